@@ -1,0 +1,149 @@
+"""Seeded synthetic inputs for the SYRK workloads.
+
+This module only draws random numbers, rounds them to the storage type and
+shapes them; it contains none of the method's arithmetic, so both the GPU tests
+and the CPU reference may take their inputs from it.  All generators are numpy
+``default_rng(seed)`` streams on the host, so the bits do not depend on torch or
+on a GPU.
+
+bf16 values travel as ``uint16`` bit patterns (numpy has no bfloat16 type).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+DTYPE_F64 = 0        # A, C binary64
+DTYPE_BF16_F32 = 1   # A bfloat16, C binary32 (binary32 accumulation)
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round binary32 values to bfloat16 (nearest, ties to even); returns uint16 bits."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    lsb = (u >> np.uint32(16)) & np.uint32(1)
+    rounded = (u + np.uint32(0x7FFF) + lsb) >> np.uint32(16)
+    return rounded.astype(np.uint16)
+
+
+def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """Widen bfloat16 bit patterns to binary32 (exact)."""
+    return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def _normal(rng: np.random.Generator, shape, std: float, chunk_rows: int = 1024) -> np.ndarray:
+    """N(0, std^2) float32 array drawn row-chunk by row-chunk (bounded host memory)."""
+    out = np.empty(shape, dtype=np.float32)
+    for r0 in range(0, shape[0], chunk_rows):
+        r1 = min(shape[0], r0 + chunk_rows)
+        out[r0:r1] = (rng.standard_normal((r1 - r0, shape[1]), dtype=np.float32) * np.float32(std))
+    return out
+
+
+def uniform_f64(N: int, M: int, seed: int) -> np.ndarray:
+    """Entries i.i.d. Uniform(-1, 1), binary64."""
+    return np.random.default_rng(seed).uniform(-1.0, 1.0, size=(N, M))
+
+
+def normal_f64(N: int, M: int, seed: int, std: float = 1.0) -> np.ndarray:
+    """Entries i.i.d. N(0, std^2), binary64."""
+    return np.random.default_rng(seed).standard_normal((N, M)) * std
+
+
+def normal_bf16(N: int, M: int, seed: int, std: float = 1.0) -> np.ndarray:
+    """Entries i.i.d. N(0, std^2) rounded to bfloat16; uint16 bit patterns."""
+    return f32_to_bf16_bits(_normal(np.random.default_rng(seed), (N, M), std))
+
+
+def small_int_f64(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
+    """Integer entries in [lo, hi] stored as binary64 (every partial sum is exact)."""
+    return np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float64)
+
+
+def small_int_bf16(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
+    """Integer entries in [lo, hi] as bfloat16 bit patterns (exactly representable)."""
+    v = np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float32)
+    return f32_to_bf16_bits(v)
+
+
+def ones(N: int, M: int, dtype: int) -> np.ndarray:
+    """All-ones A in the storage type of ``dtype``."""
+    if dtype == DTYPE_F64:
+        return np.ones((N, M), dtype=np.float64)
+    return f32_to_bf16_bits(np.ones((N, M), dtype=np.float32))
+
+
+def to_storage(values: np.ndarray, dtype: int) -> np.ndarray:
+    """Values (exactly representable in the target type) -> storage array for A."""
+    if dtype == DTYPE_F64:
+        return np.ascontiguousarray(values, dtype=np.float64)
+    return f32_to_bf16_bits(np.asarray(values, dtype=np.float32))
+
+
+def c_storage_dtype(dtype: int):
+    return np.float64 if dtype == DTYPE_F64 else np.float32
+
+
+def random_c(N: int, seed: int, dtype: int, ldc: Optional[int] = None) -> np.ndarray:
+    """A full N x ldc prior value of C (both triangles filled; N(0,1))."""
+    ldc = N if ldc is None else ldc
+    c = np.random.default_rng(seed).standard_normal((N, ldc))
+    return c.astype(c_storage_dtype(dtype))
+
+
+@dataclass
+class Workload:
+    """One benchmark configuration: shapes, scalars, type and the recipe for A."""
+    name: str
+    N: int
+    M: int
+    dtype: int
+    alpha: float
+    beta: float
+    seed: int
+    dist: str            # "uniform", "normal"
+    std: float = 1.0
+
+    def make_A(self) -> np.ndarray:
+        if self.dtype == DTYPE_F64:
+            if self.dist == "uniform":
+                return uniform_f64(self.N, self.M, self.seed)
+            return normal_f64(self.N, self.M, self.seed, self.std)
+        return normal_bf16(self.N, self.M, self.seed, self.std)
+
+    @property
+    def flops(self) -> int:
+        return self.N * (self.N + 1) * self.M
+
+
+# The four single-call configurations (the fifth is a sweep, see cholesky_sweep_*).
+CONFIGS = {
+    "c1": Workload("c1_f64_512x256", 512, 256, DTYPE_F64, 1.0, 0.0, 0, "uniform"),
+    "c2": Workload("c2_f64_4096x4096", 4096, 4096, DTYPE_F64, 1.0, 0.0, 1, "normal"),
+    "c3": Workload("c3_bf16_16384x4096", 16384, 4096, DTYPE_BF16_F32, 1.0, 0.0, 2, "normal"),
+    "c4": Workload("c4_bf16_2048x262144", 2048, 262144, DTYPE_BF16_F32, 1.0, 0.0, 3, "normal",
+                   std=2.0 ** -9),
+}
+
+# Cholesky-shaped trailing-update sweep: n = n_max, n_max - step, ..., step; inner
+# dimension 512; alpha = -1, beta = 1; seed 4.
+SWEEP_K = 512
+SWEEP_SEED = 4
+
+
+def sweep_sizes(n_max: int = 32768, step: int = 512):
+    return list(range(n_max, 0, -step))
+
+
+def sweep_panel(n: int, n_max: int = 32768) -> np.ndarray:
+    """A_n: n x 512 binary64, N(0,1)/sqrt(512); one independent stream per n."""
+    rng = np.random.default_rng([SWEEP_SEED, 1, n, n_max])
+    return rng.standard_normal((n, SWEEP_K)) / np.sqrt(float(SWEEP_K))
+
+
+def sweep_factor(n_max: int = 32768) -> np.ndarray:
+    """G: n_max x 512 binary64 N(0,1).  The swept matrix is n_max*I + G G^T / 512;
+    forming that product is input preparation and is left to the caller."""
+    rng = np.random.default_rng([SWEEP_SEED, 0, n_max])
+    return rng.standard_normal((n_max, SWEEP_K))

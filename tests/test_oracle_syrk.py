@@ -1,0 +1,187 @@
+"""Pins for the numeric reference (oracle/syrk_oracle.c), CPU only.
+
+Each test ties the reference to something other than itself: a hand-worked
+example, closed forms, exact rational arithmetic through an independent
+loop nest, symmetry, the algebra of alpha and beta.
+"""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import syrk as O
+from paper_2202_10217_b200 import inputs as I
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+BOTH = [O.DTYPE_F64, O.DTYPE_BF16_F32]
+
+
+def lower(x):
+    return x[np.tril_indices(x.shape[0])]
+
+
+def widen(A, dtype):
+    return A if dtype == O.DTYPE_F64 else I.bf16_bits_to_f32(A).astype(np.float64)
+
+
+def exact_gram_by_outer_products(Af):
+    """Full N x N Gram matrix in exact rationals, column-by-column outer products
+    (k outermost: a different loop nest from the reference's i, j, k)."""
+    N, M = Af.shape
+    G = [[Fraction(0)] * N for _ in range(N)]
+    for k in range(M):
+        col = [Fraction(float(Af[r, k])) for r in range(N)]
+        for i in range(N):
+            for j in range(N):
+                G[i][j] += col[i] * col[j]
+    return G
+
+
+def test_hand_worked_example():
+    rows = [l for l in open(os.path.join(GOLDEN, "syrk_3x2_by_hand.txt")) if not l.startswith("#")]
+    N, M = map(int, rows[0].split())
+    A = np.array([[float(v) for v in rows[1 + r].split()] for r in range(N)])
+    want = [[float(v) for v in rows[1 + N + r].split()] for r in range(N)]
+    for dtype in BOTH:
+        ref, bound = O.syrk_lower(I.to_storage(A, dtype), None, 1.0, 0.0, dtype)
+        for i in range(N):
+            for j in range(i + 1):
+                assert ref[i, j] == want[i][j]
+                assert bound[i, j] == want[i][j]        # all entries positive
+        assert np.isnan(ref[0, 1]) and np.isnan(ref[1, 2])  # upper triangle never written
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+@pytest.mark.parametrize("N,M", [(1, 1), (5, 7), (17, 64), (8, 4096)])
+def test_all_ones_gives_M(dtype, N, M):
+    ref, bound = O.syrk_lower(I.ones(N, M, dtype), None, 1.0, 0.0, dtype)
+    assert np.all(lower(ref) == float(M)) and np.all(lower(bound) == float(M))
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+def test_orthonormal_rows_give_identity(dtype):
+    N = 16
+    A = np.zeros((N, 40))
+    A[:, :N] = np.eye(N)                                    # [I | 0]
+    ref, _ = O.syrk_lower(I.to_storage(A, dtype), None, 1.0, 0.0, dtype)
+    assert np.array_equal(lower(ref), lower(np.eye(N)))
+    H = np.array([[1.0]])
+    while H.shape[0] < 64:                                   # Sylvester-Hadamard
+        H = np.block([[H, H], [H, -H]])
+    A = H / 8.0                                              # 1/sqrt(64), exact in bf16
+    ref, bound = O.syrk_lower(I.to_storage(A, dtype), None, 1.0, 0.0, dtype)
+    assert np.array_equal(lower(ref), lower(np.eye(64)))
+    assert np.all(lower(bound) == 1.0)
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+def test_single_column_is_rank_one_outer_product(dtype):
+    v = np.array([3.0, -1.0, 0.5, 2.0, -4.0, 0.25])
+    A = np.zeros((6, 9))
+    A[:, 4] = v
+    ref, bound = O.syrk_lower(I.to_storage(A, dtype), None, 1.0, 0.0, dtype)
+    assert np.array_equal(lower(ref), lower(np.outer(v, v)))
+    assert np.array_equal(lower(bound), lower(np.abs(np.outer(v, v))))
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+def test_exact_integers_match_independent_loop_nest(dtype):
+    N, M = 23, 37
+    A = I.small_int_f64(N, M, seed=11, lo=-3, hi=3)
+    G = exact_gram_by_outer_products(A)
+    ref, bound = O.syrk_lower(I.to_storage(A, dtype), None, 1.0, 0.0, dtype)
+    Gabs = exact_gram_by_outer_products(np.abs(A))
+    for i in range(N):
+        for j in range(i + 1):
+            assert Fraction(ref[i, j]) == G[i][j]
+            assert Fraction(bound[i, j]) == Gabs[i][j]
+            assert G[i][j] == G[j][i]                       # symmetry of A A^T
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+def test_real_inputs_within_dot_product_bound_of_exact(dtype):
+    N, M = 12, 50
+    A = I.uniform_f64(N, M, seed=5) if dtype == O.DTYPE_F64 else I.normal_bf16(N, M, seed=5)
+    Af = widen(A, dtype)
+    G = exact_gram_by_outer_products(Af)
+    ref, bound = O.syrk_lower(A, None, 1.0, 0.0, dtype)
+    u = 2.0 ** -53
+    for i in range(N):
+        for j in range(i + 1):
+            err = abs(Fraction(ref[i, j]) - G[i][j])
+            assert err <= Fraction(M * u * 1.01) * Fraction(bound[i, j])
+    # the reference must not be exact-by-construction: some entry does round
+    assert any(Fraction(ref[i, j]) != G[i][j] for i in range(N) for j in range(i + 1))
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+def test_row_reversal_symmetry(dtype):
+    """(P A)(P A)^T = P (A A^T) P^T: entry (i, j) of the reversed problem equals
+    entry (N-1-j, N-1-i) of the original, bit for bit (products commute exactly)."""
+    N, M = 19, 33
+    A = I.normal_f64(N, M, 3) if dtype == O.DTYPE_F64 else I.normal_bf16(N, M, 3)
+    ref, _ = O.syrk_lower(A, None, 1.0, 0.0, dtype)
+    rev, _ = O.syrk_lower(np.ascontiguousarray(A[::-1]), None, 1.0, 0.0, dtype)
+    for i in range(N):
+        for j in range(i + 1):
+            assert rev[i, j] == ref[N - 1 - j, N - 1 - i]
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+@pytest.mark.parametrize("alpha,beta", [(1, 0), (-1, 1), (0, 1), (0, 0), (2.5, -0.5), (1, 2)])
+def test_alpha_beta_algebra_on_integers(dtype, alpha, beta):
+    N, M = 9, 14
+    A = I.small_int_f64(N, M, seed=2)
+    Cin = (np.random.default_rng(8).integers(-8, 9, size=(N, N)) * 2).astype(I.c_storage_dtype(dtype))
+    base, _ = O.syrk_lower(I.to_storage(A, dtype), None, 1.0, 0.0, dtype)
+    ref, _ = O.syrk_lower(I.to_storage(A, dtype), Cin, alpha, beta, dtype)
+    want = alpha * base + beta * Cin.astype(np.float64)    # all terms exact in binary64
+    assert np.array_equal(lower(ref), lower(want))
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+def test_beta_zero_does_not_read_C(dtype):
+    A = I.small_int_f64(6, 5, seed=1)
+    poison = np.full((6, 6), np.nan, dtype=I.c_storage_dtype(dtype))
+    a, _ = O.syrk_lower(I.to_storage(A, dtype), None, 1.0, 0.0, dtype)
+    b, _ = O.syrk_lower(I.to_storage(A, dtype), poison, 1.0, 0.0, dtype)
+    assert np.array_equal(lower(a), lower(b)) and not np.isnan(lower(b)).any()
+
+
+def test_bf16_widening_bit_patterns():
+    bits = np.array([[0x3F80, 0xC000, 0x3DCD, 0x0000]], dtype=np.uint16)   # 1, -2, 0.10009765625, 0
+    ref, bound = O.syrk_lower(bits, None, 1.0, 0.0, O.DTYPE_BF16_F32)
+    assert ref[0, 0] == 1.0 + 4.0 + 0.10009765625 ** 2
+    assert bound[0, 0] == ref[0, 0]
+
+
+@pytest.mark.parametrize("dtype", BOTH)
+def test_leading_dimensions_and_entry_list(dtype):
+    N, M, lda, ldc = 13, 21, 32, 20
+    big = I.small_int_f64(N, lda, 4) if dtype == O.DTYPE_F64 else I.small_int_bf16(N, lda, 4)
+    A = big[:, :M]                                           # row pitch lda > M
+    Cbig = I.random_c(N, 6, dtype, ldc)
+    Cin = Cbig[:, :N]
+    ref, bound = O.syrk_lower(A, Cin, -1.0, 1.0, dtype)
+    ref2, bound2 = O.syrk_lower(np.ascontiguousarray(A), np.ascontiguousarray(Cin), -1.0, 1.0, dtype)
+    assert np.array_equal(lower(ref), lower(ref2)) and np.array_equal(lower(bound), lower(bound2))
+    ii, jj = np.tril_indices(N)
+    r3, b3 = O.syrk_entries(ii, jj, A, Cin, -1.0, 1.0, dtype)
+    assert np.array_equal(r3, lower(ref)) and np.array_equal(b3, lower(bound))
+    with pytest.raises(ValueError):
+        O.syrk_entries([0], [1], A, Cin, 1.0, 0.0, dtype)    # upper-triangle entry refused
+
+
+def test_bf16_rounding_of_inputs_is_nearest_even():
+    # 1 + 2^-8 is a tie between 1 and 1 + 2^-7 -> even (1.0); 1 + 3*2^-8 ties up to 1 + 2^-6.
+    x = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20], dtype=np.float32)
+    got = I.bf16_bits_to_f32(I.f32_to_bf16_bits(x))
+    assert list(got) == [1.0, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7]
+
+
+def test_tolerance_formula():
+    t = O.tolerance(4, np.array([2.0]), np.array([3.0]), -1.0, 1.0, O.DTYPE_F64)
+    assert t[0] == 8 * 2.0 ** -53 * 4 * 5.0
+    t = O.tolerance(4, np.array([2.0]), np.array([3.0]), 2.0, 0.0, O.DTYPE_BF16_F32)
+    assert t[0] == 4 * 2.0 ** -24 * 4 * 4.0
