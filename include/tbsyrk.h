@@ -1,0 +1,180 @@
+/*
+ * tbsyrk - symmetric rank-k update on the lower triangle, scheduled by triangle
+ * blocks, for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libtbsyrk.so.  Plain pointers and sizes only.  Unless a function says
+ * otherwise, matrix pointers are DEVICE pointers and the call only enqueues work
+ * on the given CUDA stream: it never synchronises the device, never aborts and
+ * never throws.  Every function returns 0 (SYRK_OK) or a negative SYRK_ERR_*.
+ *
+ * The operation (Algorithm 1 of "I/O-Optimal Algorithms for Symmetric Linear
+ * Algebra Kernels": for i, for j <= i, for k: C[i][j] += A[i][k] * A[j][k]),
+ * extended with the usual scalars:
+ *
+ *     C[i*ldc + j] <- alpha * sum_{k<M} A[i*lda + k] * A[j*lda + k] + beta * C[i*ldc + j]
+ *
+ * for all 0 <= j <= i < N.  Entries with i < j are never read or written.  The
+ * work is partitioned as in Algorithm 4 (TBS) in its tiled form (Section 5.1.4):
+ * a thread block owns the accumulators of every pair among k row-segments of A
+ * (a triangle block, Section 3.2) and streams only those k segments along M;
+ * what triangle blocks cannot cover is done with square and diagonal blocks.
+ */
+#ifndef TBSYRK_H
+#define TBSYRK_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* dtype argument */
+#define SYRK_DTYPE_F64      0  /* A and C binary64; binary64 accumulation (DMMA)          */
+#define SYRK_DTYPE_BF16_F32 1  /* A bfloat16, C binary32; binary32 accumulation (tcgen05) */
+
+/* return codes */
+#define SYRK_OK                 0
+#define SYRK_ERR_NULL          -1  /* a required pointer is null                          */
+#define SYRK_ERR_SIZE          -2  /* N < 0 or M < 0, or a size beyond a stated maximum   */
+#define SYRK_ERR_LD            -3  /* lda < max(1, M) or ldc < max(1, N)                  */
+#define SYRK_ERR_DTYPE         -4  /* unknown dtype                                       */
+#define SYRK_ERR_ALLOC         -5  /* a device or host allocation of the library failed   */
+#define SYRK_ERR_CUDA          -6  /* a CUDA runtime/driver call failed                   */
+#define SYRK_ERR_PLAN          -7  /* invalid schedule parameters                         */
+#define SYRK_ERR_DEVICE_WAIT   -8  /* a bounded wait inside a kernel ran out (see syrk_last_status) */
+#define SYRK_ERR_NO_DEVICE     -9  /* no CUDA device / not an sm_100 device               */
+
+/* schedules (syrk_set_schedule) */
+#define SYRK_SCHEDULE_TBS     0    /* triangle blocks + square/diagonal leftovers (default) */
+#define SYRK_SCHEDULE_SQUARE  1    /* square and diagonal blocks only (comparison schedule) */
+
+/*
+ * The update itself (see the formula above).
+ *
+ *   N, M     rows and columns of A; N == 0 returns at once.
+ *   A        device pointer, row-major N x M, row pitch lda >= max(1, M) elements;
+ *            read only.  binary64 for SYRK_DTYPE_F64, bfloat16 for SYRK_DTYPE_BF16_F32.
+ *   C        device pointer, row-major N x N, row pitch ldc >= max(1, N) elements;
+ *            binary64 / binary32 respectively.  Only j <= i is touched.  With
+ *            beta == 0 the old C is not read (NaN or Inf there do not propagate).
+ *   alpha, beta   scalars, passed through as given (non-finite values included).
+ *            alpha == 0 or M == 0: the lower triangle becomes beta * C (zero when
+ *            beta == 0, untouched when beta == 1).
+ *   stream   a cudaStream_t (0 = the legacy default stream).
+ *
+ * Layout and alignment: the fast kernels fetch A with TMA and need A 16-byte
+ * aligned and lda * sizeof(element) a multiple of 16; any other A takes a slower
+ * plain-load kernel with the same result.  C may have any alignment.
+ *
+ * Ownership: the caller owns A and C, keeps them alive until the stream has run
+ * the enqueued work, and must not let them overlap.  The library owns a cache of
+ * device-resident work lists (one per N, dtype and schedule) and, for the
+ * K-split path, a device workspace; both are created on first use (that first
+ * call allocates device memory) and released by syrk_shutdown().  Calls are
+ * stream-ordered; concurrent calls on different streams that need the K-split
+ * workspace are serialised by the caller.
+ */
+int syrk_lower(int64_t N, int64_t M,
+               const void* A, int64_t lda,
+               void* C, int64_t ldc,
+               double alpha, double beta,
+               int dtype, void* stream);
+
+/*
+ * Same operation with HOST buffers: copies A (and C when beta != 0) to the
+ * device, runs syrk_lower, copies the lower triangle back into C, and waits for
+ * completion.  A and C are host pointers (pageable or pinned).  The strict upper
+ * triangle of the host C is left as it was.  Device buffers are allocated per
+ * call and freed before returning.
+ */
+int syrk_lower_host(int64_t N, int64_t M,
+                    const void* A, int64_t lda,
+                    void* C, int64_t ldc,
+                    double alpha, double beta, int dtype);
+
+/* Build and upload the work list for (N, M, dtype) ahead of time, so that a later
+ * syrk_lower with these sizes allocates nothing. */
+int syrk_plan_prepare(int64_t N, int64_t M, int dtype);
+
+/* Free every cached work list and workspace of the calling process. */
+void syrk_shutdown(void);
+
+/* After the caller has synchronised `stream`: 0, or SYRK_ERR_DEVICE_WAIT when a
+ * kernel gave up on a bounded wait since the last query (the result of that call
+ * is then undefined; the context stays usable).  Clears the flag. */
+int syrk_last_status(void* stream);
+
+/* Human-readable text for a return code (static storage). */
+const char* syrk_strerror(int code);
+
+/* Select the schedule used by later calls (process-wide). */
+int syrk_set_schedule(int schedule);
+
+/* Force the number of K-slices (0 = automatic) used by later bf16 calls. */
+int syrk_set_split_k(int slices);
+
+/*
+ * What a call with these sizes would run (host only, no device needed).
+ * All counts refer to one call.  "a_loads" is the number of elements of A the
+ * work list moves from slow to fast memory in the paper's two-level model
+ * (Section 3): for every work item, rows held x M.
+ */
+typedef struct {
+    int32_t tile;            /* b: rows per segment                                  */
+    int32_t k;               /* segments per triangle block                          */
+    int32_t c;               /* zone side of the top level (in tiles)                */
+    int32_t split_k;         /* K-slices                                             */
+    int64_t n_tiles;         /* ceil(N / b)                                          */
+    int64_t items;           /* work items                                           */
+    int64_t tri_items;       /* of which triangle blocks                             */
+    int64_t rect_items;      /* of which square / rectangular blocks                 */
+    int64_t diag_items;      /* of which blocks on the diagonal                      */
+    int64_t tri_tiles;       /* b x b output tiles owned by triangle blocks          */
+    int64_t all_tiles;       /* b x b output tiles in total: n_tiles(n_tiles+1)/2    */
+    int64_t a_loads;         /* elements of A loaded (two-level model)               */
+    int64_t c_elems;         /* elements of C owned: N(N+1)/2                        */
+    int64_t s_acc;           /* accumulator elements a thread block may hold         */
+    int64_t s_total;         /* s_acc + staging elements (all pipeline stages)       */
+} syrk_schedule_stats;
+
+int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats* out);
+
+/*
+ * Work-list inspection (host only).  A plan is the tiled Algorithm 4 over
+ * n_tiles tile rows: triangle blocks of k tile rows chosen by the cyclic indexing
+ * family, square blocks (rect_rows x rect_cols tiles) for the last l tile rows and
+ * for zones too small to recurse into, and diagonal blocks (diag_side adjacent
+ * tile rows, including their diagonal tiles).  schedule == SYRK_SCHEDULE_SQUARE
+ * drops the triangle blocks.  Returns NULL on invalid parameters.
+ *
+ * An item holds n_seg tile rows ("segments") and n_tile output tiles; tile t is
+ * C[seg[tile_x[t]] , seg[tile_y[t]]] (tile row, tile column), seg[x] >= seg[y].
+ */
+#define TBS_ITEM_TRI  0
+#define TBS_ITEM_RECT 1
+#define TBS_ITEM_DIAG 2
+#define TBS_MAX_SEG   8
+#define TBS_MAX_TILE 16
+
+void*   tbs_plan_build(int64_t n_tiles, int k, int rect_rows, int rect_cols,
+                       int diag_side, int schedule);
+int64_t tbs_plan_num_items(const void* plan);
+int     tbs_plan_item(const void* plan, int64_t index, int32_t* kind,
+                      int32_t* n_seg, int32_t seg[TBS_MAX_SEG],
+                      int32_t* n_tile, int32_t tile_x[TBS_MAX_TILE],
+                      int32_t tile_y[TBS_MAX_TILE]);
+void    tbs_plan_free(void* plan);
+
+/* Replay a plan in the two-level model for an N x M matrix cut into tiles of b
+ * rows (the last tile may be ragged): elements of A and of C moved, and the
+ * smallest / largest number of items that own a lower-triangle tile (both 1 for a
+ * correct plan; tiles above the diagonal must stay at 0 and are reported through
+ * *upper_cover). */
+int tbs_plan_simulate(const void* plan, int64_t N, int64_t M, int b,
+                      int64_t* a_loads, int64_t* c_loads,
+                      int32_t* min_cover, int32_t* max_cover, int32_t* upper_cover);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TBSYRK_H */

@@ -57,7 +57,7 @@ def num_threads() -> int:
 def _check_inputs(A: np.ndarray, C_in, dtype: int):
     want_a = np.float64 if dtype == DTYPE_F64 else np.uint16
     want_c = np.float64 if dtype == DTYPE_F64 else np.float32
-    if A.dtype != want_a or A.ndim != 2 or A.strides[1] != A.itemsize:
+    if A.dtype != want_a or A.ndim != 2 or (A.size > 0 and A.strides[1] != A.itemsize):
         raise ValueError("A must be a row-major 2-D array of %s" % want_a.__name__)
     if C_in is not None and (C_in.dtype != want_c or C_in.ndim != 2
                              or C_in.strides[1] != C_in.itemsize):
@@ -74,7 +74,7 @@ def syrk_lower(A: np.ndarray, C_in, alpha: float, beta: float, dtype: int):
     """
     _check_inputs(A, C_in, dtype)
     N, M = A.shape
-    lda = A.strides[0] // A.itemsize if N > 0 else max(M, 1)
+    lda = max(A.strides[0] // A.itemsize, M, 1) if A.size > 0 else max(M, 1)
     ref = np.full((N, N), np.nan, dtype=np.float64)
     bound = np.full((N, N), np.nan, dtype=np.float64)
     cptr, ldc = None, max(N, 1)

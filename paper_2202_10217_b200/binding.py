@@ -1,0 +1,205 @@
+"""Thin ctypes binding of libtbsyrk.so: same names as the C ABI, argument
+marshalling only.  Every step of the computation runs in the library's CUDA
+kernels; there is no CPU or PyTorch fallback, and loading fails loudly when the
+shared library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libtbsyrk.so")
+
+DTYPE_F64 = 0
+DTYPE_BF16_F32 = 1
+SCHEDULE_TBS = 0
+SCHEDULE_SQUARE = 1
+ITEM_TRI, ITEM_RECT, ITEM_DIAG = 0, 1, 2
+MAX_SEG, MAX_TILE = 8, 16
+
+EXPORTS = [
+    "syrk_lower", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
+    "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_get_schedule_stats",
+    "tbs_plan_build", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
+]
+
+
+class ScheduleStats(ctypes.Structure):
+    _fields_ = [("tile", ctypes.c_int32), ("k", ctypes.c_int32), ("c", ctypes.c_int32),
+                ("split_k", ctypes.c_int32), ("n_tiles", ctypes.c_int64), ("items", ctypes.c_int64),
+                ("tri_items", ctypes.c_int64), ("rect_items", ctypes.c_int64),
+                ("diag_items", ctypes.c_int64), ("tri_tiles", ctypes.c_int64),
+                ("all_tiles", ctypes.c_int64), ("a_loads", ctypes.c_int64),
+                ("c_elems", ctypes.c_int64), ("s_acc", ctypes.c_int64), ("s_total", ctypes.c_int64)]
+
+    def as_dict(self):
+        return {name: int(getattr(self, name)) for name, _ in self._fields_}
+
+
+class SyrkError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__("tbsyrk error %d: %s" % (code, strerror(code)))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library (raises if it is not built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libtbsyrk.so is missing: run `python -m paper_2202_10217_b200.build` "
+                              "(there is no fallback implementation)")
+        L = ctypes.CDLL(LIB_PATH)
+        i64, i32, dbl, vp, ci = ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_void_p, ctypes.c_int
+        L.syrk_lower.restype = ci
+        L.syrk_lower.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
+        L.syrk_lower_host.restype = ci
+        L.syrk_lower_host.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci]
+        L.syrk_plan_prepare.restype = ci
+        L.syrk_plan_prepare.argtypes = [i64, i64, ci]
+        L.syrk_shutdown.restype = None
+        L.syrk_shutdown.argtypes = []
+        L.syrk_last_status.restype = ci
+        L.syrk_last_status.argtypes = [vp]
+        L.syrk_strerror.restype = ctypes.c_char_p
+        L.syrk_strerror.argtypes = [ci]
+        L.syrk_set_schedule.restype = ci
+        L.syrk_set_schedule.argtypes = [ci]
+        L.syrk_set_split_k.restype = ci
+        L.syrk_set_split_k.argtypes = [ci]
+        L.syrk_get_schedule_stats.restype = ci
+        L.syrk_get_schedule_stats.argtypes = [i64, i64, ci, ctypes.POINTER(ScheduleStats)]
+        L.tbs_plan_build.restype = vp
+        L.tbs_plan_build.argtypes = [i64, ci, ci, ci, ci, ci]
+        L.tbs_plan_num_items.restype = i64
+        L.tbs_plan_num_items.argtypes = [vp]
+        L.tbs_plan_item.restype = ci
+        L.tbs_plan_item.argtypes = [vp, i64, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                    ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                    ctypes.POINTER(i32)]
+        L.tbs_plan_free.restype = None
+        L.tbs_plan_free.argtypes = [vp]
+        L.tbs_plan_simulate.restype = ci
+        L.tbs_plan_simulate.argtypes = [vp, i64, i64, ci, ctypes.POINTER(i64), ctypes.POINTER(i64),
+                                        ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().syrk_strerror(int(code)).decode()
+
+
+def _check(code: int) -> None:
+    if code != 0:
+        raise SyrkError(code)
+
+
+def _ptr(x) -> Optional[int]:
+    """Raw address of a torch tensor / numpy array / int / None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return int(x.data_ptr())
+    if hasattr(x, "ctypes"):
+        return int(x.ctypes.data)
+    raise TypeError("cannot take the address of %r" % type(x))
+
+
+def syrk_lower(N: int, M: int, A, lda: int, C, ldc: int, alpha: float, beta: float, dtype: int,
+               stream: Optional[int] = None) -> None:
+    """Enqueue C_lower <- alpha * A A^T + beta * C_lower on `stream` (device pointers).
+
+    `A` and `C` are torch CUDA tensors (or raw device addresses); `stream` is a raw
+    cudaStream_t, by default torch's current stream.
+    """
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().syrk_lower(N, M, _ptr(A), lda, _ptr(C), ldc, float(alpha), float(beta), dtype, stream))
+
+
+def syrk_lower_host(N: int, M: int, A, lda: int, C, ldc: int, alpha: float, beta: float,
+                    dtype: int) -> None:
+    """Same operation on HOST buffers (numpy arrays, CPU tensors or raw addresses);
+    copies in, computes on the GPU, copies the lower triangle back, and waits."""
+    _check(lib().syrk_lower_host(N, M, _ptr(A), lda, _ptr(C), ldc, float(alpha), float(beta), dtype))
+
+
+def syrk_plan_prepare(N: int, M: int, dtype: int) -> None:
+    _check(lib().syrk_plan_prepare(N, M, dtype))
+
+
+def syrk_shutdown() -> None:
+    lib().syrk_shutdown()
+
+
+def syrk_last_status(stream: Optional[int] = None) -> int:
+    return int(lib().syrk_last_status(stream))
+
+
+def syrk_set_schedule(schedule: int) -> None:
+    _check(lib().syrk_set_schedule(schedule))
+
+
+def syrk_set_split_k(slices: int) -> None:
+    _check(lib().syrk_set_split_k(slices))
+
+
+def syrk_get_schedule_stats(N: int, M: int, dtype: int) -> dict:
+    st = ScheduleStats()
+    _check(lib().syrk_get_schedule_stats(N, M, dtype, ctypes.byref(st)))
+    return st.as_dict()
+
+
+class Plan:
+    """Host-side work list (tbs_plan_* calls); no device needed."""
+
+    def __init__(self, n_tiles: int, k: int, rect_rows: int, rect_cols: int, diag_side: int,
+                 schedule: int = SCHEDULE_TBS):
+        self._h = lib().tbs_plan_build(n_tiles, k, rect_rows, rect_cols, diag_side, schedule)
+        if not self._h:
+            raise SyrkError(-7)
+        self.n_tiles = n_tiles
+
+    def __len__(self) -> int:
+        return int(lib().tbs_plan_num_items(self._h))
+
+    def item(self, index: int):
+        """(kind, [segments], [(x_slot, y_slot), ...])"""
+        i32 = ctypes.c_int32
+        kind, n_seg, n_tile = i32(), i32(), i32()
+        seg = (i32 * MAX_SEG)()
+        tx = (i32 * MAX_TILE)()
+        ty = (i32 * MAX_TILE)()
+        _check(lib().tbs_plan_item(self._h, index, ctypes.byref(kind), ctypes.byref(n_seg), seg,
+                                   ctypes.byref(n_tile), tx, ty))
+        return (kind.value, list(seg[:n_seg.value]),
+                [(tx[t], ty[t]) for t in range(n_tile.value)])
+
+    def simulate(self, N: int, M: int, b: int) -> dict:
+        i64, i32 = ctypes.c_int64, ctypes.c_int32
+        a, c = i64(), i64()
+        lo, hi, up = i32(), i32(), i32()
+        _check(lib().tbs_plan_simulate(self._h, N, M, b, ctypes.byref(a), ctypes.byref(c),
+                                       ctypes.byref(lo), ctypes.byref(hi), ctypes.byref(up)))
+        return {"a_loads": a.value, "c_loads": c.value, "min_cover": lo.value,
+                "max_cover": hi.value, "upper_cover": up.value}
+
+    def close(self) -> None:
+        if self._h:
+            lib().tbs_plan_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,306 @@
+// C ABI of libtbsyrk.so (see include/tbsyrk.h for the contract of every call).
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+#include "../../include/tbsyrk.h"
+#include "kernels.h"
+#include "runtime.h"
+
+using namespace tbsyrk;
+
+namespace {
+
+int validate(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, int dtype) {
+    if (dtype != SYRK_DTYPE_F64 && dtype != SYRK_DTYPE_BF16_F32) return SYRK_ERR_DTYPE;
+    if (N < 0 || M < 0 || N >= (int64_t(1) << 31) - 256 || M >= (int64_t(1) << 31) - 256) return SYRK_ERR_SIZE;
+    if (N == 0) return SYRK_OK;
+    if (lda < std::max<int64_t>(1, M) || ldc < N) return SYRK_ERR_LD;
+    if (!C || (M > 0 && !A)) return SYRK_ERR_NULL;
+    return SYRK_OK;
+}
+
+size_t a_elem(int dtype) { return dtype == SYRK_DTYPE_F64 ? 8 : 2; }
+size_t c_elem(int dtype) { return dtype == SYRK_DTYPE_F64 ? 8 : 4; }
+
+bool tma_ok(const void* A, int64_t lda, int dtype) {
+    return (reinterpret_cast<uintptr_t>(A) & 15) == 0 && (size_t(lda) * a_elem(dtype)) % 16 == 0;
+}
+
+int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk) {
+    const int forced = runtime().split_k;
+    const int64_t ksteps = (M + bk - 1) / bk;
+    int s = 1;
+    if (forced > 0) s = forced;
+    else {
+        // Few items and a long inner dimension: cut M so that every SM has work.
+        const int64_t items = int64_t(dp->plan.items.size());
+        if (items > 0 && items < ds->sm_count && ksteps >= 64)
+            s = int(std::min<int64_t>((2 * ds->sm_count + items - 1) / items, ksteps / 32));
+    }
+    s = int(std::max<int64_t>(1, std::min<int64_t>(s, ksteps)));
+    return s;
+}
+
+int run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
+               double beta, int dtype, cudaStream_t stream) {
+    DeviceState* ds = nullptr;
+    int rc = get_device_state(&ds);
+    if (rc != SYRK_OK) return rc;
+    if (alpha == 0.0 || M == 0) {
+        if (beta == 1.0) return SYRK_OK;
+        return launch_scale_lower(dtype, N, C, ldc, beta, stream) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+    }
+    if (!tma_ok(A, lda, dtype))
+        return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, stream) == cudaSuccess
+                   ? SYRK_OK : SYRK_ERR_CUDA;
+    DevicePlan* dp = nullptr;
+    rc = get_device_plan(ds, N, dtype, &dp);
+    if (rc != SYRK_OK) return rc;
+    const KernelShape ks = kernel_shape(dtype);
+    CUtensorMap tm;
+    rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, ks.tile, ks.bk);
+    if (rc != SYRK_OK) return rc;
+    const int64_t n_items = int64_t(dp->plan.items.size());
+    cudaError_t e;
+    if (dtype == SYRK_DTYPE_F64) {
+        e = launch_syrk_f64(tm, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha, beta,
+                            ds->d_status, stream);
+    } else {
+        const int split = pick_split_k(ds, dp, M, ks.bk);
+        if (split > 1) {
+            const size_t want = size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float);
+            void* p = ds->d_partial;
+            rc = ensure_device_bytes(&p, &ds->partial_bytes, want);
+            ds->d_partial = static_cast<float*>(p);
+            if (rc != SYRK_OK) return rc;
+        }
+        e = launch_syrk_bf16(tm, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
+                             float(beta), split, ds->d_partial, dp->d_tile_base, ds->d_status,
+                             ds->sm_count, stream);
+    }
+    return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
+// Lower triangle of C (row pitch ldc) -> packed rows (row i has i+1 entries), on device.
+template <typename T>
+__global__ void pack_lower_kernel(int64_t N, const T* __restrict__ C, int64_t ldc, T* __restrict__ packed) {
+    const int64_t i = blockIdx.y;
+    const T* src = C + i * ldc;
+    T* dst = packed + i * (i + 1) / 2;
+    for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j <= i; j += int64_t(gridDim.x) * blockDim.x)
+        dst[j] = src[j];
+}
+
+}  // namespace
+
+extern "C" {
+
+int syrk_lower(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
+               double beta, int dtype, void* stream) {
+    int rc = validate(N, M, A, lda, C, ldc, dtype);
+    if (rc != SYRK_OK || N == 0) return rc;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    return run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream));
+}
+
+int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
+                    double beta, int dtype) {
+    int rc = validate(N, M, A, lda, C, ldc, dtype);
+    if (rc != SYRK_OK || N == 0) return rc;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    DeviceState* ds = nullptr;
+    rc = get_device_state(&ds);
+    if (rc != SYRK_OK) return rc;
+    if (!ds->host_stream && cudaStreamCreateWithFlags(&ds->host_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        cudaGetLastError();
+        return SYRK_ERR_CUDA;
+    }
+    cudaStream_t st = ds->host_stream;
+    const size_t ea = a_elem(dtype), ec = c_elem(dtype);
+    // device pitch of A rounded up so that the TMA path applies to any M
+    const int64_t dlda = (std::max<int64_t>(M, 1) * int64_t(ea) + 15) / 16 * 16 / int64_t(ea);
+    const int64_t dldc = (N + 1) / 2 * 2;
+    const size_t packed_bytes = size_t(N) * size_t(N + 1) / 2 * ec;
+    if ((rc = ensure_device_bytes(&ds->d_a, &ds->d_a_bytes, size_t(N) * dlda * ea)) != SYRK_OK) return rc;
+    if ((rc = ensure_device_bytes(&ds->d_c, &ds->d_c_bytes, size_t(N) * dldc * ec)) != SYRK_OK) return rc;
+    if ((rc = ensure_device_bytes(&ds->d_packed, &ds->d_packed_bytes, packed_bytes)) != SYRK_OK) return rc;
+    if ((rc = ensure_pinned_bytes(&ds->h_packed, &ds->h_packed_bytes, packed_bytes)) != SYRK_OK) return rc;
+    bool ok = true;
+    if (M > 0)
+        ok = ok && cudaMemcpy2DAsync(ds->d_a, dlda * ea, A, lda * ea, M * ea, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (beta != 0.0)
+        ok = ok && cudaMemcpy2DAsync(ds->d_c, dldc * ec, C, ldc * ec, N * ec, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+    rc = run_device(N, M, ds->d_a, dlda, ds->d_c, dldc, alpha, beta, dtype, st);
+    if (rc != SYRK_OK) return rc;
+    const dim3 grid(unsigned(std::min<int64_t>(64, (N + 255) / 256)), unsigned(N));
+    if (dtype == SYRK_DTYPE_F64)
+        pack_lower_kernel<double><<<grid, 256, 0, st>>>(N, static_cast<const double*>(ds->d_c), dldc,
+                                                        static_cast<double*>(ds->d_packed));
+    else
+        pack_lower_kernel<float><<<grid, 256, 0, st>>>(N, static_cast<const float*>(ds->d_c), dldc,
+                                                       static_cast<float*>(ds->d_packed));
+    ok = cudaGetLastError() == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ds->h_packed, ds->d_packed, packed_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+    const char* src = static_cast<const char*>(ds->h_packed);
+    char* dst = static_cast<char*>(C);
+    for (int64_t i = 0; i < N; ++i) {
+        std::memcpy(dst + size_t(i) * ldc * ec, src, size_t(i + 1) * ec);
+        src += size_t(i + 1) * ec;
+    }
+    int flag = 0;
+    if (cudaMemcpy(&flag, ds->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+    if (flag != 0) { cudaMemset(ds->d_status, 0, sizeof(int)); return SYRK_ERR_DEVICE_WAIT; }
+    return SYRK_OK;
+}
+
+int syrk_plan_prepare(int64_t N, int64_t M, int dtype) {
+    if (dtype != SYRK_DTYPE_F64 && dtype != SYRK_DTYPE_BF16_F32) return SYRK_ERR_DTYPE;
+    if (N < 0 || M < 0) return SYRK_ERR_SIZE;
+    if (N == 0) return SYRK_OK;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    DeviceState* ds = nullptr;
+    int rc = get_device_state(&ds);
+    if (rc != SYRK_OK) return rc;
+    DevicePlan* dp = nullptr;
+    rc = get_device_plan(ds, N, dtype, &dp);
+    if (rc != SYRK_OK) return rc;
+    if (dtype == SYRK_DTYPE_BF16_F32) {
+        const KernelShape ks = kernel_shape(dtype);
+        const int split = pick_split_k(ds, dp, M, ks.bk);
+        if (split > 1) {
+            void* p = ds->d_partial;
+            rc = ensure_device_bytes(&p, &ds->partial_bytes,
+                                     size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float));
+            ds->d_partial = static_cast<float*>(p);
+        }
+    }
+    return rc;
+}
+
+void syrk_shutdown(void) {
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    release_all();
+}
+
+int syrk_last_status(void* /*stream*/) {
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    DeviceState* ds = nullptr;
+    int rc = get_device_state(&ds);
+    if (rc != SYRK_OK) return rc;
+    int flag = 0;
+    if (cudaMemcpy(&flag, ds->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+    if (flag == 0) return SYRK_OK;
+    cudaMemset(ds->d_status, 0, sizeof(int));
+    return SYRK_ERR_DEVICE_WAIT;
+}
+
+const char* syrk_strerror(int code) {
+    switch (code) {
+        case SYRK_OK: return "success";
+        case SYRK_ERR_NULL: return "a required pointer is null";
+        case SYRK_ERR_SIZE: return "negative or too large size";
+        case SYRK_ERR_LD: return "leading dimension smaller than the row length";
+        case SYRK_ERR_DTYPE: return "unknown dtype";
+        case SYRK_ERR_ALLOC: return "allocation failed";
+        case SYRK_ERR_CUDA: return "a CUDA call failed";
+        case SYRK_ERR_PLAN: return "invalid schedule parameters";
+        case SYRK_ERR_DEVICE_WAIT: return "a bounded wait inside a kernel ran out";
+        case SYRK_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+        default: return "unknown error code";
+    }
+}
+
+int syrk_set_schedule(int schedule) {
+    if (schedule != SYRK_SCHEDULE_TBS && schedule != SYRK_SCHEDULE_SQUARE) return SYRK_ERR_PLAN;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    runtime().schedule = schedule;
+    return SYRK_OK;
+}
+
+int syrk_set_split_k(int slices) {
+    if (slices < 0 || slices > 1024) return SYRK_ERR_PLAN;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    runtime().split_k = slices;
+    return SYRK_OK;
+}
+
+int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats* out) {
+    if (!out) return SYRK_ERR_NULL;
+    if (dtype != SYRK_DTYPE_F64 && dtype != SYRK_DTYPE_BF16_F32) return SYRK_ERR_DTYPE;
+    if (N < 0 || M < 0) return SYRK_ERR_SIZE;
+    int schedule;
+    { std::lock_guard<std::mutex> lock(runtime().mu); schedule = runtime().schedule; }
+    Plan plan;
+    if (!build_host_plan(N, dtype, schedule, &plan)) return SYRK_ERR_PLAN;
+    const KernelShape ks = kernel_shape(dtype);
+    const SimResult sim = simulate_plan(plan, N, M, ks.tile);
+    std::memset(out, 0, sizeof(*out));
+    out->tile = ks.tile;
+    out->k = ks.k;
+    out->c = int32_t(plan.c_top);
+    out->split_k = 1;
+    out->n_tiles = plan.p.n_tiles;
+    out->items = int64_t(plan.items.size());
+    out->tri_items = plan.n_tri;
+    out->rect_items = plan.n_rect;
+    out->diag_items = plan.n_diag;
+    out->tri_tiles = plan.tri_tiles;
+    out->all_tiles = plan.p.n_tiles * (plan.p.n_tiles + 1) / 2;
+    out->a_loads = sim.a_loads;
+    out->c_elems = N * (N + 1) / 2;
+    out->s_acc = ks.s_acc;
+    out->s_total = ks.s_acc + int64_t(kMaxSeg) * ks.tile * ks.bk * ks.stages;
+    if (dtype == SYRK_DTYPE_BF16_F32) out->s_total = ks.s_acc + int64_t(4) * ks.tile * ks.bk * ks.stages;
+    return SYRK_OK;
+}
+
+void* tbs_plan_build(int64_t n_tiles, int k, int rect_rows, int rect_cols, int diag_side, int schedule) {
+    PlanParams p;
+    p.n_tiles = n_tiles; p.k = k; p.rect_rows = rect_rows; p.rect_cols = rect_cols;
+    p.diag_side = diag_side; p.schedule = schedule;
+    Plan* plan = new (std::nothrow) Plan();
+    if (!plan) return nullptr;
+    if (!build_plan(p, plan)) { delete plan; return nullptr; }
+    return plan;
+}
+
+int64_t tbs_plan_num_items(const void* plan) {
+    return plan ? int64_t(static_cast<const Plan*>(plan)->items.size()) : SYRK_ERR_NULL;
+}
+
+int tbs_plan_item(const void* plan, int64_t index, int32_t* kind, int32_t* n_seg, int32_t seg[TBS_MAX_SEG],
+                  int32_t* n_tile, int32_t tile_x[TBS_MAX_TILE], int32_t tile_y[TBS_MAX_TILE]) {
+    if (!plan || !kind || !n_seg || !seg || !n_tile || !tile_x || !tile_y) return SYRK_ERR_NULL;
+    const Plan* p = static_cast<const Plan*>(plan);
+    if (index < 0 || index >= int64_t(p->items.size())) return SYRK_ERR_SIZE;
+    const WorkItem& it = p->items[size_t(index)];
+    *kind = it.kind; *n_seg = it.n_seg; *n_tile = it.n_tile;
+    for (int s = 0; s < TBS_MAX_SEG; ++s) seg[s] = s < it.n_seg ? it.seg[s] : -1;
+    for (int t = 0; t < TBS_MAX_TILE; ++t) {
+        tile_x[t] = t < it.n_tile ? it.tile_x[t] : -1;
+        tile_y[t] = t < it.n_tile ? it.tile_y[t] : -1;
+    }
+    return SYRK_OK;
+}
+
+void tbs_plan_free(void* plan) { delete static_cast<Plan*>(plan); }
+
+int tbs_plan_simulate(const void* plan, int64_t N, int64_t M, int b, int64_t* a_loads, int64_t* c_loads,
+                      int32_t* min_cover, int32_t* max_cover, int32_t* upper_cover) {
+    if (!plan) return SYRK_ERR_NULL;
+    const Plan* p = static_cast<const Plan*>(plan);
+    if (N < 0 || M < 0 || b < 1 || (N + b - 1) / b != p->p.n_tiles) return SYRK_ERR_SIZE;
+    const SimResult r = simulate_plan(*p, N, M, b);
+    if (a_loads) *a_loads = r.a_loads;
+    if (c_loads) *c_loads = r.c_loads;
+    if (min_cover) *min_cover = r.min_cover;
+    if (max_cover) *max_cover = r.max_cover;
+    if (upper_cover) *upper_cover = r.upper_cover;
+    return SYRK_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,39 @@
+// Launchers of the CUDA kernels (internal to the library).
+#pragma once
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "tbs_plan.h"
+
+namespace tbsyrk {
+
+// FP64 triangle-block kernel: one thread block per work item.
+cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items,
+                            int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
+                            double beta, int* d_status, cudaStream_t stream);
+int f64_tile();
+int f64_bk();
+int f64_stages();
+
+// BF16 -> FP32 triangle-block kernel (tcgen05 / TMEM): persistent, one thread block per SM.
+// `split_k` > 1 makes every item run once per K-slice, partial tiles going to `d_partial`
+// (split_k x tiles x 128 x 128 floats) to be summed by the reduce kernel.
+cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items,
+                             int64_t N, int64_t M, float* C, int64_t ldc, float alpha, float beta,
+                             int split_k, float* d_partial, const int64_t* d_tile_base,
+                             int* d_status, int sm_count, cudaStream_t stream);
+int bf16_tile();
+int bf16_bk();
+int bf16_stages();
+
+// Plain-load kernels: one thread per lower-triangle entry.  Used when A does not meet
+// the TMA alignment rules; same result, much slower.
+cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, void* C,
+                              int64_t ldc, double alpha, double beta, cudaStream_t stream);
+
+// Lower triangle <- beta * lower triangle (zero when beta == 0, without reading C).
+cudaError_t launch_scale_lower(int dtype, int64_t N, void* C, int64_t ldc, double beta,
+                               cudaStream_t stream);
+
+}  // namespace tbsyrk

@@ -1,0 +1,183 @@
+// Host-side runtime: device state, work-list cache, TMA descriptors.
+#include "runtime.h"
+
+#include <cstdio>
+#include <cstdlib>
+#include <algorithm>
+#include <vector>
+
+#include "../../include/tbsyrk.h"
+#include "kernels.h"
+
+namespace tbsyrk {
+
+Runtime& runtime() {
+    static Runtime r;
+    return r;
+}
+
+KernelShape kernel_shape(int dtype) {
+    KernelShape s{};
+    if (dtype == SYRK_DTYPE_F64) {
+        // 32-row segments; k = 6 gives 15 of the 16 accumulator tiles a block can hold.
+        s.tile = f64_tile(); s.k = 6; s.rect_rows = 4; s.rect_cols = 4; s.diag_side = 4;
+        s.bk = f64_bk(); s.stages = f64_stages();
+        s.s_acc = int64_t(16) * s.tile * s.tile;
+    } else {
+        // 128-row segments; TMEM holds four 128 x 128 FP32 tiles, k = 3 uses three.
+        s.tile = bf16_tile(); s.k = 3; s.rect_rows = 2; s.rect_cols = 2; s.diag_side = 2;
+        s.bk = bf16_bk(); s.stages = bf16_stages();
+        s.s_acc = int64_t(4) * s.tile * s.tile;
+    }
+    return s;
+}
+
+bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out) {
+    const KernelShape ks = kernel_shape(dtype);
+    PlanParams p;
+    p.n_tiles = (N + ks.tile - 1) / ks.tile;
+    p.k = ks.k;
+    p.rect_rows = ks.rect_rows;
+    p.rect_cols = ks.rect_cols;
+    p.diag_side = ks.diag_side;
+    p.schedule = schedule;
+    return build_plan(p, out);
+}
+
+int get_device_state(DeviceState** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_NO_DEVICE; }
+    Runtime& rt = runtime();
+    auto it = rt.devices.find(dev);
+    if (it == rt.devices.end()) {
+        DeviceState ds;
+        ds.device = dev;
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_NO_DEVICE; }
+        ds.sm_count = prop.multiProcessorCount;
+        ds.cc_major = prop.major;
+        if (prop.major != 10) return SYRK_ERR_NO_DEVICE;  // kernels are built for sm_100a only
+        if (cudaMalloc(&ds.d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
+        if (cudaMemset(ds.d_status, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+        it = rt.devices.emplace(dev, std::move(ds)).first;
+    }
+    *out = &it->second;
+    return SYRK_OK;
+}
+
+int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
+    const KernelShape ks = kernel_shape(dtype);
+    const int64_t n_tiles = (N + ks.tile - 1) / ks.tile;
+    const auto key = std::make_tuple(n_tiles, dtype, runtime().schedule);
+    auto it = ds->plans.find(key);
+    if (it == ds->plans.end()) {
+        DevicePlan dp;
+        if (!build_host_plan(N, dtype, runtime().schedule, &dp.plan)) return SYRK_ERR_PLAN;
+        if (dtype == SYRK_DTYPE_BF16_F32) {
+            // The tcgen05 kernel's cost grows with the tiles an item owns: heaviest first.
+            std::stable_sort(dp.plan.items.begin(), dp.plan.items.end(),
+                             [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
+        }
+        const size_t n = dp.plan.items.size();
+        std::vector<int64_t> base(n + 1, 0);
+        for (size_t i = 0; i < n; ++i) base[i + 1] = base[i] + dp.plan.items[i].n_tile;
+        dp.total_tiles = base[n];
+        if (n > 0) {
+            if (cudaMalloc(&dp.d_items, n * sizeof(WorkItem)) != cudaSuccess ||
+                cudaMalloc(&dp.d_tile_base, (n + 1) * sizeof(int64_t)) != cudaSuccess) {
+                cudaGetLastError();
+                if (dp.d_items) cudaFree(dp.d_items);
+                return SYRK_ERR_ALLOC;
+            }
+            if (cudaMemcpy(dp.d_items, dp.plan.items.data(), n * sizeof(WorkItem), cudaMemcpyHostToDevice) != cudaSuccess ||
+                cudaMemcpy(dp.d_tile_base, base.data(), (n + 1) * sizeof(int64_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+                cudaGetLastError();
+                cudaFree(dp.d_items); cudaFree(dp.d_tile_base);
+                return SYRK_ERR_CUDA;
+            }
+        }
+        it = ds->plans.emplace(key, std::move(dp)).first;
+    }
+    *out = &it->second;
+    return SYRK_OK;
+}
+
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            p = nullptr;
+        }
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+}  // namespace
+
+int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, int64_t M,
+                         int64_t lda, int box_rows, int box_cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SYRK_ERR_CUDA;
+    const size_t es = (dtype == SYRK_DTYPE_F64) ? 8 : 2;
+    const cuuint64_t dims[2] = {cuuint64_t(M), cuuint64_t(N)};
+    const cuuint64_t strides[1] = {cuuint64_t(lda) * es};
+    const cuuint32_t box[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt =
+        (dtype == SYRK_DTYPE_F64) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult r = fn(tm, dt, 2, const_cast<void*>(A), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
+int ensure_device_bytes(void** p, size_t* have, size_t want) {
+    if (*have >= want && *p) return SYRK_OK;
+    if (*p) { cudaFree(*p); *p = nullptr; *have = 0; }
+    if (cudaMalloc(p, want) != cudaSuccess) { cudaGetLastError(); *p = nullptr; return SYRK_ERR_ALLOC; }
+    *have = want;
+    return SYRK_OK;
+}
+
+int ensure_pinned_bytes(void** p, size_t* have, size_t want) {
+    if (*have >= want && *p) return SYRK_OK;
+    if (*p) { cudaFreeHost(*p); *p = nullptr; *have = 0; }
+    if (cudaMallocHost(p, want) != cudaSuccess) { cudaGetLastError(); *p = nullptr; return SYRK_ERR_ALLOC; }
+    *have = want;
+    return SYRK_OK;
+}
+
+void release_all() {
+    Runtime& rt = runtime();
+    int prev = -1;
+    cudaGetDevice(&prev);
+    for (auto& kv : rt.devices) {
+        DeviceState& ds = kv.second;
+        cudaSetDevice(ds.device);
+        for (auto& pk : ds.plans) {
+            if (pk.second.d_items) cudaFree(pk.second.d_items);
+            if (pk.second.d_tile_base) cudaFree(pk.second.d_tile_base);
+        }
+        if (ds.d_status) cudaFree(ds.d_status);
+        if (ds.d_partial) cudaFree(ds.d_partial);
+        if (ds.d_a) cudaFree(ds.d_a);
+        if (ds.d_c) cudaFree(ds.d_c);
+        if (ds.d_packed) cudaFree(ds.d_packed);
+        if (ds.h_packed) cudaFreeHost(ds.h_packed);
+        if (ds.host_stream) cudaStreamDestroy(ds.host_stream);
+    }
+    rt.devices.clear();
+    if (prev >= 0) cudaSetDevice(prev);
+    cudaGetLastError();
+}
+
+}  // namespace tbsyrk

@@ -1,0 +1,77 @@
+// Host-side runtime of the library: per-device state, the cache of device-resident
+// work lists, TMA descriptor encoding.  Internal.
+#pragma once
+#include <cstdint>
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "tbs_plan.h"
+
+namespace tbsyrk {
+
+// Schedule parameters per dtype (tile side b, block side k, leftover shapes).
+struct KernelShape {
+    int tile;        // b
+    int k;           // segments per triangle block
+    int rect_rows, rect_cols, diag_side;
+    int bk, stages;  // staging: columns per stage, pipeline depth
+    int64_t s_acc;   // accumulator elements a thread block may hold
+};
+KernelShape kernel_shape(int dtype);
+
+struct DevicePlan {
+    Plan plan;
+    WorkItem* d_items = nullptr;
+    int64_t* d_tile_base = nullptr;  // first output-tile slot of each item (K-split workspace)
+    int64_t total_tiles = 0;
+};
+
+struct DeviceState {
+    int device = -1;
+    int sm_count = 0;
+    int cc_major = 0;
+    int* d_status = nullptr;
+    float* d_partial = nullptr;  // K-split workspace
+    size_t partial_bytes = 0;
+    // staging for the host-buffer entry point (grow-only)
+    void* d_a = nullptr; size_t d_a_bytes = 0;
+    void* d_c = nullptr; size_t d_c_bytes = 0;
+    void* d_packed = nullptr; size_t d_packed_bytes = 0;
+    void* h_packed = nullptr; size_t h_packed_bytes = 0;
+    cudaStream_t host_stream = nullptr;
+    std::map<std::tuple<int64_t, int, int>, DevicePlan> plans;  // (n_tiles, dtype, schedule)
+};
+
+struct Runtime {
+    std::mutex mu;
+    std::map<int, DeviceState> devices;
+    int schedule = 0;
+    int split_k = 0;
+};
+Runtime& runtime();
+
+// Current device's state, created on first use.  Returns a SYRK_* code.
+int get_device_state(DeviceState** out);
+
+// Plan for (N, dtype) under the current schedule, built and uploaded on first use.
+int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out);
+
+// Host-only plan (no device).
+bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out);
+
+// 2-D row-major tensor map over A (N x M, pitch lda elements) with a box of
+// box_rows x box_cols elements and 128-byte swizzle.
+int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, int64_t M,
+                         int64_t lda, int box_rows, int box_cols);
+
+// Grow-only device / pinned-host buffers.
+int ensure_device_bytes(void** p, size_t* have, size_t want);
+int ensure_pinned_bytes(void** p, size_t* have, size_t want);
+
+void release_all();
+
+}  // namespace tbsyrk

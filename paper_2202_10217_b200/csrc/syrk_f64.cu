@@ -1,0 +1,199 @@
+// FP64 triangle-block SYRK kernel for sm_100a.
+//
+// One thread block per work item of the tiled TBS schedule (Algorithm 4 and
+// Section 5.1.4 of the paper).  An item names up to 8 row segments of A (32 rows
+// each) and up to 16 output tiles C[seg x, seg y]; for a triangle block the tiles
+// are all pairs among k = 6 segments, so the block streams 6 segments per K-step
+// where a square block of the same accumulator count streams 8.
+//
+//   producer warp : plain TMA tile loads (no multicast) of the item's segments,
+//                   16 columns of A per stage, into a 6-stage shared-memory ring
+//                   (128-byte swizzle), signalled through mbarriers;
+//   16 MMA warps  : warp w owns tile w: a 32 x 32 accumulator held in registers as
+//                   4 x 4 blocks of mma.sync m8n8k4 (FP64 tensor core, DMMA);
+//   epilogue      : alpha * acc (+ beta * C) written for entries with col <= row
+//                   only, two doubles per store where alignment allows.
+//
+// Accumulators (the C block) stay on chip for the whole M loop and each entry of
+// C is read (beta != 0) and written exactly once, as in the paper's generic
+// out-of-core scheme (Algorithm 3).
+#include "device_utils.cuh"
+#include "kernels.h"
+#include "tbs_plan.h"
+
+namespace tbsyrk {
+namespace f64 {
+
+constexpr int kTile = 32;                       // b
+constexpr int kBK = 16;                         // columns of A per stage (128 bytes)
+constexpr int kStages = 6;
+constexpr int kSegBytes = kTile * kBK * 8;      // 4096
+constexpr int kStageBytes = kMaxSeg * kSegBytes;
+constexpr int kMmaWarps = 16;
+constexpr int kThreads = (kMmaWarps + 1) * 32;  // + producer warp
+constexpr int kSmemBytes = kStages * kStageBytes + 2 * kStages * 8 + 1024;
+
+__device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(c[0]), "+d"(c[1])
+                 : "d"(a), "d"(b));
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __restrict__ items,
+                    int64_t N, int32_t n_ksteps, double* __restrict__ C, int64_t ldc,
+                    double alpha, double beta, int vec_ok, int* __restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+    uint64_t* empty_bar = full_bar + kStages;
+    __shared__ WorkItem s_item;
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid < int(sizeof(WorkItem) / 4))
+        reinterpret_cast<int32_t*>(&s_item)[tid] = reinterpret_cast<const int32_t*>(&items[blockIdx.x])[tid];
+    if (tid == 0) s_abort = 0;
+    __syncthreads();
+
+    const int n_seg = s_item.n_seg, n_tile = s_item.n_tile;
+    if (tid == 0) {
+        bool ok = n_seg >= 1 && n_seg <= kMaxSeg && n_tile >= 1 && n_tile <= kMmaWarps;
+        for (int s = 0; ok && s < n_seg; ++s)
+            ok = s_item.seg[s] >= 0 && int64_t(s_item.seg[s]) * kTile < N;
+        for (int t = 0; ok && t < n_tile; ++t)
+            ok = s_item.tile_x[t] < n_seg && s_item.tile_y[t] < n_seg;
+        if (!ok) { s_abort = 1; atomicOr(status, kStatusBadItem); }
+        else {
+            for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], n_tile); }
+            mbar_fence_init();
+        }
+    }
+    __syncthreads();
+    if (s_abort) return;
+
+    if (warp == kMmaWarps) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            prefetch_tensormap(&tmA);
+            int issued = 0;
+            for (int ks = 0; ks < n_ksteps; ++ks) {
+                const int st = ks % kStages;
+                if (ks >= kStages &&
+                    !mbar_wait_bounded(&empty_bar[st], ((ks / kStages) - 1) & 1, &s_abort)) {
+                    s_abort = 1; atomicOr(status, kStatusWaitEmpty); break;
+                }
+                mbar_arrive_expect_tx(&full_bar[st], uint32_t(n_seg) * kSegBytes);
+                uint8_t* dst = smem + st * kStageBytes;
+                for (int s = 0; s < n_seg; ++s)
+                    tma_load_2d(dst + s * kSegBytes, &tmA, ks * kBK, s_item.seg[s] * kTile, &full_bar[st]);
+                issued = ks + 1;
+            }
+            if (s_abort) {
+                // Winding down: let the copies still in flight land before the block exits.
+                for (int ks = (issued > kStages ? issued - kStages : 0); ks < issued; ++ks) {
+                    int dummy = 0;
+                    mbar_wait_bounded(&full_bar[ks % kStages], (ks / kStages) & 1, &dummy);
+                }
+            }
+        }
+        return;
+    }
+    if (warp >= n_tile) return;
+
+    // ------------------------------ MMA warps ------------------------------
+    const int g = lane >> 2, t = lane & 3;
+    uint32_t off[4];
+#pragma unroll
+    for (int sl = 0; sl < 4; ++sl)
+        off[sl] = uint32_t(g * 128 + ((((sl << 1) | (t >> 1)) ^ g) << 4) + ((t & 1) << 3));
+    const int sx = s_item.tile_x[warp], sy = s_item.tile_y[warp];
+    const uint32_t xbase = uint32_t(sx) * kSegBytes, ybase = uint32_t(sy) * kSegBytes;
+
+    double acc[4][4][2];
+#pragma unroll
+    for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) acc[mi][ni][0] = acc[mi][ni][1] = 0.0;
+
+    bool alive = true;
+    for (int ks = 0; ks < n_ksteps; ++ks) {
+        const int st = ks % kStages;
+        if (!mbar_wait_bounded(&full_bar[st], (ks / kStages) & 1, &s_abort)) {
+            s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); alive = false; break;
+        }
+        const uint8_t* px = smem + st * kStageBytes + xbase;
+        const uint8_t* py = smem + st * kStageBytes + ybase;
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl) {
+            double a[4], b[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                a[j] = *reinterpret_cast<const double*>(px + off[sl] + j * 1024);
+                b[j] = *reinterpret_cast<const double*>(py + off[sl] + j * 1024);
+            }
+#pragma unroll
+            for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+                for (int ni = 0; ni < 4; ++ni) dmma884(acc[mi][ni], a[mi], b[ni]);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[st]);
+    }
+    if (!alive) return;
+
+    // ------------------------------ epilogue ------------------------------
+    const int64_t row0 = int64_t(s_item.seg[sx]) * kTile, col0 = int64_t(s_item.seg[sy]) * kTile;
+    const bool use_beta = (beta != 0.0);
+#pragma unroll
+    for (int mi = 0; mi < 4; ++mi) {
+        const int64_t r = row0 + mi * 8 + g;
+        if (r >= N) continue;
+        double* crow = C + r * ldc;
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) {
+            const int64_t c = col0 + ni * 8 + 2 * t;
+            double v0 = alpha * acc[mi][ni][0], v1 = alpha * acc[mi][ni][1];
+            if (c + 1 <= r) {
+                if (vec_ok) {
+                    double2* p = reinterpret_cast<double2*>(crow + c);
+                    if (use_beta) { const double2 o = *p; v0 += beta * o.x; v1 += beta * o.y; }
+                    *p = make_double2(v0, v1);
+                } else {
+                    if (use_beta) { v0 += beta * crow[c]; v1 += beta * crow[c + 1]; }
+                    crow[c] = v0; crow[c + 1] = v1;
+                }
+            } else if (c <= r) {
+                if (use_beta) v0 += beta * crow[c];
+                crow[c] = v0;
+            }
+        }
+    }
+}
+
+}  // namespace f64
+
+cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items,
+                            int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
+                            double beta, int* d_status, cudaStream_t stream) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(f64::syrk_f64_tbs_kernel,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, f64::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    if (n_items == 0) return cudaSuccess;
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0) ? 1 : 0;
+    const int32_t n_ksteps = int32_t((M + f64::kBK - 1) / f64::kBK);
+    f64::syrk_f64_tbs_kernel<<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
+        tmA, d_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, d_status);
+    return cudaGetLastError();
+}
+
+int f64_tile() { return f64::kTile; }
+int f64_bk() { return f64::kBK; }
+int f64_stages() { return f64::kStages; }
+
+}  // namespace tbsyrk

@@ -1,0 +1,73 @@
+// Plain-load SYRK and the scale-only kernel.
+//
+// syrk_plain: one thread per entry (i, j), j <= i, of the result of Algorithm 1 of the
+// paper with alpha/beta; no TMA, no alignment requirement.  It is the slow path for
+// inputs whose base address or row pitch is not a multiple of 16 bytes.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+
+namespace tbsyrk {
+namespace {
+
+template <typename TA, typename TC> struct Widen;
+template <> struct Widen<double, double> { static __device__ double get(const double* p) { return *p; } };
+template <> struct Widen<__nv_bfloat16, float> {
+    static __device__ float get(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+};
+
+template <typename TA, typename TC>
+__global__ void syrk_plain_kernel(int64_t N, int64_t M, const TA* __restrict__ A, int64_t lda,
+                                  TC* __restrict__ C, int64_t ldc, TC alpha, TC beta) {
+    const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
+    if (i >= N || j > i) return;
+    const TA* ai = A + i * lda;
+    const TA* aj = A + j * lda;
+    TC s = TC(0);
+    for (int64_t k = 0; k < M; ++k) s = fma(Widen<TA, TC>::get(ai + k), Widen<TA, TC>::get(aj + k), s);
+    TC* c = C + i * ldc + j;
+    *c = (beta == TC(0)) ? alpha * s : alpha * s + beta * *c;
+}
+
+template <typename TC>
+__global__ void scale_lower_kernel(int64_t N, TC* __restrict__ C, int64_t ldc, TC beta) {
+    const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
+    if (i >= N || j > i) return;
+    TC* c = C + i * ldc + j;
+    *c = (beta == TC(0)) ? TC(0) : beta * *c;
+}
+
+inline dim3 grid2d(int64_t N, dim3 block) {
+    return dim3(unsigned((N + block.x - 1) / block.x), unsigned((N + block.y - 1) / block.y));
+}
+
+}  // namespace
+
+cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, void* C,
+                              int64_t ldc, double alpha, double beta, cudaStream_t stream) {
+    if (N == 0) return cudaSuccess;
+    const dim3 block(32, 8);
+    if (dtype == 0)
+        syrk_plain_kernel<double, double><<<grid2d(N, block), block, 0, stream>>>(
+            N, M, static_cast<const double*>(A), lda, static_cast<double*>(C), ldc, alpha, beta);
+    else
+        syrk_plain_kernel<__nv_bfloat16, float><<<grid2d(N, block), block, 0, stream>>>(
+            N, M, static_cast<const __nv_bfloat16*>(A), lda, static_cast<float*>(C), ldc,
+            float(alpha), float(beta));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scale_lower(int dtype, int64_t N, void* C, int64_t ldc, double beta,
+                               cudaStream_t stream) {
+    if (N == 0) return cudaSuccess;
+    const dim3 block(32, 8);
+    if (dtype == 0)
+        scale_lower_kernel<double><<<grid2d(N, block), block, 0, stream>>>(N, static_cast<double*>(C), ldc, beta);
+    else
+        scale_lower_kernel<float><<<grid2d(N, block), block, 0, stream>>>(N, static_cast<float*>(C), ldc, float(beta));
+    return cudaGetLastError();
+}
+
+}  // namespace tbsyrk

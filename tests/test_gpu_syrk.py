@@ -1,0 +1,154 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU reference,
+entry by entry on the same seeded inputs.
+
+Tolerance (binary64 reference of the exact products):
+    |C_gpu - C_ref| <= tol * M * (|alpha| * (|A||A|^T)_ij + |beta| * |C_in,ij|)
+with tol = 8 * 2^-53 (FP64) and 4 * 2^-24 (BF16 inputs, FP32 accumulation).
+Integer-valued inputs must match bit for bit whatever the summation order.
+"""
+import numpy as np
+import pytest
+
+from oracle import syrk as O
+from paper_2202_10217_b200 import binding as B
+from paper_2202_10217_b200 import inputs as I
+
+from gpu_util import assert_within_tolerance, run_case
+
+pytestmark = pytest.mark.gpu
+BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32]
+DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16"])
+
+
+def make_A(N, M, dtype, seed, kind="normal"):
+    if kind == "int":
+        return I.small_int_f64(N, M, seed) if dtype == B.DTYPE_F64 else I.small_int_bf16(N, M, seed)
+    if dtype == B.DTYPE_F64:
+        return I.normal_f64(N, M, seed)
+    return I.normal_bf16(N, M, seed)
+
+
+# Sizes: below one tile, exact tiles, ragged tails in N and M, several tiles, and sizes
+# large enough for triangle blocks (FP64: >= 30 tile rows of 32; BF16: >= 6 tile rows of 128).
+SIZES_F64 = [(1, 1), (5, 3), (31, 17), (32, 16), (33, 50), (100, 64), (257, 130), (512, 256),
+             (1000, 70), (1300, 40)]
+SIZES_BF16 = [(1, 8), (5, 24), (127, 64), (128, 64), (129, 72), (300, 200), (512, 256),
+              (777, 136), (1100, 320), (2050, 72)]
+
+
+def sizes(dtype):
+    return SIZES_F64 if dtype == B.DTYPE_F64 else SIZES_BF16
+
+
+@DT
+def test_real_inputs_within_tolerance(dtype):
+    for n, (N, M) in enumerate(sizes(dtype)):
+        A = make_A(N, M, dtype, seed=100 + n)
+        got, ref, bound = run_case(A, dtype, 1.0, 0.0)
+        assert_within_tolerance(got, ref, bound, M, 1.0, 0.0, None, dtype)
+
+
+@DT
+def test_integer_inputs_are_bit_exact(dtype):
+    for n, (N, M) in enumerate(sizes(dtype)):
+        A = make_A(N, M, dtype, seed=200 + n, kind="int")
+        got, ref, bound = run_case(A, dtype, 1.0, 0.0)
+        assert_within_tolerance(got, ref, bound, M, 1.0, 0.0, None, dtype, exact=True)
+
+
+@DT
+@pytest.mark.parametrize("alpha,beta", [(-1.0, 1.0), (0.0, 1.0), (0.0, 0.0), (2.5, -0.5), (1.0, 2.0),
+                                        (0.0, -3.0)])
+def test_alpha_beta(dtype, alpha, beta):
+    N, M = (1000, 48) if dtype == B.DTYPE_F64 else (900, 128)
+    A = make_A(N, M, dtype, seed=7, kind="int")
+    Cin = (np.random.default_rng(9).integers(-8, 9, size=(N, N)) * 2).astype(I.c_storage_dtype(dtype))
+    got, ref, bound = run_case(A, dtype, alpha, beta, Cin=Cin)
+    if beta == 0.0:
+        ref, bound = O.syrk_lower(A, None, alpha, 0.0, dtype)
+    assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin, dtype, exact=True)
+    A = make_A(N, M, dtype, seed=8)
+    Cin = I.random_c(N, 10, dtype)
+    got, ref, bound = run_case(A, dtype, alpha, beta, Cin=Cin)
+    assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin, dtype)
+
+
+@DT
+def test_beta_zero_ignores_nan_in_C(dtype):
+    N, M = (200, 40) if dtype == B.DTYPE_F64 else (300, 64)
+    A = make_A(N, M, dtype, seed=3)
+    got, ref, bound = run_case(A, dtype, 1.0, 0.0, poison=True)
+    assert_within_tolerance(got, ref, bound, M, 1.0, 0.0, None, dtype)
+
+
+@DT
+def test_pitches_and_offsets(dtype):
+    N, M = (300, 50) if dtype == B.DTYPE_F64 else (400, 100)
+    A = make_A(N, M, dtype, seed=4)
+    Cin = I.random_c(N, 5, dtype)
+    step = 2 if dtype == B.DTYPE_F64 else 8           # keeps A 16-byte aligned (TMA path)
+    got, ref, bound = run_case(A, dtype, -1.0, 1.0, Cin=Cin, lda=M - M % step + 4 * step, ldc=N + 37,
+                               a_offset=3 * step, c_offset=5)
+    assert_within_tolerance(got, ref, bound, M, -1.0, 1.0, Cin, dtype)
+
+
+@DT
+def test_unaligned_A_takes_the_plain_kernel(dtype):
+    N, M = (150, 33) if dtype == B.DTYPE_F64 else (150, 77)
+    A = make_A(N, M, dtype, seed=6)
+    Cin = I.random_c(N, 5, dtype)
+    got, ref, bound = run_case(A, dtype, 1.5, 0.5, Cin=Cin, lda=M + (1 if dtype == B.DTYPE_F64 else 3),
+                               a_offset=1)
+    assert_within_tolerance(got, ref, bound, M, 1.5, 0.5, Cin, dtype)
+
+
+@DT
+def test_closed_forms(dtype):
+    N, M = (700, 96) if dtype == B.DTYPE_F64 else (640, 256)
+    got, ref, bound = run_case(I.ones(N, M, dtype), dtype, 1.0, 0.0)
+    assert np.all(got[np.tril_indices(N)] == float(M))
+    H = np.array([[1.0]])
+    while H.shape[0] < 256:
+        H = np.block([[H, H], [H, -H]])
+    got, ref, bound = run_case(I.to_storage(H / 16.0, dtype), dtype, 1.0, 0.0)   # orthonormal rows
+    assert np.array_equal(got[np.tril_indices(256)], np.eye(256)[np.tril_indices(256)])
+
+
+@DT
+def test_degenerate_sizes(dtype):
+    cdt = I.c_storage_dtype(dtype)
+    # M == 0: lower triangle <- beta * C
+    A = np.zeros((40, 0), dtype=np.float64 if dtype == B.DTYPE_F64 else np.uint16)
+    Cin = I.random_c(40, 1, dtype)
+    got, _, _ = run_case(A, dtype, 1.0, 2.0, Cin=Cin)
+    il = np.tril_indices(40)
+    assert np.array_equal(got[il], (cdt(2.0) * Cin[il]).astype(np.float64))
+    got, _, _ = run_case(A, dtype, 1.0, 0.0, poison=True)
+    assert np.all(got[il] == 0.0)
+    # N == 0 is a no-op
+    B.syrk_lower(0, 16, None, 16, None, 1, 1.0, 0.0, dtype)
+
+
+@DT
+def test_square_schedule_gives_the_same_result(dtype):
+    N, M = (1100, 64) if dtype == B.DTYPE_F64 else (1300, 192)
+    A = make_A(N, M, dtype, seed=12, kind="int")
+    try:
+        B.syrk_set_schedule(B.SCHEDULE_SQUARE)
+        got, ref, bound = run_case(A, dtype, 1.0, 0.0)
+    finally:
+        B.syrk_set_schedule(B.SCHEDULE_TBS)
+    assert_within_tolerance(got, ref, bound, M, 1.0, 0.0, None, dtype, exact=True)
+
+
+@DT
+def test_host_buffer_entry_point(dtype):
+    N, M = (333, 45) if dtype == B.DTYPE_F64 else (500, 90)
+    A = make_A(N, M, dtype, seed=13)
+    Cin = I.random_c(N, 14, dtype)
+    C = Cin.copy()
+    B.syrk_lower_host(N, M, A, M, C, N, -1.0, 1.0, dtype)
+    ref, bound = O.syrk_lower(A, Cin, -1.0, 1.0, dtype)
+    assert_within_tolerance(C.astype(np.float64), ref, bound, M, -1.0, 1.0, Cin, dtype)
+    iu = np.triu_indices(N, 1)
+    assert np.array_equal(C[iu], Cin[iu])               # host upper triangle untouched
