@@ -76,7 +76,7 @@ int run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_
             if (rc != SYRK_OK) return rc;
         }
         e = launch_syrk_bf16(tm, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
-                             float(beta), split, ds->d_partial, dp->d_tile_base, ds->d_status,
+                             float(beta), split, ds->d_partial, dp->d_tile_base, dp->total_tiles, ds->d_status,
                              ds->sm_count, stream);
     }
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
@@ -254,7 +254,7 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->c_elems = N * (N + 1) / 2;
     out->s_acc = ks.s_acc;
     out->s_total = ks.s_acc + int64_t(kMaxSeg) * ks.tile * ks.bk * ks.stages;
-    if (dtype == SYRK_DTYPE_BF16_F32) out->s_total = ks.s_acc + int64_t(4) * ks.tile * ks.bk * ks.stages;
+    if (dtype == SYRK_DTYPE_BF16_F32) out->s_total = ks.s_acc + int64_t(bf16_seg_slots()) * ks.tile * ks.bk * ks.stages;
     return SYRK_OK;
 }
 

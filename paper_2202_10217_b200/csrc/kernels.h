@@ -22,10 +22,11 @@ int f64_stages();
 cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items,
                              int64_t N, int64_t M, float* C, int64_t ldc, float alpha, float beta,
                              int split_k, float* d_partial, const int64_t* d_tile_base,
-                             int* d_status, int sm_count, cudaStream_t stream);
+                             int64_t total_tiles, int* d_status, int sm_count, cudaStream_t stream);
 int bf16_tile();
 int bf16_bk();
 int bf16_stages();
+int bf16_seg_slots();
 
 // Plain-load kernels: one thread per lower-triangle entry.  Used when A does not meet
 // the TMA alignment rules; same result, much slower.

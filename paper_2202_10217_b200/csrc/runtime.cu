@@ -24,10 +24,11 @@ KernelShape kernel_shape(int dtype) {
         s.bk = f64_bk(); s.stages = f64_stages();
         s.s_acc = int64_t(16) * s.tile * s.tile;
     } else {
-        // 128-row segments; TMEM holds four 128 x 128 FP32 tiles, k = 3 uses three.
-        s.tile = bf16_tile(); s.k = 3; s.rect_rows = 2; s.rect_cols = 2; s.diag_side = 2;
+        // 128-row segments, three per pipeline stage and three 128 x 128 FP32 accumulators in
+        // TMEM: a triangle block with k = 3, or a 1 x 2 rectangle, or two diagonal tile rows.
+        s.tile = bf16_tile(); s.k = 3; s.rect_rows = 1; s.rect_cols = 2; s.diag_side = 2;
         s.bk = bf16_bk(); s.stages = bf16_stages();
-        s.s_acc = int64_t(4) * s.tile * s.tile;
+        s.s_acc = int64_t(3) * s.tile * s.tile;
     }
     return s;
 }
@@ -78,6 +79,10 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
             std::stable_sort(dp.plan.items.begin(), dp.plan.items.end(),
                              [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
         }
+        const int max_seg = (dtype == SYRK_DTYPE_F64) ? kMaxSeg : bf16_seg_slots();
+        const int max_tile = (dtype == SYRK_DTYPE_F64) ? kMaxTile : 3;
+        for (const WorkItem& it : dp.plan.items)
+            if (it.n_seg > max_seg || it.n_tile > max_tile) return SYRK_ERR_PLAN;
         const size_t n = dp.plan.items.size();
         std::vector<int64_t> base(n + 1, 0);
         for (size_t i = 0; i < n; ++i) base[i + 1] = base[i] + dp.plan.items[i].n_tile;

@@ -1,11 +1,356 @@
-// placeholder until the tcgen05 kernel lands
+// BF16-in / FP32-accumulate triangle-block SYRK kernel for sm_100a (tcgen05 + TMEM).
+//
+// Persistent kernel, one thread block per SM, work units dealt round-robin.  A work
+// unit is one item of the tiled TBS schedule (Algorithm 4 / Section 5.1.4 of the
+// paper) restricted to one K-slice.  An item names up to 3 row segments of A (128
+// rows each) and up to 3 output tiles; for a triangle block (k = 3) the tiles are
+// (s1,s0), (s2,s0), (s2,s1): three 128 x 128 accumulators fed by three segments per
+// K-step, where a rectangle of the same staging footprint owns two.
+//
+//   warp 0   : producer - plain TMA tile loads (no multicast) of the item's segments,
+//              64 columns of A per stage, 4-stage ring, 128-byte swizzle;
+//   warp 1   : allocates tensor memory; one lane issues tcgen05.mma (M = 128,
+//              N = 128 or 256, K = 16) from shared-memory descriptors into TMEM
+//              accumulators and frees ring stages with tcgen05.commit;
+//   warps 2-5: epilogue - tcgen05.ld of the accumulators, alpha/beta, stores of the
+//              entries with col <= row only (or raw partial tiles when M is split).
+//
+// Both MMA operands come from the same row-major A (K contiguous): segment x is the
+// M-operand, segment y (or the adjacent pair y, y+1) the N-operand, both K-major.
+#include "device_utils.cuh"
 #include "kernels.h"
+#include "tbs_plan.h"
+
 namespace tbsyrk {
-cudaError_t launch_syrk_bf16(const CUtensorMap&, const WorkItem*, int64_t, int64_t, int64_t, float*, int64_t,
-                             float, float, int, float*, const int64_t*, int*, int, cudaStream_t) {
-    return cudaErrorNotSupported;
+namespace bf16 {
+
+constexpr int kTile = 128;                        // b
+constexpr int kBK = 64;                           // columns of A per stage (128 bytes)
+constexpr int kStages = 4;
+constexpr int kSegSlots = 3;                      // segments per stage
+constexpr int kSegBytes = kTile * kBK * 2;        // 16384
+constexpr int kStageBytes = kSegSlots * kSegBytes;
+constexpr int kMaxTiles = 3;                      // 3 x 128 TMEM columns of 512
+constexpr int kTmemCols = 512;
+constexpr int kThreads = 192;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+
+// ---- tcgen05 wrappers -------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
-int bf16_tile() { return 128; }
-int bf16_bk() { return 64; }
-int bf16_stages() { return 4; }
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, BF16 inputs, FP32 accumulation, M = 128.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (base + i).
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128
+// bytes, 8-row groups 1024 bytes apart; `addr` is the shared-memory byte address of
+// the first row (+ 32 bytes per K = 16 step inside the swizzle atom).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= uint64_t((addr & 0x3FFFF) >> 4);          // start address
+    d |= uint64_t(1024 >> 4) << 32;                // stride byte offset (between 8-row groups)
+    d |= uint64_t(1) << 46;                        // descriptor version of sm_100
+    d |= uint64_t(2) << 61;                        // layout: 128-byte swizzle
+    return d;
+}
+// Instruction descriptor, kind::f16: D = FP32, A = B = BF16, both K-major, M = 128.
+__device__ __forceinline__ uint32_t instr_desc_bf16(uint32_t n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+struct Unit {       // one work unit: an item and a range of K-steps
+    int64_t item;
+    int32_t slice;
+    int32_t k0, k1;
+};
+__device__ __forceinline__ Unit unit_of(int64_t w, int64_t n_items, int32_t n_ksteps, int32_t split) {
+    Unit u;
+    u.slice = int32_t(w / n_items);               // slice-major: a wave shares one K-slab of A
+    u.item = w % n_items;
+    u.k0 = int32_t(int64_t(n_ksteps) * u.slice / split);
+    u.k1 = int32_t(int64_t(n_ksteps) * (u.slice + 1) / split);
+    return u;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __restrict__ items,
+                     int64_t n_items, int64_t N, int32_t n_ksteps, float* __restrict__ C, int64_t ldc,
+                     float alpha, float beta, int vec_ok, int32_t split, float* __restrict__ partial,
+                     const int64_t* __restrict__ tile_base, int64_t total_tiles, int* __restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+    uint64_t* empty_bar = full_bar + kStages;
+    uint64_t* tmem_full_bar = empty_bar + kStages;
+    uint64_t* tmem_empty_bar = tmem_full_bar + 1;
+    uint64_t* drain_bar = tmem_empty_bar + 1;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ volatile int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t n_units = n_items * split;
+
+    if (tid == 0) {
+        s_abort = 0;
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(tmem_full_bar, 1);
+        mbar_init(tmem_empty_bar, 4);
+        mbar_init(drain_bar, 1);
+        mbar_fence_init();
+    }
+    if (warp == 1) tmem_alloc(&s_tmem_base, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            prefetch_tensormap(&tmA);
+            uint32_t g = 0;
+            for (int64_t w = blockIdx.x; w < n_units && !s_abort; w += gridDim.x) {
+                const Unit u = unit_of(w, n_items, n_ksteps, split);
+                const WorkItem* it = &items[u.item];
+                const int n_seg = it->n_seg;
+                int32_t rows[kSegSlots];
+                for (int s = 0; s < kSegSlots; ++s) rows[s] = (s < n_seg) ? it->seg[s] * kTile : 0;
+                for (int ks = u.k0; ks < u.k1; ++ks, ++g) {
+                    const uint32_t st = g % kStages;
+                    if (g >= kStages && !mbar_wait_bounded(&empty_bar[st], ((g / kStages) - 1) & 1, &s_abort)) {
+                        s_abort = 1; atomicOr(status, kStatusWaitEmpty); break;
+                    }
+                    mbar_arrive_expect_tx(&full_bar[st], uint32_t(n_seg) * kSegBytes);
+                    uint8_t* dst = smem + st * kStageBytes;
+                    for (int s = 0; s < n_seg; ++s)
+                        tma_load_2d(dst + s * kSegBytes, &tmA, ks * kBK, rows[s], &full_bar[st]);
+                }
+            }
+            if (s_abort) {   // winding down: let the copies still in flight land first
+                volatile int dummy = 0;
+                for (uint32_t i = (g > kStages ? g - kStages : 0); i < g; ++i)
+                    mbar_wait_bounded(&full_bar[i % kStages], (i / kStages) & 1, &dummy);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            uint32_t g = 0, n_done = 0;
+            const uint32_t smem_base = smem_u32(smem);
+            for (int64_t w = blockIdx.x; w < n_units && !s_abort; w += gridDim.x, ++n_done) {
+                const Unit u = unit_of(w, n_items, n_ksteps, split);
+                const WorkItem* it = &items[u.item];
+                const int n_tile = it->n_tile;
+                // MMA groups: tile t alone (N = 128), or tiles t, t+1 with the same M-operand
+                // and adjacent N-operand segments (N = 256).
+                int gx[kMaxTiles], gy[kMaxTiles], gn[kMaxTiles], gcol[kMaxTiles], n_grp = 0;
+                for (int t = 0; t < n_tile;) {
+                    const int x = it->tile_x[t], y = it->tile_y[t];
+                    const bool pair = (t + 1 < n_tile) && it->tile_x[t + 1] == x && it->tile_y[t + 1] == y + 1;
+                    gx[n_grp] = x; gy[n_grp] = y; gn[n_grp] = pair ? 256 : 128; gcol[n_grp] = t * kTile;
+                    ++n_grp;
+                    t += pair ? 2 : 1;
+                }
+                if (n_done > 0 && !mbar_wait_bounded(tmem_empty_bar, (n_done - 1) & 1, &s_abort)) {
+                    s_abort = 1; atomicOr(status, kStatusWaitTmem); break;
+                }
+                tc_fence_after();
+                bool ok = true;
+                for (int ks = u.k0; ks < u.k1; ++ks, ++g) {
+                    const uint32_t st = g % kStages;
+                    if (!mbar_wait_bounded(&full_bar[st], (g / kStages) & 1, &s_abort)) {
+                        s_abort = 1; atomicOr(status, kStatusWaitFull); ok = false; break;
+                    }
+                    tc_fence_after();
+                    const uint32_t stage_addr = smem_base + st * kStageBytes;
+                    for (int q = 0; q < n_grp; ++q) {
+                        const uint32_t a_addr = stage_addr + gx[q] * kSegBytes;
+                        const uint32_t b_addr = stage_addr + gy[q] * kSegBytes;
+                        const uint32_t idesc = instr_desc_bf16(uint32_t(gn[q]));
+#pragma unroll
+                        for (int kk = 0; kk < kBK / 16; ++kk)
+                            tc_mma_bf16(tmem_base + uint32_t(gcol[q]), smem_desc_sw128(a_addr + kk * 32),
+                                        smem_desc_sw128(b_addr + kk * 32), idesc, (ks > u.k0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(&empty_bar[st]);    // stage reusable once these MMAs have read it
+                }
+                if (!ok) break;
+                tc_commit(tmem_full_bar);         // accumulators complete
+            }
+            if (s_abort) {                        // let issued MMAs finish before TMEM is freed
+                volatile int dummy = 0;
+                tc_commit(drain_bar);
+                mbar_wait_bounded(drain_bar, 0, &dummy);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------ epilogue ------------------------------
+        const int quarter = warp & 3;                     // TMEM lanes this warp may read
+        const int row_in_tile = quarter * 32 + lane;
+        uint32_t n_done = 0;
+        for (int64_t w = blockIdx.x; w < n_units && !s_abort; w += gridDim.x, ++n_done) {
+            const Unit u = unit_of(w, n_items, n_ksteps, split);
+            const WorkItem* it = &items[u.item];
+            const int n_tile = it->n_tile;
+            if (!mbar_wait_bounded(tmem_full_bar, n_done & 1, &s_abort)) {
+                s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitMma); break;
+            }
+            tc_fence_after();
+            for (int t = 0; t < n_tile; ++t) {
+                const int64_t trow = it->seg[it->tile_x[t]], tcol = it->seg[it->tile_y[t]];
+                const int64_t r = trow * kTile + row_in_tile;
+                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(t * kTile);
+#pragma unroll 1
+                for (int cb = 0; cb < kTile; cb += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(taddr + cb, v);
+                    if (split > 1) {
+                        float4* dst = reinterpret_cast<float4*>(
+                            partial + ((int64_t(u.slice) * total_tiles + tile_base[u.item] + t) * kTile + row_in_tile) * kTile + cb);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                 __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        continue;
+                    }
+                    if (r >= N) continue;
+                    const int64_t c0 = tcol * kTile + cb;
+                    float* crow = C + r * ldc + c0;
+                    if (c0 + 31 <= r && vec_ok) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            float4 o = make_float4(alpha * __uint_as_float(v[4 * j]), alpha * __uint_as_float(v[4 * j + 1]),
+                                                   alpha * __uint_as_float(v[4 * j + 2]), alpha * __uint_as_float(v[4 * j + 3]));
+                            float4* p = reinterpret_cast<float4*>(crow) + j;
+                            if (beta != 0.f) {
+                                const float4 old = *p;
+                                o.x += beta * old.x; o.y += beta * old.y; o.z += beta * old.z; o.w += beta * old.w;
+                            }
+                            *p = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (c0 + j <= r) {
+                                float o = alpha * __uint_as_float(v[j]);
+                                if (beta != 0.f) o += beta * crow[j];
+                                crow[j] = o;
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tmem_empty_bar);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// Sum of the K-slices' partial tiles in slice order, then alpha/beta and the triangle mask.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const WorkItem* __restrict__ items, const int64_t* __restrict__ tile_base,
+                     int64_t total_tiles, int32_t split, const float* __restrict__ partial, int64_t N,
+                     float* __restrict__ C, int64_t ldc, float alpha, float beta) {
+    const WorkItem* it = &items[blockIdx.x];
+    const int t = blockIdx.y;
+    if (t >= it->n_tile) return;
+    const int64_t slot = tile_base[blockIdx.x] + t;
+    const int64_t row0 = int64_t(it->seg[it->tile_x[t]]) * kTile, col0 = int64_t(it->seg[it->tile_y[t]]) * kTile;
+    for (int e = threadIdx.x; e < kTile * kTile / 4; e += blockDim.x) {
+        const int rr = e / (kTile / 4), cc = (e % (kTile / 4)) * 4;
+        const int64_t r = row0 + rr;
+        if (r >= N) continue;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sl = 0; sl < split; ++sl) {
+            const float4 p = *reinterpret_cast<const float4*>(
+                partial + ((int64_t(sl) * total_tiles + slot) * kTile + rr) * kTile + cc);
+            s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+        }
+        const float vals[4] = {s.x, s.y, s.z, s.w};
+        float* crow = C + r * ldc + col0 + cc;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (col0 + cc + j <= r) {
+                float o = alpha * vals[j];
+                if (beta != 0.f) o += beta * crow[j];
+                crow[j] = o;
+            }
+        }
+    }
+}
+
+}  // namespace bf16
+
+cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items, int64_t N,
+                             int64_t M, float* C, int64_t ldc, float alpha, float beta, int split_k,
+                             float* d_partial, const int64_t* d_tile_base, int64_t total_tiles,
+                             int* d_status, int sm_count, cudaStream_t stream) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(bf16::syrk_bf16_tbs_kernel,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, bf16::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    if (n_items == 0) return cudaSuccess;
+    const int32_t n_ksteps = int32_t((M + bf16::kBK - 1) / bf16::kBK);
+    const int split = split_k < 1 ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
+    const int64_t n_units = n_items * split;
+    const unsigned grid = unsigned(n_units < sm_count ? n_units : sm_count);
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0) ? 1 : 0;
+    bf16::syrk_bf16_tbs_kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
+        tmA, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, split, d_partial, d_tile_base,
+        total_tiles, d_status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || split == 1) return e;
+    bf16::splitk_reduce_kernel<<<dim3(unsigned(n_items), bf16::kMaxTiles), 256, 0, stream>>>(
+        d_items, d_tile_base, total_tiles, split, d_partial, N, C, ldc, alpha, beta);
+    return cudaGetLastError();
+}
+
+int bf16_tile() { return bf16::kTile; }
+int bf16_bk() { return bf16::kBK; }
+int bf16_stages() { return bf16::kStages; }
+int bf16_seg_slots() { return bf16::kSegSlots; }
+
 }  // namespace tbsyrk

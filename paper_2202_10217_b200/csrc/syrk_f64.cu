@@ -48,7 +48,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
     uint64_t* empty_bar = full_bar + kStages;
     __shared__ WorkItem s_item;
-    __shared__ int s_abort;
+    __shared__ volatile int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -93,7 +93,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
             if (s_abort) {
                 // Winding down: let the copies still in flight land before the block exits.
                 for (int ks = (issued > kStages ? issued - kStages : 0); ks < issued; ++ks) {
-                    int dummy = 0;
+                    volatile int dummy = 0;
                     mbar_wait_bounded(&full_bar[ks % kStages], (ks / kStages) & 1, &dummy);
                 }
             }

@@ -10,7 +10,7 @@
 //              rows  r_u = u*c + f(u),  f(0) = j,  f(u) = (i + j*(u-1)) mod c
 //              (cyclic indexing family, Section 5.1.2).
 // Integer arithmetic only.  The square-block fallback is only cited by the paper;
-// here it is a band decomposition: bands of `rect_rows` tile rows, each cut into
+// here it is a band decomposition: bands of `diag_side` tile rows, each cut into
 // rect_rows x rect_cols rectangles left of the diagonal plus one diagonal block.
 #include "tbs_plan.h"
 
@@ -90,10 +90,12 @@ struct Builder {
 
     // {(r, t) : row_lo <= r < row_hi, col_lo <= t <= r}, col_lo <= row_lo
     void square_blocks(int64_t row_lo, int64_t row_hi, int64_t col_lo) {
-        for (int64_t r0 = row_lo; r0 < row_hi; r0 += p.rect_rows) {
-            const int64_t r1 = std::min<int64_t>(r0 + p.rect_rows, row_hi);
-            for (int64_t c0 = col_lo; c0 < r0; c0 += p.rect_cols)
-                rect_item(r0, r1, c0, std::min<int64_t>(c0 + p.rect_cols, r0));
+        for (int64_t r0 = row_lo; r0 < row_hi; r0 += p.diag_side) {
+            const int64_t r1 = std::min<int64_t>(r0 + p.diag_side, row_hi);
+            for (int64_t q0 = r0; q0 < r1; q0 += p.rect_rows)
+                for (int64_t c0 = col_lo; c0 < r0; c0 += p.rect_cols)
+                    rect_item(q0, std::min<int64_t>(q0 + p.rect_rows, r1), c0,
+                              std::min<int64_t>(c0 + p.rect_cols, r0));
             diag_item(r0, r1);
         }
     }
@@ -148,7 +150,7 @@ bool build_plan(const PlanParams& p, Plan* out) {
     if (p.rect_rows < 1 || p.rect_cols < 1 || p.rect_rows + p.rect_cols > kMaxSeg ||
         p.rect_rows * p.rect_cols > kMaxTile)
         return false;
-    if (p.diag_side != p.rect_rows || p.diag_side * (p.diag_side + 1) / 2 > kMaxTile) return false;
+    if (p.diag_side < p.rect_rows || p.diag_side > kMaxSeg || p.diag_side * (p.diag_side + 1) / 2 > kMaxTile) return false;
     if (p.schedule != 0 && p.schedule != 1) return false;
     out->p = p;
     out->c_top = 0;

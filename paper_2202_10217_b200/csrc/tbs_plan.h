@@ -30,7 +30,7 @@ struct PlanParams {
     int k = 3;            // segments per triangle block
     int rect_rows = 2;    // square-block fallback: rows x cols tiles per item
     int rect_cols = 2;
-    int diag_side = 2;    // adjacent tile rows per diagonal item (== rect_rows)
+    int diag_side = 2;    // adjacent tile rows per diagonal item and per band (>= rect_rows)
     int schedule = 0;     // 0: triangle blocks + leftovers, 1: squares only
 };
 

@@ -57,11 +57,11 @@ def plan_ops(plan):
     return ops
 
 
-@pytest.mark.parametrize("k,rr,rc", [(3, 2, 2), (6, 4, 4), (4, 3, 3), (5, 4, 4)])
+@pytest.mark.parametrize("k,rr,rc,dg", [(3, 2, 2, 2), (6, 4, 4, 4), (4, 3, 3, 3), (5, 4, 4, 4), (3, 1, 2, 2), (4, 2, 3, 5)])
 @pytest.mark.parametrize("schedule", [B.SCHEDULE_TBS, B.SCHEDULE_SQUARE])
-def test_work_list_covers_every_tile_exactly_once(k, rr, rc, schedule):
+def test_work_list_covers_every_tile_exactly_once(k, rr, rc, dg, schedule):
     for n_t in list(range(0, 41)) + [64, 128, 131, 256]:
-        plan = B.Plan(n_t, k, rr, rc, rr, schedule)
+        plan = B.Plan(n_t, k, rr, rc, dg, schedule)
         cover = np.zeros((n_t, n_t), dtype=np.int64)
         for kind, seg, pairs in plan_ops(plan):
             assert len(set(seg)) == len(seg) and all(0 <= s < n_t for s in seg)
