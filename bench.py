@@ -1,0 +1,306 @@
+#!/usr/bin/env python
+"""Benchmark of the triangle-block SYRK library on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c1]
+                    [--impl ours|reference]
+
+A step is one SYRK call (the whole hot path: work-list lookup, TMA streaming, tensor-core
+update, epilogue) on one seeded synthetic workload.  Prints ONE JSON line (rank 0).
+With N > 1 every rank runs an independent replica on its own GPU (the path has no
+exchange step); the value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2202_10217_b200 import inputs as I
+
+METRIC = "syrk_tflops_N(N+1)M"
+UNIT = "TFLOP/s"
+DTYPE_NAME = {I.DTYPE_F64: "f64", I.DTYPE_BF16_F32: "bf16_in_f32_acc"}
+ELEM_A = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 2}
+ELEM_C = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 4}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons (one `nvidia-smi -lms` process) while the
+    timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int, period_ms: int = 20):
+        self.cmd = ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
+                    "--format=csv,noheader,nounits", "-lms", str(period_ms)]
+        self.proc = None
+        self.rows = []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            time.sleep(0.15)                      # let the first samples arrive before the load starts
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is None:
+            return
+        self.proc.terminate()                     # the exact process started above
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        self.rows = [[x.strip() for x in line.split(",")] for line in out.splitlines() if line.strip()]
+
+    def summary(self):
+        sm, mx, power, reasons = [], 0.0, [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = max(mx, float(r[1]))
+                power.append(float(r[2]))
+                for name, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        # "under load": samples drawing more than half of the largest power seen
+        load = [c for c, w in zip(sm, power) if power and w >= 0.5 * max(power)]
+        return {"sm_mhz": float(np.median(load)) if load else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm), "samples_under_load": len(load),
+                "power_w_max": max(power) if power else None}
+
+
+def cpu_reference_sample(wl: I.Workload, A: np.ndarray, target_macs: float = 2.0e11):
+    """Times the CPU reference, as it stands, on a bounded sample of the workload.
+
+    The sample is the first R rows of the lower triangle (R chosen so that the work is
+    about `target_macs` multiply-adds); throughput is scaled to the metric's unit by the
+    flops of the sampled part, 2 * M per entry.
+    """
+    from oracle import syrk as O
+    N, M = wl.N, wl.M
+    R = int(min(N, max(64, np.sqrt(2.0 * target_macs / M))))
+    sub = np.ascontiguousarray(A[:R])
+    t0 = time.perf_counter()
+    O.syrk_lower(sub, None, wl.alpha, 0.0, wl.dtype)
+    dt = time.perf_counter() - t0
+    flops = R * (R + 1) * M
+    return {"value": flops / dt * 1e-12, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": "first %d of %d rows of the lower triangle (%.3g flops, %.1f s)" % (R, N, flops, dt)}
+
+
+def run_reference(args, wl: I.Workload, rank: int):
+    """--impl reference: the CPU oracle on host cores, rank 0 only."""
+    if rank != 0:
+        return
+    A = wl.make_A()
+    target = 6.0e9
+    for _ in range(args.warmup):
+        cpu_reference_sample(wl, A, target_macs=target / 8)
+    vals, t0 = [], time.perf_counter()
+    for _ in range(args.steps):
+        vals.append(cpu_reference_sample(wl, A, target_macs=target))
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    last = vals[-1]
+    value = float(np.mean([v["value"] for v in vals]))
+    base = dict(last)
+    base["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "N": wl.N, "M": wl.M, "alpha": wl.alpha, "beta": wl.beta,
+                   "note": "CPU oracle (plain triple loop) on a bounded sample per step"},
+        "cpu_baseline": base,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/.  Valid only for the kernel source it was taken on.
+NCU_TRAFFIC = {
+    # workload: (bytes per launch, sha256 of the kernel source at capture time)
+}
+
+
+def kernel_source_hash(dtype: int) -> str:
+    import hashlib
+    name = "syrk_f64.cu" if dtype == I.DTYPE_F64 else "syrk_bf16.cu"
+    with open(os.path.join(ROOT, "paper_2202_10217_b200", "csrc", name), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()
+
+
+def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
+    import torch
+    from paper_2202_10217_b200 import binding as B
+
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    N, M, dtype = wl.N, wl.M, wl.dtype
+    A_host = wl.make_A()
+    cdt = I.c_storage_dtype(dtype)
+    if dtype == I.DTYPE_F64:
+        A_pinned = torch.from_numpy(A_host).pin_memory()
+        dA = A_pinned.cuda()
+    else:
+        A_pinned = torch.from_numpy(A_host.view(np.int16)).pin_memory()
+        dA = A_pinned.cuda().view(torch.bfloat16)
+    C_pinned = torch.zeros((N, N), dtype=torch.float64 if dtype == I.DTYPE_F64 else torch.float32).pin_memory()
+    dC = torch.zeros((N, N), dtype=C_pinned.dtype, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > L2 (126 MB)
+
+    B.syrk_plan_prepare(N, M, dtype)
+    stats = B.syrk_get_schedule_stats(N, M, dtype)
+    n_warm = args.warmup if args.kernel_only else max(args.warmup, 3)
+    for _ in range(n_warm):
+        B.syrk_lower(N, M, dA, M, dC, N, wl.alpha, wl.beta, dtype)
+    torch.cuda.synchronize()
+    assert B.syrk_last_status() == 0
+
+    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        for i in range(args.steps):
+            flush.zero_()                                  # evict A and C from L2 (not timed)
+            ev0[i].record()
+            B.syrk_lower(N, M, dA, M, dC, N, wl.alpha, wl.beta, dtype)
+            ev1[i].record()
+        barrier()
+    assert B.syrk_last_status() == 0
+    times = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
+    total_ms = float(sum(times))
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * wl.flops / (ms_per_step * 1e-3) * 1e-12
+
+    if args.kernel_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+                              "steps": args.steps, "ms_per_step": ms_per_step, "kernel_only": True,
+                              "config": {"workload": wl.name, "N": N, "M": M}}))
+        return
+
+    # end to end: host buffers through the C ABI, copies inside the timed region
+    e2e_steps = max(1, min(args.steps, 3))
+    B.syrk_lower_host(N, M, A_pinned, M, C_pinned, N, wl.alpha, wl.beta, dtype)      # warm-up (allocates staging)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        B.syrk_lower_host(N, M, A_pinned, M, C_pinned, N, wl.alpha, wl.beta, dtype)
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * wl.flops / e2e_s * 1e-12, "unit": UNIT,
+           "h2d_bytes_per_step": N * M * ELEM_A[dtype] + (N * N * ELEM_C[dtype] if wl.beta != 0 else 0),
+           "d2h_bytes_per_step": N * (N + 1) // 2 * ELEM_C[dtype]}
+
+    if rank != 0:
+        return
+    peaks, peak_kind = measured_peaks()
+    kernel_ms = float(np.mean(times))
+    achieved = wl.flops / (kernel_ms * 1e-3) * 1e-12
+    if dtype == I.DTYPE_F64:
+        peak = B.syrk_probe_f64_mma_peak(20000)
+        peak_note = ("FP64 tensor-core (DMMA) rate measured in this run by the library's register-only "
+                     "mma.sync probe; MEASURED_PEAKS.json has no FP64 figure (bf16 %s %.1f x 40/2250 = %.1f)"
+                     % (peak_kind, peaks["bf16_tflops"], peaks["bf16_tflops"] * 40.0 / 2250.0))
+    else:
+        peak = float(peaks["bf16_tflops"])
+        peak_note = "cuBLAS bf16 burst, MEASURED_PEAKS.json (%s); sustained %.1f" % (
+            peak_kind, peaks.get("bf16_tflops_sustained", float("nan")))
+    traffic = None
+    if wl.name in NCU_TRAFFIC and NCU_TRAFFIC[wl.name][1] == kernel_source_hash(dtype):
+        traffic = NCU_TRAFFIC[wl.name][0]
+    launches_per_step = 1 if dtype == I.DTYPE_F64 else (2 if stats["split_k"] > 1 else 1)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": DTYPE_NAME[dtype], "data": "synthetic",
+        "config": {"workload": wl.name, "N": N, "M": M, "alpha": wl.alpha, "beta": wl.beta,
+                   "schedule": "tbs", "tile": stats["tile"], "k": stats["k"], "items": stats["items"],
+                   "tri_items": stats["tri_items"], "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "l2": "256 MiB buffer written between timed steps (L2 flush)"},
+        "clocks": clocks.summary(),
+        "e2e": e2e,
+        "gpu_launches": args.steps * launches_per_step,
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": UNIT,
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_note,
+                     "algorithmic_flops_per_launch": wl.flops,
+                     "model_a_bytes_per_launch": stats["a_loads"] * ELEM_A[dtype]},
+    }
+    if world == 1:
+        line["cpu_baseline"] = cpu_reference_sample(wl, A_host)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2", choices=sorted(I.CONFIGS))
+    ap.add_argument("--shape", default=None,
+                    help="N,M,dtype,alpha,beta (dtype f64|bf16): a custom seeded N(0,1) workload")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="device-timed kernel steps only (no end-to-end leg, CPU baseline or peak probe); "
+                         "for short profiler runs")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = I.CONFIGS[args.workload]
+    if args.shape:
+        n, m, dt, al, be = args.shape.split(",")
+        dtype = I.DTYPE_F64 if dt == "f64" else I.DTYPE_BF16_F32
+        wl = I.Workload("custom_%s_%sx%s" % (dt, n, m), int(n), int(m), dtype, float(al), float(be), 99, "normal")
+    if args.impl == "reference":
+        run_reference(args, wl, rank)
+        return
+    run_ours(args, wl, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -82,10 +82,11 @@ int syrk_lower(int64_t N, int64_t M,
 
 /*
  * Same operation with HOST buffers: copies A (and C when beta != 0) to the
- * device, runs syrk_lower, copies the lower triangle back into C, and waits for
- * completion.  A and C are host pointers (pageable or pinned).  The strict upper
- * triangle of the host C is left as it was.  Device buffers are allocated per
- * call and freed before returning.
+ * device, runs syrk_lower on a stream of the library, copies the lower triangle
+ * back into C, and waits for completion.  A and C are host pointers (pageable or
+ * pinned; pinned memory copies faster).  The strict upper triangle of the host C is
+ * left as it was.  The device and pinned staging buffers are kept by the library
+ * (they only grow) and are released by syrk_shutdown().
  */
 int syrk_lower_host(int64_t N, int64_t M,
                     const void* A, int64_t lda,
@@ -109,6 +110,14 @@ const char* syrk_strerror(int code);
 
 /* Select the schedule used by later calls (process-wide). */
 int syrk_set_schedule(int schedule);
+
+/*
+ * Diagnostic, no counterpart in the paper: measures this GPU's FP64 tensor-core
+ * (DMMA) throughput with a register-only mma.sync loop of `iters` iterations per
+ * warp (about 20000 gives ~20 ms) on the current device and default stream, waits
+ * for it, and returns TFLOP/s in *tflops.  Allocates and frees a small device buffer.
+ */
+int syrk_probe_f64_mma_peak(int iters, double* tflops);
 
 /* Force the number of K-slices (0 = automatic) used by later bf16 calls. */
 int syrk_set_split_k(int slices);

@@ -22,6 +22,7 @@ MAX_SEG, MAX_TILE = 8, 16
 EXPORTS = [
     "syrk_lower", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_get_schedule_stats",
+    "syrk_probe_f64_mma_peak",
     "tbs_plan_build", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
 ]
 
@@ -74,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.syrk_set_split_k.argtypes = [ci]
         L.syrk_get_schedule_stats.restype = ci
         L.syrk_get_schedule_stats.argtypes = [i64, i64, ci, ctypes.POINTER(ScheduleStats)]
+        L.syrk_probe_f64_mma_peak.restype = ci
+        L.syrk_probe_f64_mma_peak.argtypes = [ci, ctypes.POINTER(dbl)]
         L.tbs_plan_build.restype = vp
         L.tbs_plan_build.argtypes = [i64, ci, ci, ci, ci, ci]
         L.tbs_plan_num_items.restype = i64
@@ -157,6 +160,13 @@ def syrk_get_schedule_stats(N: int, M: int, dtype: int) -> dict:
     st = ScheduleStats()
     _check(lib().syrk_get_schedule_stats(N, M, dtype, ctypes.byref(st)))
     return st.as_dict()
+
+
+def syrk_probe_f64_mma_peak(iters: int = 20000) -> float:
+    """Measured FP64 tensor-core throughput of the current GPU, TFLOP/s."""
+    out = ctypes.c_double()
+    _check(lib().syrk_probe_f64_mma_peak(iters, ctypes.byref(out)))
+    return float(out.value)
 
 
 class Plan:
