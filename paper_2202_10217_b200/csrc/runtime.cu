@@ -81,8 +81,19 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
         }
         const int max_seg = (dtype == SYRK_DTYPE_F64) ? kMaxSeg : bf16_seg_slots();
         const int max_tile = (dtype == SYRK_DTYPE_F64) ? kMaxTile : 3;
-        for (const WorkItem& it : dp.plan.items)
+        for (const WorkItem& it : dp.plan.items) {
             if (it.n_seg > max_seg || it.n_tile > max_tile) return SYRK_ERR_PLAN;
+            if (dtype == SYRK_DTYPE_BF16_F32) {   // TMEM layout: at most one lone tile and one adjacent pair
+                int lone = 0, pairs = 0;
+                for (int t = 0; t < it.n_tile;) {
+                    const bool pair = t + 1 < it.n_tile && it.tile_x[t + 1] == it.tile_x[t] &&
+                                      it.tile_y[t + 1] == it.tile_y[t] + 1;
+                    pair ? ++pairs : ++lone;
+                    t += pair ? 2 : 1;
+                }
+                if (lone > 1 || pairs > 1) return SYRK_ERR_PLAN;
+            }
+        }
         const size_t n = dp.plan.items.size();
         std::vector<int64_t> base(n + 1, 0);
         for (size_t i = 0; i < n; ++i) base[i + 1] = base[i] + dp.plan.items[i].n_tile;
@@ -142,6 +153,19 @@ int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, i
     const CUresult r = fn(tm, dt, 2, const_cast<void*>(A), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
+int encode_tensor_map_c_f32(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SYRK_ERR_CUDA;
+    const cuuint64_t dims[2] = {cuuint64_t(N), cuuint64_t(N)};
+    const cuuint64_t strides[1] = {cuuint64_t(ldc) * 4};
+    const cuuint32_t bx[2] = {cuuint32_t(box), cuuint32_t(box)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(C), dims, strides, bx, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
 }
 

@@ -68,6 +68,9 @@ bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out);
 int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, int64_t M,
                          int64_t lda, int box_rows, int box_cols);
 
+// 2-D row-major FP32 tensor map over C (N x N, pitch ldc) with box x box boxes, 128-byte swizzle.
+int encode_tensor_map_c_f32(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box);
+
 // Grow-only device / pinned-host buffers.
 int ensure_device_bytes(void** p, size_t* have, size_t want);
 int ensure_pinned_bytes(void** p, size_t* have, size_t want);

@@ -12,8 +12,15 @@
 //   warp 1   : allocates tensor memory; one lane issues tcgen05.mma (M = 128,
 //              N = 128 or 256, K = 16) from shared-memory descriptors into TMEM
 //              accumulators and frees ring stages with tcgen05.commit;
-//   warps 2-5: epilogue - tcgen05.ld of the accumulators, alpha/beta, stores of the
-//              entries with col <= row only (or raw partial tiles when M is split).
+//   warps 2-5: epilogue - tcgen05.ld of the accumulators, alpha/beta, and either
+//              swizzled shared-memory staging + asynchronous TMA stores (tiles below the
+//              diagonal, beta == 0) or masked direct stores of the entries with
+//              col <= row (diagonal tiles, beta != 0), or raw partial tiles when M is split.
+//
+// TMEM holds four 128-column slots.  The N = 256 accumulator pair of an item always
+// lives in slots 1-2; its N = 128 accumulator alternates between slot 0 and slot 3
+// from one item to the next.  The epilogue drains the pair first, so the next item's
+// MMAs start while the previous item's third tile is still being written out.
 //
 // Both MMA operands come from the same row-major A (K contiguous): segment x is the
 // M-operand, segment y (or the adjacent pair y, y+1) the N-operand, both K-major.
@@ -33,7 +40,10 @@ constexpr int kStageBytes = kSegSlots * kSegBytes;
 constexpr int kMaxTiles = 3;                      // 3 x 128 TMEM columns of 512
 constexpr int kTmemCols = 512;
 constexpr int kThreads = 192;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+constexpr int kStoreBox = 32;                      // rows and FP32 columns per TMA store
+constexpr int kStageBufBytes = kStoreBox * kStoreBox * 4;   // 4096
+constexpr int kStagingBytes = 4 * 2 * kStageBufBytes;        // 4 epilogue warps x 2 buffers
+constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024 + 256;
 
 // ---- tcgen05 wrappers -------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
@@ -88,6 +98,16 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(uint32_t n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// ---- bulk-async (TMA) store helpers ---------------------------------------------------
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, const void* smem_src, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(smem_src)) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 struct Unit {       // one work unit: an item and a range of K-steps
     int64_t item;
     int32_t slice;
@@ -102,18 +122,46 @@ __device__ __forceinline__ Unit unit_of(int64_t w, int64_t n_items, int32_t n_ks
     return u;
 }
 
+// Where an item's accumulators live.  Tiles t, t+1 with the same M-operand segment and
+// adjacent N-operand segments form one N = 256 MMA group in TMEM slots 1-2; a lone tile
+// is an N = 128 group in the single slot (0 or 3, alternating per item).  A valid item has
+// at most one group of each kind.
+struct Layout {
+    int n_grp;
+    int gx[2], gy[2], gn[2];
+    uint32_t gcol[2];
+    uint32_t tile_col[kMaxTiles];
+    bool tile_in_pair[kMaxTiles];
+};
+__device__ __forceinline__ void layout_of(const WorkItem* it, int n_tile, uint32_t single_col, Layout& L) {
+    L.n_grp = 0;
+    for (int t = 0; t < n_tile && L.n_grp < 2;) {
+        const int x = it->tile_x[t], y = it->tile_y[t];
+        const bool pair = (t + 1 < n_tile) && it->tile_x[t + 1] == x && it->tile_y[t + 1] == y + 1;
+        const int q = L.n_grp++;
+        L.gx[q] = x; L.gy[q] = y; L.gn[q] = pair ? 256 : 128;
+        L.gcol[q] = pair ? uint32_t(kTile) : single_col;
+        L.tile_col[t] = L.gcol[q]; L.tile_in_pair[t] = pair;
+        if (pair) { L.tile_col[t + 1] = L.gcol[q] + kTile; L.tile_in_pair[t + 1] = true; }
+        t += pair ? 2 : 1;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __restrict__ items,
-                     int64_t n_items, int64_t N, int32_t n_ksteps, float* __restrict__ C, int64_t ldc,
-                     float alpha, float beta, int vec_ok, int32_t split, float* __restrict__ partial,
-                     const int64_t* __restrict__ tile_base, int64_t total_tiles, int* __restrict__ status) {
+syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
+                     const WorkItem* __restrict__ items, int64_t n_items, int64_t N, int32_t n_ksteps,
+                     float* __restrict__ C, int64_t ldc, float alpha, float beta, int vec_ok, int tma_store_ok,
+                     int32_t split, float* __restrict__ partial, const int64_t* __restrict__ tile_base,
+                     int64_t total_tiles, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+    uint8_t* staging = smem + kStages * kStageBytes;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(staging + kStagingBytes);
     uint64_t* empty_bar = full_bar + kStages;
     uint64_t* tmem_full_bar = empty_bar + kStages;
-    uint64_t* tmem_empty_bar = tmem_full_bar + 1;
-    uint64_t* drain_bar = tmem_empty_bar + 1;
+    uint64_t* pair_free_bar = tmem_full_bar + 1;
+    uint64_t* single_free_bar = pair_free_bar + 1;     // [2]
+    uint64_t* drain_bar = single_free_bar + 2;
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
 
@@ -124,7 +172,9 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __
         s_abort = 0;
         for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         mbar_init(tmem_full_bar, 1);
-        mbar_init(tmem_empty_bar, 4);
+        mbar_init(pair_free_bar, 4);
+        mbar_init(&single_free_bar[0], 4);
+        mbar_init(&single_free_bar[1], 4);
         mbar_init(drain_bar, 1);
         mbar_fence_init();
     }
@@ -168,21 +218,25 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __
         if (lane == 0) {
             uint32_t g = 0, n_done = 0;
             const uint32_t smem_base = smem_u32(smem);
+            const uint64_t desc_hi = smem_desc_sw128(0);
             for (int64_t w = blockIdx.x; w < n_units && !s_abort; w += gridDim.x, ++n_done) {
                 const Unit u = unit_of(w, n_items, n_ksteps, split);
                 const WorkItem* it = &items[u.item];
-                const int n_tile = it->n_tile;
-                // MMA groups: tile t alone (N = 128), or tiles t, t+1 with the same M-operand
-                // and adjacent N-operand segments (N = 256).
-                int gx[kMaxTiles], gy[kMaxTiles], gn[kMaxTiles], gcol[kMaxTiles], n_grp = 0;
-                for (int t = 0; t < n_tile;) {
-                    const int x = it->tile_x[t], y = it->tile_y[t];
-                    const bool pair = (t + 1 < n_tile) && it->tile_x[t + 1] == x && it->tile_y[t + 1] == y + 1;
-                    gx[n_grp] = x; gy[n_grp] = y; gn[n_grp] = pair ? 256 : 128; gcol[n_grp] = t * kTile;
-                    ++n_grp;
-                    t += pair ? 2 : 1;
+                Layout L;
+                layout_of(it, it->n_tile, (n_done & 1) ? 3u * kTile : 0u, L);
+                uint32_t a_lo[2], b_lo[2], idesc[2], d_addr[2];
+                for (int q = 0; q < 2; ++q) {
+                    const int qq = q < L.n_grp ? q : 0;
+                    a_lo[q] = (smem_base + uint32_t(L.gx[qq]) * kSegBytes) >> 4;
+                    b_lo[q] = (smem_base + uint32_t(L.gy[qq]) * kSegBytes) >> 4;
+                    idesc[q] = instr_desc_bf16(uint32_t(L.gn[qq]));
+                    d_addr[q] = tmem_base + L.gcol[qq];
                 }
-                if (n_done > 0 && !mbar_wait_bounded(tmem_empty_bar, (n_done - 1) & 1, &s_abort)) {
+                // accumulators of this item must have been drained by the epilogue
+                if (n_done >= 1 && !mbar_wait_bounded(pair_free_bar, (n_done - 1) & 1, &s_abort)) {
+                    s_abort = 1; atomicOr(status, kStatusWaitTmem); break;
+                }
+                if (n_done >= 2 && !mbar_wait_bounded(&single_free_bar[n_done & 1], ((n_done >> 1) - 1) & 1, &s_abort)) {
                     s_abort = 1; atomicOr(status, kStatusWaitTmem); break;
                 }
                 tc_fence_after();
@@ -193,15 +247,14 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __
                         s_abort = 1; atomicOr(status, kStatusWaitFull); ok = false; break;
                     }
                     tc_fence_after();
-                    const uint32_t stage_addr = smem_base + st * kStageBytes;
-                    for (int q = 0; q < n_grp; ++q) {
-                        const uint32_t a_addr = stage_addr + gx[q] * kSegBytes;
-                        const uint32_t b_addr = stage_addr + gy[q] * kSegBytes;
-                        const uint32_t idesc = instr_desc_bf16(uint32_t(gn[q]));
+                    const uint32_t st_off = (st * kStageBytes) >> 4;
+                    const uint32_t first = (ks > u.k0) ? 1u : 0u;
+                    for (int q = 0; q < L.n_grp; ++q) {
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk)
-                            tc_mma_bf16(tmem_base + uint32_t(gcol[q]), smem_desc_sw128(a_addr + kk * 32),
-                                        smem_desc_sw128(b_addr + kk * 32), idesc, (ks > u.k0 || kk > 0) ? 1u : 0u);
+                            tc_mma_bf16(d_addr[q], desc_hi | uint64_t(a_lo[q] + st_off + 2 * kk),
+                                        desc_hi | uint64_t(b_lo[q] + st_off + 2 * kk), idesc[q],
+                                        (kk > 0) ? 1u : first);
                     }
                     tc_commit(&empty_bar[st]);    // stage reusable once these MMAs have read it
                 }
@@ -219,63 +272,95 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __
         // ------------------------------ epilogue ------------------------------
         const int quarter = warp & 3;                     // TMEM lanes this warp may read
         const int row_in_tile = quarter * 32 + lane;
-        uint32_t n_done = 0;
+        uint8_t* my_staging = staging + (warp - 2) * 2 * kStageBufBytes;
+        uint32_t n_done = 0, n_stores = 0;
         for (int64_t w = blockIdx.x; w < n_units && !s_abort; w += gridDim.x, ++n_done) {
             const Unit u = unit_of(w, n_items, n_ksteps, split);
             const WorkItem* it = &items[u.item];
             const int n_tile = it->n_tile;
+            Layout L;
+            layout_of(it, n_tile, (n_done & 1) ? 3u * kTile : 0u, L);
+            int64_t trow[kMaxTiles], tcol[kMaxTiles];
+            for (int t = 0; t < kMaxTiles; ++t) {
+                trow[t] = (t < n_tile) ? it->seg[it->tile_x[t]] : 0;
+                tcol[t] = (t < n_tile) ? it->seg[it->tile_y[t]] : 0;
+            }
+            const int64_t slot0 = (split > 1) ? tile_base[u.item] : 0;
             if (!mbar_wait_bounded(tmem_full_bar, n_done & 1, &s_abort)) {
                 s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitMma); break;
             }
             tc_fence_after();
-            for (int t = 0; t < n_tile; ++t) {
-                const int64_t trow = it->seg[it->tile_x[t]], tcol = it->seg[it->tile_y[t]];
-                const int64_t r = trow * kTile + row_in_tile;
-                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(t * kTile);
+            for (int pass = 0; pass < 2; ++pass) {        // the N = 256 pair first, then the lone tile
+                for (int t = 0; t < n_tile; ++t) {
+                    if (L.tile_in_pair[t] != (pass == 0)) continue;
+                    const int64_t r = trow[t] * kTile + row_in_tile;
+                    const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + L.tile_col[t];
+                    const bool staged = tma_store_ok && split == 1 && beta == 0.f && trow[t] != tcol[t] &&
+                                        trow[t] * kTile + quarter * 32 < N;
 #pragma unroll 1
-                for (int cb = 0; cb < kTile; cb += 32) {
-                    uint32_t v[32];
-                    tmem_ld_32x32(taddr + cb, v);
-                    if (split > 1) {
-                        float4* dst = reinterpret_cast<float4*>(
-                            partial + ((int64_t(u.slice) * total_tiles + tile_base[u.item] + t) * kTile + row_in_tile) * kTile + cb);
+                    for (int cb = 0; cb < kTile; cb += 32) {
+                        uint32_t v[32];
+                        tmem_ld_32x32(taddr + cb, v);
+                        if (split > 1) {
+                            float4* dst = reinterpret_cast<float4*>(
+                                partial + ((int64_t(u.slice) * total_tiles + slot0 + t) * kTile + row_in_tile) * kTile + cb);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                                 __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                        continue;
-                    }
-                    if (r >= N) continue;
-                    const int64_t c0 = tcol * kTile + cb;
-                    float* crow = C + r * ldc + c0;
-                    if (c0 + 31 <= r && vec_ok) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            float4 o = make_float4(alpha * __uint_as_float(v[4 * j]), alpha * __uint_as_float(v[4 * j + 1]),
-                                                   alpha * __uint_as_float(v[4 * j + 2]), alpha * __uint_as_float(v[4 * j + 3]));
-                            float4* p = reinterpret_cast<float4*>(crow) + j;
-                            if (beta != 0.f) {
-                                const float4 old = *p;
-                                o.x += beta * old.x; o.y += beta * old.y; o.z += beta * old.z; o.w += beta * old.w;
-                            }
-                            *p = o;
+                            for (int j = 0; j < 8; ++j)
+                                dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                            continue;
                         }
-                    } else {
+                        const int64_t c0 = tcol[t] * kTile + cb;
+                        if (staged) {
+                            // 32 x 32 block -> swizzled staging buffer -> asynchronous TMA store
+                            uint8_t* buf = my_staging + (n_stores & 1) * kStageBufBytes;
+                            if (lane == 0) tma_store_wait_read_1();   // the store that last used `buf` has read it
+                            __syncwarp();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (c0 + j <= r) {
-                                float o = alpha * __uint_as_float(v[j]);
-                                if (beta != 0.f) o += beta * crow[j];
-                                crow[j] = o;
+                            for (int j = 0; j < 8; ++j)
+                                *reinterpret_cast<float4*>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                                    make_float4(alpha * __uint_as_float(v[4 * j]), alpha * __uint_as_float(v[4 * j + 1]),
+                                                alpha * __uint_as_float(v[4 * j + 2]), alpha * __uint_as_float(v[4 * j + 3]));
+                            fence_async_smem();
+                            __syncwarp();
+                            if (lane == 0)
+                                tma_store_2d(&tmC, buf, int32_t(c0), int32_t(trow[t] * kTile + quarter * 32));
+                            ++n_stores;
+                            continue;
+                        }
+                        if (r >= N) continue;
+                        float* crow = C + r * ldc + c0;
+                        if (c0 + 31 <= r && vec_ok) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                float4 o = make_float4(alpha * __uint_as_float(v[4 * j]), alpha * __uint_as_float(v[4 * j + 1]),
+                                                       alpha * __uint_as_float(v[4 * j + 2]), alpha * __uint_as_float(v[4 * j + 3]));
+                                float4* p = reinterpret_cast<float4*>(crow) + j;
+                                if (beta != 0.f) {
+                                    const float4 old = *p;
+                                    o.x += beta * old.x; o.y += beta * old.y; o.z += beta * old.z; o.w += beta * old.w;
+                                }
+                                *p = o;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                if (c0 + j <= r) {
+                                    float o = alpha * __uint_as_float(v[j]);
+                                    if (beta != 0.f) o += beta * crow[j];
+                                    crow[j] = o;
+                                }
                             }
                         }
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pass == 0 ? pair_free_bar : &single_free_bar[n_done & 1]);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tmem_empty_bar);
         }
+        if (lane == 0) tma_store_wait_all();              // staged tiles are in global memory
+        __syncwarp();
     }
 
     tc_fence_before();
@@ -321,10 +406,10 @@ splitk_reduce_kernel(const WorkItem* __restrict__ items, const int64_t* __restri
 
 }  // namespace bf16
 
-cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items, int64_t N,
-                             int64_t M, float* C, int64_t ldc, float alpha, float beta, int split_k,
-                             float* d_partial, const int64_t* d_tile_base, int64_t total_tiles,
-                             int* d_status, int sm_count, cudaStream_t stream) {
+cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
+                             int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
+                             float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
+                             int64_t total_tiles, int* d_status, int sm_count, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(bf16::syrk_bf16_tbs_kernel,
@@ -338,9 +423,10 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const WorkItem* d_items, in
     const int64_t n_units = n_items * split;
     const unsigned grid = unsigned(n_units < sm_count ? n_units : sm_count);
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0) ? 1 : 0;
+    CUtensorMap none{};
     bf16::syrk_bf16_tbs_kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
-        tmA, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, split, d_partial, d_tile_base,
-        total_tiles, d_status);
+        tmA, tmC ? *tmC : none, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, split,
+        d_partial, d_tile_base, total_tiles, d_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || split == 1) return e;
     bf16::splitk_reduce_kernel<<<dim3(unsigned(n_items), bf16::kMaxTiles), 256, 0, stream>>>(
@@ -352,5 +438,6 @@ int bf16_tile() { return bf16::kTile; }
 int bf16_bk() { return bf16::kBK; }
 int bf16_stages() { return bf16::kStages; }
 int bf16_seg_slots() { return bf16::kSegSlots; }
+int bf16_store_box() { return bf16::kStoreBox; }
 
 }  // namespace tbsyrk
