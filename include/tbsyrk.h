@@ -43,6 +43,7 @@ extern "C" {
 #define SYRK_ERR_PLAN          -7  /* invalid schedule parameters                         */
 #define SYRK_ERR_DEVICE_WAIT   -8  /* a bounded wait inside a kernel ran out (see syrk_last_status) */
 #define SYRK_ERR_NO_DEVICE     -9  /* no CUDA device / not an sm_100 device               */
+#define SYRK_ERR_STATIC_LIMIT -10  /* syrk_lower_bf16_static: problem exceeds its fixed arrays */
 
 /* schedules (syrk_set_schedule) */
 #define SYRK_SCHEDULE_TBS     0    /* triangle blocks + square/diagonal leftovers (default) */
@@ -92,6 +93,41 @@ int syrk_lower_host(int64_t N, int64_t M,
                     const void* A, int64_t lda,
                     void* C, int64_t ldc,
                     double alpha, double beta, int dtype);
+
+/*
+ * Allocation-free variant of the K-split BF16 path (no counterpart in the paper; it
+ * exists for callers that cannot let a library call cudaMalloc: code that runs while
+ * another allocator owns the device heap, services whose device memory budget is fixed
+ * at start-up, loops where the implicit synchronisation of an allocation is not
+ * acceptable).
+ *
+ * Same operation, arguments and result as syrk_lower with dtype SYRK_DTYPE_BF16_F32,
+ * computed as `slices` >= 2 partial products over M that are summed in slice order.
+ * The work list, the partial tiles and the status word live in fixed device arrays
+ * inside the library image (about 34 MiB on every GPU that loads the library, held
+ * until the process exits) instead of cudaMalloc'ed memory; the call itself makes no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * Limits: at most 1024 work items and
+ *     slices * (number of 128 x 128 output tiles) <= SYRK_STATIC_MAX_SLICE_TILES
+ * (e.g. N = 2048: 136 tiles, up to 3 slices; N = 1024: 36 tiles, up to 14 slices).
+ * Larger problems are refused with SYRK_ERR_STATIC_LIMIT and nothing is enqueued.
+ * A must meet the TMA rules (16-byte aligned, lda * 2 a multiple of 16), else
+ * SYRK_ERR_LD; alpha == 0 or M == 0 have nothing to split and return SYRK_ERR_SIZE.
+ *
+ * The first call on a device also resolves the device addresses of those arrays
+ * (cudaGetSymbolAddress); make that first call outside any stream capture.
+ * Every call rewrites the shared arrays, so calls whose GPU work may overlap (other
+ * streams, other host threads) race: serialise them.  A bounded-wait failure inside
+ * this variant's kernels is recorded in its own status word and is not reported by
+ * syrk_last_status.
+ */
+#define SYRK_STATIC_MAX_SLICE_TILES 512
+int syrk_lower_bf16_static(int64_t N, int64_t M,
+                           const void* A, int64_t lda,
+                           void* C, int64_t ldc,
+                           double alpha, double beta,
+                           int slices, void* stream);
 
 /* Build and upload the work list for (N, M, dtype) ahead of time, so that a later
  * syrk_lower with these sizes allocates nothing. */

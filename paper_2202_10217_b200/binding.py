@@ -22,7 +22,7 @@ MAX_SEG, MAX_TILE = 8, 16
 EXPORTS = [
     "syrk_lower", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_get_schedule_stats",
-    "syrk_probe_f64_mma_peak",
+    "syrk_probe_f64_mma_peak", "syrk_lower_bf16_static",
     "tbs_plan_build", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
 ]
 
@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.syrk_get_schedule_stats.argtypes = [i64, i64, ci, ctypes.POINTER(ScheduleStats)]
         L.syrk_probe_f64_mma_peak.restype = ci
         L.syrk_probe_f64_mma_peak.argtypes = [ci, ctypes.POINTER(dbl)]
+        L.syrk_lower_bf16_static.restype = ci
+        L.syrk_lower_bf16_static.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
         L.tbs_plan_build.restype = vp
         L.tbs_plan_build.argtypes = [i64, ci, ci, ci, ci, ci]
         L.tbs_plan_num_items.restype = i64
@@ -134,6 +136,19 @@ def syrk_lower_host(N: int, M: int, A, lda: int, C, ldc: int, alpha: float, beta
     """Same operation on HOST buffers (numpy arrays, CPU tensors or raw addresses);
     copies in, computes on the GPU, copies the lower triangle back, and waits."""
     _check(lib().syrk_lower_host(N, M, _ptr(A), lda, _ptr(C), ldc, float(alpha), float(beta), dtype))
+
+
+def syrk_lower_bf16_static(N: int, M: int, A, lda: int, C, ldc: int, alpha: float, beta: float,
+                           slices: int, stream: Optional[int] = None) -> None:
+    """K-split BF16 update that allocates nothing: its work list and partial tiles live in
+    fixed device arrays of the library (for callers that cannot let a library call
+    cudaMalloc).  Raises SyrkError(-10) when the problem exceeds those arrays.  Calls share
+    the arrays, so overlapping calls must be serialised by the caller."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().syrk_lower_bf16_static(N, M, _ptr(A), lda, _ptr(C), ldc, float(alpha), float(beta),
+                                        int(slices), stream))
 
 
 def syrk_plan_prepare(N: int, M: int, dtype: int) -> None:

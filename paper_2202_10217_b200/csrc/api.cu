@@ -213,6 +213,7 @@ const char* syrk_strerror(int code) {
         case SYRK_ERR_PLAN: return "invalid schedule parameters";
         case SYRK_ERR_DEVICE_WAIT: return "a bounded wait inside a kernel ran out";
         case SYRK_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+        case SYRK_ERR_STATIC_LIMIT: return "problem too large for the fixed arrays of syrk_lower_bf16_static (work items or slices x tiles)";
         default: return "unknown error code";
     }
 }
