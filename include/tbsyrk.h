@@ -203,6 +203,10 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
 
 void*   tbs_plan_build(int64_t n_tiles, int k, int rect_rows, int rect_cols,
                        int diag_side, int schedule);
+/* Reorder a plan for a machine that runs `slots` items at a time (heaviest items first, some
+ * full rectangles at the end cut into quarters so that the last wave fills evenly); the set of
+ * tiles covered does not change.  The FP64 path applies this with slots = 148. */
+int     tbs_plan_balance(void* plan, int slots);
 int64_t tbs_plan_num_items(const void* plan);
 int     tbs_plan_item(const void* plan, int64_t index, int32_t* kind,
                       int32_t* n_seg, int32_t seg[TBS_MAX_SEG],

@@ -23,7 +23,7 @@ EXPORTS = [
     "syrk_lower", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_get_schedule_stats",
     "syrk_probe_f64_mma_peak", "syrk_lower_bf16_static",
-    "tbs_plan_build", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
+    "tbs_plan_build", "tbs_plan_balance", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
 ]
 
 
@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.syrk_lower_bf16_static.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
         L.tbs_plan_build.restype = vp
         L.tbs_plan_build.argtypes = [i64, ci, ci, ci, ci, ci]
+        L.tbs_plan_balance.restype = ci
+        L.tbs_plan_balance.argtypes = [vp, ci]
         L.tbs_plan_num_items.restype = i64
         L.tbs_plan_num_items.argtypes = [vp]
         L.tbs_plan_item.restype = ci
@@ -193,6 +195,9 @@ class Plan:
         if not self._h:
             raise SyrkError(-7)
         self.n_tiles = n_tiles
+
+    def balance(self, slots: int) -> None:
+        _check(lib().tbs_plan_balance(self._h, slots))
 
     def __len__(self) -> int:
         return int(lib().tbs_plan_num_items(self._h))

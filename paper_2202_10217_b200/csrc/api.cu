@@ -272,6 +272,13 @@ void* tbs_plan_build(int64_t n_tiles, int k, int rect_rows, int rect_cols, int d
     return plan;
 }
 
+int tbs_plan_balance(void* plan, int slots) {
+    if (!plan) return SYRK_ERR_NULL;
+    if (slots < 1) return SYRK_ERR_SIZE;
+    balance_for_slots(static_cast<Plan*>(plan), slots);
+    return SYRK_OK;
+}
+
 int64_t tbs_plan_num_items(const void* plan) {
     return plan ? int64_t(static_cast<const Plan*>(plan)->items.size()) : SYRK_ERR_NULL;
 }

@@ -42,7 +42,13 @@ bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out) {
     p.rect_cols = ks.rect_cols;
     p.diag_side = ks.diag_side;
     p.schedule = schedule;
-    return build_plan(p, out);
+    if (!build_plan(p, out)) return false;
+    // FP64: one thread block per item, dispatched in list order onto 148 SMs (B200); the BF16
+    // kernel is persistent and deals items round-robin, heaviest first.
+    if (dtype == SYRK_DTYPE_F64) balance_for_slots(out, 148);
+    else std::stable_sort(out->items.begin(), out->items.end(),
+                          [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
+    return true;
 }
 
 int get_device_state(DeviceState** out) {
@@ -74,11 +80,6 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
     if (it == ds->plans.end()) {
         DevicePlan dp;
         if (!build_host_plan(N, dtype, runtime().schedule, &dp.plan)) return SYRK_ERR_PLAN;
-        if (dtype == SYRK_DTYPE_BF16_F32) {
-            // The tcgen05 kernel's cost grows with the tiles an item owns: heaviest first.
-            std::stable_sort(dp.plan.items.begin(), dp.plan.items.end(),
-                             [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
-        }
         const int max_seg = (dtype == SYRK_DTYPE_F64) ? kMaxSeg : bf16_seg_slots();
         const int max_tile = (dtype == SYRK_DTYPE_F64) ? kMaxTile : 3;
         for (const WorkItem& it : dp.plan.items) {

@@ -10,7 +10,12 @@
 //                   16 columns of A per stage, into a 6-stage shared-memory ring
 //                   (128-byte swizzle), signalled through mbarriers;
 //   16 MMA warps  : warp w owns tile w: a 32 x 32 accumulator held in registers as
-//                   4 x 4 blocks of mma.sync m8n8k4 (FP64 tensor core, DMMA);
+//                   4 x 4 blocks of mma.sync m8n8k4 (FP64 tensor core, DMMA).  Each of the
+//                   SM's four schedulers has its own DMMA pipe, so an item lasts as long as
+//                   its busiest scheduler.  A triangle block has 15 tiles: its 15 warps then
+//                   leave out their last 8 x 8 block and the 16th warp owns those 15 blocks -
+//                   itself a triangle block over the last 8 rows of the six segments - so
+//                   that every warp issues 15 DMMAs per k-slice instead of 16, 16, 16, 12;
 //   epilogue      : alpha * acc (+ beta * C) written for entries with col <= row
 //                   only, two doubles per store where alignment allows.
 //
@@ -39,6 +44,38 @@ __device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
                  : "d"(a), "d"(b));
 }
 
+// The M loop of one warp's tile.  kSkipLast leaves out block (3, 3), which the 16th warp of
+// a triangle block computes.  Returns false when a bounded wait ran out.
+template <bool kSkipLast>
+__device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const uint8_t* smem, uint32_t xbase,
+                                              uint32_t ybase, const uint32_t (&off)[4], int n_ksteps,
+                                              uint64_t* full_bar, uint64_t* empty_bar, volatile int* abort_flag,
+                                              int lane) {
+    for (int ks = 0; ks < n_ksteps; ++ks) {
+        const int st = ks % kStages;
+        if (!mbar_wait_bounded(&full_bar[st], (ks / kStages) & 1, abort_flag)) return false;
+        const uint8_t* px = smem + st * kStageBytes + xbase;
+        const uint8_t* py = smem + st * kStageBytes + ybase;
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl) {
+            double a[4], b[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                a[j] = *reinterpret_cast<const double*>(px + off[sl] + j * 1024);
+                b[j] = *reinterpret_cast<const double*>(py + off[sl] + j * 1024);
+            }
+#pragma unroll
+            for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+                for (int ni = 0; ni < 4; ++ni)
+                    if (!(kSkipLast && mi == 3 && ni == 3)) dmma884(acc[mi][ni], a[mi], b[ni]);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[st]);
+    }
+    return true;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __restrict__ items,
                     int64_t N, int32_t n_ksteps, double* __restrict__ C, int64_t ldc,
@@ -49,6 +86,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
     uint64_t* empty_bar = full_bar + kStages;
     __shared__ WorkItem s_item;
     __shared__ volatile int s_abort;
+    __shared__ int s_scavenge;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -64,9 +102,17 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
             ok = s_item.seg[s] >= 0 && int64_t(s_item.seg[s]) * kTile < N;
         for (int t = 0; ok && t < n_tile; ++t)
             ok = s_item.tile_x[t] < n_seg && s_item.tile_y[t] < n_seg;
+        // A triangle block in the generator's tile order (x = 1..5, y < x): the 16th warp helps.
+        bool tri = ok && s_item.kind == kTri && n_seg == 6 && n_tile == 15;
+        for (int x = 1, t = 0; tri && x < 6; ++x)
+            for (int y = 0; y < x; ++y, ++t) tri = tri && s_item.tile_x[t] == x && s_item.tile_y[t] == y;
+        s_scavenge = tri ? 1 : 0;
         if (!ok) { s_abort = 1; atomicOr(status, kStatusBadItem); }
         else {
-            for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], n_tile); }
+            for (int s = 0; s < kStages; ++s) {
+                mbar_init(&full_bar[s], 1);
+                mbar_init(&empty_bar[s], tri ? kMmaWarps : n_tile);
+            }
             mbar_fence_init();
         }
     }
@@ -100,14 +146,64 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
         }
         return;
     }
-    if (warp >= n_tile) return;
+    const bool scavenge = s_scavenge != 0;
+    if (warp >= n_tile && !scavenge) return;
 
     // ------------------------------ MMA warps ------------------------------
+    // Fragment addressing.  Lane (g, t) of an m8n8k4 fragment holds (row g, k = t).  The four
+    // k-slices of a stage take k = 8*(t>>1) + 2*sl + (t&1): any assignment of the stage's 16
+    // columns to (slice, t) is valid as long as both operands use the same one, and this one
+    // makes every half-warp's 16 loads hit 16 different 8-byte bank pairs under the 128-byte
+    // swizzle (16-byte chunk index ^ row % 8).
     const int g = lane >> 2, t = lane & 3;
     uint32_t off[4];
 #pragma unroll
     for (int sl = 0; sl < 4; ++sl)
-        off[sl] = uint32_t(g * 128 + ((((sl << 1) | (t >> 1)) ^ g) << 4) + ((t & 1) << 3));
+        off[sl] = uint32_t(g * 128 + ((((t >> 1) << 2 | sl) ^ g) << 4) + ((t & 1) << 3));
+    const bool use_beta = (beta != 0.0);
+
+    if (scavenge && warp == kMmaWarps - 1) {
+        // ------------- 16th warp of a triangle block: the 15 left-out 8 x 8 blocks -------------
+        double sacc[15][2];
+#pragma unroll
+        for (int q = 0; q < 15; ++q) sacc[q][0] = sacc[q][1] = 0.0;
+        for (int ks = 0; ks < n_ksteps; ++ks) {
+            const int st = ks % kStages;
+            if (!mbar_wait_bounded(&full_bar[st], (ks / kStages) & 1, &s_abort)) {
+                s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return;
+            }
+            const uint8_t* base = smem + st * kStageBytes + 3 * 1024;      // rows 24..31 of every segment
+#pragma unroll
+            for (int sl = 0; sl < 4; ++sl) {
+                double f[6];
+#pragma unroll
+                for (int s = 0; s < 6; ++s) f[s] = *reinterpret_cast<const double*>(base + s * kSegBytes + off[sl]);
+                int q = 0;
+#pragma unroll
+                for (int x = 1; x < 6; ++x)
+#pragma unroll
+                    for (int y = 0; y < x; ++y, ++q) dmma884(sacc[q], f[x], f[y]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[st]);
+        }
+        int q = 0;
+#pragma unroll
+        for (int x = 1; x < 6; ++x)
+#pragma unroll
+            for (int y = 0; y < x; ++y, ++q) {
+                const int64_t r = int64_t(s_item.seg[x]) * kTile + 24 + g;
+                const int64_t c = int64_t(s_item.seg[y]) * kTile + 24 + 2 * t;
+                if (r >= N) continue;                                   // tile below the diagonal: c + 1 < r
+                double* p = C + r * ldc + c;
+                double v0 = alpha * sacc[q][0], v1 = alpha * sacc[q][1];
+                if (use_beta) { v0 += beta * p[0]; v1 += beta * p[1]; }
+                if (vec_ok) *reinterpret_cast<double2*>(p) = make_double2(v0, v1);
+                else { p[0] = v0; p[1] = v1; }
+            }
+        return;
+    }
+
     const int sx = s_item.tile_x[warp], sy = s_item.tile_y[warp];
     const uint32_t xbase = uint32_t(sx) * kSegBytes, ybase = uint32_t(sy) * kSegBytes;
 
@@ -117,35 +213,13 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
 #pragma unroll
         for (int ni = 0; ni < 4; ++ni) acc[mi][ni][0] = acc[mi][ni][1] = 0.0;
 
-    bool alive = true;
-    for (int ks = 0; ks < n_ksteps; ++ks) {
-        const int st = ks % kStages;
-        if (!mbar_wait_bounded(&full_bar[st], (ks / kStages) & 1, &s_abort)) {
-            s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); alive = false; break;
-        }
-        const uint8_t* px = smem + st * kStageBytes + xbase;
-        const uint8_t* py = smem + st * kStageBytes + ybase;
-#pragma unroll
-        for (int sl = 0; sl < 4; ++sl) {
-            double a[4], b[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                a[j] = *reinterpret_cast<const double*>(px + off[sl] + j * 1024);
-                b[j] = *reinterpret_cast<const double*>(py + off[sl] + j * 1024);
-            }
-#pragma unroll
-            for (int mi = 0; mi < 4; ++mi)
-#pragma unroll
-                for (int ni = 0; ni < 4; ++ni) dmma884(acc[mi][ni], a[mi], b[ni]);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[st]);
-    }
-    if (!alive) return;
+    const bool alive = scavenge
+        ? tile_mainloop<true>(acc, smem, xbase, ybase, off, n_ksteps, full_bar, empty_bar, &s_abort, lane)
+        : tile_mainloop<false>(acc, smem, xbase, ybase, off, n_ksteps, full_bar, empty_bar, &s_abort, lane);
+    if (!alive) { s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return; }
 
     // ------------------------------ epilogue ------------------------------
     const int64_t row0 = int64_t(s_item.seg[sx]) * kTile, col0 = int64_t(s_item.seg[sy]) * kTile;
-    const bool use_beta = (beta != 0.0);
 #pragma unroll
     for (int mi = 0; mi < 4; ++mi) {
         const int64_t r = row0 + mi * 8 + g;
@@ -153,6 +227,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
         double* crow = C + r * ldc;
 #pragma unroll
         for (int ni = 0; ni < 4; ++ni) {
+            if (scavenge && mi == 3 && ni == 3) continue;             // written by the 16th warp
             const int64_t c = col0 + ni * 8 + 2 * t;
             double v0 = alpha * acc[mi][ni][0], v1 = alpha * acc[mi][ni][1];
             if (c + 1 <= r) {

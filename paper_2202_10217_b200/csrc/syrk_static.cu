@@ -99,8 +99,6 @@ extern "C" int syrk_lower_bf16_static(int64_t N, int64_t M, const void* A, int64
     // Host-side work list (the same generator and ordering as the regular path).
     Plan plan;
     if (!build_host_plan(N, SYRK_DTYPE_BF16_F32, SYRK_SCHEDULE_TBS, &plan)) return SYRK_ERR_PLAN;
-    std::stable_sort(plan.items.begin(), plan.items.end(),
-                     [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
     const int64_t n_items = int64_t(plan.items.size());
     if (n_items > kStaticMaxItems) return SYRK_ERR_STATIC_LIMIT;
     std::vector<int64_t> base(size_t(n_items) + 1, 0);

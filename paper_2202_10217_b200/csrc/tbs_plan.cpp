@@ -161,6 +161,47 @@ bool build_plan(const PlanParams& p, Plan* out) {
     return true;
 }
 
+void balance_for_slots(Plan* plan, int slots) {
+    auto by_cost = [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; };
+    std::stable_sort(plan->items.begin(), plan->items.end(), by_cost);
+    const PlanParams& p = plan->p;
+    const int full = p.rect_rows * p.rect_cols;
+    if (slots <= 0 || p.rect_rows % 2 != 0 || p.rect_cols % 2 != 0 || full < 4) return;
+    int64_t total = 0;
+    for (const WorkItem& it : plan->items) total += it.n_tile;
+    if (total < int64_t(slots) * full) return;            // less than one wave: nothing to even out
+    const int64_t want = int64_t(slots) * full / 2;        // tiles to turn into small items
+    std::vector<WorkItem> out, small;
+    int64_t cut = 0;
+    for (auto it = plan->items.rbegin(); it != plan->items.rend(); ++it) {
+        if (cut < want && it->kind == kRect && it->n_tile == full) {
+            const int nc = p.rect_cols, nr = p.rect_rows;  // seg = [cols..., rows...]
+            for (int qr = 0; qr < 2; ++qr)
+                for (int qc = 0; qc < 2; ++qc) {
+                    WorkItem q{};
+                    q.kind = kRect;
+                    const int hc = nc / 2, hr = nr / 2;
+                    for (int y = 0; y < hc; ++y) q.seg[y] = it->seg[qc * hc + y];
+                    for (int x = 0; x < hr; ++x) q.seg[hc + x] = it->seg[nc + qr * hr + x];
+                    q.n_seg = hc + hr;
+                    int t = 0;
+                    for (int x = 0; x < hr; ++x)
+                        for (int y = 0; y < hc; ++y) { q.tile_x[t] = uint8_t(hc + x); q.tile_y[t] = uint8_t(y); ++t; }
+                    q.n_tile = t;
+                    small.push_back(q);
+                }
+            cut += full;
+            plan->n_rect += 3;
+        } else {
+            out.push_back(*it);
+        }
+    }
+    std::reverse(out.begin(), out.end());
+    out.insert(out.end(), small.begin(), small.end());
+    std::stable_sort(out.begin(), out.end(), by_cost);
+    plan->items.swap(out);
+}
+
 SimResult simulate_plan(const Plan& plan, int64_t N, int64_t M, int b) {
     SimResult r;
     const int64_t nt = plan.p.n_tiles;

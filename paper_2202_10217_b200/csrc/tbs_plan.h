@@ -48,6 +48,12 @@ int64_t pick_zone_side(int64_t n, int k);
 // Builds the item list; returns false on invalid parameters.
 bool build_plan(const PlanParams& p, Plan* out);
 
+// Ordering for a machine that runs `slots` items at a time, each item costing about its tile
+// count (ours; the paper's block loop is order-free): heaviest first, and enough full
+// rect_rows x rect_cols rectangles at the end cut into quarters to leave about half a wave of
+// small items that fill the last wave evenly.  Coverage is unchanged.
+void balance_for_slots(Plan* plan, int slots);
+
 // Two-level-model replay (Section 3): elements of A and C moved, tile coverage.
 struct SimResult {
     int64_t a_loads = 0, c_loads = 0;

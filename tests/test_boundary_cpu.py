@@ -47,6 +47,23 @@ def test_strerror_and_argument_validation_need_no_device():
         B.Plan(10, 9, 2, 2, 2)                                                # k(k-1)/2 tiles > 16
 
 
+def test_balancing_keeps_exact_once_coverage_and_puts_small_items_last():
+    for n_t, k, rr, rc in [(128, 6, 4, 4), (40, 6, 4, 4), (257, 6, 4, 4), (64, 3, 2, 2), (31, 4, 2, 4)]:
+        plan = B.Plan(n_t, k, rr, rc, rr)
+        before = len(plan)
+        plan.balance(148)
+        cover = np.zeros((n_t, n_t), dtype=np.int64)
+        sizes = []
+        for kind, seg, pairs in plan_ops(plan):
+            sizes.append(len(pairs))
+            assert len(set(seg)) == len(seg)
+            for (r, t) in pairs:
+                cover[r, t] += 1
+        assert np.array_equal(cover, np.tril(np.ones((n_t, n_t), dtype=np.int64)))
+        assert sizes == sorted(sizes, reverse=True) and len(plan) >= before
+        plan.close()
+
+
 def plan_ops(plan):
     """Library work list -> operations of the reference simulator."""
     ops = []
