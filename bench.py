@@ -145,6 +145,8 @@ def run_reference(args, wl: I.Workload, rank: int):
 # captures summarised under profiles/.  Valid only for the kernel source it was taken on.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, sha256 of the kernel source at capture time)
+    "c2_f64_4096x4096": (786_889_472, "c682423e7463c2af270ecf695a4e4cacf991ea8694e2352a6c3dcbca70e44220"),
+    "c3_bf16_16384x4096": (1_808_215_984, "a0c0b2d9ad91a1e0684e744e9ead0eb8b753a9131f407e699dc879ce4431e556"),
 }
 
 

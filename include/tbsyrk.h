@@ -168,7 +168,7 @@ typedef struct {
     int32_t tile;            /* b: rows per segment                                  */
     int32_t k;               /* segments per triangle block                          */
     int32_t c;               /* zone side of the top level (in tiles)                */
-    int32_t split_k;         /* K-slices                                             */
+    int32_t split_k;         /* K-slices a BF16 call would use on a 148-SM device    */
     int64_t n_tiles;         /* ceil(N / b)                                          */
     int64_t items;           /* work items                                           */
     int64_t tri_items;       /* of which triangle blocks                             */

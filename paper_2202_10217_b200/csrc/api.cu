@@ -27,19 +27,19 @@ bool tma_ok(const void* A, int64_t lda, int dtype) {
     return (reinterpret_cast<uintptr_t>(A) & 15) == 0 && (size_t(lda) * a_elem(dtype)) % 16 == 0;
 }
 
-int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk) {
-    const int forced = runtime().split_k;
+// K-slices for a BF16 call: few items and a long inner dimension are cut along M so that
+// every SM has work.
+int auto_split_k(int64_t items, int64_t M, int bk, int sm_count, int forced) {
     const int64_t ksteps = (M + bk - 1) / bk;
-    int s = 1;
+    int64_t s = 1;
     if (forced > 0) s = forced;
-    else {
-        // Few items and a long inner dimension: cut M so that every SM has work.
-        const int64_t items = int64_t(dp->plan.items.size());
-        if (items > 0 && items < ds->sm_count && ksteps >= 64)
-            s = int(std::min<int64_t>((2 * ds->sm_count + items - 1) / items, ksteps / 32));
-    }
-    s = int(std::max<int64_t>(1, std::min<int64_t>(s, ksteps)));
-    return s;
+    else if (items > 0 && items < sm_count && ksteps >= 64)
+        s = std::min<int64_t>((2 * int64_t(sm_count) + items - 1) / items, ksteps / 32);
+    return int(std::max<int64_t>(1, std::min<int64_t>(s, ksteps)));
+}
+
+int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk) {
+    return auto_split_k(int64_t(dp->plan.items.size()), M, bk, ds->sm_count, runtime().split_k);
 }
 
 int run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
@@ -236,8 +236,8 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     if (!out) return SYRK_ERR_NULL;
     if (dtype != SYRK_DTYPE_F64 && dtype != SYRK_DTYPE_BF16_F32) return SYRK_ERR_DTYPE;
     if (N < 0 || M < 0) return SYRK_ERR_SIZE;
-    int schedule;
-    { std::lock_guard<std::mutex> lock(runtime().mu); schedule = runtime().schedule; }
+    int schedule, forced_split;
+    { std::lock_guard<std::mutex> lock(runtime().mu); schedule = runtime().schedule; forced_split = runtime().split_k; }
     Plan plan;
     if (!build_host_plan(N, dtype, schedule, &plan)) return SYRK_ERR_PLAN;
     const KernelShape ks = kernel_shape(dtype);
@@ -246,7 +246,8 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->tile = ks.tile;
     out->k = ks.k;
     out->c = int32_t(plan.c_top);
-    out->split_k = 1;
+    out->split_k = (dtype == SYRK_DTYPE_BF16_F32 && M > 0)
+                       ? auto_split_k(int64_t(plan.items.size()), M, ks.bk, 148, forced_split) : 1;
     out->n_tiles = plan.p.n_tiles;
     out->items = int64_t(plan.items.size());
     out->tri_items = plan.n_tri;
