@@ -150,6 +150,21 @@ NCU_TRAFFIC = {
 }
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """Slowest rank's time (every rank gets it); the identity without a process group."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_replica: int, world: int, seconds: float) -> float:
+    """Replicas only: every rank does the same work, the job lasts as long as its slowest rank."""
+    return world * flops_per_replica / seconds * 1e-12
+
+
 def kernel_source_hash(dtype: int) -> str:
     import hashlib
     name = "syrk_f64.cu" if dtype == I.DTYPE_F64 else "syrk_bf16.cu"
@@ -206,12 +221,9 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
     assert B.syrk_last_status() == 0
     times = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
     total_ms = float(sum(times))
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * wl.flops / (ms_per_step * 1e-3) * 1e-12
+    value = whole_job_tflops(wl.flops, world, ms_per_step * 1e-3)
 
     if args.kernel_only:
         if rank == 0:
@@ -228,11 +240,8 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
     for _ in range(e2e_steps):
         B.syrk_lower_host(N, M, A_pinned, M, C_pinned, N, wl.alpha, wl.beta, dtype)
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e = {"value": world * wl.flops / e2e_s * 1e-12, "unit": UNIT,
+    e2e_s = max_over_ranks(e2e_s, dist, "cuda")
+    e2e = {"value": whole_job_tflops(wl.flops, world, e2e_s), "unit": UNIT,
            "h2d_bytes_per_step": N * M * ELEM_A[dtype] + (N * N * ELEM_C[dtype] if wl.beta != 0 else 0),
            "d2h_bytes_per_step": N * (N + 1) // 2 * ELEM_C[dtype]}
 

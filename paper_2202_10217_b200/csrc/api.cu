@@ -27,19 +27,40 @@ bool tma_ok(const void* A, int64_t lda, int dtype) {
     return (reinterpret_cast<uintptr_t>(A) & 15) == 0 && (size_t(lda) * a_elem(dtype)) % 16 == 0;
 }
 
-// K-slices for a BF16 call: few items and a long inner dimension are cut along M so that
-// every SM has work.
-int auto_split_k(int64_t items, int64_t M, int bk, int sm_count, int forced) {
+// K-slices for a BF16 call.  The persistent kernel deals its units (item x K-slice) round-robin
+// to min(units, SMs) thread blocks; with few items the inner dimension is cut so that every SM
+// has work.  The number of slices is the one with the smallest modelled makespan, in units of
+// one 128 x 128 x 64 tile step: a unit costs tiles x its K-steps plus about 20 per tile for the
+// write-out, and the reduction pass adds about 0.1 per partial tile.
+int auto_split_k(const std::vector<WorkItem>& items, int64_t M, int bk, int sm_count, int forced) {
     const int64_t ksteps = (M + bk - 1) / bk;
-    int64_t s = 1;
-    if (forced > 0) s = forced;
-    else if (items > 0 && items < sm_count && ksteps >= 64)
-        s = std::min<int64_t>((2 * int64_t(sm_count) + items - 1) / items, ksteps / 32);
-    return int(std::max<int64_t>(1, std::min<int64_t>(s, ksteps)));
+    if (forced > 0) return int(std::max<int64_t>(1, std::min<int64_t>(forced, ksteps)));
+    const int64_t n = int64_t(items.size());
+    if (n == 0 || n >= 4 * int64_t(sm_count) || ksteps < 16) return 1;
+    int64_t total_tiles = 0;
+    for (const WorkItem& it : items) total_tiles += it.n_tile;
+    int best = 1;
+    double best_cost = 0.0;
+    std::vector<double> load;
+    for (int s = 1; s <= 32 && s <= ksteps / 8; ++s) {
+        const int64_t units = n * s;
+        const int64_t grid = std::min<int64_t>(units, sm_count);
+        load.assign(size_t(grid), 0.0);
+        for (int64_t w = 0; w < units; ++w) {
+            const WorkItem& it = items[size_t(w % n)];
+            const int64_t slice = w / n;
+            const int64_t kk = ksteps * (slice + 1) / s - ksteps * slice / s;
+            load[size_t(w % grid)] += double(it.n_tile) * double(kk + 20);
+        }
+        double cost = *std::max_element(load.begin(), load.end());
+        if (s > 1) cost += 0.1 * double(s) * double(total_tiles) + 40.0;
+        if (s == 1 || cost < best_cost) { best = s; best_cost = cost; }
+    }
+    return best;
 }
 
 int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk) {
-    return auto_split_k(int64_t(dp->plan.items.size()), M, bk, ds->sm_count, runtime().split_k);
+    return auto_split_k(dp->plan.items, M, bk, ds->sm_count, runtime().split_k);
 }
 
 int run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
@@ -247,7 +268,7 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->k = ks.k;
     out->c = int32_t(plan.c_top);
     out->split_k = (dtype == SYRK_DTYPE_BF16_F32 && M > 0)
-                       ? auto_split_k(int64_t(plan.items.size()), M, ks.bk, 148, forced_split) : 1;
+                       ? auto_split_k(plan.items, M, ks.bk, 148, forced_split) : 1;
     out->n_tiles = plan.p.n_tiles;
     out->items = int64_t(plan.items.size());
     out->tri_items = plan.n_tri;
