@@ -85,8 +85,11 @@ int run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_
     const int64_t n_items = int64_t(dp->plan.items.size());
     cudaError_t e;
     if (dtype == SYRK_DTYPE_F64) {
-        e = launch_syrk_f64(tm, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha, beta,
-                            ds->d_status, stream);
+        CUtensorMap tmc;
+        const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
+                           encode_tensor_map_c_f64(&tmc, C, N, ldc, f64_tile()) == SYRK_OK;
+        e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc,
+                            alpha, beta, ds->d_status, stream);
     } else {
         const int split = pick_split_k(ds, dp, M, ks.bk);
         if (split > 1) {

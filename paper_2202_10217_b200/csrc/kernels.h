@@ -9,8 +9,10 @@
 namespace tbsyrk {
 
 // FP64 triangle-block kernel: one thread block per work item.
-cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items,
-                            int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
+// `tmC` (may be null): tensor map over C with 32 x 32 FP64 boxes, no swizzle, through which the
+// old C tiles are fetched when beta != 0.
+cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
+                            int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int* d_status, cudaStream_t stream);
 int f64_tile();
 int f64_bk();

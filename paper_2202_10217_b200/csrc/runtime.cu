@@ -170,6 +170,19 @@ int encode_tensor_map_c_f32(CUtensorMap* tm, const void* C, int64_t N, int64_t l
     return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
+int encode_tensor_map_c_f64(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SYRK_ERR_CUDA;
+    const cuuint64_t dims[2] = {cuuint64_t(N), cuuint64_t(N)};
+    const cuuint64_t strides[1] = {cuuint64_t(ldc) * 8};
+    const cuuint32_t bx[2] = {cuuint32_t(box), cuuint32_t(box)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, 2, const_cast<void*>(C), dims, strides, bx, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
 int ensure_device_bytes(void** p, size_t* have, size_t want) {
     if (*have >= want && *p) return SYRK_OK;
     if (*p) { cudaFree(*p); *p = nullptr; *have = 0; }

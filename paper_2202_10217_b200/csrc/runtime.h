@@ -70,6 +70,8 @@ int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, i
 
 // 2-D row-major FP32 tensor map over C (N x N, pitch ldc) with box x box boxes, 128-byte swizzle.
 int encode_tensor_map_c_f32(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box);
+// The same over an FP64 C, without swizzle (a box row of 32 doubles is 256 bytes).
+int encode_tensor_map_c_f64(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box);
 
 // Grow-only device / pinned-host buffers.
 int ensure_device_bytes(void** p, size_t* have, size_t want);

@@ -17,7 +17,10 @@
 //                   itself a triangle block over the last 8 rows of the six segments - so
 //                   that every warp issues 15 DMMAs per k-slice instead of 16, 16, 16, 12;
 //   epilogue      : alpha * acc (+ beta * C) written for entries with col <= row
-//                   only, two doubles per store where alignment allows.
+//                   only, two doubles per store where alignment allows.  With beta != 0
+//                   the producer also TMA-loads the item's old C tiles (those below the
+//                   diagonal) into the ring's stages as the last K-steps release them, so
+//                   the epilogue reads them from shared memory instead of waiting on HBM.
 //
 // Accumulators (the C block) stay on chip for the whole M loop and each entry of
 // C is read (beta != 0) and written exactly once, as in the paper's generic
@@ -36,6 +39,7 @@ constexpr int kSegBytes = kTile * kBK * 8;      // 4096
 constexpr int kStageBytes = kMaxSeg * kSegBytes;
 constexpr int kMmaWarps = 16;
 constexpr int kThreads = (kMmaWarps + 1) * 32;  // + producer warp
+constexpr int kCTileBytes = kTile * kTile * 8;   // one old C tile in a ring stage (4 per stage)
 constexpr int kSmemBytes = kStages * kStageBytes + 2 * kStages * 8 + 1024;
 
 __device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
@@ -77,9 +81,10 @@ __device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const uint
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __restrict__ items,
-                    int64_t N, int32_t n_ksteps, double* __restrict__ C, int64_t ldc,
-                    double alpha, double beta, int vec_ok, int* __restrict__ status) {
+syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
+                    const WorkItem* __restrict__ items, int64_t N, int32_t n_ksteps,
+                    double* __restrict__ C, int64_t ldc, double alpha, double beta, int vec_ok,
+                    int c_tma, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
@@ -136,6 +141,27 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
                     tma_load_2d(dst + s * kSegBytes, &tmA, ks * kBK, s_item.seg[s] * kTile, &full_bar[st]);
                 issued = ks + 1;
             }
+            if (c_tma && !s_abort) {
+                // Old C: ring step n_ksteps + j carries tiles 4j .. 4j+3 (8 KB each, row pitch 256 B).
+                prefetch_tensormap(&tmC);
+                for (int j = 0; 4 * j < n_tile; ++j) {
+                    const int q = n_ksteps + j, st = q % kStages;
+                    if (q >= kStages && !mbar_wait_bounded(&empty_bar[st], ((q / kStages) - 1) & 1, &s_abort)) {
+                        s_abort = 1; atomicOr(status, kStatusWaitEmpty); break;
+                    }
+                    int below = 0;
+                    for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt)
+                        below += (s_item.seg[s_item.tile_x[tt]] != s_item.seg[s_item.tile_y[tt]]) ? 1 : 0;
+                    if (below == 0) { mbar_arrive(&full_bar[st]); continue; }
+                    mbar_arrive_expect_tx(&full_bar[st], uint32_t(below) * kCTileBytes);
+                    uint8_t* dst = smem + st * kStageBytes;
+                    for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt) {
+                        const int rx = s_item.seg[s_item.tile_x[tt]], cy = s_item.seg[s_item.tile_y[tt]];
+                        if (rx != cy) tma_load_2d(dst + (tt & 3) * kCTileBytes, &tmC, cy * kTile, rx * kTile, &full_bar[st]);
+                    }
+                    issued = q + 1;
+                }
+            }
             if (s_abort) {
                 // Winding down: let the copies still in flight land before the block exits.
                 for (int ks = (issued > kStages ? issued - kStages : 0); ks < issued; ++ks) {
@@ -187,6 +213,14 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);
         }
+        if (c_tma) {                                                    // all four old-C ring steps
+            for (int j = 0; j < 4; ++j) {
+                const int qs = n_ksteps + j;
+                if (!mbar_wait_bounded(&full_bar[qs % kStages], (qs / kStages) & 1, &s_abort)) {
+                    s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return;
+                }
+            }
+        }
         int q = 0;
 #pragma unroll
         for (int x = 1; x < 6; ++x)
@@ -197,7 +231,12 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
                 if (r >= N) continue;                                   // tile below the diagonal: c + 1 < r
                 double* p = C + r * ldc + c;
                 double v0 = alpha * sacc[q][0], v1 = alpha * sacc[q][1];
-                if (use_beta) { v0 += beta * p[0]; v1 += beta * p[1]; }
+                if (c_tma) {
+                    const double2 o = *reinterpret_cast<const double2*>(
+                        smem + ((n_ksteps + (q >> 2)) % kStages) * kStageBytes + (q & 3) * kCTileBytes +
+                        (24 + g) * (kTile * 8) + (24 + 2 * t) * 8);
+                    v0 += beta * o.x; v1 += beta * o.y;
+                } else if (use_beta) { v0 += beta * p[0]; v1 += beta * p[1]; }
                 if (vec_ok) *reinterpret_cast<double2*>(p) = make_double2(v0, v1);
                 else { p[0] = v0; p[1] = v1; }
             }
@@ -220,6 +259,14 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
 
     // ------------------------------ epilogue ------------------------------
     const int64_t row0 = int64_t(s_item.seg[sx]) * kTile, col0 = int64_t(s_item.seg[sy]) * kTile;
+    const uint8_t* old_tile = nullptr;                  // this warp's old C tile in shared memory
+    if (c_tma && row0 != col0) {
+        const int qs = n_ksteps + (warp >> 2);
+        if (!mbar_wait_bounded(&full_bar[qs % kStages], (qs / kStages) & 1, &s_abort)) {
+            s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return;
+        }
+        old_tile = smem + (qs % kStages) * kStageBytes + (warp & 3) * kCTileBytes;
+    }
 #pragma unroll
     for (int mi = 0; mi < 4; ++mi) {
         const int64_t r = row0 + mi * 8 + g;
@@ -230,7 +277,10 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
             if (scavenge && mi == 3 && ni == 3) continue;             // written by the 16th warp
             const int64_t c = col0 + ni * 8 + 2 * t;
             double v0 = alpha * acc[mi][ni][0], v1 = alpha * acc[mi][ni][1];
-            if (c + 1 <= r) {
+            if (old_tile) {                                           // tile below the diagonal, vec_ok holds
+                const double2 o = *reinterpret_cast<const double2*>(old_tile + (mi * 8 + g) * (kTile * 8) + (ni * 8 + 2 * t) * 8);
+                *reinterpret_cast<double2*>(crow + c) = make_double2(v0 + beta * o.x, v1 + beta * o.y);
+            } else if (c + 1 <= r) {
                 if (vec_ok) {
                     double2* p = reinterpret_cast<double2*>(crow + c);
                     if (use_beta) { const double2 o = *p; v0 += beta * o.x; v1 += beta * o.y; }
@@ -249,8 +299,8 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __r
 
 }  // namespace f64
 
-cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items,
-                            int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
+cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
+                            int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int* d_status, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
@@ -262,8 +312,10 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int
     if (n_items == 0) return cudaSuccess;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0) ? 1 : 0;
     const int32_t n_ksteps = int32_t((M + f64::kBK - 1) / f64::kBK);
+    const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
+    CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
-        tmA, d_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, d_status);
+        tmA, c_tma ? *tmC : none, d_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
     return cudaGetLastError();
 }
 
