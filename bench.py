@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the triangle-block SYRK library on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c1]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c1|c5]
                     [--impl ours|reference]
 
 A step is one SYRK call (the whole hot path: work-list lookup, TMA streaming, tensor-core
@@ -286,12 +286,113 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
         dist.destroy_process_group()
 
 
+def run_sweep(args, rank: int, world: int, local_rank: int):
+    """Config 5: C_n <- C_n - A_n A_n^T on the trailing n x n view of one 32768^2 FP64 matrix,
+    n = 32768, 32256, ..., 512 (64 calls, M = 512, ldc = 32768).  One step = the whole sweep."""
+    import torch
+    from paper_2202_10217_b200 import binding as B
+
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    n_max, step, M = 32768, 512, I.SWEEP_K
+    sizes = I.sweep_sizes(n_max, step)
+    flops = sum(n * (n + 1) * M for n in sizes)
+    # A_n = the trailing n rows of one seeded n_max x 512 panel (same shapes, pitches and value
+    # distribution as a fresh panel per step); C = n_max * I + G G^T / 512 prepared with torch.
+    A_pinned = torch.from_numpy(I.sweep_panel(n_max, n_max)).pin_memory()
+    dA = A_pinned.cuda()
+    G = torch.from_numpy(I.sweep_factor(n_max)).cuda()
+    C = torch.matmul(G, G.T) / float(M)
+    C.diagonal().add_(float(n_max))
+    del G
+    diag_host = torch.empty(n_max, dtype=torch.float64).pin_memory()
+    for n in sizes:
+        B.syrk_plan_prepare(n, M, I.DTYPE_F64)
+
+    def sweep(src):
+        for n in sizes:
+            off = n_max - n
+            B.syrk_lower(n, M, src.data_ptr() + off * M * 8, M, C.data_ptr() + (off * n_max + off) * 8, n_max,
+                         -1.0, 1.0, I.DTYPE_F64)
+
+    steps = max(1, min(args.steps, 10))
+    for _ in range(1 if args.kernel_only else 3):
+        sweep(dA)
+    torch.cuda.synchronize()
+    assert B.syrk_last_status() == 0
+    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        for i in range(steps):
+            ev0[i].record()
+            sweep(dA)
+            ev1[i].record()
+        barrier()
+    assert B.syrk_last_status() == 0
+    times = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
+    ms_per_step = max_over_ranks(float(sum(times)), dist, "cuda") / steps
+    value = whole_job_tflops(flops, world, ms_per_step * 1e-3)
+    if args.kernel_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+                              "ms_per_step": ms_per_step, "kernel_only": True,
+                              "config": {"workload": "c5_f64_sweep_32768..512_x512"}}))
+        return
+    # end to end: every panel copied from pinned host memory before its call, the diagonal read back
+    dA2 = torch.empty_like(dA)
+    barrier()
+    t0 = time.perf_counter()
+    for n in sizes:
+        off = n_max - n
+        dA2[off:].copy_(A_pinned[off:], non_blocking=True)
+        B.syrk_lower(n, M, dA2.data_ptr() + off * M * 8, M, C.data_ptr() + (off * n_max + off) * 8, n_max,
+                     -1.0, 1.0, I.DTYPE_F64)
+    diag_host.copy_(C.diagonal(), non_blocking=True)
+    torch.cuda.synchronize()
+    e2e_s = max_over_ranks(time.perf_counter() - t0, dist, "cuda")
+    if rank != 0:
+        return
+    peak = B.syrk_probe_f64_mma_peak(20000)
+    achieved = flops / (float(np.mean(times)) * 1e-3) * 1e-12
+    small = I.Workload("c5_step_n4096", 4096, M, I.DTYPE_F64, -1.0, 1.0, I.SWEEP_SEED, "normal", std=M ** -0.5)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": 3,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "c5_f64_sweep_32768..512_x512", "calls_per_step": len(sizes), "M": M, "alpha": -1.0,
+                   "beta": 1.0, "ldc": n_max, "schedule": "tbs",
+                   "l2": "inputs larger than L2 (C view 8.6 GB .. 2 MB, read and written once per call)"},
+        "clocks": clocks.summary(),
+        "e2e": {"value": whole_job_tflops(flops, world, e2e_s), "unit": UNIT,
+                "h2d_bytes_per_step": sum(n * M * 8 for n in sizes), "d2h_bytes_per_step": n_max * 8},
+        "gpu_launches": steps * len(sizes),
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": UNIT, "frac": achieved / peak,
+                     "traffic": None, "peak_source": "FP64 DMMA rate measured in this run by the library's probe",
+                     "algorithmic_flops_per_launch": flops / len(sizes)},
+    }
+    if world == 1:
+        line["cpu_baseline"] = cpu_reference_sample(small, small.make_A())
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c2", choices=sorted(I.CONFIGS))
+    ap.add_argument("--workload", default="c2", choices=sorted(I.CONFIGS) + ["c5"])
     ap.add_argument("--shape", default=None,
                     help="N,M,dtype,alpha,beta (dtype f64|bf16): a custom seeded N(0,1) workload")
     ap.add_argument("--kernel-only", action="store_true",
@@ -302,6 +403,12 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.workload == "c5" and not args.shape:
+        if args.impl == "reference":
+            args.workload = "c2"                     # the oracle arm samples a single FP64 call
+        else:
+            run_sweep(args, rank, world, local_rank)
+            return
     wl = I.CONFIGS[args.workload]
     if args.shape:
         n, m, dt, al, be = args.shape.split(",")
