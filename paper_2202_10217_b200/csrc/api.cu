@@ -103,7 +103,7 @@ int run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_
         const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                            encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
         e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
-                             float(beta), split, ds->d_partial, dp->d_tile_base, dp->total_tiles, ds->d_status,
+                             float(beta), split, ds->d_partial, dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, ds->d_status,
                              ds->sm_count, stream);
     }
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;

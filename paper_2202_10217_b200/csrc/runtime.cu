@@ -95,6 +95,43 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
                 if (lone > 1 || pairs > 1) return SYRK_ERR_PLAN;
             }
         }
+        std::vector<int64_t> cta_begin;
+        if (dtype == SYRK_DTYPE_BF16_F32 && !dp.plan.items.empty()) {
+            // Persistent kernel: items go to thread blocks (one per SM) longest first, each to the
+            // block with the least work so far.  The kernel is bound by shared-memory traffic, so
+            // an item costs, per K-step, 16 KB per segment written by TMA plus the operand reads of
+            // its MMAs (16 KB for the M-operand and 16 KB per 128 columns of N), and about 600 KB
+            // worth of time per tile for the write-out.  K-steps are not known here; 64 (M = 4096)
+            // weighs the two terms.
+            const int n_ctas = int(std::min<size_t>(dp.plan.items.size(), size_t(ds->sm_count)));
+            auto cost = [](const WorkItem& it) {
+                int64_t kb = 16 * it.n_seg;
+                for (int t = 0; t < it.n_tile;) {
+                    const bool pair = t + 1 < it.n_tile && it.tile_x[t + 1] == it.tile_x[t] &&
+                                      it.tile_y[t + 1] == it.tile_y[t] + 1;
+                    kb += pair ? 48 : 32;
+                    t += pair ? 2 : 1;
+                }
+                return 64 * kb + 600 * int64_t(it.n_tile);
+            };
+            std::vector<WorkItem> sorted = dp.plan.items;
+            std::stable_sort(sorted.begin(), sorted.end(),
+                             [&](const WorkItem& a, const WorkItem& b) { return cost(a) > cost(b); });
+            std::vector<std::vector<WorkItem>> per_block(static_cast<size_t>(n_ctas));
+            std::vector<int64_t> load(size_t(n_ctas), 0);
+            for (const WorkItem& it : sorted) {
+                const size_t b = size_t(std::min_element(load.begin(), load.end()) - load.begin());
+                per_block[b].push_back(it);
+                load[b] += cost(it);
+            }
+            dp.plan.items.clear();
+            cta_begin.push_back(0);
+            for (int b = 0; b < n_ctas; ++b) {
+                dp.plan.items.insert(dp.plan.items.end(), per_block[size_t(b)].begin(), per_block[size_t(b)].end());
+                cta_begin.push_back(int64_t(dp.plan.items.size()));
+            }
+            dp.n_ctas = n_ctas;
+        }
         const size_t n = dp.plan.items.size();
         std::vector<int64_t> base(n + 1, 0);
         for (size_t i = 0; i < n; ++i) base[i + 1] = base[i] + dp.plan.items[i].n_tile;
@@ -111,6 +148,14 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
                 cudaGetLastError();
                 cudaFree(dp.d_items); cudaFree(dp.d_tile_base);
                 return SYRK_ERR_CUDA;
+            }
+        }
+        if (!cta_begin.empty()) {
+            if (cudaMalloc(&dp.d_cta_begin, cta_begin.size() * sizeof(int64_t)) != cudaSuccess) {
+                cudaGetLastError(); cudaFree(dp.d_items); cudaFree(dp.d_tile_base); return SYRK_ERR_ALLOC;
+            }
+            if (cudaMemcpy(dp.d_cta_begin, cta_begin.data(), cta_begin.size() * sizeof(int64_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+                cudaGetLastError(); cudaFree(dp.d_items); cudaFree(dp.d_tile_base); cudaFree(dp.d_cta_begin); return SYRK_ERR_CUDA;
             }
         }
         it = ds->plans.emplace(key, std::move(dp)).first;
@@ -209,6 +254,7 @@ void release_all() {
         for (auto& pk : ds.plans) {
             if (pk.second.d_items) cudaFree(pk.second.d_items);
             if (pk.second.d_tile_base) cudaFree(pk.second.d_tile_base);
+            if (pk.second.d_cta_begin) cudaFree(pk.second.d_cta_begin);
         }
         if (ds.d_status) cudaFree(ds.d_status);
         if (ds.d_partial) cudaFree(ds.d_partial);

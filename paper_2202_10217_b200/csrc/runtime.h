@@ -28,6 +28,8 @@ struct DevicePlan {
     WorkItem* d_items = nullptr;
     int64_t* d_tile_base = nullptr;  // first output-tile slot of each item (K-split workspace)
     int64_t total_tiles = 0;
+    int64_t* d_cta_begin = nullptr;  // BF16: first item of each persistent thread block (n_ctas + 1)
+    int n_ctas = 0;
 };
 
 struct DeviceState {

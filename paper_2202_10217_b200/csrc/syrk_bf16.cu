@@ -152,7 +152,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                      const WorkItem* __restrict__ items, int64_t n_items, int64_t N, int32_t n_ksteps,
                      float* __restrict__ C, int64_t ldc, float alpha, float beta, int vec_ok, int tma_store_ok,
                      int32_t split, float* __restrict__ partial, const int64_t* __restrict__ tile_base,
-                     int64_t total_tiles, int* __restrict__ status) {
+                     int64_t total_tiles, const int64_t* __restrict__ cta_begin, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* staging = smem + kStages * kStageBytes;
@@ -167,6 +167,11 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t n_units = n_items * split;
+    // This block's units: its own contiguous range of a list ordered block by block on the host,
+    // or (K-split calls) every gridDim.x-th unit of the slice-major list.
+    const int64_t w_first = cta_begin ? cta_begin[blockIdx.x] : int64_t(blockIdx.x);
+    const int64_t w_last = cta_begin ? cta_begin[blockIdx.x + 1] : n_units;
+    const int64_t w_stride = cta_begin ? 1 : int64_t(gridDim.x);
 
     if (tid == 0) {
         s_abort = 0;
@@ -189,7 +194,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if (lane == 0) {
             prefetch_tensormap(&tmA);
             uint32_t g = 0;
-            for (int64_t w = blockIdx.x; w < n_units && !s_abort; w += gridDim.x) {
+            for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride) {
                 const Unit u = unit_of(w, n_items, n_ksteps, split);
                 const WorkItem* it = &items[u.item];
                 const int n_seg = it->n_seg;
@@ -219,7 +224,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             uint32_t g = 0, n_done = 0;
             const uint32_t smem_base = smem_u32(smem);
             const uint64_t desc_hi = smem_desc_sw128(0);
-            for (int64_t w = blockIdx.x; w < n_units && !s_abort; w += gridDim.x, ++n_done) {
+            for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride, ++n_done) {
                 const Unit u = unit_of(w, n_items, n_ksteps, split);
                 const WorkItem* it = &items[u.item];
                 Layout L;
@@ -274,7 +279,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const int row_in_tile = quarter * 32 + lane;
         uint8_t* my_staging = staging + (warp - 2) * 2 * kStageBufBytes;
         uint32_t n_done = 0, n_stores = 0;
-        for (int64_t w = blockIdx.x; w < n_units && !s_abort; w += gridDim.x, ++n_done) {
+        for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride, ++n_done) {
             const Unit u = unit_of(w, n_items, n_ksteps, split);
             const WorkItem* it = &items[u.item];
             const int n_tile = it->n_tile;
@@ -409,7 +414,8 @@ splitk_reduce_kernel(const WorkItem* __restrict__ items, const int64_t* __restri
 cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                              int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
-                             int64_t total_tiles, int* d_status, int sm_count, cudaStream_t stream) {
+                             int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int* d_status,
+                             int sm_count, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(bf16::syrk_bf16_tbs_kernel,
@@ -421,12 +427,13 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     const int32_t n_ksteps = int32_t((M + bf16::kBK - 1) / bf16::kBK);
     const int split = split_k < 1 ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
     const int64_t n_units = n_items * split;
-    const unsigned grid = unsigned(n_units < sm_count ? n_units : sm_count);
+    const bool ranges = (d_cta_begin != nullptr && split == 1 && n_ctas > 0);
+    const unsigned grid = ranges ? unsigned(n_ctas) : unsigned(n_units < sm_count ? n_units : sm_count);
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0) ? 1 : 0;
     CUtensorMap none{};
     bf16::syrk_bf16_tbs_kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
         tmA, tmC ? *tmC : none, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, split,
-        d_partial, d_tile_base, total_tiles, d_status);
+        d_partial, d_tile_base, total_tiles, ranges ? d_cta_begin : nullptr, d_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || split == 1) return e;
     bf16::splitk_reduce_kernel<<<dim3(unsigned(n_items), bf16::kMaxTiles), 256, 0, stream>>>(
