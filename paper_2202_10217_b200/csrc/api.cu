@@ -1,6 +1,8 @@
 // C ABI of libtbsyrk.so (see include/tbsyrk.h for the contract of every call).
 #include <algorithm>
+#include <cmath>
 #include <cstring>
+#include <thread>
 #include <vector>
 
 #include "../../include/tbsyrk.h"
@@ -172,11 +174,26 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     ok = ok && cudaMemcpyAsync(ds->h_packed, ds->d_packed, packed_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return SYRK_ERR_CUDA; }
-    const char* src = static_cast<const char*>(ds->h_packed);
-    char* dst = static_cast<char*>(C);
-    for (int64_t i = 0; i < N; ++i) {
-        std::memcpy(dst + size_t(i) * ldc * ec, src, size_t(i + 1) * ec);
-        src += size_t(i + 1) * ec;
+    // Packed rows -> the caller's lower triangle, on a few host threads with equal byte shares
+    // (row i starts at element i(i+1)/2, so thread t gets rows up to N * sqrt((t+1)/T)).
+    {
+        const char* src = static_cast<const char*>(ds->h_packed);
+        char* dst = static_cast<char*>(C);
+        const unsigned hw = std::thread::hardware_concurrency();
+        const int T = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(hw ? hw : 1), int64_t(8), N / 256})));
+        auto rows = [=](int64_t r0, int64_t r1) {
+            for (int64_t i = r0; i < r1; ++i)
+                std::memcpy(dst + size_t(i) * ldc * ec, src + size_t(i) * size_t(i + 1) / 2 * ec, size_t(i + 1) * ec);
+        };
+        std::vector<std::thread> pool;
+        int64_t r0 = 0;
+        for (int t = 0; t < T; ++t) {
+            const int64_t r1 = (t == T - 1) ? N : int64_t(double(N) * std::sqrt(double(t + 1) / T));
+            if (t == T - 1) rows(r0, r1);
+            else pool.emplace_back(rows, r0, std::max(r0, r1));
+            r0 = std::max(r0, r1);
+        }
+        for (std::thread& th : pool) th.join();
     }
     int flag = 0;
     if (cudaMemcpy(&flag, ds->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
