@@ -43,6 +43,7 @@ extern "C" {
 #define SYRK_ERR_PLAN          -7  /* invalid schedule parameters                         */
 #define SYRK_ERR_DEVICE_WAIT   -8  /* a bounded wait inside a kernel ran out (see syrk_last_status) */
 #define SYRK_ERR_NO_DEVICE     -9  /* no CUDA device / not an sm_100 device               */
+#define SYRK_ERR_NOT_SPD      -11  /* cholesky_lower met a non-positive pivot (see cholesky_last_info) */
 #define SYRK_ERR_STATIC_LIMIT -10  /* syrk_lower_bf16_static: problem exceeds its fixed arrays */
 
 /* schedules (syrk_set_schedule) */
@@ -128,6 +129,24 @@ int syrk_lower_bf16_static(int64_t N, int64_t M,
                            void* C, int64_t ldc,
                            double alpha, double beta,
                            int slices, void* stream);
+
+/*
+ * Cholesky factorisation by Large Block Cholesky (Algorithm 5 of the paper, LBC): replaces the
+ * lower triangle of the symmetric positive definite FP64 matrix A (device pointer, row-major
+ * N x N, row pitch lda >= N) by L with A = L * L^T.  Entries above the diagonal are never read
+ * or written.  Right-looking with panels of `block` columns (0 = 512; a multiple of 128 up to
+ * 4096; the paper suggests about sqrt(N)): each panel is factored and the rows below it solved
+ * in 128-column steps, then the trailing matrix gets A[I1,I1] -= A[I1,I0] * A[I1,I0]^T through
+ * syrk_lower's triangle-block kernel, which is where almost all the arithmetic is.
+ *
+ * A must be 16-byte aligned and lda even (SYRK_ERR_LD otherwise).  The call enqueues all work on
+ * `stream` and returns; workspaces (N x 128 doubles and a few 128 x 128 blocks) are created on
+ * first use and kept until syrk_shutdown().  A non-positive pivot does not stop the enqueued
+ * work: after synchronising the stream, cholesky_last_info() returns 0, or k + 1 for the first
+ * pivot k that was not positive (the contents of A are then undefined from column k on).
+ */
+int     cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, void* stream);
+int64_t cholesky_last_info(void* stream);
 
 /* Build and upload the work list for (N, M, dtype) ahead of time, so that a later
  * syrk_lower with these sizes allocates nothing. */

@@ -22,7 +22,7 @@ MAX_SEG, MAX_TILE = 8, 16
 EXPORTS = [
     "syrk_lower", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_get_schedule_stats",
-    "syrk_probe_f64_mma_peak", "syrk_lower_bf16_static",
+    "syrk_probe_f64_mma_peak", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
     "tbs_plan_build", "tbs_plan_balance", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
 ]
 
@@ -79,6 +79,10 @@ def lib() -> ctypes.CDLL:
         L.syrk_probe_f64_mma_peak.argtypes = [ci, ctypes.POINTER(dbl)]
         L.syrk_lower_bf16_static.restype = ci
         L.syrk_lower_bf16_static.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
+        L.cholesky_lower.restype = ci
+        L.cholesky_lower.argtypes = [i64, vp, i64, i64, vp]
+        L.cholesky_last_info.restype = i64
+        L.cholesky_last_info.argtypes = [vp]
         L.tbs_plan_build.restype = vp
         L.tbs_plan_build.argtypes = [i64, ci, ci, ci, ci, ci]
         L.tbs_plan_balance.restype = ci
@@ -151,6 +155,20 @@ def syrk_lower_bf16_static(N: int, M: int, A, lda: int, C, ldc: int, alpha: floa
         stream = torch.cuda.current_stream().cuda_stream
     _check(lib().syrk_lower_bf16_static(N, M, _ptr(A), lda, _ptr(C), ldc, float(alpha), float(beta),
                                         int(slices), stream))
+
+
+def cholesky_lower(N: int, A, lda: int, block: int = 0, stream: Optional[int] = None) -> None:
+    """Enqueue the in-place lower Cholesky factorisation (Large Block Cholesky) of the FP64 device
+    matrix A; check cholesky_last_info() after synchronising."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().cholesky_lower(N, _ptr(A), lda, block, stream))
+
+
+def cholesky_last_info(stream: Optional[int] = None) -> int:
+    """0, or k + 1 for the first non-positive pivot k of the last factorisation (after a sync)."""
+    return int(lib().cholesky_last_info(stream))
 
 
 def syrk_plan_prepare(N: int, M: int, dtype: int) -> None:

@@ -65,8 +65,10 @@ int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk)
     return auto_split_k(dp->plan.items, M, bk, ds->sm_count, runtime().split_k);
 }
 
-int run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
-               double beta, int dtype, cudaStream_t stream) {
+}  // namespace
+
+int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
+                            double beta, int dtype, cudaStream_t stream) {
     DeviceState* ds = nullptr;
     int rc = get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
@@ -111,6 +113,8 @@ int run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
+namespace {
+
 // Lower triangle of C (row pitch ldc) -> packed rows (row i has i+1 entries), on device.
 template <typename T>
 __global__ void pack_lower_kernel(int64_t N, const T* __restrict__ C, int64_t ldc, T* __restrict__ packed) {
@@ -130,7 +134,7 @@ int syrk_lower(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_
     int rc = validate(N, M, A, lda, C, ldc, dtype);
     if (rc != SYRK_OK || N == 0) return rc;
     std::lock_guard<std::mutex> lock(runtime().mu);
-    return run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream));
+    return syrk_run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream));
 }
 
 int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
@@ -161,7 +165,7 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     if (beta != 0.0)
         ok = ok && cudaMemcpy2DAsync(ds->d_c, dldc * ec, C, ldc * ec, N * ec, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return SYRK_ERR_CUDA; }
-    rc = run_device(N, M, ds->d_a, dlda, ds->d_c, dldc, alpha, beta, dtype, st);
+    rc = syrk_run_device(N, M, ds->d_a, dlda, ds->d_c, dldc, alpha, beta, dtype, st);
     if (rc != SYRK_OK) return rc;
     const dim3 grid(unsigned(std::min<int64_t>(64, (N + 255) / 256)), unsigned(N));
     if (dtype == SYRK_DTYPE_F64)
@@ -254,6 +258,7 @@ const char* syrk_strerror(int code) {
         case SYRK_ERR_PLAN: return "invalid schedule parameters";
         case SYRK_ERR_DEVICE_WAIT: return "a bounded wait inside a kernel ran out";
         case SYRK_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+        case SYRK_ERR_NOT_SPD: return "matrix is not positive definite";
         case SYRK_ERR_STATIC_LIMIT: return "problem too large for the fixed arrays of syrk_lower_bf16_static (work items or slices x tiles)";
         default: return "unknown error code";
     }

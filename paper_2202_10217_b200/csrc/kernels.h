@@ -14,6 +14,12 @@ namespace tbsyrk {
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int* d_status, cudaStream_t stream);
+// The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
+// P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
+// columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.
+cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, const CUtensorMap* tmD,
+                               int64_t nrows, int64_t ncols, int64_t K, double* D, int64_t ldd, double alpha,
+                               double beta, int* d_status, cudaStream_t stream);
 int f64_tile();
 int f64_bk();
 int f64_stages();

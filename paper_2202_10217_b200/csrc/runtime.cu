@@ -215,6 +215,20 @@ int encode_tensor_map_c_f32(CUtensorMap* tm, const void* C, int64_t N, int64_t l
     return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
+int encode_tensor_map_f64_plain(CUtensorMap* tm, const void* p, int64_t rows, int64_t cols, int64_t ld,
+                                int box_rows, int box_cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SYRK_ERR_CUDA;
+    const cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
+    const cuuint64_t strides[1] = {cuuint64_t(ld) * 8};
+    const cuuint32_t bx[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, 2, const_cast<void*>(p), dims, strides, bx, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
 int encode_tensor_map_c_f64(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return SYRK_ERR_CUDA;
@@ -245,6 +259,7 @@ int ensure_pinned_bytes(void** p, size_t* have, size_t want) {
 }
 
 void release_all() {
+    release_cholesky_workspaces();
     Runtime& rt = runtime();
     int prev = -1;
     cudaGetDevice(&prev);

@@ -75,6 +75,16 @@ int encode_tensor_map_c_f32(CUtensorMap* tm, const void* C, int64_t N, int64_t l
 // The same over an FP64 C, without swizzle (a box row of 32 doubles is 256 bytes).
 int encode_tensor_map_c_f64(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box);
 
+// Plain (unswizzled) FP64 tensor map over a rows x cols row-major matrix with pitch ld.
+int encode_tensor_map_f64_plain(CUtensorMap* tm, const void* p, int64_t rows, int64_t cols, int64_t ld,
+                                int box_rows, int box_cols);
+
+// The device path of syrk_lower (arguments already validated; the caller holds the runtime lock).
+int syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
+                    double beta, int dtype, cudaStream_t stream);
+
+void release_cholesky_workspaces();
+
 // Grow-only device / pinned-host buffers.
 int ensure_device_bytes(void** p, size_t* have, size_t want);
 int ensure_pinned_bytes(void** p, size_t* have, size_t want);

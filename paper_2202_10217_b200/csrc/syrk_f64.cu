@@ -81,10 +81,10 @@ __device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const uint
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
-                    const WorkItem* __restrict__ items, int64_t N, int32_t n_ksteps,
-                    double* __restrict__ C, int64_t ldc, double alpha, double beta, int vec_ok,
-                    int c_tma, int* __restrict__ status) {
+syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
+                    int64_t ncols, int32_t gemm_col_tiles, int32_t n_ksteps, double* __restrict__ C,
+                    int64_t ldc, double alpha, double beta, int vec_ok, int c_tma, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
@@ -95,8 +95,27 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    if (tid < int(sizeof(WorkItem) / 4))
+    // Two-operand mode (gemm_col_tiles > 0): D = alpha * P * Q^T + beta * D without a triangle
+    // mask; block b owns the 4 x 4 tile rectangle (b / column groups, b % column groups), its
+    // column segments come from Q (tmB, the first `pad` segments), its row segments from P (tmA).
+    const bool gemm = gemm_col_tiles > 0;
+    if (gemm) {
+        if (tid == 0) {
+            const int n_cg = (gemm_col_tiles + 3) / 4;
+            const int64_t row_tiles = (N + kTile - 1) / kTile;
+            const int64_t rg = blockIdx.x / n_cg, cg = blockIdx.x % n_cg;
+            const int nc = int(min(int64_t(4), int64_t(gemm_col_tiles) - cg * 4));
+            const int nr = int(min(int64_t(4), row_tiles - rg * 4));
+            for (int y = 0; y < nc; ++y) s_item.seg[y] = int32_t(cg * 4 + y);
+            for (int x = 0; x < nr; ++x) s_item.seg[nc + x] = int32_t(rg * 4 + x);
+            int tt = 0;
+            for (int x = 0; x < nr; ++x)
+                for (int y = 0; y < nc; ++y) { s_item.tile_x[tt] = uint8_t(nc + x); s_item.tile_y[tt] = uint8_t(y); ++tt; }
+            s_item.n_seg = nc + nr; s_item.n_tile = tt; s_item.kind = kRect; s_item.pad = nc;
+        }
+    } else if (tid < int(sizeof(WorkItem) / 4)) {
         reinterpret_cast<int32_t*>(&s_item)[tid] = reinterpret_cast<const int32_t*>(&items[blockIdx.x])[tid];
+    }
     if (tid == 0) s_abort = 0;
     __syncthreads();
 
@@ -104,7 +123,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (tid == 0) {
         bool ok = n_seg >= 1 && n_seg <= kMaxSeg && n_tile >= 1 && n_tile <= kMmaWarps;
         for (int s = 0; ok && s < n_seg; ++s)
-            ok = s_item.seg[s] >= 0 && int64_t(s_item.seg[s]) * kTile < N;
+            ok = s_item.seg[s] >= 0 && int64_t(s_item.seg[s]) * kTile < ((gemm && s < s_item.pad) ? ncols : N);
         for (int t = 0; ok && t < n_tile; ++t)
             ok = s_item.tile_x[t] < n_seg && s_item.tile_y[t] < n_seg;
         // A triangle block in the generator's tile order (x = 1..5, y < x): the 16th warp helps.
@@ -138,7 +157,8 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 mbar_arrive_expect_tx(&full_bar[st], uint32_t(n_seg) * kSegBytes);
                 uint8_t* dst = smem + st * kStageBytes;
                 for (int s = 0; s < n_seg; ++s)
-                    tma_load_2d(dst + s * kSegBytes, &tmA, ks * kBK, s_item.seg[s] * kTile, &full_bar[st]);
+                    tma_load_2d(dst + s * kSegBytes, (gemm && s < s_item.pad) ? &tmB : &tmA, ks * kBK,
+                                s_item.seg[s] * kTile, &full_bar[st]);
                 issued = ks + 1;
             }
             if (c_tma && !s_abort) {
@@ -151,13 +171,13 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     }
                     int below = 0;
                     for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt)
-                        below += (s_item.seg[s_item.tile_x[tt]] != s_item.seg[s_item.tile_y[tt]]) ? 1 : 0;
+                        below += (gemm || s_item.seg[s_item.tile_x[tt]] != s_item.seg[s_item.tile_y[tt]]) ? 1 : 0;
                     if (below == 0) { mbar_arrive(&full_bar[st]); continue; }
                     mbar_arrive_expect_tx(&full_bar[st], uint32_t(below) * kCTileBytes);
                     uint8_t* dst = smem + st * kStageBytes;
                     for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt) {
                         const int rx = s_item.seg[s_item.tile_x[tt]], cy = s_item.seg[s_item.tile_y[tt]];
-                        if (rx != cy) tma_load_2d(dst + (tt & 3) * kCTileBytes, &tmC, cy * kTile, rx * kTile, &full_bar[st]);
+                        if (gemm || rx != cy) tma_load_2d(dst + (tt & 3) * kCTileBytes, &tmC, cy * kTile, rx * kTile, &full_bar[st]);
                     }
                     issued = q + 1;
                 }
@@ -260,7 +280,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ------------------------------ epilogue ------------------------------
     const int64_t row0 = int64_t(s_item.seg[sx]) * kTile, col0 = int64_t(s_item.seg[sy]) * kTile;
     const uint8_t* old_tile = nullptr;                  // this warp's old C tile in shared memory
-    if (c_tma && row0 != col0) {
+    if (c_tma && (gemm || row0 != col0)) {
         const int qs = n_ksteps + (warp >> 2);
         if (!mbar_wait_bounded(&full_bar[qs % kStages], (qs / kStages) & 1, &s_abort)) {
             s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return;
@@ -271,26 +291,26 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     for (int mi = 0; mi < 4; ++mi) {
         const int64_t r = row0 + mi * 8 + g;
         if (r >= N) continue;
+        const int64_t cmax = gemm ? ncols - 1 : r;      // last column this row may touch
         double* crow = C + r * ldc;
 #pragma unroll
         for (int ni = 0; ni < 4; ++ni) {
             if (scavenge && mi == 3 && ni == 3) continue;             // written by the 16th warp
             const int64_t c = col0 + ni * 8 + 2 * t;
+            if (c > cmax) continue;
+            const bool both = (c + 1 <= cmax);
             double v0 = alpha * acc[mi][ni][0], v1 = alpha * acc[mi][ni][1];
-            if (old_tile) {                                           // tile below the diagonal, vec_ok holds
-                const double2 o = *reinterpret_cast<const double2*>(old_tile + (mi * 8 + g) * (kTile * 8) + (ni * 8 + 2 * t) * 8);
-                *reinterpret_cast<double2*>(crow + c) = make_double2(v0 + beta * o.x, v1 + beta * o.y);
-            } else if (c + 1 <= r) {
-                if (vec_ok) {
-                    double2* p = reinterpret_cast<double2*>(crow + c);
-                    if (use_beta) { const double2 o = *p; v0 += beta * o.x; v1 += beta * o.y; }
-                    *p = make_double2(v0, v1);
-                } else {
-                    if (use_beta) { v0 += beta * crow[c]; v1 += beta * crow[c + 1]; }
-                    crow[c] = v0; crow[c + 1] = v1;
-                }
-            } else if (c <= r) {
-                if (use_beta) v0 += beta * crow[c];
+            if (use_beta) {
+                double2 o = make_double2(0.0, 0.0);
+                if (old_tile) o = *reinterpret_cast<const double2*>(old_tile + (mi * 8 + g) * (kTile * 8) + (ni * 8 + 2 * t) * 8);
+                else if (both && vec_ok) o = *reinterpret_cast<const double2*>(crow + c);
+                else { o.x = crow[c]; if (both) o.y = crow[c + 1]; }
+                v0 += beta * o.x; v1 += beta * o.y;
+            }
+            if (both) {
+                if (vec_ok) *reinterpret_cast<double2*>(crow + c) = make_double2(v0, v1);
+                else { crow[c] = v0; crow[c + 1] = v1; }
+            } else {
                 crow[c] = v0;
             }
         }
@@ -299,9 +319,8 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
 }  // namespace f64
 
-cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
-                            int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
-                            double beta, int* d_status, cudaStream_t stream) {
+namespace {
+cudaError_t configure_f64_kernel() {
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(f64::syrk_f64_tbs_kernel,
@@ -309,13 +328,40 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
         if (e != cudaSuccess) return e;
         configured = true;
     }
+    return cudaSuccess;
+}
+}  // namespace
+
+cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
+                            int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
+                            double beta, int* d_status, cudaStream_t stream) {
+    cudaError_t e = configure_f64_kernel();
+    if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0) ? 1 : 0;
     const int32_t n_ksteps = int32_t((M + f64::kBK - 1) / f64::kBK);
     const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
     CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
-        tmA, c_tma ? *tmC : none, d_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
+        tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, const CUtensorMap* tmD,
+                               int64_t nrows, int64_t ncols, int64_t K, double* D, int64_t ldd, double alpha,
+                               double beta, int* d_status, cudaStream_t stream) {
+    cudaError_t e = configure_f64_kernel();
+    if (e != cudaSuccess) return e;
+    if (nrows == 0 || ncols == 0) return cudaSuccess;
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0 && (ldd & 1) == 0) ? 1 : 0;
+    const int32_t n_ksteps = int32_t((K + f64::kBK - 1) / f64::kBK);
+    const int c_tma = (tmD != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
+    const int64_t row_tiles = (nrows + f64::kTile - 1) / f64::kTile, col_tiles = (ncols + f64::kTile - 1) / f64::kTile;
+    const int64_t blocks = ((row_tiles + 3) / 4) * ((col_tiles + 3) / 4);
+    CUtensorMap none{};
+    f64::syrk_f64_tbs_kernel<<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
+        tmP, tmQ, c_tma ? *tmD : none, nullptr, nrows, ncols, int32_t(col_tiles), n_ksteps, D, ldd, alpha, beta,
+        vec_ok, c_tma, d_status);
     return cudaGetLastError();
 }
 
