@@ -387,12 +387,55 @@ def run_sweep(args, rank: int, world: int, local_rank: int):
         dist.destroy_process_group()
 
 
+def run_cholesky(args, rank: int, world: int, local_rank: int):
+    """Large Block Cholesky of a seeded 32768^2 FP64 matrix (n*I + G G^T / 512); a step is one
+    factorisation (the matrix is restored from a device copy between steps, outside the timing)."""
+    import torch
+    from paper_2202_10217_b200 import binding as B
+
+    torch.cuda.set_device(local_rank)
+    n, M = 32768, I.SWEEP_K
+    G = torch.from_numpy(I.sweep_factor(n)).cuda()
+    A0 = torch.matmul(G, G.T) / float(M)
+    A0.diagonal().add_(float(n))
+    del G
+    A = A0.clone()
+    flops = n ** 3 / 3.0
+    steps = max(1, min(args.steps, 5))
+    times = []
+    for i in range(steps + 1):                       # first pass is the warm-up (allocates work lists)
+        A.copy_(A0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.cholesky_lower(n, A, n, args.block)
+        e1.record()
+        torch.cuda.synchronize()
+        assert B.syrk_last_status() == 0 and B.cholesky_last_info() == 0
+        if i > 0:
+            times.append(e0.elapsed_time(e1))
+    ms = float(np.mean(times))
+    # residual on sampled entries: (L L^T)_ij against A0_ij
+    idx = torch.randint(0, n, (4096,), device="cuda")
+    jdx = (torch.rand(4096, device="cuda") * (idx + 1)).long()
+    L = torch.tril(A)
+    rec = (L[idx] * L[jdx]).sum(dim=1)
+    err = float((rec - A0[idx, jdx]).abs().max() / A0.abs().max())
+    peak = B.syrk_probe_f64_mma_peak(20000)
+    print(json.dumps({"metric": "cholesky_tflops_N^3/3", "value": flops / (ms * 1e-3) * 1e-12, "unit": UNIT,
+                      "n_gpus": 1, "steps": steps, "ms_per_step": ms, "higher_is_better": True, "dtype": "f64",
+                      "data": "synthetic", "config": {"workload": "lbc_f64_32768", "block": args.block or 512},
+                      "sampled_relative_residual": err, "gpu_launches": None,
+                      "roofline": {"bound": "tensor", "achieved": flops / (ms * 1e-3) * 1e-12, "peak": peak,
+                                   "unit": UNIT, "frac": flops / (ms * 1e-3) * 1e-12 / peak, "traffic": None}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c2", choices=sorted(I.CONFIGS) + ["c5"])
+    ap.add_argument("--workload", default="c2", choices=sorted(I.CONFIGS) + ["c5", "lbc"])
+    ap.add_argument("--block", type=int, default=0, help="panel width of --workload lbc (0 = library default)")
     ap.add_argument("--shape", default=None,
                     help="N,M,dtype,alpha,beta (dtype f64|bf16): a custom seeded N(0,1) workload")
     ap.add_argument("--kernel-only", action="store_true",
@@ -403,6 +446,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.workload == "lbc":
+        if rank == 0 and args.impl != "reference":
+            run_cholesky(args, rank, world, local_rank)
+        return
     if args.workload == "c5" and not args.shape:
         if args.impl == "reference":
             args.workload = "c2"                     # the oracle arm samples a single FP64 call
