@@ -394,7 +394,7 @@ def run_cholesky(args, rank: int, world: int, local_rank: int):
     from paper_2202_10217_b200 import binding as B
 
     torch.cuda.set_device(local_rank)
-    n, M = 32768, I.SWEEP_K
+    n, M = args.lbc_n, I.SWEEP_K
     G = torch.from_numpy(I.sweep_factor(n)).cuda()
     A0 = torch.matmul(G, G.T) / float(M)
     A0.diagonal().add_(float(n))
@@ -423,7 +423,7 @@ def run_cholesky(args, rank: int, world: int, local_rank: int):
     peak = B.syrk_probe_f64_mma_peak(20000)
     print(json.dumps({"metric": "cholesky_tflops_N^3/3", "value": flops / (ms * 1e-3) * 1e-12, "unit": UNIT,
                       "n_gpus": 1, "steps": steps, "ms_per_step": ms, "higher_is_better": True, "dtype": "f64",
-                      "data": "synthetic", "config": {"workload": "lbc_f64_32768", "block": args.block or 512},
+                      "data": "synthetic", "config": {"workload": "lbc_f64_%d" % n, "block": args.block or 512},
                       "sampled_relative_residual": err, "gpu_launches": None,
                       "roofline": {"bound": "tensor", "achieved": flops / (ms * 1e-3) * 1e-12, "peak": peak,
                                    "unit": UNIT, "frac": flops / (ms * 1e-3) * 1e-12 / peak, "traffic": None}}))
@@ -435,6 +435,7 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c2", choices=sorted(I.CONFIGS) + ["c5", "lbc"])
+    ap.add_argument("--lbc-n", type=int, default=32768, help="matrix size of --workload lbc")
     ap.add_argument("--block", type=int, default=0, help="panel width of --workload lbc (0 = library default)")
     ap.add_argument("--shape", default=None,
                     help="N,M,dtype,alpha,beta (dtype f64|bf16): a custom seeded N(0,1) workload")

