@@ -134,13 +134,14 @@ int syrk_lower_bf16_static(int64_t N, int64_t M,
  * Cholesky factorisation by Large Block Cholesky (Algorithm 5 of the paper, LBC): replaces the
  * lower triangle of the symmetric positive definite FP64 matrix A (device pointer, row-major
  * N x N, row pitch lda >= N) by L with A = L * L^T.  Entries above the diagonal are never read
- * or written.  Right-looking with panels of `block` columns (0 = 512; a multiple of 128 up to
- * 4096; the paper suggests about sqrt(N)): each panel is factored and the rows below it solved
+ * or written.  Right-looking with panels of `block` columns (0 = 512, or 1024 from N = 16384 on; a
+ * multiple of 128 up to 4096; the paper suggests about sqrt(N)): each panel is factored and the rows below it solved
  * in 128-column steps, then the trailing matrix gets A[I1,I1] -= A[I1,I0] * A[I1,I0]^T through
  * syrk_lower's triangle-block kernel, which is where almost all the arithmetic is.
  *
  * A must be 16-byte aligned and lda even (SYRK_ERR_LD otherwise).  The call enqueues all work on
- * `stream` and returns; workspaces (N x 128 doubles and a few 128 x 128 blocks) are created on
+ * `stream` and returns (part of it runs on a second stream of the library that is ordered after the
+ * work already in `stream` and joined back into it before the call returns); workspaces (N x 128 doubles and a few 128 x 128 blocks) are created on
  * first use and kept until syrk_shutdown().  A non-positive pivot does not stop the enqueued
  * work: after synchronising the stream, cholesky_last_info() returns 0, or k + 1 for the first
  * pivot k that was not positive (the contents of A are then undefined from column k on).

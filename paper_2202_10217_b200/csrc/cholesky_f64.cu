@@ -1,6 +1,6 @@
 // Large Block Cholesky (Algorithm 5 of the paper, LBC) in FP64, lower triangle, in place.
 //
-// Right-looking blocked factorisation with block size b (default 512).  For the panel of
+// Right-looking blocked factorisation with block size b (default 512, 1024 from N = 16384 on).  For the panel of
 // columns I0 = [o, o + b):
 //   1. A[I0, I0] <- its Cholesky factor                      (the paper's OOC_CHOL step)
 //   2. A[I1, I0] <- A[I1, I0] * L00^-T, I1 = [o + b, N)      (the paper's OOC_TRSM step)
@@ -184,6 +184,8 @@ struct CholWorkspace {
     double* t = nullptr;          // N x 128 staging of a solved column block
     size_t t_bytes = 0;
     long long* info = nullptr;
+    cudaStream_t panel_stream = nullptr;   // panel factorisations run here, ahead of the trailing update
+    cudaEvent_t ev_panel = nullptr, ev_rest = nullptr;
 };
 std::mutex g_chol_mu;
 CholWorkspace g_ws[64];
@@ -213,7 +215,7 @@ extern "C" int cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, 
     if (!A) return SYRK_ERR_NULL;
     if (lda < N) return SYRK_ERR_LD;
     if ((reinterpret_cast<uintptr_t>(A) & 15) != 0 || (lda & 1) != 0) return SYRK_ERR_LD;   // TMA rules for the panels
-    if (block == 0) block = 512;
+    if (block == 0) block = (N >= 16384) ? 1024 : 512;
     if (block < kLeaf || block > 4096 || block % kLeaf != 0) return SYRK_ERR_SIZE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
@@ -232,6 +234,15 @@ extern "C" int cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, 
         if ((rc = ensure_device_bytes(&p, &ws.t_bytes, size_t(N) * kLeaf * sizeof(double))) != SYRK_OK) return rc;
         ws.t = static_cast<double*>(p);
         if (!ws.info && cudaMalloc(&ws.info, sizeof(long long)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
+        if (!ws.panel_stream) {
+            int lo = 0, hi = 0;
+            cudaDeviceGetStreamPriorityRange(&lo, &hi);
+            if (cudaStreamCreateWithPriority(&ws.panel_stream, cudaStreamNonBlocking, hi) != cudaSuccess ||
+                cudaEventCreateWithFlags(&ws.ev_panel, cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&ws.ev_rest, cudaEventDisableTiming) != cudaSuccess) {
+                cudaGetLastError(); return SYRK_ERR_CUDA;
+            }
+        }
         static bool leaf_configured = false;
         if (!leaf_configured) {
             if (cudaFuncSetAttribute(chol_leaf_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLeafSmem) != cudaSuccess) {
@@ -242,36 +253,62 @@ extern "C" int cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, 
     }
     if (cudaMemsetAsync(ws.info, 0, sizeof(long long), st) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
 
+    // One panel of look-ahead: the trailing update of panel p is split into the columns of panel
+    // p + 1 (done first, on the panel stream) and the rest (on the caller's stream); panel p + 1
+    // is then factored on the panel stream while the rest of update p is still running.
+    cudaStream_t sp = ws.panel_stream;
+    cudaEvent_t ev_panel = ws.ev_panel, ev_rest = ws.ev_rest;
+    auto chk = [](cudaError_t e) { if (e != cudaSuccess) { cudaGetLastError(); return false; } return true; };
+    if (!chk(cudaEventRecord(ev_rest, st)) || !chk(cudaStreamWaitEvent(sp, ev_rest, 0))) return SYRK_ERR_CUDA;   // sp starts after the caller's prior work
+
     for (int64_t o = 0; o < N; o += block) {
         const int64_t bb = std::min<int64_t>(block, N - o);
+        // ---- panel [o, o + bb) on the panel stream: factor, solve the rows below ----
         for (int64_t cj = o; cj < o + bb; cj += kLeaf) {
             const int m = int(std::min<int64_t>(kLeaf, o + bb - cj));
             double* Wj = ws.w + size_t((cj - o) / kLeaf) * kLeaf * kLeaf;
-            chol_leaf_kernel<<<1, kLeafThreads, kLeafSmem, st>>>(A + cj * lda + cj, lda, m, Wj, ws.info, cj);
+            chol_leaf_kernel<<<1, kLeafThreads, kLeafSmem, sp>>>(A + cj * lda + cj, lda, m, Wj, ws.info, cj);
             if (cudaGetLastError() != cudaSuccess) return SYRK_ERR_CUDA;
             const int64_t below = N - (cj + m);
             if (below <= 0) continue;
             double* panel = A + (cj + m) * lda + cj;              // rows below the leaf, its m columns
             // solve: panel <- panel * L_jj^-T  (through the staging buffer: the product is not in place)
-            if ((rc = gemm_nt(ds, below, m, m, panel, lda, Wj, kLeaf, ws.t, kLeaf, 1.0, 0.0, st)) != SYRK_OK) return rc;
-            if (cudaMemcpy2DAsync(panel, size_t(lda) * 8, ws.t, size_t(kLeaf) * 8, size_t(m) * 8, size_t(below),
-                                  cudaMemcpyDeviceToDevice, st) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+            if ((rc = gemm_nt(ds, below, m, m, panel, lda, Wj, kLeaf, ws.t, kLeaf, 1.0, 0.0, sp)) != SYRK_OK) return rc;
+            if (!chk(cudaMemcpy2DAsync(panel, size_t(lda) * 8, ws.t, size_t(kLeaf) * 8, size_t(m) * 8, size_t(below),
+                                       cudaMemcpyDeviceToDevice, sp))) return SYRK_ERR_CUDA;
             const int64_t rem = o + bb - (cj + m);                // panel columns still to be updated
             if (rem <= 0) continue;
             // inside the panel: square block [cj+m, o+bb)^2, lower triangle
             if ((rc = syrk_run_device(rem, m, panel, lda, A + (cj + m) * lda + (cj + m), lda, -1.0, 1.0,
-                                      SYRK_DTYPE_F64, st)) != SYRK_OK) return rc;
+                                      SYRK_DTYPE_F64, sp)) != SYRK_OK) return rc;
             // below the panel: rows [o+bb, N) x columns [cj+m, o+bb)
             const int64_t nb = N - (o + bb);
             if ((rc = gemm_nt(ds, nb, rem, m, A + (o + bb) * lda + cj, lda, panel, lda, A + (o + bb) * lda + (cj + m), lda,
-                              -1.0, 1.0, st)) != SYRK_OK) return rc;
+                              -1.0, 1.0, sp)) != SYRK_OK) return rc;
         }
-        const int64_t nb = N - (o + bb);
-        if (nb > 0) {                                             // the TBS step of Algorithm 5
-            if ((rc = syrk_run_device(nb, bb, A + (o + bb) * lda + o, lda, A + (o + bb) * lda + (o + bb), lda, -1.0, 1.0,
+        const int64_t o1 = o + bb, nb = N - o1;
+        if (nb <= 0) break;
+        // ---- trailing update A[I1,I1] -= A[I1,I0] A[I1,I0]^T (the TBS step of Algorithm 5), in two parts ----
+        const double* P = A + o1 * lda + o;                       // A[I1, I0]: nb x bb
+        const int64_t b1 = std::min<int64_t>(block, nb);          // width of the next panel
+        // (a) columns of the next panel, on the panel stream: its diagonal block and the rows below it.
+        //     They lie inside the region part (b) of the previous update wrote: wait for it.
+        if (!chk(cudaStreamWaitEvent(sp, ev_rest, 0))) return SYRK_ERR_CUDA;
+        if ((rc = syrk_run_device(b1, bb, P, lda, A + o1 * lda + o1, lda, -1.0, 1.0, SYRK_DTYPE_F64, sp)) != SYRK_OK) return rc;
+        if ((rc = gemm_nt(ds, nb - b1, b1, bb, P + b1 * lda, lda, P, lda, A + (o1 + b1) * lda + o1, lda, -1.0, 1.0, sp)) != SYRK_OK) return rc;
+        if (!chk(cudaEventRecord(ev_panel, sp))) return SYRK_ERR_CUDA;
+        // (b) the rest, on the caller's stream, concurrently with the next panel's factorisation
+        if (nb - b1 > 0) {
+            if (!chk(cudaStreamWaitEvent(st, ev_panel, 0))) return SYRK_ERR_CUDA;
+            if ((rc = syrk_run_device(nb - b1, bb, P + b1 * lda, lda, A + (o1 + b1) * lda + (o1 + b1), lda, -1.0, 1.0,
                                       SYRK_DTYPE_F64, st)) != SYRK_OK) return rc;
+            if (!chk(cudaEventRecord(ev_rest, st))) return SYRK_ERR_CUDA;
         }
+        // The next panel's factorisation (next iteration, panel stream) touches only the columns that
+        // part (a) wrote, so it runs concurrently with part (b).
     }
+    // the caller's stream continues after everything on the panel stream
+    if (!chk(cudaEventRecord(ev_panel, sp)) || !chk(cudaStreamWaitEvent(st, ev_panel, 0))) return SYRK_ERR_CUDA;
     return SYRK_OK;
 }
 
@@ -293,6 +330,9 @@ void release_cholesky_workspaces() {
         if (ws.w) cudaFree(ws.w);
         if (ws.t) cudaFree(ws.t);
         if (ws.info) cudaFree(ws.info);
+        if (ws.panel_stream) cudaStreamDestroy(ws.panel_stream);
+        if (ws.ev_panel) cudaEventDestroy(ws.ev_panel);
+        if (ws.ev_rest) cudaEventDestroy(ws.ev_rest);
         ws = CholWorkspace{};
     }
     cudaGetLastError();
