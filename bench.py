@@ -145,8 +145,9 @@ def run_reference(args, wl: I.Workload, rank: int):
 # captures summarised under profiles/.  Valid only for the kernel source it was taken on.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, sha256 of the kernel source at capture time)
-    "c2_f64_4096x4096": (786_889_472, "c682423e7463c2af270ecf695a4e4cacf991ea8694e2352a6c3dcbca70e44220"),
-    "c3_bf16_16384x4096": (1_808_215_984, "a0c0b2d9ad91a1e0684e744e9ead0eb8b753a9131f407e699dc879ce4431e556"),
+    "c2_f64_4096x4096": (776_841_984, "ffce25a1242a9bc40445b184443a2f5909a376bec13969b80b348bd5580269a9"),
+    "c3_bf16_16384x4096": (1_901_564_240, "6d3634d1378014482fc34c494f00de6ae799fe5a2c202f4d6b6394ab679ed5f1"),
+    "c4_bf16_2048x262144": (2_829_940_056, "6d3634d1378014482fc34c494f00de6ae799fe5a2c202f4d6b6394ab679ed5f1"),
 }
 
 
