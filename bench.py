@@ -145,9 +145,9 @@ def run_reference(args, wl: I.Workload, rank: int):
 # captures summarised under profiles/.  Valid only for the kernel source it was taken on.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, sha256 of the kernel source at capture time)
-    "c2_f64_4096x4096": (776_841_984, "ffce25a1242a9bc40445b184443a2f5909a376bec13969b80b348bd5580269a9"),
-    "c3_bf16_16384x4096": (1_901_564_240, "6d3634d1378014482fc34c494f00de6ae799fe5a2c202f4d6b6394ab679ed5f1"),
-    "c4_bf16_2048x262144": (2_829_940_056, "6d3634d1378014482fc34c494f00de6ae799fe5a2c202f4d6b6394ab679ed5f1"),
+    "c2_f64_4096x4096": (777_772_288, "7b8c18f67a7ae93954eaacd0a2b84ee81904352564189c45e601f2351a35338d"),
+    "c3_bf16_16384x4096": (1_929_455_616, "bdbdbe0287129decd338866798941c9d5382b66f3e0cefd7d9cbb2e9065a3296"),
+    "c4_bf16_2048x262144": (2_859_560_192, "bdbdbe0287129decd338866798941c9d5382b66f3e0cefd7d9cbb2e9065a3296"),
 }
 
 

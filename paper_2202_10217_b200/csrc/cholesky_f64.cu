@@ -243,12 +243,12 @@ extern "C" int cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, 
                 cudaGetLastError(); return SYRK_ERR_CUDA;
             }
         }
-        static bool leaf_configured = false;
-        if (!leaf_configured) {
+        static bool leaf_configured[64] = {};
+        if (!leaf_configured[ds->device]) {
             if (cudaFuncSetAttribute(chol_leaf_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLeafSmem) != cudaSuccess) {
                 cudaGetLastError(); return SYRK_ERR_CUDA;
             }
-            leaf_configured = true;
+            leaf_configured[ds->device] = true;
         }
     }
     if (cudaMemsetAsync(ws.info, 0, sizeof(long long), st) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }

@@ -416,12 +416,16 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int* d_status,
                              int sm_count, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
+    // The shared-memory attribute belongs to a device's context: set it once per device.
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(bf16::syrk_bf16_tbs_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, bf16::kSmemBytes);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
     if (n_items == 0) return cudaSuccess;
     const int32_t n_ksteps = int32_t((M + bf16::kBK - 1) / bf16::kBK);

@@ -321,12 +321,16 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
 namespace {
 cudaError_t configure_f64_kernel() {
-    static bool configured = false;
-    if (!configured) {
+    // The shared-memory attribute belongs to a device's context: set it once per device.
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(f64::syrk_f64_tbs_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, f64::kSmemBytes);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
     return cudaSuccess;
 }

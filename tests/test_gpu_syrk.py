@@ -152,3 +152,39 @@ def test_host_buffer_entry_point(dtype):
     assert_within_tolerance(C.astype(np.float64), ref, bound, M, -1.0, 1.0, Cin, dtype)
     iu = np.triu_indices(N, 1)
     assert np.array_equal(C[iu], Cin[iu])               # host upper triangle untouched
+
+
+def test_shutdown_releases_everything_and_the_library_can_be_used_again():
+    N, M = 300, 64
+    A = make_A(N, M, B.DTYPE_F64, seed=21, kind="int")
+    got1, ref, bound = run_case(A, B.DTYPE_F64, 1.0, 0.0)
+    B.syrk_shutdown()
+    B.syrk_plan_prepare(N, M, B.DTYPE_F64)               # rebuilds the cached work list
+    got2, _, _ = run_case(A, B.DTYPE_F64, 1.0, 0.0)
+    assert_within_tolerance(got2, ref, bound, M, 1.0, 0.0, None, B.DTYPE_F64, exact=True)
+    assert np.array_equal(got1[np.tril_indices(N)], got2[np.tril_indices(N)])
+    A16 = make_A(400, 128, B.DTYPE_BF16_F32, seed=22, kind="int")
+    got, ref, bound = run_case(A16, B.DTYPE_BF16_F32, 1.0, 0.0)
+    assert_within_tolerance(got, ref, bound, 128, 1.0, 0.0, None, B.DTYPE_BF16_F32, exact=True)
+
+
+def test_two_streams_back_to_back():
+    """Calls on two streams that do not overlap in C run correctly one after the other."""
+    import torch
+    N, M = 600, 96
+    A = make_A(N, M, B.DTYPE_F64, seed=23, kind="int")
+    dA = torch.from_numpy(A).cuda()
+    outs = []
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for s in streams:
+        dC = torch.zeros((N, N), dtype=torch.float64, device="cuda")
+        with torch.cuda.stream(s):
+            B.syrk_lower(N, M, dA, M, dC, N, 1.0, 0.0, B.DTYPE_F64, stream=s.cuda_stream)
+        outs.append(dC)
+    torch.cuda.synchronize()
+    assert B.syrk_last_status() == 0
+    ref, _ = O.syrk_lower(A, None, 1.0, 0.0, B.DTYPE_F64)
+    il = np.tril_indices(N)
+    for dC in outs:
+        assert np.array_equal(dC.cpu().numpy()[il], ref[il])
