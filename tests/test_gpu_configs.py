@@ -155,3 +155,28 @@ def test_forced_split_k_matches_reference(split):
     il, iu = np.tril_indices(N), np.triu_indices(N, 1)
     assert np.array_equal(got[il], ref[il])                          # integers: exact in any order
     assert np.array_equal(got[iu], Cin[iu].astype(np.float64))
+
+
+@pytest.mark.parametrize("dtype,N,M", [(B.DTYPE_BF16_F32, 20001, 104), (B.DTYPE_F64, 12003, 50)])
+def test_large_ragged_sizes_sampled(dtype, N, M):
+    """Hundreds of tile rows with a ragged last tile and a ragged last K-step; alpha/beta general."""
+    A = I.normal_f64(N, M, 77) if dtype == B.DTYPE_F64 else I.normal_bf16(N, M, 77)
+    dA = upload_A(A, dtype)
+    tdt = torch.float64 if dtype == B.DTYPE_F64 else torch.float32
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    dC = torch.randn((N, N), dtype=tdt, device="cuda", generator=gen)
+    ii, jj = sample_pairs(N, 1 << 16, 32 if dtype == B.DTYPE_F64 else 128, seed=78)
+    gi, gj = torch.from_numpy(ii).cuda(), torch.from_numpy(jj).cuda()
+    before = dC[gi, gj].cpu().numpy().astype(np.float64)
+    up_before = dC[gj[:256], gi[:256]].clone()
+    alpha, beta = 0.75, -1.25
+    B.syrk_lower(N, M, dA, M, dC, N, alpha, beta, dtype)
+    torch.cuda.synchronize()
+    assert B.syrk_last_status() == 0
+    got = dC[gi, gj].cpu().numpy().astype(np.float64)
+    ref, bound = O.syrk_entries(ii, jj, A, None, alpha, 0.0, dtype)
+    ref = ref + beta * before
+    tol = O.tolerance(M, bound, np.abs(before), alpha, beta, dtype)
+    assert np.all(np.abs(got - ref) <= tol)
+    strict = torch.from_numpy(ii[:256] != jj[:256]).cuda()
+    assert torch.equal(dC[gj[:256], gi[:256]][strict], up_before[strict])
