@@ -179,6 +179,21 @@ int syrk_probe_f64_mma_peak(int iters, double* tflops);
 int syrk_set_split_k(int slices);
 
 /*
+ * How later FP64 calls hand the work items of the schedule (Algorithm 4, tiled as in
+ * Section 5.1.4) to thread blocks; the paper has no counterpart, results are the same
+ * entry for entry.  PER_ITEM: one thread block per item.  PERSISTENT: one block per SM
+ * that draws items from a device-side counter, so an item's first loads overlap the
+ * previous item's write-out; used only outside stream capture and for at most 256
+ * distinct streams per device, else the call falls back to PER_ITEM.  AUTO (default):
+ * PERSISTENT when M <= 1024 and the list has at least four items per SM.
+ * Returns SYRK_ERR_PLAN for another value.  Process-wide.
+ */
+#define SYRK_F64_LAUNCH_AUTO 0
+#define SYRK_F64_LAUNCH_PER_ITEM 1
+#define SYRK_F64_LAUNCH_PERSISTENT 2
+int syrk_set_f64_launch(int mode);
+
+/*
  * What a call with these sizes would run (host only, no device needed).
  * All counts refer to one call.  "a_loads" is the number of elements of A the
  * work list moves from slow to fast memory in the paper's two-level model

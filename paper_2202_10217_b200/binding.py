@@ -21,7 +21,7 @@ MAX_SEG, MAX_TILE = 8, 16
 
 EXPORTS = [
     "syrk_lower", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
-    "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_get_schedule_stats",
+    "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_set_f64_launch", "syrk_get_schedule_stats",
     "syrk_probe_f64_mma_peak", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
     "tbs_plan_build", "tbs_plan_balance", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
 ]
@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.syrk_set_schedule.argtypes = [ci]
         L.syrk_set_split_k.restype = ci
         L.syrk_set_split_k.argtypes = [ci]
+        L.syrk_set_f64_launch.restype = ci
+        L.syrk_set_f64_launch.argtypes = [ci]
         L.syrk_get_schedule_stats.restype = ci
         L.syrk_get_schedule_stats.argtypes = [i64, i64, ci, ctypes.POINTER(ScheduleStats)]
         L.syrk_probe_f64_mma_peak.restype = ci
@@ -185,6 +187,13 @@ def syrk_last_status(stream: Optional[int] = None) -> int:
 
 def syrk_set_schedule(schedule: int) -> None:
     _check(lib().syrk_set_schedule(schedule))
+
+
+F64_LAUNCH_AUTO, F64_LAUNCH_PER_ITEM, F64_LAUNCH_PERSISTENT = 0, 1, 2
+
+
+def syrk_set_f64_launch(mode: int) -> None:
+    _check(lib().syrk_set_f64_launch(mode))
 
 
 def syrk_set_split_k(slices: int) -> None:

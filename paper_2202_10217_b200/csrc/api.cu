@@ -68,7 +68,7 @@ int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk)
 }  // namespace
 
 int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
-                            double beta, int dtype, cudaStream_t stream) {
+                            double beta, int dtype, cudaStream_t stream, int f64_launch) {
     DeviceState* ds = nullptr;
     int rc = get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
@@ -92,8 +92,15 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         CUtensorMap tmc;
         const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
                            encode_tensor_map_c_f64(&tmc, C, N, ldc, f64_tile()) == SYRK_OK;
+        // Persistent blocks hide each item's start-up (a few microseconds) behind the previous item.
+        // That pays when items are short (M <= 1024: at most 64 stages each) and the list fills the
+        // device several times over; for long items one block per item is the faster form.
+        const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
+        const bool persistent = mode == SYRK_F64_LAUNCH_PERSISTENT ||
+                                (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count));
+        int* tickets = persistent ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc,
-                            alpha, beta, ds->d_status, stream);
+                            alpha, beta, tickets, ds->sm_count, ds->d_status, stream);
     } else {
         const int split = pick_split_k(ds, dp, M, ks.bk);
         if (split > 1) {
@@ -268,6 +275,14 @@ int syrk_set_schedule(int schedule) {
     if (schedule != SYRK_SCHEDULE_TBS && schedule != SYRK_SCHEDULE_SQUARE) return SYRK_ERR_PLAN;
     std::lock_guard<std::mutex> lock(runtime().mu);
     runtime().schedule = schedule;
+    return SYRK_OK;
+}
+
+int syrk_set_f64_launch(int mode) {
+    if (mode != SYRK_F64_LAUNCH_AUTO && mode != SYRK_F64_LAUNCH_PER_ITEM && mode != SYRK_F64_LAUNCH_PERSISTENT)
+        return SYRK_ERR_PLAN;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    runtime().f64_launch = mode;
     return SYRK_OK;
 }
 

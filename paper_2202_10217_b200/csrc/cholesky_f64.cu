@@ -300,8 +300,11 @@ extern "C" int cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, 
         // (b) the rest, on the caller's stream, concurrently with the next panel's factorisation
         if (nb - b1 > 0) {
             if (!chk(cudaStreamWaitEvent(st, ev_panel, 0))) return SYRK_ERR_CUDA;
+            // One block per item: the panel stream's blocks, of higher priority, then get the SMs
+            // that this update's blocks free one by one; persistent blocks would hold every SM
+            // until the update ends and the look-ahead would wait behind it.
             if ((rc = syrk_run_device(nb - b1, bb, P + b1 * lda, lda, A + (o1 + b1) * lda + (o1 + b1), lda, -1.0, 1.0,
-                                      SYRK_DTYPE_F64, st)) != SYRK_OK) return rc;
+                                      SYRK_DTYPE_F64, st, SYRK_F64_LAUNCH_PER_ITEM)) != SYRK_OK) return rc;
             if (!chk(cudaEventRecord(ev_rest, st))) return SYRK_ERR_CUDA;
         }
         // The next panel's factorisation (next iteration, panel stream) touches only the columns that

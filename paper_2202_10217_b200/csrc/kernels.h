@@ -8,12 +8,14 @@
 
 namespace tbsyrk {
 
-// FP64 triangle-block kernel: one thread block per work item.
-// `tmC` (may be null): tensor map over C with 32 x 32 FP64 boxes, no swizzle, through which the
-// old C tiles are fetched when beta != 0.
+// FP64 triangle-block kernel.  `tmC` (may be null): tensor map over C with 32 x 32 FP64 boxes, no
+// swizzle, through which the old C tiles are fetched when beta != 0.  With `d_tickets` null there
+// is one thread block per work item; otherwise `n_blocks` persistent blocks draw the items from
+// d_tickets[0] (d_tickets[0..1] must be zero and must not be shared with a launch that can run at
+// the same time; the kernel leaves them zero).
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
-                            double beta, int* d_status, cudaStream_t stream);
+                            double beta, int* d_tickets, int n_blocks, int* d_status, cudaStream_t stream);
 // The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
 // P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
 // columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.

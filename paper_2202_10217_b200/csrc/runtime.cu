@@ -66,10 +66,24 @@ int get_device_state(DeviceState** out) {
         if (prop.major != 10) return SYRK_ERR_NO_DEVICE;  // kernels are built for sm_100a only
         if (cudaMalloc(&ds.d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
         if (cudaMemset(ds.d_status, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+        if (cudaMalloc(&ds.d_tickets, 2 * kTicketStreams * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
+        if (cudaMemset(ds.d_tickets, 0, 2 * kTicketStreams * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
         it = rt.devices.emplace(dev, std::move(ds)).first;
     }
     *out = &it->second;
     return SYRK_OK;
+}
+
+int* tickets_for_stream(DeviceState* ds, cudaStream_t stream) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (cap != cudaStreamCaptureStatusNone) return nullptr;
+    auto it = ds->ticket_slot.find(stream);
+    if (it == ds->ticket_slot.end()) {
+        if (int(ds->ticket_slot.size()) >= kTicketStreams) return nullptr;
+        it = ds->ticket_slot.emplace(stream, int(ds->ticket_slot.size())).first;
+    }
+    return ds->d_tickets + 2 * it->second;
 }
 
 int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
@@ -272,6 +286,7 @@ void release_all() {
             if (pk.second.d_cta_begin) cudaFree(pk.second.d_cta_begin);
         }
         if (ds.d_status) cudaFree(ds.d_status);
+        if (ds.d_tickets) cudaFree(ds.d_tickets);
         if (ds.d_partial) cudaFree(ds.d_partial);
         if (ds.d_a) cudaFree(ds.d_a);
         if (ds.d_c) cudaFree(ds.d_c);

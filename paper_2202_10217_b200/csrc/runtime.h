@@ -37,6 +37,10 @@ struct DeviceState {
     int sm_count = 0;
     int cc_major = 0;
     int* d_status = nullptr;
+    // FP64 persistent launches: a pair of tickets per stream (launches on one stream run one
+    // after another, so they can share a pair; launches on different streams cannot).
+    int* d_tickets = nullptr;
+    std::map<cudaStream_t, int> ticket_slot;
     float* d_partial = nullptr;  // K-split workspace
     size_t partial_bytes = 0;
     // staging for the host-buffer entry point (grow-only)
@@ -53,7 +57,13 @@ struct Runtime {
     std::map<int, DeviceState> devices;
     int schedule = 0;
     int split_k = 0;
+    int f64_launch = 0;
 };
+constexpr int kTicketStreams = 256;
+
+// The ticket pair of `stream` on this device, or null when the persistent form must not be used
+// (all pairs taken, or the stream is being captured into a graph, whose replays may overlap).
+int* tickets_for_stream(DeviceState* ds, cudaStream_t stream);
 Runtime& runtime();
 
 // Current device's state, created on first use.  Returns a SYRK_* code.
@@ -80,8 +90,9 @@ int encode_tensor_map_f64_plain(CUtensorMap* tm, const void* p, int64_t rows, in
                                 int box_rows, int box_cols);
 
 // The device path of syrk_lower (arguments already validated; the caller holds the runtime lock).
+// `f64_launch` >= 0 overrides the process-wide FP64 launch form for this call.
 int syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
-                    double beta, int dtype, cudaStream_t stream);
+                    double beta, int dtype, cudaStream_t stream, int f64_launch = -1);
 
 void release_cholesky_workspaces();
 

@@ -1,10 +1,10 @@
-// FP64 triangle-block SYRK kernel for sm_100a.
+// FP64 triangle-block SYRK kernels for sm_100a.
 //
-// One thread block per work item of the tiled TBS schedule (Algorithm 4 and
-// Section 5.1.4 of the paper).  An item names up to 8 row segments of A (32 rows
-// each) and up to 16 output tiles C[seg x, seg y]; for a triangle block the tiles
-// are all pairs among k = 6 segments, so the block streams 6 segments per K-step
-// where a square block of the same accumulator count streams 8.
+// Work items of the tiled TBS schedule (Algorithm 4 and Section 5.1.4 of the paper) are run
+// by thread blocks of 16 MMA warps and one producer warp.  An item names up to 8 row
+// segments of A (32 rows each) and up to 16 output tiles C[seg x, seg y]; for a triangle
+// block the tiles are all pairs among k = 6 segments, so the block streams 6 segments per
+// K-step where a square block of the same accumulator count streams 8.
 //
 //   producer warp : plain TMA tile loads (no multicast) of the item's segments,
 //                   16 columns of A per stage, into a 6-stage shared-memory ring
@@ -21,6 +21,13 @@
 //                   the producer also TMA-loads the item's old C tiles (those below the
 //                   diagonal) into the ring's stages as the last K-steps release them, so
 //                   the epilogue reads them from shared memory instead of waiting on HBM.
+//
+// Two launch forms share this code.  One block per item (the hardware block scheduler hands
+// out the items; used for short lists and for the two-operand mode), and a persistent form,
+// one block per SM, whose producer draws the next item from a global counter and publishes
+// it to the MMA warps through a small ring in shared memory: the ring of stages then runs on
+// across items and the next item's first stages are in flight while the current one is
+// finished and written out.
 //
 // Accumulators (the C block) stay on chip for the whole M loop and each entry of
 // C is read (beta != 0) and written exactly once, as in the paper's generic
@@ -39,8 +46,9 @@ constexpr int kSegBytes = kTile * kBK * 8;      // 4096
 constexpr int kStageBytes = kMaxSeg * kSegBytes;
 constexpr int kMmaWarps = 16;
 constexpr int kThreads = (kMmaWarps + 1) * 32;  // + producer warp
-constexpr int kCTileBytes = kTile * kTile * 8;   // one old C tile in a ring stage (4 per stage)
+constexpr int kCTileBytes = kTile * kTile * 8;  // one old C tile in a ring stage (4 per stage)
 constexpr int kSmemBytes = kStages * kStageBytes + 2 * kStages * 8 + 1024;
+constexpr int kItemRing = 16;                   // published items in flight (persistent form)
 
 __device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
@@ -48,25 +56,154 @@ __device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
                  : "d"(a), "d"(b));
 }
 
+// What every role of a block needs to know about the call.
+struct Call {
+    uint8_t* smem;                 // the ring of stages
+    uint32_t smem32, bars32;       // shared-space addresses of the ring and of full_bar[0] (MMA warps use these)
+    uint64_t* full_bar;
+    uint64_t* empty_bar;           // 16 arrivals (one per MMA warp) free a stage
+    volatile int* abort_flag;
+    int* status;
+    const CUtensorMap* tmA;        // row segments
+    const CUtensorMap* tmB;        // column segments of the two-operand mode (else == tmA)
+    const CUtensorMap* tmC;        // old C tiles (c_tma)
+    int64_t N, ncols;
+    int32_t n_ksteps;
+    double* C;
+    int64_t ldc;
+    double alpha, beta;
+    int vec_ok, c_tma;
+    bool gemm;
+};
+
+// Ring steps of one item: its K-steps, then (c_tma) one step per group of four tiles of old C.
+__device__ __forceinline__ int c_steps_of(const Call& k, int n_tile) { return k.c_tma ? (n_tile + 3) / 4 : 0; }
+
+// ---------------------------------------------------------------------------------------------
+// Producer (one thread): fetch one item's ring steps, starting at global step g.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, uint32_t& g) {
+    const int n_seg = it.n_seg, n_tile = it.n_tile;
+    for (int ks = 0; ks < k.n_ksteps; ++ks, ++g) {
+        const uint32_t st = g % kStages;
+        if (g >= kStages && !mbar_wait_bounded(&k.empty_bar[st], ((g / kStages) - 1) & 1, k.abort_flag)) {
+            *k.abort_flag = 1; atomicOr(k.status, kStatusWaitEmpty); return false;
+        }
+        mbar_arrive_expect_tx(&k.full_bar[st], uint32_t(n_seg) * kSegBytes);
+        uint8_t* dst = k.smem + st * kStageBytes;
+        for (int s = 0; s < n_seg; ++s)
+            tma_load_2d(dst + s * kSegBytes, (k.gemm && s < it.pad) ? k.tmB : k.tmA, ks * kBK, it.seg[s] * kTile,
+                        &k.full_bar[st]);
+    }
+    // Old C: ring step j carries tiles 4j .. 4j+3 (8 KB each, row pitch 256 B), those below the diagonal.
+    const int n_c = c_steps_of(k, n_tile);
+    for (int j = 0; j < n_c; ++j, ++g) {
+        const uint32_t st = g % kStages;
+        if (g >= kStages && !mbar_wait_bounded(&k.empty_bar[st], ((g / kStages) - 1) & 1, k.abort_flag)) {
+            *k.abort_flag = 1; atomicOr(k.status, kStatusWaitEmpty); return false;
+        }
+        int below = 0;
+        for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt)
+            below += (k.gemm || it.seg[it.tile_x[tt]] != it.seg[it.tile_y[tt]]) ? 1 : 0;
+        if (below == 0) { mbar_arrive(&k.full_bar[st]); continue; }
+        mbar_arrive_expect_tx(&k.full_bar[st], uint32_t(below) * kCTileBytes);
+        uint8_t* dst = k.smem + st * kStageBytes;
+        for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt) {
+            const int rx = it.seg[it.tile_x[tt]], cy = it.seg[it.tile_y[tt]];
+            if (k.gemm || rx != cy) tma_load_2d(dst + (tt & 3) * kCTileBytes, k.tmC, cy * kTile, rx * kTile, &k.full_bar[st]);
+        }
+    }
+    return true;
+}
+
+// After a give-up: let the copies still in flight land before the block exits.
+__device__ void drain_producer(const Call& k, uint32_t g) {
+    for (uint32_t i = (g > kStages ? g - kStages : 0); i < g; ++i) {
+        volatile int dummy = 0;
+        mbar_wait_bounded(&k.full_bar[i % kStages], (i / kStages) & 1, &dummy);
+    }
+}
+
+// Checks an item before any role uses it and, outside the two-operand mode, records in `pad`
+// whether it is a triangle block in the generator's tile order (x = 1..5, y < x): for those
+// the 16th MMA warp takes the last 8 x 8 block of every tile.  (One thread decides this once per
+// item; the MMA warps only read the flag.)
+__device__ bool prepare_item(const Call& k, WorkItem& it) {
+    bool ok = it.n_seg >= 1 && it.n_seg <= kMaxSeg && it.n_tile >= 1 && it.n_tile <= kMmaWarps;
+    for (int s = 0; ok && s < it.n_seg; ++s)
+        ok = it.seg[s] >= 0 && int64_t(it.seg[s]) * kTile < ((k.gemm && s < it.pad) ? k.ncols : k.N);
+    for (int t = 0; ok && t < it.n_tile; ++t) ok = it.tile_x[t] < it.n_seg && it.tile_y[t] < it.n_seg;
+    if (ok && !k.gemm) {
+        bool tri = it.kind == kTri && it.n_seg == 6 && it.n_tile == 15;
+        for (int x = 1, q = 0; tri && x < 6; ++x)
+            for (int y = 0; y < x; ++y, ++q) tri = tri && it.tile_x[q] == x && it.tile_y[q] == y;
+        it.pad = tri ? 1 : 0;
+    }
+    return ok;
+}
+
+// ---------------------------------------------------------------------------------------------
+// MMA warps
+// ---------------------------------------------------------------------------------------------
+// The MMA warps address shared memory by 32-bit shared-space addresses: fewer registers held
+// across the M loop than with generic pointers.
+__device__ __forceinline__ double lds_f64(uint32_t addr) {
+    double v;
+    asm volatile("ld.shared.f64 %0, [%1];" : "=d"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ bool try_wait32(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool wait_full_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int lane) {
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (!try_wait32(bar, parity)) {
+        if ((++spins & 0x3FFu) == 0 && (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs)) {
+            *abort_flag = 1;
+            if (lane == 0) atomicOr(status, kStatusWaitFull);
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ bool wait_full_at(const Call& k, uint32_t st, uint32_t parity, int lane) {
+    const uint32_t bar = k.bars32 + st * 8;
+    if (try_wait32(bar, parity)) return true;
+    return wait_full_slow(bar, parity, k.abort_flag, k.status, lane);
+}
+__device__ __forceinline__ void release_at(const Call& k, uint32_t st, int lane) {
+    __syncwarp();
+    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(k.bars32 + (kStages + st) * 8) : "memory");
+}
+__device__ __forceinline__ bool wait_full(const Call& k, uint32_t g, int lane) {
+    return wait_full_at(k, g % kStages, (g / kStages) & 1, lane);
+}
+__device__ __forceinline__ void release(const Call& k, uint32_t g, int lane) { release_at(k, g % kStages, lane); }
+
 // The M loop of one warp's tile.  kSkipLast leaves out block (3, 3), which the 16th warp of
 // a triangle block computes.  Returns false when a bounded wait ran out.
 template <bool kSkipLast>
-__device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const uint8_t* smem, uint32_t xbase,
-                                              uint32_t ybase, const uint32_t (&off)[4], int n_ksteps,
-                                              uint64_t* full_bar, uint64_t* empty_bar, volatile int* abort_flag,
-                                              int lane) {
-    for (int ks = 0; ks < n_ksteps; ++ks) {
-        const int st = ks % kStages;
-        if (!mbar_wait_bounded(&full_bar[st], (ks / kStages) & 1, abort_flag)) return false;
-        const uint8_t* px = smem + st * kStageBytes + xbase;
-        const uint8_t* py = smem + st * kStageBytes + ybase;
+__device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const Call& k, uint32_t xbase, uint32_t ybase,
+                                              uint32_t off0, uint32_t g0, int lane) {
+    uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;      // stage and phase, advanced step by step
+    for (int ks = 0; ks < k.n_ksteps; ++ks) {
+        if (!wait_full_at(k, st, parity, lane)) return false;
+        const uint32_t stage = k.smem32 + st * kStageBytes;
+        const uint32_t px = (stage + xbase) | off0, py = (stage + ybase) | off0;   // 1024-aligned | offset < 1024
 #pragma unroll
         for (int sl = 0; sl < 4; ++sl) {
             double a[4], b[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                a[j] = *reinterpret_cast<const double*>(px + off[sl] + j * 1024);
-                b[j] = *reinterpret_cast<const double*>(py + off[sl] + j * 1024);
+                a[j] = lds_f64((px ^ (sl << 4)) + j * 1024);
+                b[j] = lds_f64((py ^ (sl << 4)) + j * 1024);
             }
 #pragma unroll
             for (int mi = 0; mi < 4; ++mi)
@@ -74,12 +211,161 @@ __device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const uint
                 for (int ni = 0; ni < 4; ++ni)
                     if (!(kSkipLast && mi == 3 && ni == 3)) dmma884(acc[mi][ni], a[mi], b[ni]);
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[st]);
+        release_at(k, st, lane);
+        if (++st == kStages) { st = 0; parity ^= 1; }
     }
     return true;
 }
 
+
+__device__ __forceinline__ uint32_t fragment_offset(int lane) {
+    // Lane (g, t) of an m8n8k4 fragment holds (row g, k = t).  The four k-slices of a stage take
+    // k = 8*(t>>1) + 2*sl + (t&1): any assignment of the stage's 16 columns to (slice, t) is valid as
+    // long as both operands use the same one, and this one makes every half-warp's 16 loads hit 16
+    // different 8-byte bank pairs under the 128-byte swizzle (16-byte chunk index ^ row % 8).
+    // Byte offset of slice sl within a 1024-byte group of 8 rows:
+    //   g*128 + ((((t>>1)<<2 | sl) ^ g) << 4) + ((t&1) << 3)  ==  (slice 0's offset) ^ (sl << 4).
+    const int g = lane >> 2, t = lane & 3;
+    return uint32_t(g * 128 + ((((t >> 1) << 2) ^ g) << 4) + ((t & 1) << 3));
+}
+
+// 16th warp of a triangle block: the 15 left-out 8 x 8 blocks.  g0 = the item's first ring step,
+// n_c = its old-C steps.
+__device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, int lane) {
+    const int gq = lane >> 2, t = lane & 3;
+    const uint32_t gc = g0 + uint32_t(k.n_ksteps);
+    const bool use_beta = (k.beta != 0.0);
+    const uint32_t off0 = fragment_offset(lane);
+    int32_t seg[6];
+#pragma unroll
+    for (int s = 0; s < 6; ++s) seg[s] = it.seg[s];
+    double sacc[15][2];
+#pragma unroll
+    for (int q = 0; q < 15; ++q) sacc[q][0] = sacc[q][1] = 0.0;
+    uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;
+    for (int ks = 0; ks < k.n_ksteps; ++ks) {
+        if (!wait_full_at(k, st, parity, lane)) return false;
+        const uint32_t base = (k.smem32 + st * kStageBytes + 3 * 1024) | off0;   // rows 24..31 of every segment
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl) {
+            double f[6];
+#pragma unroll
+            for (int j = 0; j < 6; ++j) f[j] = lds_f64((base ^ (sl << 4)) + j * kSegBytes);
+            int q = 0;
+#pragma unroll
+            for (int x = 1; x < 6; ++x)
+#pragma unroll
+                for (int y = 0; y < x; ++y, ++q) dmma884(sacc[q], f[x], f[y]);
+        }
+        release_at(k, st, lane);
+        if (++st == kStages) { st = 0; parity ^= 1; }
+    }
+    for (int j = 0; j < n_c; ++j)
+        if (!wait_full(k, gc + j, lane)) return false;
+    int q = 0;
+#pragma unroll
+    for (int x = 1; x < 6; ++x)
+#pragma unroll
+        for (int y = 0; y < x; ++y, ++q) {
+            const int64_t r = int64_t(seg[x]) * kTile + 24 + gq;
+            const int64_t c = int64_t(seg[y]) * kTile + 24 + 2 * t;
+            if (r >= k.N) continue;                                 // tile below the diagonal: c + 1 < r
+            double* p = k.C + r * k.ldc + c;
+            double v0 = k.alpha * sacc[q][0], v1 = k.alpha * sacc[q][1];
+            if (n_c > 0) {
+                const double2 o = *reinterpret_cast<const double2*>(
+                    k.smem + ((gc + (q >> 2)) % kStages) * kStageBytes + (q & 3) * kCTileBytes +
+                    (24 + gq) * (kTile * 8) + (24 + 2 * t) * 8);
+                v0 += k.beta * o.x; v1 += k.beta * o.y;
+            } else if (use_beta) { v0 += k.beta * p[0]; v1 += k.beta * p[1]; }
+            if (k.vec_ok) *reinterpret_cast<double2*>(p) = make_double2(v0, v1);
+            else { p[0] = v0; p[1] = v1; }
+        }
+    for (int j = 0; j < n_c; ++j) release(k, gc + j, lane);
+    return true;
+}
+
+// A warp with a tile (tile number `warp` of the item).  `scavenge`: block (3, 3) is left to the 16th warp.
+__device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, bool scavenge,
+                                          int warp, int lane) {
+    const int gq = lane >> 2, t = lane & 3;
+    const uint32_t gc = g0 + uint32_t(k.n_ksteps);
+    const bool use_beta = (k.beta != 0.0);
+    const uint32_t off0 = fragment_offset(lane);
+    const int sx = it.tile_x[warp], sy = it.tile_y[warp];
+    const int64_t row0 = int64_t(it.seg[sx]) * kTile, col0 = int64_t(it.seg[sy]) * kTile;
+    const uint32_t xbase = uint32_t(sx) * kSegBytes, ybase = uint32_t(sy) * kSegBytes;
+
+    double acc[4][4][2];
+#pragma unroll
+    for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) acc[mi][ni][0] = acc[mi][ni][1] = 0.0;
+
+    const bool alive = scavenge ? tile_mainloop<true>(acc, k, xbase, ybase, off0, g0, lane)
+                                : tile_mainloop<false>(acc, k, xbase, ybase, off0, g0, lane);
+    if (!alive) return false;
+
+    for (int j = 0; j < n_c; ++j)
+        if (!wait_full(k, gc + j, lane)) return false;
+    const uint8_t* old_tile = nullptr;                  // this warp's old C tile in shared memory
+    if (n_c > 0 && (k.gemm || row0 != col0))
+        old_tile = k.smem + ((gc + (warp >> 2)) % kStages) * kStageBytes + (warp & 3) * kCTileBytes;
+#pragma unroll
+    for (int mi = 0; mi < 4; ++mi) {
+        const int64_t r = row0 + mi * 8 + gq;
+        if (r >= k.N) continue;
+        const int64_t cmax = k.gemm ? k.ncols - 1 : r;  // last column this row may touch
+        double* crow = k.C + r * k.ldc;
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) {
+            if (scavenge && mi == 3 && ni == 3) continue;             // written by the 16th warp
+            const int64_t c = col0 + ni * 8 + 2 * t;
+            if (c > cmax) continue;
+            const bool both = (c + 1 <= cmax);
+            double v0 = k.alpha * acc[mi][ni][0], v1 = k.alpha * acc[mi][ni][1];
+            if (use_beta) {
+                double2 o = make_double2(0.0, 0.0);
+                if (old_tile) o = *reinterpret_cast<const double2*>(old_tile + (mi * 8 + gq) * (kTile * 8) + (ni * 8 + 2 * t) * 8);
+                else if (both && k.vec_ok) o = *reinterpret_cast<const double2*>(crow + c);
+                else { o.x = crow[c]; if (both) o.y = crow[c + 1]; }
+                v0 += k.beta * o.x; v1 += k.beta * o.y;
+            }
+            if (both) {
+                if (k.vec_ok) *reinterpret_cast<double2*>(crow + c) = make_double2(v0, v1);
+                else { crow[c] = v0; crow[c + 1] = v1; }
+            } else {
+                crow[c] = v0;
+            }
+        }
+    }
+    for (int j = 0; j < n_c; ++j) release(k, gc + j, lane);
+    return true;
+}
+
+// One MMA warp's share of one item: its ring steps from global step g on, then its write-out.
+// Every warp waits for and releases every ring step of the item, with or without work in it.
+__device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it, uint32_t& g, int warp, int lane) {
+    const int n_tile = it.n_tile;
+    const int n_c = c_steps_of(k, n_tile);
+    const uint32_t g0 = g;
+    g += uint32_t(k.n_ksteps + n_c);
+    const bool scavenge = !k.gemm && it.pad != 0;      // set by prepare_item
+    if (scavenge && warp == kMmaWarps - 1) return scavenger_role(k, it, g0, n_c, lane);
+    if (warp < n_tile) return tile_role(k, it, g0, n_c, scavenge, warp, lane);
+    for (uint32_t s = g0; s < g; ++s) {                 // no tile in this item: keep the ring moving
+        if (!wait_full(k, s, lane)) return false;
+        release(k, s, lane);
+    }
+    return true;
+}
+
+// ---------------------------------------------------------------------------------------------
+// One block per item.  Two-operand mode (gemm_col_tiles > 0): D = alpha * P * Q^T + beta * D
+// without a triangle mask; block b owns the 4 x 4 tile rectangle (b / column groups, b % column
+// groups), its column segments come from Q (tmB, the first `pad` segments), its row segments
+// from P (tmA).
+// ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
@@ -87,19 +373,21 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     int64_t ldc, double alpha, double beta, int vec_ok, int c_tma, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
-    uint64_t* empty_bar = full_bar + kStages;
     __shared__ WorkItem s_item;
     __shared__ volatile int s_abort;
-    __shared__ int s_scavenge;
-
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // Two-operand mode (gemm_col_tiles > 0): D = alpha * P * Q^T + beta * D without a triangle
-    // mask; block b owns the 4 x 4 tile rectangle (b / column groups, b % column groups), its
-    // column segments come from Q (tmB, the first `pad` segments), its row segments from P (tmA).
-    const bool gemm = gemm_col_tiles > 0;
-    if (gemm) {
+    Call k;
+    k.smem = smem;
+    k.full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+    k.empty_bar = k.full_bar + kStages;
+    k.smem32 = smem_u32(smem); k.bars32 = smem_u32(k.full_bar);
+    k.abort_flag = &s_abort; k.status = status;
+    k.tmA = &tmA; k.tmB = &tmB; k.tmC = &tmC;
+    k.N = N; k.ncols = ncols; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
+    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = gemm_col_tiles > 0;
+
+    if (k.gemm) {
         if (tid == 0) {
             const int n_cg = (gemm_col_tiles + 3) / 4;
             const int64_t row_tiles = (N + kTile - 1) / kTile;
@@ -118,209 +406,111 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     if (tid == 0) s_abort = 0;
     __syncthreads();
-
-    const int n_seg = s_item.n_seg, n_tile = s_item.n_tile;
     if (tid == 0) {
-        bool ok = n_seg >= 1 && n_seg <= kMaxSeg && n_tile >= 1 && n_tile <= kMmaWarps;
-        for (int s = 0; ok && s < n_seg; ++s)
-            ok = s_item.seg[s] >= 0 && int64_t(s_item.seg[s]) * kTile < ((gemm && s < s_item.pad) ? ncols : N);
-        for (int t = 0; ok && t < n_tile; ++t)
-            ok = s_item.tile_x[t] < n_seg && s_item.tile_y[t] < n_seg;
-        // A triangle block in the generator's tile order (x = 1..5, y < x): the 16th warp helps.
-        bool tri = ok && s_item.kind == kTri && n_seg == 6 && n_tile == 15;
-        for (int x = 1, t = 0; tri && x < 6; ++x)
-            for (int y = 0; y < x; ++y, ++t) tri = tri && s_item.tile_x[t] == x && s_item.tile_y[t] == y;
-        s_scavenge = tri ? 1 : 0;
-        if (!ok) { s_abort = 1; atomicOr(status, kStatusBadItem); }
+        if (!prepare_item(k, s_item)) { s_abort = 1; atomicOr(status, kStatusBadItem); }
         else {
-            for (int s = 0; s < kStages; ++s) {
-                mbar_init(&full_bar[s], 1);
-                mbar_init(&empty_bar[s], tri ? kMmaWarps : n_tile);
-            }
+            for (int s = 0; s < kStages; ++s) { mbar_init(&k.full_bar[s], 1); mbar_init(&k.empty_bar[s], kMmaWarps); }
             mbar_fence_init();
         }
     }
     __syncthreads();
     if (s_abort) return;
 
+    uint32_t g = 0;
     if (warp == kMmaWarps) {
-        // ------------------------------ producer ------------------------------
         if (lane == 0) {
             prefetch_tensormap(&tmA);
-            int issued = 0;
-            for (int ks = 0; ks < n_ksteps; ++ks) {
-                const int st = ks % kStages;
-                if (ks >= kStages &&
-                    !mbar_wait_bounded(&empty_bar[st], ((ks / kStages) - 1) & 1, &s_abort)) {
-                    s_abort = 1; atomicOr(status, kStatusWaitEmpty); break;
-                }
-                mbar_arrive_expect_tx(&full_bar[st], uint32_t(n_seg) * kSegBytes);
-                uint8_t* dst = smem + st * kStageBytes;
-                for (int s = 0; s < n_seg; ++s)
-                    tma_load_2d(dst + s * kSegBytes, (gemm && s < s_item.pad) ? &tmB : &tmA, ks * kBK,
-                                s_item.seg[s] * kTile, &full_bar[st]);
-                issued = ks + 1;
-            }
-            if (c_tma && !s_abort) {
-                // Old C: ring step n_ksteps + j carries tiles 4j .. 4j+3 (8 KB each, row pitch 256 B).
-                prefetch_tensormap(&tmC);
-                for (int j = 0; 4 * j < n_tile; ++j) {
-                    const int q = n_ksteps + j, st = q % kStages;
-                    if (q >= kStages && !mbar_wait_bounded(&empty_bar[st], ((q / kStages) - 1) & 1, &s_abort)) {
-                        s_abort = 1; atomicOr(status, kStatusWaitEmpty); break;
-                    }
-                    int below = 0;
-                    for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt)
-                        below += (gemm || s_item.seg[s_item.tile_x[tt]] != s_item.seg[s_item.tile_y[tt]]) ? 1 : 0;
-                    if (below == 0) { mbar_arrive(&full_bar[st]); continue; }
-                    mbar_arrive_expect_tx(&full_bar[st], uint32_t(below) * kCTileBytes);
-                    uint8_t* dst = smem + st * kStageBytes;
-                    for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt) {
-                        const int rx = s_item.seg[s_item.tile_x[tt]], cy = s_item.seg[s_item.tile_y[tt]];
-                        if (gemm || rx != cy) tma_load_2d(dst + (tt & 3) * kCTileBytes, &tmC, cy * kTile, rx * kTile, &full_bar[st]);
-                    }
-                    issued = q + 1;
-                }
-            }
-            if (s_abort) {
-                // Winding down: let the copies still in flight land before the block exits.
-                for (int ks = (issued > kStages ? issued - kStages : 0); ks < issued; ++ks) {
-                    volatile int dummy = 0;
-                    mbar_wait_bounded(&full_bar[ks % kStages], (ks / kStages) & 1, &dummy);
-                }
-            }
+            if (c_tma) prefetch_tensormap(&tmC);
+            produce_item(k, s_item, g);
+            if (s_abort) drain_producer(k, g);
         }
         return;
     }
-    const bool scavenge = s_scavenge != 0;
-    if (warp >= n_tile && !scavenge) return;
+    mma_warp_item(k, s_item, g, warp, lane);
+}
 
-    // ------------------------------ MMA warps ------------------------------
-    // Fragment addressing.  Lane (g, t) of an m8n8k4 fragment holds (row g, k = t).  The four
-    // k-slices of a stage take k = 8*(t>>1) + 2*sl + (t&1): any assignment of the stage's 16
-    // columns to (slice, t) is valid as long as both operands use the same one, and this one
-    // makes every half-warp's 16 loads hit 16 different 8-byte bank pairs under the 128-byte
-    // swizzle (16-byte chunk index ^ row % 8).
-    const int g = lane >> 2, t = lane & 3;
-    uint32_t off[4];
-#pragma unroll
-    for (int sl = 0; sl < 4; ++sl)
-        off[sl] = uint32_t(g * 128 + ((((t >> 1) << 2 | sl) ^ g) << 4) + ((t & 1) << 3));
-    const bool use_beta = (beta != 0.0);
+// ---------------------------------------------------------------------------------------------
+// Persistent form: one block per SM; the producer draws items from counter[0] (zero at launch;
+// counter[1] counts the producers that are done) and publishes them through a ring of kItemRing
+// slots.  The producer is never more than
+// kStages ring steps - hence fewer than kItemRing items - ahead of the slowest MMA warp, so a
+// slot is rewritten only after every warp has read it.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
+                               const WorkItem* __restrict__ items, int64_t n_items, int* __restrict__ counter,
+                               int64_t N, int32_t n_ksteps, double* __restrict__ C, int64_t ldc, double alpha,
+                               double beta, int vec_ok, int c_tma, int* __restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ WorkItem s_ring[kItemRing];
+    __shared__ uint64_t s_item_bar[kItemRing];
+    __shared__ volatile int s_abort;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    if (scavenge && warp == kMmaWarps - 1) {
-        // ------------- 16th warp of a triangle block: the 15 left-out 8 x 8 blocks -------------
-        double sacc[15][2];
-#pragma unroll
-        for (int q = 0; q < 15; ++q) sacc[q][0] = sacc[q][1] = 0.0;
-        for (int ks = 0; ks < n_ksteps; ++ks) {
-            const int st = ks % kStages;
-            if (!mbar_wait_bounded(&full_bar[st], (ks / kStages) & 1, &s_abort)) {
-                s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return;
-            }
-            const uint8_t* base = smem + st * kStageBytes + 3 * 1024;      // rows 24..31 of every segment
-#pragma unroll
-            for (int sl = 0; sl < 4; ++sl) {
-                double f[6];
-#pragma unroll
-                for (int s = 0; s < 6; ++s) f[s] = *reinterpret_cast<const double*>(base + s * kSegBytes + off[sl]);
-                int q = 0;
-#pragma unroll
-                for (int x = 1; x < 6; ++x)
-#pragma unroll
-                    for (int y = 0; y < x; ++y, ++q) dmma884(sacc[q], f[x], f[y]);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[st]);
-        }
-        if (c_tma) {                                                    // all four old-C ring steps
-            for (int j = 0; j < 4; ++j) {
-                const int qs = n_ksteps + j;
-                if (!mbar_wait_bounded(&full_bar[qs % kStages], (qs / kStages) & 1, &s_abort)) {
-                    s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return;
+    Call k;
+    k.smem = smem;
+    k.full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+    k.empty_bar = k.full_bar + kStages;
+    k.smem32 = smem_u32(smem); k.bars32 = smem_u32(k.full_bar);
+    k.abort_flag = &s_abort; k.status = status;
+    k.tmA = &tmA; k.tmB = &tmA; k.tmC = &tmC;
+    k.N = N; k.ncols = N; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
+    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false;
+
+    if (tid == 0) {
+        s_abort = 0;
+        for (int s = 0; s < kStages; ++s) { mbar_init(&k.full_bar[s], 1); mbar_init(&k.empty_bar[s], kMmaWarps); }
+        for (int s = 0; s < kItemRing; ++s) mbar_init(&s_item_bar[s], 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    uint32_t g = 0;
+    if (warp == kMmaWarps) {
+        if (lane == 0) {
+            prefetch_tensormap(&tmA);
+            if (c_tma) prefetch_tensormap(&tmC);
+            for (uint32_t slot = 0;; ++slot) {
+                WorkItem& dst = s_ring[slot % kItemRing];
+                const int64_t idx = s_abort ? n_items : int64_t(atomicAdd(counter, 1));
+                bool last = idx >= n_items;
+                if (!last) {
+                    for (int w = 0; w < int(sizeof(WorkItem) / 4); ++w)
+                        reinterpret_cast<int32_t*>(&dst)[w] = reinterpret_cast<const int32_t*>(&items[idx])[w];
+                    if (!prepare_item(k, dst)) { s_abort = 1; atomicOr(status, kStatusBadItem); last = true; }
+                }
+                if (last) dst.n_tile = -1;                        // end marker
+                mbar_arrive(&s_item_bar[slot % kItemRing]);       // publishes the slot (release)
+                if (last) break;
+                if (!produce_item(k, dst, g)) {                   // gave up: tell the MMA warps to stop as well
+                    WorkItem& end = s_ring[(slot + 1) % kItemRing];
+                    end.n_tile = -1;
+                    mbar_arrive(&s_item_bar[(slot + 1) % kItemRing]);
+                    break;
                 }
             }
+            if (s_abort) drain_producer(k, g);
+            // The last producer to get here puts both tickets back to zero for the next launch
+            // on this stream: by then no block draws any more.
+            if (atomicAdd(counter + 1, 1) == int(gridDim.x) - 1) { atomicExch(counter, 0); atomicExch(counter + 1, 0); }
         }
-        int q = 0;
-#pragma unroll
-        for (int x = 1; x < 6; ++x)
-#pragma unroll
-            for (int y = 0; y < x; ++y, ++q) {
-                const int64_t r = int64_t(s_item.seg[x]) * kTile + 24 + g;
-                const int64_t c = int64_t(s_item.seg[y]) * kTile + 24 + 2 * t;
-                if (r >= N) continue;                                   // tile below the diagonal: c + 1 < r
-                double* p = C + r * ldc + c;
-                double v0 = alpha * sacc[q][0], v1 = alpha * sacc[q][1];
-                if (c_tma) {
-                    const double2 o = *reinterpret_cast<const double2*>(
-                        smem + ((n_ksteps + (q >> 2)) % kStages) * kStageBytes + (q & 3) * kCTileBytes +
-                        (24 + g) * (kTile * 8) + (24 + 2 * t) * 8);
-                    v0 += beta * o.x; v1 += beta * o.y;
-                } else if (use_beta) { v0 += beta * p[0]; v1 += beta * p[1]; }
-                if (vec_ok) *reinterpret_cast<double2*>(p) = make_double2(v0, v1);
-                else { p[0] = v0; p[1] = v1; }
-            }
         return;
     }
-
-    const int sx = s_item.tile_x[warp], sy = s_item.tile_y[warp];
-    const uint32_t xbase = uint32_t(sx) * kSegBytes, ybase = uint32_t(sy) * kSegBytes;
-
-    double acc[4][4][2];
-#pragma unroll
-    for (int mi = 0; mi < 4; ++mi)
-#pragma unroll
-        for (int ni = 0; ni < 4; ++ni) acc[mi][ni][0] = acc[mi][ni][1] = 0.0;
-
-    const bool alive = scavenge
-        ? tile_mainloop<true>(acc, smem, xbase, ybase, off, n_ksteps, full_bar, empty_bar, &s_abort, lane)
-        : tile_mainloop<false>(acc, smem, xbase, ybase, off, n_ksteps, full_bar, empty_bar, &s_abort, lane);
-    if (!alive) { s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return; }
-
-    // ------------------------------ epilogue ------------------------------
-    const int64_t row0 = int64_t(s_item.seg[sx]) * kTile, col0 = int64_t(s_item.seg[sy]) * kTile;
-    const uint8_t* old_tile = nullptr;                  // this warp's old C tile in shared memory
-    if (c_tma && (gemm || row0 != col0)) {
-        const int qs = n_ksteps + (warp >> 2);
-        if (!mbar_wait_bounded(&full_bar[qs % kStages], (qs / kStages) & 1, &s_abort)) {
+    for (uint32_t slot = 0;; ++slot) {
+        if (!mbar_wait_bounded(&s_item_bar[slot % kItemRing], (slot / kItemRing) & 1, &s_abort)) {
             s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return;
         }
-        old_tile = smem + (qs % kStages) * kStageBytes + (warp & 3) * kCTileBytes;
-    }
-#pragma unroll
-    for (int mi = 0; mi < 4; ++mi) {
-        const int64_t r = row0 + mi * 8 + g;
-        if (r >= N) continue;
-        const int64_t cmax = gemm ? ncols - 1 : r;      // last column this row may touch
-        double* crow = C + r * ldc;
-#pragma unroll
-        for (int ni = 0; ni < 4; ++ni) {
-            if (scavenge && mi == 3 && ni == 3) continue;             // written by the 16th warp
-            const int64_t c = col0 + ni * 8 + 2 * t;
-            if (c > cmax) continue;
-            const bool both = (c + 1 <= cmax);
-            double v0 = alpha * acc[mi][ni][0], v1 = alpha * acc[mi][ni][1];
-            if (use_beta) {
-                double2 o = make_double2(0.0, 0.0);
-                if (old_tile) o = *reinterpret_cast<const double2*>(old_tile + (mi * 8 + g) * (kTile * 8) + (ni * 8 + 2 * t) * 8);
-                else if (both && vec_ok) o = *reinterpret_cast<const double2*>(crow + c);
-                else { o.x = crow[c]; if (both) o.y = crow[c + 1]; }
-                v0 += beta * o.x; v1 += beta * o.y;
-            }
-            if (both) {
-                if (vec_ok) *reinterpret_cast<double2*>(crow + c) = make_double2(v0, v1);
-                else { crow[c] = v0; crow[c + 1] = v1; }
-            } else {
-                crow[c] = v0;
-            }
-        }
+        const WorkItem& it = s_ring[slot % kItemRing];
+        if (it.n_tile < 0) return;
+        if (!mma_warp_item(k, it, g, warp, lane)) return;
     }
 }
 
 }  // namespace f64
 
 namespace {
-cudaError_t configure_f64_kernel() {
+cudaError_t configure_f64_kernels() {
     // The shared-memory attribute belongs to a device's context: set it once per device.
     static bool configured[64] = {};
     int dev = 0;
@@ -330,6 +520,9 @@ cudaError_t configure_f64_kernel() {
         cudaError_t e = cudaFuncSetAttribute(f64::syrk_f64_tbs_kernel,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, f64::kSmemBytes);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(f64::syrk_f64_tbs_persistent_kernel,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, f64::kSmemBytes);
+        if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
     return cudaSuccess;
@@ -338,14 +531,21 @@ cudaError_t configure_f64_kernel() {
 
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
-                            double beta, int* d_status, cudaStream_t stream) {
-    cudaError_t e = configure_f64_kernel();
+                            double beta, int* d_tickets, int n_blocks, int* d_status, cudaStream_t stream) {
+    cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0) ? 1 : 0;
     const int32_t n_ksteps = int32_t((M + f64::kBK - 1) / f64::kBK);
     const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
     CUtensorMap none{};
+    if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
+        const int64_t blocks = n_items < n_blocks ? n_items : int64_t(n_blocks);
+        f64::syrk_f64_tbs_persistent_kernel<<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
+            tmA, c_tma ? *tmC : none, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma,
+            d_status);
+        return cudaGetLastError();
+    }
     f64::syrk_f64_tbs_kernel<<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
     return cudaGetLastError();
@@ -354,7 +554,7 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
 cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, const CUtensorMap* tmD,
                                int64_t nrows, int64_t ncols, int64_t K, double* D, int64_t ldd, double alpha,
                                double beta, int* d_status, cudaStream_t stream) {
-    cudaError_t e = configure_f64_kernel();
+    cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (nrows == 0 || ncols == 0) return cudaSuccess;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0 && (ldd & 1) == 0) ? 1 : 0;

@@ -188,3 +188,82 @@ def test_two_streams_back_to_back():
     il = np.tril_indices(N)
     for dC in outs:
         assert np.array_equal(dC.cpu().numpy()[il], ref[il])
+
+
+# ---- FP64 launch forms: one block per item / persistent blocks drawing items from a counter ----
+
+@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-1.0, 1.0)])
+def test_f64_launch_forms_agree_bit_for_bit(alpha, beta):
+    """Both forms run every tile with the same arithmetic in the same order: identical bits,
+    and both within tolerance of the reference.  Sizes span one item, a ragged edge, and a list
+    several times longer than the SM count."""
+    for n, (N, M) in enumerate([(33, 50), (1000, 70), (1300, 40), (2500, 33), (5000, 48)]):
+        A = make_A(N, M, B.DTYPE_F64, seed=300 + n)
+        Cin = I.random_c(N, 7, B.DTYPE_F64) if beta != 0.0 else None
+        outs = []
+        for mode in (B.F64_LAUNCH_PER_ITEM, B.F64_LAUNCH_PERSISTENT, B.F64_LAUNCH_AUTO):
+            try:
+                B.syrk_set_f64_launch(mode)
+                got, ref, bound = run_case(A, B.DTYPE_F64, alpha, beta, Cin)
+            finally:
+                B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+            assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin, B.DTYPE_F64)
+            outs.append(got)
+        il = np.tril_indices(N)
+        assert np.array_equal(outs[0][il], outs[1][il]) and np.array_equal(outs[0][il], outs[2][il])
+
+
+def test_f64_persistent_form_repeated_and_on_two_streams():
+    """The item counter is left at zero by every launch, and each stream has its own: repeated
+    calls on one stream and interleaved calls on two streams all give the reference result."""
+    import torch
+    N, M = 2100, 64
+    A = make_A(N, M, B.DTYPE_F64, seed=31, kind="int")
+    dA = torch.from_numpy(A).cuda()
+    ref, _ = O.syrk_lower(A, None, 1.0, 0.0, B.DTYPE_F64)
+    il = np.tril_indices(N)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = []
+    try:
+        B.syrk_set_f64_launch(B.F64_LAUNCH_PERSISTENT)
+        torch.cuda.synchronize()
+        for rep in range(3):
+            for s in streams:
+                dC = torch.zeros((N, N), dtype=torch.float64, device="cuda")
+                s.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(s):
+                    B.syrk_lower(N, M, dA, M, dC, N, 1.0, 0.0, B.DTYPE_F64, stream=s.cuda_stream)
+                outs.append(dC)
+        torch.cuda.synchronize()
+    finally:
+        B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+    assert B.syrk_last_status() == 0
+    for dC in outs:
+        assert np.array_equal(dC.cpu().numpy()[il], ref[il])
+
+
+def test_f64_call_inside_stream_capture_replays_correctly():
+    """During stream capture the library uses the one-block-per-item form (a captured graph may be
+    replayed on several streams at once); the replayed graph gives the reference result."""
+    import torch
+    N, M = 1500, 48
+    A = make_A(N, M, B.DTYPE_F64, seed=32, kind="int")
+    dA = torch.from_numpy(A).cuda()
+    dC = torch.zeros((N, N), dtype=torch.float64, device="cuda")
+    B.syrk_lower(N, M, dA, M, dC, N, 1.0, 0.0, B.DTYPE_F64)          # builds the cached work list first
+    torch.cuda.synchronize()
+    dC.zero_()
+    g = torch.cuda.CUDAGraph()
+    try:
+        B.syrk_set_f64_launch(B.F64_LAUNCH_PERSISTENT)
+        with torch.cuda.graph(g):
+            B.syrk_lower(N, M, dA, M, dC, N, 1.0, 1.0, B.DTYPE_F64,
+                         stream=torch.cuda.current_stream().cuda_stream)
+    finally:
+        B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+    g.replay(); g.replay()
+    torch.cuda.synchronize()
+    assert B.syrk_last_status() == 0
+    ref, _ = O.syrk_lower(A, None, 2.0, 0.0, B.DTYPE_F64)             # two accumulating replays
+    il = np.tril_indices(N)
+    assert np.array_equal(dC.cpu().numpy()[il], ref[il])
