@@ -204,8 +204,13 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
     B.syrk_plan_prepare(N, M, dtype)
     stats = B.syrk_get_schedule_stats(N, M, dtype)
     n_warm = args.warmup if args.kernel_only else max(args.warmup, 3)
+    if args.gram:                                          # same operand stored M x N: C = A^T A
+        dA = dA.t().contiguous()
+        device_call = lambda: B.syrk_lower_tn(N, M, dA, N, dC, N, wl.alpha, wl.beta, dtype)
+    else:
+        device_call = lambda: B.syrk_lower(N, M, dA, M, dC, N, wl.alpha, wl.beta, dtype)
     for _ in range(n_warm):
-        B.syrk_lower(N, M, dA, M, dC, N, wl.alpha, wl.beta, dtype)
+        device_call()
     torch.cuda.synchronize()
     assert B.syrk_last_status() == 0
 
@@ -216,7 +221,7 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
         for i in range(args.steps):
             flush.zero_()                                  # evict A and C from L2 (not timed)
             ev0[i].record()
-            B.syrk_lower(N, M, dA, M, dC, N, wl.alpha, wl.beta, dtype)
+            device_call()
             ev1[i].record()
         barrier()
     assert B.syrk_last_status() == 0
@@ -230,7 +235,8 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
                               "steps": args.steps, "ms_per_step": ms_per_step, "kernel_only": True,
-                              "config": {"workload": wl.name, "N": N, "M": M}}))
+                              "config": {"workload": wl.name, "N": N, "M": M,
+                                         "operand": "M x N (Gram form)" if args.gram else "N x M"}}))
         return
 
     # end to end: host buffers through the C ABI, copies inside the timed region
@@ -443,8 +449,12 @@ def main():
     ap.add_argument("--kernel-only", action="store_true",
                     help="device-timed kernel steps only (no end-to-end leg, CPU baseline or peak probe); "
                          "for short profiler runs")
+    ap.add_argument("--gram", action="store_true",
+                    help="with --kernel-only: hand the operand over stored M x N and time syrk_lower_tn (C = A^T A)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
+    if args.gram and not args.kernel_only:
+        ap.error("--gram needs --kernel-only (the host-buffer entry point takes the N x M form)")
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

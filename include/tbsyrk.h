@@ -83,6 +83,26 @@ int syrk_lower(int64_t N, int64_t M,
                int dtype, void* stream);
 
 /*
+ * The same update for the other storage order of the operand (the Gram-matrix form):
+ *
+ *     C[i][j] = alpha * sum_k A[k][i] * A[k][j] + beta * C[i][j]      for 0 <= j <= i < N,
+ *
+ * i.e. Algorithm 1 of the paper applied to the N x M matrix A^T, where A is a DEVICE
+ * pointer to an M x N row-major array with row pitch lda >= max(1, N) elements.  The
+ * paper states the operation for an N x M operand only; the work list (Algorithm 4,
+ * Section 5.1.4), C, alpha, beta, dtype, stream, alignment rule (A 16-byte aligned and
+ * lda * sizeof(element) a multiple of 16, else a slower plain-load kernel), ownership
+ * and error codes are those of syrk_lower (SYRK_ERR_LD refers to lda < N here).
+ * FP64 runs on the FP64 tensor cores in both launch forms; BF16 inputs in this storage
+ * order currently take the plain-load kernel.
+ */
+int syrk_lower_tn(int64_t N, int64_t M,
+                  const void* A, int64_t lda,
+                  void* C, int64_t ldc,
+                  double alpha, double beta,
+                  int dtype, void* stream);
+
+/*
  * Same operation with HOST buffers: copies A (and C when beta != 0) to the
  * device, runs syrk_lower on a stream of the library, copies the lower triangle
  * back into C, and waits for completion.  A and C are host pointers (pageable or

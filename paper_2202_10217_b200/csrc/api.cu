@@ -13,11 +13,12 @@ using namespace tbsyrk;
 
 namespace {
 
-int validate(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, int dtype) {
+int validate(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, int dtype,
+             bool a_is_m_by_n = false) {
     if (dtype != SYRK_DTYPE_F64 && dtype != SYRK_DTYPE_BF16_F32) return SYRK_ERR_DTYPE;
     if (N < 0 || M < 0 || N >= (int64_t(1) << 31) - 256 || M >= (int64_t(1) << 31) - 256) return SYRK_ERR_SIZE;
     if (N == 0) return SYRK_OK;
-    if (lda < std::max<int64_t>(1, M) || ldc < N) return SYRK_ERR_LD;
+    if (lda < std::max<int64_t>(1, a_is_m_by_n ? N : M) || ldc < N) return SYRK_ERR_LD;
     if (!C || (M > 0 && !A)) return SYRK_ERR_NULL;
     return SYRK_OK;
 }
@@ -68,7 +69,7 @@ int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk)
 }  // namespace
 
 int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
-                            double beta, int dtype, cudaStream_t stream, int f64_launch) {
+                            double beta, int dtype, cudaStream_t stream, int f64_launch, int a_is_m_by_n) {
     DeviceState* ds = nullptr;
     int rc = get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
@@ -76,15 +77,17 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         if (beta == 1.0) return SYRK_OK;
         return launch_scale_lower(dtype, N, C, ldc, beta, stream) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
     }
-    if (!tma_ok(A, lda, dtype))
-        return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, stream) == cudaSuccess
+    // The M x N storage order has a tensor-core path in FP64 only so far.
+    if (!tma_ok(A, lda, dtype) || (a_is_m_by_n && dtype != SYRK_DTYPE_F64))
+        return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
     DevicePlan* dp = nullptr;
     rc = get_device_plan(ds, N, dtype, &dp);
     if (rc != SYRK_OK) return rc;
     const KernelShape ks = kernel_shape(dtype);
     CUtensorMap tm;
-    rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, ks.tile, ks.bk);
+    if (a_is_m_by_n) rc = encode_tensor_map_2d(&tm, dtype, A, M, N, lda, ks.bk, 16);   // boxes of 16 k-rows x 16 columns
+    else rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, ks.tile, ks.bk);
     if (rc != SYRK_OK) return rc;
     const int64_t n_items = int64_t(dp->plan.items.size());
     cudaError_t e;
@@ -100,7 +103,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
                                 (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count));
         int* tickets = persistent ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc,
-                            alpha, beta, tickets, ds->sm_count, ds->d_status, stream);
+                            alpha, beta, a_is_m_by_n, tickets, ds->sm_count, ds->d_status, stream);
     } else {
         const int split = pick_split_k(ds, dp, M, ks.bk);
         if (split > 1) {
@@ -142,6 +145,14 @@ int syrk_lower(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_
     if (rc != SYRK_OK || N == 0) return rc;
     std::lock_guard<std::mutex> lock(runtime().mu);
     return syrk_run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream));
+}
+
+int syrk_lower_tn(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
+                  double beta, int dtype, void* stream) {
+    int rc = validate(N, M, A, lda, C, ldc, dtype, true);
+    if (rc != SYRK_OK || N == 0) return rc;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    return syrk_run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream), -1, 1);
 }
 
 int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,

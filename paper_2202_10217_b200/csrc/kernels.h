@@ -12,10 +12,12 @@ namespace tbsyrk {
 // swizzle, through which the old C tiles are fetched when beta != 0.  With `d_tickets` null there
 // is one thread block per work item; otherwise `n_blocks` persistent blocks draw the items from
 // d_tickets[0] (d_tickets[0..1] must be zero and must not be shared with a launch that can run at
-// the same time; the kernel leaves them zero).
+// the same time; the kernel leaves them zero).  `a_is_m_by_n`: A is stored M x N row-major (the
+// Gram form C = A^T A); `tmA` then has boxes of 16 rows x 16 columns over that array.
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
-                            double beta, int* d_tickets, int n_blocks, int* d_status, cudaStream_t stream);
+                            double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
+                            cudaStream_t stream);
 // The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
 // P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
 // columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.
@@ -46,7 +48,7 @@ int bf16_store_box();
 // Plain-load kernels: one thread per lower-triangle entry.  Used when A does not meet
 // the TMA alignment rules; same result, much slower.
 cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, void* C,
-                              int64_t ldc, double alpha, double beta, cudaStream_t stream);
+                              int64_t ldc, double alpha, double beta, int a_is_m_by_n, cudaStream_t stream);
 
 // Lower triangle <- beta * lower triangle (zero when beta == 0, without reading C).
 cudaError_t launch_scale_lower(int dtype, int64_t N, void* C, int64_t ldc, double beta,

@@ -90,9 +90,10 @@ int encode_tensor_map_f64_plain(CUtensorMap* tm, const void* p, int64_t rows, in
                                 int box_rows, int box_cols);
 
 // The device path of syrk_lower (arguments already validated; the caller holds the runtime lock).
-// `f64_launch` >= 0 overrides the process-wide FP64 launch form for this call.
+// `f64_launch` >= 0 overrides the process-wide FP64 launch form for this call.  `a_is_m_by_n`: A is
+// stored M x N row-major (pitch lda >= N) and the call computes alpha * A^T A + beta * C.
 int syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
-                    double beta, int dtype, cudaStream_t stream, int f64_launch = -1);
+                    double beta, int dtype, cudaStream_t stream, int f64_launch = -1, int a_is_m_by_n = 0);
 
 void release_cholesky_workspaces();
 

@@ -82,6 +82,7 @@ __device__ __forceinline__ int c_steps_of(const Call& k, int n_tile) { return k.
 // ---------------------------------------------------------------------------------------------
 // Producer (one thread): fetch one item's ring steps, starting at global step g.
 // ---------------------------------------------------------------------------------------------
+template <bool kTN>
 __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, uint32_t& g) {
     const int n_seg = it.n_seg, n_tile = it.n_tile;
     for (int ks = 0; ks < k.n_ksteps; ++ks, ++g) {
@@ -91,9 +92,18 @@ __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, 
         }
         mbar_arrive_expect_tx(&k.full_bar[st], uint32_t(n_seg) * kSegBytes);
         uint8_t* dst = k.smem + st * kStageBytes;
-        for (int s = 0; s < n_seg; ++s)
-            tma_load_2d(dst + s * kSegBytes, (k.gemm && s < it.pad) ? k.tmB : k.tmA, ks * kBK, it.seg[s] * kTile,
-                        &k.full_bar[st]);
+        if (kTN) {
+            // A stored M x N: a segment's 32 columns x 16 rows of A arrive as two boxes of 16 x 16
+            // (128-byte rows of 16 columns, one row per k), 2 KB each.
+            for (int s = 0; s < n_seg; ++s)
+                for (int h = 0; h < 2; ++h)
+                    tma_load_2d(dst + s * kSegBytes + h * (kSegBytes / 2), k.tmA, it.seg[s] * kTile + h * 16, ks * kBK,
+                                &k.full_bar[st]);
+        } else {
+            for (int s = 0; s < n_seg; ++s)
+                tma_load_2d(dst + s * kSegBytes, (k.gemm && s < it.pad) ? k.tmB : k.tmA, ks * kBK, it.seg[s] * kTile,
+                            &k.full_bar[st]);
+        }
     }
     // Old C: ring step j carries tiles 4j .. 4j+3 (8 KB each, row pitch 256 B), those below the diagonal.
     const int n_c = c_steps_of(k, n_tile);
@@ -189,7 +199,16 @@ __device__ __forceinline__ void release(const Call& k, uint32_t g, int lane) { r
 
 // The M loop of one warp's tile.  kSkipLast leaves out block (3, 3), which the 16th warp of
 // a triangle block computes.  Returns false when a bounded wait ran out.
-template <bool kSkipLast>
+// Shared-memory address of a fragment element.  A stored N x M (kTN false): 8-row group j of a
+// segment is 1024 bytes further, k-slice sl flips the 16-byte chunk.  A stored M x N (kTN true):
+// see fragment_offset_tn.
+template <bool kTN>
+__device__ __forceinline__ uint32_t frag_addr(uint32_t p, int j, int sl) {
+    if (kTN) return (p ^ uint32_t(((sl & 1) << 5) ^ ((j & 1) << 6))) + uint32_t((sl & 1) * 256 + (sl >> 1) * 1024 + (j >> 1) * 2048);
+    return (p ^ uint32_t(sl << 4)) + uint32_t(j * 1024);
+}
+
+template <bool kSkipLast, bool kTN>
 __device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const Call& k, uint32_t xbase, uint32_t ybase,
                                               uint32_t off0, uint32_t g0, int lane) {
     uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;      // stage and phase, advanced step by step
@@ -202,8 +221,8 @@ __device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const Call
             double a[4], b[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                a[j] = lds_f64((px ^ (sl << 4)) + j * 1024);
-                b[j] = lds_f64((py ^ (sl << 4)) + j * 1024);
+                a[j] = lds_f64(frag_addr<kTN>(px, j, sl));
+                b[j] = lds_f64(frag_addr<kTN>(py, j, sl));
             }
 #pragma unroll
             for (int mi = 0; mi < 4; ++mi)
@@ -229,13 +248,26 @@ __device__ __forceinline__ uint32_t fragment_offset(int lane) {
     return uint32_t(g * 128 + ((((t >> 1) << 2) ^ g) << 4) + ((t & 1) << 3));
 }
 
+__device__ __forceinline__ uint32_t fragment_offset_tn(int lane) {
+    // A stored M x N: a stage holds, per segment, two boxes of 16 k-rows x 16 columns (128-byte rows,
+    // 16-byte chunk index ^ k % 8).  Column n = 8j + g of the segment is in box j>>1, chunk
+    // 4(j&1) + (g>>1), half g&1.  Slice sl and lane t take k = (t&1) + 4(t>>1) + 2(sl&1) + 8(sl>>1): the
+    // four k rows of a slice then fall on both halves of the banks (rows k and k^4 differ in chunk
+    // bit 2), so a warp's 256 bytes take the minimum of two wavefronts.  With disjoint bits, the
+    // address of (j, sl) is  (lane part ^ ((sl&1)<<5 ^ (j&1)<<6)) + (sl&1)*256 + (sl>>1)*1024 + (j>>1)*2048.
+    const int g = lane >> 2, t = lane & 3;
+    const int k_lane = (t & 1) + 4 * (t >> 1);
+    return uint32_t(k_lane * 128 + ((((g >> 1) ^ k_lane)) << 4) + ((g & 1) << 3));
+}
+
 // 16th warp of a triangle block: the 15 left-out 8 x 8 blocks.  g0 = the item's first ring step,
 // n_c = its old-C steps.
+template <bool kTN>
 __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, int lane) {
     const int gq = lane >> 2, t = lane & 3;
     const uint32_t gc = g0 + uint32_t(k.n_ksteps);
     const bool use_beta = (k.beta != 0.0);
-    const uint32_t off0 = fragment_offset(lane);
+    const uint32_t off0 = kTN ? fragment_offset_tn(lane) : fragment_offset(lane);
     int32_t seg[6];
 #pragma unroll
     for (int s = 0; s < 6; ++s) seg[s] = it.seg[s];
@@ -245,12 +277,12 @@ __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it
     uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;
     for (int ks = 0; ks < k.n_ksteps; ++ks) {
         if (!wait_full_at(k, st, parity, lane)) return false;
-        const uint32_t base = (k.smem32 + st * kStageBytes + 3 * 1024) | off0;   // rows 24..31 of every segment
+        const uint32_t base = (k.smem32 + st * kStageBytes) | off0;
 #pragma unroll
         for (int sl = 0; sl < 4; ++sl) {
             double f[6];
 #pragma unroll
-            for (int j = 0; j < 6; ++j) f[j] = lds_f64((base ^ (sl << 4)) + j * kSegBytes);
+            for (int j = 0; j < 6; ++j) f[j] = lds_f64(frag_addr<kTN>(base, 3, sl) + j * kSegBytes);   // rows 24..31 of every segment
             int q = 0;
 #pragma unroll
             for (int x = 1; x < 6; ++x)
@@ -286,12 +318,13 @@ __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it
 }
 
 // A warp with a tile (tile number `warp` of the item).  `scavenge`: block (3, 3) is left to the 16th warp.
+template <bool kTN>
 __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, bool scavenge,
                                           int warp, int lane) {
     const int gq = lane >> 2, t = lane & 3;
     const uint32_t gc = g0 + uint32_t(k.n_ksteps);
     const bool use_beta = (k.beta != 0.0);
-    const uint32_t off0 = fragment_offset(lane);
+    const uint32_t off0 = kTN ? fragment_offset_tn(lane) : fragment_offset(lane);
     const int sx = it.tile_x[warp], sy = it.tile_y[warp];
     const int64_t row0 = int64_t(it.seg[sx]) * kTile, col0 = int64_t(it.seg[sy]) * kTile;
     const uint32_t xbase = uint32_t(sx) * kSegBytes, ybase = uint32_t(sy) * kSegBytes;
@@ -302,8 +335,8 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
 #pragma unroll
         for (int ni = 0; ni < 4; ++ni) acc[mi][ni][0] = acc[mi][ni][1] = 0.0;
 
-    const bool alive = scavenge ? tile_mainloop<true>(acc, k, xbase, ybase, off0, g0, lane)
-                                : tile_mainloop<false>(acc, k, xbase, ybase, off0, g0, lane);
+    const bool alive = scavenge ? tile_mainloop<true, kTN>(acc, k, xbase, ybase, off0, g0, lane)
+                                : tile_mainloop<false, kTN>(acc, k, xbase, ybase, off0, g0, lane);
     if (!alive) return false;
 
     for (int j = 0; j < n_c; ++j)
@@ -345,14 +378,15 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
 
 // One MMA warp's share of one item: its ring steps from global step g on, then its write-out.
 // Every warp waits for and releases every ring step of the item, with or without work in it.
+template <bool kTN>
 __device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it, uint32_t& g, int warp, int lane) {
     const int n_tile = it.n_tile;
     const int n_c = c_steps_of(k, n_tile);
     const uint32_t g0 = g;
     g += uint32_t(k.n_ksteps + n_c);
     const bool scavenge = !k.gemm && it.pad != 0;      // set by prepare_item
-    if (scavenge && warp == kMmaWarps - 1) return scavenger_role(k, it, g0, n_c, lane);
-    if (warp < n_tile) return tile_role(k, it, g0, n_c, scavenge, warp, lane);
+    if (scavenge && warp == kMmaWarps - 1) return scavenger_role<kTN>(k, it, g0, n_c, lane);
+    if (warp < n_tile) return tile_role<kTN>(k, it, g0, n_c, scavenge, warp, lane);
     for (uint32_t s = g0; s < g; ++s) {                 // no tile in this item: keep the ring moving
         if (!wait_full(k, s, lane)) return false;
         release(k, s, lane);
@@ -366,6 +400,7 @@ __device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it,
 // groups), its column segments come from Q (tmB, the first `pad` segments), its row segments
 // from P (tmA).
 // ---------------------------------------------------------------------------------------------
+template <bool kTN>
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
@@ -421,12 +456,12 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (lane == 0) {
             prefetch_tensormap(&tmA);
             if (c_tma) prefetch_tensormap(&tmC);
-            produce_item(k, s_item, g);
+            produce_item<kTN>(k, s_item, g);
             if (s_abort) drain_producer(k, g);
         }
         return;
     }
-    mma_warp_item(k, s_item, g, warp, lane);
+    mma_warp_item<kTN>(k, s_item, g, warp, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -436,6 +471,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 // kStages ring steps - hence fewer than kItemRing items - ahead of the slowest MMA warp, so a
 // slot is rewritten only after every warp has read it.
 // ---------------------------------------------------------------------------------------------
+template <bool kTN>
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
                                const WorkItem* __restrict__ items, int64_t n_items, int* __restrict__ counter,
@@ -483,7 +519,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                 if (last) dst.n_tile = -1;                        // end marker
                 mbar_arrive(&s_item_bar[slot % kItemRing]);       // publishes the slot (release)
                 if (last) break;
-                if (!produce_item(k, dst, g)) {                   // gave up: tell the MMA warps to stop as well
+                if (!produce_item<kTN>(k, dst, g)) {                   // gave up: tell the MMA warps to stop as well
                     WorkItem& end = s_ring[(slot + 1) % kItemRing];
                     end.n_tile = -1;
                     mbar_arrive(&s_item_bar[(slot + 1) % kItemRing]);
@@ -503,7 +539,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
         }
         const WorkItem& it = s_ring[slot % kItemRing];
         if (it.n_tile < 0) return;
-        if (!mma_warp_item(k, it, g, warp, lane)) return;
+        if (!mma_warp_item<kTN>(k, it, g, warp, lane)) return;
     }
 }
 
@@ -517,12 +553,14 @@ cudaError_t configure_f64_kernels() {
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(f64::syrk_f64_tbs_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, f64::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(f64::syrk_f64_tbs_persistent_kernel,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, f64::kSmemBytes);
-        if (e != cudaSuccess) return e;
+        const void* kernels[4] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true>)};
+        for (const void* fn : kernels) {
+            cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, f64::kSmemBytes);
+            if (e != cudaSuccess) return e;
+        }
         configured[dev] = true;
     }
     return cudaSuccess;
@@ -531,7 +569,8 @@ cudaError_t configure_f64_kernels() {
 
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
-                            double beta, int* d_tickets, int n_blocks, int* d_status, cudaStream_t stream) {
+                            double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
+                            cudaStream_t stream) {
     cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
@@ -539,14 +578,16 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
     const int32_t n_ksteps = int32_t((M + f64::kBK - 1) / f64::kBK);
     const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
     CUtensorMap none{};
+    const dim3 threads(f64::kThreads);
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
-        const int64_t blocks = n_items < n_blocks ? n_items : int64_t(n_blocks);
-        f64::syrk_f64_tbs_persistent_kernel<<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
-            tmA, c_tma ? *tmC : none, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma,
-            d_status);
+        const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
+        auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true> : f64::syrk_f64_tbs_persistent_kernel<false>;
+        kernel<<<grid, threads, f64::kSmemBytes, stream>>>(tmA, c_tma ? *tmC : none, d_items, n_items, d_tickets, N,
+                                                           n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
         return cudaGetLastError();
     }
-    f64::syrk_f64_tbs_kernel<<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
+    auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
+    kernel<<<dim3(unsigned(n_items)), threads, f64::kSmemBytes, stream>>>(
         tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
     return cudaGetLastError();
 }
@@ -563,7 +604,7 @@ cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, c
     const int64_t row_tiles = (nrows + f64::kTile - 1) / f64::kTile, col_tiles = (ncols + f64::kTile - 1) / f64::kTile;
     const int64_t blocks = ((row_tiles + 3) / 4) * ((col_tiles + 3) / 4);
     CUtensorMap none{};
-    f64::syrk_f64_tbs_kernel<<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
+    f64::syrk_f64_tbs_kernel<false><<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmP, tmQ, c_tma ? *tmD : none, nullptr, nrows, ncols, int32_t(col_tiles), n_ksteps, D, ldd, alpha, beta,
         vec_ok, c_tma, d_status);
     return cudaGetLastError();

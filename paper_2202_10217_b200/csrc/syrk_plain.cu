@@ -2,7 +2,8 @@
 //
 // syrk_plain: one thread per entry (i, j), j <= i, of the result of Algorithm 1 of the
 // paper with alpha/beta; no TMA, no alignment requirement.  It is the slow path for
-// inputs whose base address or row pitch is not a multiple of 16 bytes.
+// inputs whose base address or row pitch is not a multiple of 16 bytes, for either storage
+// order of A (N x M, or M x N for the Gram form).
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -17,15 +18,16 @@ template <> struct Widen<__nv_bfloat16, float> {
 };
 
 template <typename TA, typename TC>
-__global__ void syrk_plain_kernel(int64_t N, int64_t M, const TA* __restrict__ A, int64_t lda,
-                                  TC* __restrict__ C, int64_t ldc, TC alpha, TC beta) {
+__global__ void syrk_plain_kernel(int64_t N, int64_t M, const TA* __restrict__ A, int64_t row_stride,
+                                  int64_t col_stride, TC* __restrict__ C, int64_t ldc, TC alpha, TC beta) {
     const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
     if (i >= N || j > i) return;
-    const TA* ai = A + i * lda;
-    const TA* aj = A + j * lda;
+    const TA* ai = A + i * row_stride;       // row i of the N x M operand, whichever way it is stored
+    const TA* aj = A + j * row_stride;
     TC s = TC(0);
-    for (int64_t k = 0; k < M; ++k) s = fma(Widen<TA, TC>::get(ai + k), Widen<TA, TC>::get(aj + k), s);
+    for (int64_t k = 0; k < M; ++k)
+        s = fma(Widen<TA, TC>::get(ai + k * col_stride), Widen<TA, TC>::get(aj + k * col_stride), s);
     TC* c = C + i * ldc + j;
     *c = (beta == TC(0)) ? alpha * s : alpha * s + beta * *c;
 }
@@ -46,15 +48,16 @@ inline dim3 grid2d(int64_t N, dim3 block) {
 }  // namespace
 
 cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, void* C,
-                              int64_t ldc, double alpha, double beta, cudaStream_t stream) {
+                              int64_t ldc, double alpha, double beta, int a_is_m_by_n, cudaStream_t stream) {
     if (N == 0) return cudaSuccess;
     const dim3 block(32, 8);
+    const int64_t rs = a_is_m_by_n ? 1 : lda, cs = a_is_m_by_n ? lda : 1;
     if (dtype == 0)
         syrk_plain_kernel<double, double><<<grid2d(N, block), block, 0, stream>>>(
-            N, M, static_cast<const double*>(A), lda, static_cast<double*>(C), ldc, alpha, beta);
+            N, M, static_cast<const double*>(A), rs, cs, static_cast<double*>(C), ldc, alpha, beta);
     else
         syrk_plain_kernel<__nv_bfloat16, float><<<grid2d(N, block), block, 0, stream>>>(
-            N, M, static_cast<const __nv_bfloat16*>(A), lda, static_cast<float*>(C), ldc,
+            N, M, static_cast<const __nv_bfloat16*>(A), rs, cs, static_cast<float*>(C), ldc,
             float(alpha), float(beta));
     return cudaGetLastError();
 }

@@ -37,8 +37,11 @@ def sentinel_array(shape, np_dtype):
 
 def run_case(A: np.ndarray, dtype: int, alpha: float, beta: float, Cin: np.ndarray | None = None,
              lda: int | None = None, ldc: int | None = None, a_offset: int = 0, c_offset: int = 0,
-             poison: bool = False):
-    """One call; returns (got, ref, bound, Cin_used).  Checks canaries and status itself."""
+             poison: bool = False, tn: bool = False):
+    """One call; returns (got, ref, bound).  Checks canaries and status itself.
+
+    `A` is always the N x M operand of the reference.  With `tn` it is handed to the library
+    transposed (an M x N row-major array, pitch lda >= N) through syrk_lower_tn."""
     N, M = A.shape
     cdt = I.c_storage_dtype(dtype)
     ldc = max(N, 1) if ldc is None else ldc
@@ -52,9 +55,13 @@ def run_case(A: np.ndarray, dtype: int, alpha: float, beta: float, Cin: np.ndarr
         body[np.tril_indices(N)] = np.nan
     before = host_c.copy()
     dev_c = torch.from_numpy(host_c).cuda()
-    keep, a_ptr = a_to_device(A, dtype, lda, a_offset)
     c_ptr = dev_c.data_ptr() + (GUARD * (ldc + c_offset) + c_offset) * dev_c.element_size()
-    B.syrk_lower(N, M, a_ptr, max(M, 1) if lda is None else lda, c_ptr, ldc + c_offset, alpha, beta, dtype)
+    if tn:
+        keep, a_ptr = a_to_device(np.ascontiguousarray(A.T), dtype, lda, a_offset)
+        B.syrk_lower_tn(N, M, a_ptr, max(N, 1) if lda is None else lda, c_ptr, ldc + c_offset, alpha, beta, dtype)
+    else:
+        keep, a_ptr = a_to_device(A, dtype, lda, a_offset)
+        B.syrk_lower(N, M, a_ptr, max(M, 1) if lda is None else lda, c_ptr, ldc + c_offset, alpha, beta, dtype)
     torch.cuda.synchronize()
     assert B.syrk_last_status() == 0
     after = dev_c.cpu().numpy()
