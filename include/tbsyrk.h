@@ -93,8 +93,8 @@ int syrk_lower(int64_t N, int64_t M,
  * Section 5.1.4), C, alpha, beta, dtype, stream, alignment rule (A 16-byte aligned and
  * lda * sizeof(element) a multiple of 16, else a slower plain-load kernel), ownership
  * and error codes are those of syrk_lower (SYRK_ERR_LD refers to lda < N here).
- * FP64 runs on the FP64 tensor cores in both launch forms; BF16 inputs in this storage
- * order currently take the plain-load kernel.
+ * Both dtypes run on the tensor-core kernels (FP64: both launch forms; BF16: tcgen05
+ * with MN-major operands, K-split included).
  */
 int syrk_lower_tn(int64_t N, int64_t M,
                   const void* A, int64_t lda,

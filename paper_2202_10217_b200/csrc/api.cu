@@ -77,8 +77,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         if (beta == 1.0) return SYRK_OK;
         return launch_scale_lower(dtype, N, C, ldc, beta, stream) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
     }
-    // The M x N storage order has a tensor-core path in FP64 only so far.
-    if (!tma_ok(A, lda, dtype) || (a_is_m_by_n && dtype != SYRK_DTYPE_F64))
+    if (!tma_ok(A, lda, dtype))
         return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
     DevicePlan* dp = nullptr;
@@ -86,7 +85,8 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
     if (rc != SYRK_OK) return rc;
     const KernelShape ks = kernel_shape(dtype);
     CUtensorMap tm;
-    if (a_is_m_by_n) rc = encode_tensor_map_2d(&tm, dtype, A, M, N, lda, ks.bk, 16);   // boxes of 16 k-rows x 16 columns
+    // A stored M x N: boxes of one stage's k-rows x 128 bytes of columns (16 doubles, 64 bf16)
+    if (a_is_m_by_n) rc = encode_tensor_map_2d(&tm, dtype, A, M, N, lda, ks.bk, dtype == SYRK_DTYPE_F64 ? 16 : 64);
     else rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, ks.tile, ks.bk);
     if (rc != SYRK_OK) return rc;
     const int64_t n_items = int64_t(dp->plan.items.size());
@@ -117,8 +117,8 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                            encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
         e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
-                             float(beta), split, ds->d_partial, dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, ds->d_status,
-                             ds->sm_count, stream);
+                             float(beta), split, ds->d_partial, dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, a_is_m_by_n,
+                             ds->d_status, ds->sm_count, stream);
     }
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }

@@ -23,7 +23,9 @@
 // MMAs start while the previous item's third tile is still being written out.
 //
 // Both MMA operands come from the same row-major A (K contiguous): segment x is the
-// M-operand, segment y (or the adjacent pair y, y+1) the N-operand, both K-major.
+// M-operand, segment y (or the adjacent pair y, y+1) the N-operand, both K-major.  When A is
+// stored M x N (the Gram form) the stages hold 64 k-rows of 64 columns per box and both
+// operands are MN-major; everything after the MMA is the same.
 #include "device_utils.cuh"
 #include "kernels.h"
 #include "tbs_plan.h"
@@ -93,9 +95,23 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     d |= uint64_t(2) << 61;                        // layout: 128-byte swizzle
     return d;
 }
-// Instruction descriptor, kind::f16: D = FP32, A = B = BF16, both K-major, M = 128.
-__device__ __forceinline__ uint32_t instr_desc_bf16(uint32_t n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+// The same for an MN-major operand (A stored M x N: a segment's 128 columns are contiguous in
+// memory, one 128-byte row of 64 columns per k).  A segment slot holds two groups of 64 columns,
+// 8192 bytes apart (leading byte offset); within a group, 8-row k groups are 1024 bytes apart
+// (stride byte offset); `addr` advances by 2048 bytes per K = 16 step.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= uint64_t((addr & 0x3FFFF) >> 4);
+    d |= uint64_t(8192 >> 4) << 16;                // leading byte offset (between 64-column groups)
+    d |= uint64_t(1024 >> 4) << 32;                // stride byte offset (between 8-row k groups)
+    d |= uint64_t(1) << 46;
+    d |= uint64_t(2) << 61;
+    return d;
+}
+// Instruction descriptor, kind::f16: D = FP32, A = B = BF16, M = 128; both operands K-major, or
+// both MN-major (bits 15 and 16) when A is stored M x N.
+__device__ __forceinline__ uint32_t instr_desc_bf16(uint32_t n, bool mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (mn_major ? (3u << 15) : 0u) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // ---- bulk-async (TMA) store helpers ---------------------------------------------------
@@ -147,6 +163,7 @@ __device__ __forceinline__ void layout_of(const WorkItem* it, int n_tile, uint32
     }
 }
 
+template <bool kTN>
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
                      const WorkItem* __restrict__ items, int64_t n_items, int64_t N, int32_t n_ksteps,
@@ -207,8 +224,15 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     }
                     mbar_arrive_expect_tx(&full_bar[st], uint32_t(n_seg) * kSegBytes);
                     uint8_t* dst = smem + st * kStageBytes;
-                    for (int s = 0; s < n_seg; ++s)
-                        tma_load_2d(dst + s * kSegBytes, &tmA, ks * kBK, rows[s], &full_bar[st]);
+                    if (kTN) {   // A stored M x N: two boxes of 64 k-rows x 64 columns per segment
+                        for (int s = 0; s < n_seg; ++s)
+                            for (int h = 0; h < 2; ++h)
+                                tma_load_2d(dst + s * kSegBytes + h * (kSegBytes / 2), &tmA, rows[s] + h * 64, ks * kBK,
+                                            &full_bar[st]);
+                    } else {
+                        for (int s = 0; s < n_seg; ++s)
+                            tma_load_2d(dst + s * kSegBytes, &tmA, ks * kBK, rows[s], &full_bar[st]);
+                    }
                 }
             }
             if (s_abort) {   // winding down: let the copies still in flight land first
@@ -223,7 +247,8 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if (lane == 0) {
             uint32_t g = 0, n_done = 0;
             const uint32_t smem_base = smem_u32(smem);
-            const uint64_t desc_hi = smem_desc_sw128(0);
+            const uint64_t desc_hi = kTN ? smem_desc_mn_sw128(0) : smem_desc_sw128(0);
+            constexpr uint32_t kk_step = kTN ? (2048u >> 4) : (32u >> 4);   // descriptor advance per K = 16
             for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride, ++n_done) {
                 const Unit u = unit_of(w, n_items, n_ksteps, split);
                 const WorkItem* it = &items[u.item];
@@ -234,7 +259,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const int qq = q < L.n_grp ? q : 0;
                     a_lo[q] = (smem_base + uint32_t(L.gx[qq]) * kSegBytes) >> 4;
                     b_lo[q] = (smem_base + uint32_t(L.gy[qq]) * kSegBytes) >> 4;
-                    idesc[q] = instr_desc_bf16(uint32_t(L.gn[qq]));
+                    idesc[q] = instr_desc_bf16(uint32_t(L.gn[qq]), kTN);
                     d_addr[q] = tmem_base + L.gcol[qq];
                 }
                 // accumulators of this item must have been drained by the epilogue
@@ -257,8 +282,8 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     for (int q = 0; q < L.n_grp; ++q) {
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk)
-                            tc_mma_bf16(d_addr[q], desc_hi | uint64_t(a_lo[q] + st_off + 2 * kk),
-                                        desc_hi | uint64_t(b_lo[q] + st_off + 2 * kk), idesc[q],
+                            tc_mma_bf16(d_addr[q], desc_hi | uint64_t(a_lo[q] + st_off + kk_step * kk),
+                                        desc_hi | uint64_t(b_lo[q] + st_off + kk_step * kk), idesc[q],
                                         (kk > 0) ? 1u : first);
                     }
                     tc_commit(&empty_bar[st]);    // stage reusable once these MMAs have read it
@@ -414,16 +439,19 @@ splitk_reduce_kernel(const WorkItem* __restrict__ items, const int64_t* __restri
 cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                              int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
-                             int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int* d_status,
-                             int sm_count, cudaStream_t stream) {
+                             int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
+                             int* d_status, int sm_count, cudaStream_t stream) {
     // The shared-memory attribute belongs to a device's context: set it once per device.
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(bf16::syrk_bf16_tbs_kernel,
+        cudaError_t e = cudaFuncSetAttribute(bf16::syrk_bf16_tbs_kernel<false>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, bf16::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(bf16::syrk_bf16_tbs_kernel<true>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, bf16::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -435,7 +463,8 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     const unsigned grid = ranges ? unsigned(n_ctas) : unsigned(n_units < sm_count ? n_units : sm_count);
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0) ? 1 : 0;
     CUtensorMap none{};
-    bf16::syrk_bf16_tbs_kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
+    auto kernel = a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true> : bf16::syrk_bf16_tbs_kernel<false>;
+    kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
         tmA, tmC ? *tmC : none, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, split,
         d_partial, d_tile_base, total_tiles, ranges ? d_cta_begin : nullptr, d_status);
     cudaError_t e = cudaGetLastError();

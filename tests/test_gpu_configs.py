@@ -51,14 +51,19 @@ def check_sampled(dC, Cin_vals, A, wl, ii, jj):
     return float(np.max(err / np.maximum(tol, 1e-300)))
 
 
-def run_config(key, samples):
+def run_config(key, samples, gram=False):
+    """`gram`: the same operand handed over stored M x N, through syrk_lower_tn."""
     wl = I.CONFIGS[key]
     A = wl.make_A()
     dA = upload_A(A, wl.dtype)
     sentinel = float("nan")
     dC = torch.full((wl.N, wl.N), sentinel, dtype=torch.float64 if wl.dtype == B.DTYPE_F64 else torch.float32,
                     device="cuda")
-    B.syrk_lower(wl.N, wl.M, dA, wl.M, dC, wl.N, wl.alpha, wl.beta, wl.dtype)
+    if gram:
+        dA = dA.t().contiguous()
+        B.syrk_lower_tn(wl.N, wl.M, dA, wl.N, dC, wl.N, wl.alpha, wl.beta, wl.dtype)
+    else:
+        B.syrk_lower(wl.N, wl.M, dA, wl.M, dC, wl.N, wl.alpha, wl.beta, wl.dtype)
     torch.cuda.synchronize()
     assert B.syrk_last_status() == 0
     # strict upper triangle untouched (still NaN), lower triangle fully written
@@ -81,6 +86,26 @@ def test_config2_full_triangle():
     il = np.tril_indices(wl.N)
     got = dC.cpu().numpy()
     assert np.all(np.abs(got[il] - ref[il]) <= O.tolerance(wl.M, bound[il], None, 1.0, 0.0, wl.dtype))
+
+
+def test_config2_gram_form_full_triangle():
+    wl, A, dC = run_config("c2", 0, gram=True)
+    ref, bound = O.syrk_lower(A, None, wl.alpha, 0.0, wl.dtype)
+    il = np.tril_indices(wl.N)
+    got = dC.cpu().numpy()
+    assert np.all(np.abs(got[il] - ref[il]) <= O.tolerance(wl.M, bound[il], None, 1.0, 0.0, wl.dtype))
+
+
+def test_config3_gram_form_sampled():
+    wl, A, dC = run_config("c3", 1 << 20, gram=True)
+    ii, jj = sample_pairs(wl.N, 1 << 20, 128, seed=35)
+    check_sampled(dC, None, A, wl, ii, jj)
+
+
+def test_config4_gram_form_sampled_split_k():
+    wl, A, dC = run_config("c4", 1 << 14, gram=True)
+    ii, jj = sample_pairs(wl.N, 1 << 14, 128, seed=45)
+    check_sampled(dC, None, A, wl, ii, jj)
 
 
 def test_config3_sampled():

@@ -22,7 +22,8 @@ DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16"])
 # K-steps (M not a multiple of 16) are both covered.
 SIZES = {B.DTYPE_F64: [(2, 1), (6, 3), (30, 17), (32, 16), (34, 50), (100, 64), (258, 130), (512, 256),
                        (1000, 70), (1300, 40), (2500, 33), (33, 20), (257, 19)],
-         B.DTYPE_BF16_F32: [(8, 8), (40, 24), (128, 64), (136, 72), (304, 200), (777, 136)]}
+         B.DTYPE_BF16_F32: [(8, 8), (40, 24), (128, 64), (136, 72), (304, 200), (777, 136), (512, 256),
+                            (1104, 320), (2056, 72), (1304, 1000)]}
 
 
 @DT
@@ -91,3 +92,16 @@ def test_both_launch_forms_agree_bit_for_bit_in_this_storage_order():
 def test_leading_dimension_smaller_than_N_is_refused():
     with pytest.raises(Exception):
         B.syrk_lower_tn(64, 16, 8, 32, 8, 64, 1.0, 0.0, B.DTYPE_F64, stream=0)
+
+
+@pytest.mark.parametrize("split", [0, 2, 5])
+def test_bf16_k_split_in_this_storage_order(split):
+    N, M = 704, 1280
+    A = I.small_int_bf16(N, M, seed=40 + split)
+    Cin = I.random_c(N, 41, B.DTYPE_BF16_F32)
+    try:
+        B.syrk_set_split_k(split)
+        got, ref, bound = run_case(A, B.DTYPE_BF16_F32, 2.0, -1.0, Cin, tn=True)
+    finally:
+        B.syrk_set_split_k(0)
+    assert_within_tolerance(got, ref, bound, M, 2.0, -1.0, Cin, B.DTYPE_BF16_F32)
