@@ -17,6 +17,12 @@
  * the numeric reference.  Everything is done in binary64: bf16 inputs are
  * widened exactly (their 16 bits are the upper half of a binary32), products of
  * two widened bf16 values are exact in binary64, and only the k-sum rounds.
+ * TF32 inputs are binary32 values of which only the TF32 part counts: sign, 8
+ * exponent bits and the 10 leading fraction bits, i.e. the 19 high-order bits of
+ * the encoding; the 13 low-order bits are dropped (not rounded) before the value
+ * is widened.  This is the published TF32 format; the paper itself fixes no
+ * input precision.  Products of two such values have at most 22 significant
+ * bits and are exact in binary64.
  * The k-sum is sequential, with no reassociation and no fused multiply-add
  * (compile with -ffp-contract=off).
  *
@@ -39,7 +45,7 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_DTYPE_F64 = 0, ORACLE_DTYPE_BF16_F32 = 1 };
+enum { ORACLE_DTYPE_F64 = 0, ORACLE_DTYPE_BF16_F32 = 1, ORACLE_DTYPE_TF32_F32 = 2 };
 
 static inline double widen_bf16(uint16_t bits) {
     union { uint32_t u; float f; } x;
@@ -47,13 +53,20 @@ static inline double widen_bf16(uint16_t bits) {
     return (double)x.f;
 }
 
-/* Element A[r][k] as a double, for either input type. */
+static inline double widen_tf32(uint32_t bits) {
+    union { uint32_t u; float f; } x;
+    x.u = bits & 0xFFFFE000u;              /* keep sign, exponent, 10 fraction bits */
+    return (double)x.f;
+}
+
+/* Element A[r][k] as a double, for any input type. */
 static inline double a_at(const void* A, int64_t lda, int dtype, int64_t r, int64_t k) {
     if (dtype == ORACLE_DTYPE_F64) return ((const double*)A)[r * lda + k];
+    if (dtype == ORACLE_DTYPE_TF32_F32) return widen_tf32(((const uint32_t*)A)[r * lda + k]);
     return widen_bf16(((const uint16_t*)A)[r * lda + k]);
 }
 
-/* Element C_in[i][j] as a double (binary64 C, or binary32 C for bf16 inputs). */
+/* Element C_in[i][j] as a double (binary64 C, or binary32 C for bf16 and TF32 inputs). */
 static inline double c_at(const void* C, int64_t ldc, int dtype, int64_t i, int64_t j) {
     if (dtype == ORACLE_DTYPE_F64) return ((const double*)C)[i * ldc + j];
     return (double)((const float*)C)[i * ldc + j];
@@ -83,7 +96,7 @@ static void one_entry(int64_t M, const void* A, int64_t lda, int dtype,
 int oracle_syrk_lower(int64_t N, int64_t M, const void* A, int64_t lda,
                       const void* Cin, int64_t ldc, double alpha, double beta,
                       int dtype, double* Cref, double* Bound, int64_t ldr) {
-    if (N < 0 || M < 0 || (dtype != ORACLE_DTYPE_F64 && dtype != ORACLE_DTYPE_BF16_F32)) return -1;
+    if (N < 0 || M < 0 || dtype < ORACLE_DTYPE_F64 || dtype > ORACLE_DTYPE_TF32_F32) return -1;
     if (N > 0 && (!Cref || !Bound || ldr < N)) return -1;
     if (N > 0 && M > 0 && (!A || lda < M)) return -1;
     if (N > 0 && beta != 0.0 && (!Cin || ldc < N)) return -1;
@@ -107,7 +120,7 @@ int oracle_syrk_entries(int64_t P, const int64_t* I, const int64_t* J,
                         const void* Cin, int64_t ldc, double alpha, double beta,
                         int dtype, double* ref, double* bound) {
     if (P < 0 || N < 0 || M < 0) return -1;
-    if (dtype != ORACLE_DTYPE_F64 && dtype != ORACLE_DTYPE_BF16_F32) return -1;
+    if (dtype < ORACLE_DTYPE_F64 || dtype > ORACLE_DTYPE_TF32_F32) return -1;
     for (int64_t p = 0; p < P; ++p)
         if (I[p] < J[p] || J[p] < 0 || I[p] >= N) return -1;
 #pragma omp parallel for schedule(dynamic, 64)

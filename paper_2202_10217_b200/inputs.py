@@ -17,6 +17,7 @@ import numpy as np
 
 DTYPE_F64 = 0        # A, C binary64
 DTYPE_BF16_F32 = 1   # A bfloat16, C binary32 (binary32 accumulation)
+DTYPE_TF32_F32 = 2   # A binary32 read as TF32 (19 high-order bits), C binary32
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -30,6 +31,12 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
 def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     """Widen bfloat16 bit patterns to binary32 (exact)."""
     return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def f32_keep_tf32_bits(x: np.ndarray) -> np.ndarray:
+    """binary32 values with the 13 low-order bits cleared (exactly representable in TF32)."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32) & np.uint32(0xFFFFE000)
+    return u.view(np.float32)
 
 
 def _normal(rng: np.random.Generator, shape, std: float, chunk_rows: int = 1024) -> np.ndarray:
@@ -56,6 +63,17 @@ def normal_bf16(N: int, M: int, seed: int, std: float = 1.0) -> np.ndarray:
     return f32_to_bf16_bits(_normal(np.random.default_rng(seed), (N, M), std))
 
 
+def normal_f32(N: int, M: int, seed: int, std: float = 1.0, tf32_exact: bool = False) -> np.ndarray:
+    """Entries i.i.d. N(0, std^2), binary32; with ``tf32_exact`` the low 13 bits are cleared."""
+    v = _normal(np.random.default_rng(seed), (N, M), std)
+    return f32_keep_tf32_bits(v) if tf32_exact else v
+
+
+def small_int_f32(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
+    """Integer entries in [lo, hi] stored as binary32 (exact in TF32)."""
+    return np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float32)
+
+
 def small_int_f64(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
     """Integer entries in [lo, hi] stored as binary64 (every partial sum is exact)."""
     return np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float64)
@@ -71,6 +89,8 @@ def ones(N: int, M: int, dtype: int) -> np.ndarray:
     """All-ones A in the storage type of ``dtype``."""
     if dtype == DTYPE_F64:
         return np.ones((N, M), dtype=np.float64)
+    if dtype == DTYPE_TF32_F32:
+        return np.ones((N, M), dtype=np.float32)
     return f32_to_bf16_bits(np.ones((N, M), dtype=np.float32))
 
 
@@ -78,6 +98,8 @@ def to_storage(values: np.ndarray, dtype: int) -> np.ndarray:
     """Values (exactly representable in the target type) -> storage array for A."""
     if dtype == DTYPE_F64:
         return np.ascontiguousarray(values, dtype=np.float64)
+    if dtype == DTYPE_TF32_F32:
+        return np.ascontiguousarray(values, dtype=np.float32)
     return f32_to_bf16_bits(np.asarray(values, dtype=np.float32))
 
 
@@ -110,6 +132,8 @@ class Workload:
             if self.dist == "uniform":
                 return uniform_f64(self.N, self.M, self.seed)
             return normal_f64(self.N, self.M, self.seed, self.std)
+        if self.dtype == DTYPE_TF32_F32:
+            return normal_f32(self.N, self.M, self.seed, self.std)
         return normal_bf16(self.N, self.M, self.seed, self.std)
 
     @property

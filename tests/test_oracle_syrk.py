@@ -14,7 +14,7 @@ from oracle import syrk as O
 from paper_2202_10217_b200 import inputs as I
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
-BOTH = [O.DTYPE_F64, O.DTYPE_BF16_F32]
+BOTH = [O.DTYPE_F64, O.DTYPE_BF16_F32, O.DTYPE_TF32_F32]      # every input type of the reference
 
 
 def lower(x):
@@ -22,7 +22,19 @@ def lower(x):
 
 
 def widen(A, dtype):
-    return A if dtype == O.DTYPE_F64 else I.bf16_bits_to_f32(A).astype(np.float64)
+    if dtype == O.DTYPE_F64:
+        return A
+    if dtype == O.DTYPE_TF32_F32:
+        return I.f32_keep_tf32_bits(A).astype(np.float64)
+    return I.bf16_bits_to_f32(A).astype(np.float64)
+
+
+def real_inputs(N, M, seed, dtype):
+    if dtype == O.DTYPE_F64:
+        return I.normal_f64(N, M, seed)
+    if dtype == O.DTYPE_TF32_F32:
+        return I.normal_f32(N, M, seed)          # low-order bits set: the reference must drop them
+    return I.normal_bf16(N, M, seed)
 
 
 def exact_gram_by_outer_products(Af):
@@ -102,7 +114,7 @@ def test_exact_integers_match_independent_loop_nest(dtype):
 @pytest.mark.parametrize("dtype", BOTH)
 def test_real_inputs_within_dot_product_bound_of_exact(dtype):
     N, M = 12, 50
-    A = I.uniform_f64(N, M, seed=5) if dtype == O.DTYPE_F64 else I.normal_bf16(N, M, seed=5)
+    A = I.uniform_f64(N, M, seed=5) if dtype == O.DTYPE_F64 else real_inputs(N, M, 5, dtype)
     Af = widen(A, dtype)
     G = exact_gram_by_outer_products(Af)
     ref, bound = O.syrk_lower(A, None, 1.0, 0.0, dtype)
@@ -120,7 +132,7 @@ def test_row_reversal_symmetry(dtype):
     """(P A)(P A)^T = P (A A^T) P^T: entry (i, j) of the reversed problem equals
     entry (N-1-j, N-1-i) of the original, bit for bit (products commute exactly)."""
     N, M = 19, 33
-    A = I.normal_f64(N, M, 3) if dtype == O.DTYPE_F64 else I.normal_bf16(N, M, 3)
+    A = real_inputs(N, M, 3, dtype)
     ref, _ = O.syrk_lower(A, None, 1.0, 0.0, dtype)
     rev, _ = O.syrk_lower(np.ascontiguousarray(A[::-1]), None, 1.0, 0.0, dtype)
     for i in range(N):
@@ -159,7 +171,7 @@ def test_bf16_widening_bit_patterns():
 @pytest.mark.parametrize("dtype", BOTH)
 def test_leading_dimensions_and_entry_list(dtype):
     N, M, lda, ldc = 13, 21, 32, 20
-    big = I.small_int_f64(N, lda, 4) if dtype == O.DTYPE_F64 else I.small_int_bf16(N, lda, 4)
+    big = {O.DTYPE_F64: I.small_int_f64, O.DTYPE_BF16_F32: I.small_int_bf16, O.DTYPE_TF32_F32: I.small_int_f32}[dtype](N, lda, 4)
     A = big[:, :M]                                           # row pitch lda > M
     Cbig = I.random_c(N, 6, dtype, ldc)
     Cin = Cbig[:, :N]
@@ -171,6 +183,21 @@ def test_leading_dimensions_and_entry_list(dtype):
     assert np.array_equal(r3, lower(ref)) and np.array_equal(b3, lower(bound))
     with pytest.raises(ValueError):
         O.syrk_entries([0], [1], A, Cin, 1.0, 0.0, dtype)    # upper-triangle entry refused
+
+
+def test_tf32_reading_drops_the_13_low_order_bits():
+    """TF32 keeps 10 fraction bits.  1 + 2^-10 survives; 1 + 2^-11 + 2^-12 (0.75 ulp above 1) and
+    1 + 2^-10 - 2^-23 (just below the next TF32 value) are cut down, not rounded up; signs follow."""
+    x = np.array([[1.0 + 2.0 ** -10, 1.0 + 2.0 ** -11 + 2.0 ** -12, -(1.0 + 2.0 ** -10 - 2.0 ** -23), 3.0]],
+                 dtype=np.float32)
+    ref, bound = O.syrk_lower(x, None, 1.0, 0.0, O.DTYPE_TF32_F32)
+    assert ref[0, 0] == (1.0 + 2.0 ** -10) ** 2 + 1.0 + 1.0 + 9.0
+    assert bound[0, 0] == ref[0, 0]
+    two = np.array([[1.0 + 2.0 ** -11 + 2.0 ** -12], [-(1.0 + 2.0 ** -10 - 2.0 ** -23)]], dtype=np.float32)
+    ref, bound = O.syrk_lower(two, None, 1.0, 0.0, O.DTYPE_TF32_F32)
+    assert ref[1, 0] == -1.0 and bound[1, 0] == 1.0
+    kept = I.f32_keep_tf32_bits(x)
+    assert list(kept[0]) == [np.float32(1.0 + 2.0 ** -10), 1.0, -1.0, 3.0]
 
 
 def test_bf16_rounding_of_inputs_is_nearest_even():
