@@ -31,6 +31,12 @@ extern "C" {
 /* dtype argument */
 #define SYRK_DTYPE_F64      0  /* A and C binary64; binary64 accumulation (DMMA)          */
 #define SYRK_DTYPE_BF16_F32 1  /* A bfloat16, C binary32; binary32 accumulation (tcgen05) */
+#define SYRK_DTYPE_TF32_F32 2  /* A binary32 read as TF32 (sign, exponent and the 10 leading
+                                  fraction bits: the 13 low-order bits of every element are
+                                  ignored), C binary32; binary32 accumulation (tcgen05
+                                  kind::tf32).  The paper fixes no input precision; this is
+                                  the same update on FP32 data.  syrk_lower_tn takes this
+                                  type through the plain-load kernel only.                */
 
 /* return codes */
 #define SYRK_OK                 0

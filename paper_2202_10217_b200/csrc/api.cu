@@ -15,7 +15,7 @@ namespace {
 
 int validate(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, int dtype,
              bool a_is_m_by_n = false) {
-    if (dtype != SYRK_DTYPE_F64 && dtype != SYRK_DTYPE_BF16_F32) return SYRK_ERR_DTYPE;
+    if (!known_dtype(dtype)) return SYRK_ERR_DTYPE;
     if (N < 0 || M < 0 || N >= (int64_t(1) << 31) - 256 || M >= (int64_t(1) << 31) - 256) return SYRK_ERR_SIZE;
     if (N == 0) return SYRK_OK;
     if (lda < std::max<int64_t>(1, a_is_m_by_n ? N : M) || ldc < N) return SYRK_ERR_LD;
@@ -23,8 +23,8 @@ int validate(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t 
     return SYRK_OK;
 }
 
-size_t a_elem(int dtype) { return dtype == SYRK_DTYPE_F64 ? 8 : 2; }
-size_t c_elem(int dtype) { return dtype == SYRK_DTYPE_F64 ? 8 : 4; }
+size_t a_elem(int dtype) { return a_elem_size(dtype); }
+size_t c_elem(int dtype) { return c_elem_size(dtype); }
 
 bool tma_ok(const void* A, int64_t lda, int dtype) {
     return (reinterpret_cast<uintptr_t>(A) & 15) == 0 && (size_t(lda) * a_elem(dtype)) % 16 == 0;
@@ -77,7 +77,8 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         if (beta == 1.0) return SYRK_OK;
         return launch_scale_lower(dtype, N, C, ldc, beta, stream) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
     }
-    if (!tma_ok(A, lda, dtype))
+    // TF32 inputs stored M x N have no tensor-core path (MN-major TF32 operands are not used here).
+    if (!tma_ok(A, lda, dtype) || (a_is_m_by_n && dtype == SYRK_DTYPE_TF32_F32))
         return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
     DevicePlan* dp = nullptr;
@@ -118,7 +119,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
                            encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
         e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
                              float(beta), split, ds->d_partial, dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, a_is_m_by_n,
-                             ds->d_status, ds->sm_count, stream);
+                             dtype == SYRK_DTYPE_TF32_F32, ds->d_status, ds->sm_count, stream);
     }
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
@@ -224,7 +225,7 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
 }
 
 int syrk_plan_prepare(int64_t N, int64_t M, int dtype) {
-    if (dtype != SYRK_DTYPE_F64 && dtype != SYRK_DTYPE_BF16_F32) return SYRK_ERR_DTYPE;
+    if (!known_dtype(dtype)) return SYRK_ERR_DTYPE;
     if (N < 0 || M < 0) return SYRK_ERR_SIZE;
     if (N == 0) return SYRK_OK;
     std::lock_guard<std::mutex> lock(runtime().mu);
@@ -234,7 +235,7 @@ int syrk_plan_prepare(int64_t N, int64_t M, int dtype) {
     DevicePlan* dp = nullptr;
     rc = get_device_plan(ds, N, dtype, &dp);
     if (rc != SYRK_OK) return rc;
-    if (dtype == SYRK_DTYPE_BF16_F32) {
+    if (is_tcgen05_dtype(dtype)) {
         const KernelShape ks = kernel_shape(dtype);
         const int split = pick_split_k(ds, dp, M, ks.bk);
         if (split > 1) {
@@ -306,7 +307,7 @@ int syrk_set_split_k(int slices) {
 
 int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats* out) {
     if (!out) return SYRK_ERR_NULL;
-    if (dtype != SYRK_DTYPE_F64 && dtype != SYRK_DTYPE_BF16_F32) return SYRK_ERR_DTYPE;
+    if (!known_dtype(dtype)) return SYRK_ERR_DTYPE;
     if (N < 0 || M < 0) return SYRK_ERR_SIZE;
     int schedule, forced_split;
     { std::lock_guard<std::mutex> lock(runtime().mu); schedule = runtime().schedule; forced_split = runtime().split_k; }
@@ -318,7 +319,7 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->tile = ks.tile;
     out->k = ks.k;
     out->c = int32_t(plan.c_top);
-    out->split_k = (dtype == SYRK_DTYPE_BF16_F32 && M > 0)
+    out->split_k = (is_tcgen05_dtype(dtype) && M > 0)
                        ? auto_split_k(plan.items, M, ks.bk, 148, forced_split) : 1;
     out->n_tiles = plan.p.n_tiles;
     out->items = int64_t(plan.items.size());
@@ -331,7 +332,7 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->c_elems = N * (N + 1) / 2;
     out->s_acc = ks.s_acc;
     out->s_total = ks.s_acc + int64_t(kMaxSeg) * ks.tile * ks.bk * ks.stages;
-    if (dtype == SYRK_DTYPE_BF16_F32) out->s_total = ks.s_acc + int64_t(bf16_seg_slots()) * ks.tile * ks.bk * ks.stages;
+    if (is_tcgen05_dtype(dtype)) out->s_total = ks.s_acc + int64_t(bf16_seg_slots()) * ks.tile * ks.bk * ks.stages;
     return SYRK_OK;
 }
 

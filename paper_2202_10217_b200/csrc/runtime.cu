@@ -26,8 +26,9 @@ KernelShape kernel_shape(int dtype) {
     } else {
         // 128-row segments, three per pipeline stage and three 128 x 128 FP32 accumulators in
         // TMEM: a triangle block with k = 3, or a 1 x 2 rectangle, or two diagonal tile rows.
+        // A stage row is 128 bytes: 64 bfloat16 or 32 binary32 (TF32) columns.
         s.tile = bf16_tile(); s.k = 3; s.rect_rows = 1; s.rect_cols = 2; s.diag_side = 2;
-        s.bk = bf16_bk(); s.stages = bf16_stages();
+        s.bk = (dtype == SYRK_DTYPE_TF32_F32) ? bf16_bk() / 2 : bf16_bk(); s.stages = bf16_stages();
         s.s_acc = int64_t(3) * s.tile * s.tile;
     }
     return s;
@@ -98,7 +99,7 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
         const int max_tile = (dtype == SYRK_DTYPE_F64) ? kMaxTile : 3;
         for (const WorkItem& it : dp.plan.items) {
             if (it.n_seg > max_seg || it.n_tile > max_tile) return SYRK_ERR_PLAN;
-            if (dtype == SYRK_DTYPE_BF16_F32) {   // TMEM layout: at most one lone tile and one adjacent pair
+            if (is_tcgen05_dtype(dtype)) {   // TMEM layout: at most one lone tile and one adjacent pair
                 int lone = 0, pairs = 0;
                 for (int t = 0; t < it.n_tile;) {
                     const bool pair = t + 1 < it.n_tile && it.tile_x[t + 1] == it.tile_x[t] &&
@@ -110,7 +111,7 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
             }
         }
         std::vector<int64_t> cta_begin;
-        if (dtype == SYRK_DTYPE_BF16_F32 && !dp.plan.items.empty()) {
+        if (is_tcgen05_dtype(dtype) && !dp.plan.items.empty()) {
             // Persistent kernel: items go to thread blocks (one per SM) longest first, each to the
             // block with the least work so far.  The kernel is bound by shared-memory traffic, so
             // an item costs, per K-step, 16 KB per segment written by TMA plus the operand reads of
@@ -203,13 +204,15 @@ int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, i
                          int64_t lda, int box_rows, int box_cols) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return SYRK_ERR_CUDA;
-    const size_t es = (dtype == SYRK_DTYPE_F64) ? 8 : 2;
+    const size_t es = a_elem_size(dtype);
     const cuuint64_t dims[2] = {cuuint64_t(M), cuuint64_t(N)};
     const cuuint64_t strides[1] = {cuuint64_t(lda) * es};
     const cuuint32_t box[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
+    // TF32 operands travel as plain binary32 (bits untouched; the tensor core ignores the low 13).
     const CUtensorMapDataType dt =
-        (dtype == SYRK_DTYPE_F64) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+        (dtype == SYRK_DTYPE_F64) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64
+        : (dtype == SYRK_DTYPE_TF32_F32) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUresult r = fn(tm, dt, 2, const_cast<void*>(A), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

@@ -17,6 +17,11 @@ template <> struct Widen<__nv_bfloat16, float> {
     static __device__ float get(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 };
 
+// binary32 read as TF32: the 13 low-order bits of the encoding are dropped.
+template <> struct Widen<float, float> {
+    static __device__ float get(const float* p) { return __uint_as_float(__float_as_uint(*p) & 0xFFFFE000u); }
+};
+
 template <typename TA, typename TC>
 __global__ void syrk_plain_kernel(int64_t N, int64_t M, const TA* __restrict__ A, int64_t row_stride,
                                   int64_t col_stride, TC* __restrict__ C, int64_t ldc, TC alpha, TC beta) {
@@ -55,6 +60,9 @@ cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, in
     if (dtype == 0)
         syrk_plain_kernel<double, double><<<grid2d(N, block), block, 0, stream>>>(
             N, M, static_cast<const double*>(A), rs, cs, static_cast<double*>(C), ldc, alpha, beta);
+    else if (dtype == 2)
+        syrk_plain_kernel<float, float><<<grid2d(N, block), block, 0, stream>>>(
+            N, M, static_cast<const float*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));
     else
         syrk_plain_kernel<__nv_bfloat16, float><<<grid2d(N, block), block, 0, stream>>>(
             N, M, static_cast<const __nv_bfloat16*>(A), rs, cs, static_cast<float*>(C), ldc,

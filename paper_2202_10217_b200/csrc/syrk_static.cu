@@ -125,6 +125,6 @@ extern "C" int syrk_lower_bf16_static(int64_t N, int64_t M, const void* A, int64
     if (rc != SYRK_OK) return rc;
     const cudaError_t e = launch_syrk_bf16(tm, nullptr, a->items, n_items, N, M, static_cast<float*>(C), ldc,
                                            float(alpha), float(beta), slices, a->partial, a->tile_base,
-                                           total_tiles, nullptr, 0, 0, a->status, a->sm_count, st);
+                                           total_tiles, nullptr, 0, 0, 0, a->status, a->sm_count, st);
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }

@@ -14,15 +14,16 @@ SENTINEL = {np.dtype(np.float64): 0x7FF8DEADBEEF1234, np.dtype(np.float32): 0x7F
 
 
 def a_to_device(A: np.ndarray, dtype: int, lda: int | None = None, offset_elems: int = 0):
-    """Upload A (float64, or uint16 bf16 bits) with row pitch lda; returns (tensor_keepalive, ptr)."""
+    """Upload A (float64, uint16 bf16 bits, or float32 for TF32) with row pitch lda; returns
+    (tensor_keepalive, ptr)."""
     N, M = A.shape
     lda = max(M, 1) if lda is None else lda
-    tdt = torch.float64 if dtype == B.DTYPE_F64 else torch.bfloat16
+    tdt = {B.DTYPE_F64: torch.float64, B.DTYPE_BF16_F32: torch.bfloat16, B.DTYPE_TF32_F32: torch.float32}[dtype]
     buf = torch.zeros(offset_elems + max(N, 1) * lda, dtype=tdt, device="cuda")
     if N and M:
-        host = torch.from_numpy(np.ascontiguousarray(A) if dtype == B.DTYPE_F64
-                                else np.ascontiguousarray(A).view(np.int16))
-        if dtype != B.DTYPE_F64:
+        host = torch.from_numpy(np.ascontiguousarray(A).view(np.int16) if dtype == B.DTYPE_BF16_F32
+                                else np.ascontiguousarray(A))
+        if dtype == B.DTYPE_BF16_F32:
             host = host.view(torch.bfloat16)
         view = buf[offset_elems:offset_elems + N * lda].view(N, lda)
         view[:, :M].copy_(host)

@@ -16,16 +16,18 @@ from paper_2202_10217_b200 import inputs as I
 from gpu_util import assert_within_tolerance, run_case
 
 pytestmark = pytest.mark.gpu
-BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32]
-DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16"])
+BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32]     # every input type of the library
+DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "tf32"])
+A_NUMPY = {B.DTYPE_F64: np.float64, B.DTYPE_BF16_F32: np.uint16, B.DTYPE_TF32_F32: np.float32}
+ALIGN_ELEMS = {B.DTYPE_F64: 2, B.DTYPE_BF16_F32: 8, B.DTYPE_TF32_F32: 4}     # elements per 16 bytes
 
 
 def make_A(N, M, dtype, seed, kind="normal"):
+    """Real-valued TF32 inputs keep their low-order bits: the library must ignore them."""
     if kind == "int":
-        return I.small_int_f64(N, M, seed) if dtype == B.DTYPE_F64 else I.small_int_bf16(N, M, seed)
-    if dtype == B.DTYPE_F64:
-        return I.normal_f64(N, M, seed)
-    return I.normal_bf16(N, M, seed)
+        return {B.DTYPE_F64: I.small_int_f64, B.DTYPE_BF16_F32: I.small_int_bf16,
+                B.DTYPE_TF32_F32: I.small_int_f32}[dtype](N, M, seed)
+    return {B.DTYPE_F64: I.normal_f64, B.DTYPE_BF16_F32: I.normal_bf16, B.DTYPE_TF32_F32: I.normal_f32}[dtype](N, M, seed)
 
 
 # Sizes: below one tile, exact tiles, ragged tails in N and M, several tiles, and sizes
@@ -34,10 +36,12 @@ SIZES_F64 = [(1, 1), (5, 3), (31, 17), (32, 16), (33, 50), (100, 64), (257, 130)
              (1000, 70), (1300, 40)]
 SIZES_BF16 = [(1, 8), (5, 24), (127, 64), (128, 64), (129, 72), (300, 200), (512, 256),
               (777, 136), (1100, 320), (2050, 72)]
+SIZES_TF32 = [(1, 4), (5, 12), (127, 32), (128, 64), (129, 36), (300, 100), (512, 256),
+              (777, 68), (1100, 160), (2050, 44)]
 
 
 def sizes(dtype):
-    return SIZES_F64 if dtype == B.DTYPE_F64 else SIZES_BF16
+    return {B.DTYPE_F64: SIZES_F64, B.DTYPE_BF16_F32: SIZES_BF16, B.DTYPE_TF32_F32: SIZES_TF32}[dtype]
 
 
 @DT
@@ -86,7 +90,7 @@ def test_pitches_and_offsets(dtype):
     N, M = (300, 50) if dtype == B.DTYPE_F64 else (400, 100)
     A = make_A(N, M, dtype, seed=4)
     Cin = I.random_c(N, 5, dtype)
-    step = 2 if dtype == B.DTYPE_F64 else 8           # keeps A 16-byte aligned (TMA path)
+    step = ALIGN_ELEMS[dtype]                         # keeps A 16-byte aligned (TMA path)
     got, ref, bound = run_case(A, dtype, -1.0, 1.0, Cin=Cin, lda=M - M % step + 4 * step, ldc=N + 37,
                                a_offset=3 * step, c_offset=5)
     assert_within_tolerance(got, ref, bound, M, -1.0, 1.0, Cin, dtype)
@@ -97,7 +101,7 @@ def test_unaligned_A_takes_the_plain_kernel(dtype):
     N, M = (150, 33) if dtype == B.DTYPE_F64 else (150, 77)
     A = make_A(N, M, dtype, seed=6)
     Cin = I.random_c(N, 5, dtype)
-    got, ref, bound = run_case(A, dtype, 1.5, 0.5, Cin=Cin, lda=M + (1 if dtype == B.DTYPE_F64 else 3),
+    got, ref, bound = run_case(A, dtype, 1.5, 0.5, Cin=Cin, lda=M + 3,
                                a_offset=1)
     assert_within_tolerance(got, ref, bound, M, 1.5, 0.5, Cin, dtype)
 
@@ -118,7 +122,7 @@ def test_closed_forms(dtype):
 def test_degenerate_sizes(dtype):
     cdt = I.c_storage_dtype(dtype)
     # M == 0: lower triangle <- beta * C
-    A = np.zeros((40, 0), dtype=np.float64 if dtype == B.DTYPE_F64 else np.uint16)
+    A = np.zeros((40, 0), dtype=A_NUMPY[dtype])
     Cin = I.random_c(40, 1, dtype)
     got, _, _ = run_case(A, dtype, 1.0, 2.0, Cin=Cin)
     il = np.tril_indices(40)
@@ -267,3 +271,23 @@ def test_f64_call_inside_stream_capture_replays_correctly():
     ref, _ = O.syrk_lower(A, None, 2.0, 0.0, B.DTYPE_F64)             # two accumulating replays
     il = np.tril_indices(N)
     assert np.array_equal(dC.cpu().numpy()[il], ref[il])
+
+
+def test_tf32_low_order_bits_of_the_inputs_are_ignored():
+    """The tensor core reads the 19 high-order bits of every binary32 input.  With values whose
+    low 13 bits are set the result must equal, bit for bit, the result for the same values with
+    those bits cleared (all products and sums below are exact in binary32)."""
+    N, M = 300, 64
+    rng = np.random.default_rng(77)
+    base = rng.integers(-2, 3, size=(N, M)).astype(np.float32)             # exact in TF32
+    noise = (rng.integers(1, 1 << 13, size=(N, M)).astype(np.uint32))      # only bits 0..12
+    dirty = (base.view(np.uint32) | np.where(base != 0, noise, 0).astype(np.uint32)).view(np.float32)
+    assert np.array_equal(I.f32_keep_tf32_bits(dirty), base) and not np.array_equal(dirty, base)
+    got_dirty, ref, bound = run_case(dirty, B.DTYPE_TF32_F32, 1.0, 0.0)
+    got_clean, _, _ = run_case(base, B.DTYPE_TF32_F32, 1.0, 0.0)
+    il = np.tril_indices(N)
+    assert np.array_equal(got_dirty[il], got_clean[il])
+    assert np.array_equal(got_dirty[il], ref[il])                           # the reference drops them too
+    # the plain-load path (unaligned A) makes the same reading
+    got_plain, _, _ = run_case(dirty, B.DTYPE_TF32_F32, 1.0, 0.0, lda=M + 3, a_offset=1)
+    assert np.array_equal(got_plain[il], ref[il])
