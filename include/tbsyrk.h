@@ -115,6 +115,12 @@ int syrk_lower_tn(int64_t N, int64_t M,
  * pinned; pinned memory copies faster).  The strict upper triangle of the host C is
  * left as it was.  The device and pinned staging buffers are kept by the library
  * (they only grow) and are released by syrk_shutdown().
+ * Large inputs are pipelined: A is uploaded in blocks of columns (multiples of 256,
+ * at least 32 MB each, at most 8) and each block's update
+ * C <- alpha * A_c A_c^T + (beta for the first block, 1 after) * C runs while the next
+ * block is in flight; the result comes back in four bands of rows that are moved into
+ * the caller's C while the next band is copied.  The sum over k is thereby taken block
+ * by block, which stays within the stated tolerance of the one-call result.
  */
 int syrk_lower_host(int64_t N, int64_t M,
                     const void* A, int64_t lda,

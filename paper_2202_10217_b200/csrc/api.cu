@@ -126,14 +126,17 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
 
 namespace {
 
-// Lower triangle of C (row pitch ldc) -> packed rows (row i has i+1 entries), on device.
+// Rows row0 .. row1 - 1 of the lower triangle of C (row pitch ldc) -> packed rows (row
+// i has i + 1 entries and starts at element i (i + 1) / 2), on device.
 template <typename T>
-__global__ void pack_lower_kernel(int64_t N, const T* __restrict__ C, int64_t ldc, T* __restrict__ packed) {
-    const int64_t i = blockIdx.y;
-    const T* src = C + i * ldc;
-    T* dst = packed + i * (i + 1) / 2;
-    for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j <= i; j += int64_t(gridDim.x) * blockDim.x)
-        dst[j] = src[j];
+__global__ void pack_lower_kernel(int64_t row0, int64_t row1, const T* __restrict__ C, int64_t ldc,
+                                  T* __restrict__ packed) {
+    for (int64_t i = row0 + blockIdx.y; i < row1; i += gridDim.y) {
+        const T* src = C + i * ldc;
+        T* dst = packed + i * (i + 1) / 2;
+        for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j <= i; j += int64_t(gridDim.x) * blockDim.x)
+            dst[j] = src[j];
+    }
 }
 
 }  // namespace
@@ -164,11 +167,15 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     DeviceState* ds = nullptr;
     rc = get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
-    if (!ds->host_stream && cudaStreamCreateWithFlags(&ds->host_stream, cudaStreamNonBlocking) != cudaSuccess) {
-        cudaGetLastError();
-        return SYRK_ERR_CUDA;
+    constexpr int kMaxChunks = 8, kBands = 4;
+    if (!ds->host_stream) {
+        bool ok = cudaStreamCreateWithFlags(&ds->host_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&ds->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; ok && i < kMaxChunks; ++i)
+            ok = cudaEventCreateWithFlags(&ds->host_events[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); return SYRK_ERR_CUDA; }
     }
-    cudaStream_t st = ds->host_stream;
+    cudaStream_t st = ds->host_stream, cp = ds->copy_stream;
     const size_t ea = a_elem(dtype), ec = c_elem(dtype);
     // device pitch of A rounded up so that the TMA path applies to any M
     const int64_t dlda = (std::max<int64_t>(M, 1) * int64_t(ea) + 15) / 16 * 16 / int64_t(ea);
@@ -178,46 +185,79 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     if ((rc = ensure_device_bytes(&ds->d_c, &ds->d_c_bytes, size_t(N) * dldc * ec)) != SYRK_OK) return rc;
     if ((rc = ensure_device_bytes(&ds->d_packed, &ds->d_packed_bytes, packed_bytes)) != SYRK_OK) return rc;
     if ((rc = ensure_pinned_bytes(&ds->h_packed, &ds->h_packed_bytes, packed_bytes)) != SYRK_OK) return rc;
-    bool ok = true;
-    if (M > 0)
-        ok = ok && cudaMemcpy2DAsync(ds->d_a, dlda * ea, A, lda * ea, M * ea, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (beta != 0.0)
-        ok = ok && cudaMemcpy2DAsync(ds->d_c, dldc * ec, C, ldc * ec, N * ec, N, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return SYRK_ERR_CUDA; }
-    rc = syrk_run_device(N, M, ds->d_a, dlda, ds->d_c, dldc, alpha, beta, dtype, st);
-    if (rc != SYRK_OK) return rc;
-    const dim3 grid(unsigned(std::min<int64_t>(64, (N + 255) / 256)), unsigned(N));
-    if (dtype == SYRK_DTYPE_F64)
-        pack_lower_kernel<double><<<grid, 256, 0, st>>>(N, static_cast<const double*>(ds->d_c), dldc,
-                                                        static_cast<double*>(ds->d_packed));
-    else
-        pack_lower_kernel<float><<<grid, 256, 0, st>>>(N, static_cast<const float*>(ds->d_c), dldc,
-                                                       static_cast<float*>(ds->d_packed));
-    ok = cudaGetLastError() == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(ds->h_packed, ds->d_packed, packed_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return SYRK_ERR_CUDA; }
-    // Packed rows -> the caller's lower triangle, on a few host threads with equal byte shares
-    // (row i starts at element i(i+1)/2, so thread t gets rows up to N * sqrt((t+1)/T)).
-    {
+    auto chk = [](cudaError_t e) { if (e != cudaSuccess) { cudaGetLastError(); return false; } return true; };
+
+    // Upload and compute overlap: A goes up in column blocks on the copy stream and each block's
+    // rank-update C <- alpha A_c A_c^T + (beta or 1) C runs on the compute stream as soon as its
+    // block has landed.  Blocks are multiples of 256 columns (16-byte aligned for every dtype, whole
+    // pipeline stages) and at least 32 MB of A each, so short inputs stay one call.
+    int64_t n_chunks = 1;
+    if (M > 0) {
+        const size_t a_bytes = size_t(N) * size_t(M) * ea;
+        n_chunks = std::max<int64_t>(1, std::min<int64_t>({int64_t(kMaxChunks), int64_t(a_bytes >> 25), M / 256}));
+    }
+    const int64_t chunk_cols = M > 0 ? ((M + n_chunks - 1) / n_chunks + 255) / 256 * 256 : 0;
+    if (beta != 0.0 && !chk(cudaMemcpy2DAsync(ds->d_c, dldc * ec, C, ldc * ec, N * ec, N, cudaMemcpyHostToDevice, cp)))
+        return SYRK_ERR_CUDA;
+    if (M == 0) {
+        if (!chk(cudaEventRecord(ds->host_events[0], cp)) || !chk(cudaStreamWaitEvent(st, ds->host_events[0], 0)))
+            return SYRK_ERR_CUDA;
+        rc = syrk_run_device(N, 0, ds->d_a, dlda, ds->d_c, dldc, alpha, beta, dtype, st);
+        if (rc != SYRK_OK) return rc;
+    }
+    for (int64_t c = 0, col0 = 0; col0 < M; ++c, col0 += chunk_cols) {
+        const int64_t cols = std::min<int64_t>(chunk_cols, M - col0);
+        const char* src = static_cast<const char*>(A) + size_t(col0) * ea;
+        char* dst = static_cast<char*>(ds->d_a) + size_t(col0) * ea;
+        if (!chk(cudaMemcpy2DAsync(dst, dlda * ea, src, lda * ea, cols * ea, N, cudaMemcpyHostToDevice, cp)) ||
+            !chk(cudaEventRecord(ds->host_events[c], cp)) || !chk(cudaStreamWaitEvent(st, ds->host_events[c], 0)))
+            return SYRK_ERR_CUDA;
+        rc = syrk_run_device(N, cols, dst, dlda, ds->d_c, dldc, alpha, c == 0 ? beta : 1.0, dtype, st);
+        if (rc != SYRK_OK) return rc;
+    }
+
+    // Download and unpack overlap: the lower triangle comes back packed (row i has i + 1 entries) in
+    // bands of rows of about equal bytes; while band b + 1 is copied, host threads move band b into
+    // the caller's C.
+    int64_t band_row[kBands + 1];
+    for (int b = 0; b <= kBands; ++b) band_row[b] = (b == kBands) ? N : int64_t(double(N) * std::sqrt(double(b) / kBands));
+    for (int b = 0; b < kBands; ++b) {
+        const int64_t r0 = band_row[b], r1 = std::max(band_row[b + 1], band_row[b]);
+        band_row[b + 1] = r1;
+        if (r1 > r0) {
+            const dim3 grid(unsigned(std::min<int64_t>(64, (r1 + 255) / 256)), unsigned(std::min<int64_t>(r1 - r0, 32768)));
+            if (dtype == SYRK_DTYPE_F64)
+                pack_lower_kernel<double><<<grid, 256, 0, st>>>(r0, r1, static_cast<const double*>(ds->d_c), dldc,
+                                                                static_cast<double*>(ds->d_packed));
+            else
+                pack_lower_kernel<float><<<grid, 256, 0, st>>>(r0, r1, static_cast<const float*>(ds->d_c), dldc,
+                                                               static_cast<float*>(ds->d_packed));
+            const size_t off = size_t(r0) * size_t(r0 + 1) / 2 * ec, end = size_t(r1) * size_t(r1 + 1) / 2 * ec;
+            if (!chk(cudaGetLastError()) ||
+                !chk(cudaMemcpyAsync(static_cast<char*>(ds->h_packed) + off, static_cast<char*>(ds->d_packed) + off,
+                                     end - off, cudaMemcpyDeviceToHost, st)))
+                return SYRK_ERR_CUDA;
+        }
+        if (!chk(cudaEventRecord(ds->host_events[b], st))) return SYRK_ERR_CUDA;
+    }
+    const unsigned hw = std::thread::hardware_concurrency();
+    for (int b = 0; b < kBands; ++b) {
+        if (!chk(cudaEventSynchronize(ds->host_events[b]))) return SYRK_ERR_CUDA;
+        const int64_t r0 = band_row[b], r1 = band_row[b + 1];
+        if (r1 <= r0) continue;
         const char* src = static_cast<const char*>(ds->h_packed);
         char* dst = static_cast<char*>(C);
-        const unsigned hw = std::thread::hardware_concurrency();
-        const int T = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(hw ? hw : 1), int64_t(8), N / 256})));
-        auto rows = [=](int64_t r0, int64_t r1) {
-            for (int64_t i = r0; i < r1; ++i)
+        auto rows = [=](int64_t a0, int64_t a1) {
+            for (int64_t i = a0; i < a1; ++i)
                 std::memcpy(dst + size_t(i) * ldc * ec, src + size_t(i) * size_t(i + 1) / 2 * ec, size_t(i + 1) * ec);
         };
+        const int T = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(hw ? hw : 1), int64_t(8), (r1 - r0) / 64})));
         std::vector<std::thread> pool;
-        int64_t r0 = 0;
-        for (int t = 0; t < T; ++t) {
-            const int64_t r1 = (t == T - 1) ? N : int64_t(double(N) * std::sqrt(double(t + 1) / T));
-            if (t == T - 1) rows(r0, r1);
-            else pool.emplace_back(rows, r0, std::max(r0, r1));
-            r0 = std::max(r0, r1);
-        }
+        for (int t = 1; t < T; ++t) pool.emplace_back(rows, r0 + (r1 - r0) * t / T, r0 + (r1 - r0) * (t + 1) / T);
+        rows(r0, r0 + (r1 - r0) / T);
         for (std::thread& th : pool) th.join();
     }
+    if (!chk(cudaStreamSynchronize(st))) return SYRK_ERR_CUDA;
     int flag = 0;
     if (cudaMemcpy(&flag, ds->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
     if (flag != 0) { cudaMemset(ds->d_status, 0, sizeof(int)); return SYRK_ERR_DEVICE_WAIT; }

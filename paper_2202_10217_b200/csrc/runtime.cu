@@ -296,6 +296,8 @@ void release_all() {
         if (ds.d_packed) cudaFree(ds.d_packed);
         if (ds.h_packed) cudaFreeHost(ds.h_packed);
         if (ds.host_stream) cudaStreamDestroy(ds.host_stream);
+        if (ds.copy_stream) cudaStreamDestroy(ds.copy_stream);
+        for (cudaEvent_t ev : ds.host_events) if (ev) cudaEventDestroy(ev);
     }
     rt.devices.clear();
     if (prev >= 0) cudaSetDevice(prev);

@@ -53,7 +53,9 @@ struct DeviceState {
     void* d_c = nullptr; size_t d_c_bytes = 0;
     void* d_packed = nullptr; size_t d_packed_bytes = 0;
     void* h_packed = nullptr; size_t h_packed_bytes = 0;
-    cudaStream_t host_stream = nullptr;
+    cudaStream_t host_stream = nullptr;      // compute stream of the host-buffer entry point
+    cudaStream_t copy_stream = nullptr;      // its upload stream
+    cudaEvent_t host_events[8] = {};         // block-landed / band-ready events of that entry point
     std::map<std::tuple<int64_t, int, int>, DevicePlan> plans;  // (n_tiles, dtype, schedule)
 };
 

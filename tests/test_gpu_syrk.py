@@ -291,3 +291,27 @@ def test_tf32_low_order_bits_of_the_inputs_are_ignored():
     # the plain-load path (unaligned A) makes the same reading
     got_plain, _, _ = run_case(dirty, B.DTYPE_TF32_F32, 1.0, 0.0, lda=M + 3, a_offset=1)
     assert np.array_equal(got_plain[il], ref[il])
+
+
+@DT
+def test_host_buffer_entry_point_pipelined_blocks(dtype):
+    """Inputs large enough for the host entry point to upload A in several column blocks and to
+    bring C back in bands (A > 64 MB), with beta != 0, a ragged last block and host pitches."""
+    N, M = {B.DTYPE_F64: (1500, 9000), B.DTYPE_BF16_F32: (2304, 24000), B.DTYPE_TF32_F32: (1800, 12100)}[dtype]
+    A = make_A(N, M, dtype, seed=51)
+    lda, ldc = M + 16, N + 5
+    Abig = np.zeros((N, lda), dtype=A.dtype)
+    Abig[:, :M] = A
+    Cin = I.random_c(N, 52, dtype, ldc)
+    C = Cin.copy()
+    B.syrk_lower_host(N, M, Abig, lda, C, ldc, 0.5, -1.0, dtype)
+    ii, jj = np.tril_indices(N)
+    pick = np.random.default_rng(53).choice(ii.size, size=20000, replace=False)
+    ii, jj = ii[pick], jj[pick]
+    ref, bound = O.syrk_entries(ii, jj, A, None, 0.5, 0.0, dtype)
+    ref = ref - Cin[ii, jj].astype(np.float64)
+    tol = O.tolerance(M, bound, np.abs(Cin[ii, jj]), 0.5, -1.0, dtype)
+    assert np.all(np.abs(C[ii, jj].astype(np.float64) - ref) <= tol)
+    iu = np.triu_indices(N, 1)
+    assert np.array_equal(C[:, :N][iu], Cin[:, :N][iu])           # strict upper triangle untouched
+    assert np.array_equal(C[:, N:], Cin[:, N:])                   # and the padding columns
