@@ -145,9 +145,9 @@ def run_reference(args, wl: I.Workload, rank: int):
 # captures summarised under profiles/.  Valid only for the kernel source it was taken on.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, sha256 of the kernel source at capture time)
-    "c2_f64_4096x4096": (775_598_848, "43711a695e4e772b7a1952e5503b50c48c2f0088bd49c535efebe3900ce32025"),
-    "c3_bf16_16384x4096": (1_929_455_616, "bdbdbe0287129decd338866798941c9d5382b66f3e0cefd7d9cbb2e9065a3296"),
-    "c4_bf16_2048x262144": (2_859_560_192, "bdbdbe0287129decd338866798941c9d5382b66f3e0cefd7d9cbb2e9065a3296"),
+    "c2_f64_4096x4096": (777_209_088, "de13754c66e41a84278a15bcafeb6e1758756338eb3106d2a42b6f422c6761c4"),
+    "c3_bf16_16384x4096": (1_923_674_112, "e7088eee8b3a4de2d4426963ceffe7d3d18aac3a023a141dff24a45c2e2d4309"),
+    "c4_bf16_2048x262144": (2_854_155_264, "e7088eee8b3a4de2d4426963ceffe7d3d18aac3a023a141dff24a45c2e2d4309"),
 }
 
 
