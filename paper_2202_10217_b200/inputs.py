@@ -6,7 +6,8 @@ and the CPU reference may take their inputs from it.  All generators are numpy
 ``default_rng(seed)`` streams on the host, so the bits do not depend on torch or
 on a GPU.
 
-bf16 values travel as ``uint16`` bit patterns (numpy has no bfloat16 type).
+bf16 values travel as ``uint16`` bit patterns and FP8 E4M3 values as ``uint8`` bytes (numpy has
+neither type).
 """
 from __future__ import annotations
 
@@ -18,6 +19,7 @@ import numpy as np
 DTYPE_F64 = 0        # A, C binary64
 DTYPE_BF16_F32 = 1   # A bfloat16, C binary32 (binary32 accumulation)
 DTYPE_TF32_F32 = 2   # A binary32 read as TF32 (19 high-order bits), C binary32
+DTYPE_E4M3_F32 = 3   # A FP8 E4M3 bytes (uint8), C binary32
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -37,6 +39,28 @@ def f32_keep_tf32_bits(x: np.ndarray) -> np.ndarray:
     """binary32 values with the 13 low-order bits cleared (exactly representable in TF32)."""
     u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32) & np.uint32(0xFFFFE000)
     return u.view(np.float32)
+
+
+def e4m3_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """Decode FP8 E4M3 bytes (1-4-3, bias 7, no infinities, NaN = 0x7F / 0xFF) to binary32 (exact)."""
+    b = np.ascontiguousarray(bits, dtype=np.uint8).astype(np.int32)
+    e, f = (b >> 3) & 15, b & 7
+    mag = np.where(e == 0, np.ldexp(f.astype(np.float32), -9), np.ldexp((8 + f).astype(np.float32), e - 10))
+    mag = np.where((e == 15) & (f == 7), np.float32(np.nan), mag).astype(np.float32)
+    return np.where(b >> 7 == 1, -mag, mag).astype(np.float32)
+
+
+def f32_to_e4m3_bits(x: np.ndarray) -> np.ndarray:
+    """Round binary32 values to FP8 E4M3 (nearest, ties to the even code, saturating at +-448)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    grid = e4m3_bits_to_f32(np.arange(0, 127, dtype=np.uint8)).astype(np.float64)     # codes 0..126: 0..448
+    a = np.minimum(np.abs(x).astype(np.float64), 448.0)
+    hi = np.clip(np.searchsorted(grid, a, side="left"), 0, 126)
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = a - grid[lo], grid[hi] - a
+    take_lo = (d_lo < d_hi) | ((d_lo == d_hi) & (lo % 2 == 0))
+    code = np.where(take_lo, lo, hi).astype(np.uint8)
+    return (code | (np.signbit(x).astype(np.uint8) << 7)).astype(np.uint8)
 
 
 def _normal(rng: np.random.Generator, shape, std: float, chunk_rows: int = 1024) -> np.ndarray:
@@ -74,6 +98,16 @@ def small_int_f32(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.nd
     return np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float32)
 
 
+def normal_e4m3(N: int, M: int, seed: int, std: float = 1.0) -> np.ndarray:
+    """Entries i.i.d. N(0, std^2) rounded to FP8 E4M3; uint8 bytes."""
+    return f32_to_e4m3_bits(_normal(np.random.default_rng(seed), (N, M), std))
+
+
+def small_int_e4m3(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
+    """Integer entries in [lo, hi] as FP8 E4M3 bytes (exactly representable)."""
+    return f32_to_e4m3_bits(np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float32))
+
+
 def small_int_f64(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
     """Integer entries in [lo, hi] stored as binary64 (every partial sum is exact)."""
     return np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float64)
@@ -91,6 +125,8 @@ def ones(N: int, M: int, dtype: int) -> np.ndarray:
         return np.ones((N, M), dtype=np.float64)
     if dtype == DTYPE_TF32_F32:
         return np.ones((N, M), dtype=np.float32)
+    if dtype == DTYPE_E4M3_F32:
+        return f32_to_e4m3_bits(np.ones((N, M), dtype=np.float32))
     return f32_to_bf16_bits(np.ones((N, M), dtype=np.float32))
 
 
@@ -100,6 +136,8 @@ def to_storage(values: np.ndarray, dtype: int) -> np.ndarray:
         return np.ascontiguousarray(values, dtype=np.float64)
     if dtype == DTYPE_TF32_F32:
         return np.ascontiguousarray(values, dtype=np.float32)
+    if dtype == DTYPE_E4M3_F32:
+        return f32_to_e4m3_bits(np.asarray(values, dtype=np.float32))
     return f32_to_bf16_bits(np.asarray(values, dtype=np.float32))
 
 
@@ -134,6 +172,8 @@ class Workload:
             return normal_f64(self.N, self.M, self.seed, self.std)
         if self.dtype == DTYPE_TF32_F32:
             return normal_f32(self.N, self.M, self.seed, self.std)
+        if self.dtype == DTYPE_E4M3_F32:
+            return normal_e4m3(self.N, self.M, self.seed, self.std)
         return normal_bf16(self.N, self.M, self.seed, self.std)
 
     @property

@@ -14,7 +14,7 @@ from oracle import syrk as O
 from paper_2202_10217_b200 import inputs as I
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
-BOTH = [O.DTYPE_F64, O.DTYPE_BF16_F32, O.DTYPE_TF32_F32]      # every input type of the reference
+BOTH = [O.DTYPE_F64, O.DTYPE_BF16_F32, O.DTYPE_TF32_F32, O.DTYPE_E4M3_F32]      # every input type of the reference
 
 
 def lower(x):
@@ -26,6 +26,8 @@ def widen(A, dtype):
         return A
     if dtype == O.DTYPE_TF32_F32:
         return I.f32_keep_tf32_bits(A).astype(np.float64)
+    if dtype == O.DTYPE_E4M3_F32:
+        return I.e4m3_bits_to_f32(A).astype(np.float64)
     return I.bf16_bits_to_f32(A).astype(np.float64)
 
 
@@ -34,6 +36,8 @@ def real_inputs(N, M, seed, dtype):
         return I.normal_f64(N, M, seed)
     if dtype == O.DTYPE_TF32_F32:
         return I.normal_f32(N, M, seed)          # low-order bits set: the reference must drop them
+    if dtype == O.DTYPE_E4M3_F32:
+        return I.normal_e4m3(N, M, seed)
     return I.normal_bf16(N, M, seed)
 
 
@@ -123,8 +127,12 @@ def test_real_inputs_within_dot_product_bound_of_exact(dtype):
         for j in range(i + 1):
             err = abs(Fraction(ref[i, j]) - G[i][j])
             assert err <= Fraction(M * u * 1.01) * Fraction(bound[i, j])
-    # the reference must not be exact-by-construction: some entry does round
-    assert any(Fraction(ref[i, j]) != G[i][j] for i in range(N) for j in range(i + 1))
+    # the reference must not be exact-by-construction: some entry does round.  (FP8 products are
+    # multiples of 2^-18 below 2^18, so their binary64 sums are exact for any M used here.)
+    if dtype == O.DTYPE_E4M3_F32:
+        assert all(Fraction(ref[i, j]) == G[i][j] for i in range(N) for j in range(i + 1))
+    else:
+        assert any(Fraction(ref[i, j]) != G[i][j] for i in range(N) for j in range(i + 1))
 
 
 @pytest.mark.parametrize("dtype", BOTH)
@@ -171,7 +179,8 @@ def test_bf16_widening_bit_patterns():
 @pytest.mark.parametrize("dtype", BOTH)
 def test_leading_dimensions_and_entry_list(dtype):
     N, M, lda, ldc = 13, 21, 32, 20
-    big = {O.DTYPE_F64: I.small_int_f64, O.DTYPE_BF16_F32: I.small_int_bf16, O.DTYPE_TF32_F32: I.small_int_f32}[dtype](N, lda, 4)
+    big = {O.DTYPE_F64: I.small_int_f64, O.DTYPE_BF16_F32: I.small_int_bf16, O.DTYPE_TF32_F32: I.small_int_f32,
+           O.DTYPE_E4M3_F32: I.small_int_e4m3}[dtype](N, lda, 4)
     A = big[:, :M]                                           # row pitch lda > M
     Cbig = I.random_c(N, 6, dtype, ldc)
     Cin = Cbig[:, :N]
@@ -198,6 +207,38 @@ def test_tf32_reading_drops_the_13_low_order_bits():
     assert ref[1, 0] == -1.0 and bound[1, 0] == 1.0
     kept = I.f32_keep_tf32_bits(x)
     assert list(kept[0]) == [np.float32(1.0 + 2.0 ** -10), 1.0, -1.0, 3.0]
+
+
+def test_e4m3_decoding_of_every_byte():
+    """All 256 bytes against the format's definition written out independently: value =
+    (-1)^s * 2^(e-7) * (1 + f/8), subnormals 2^-6 * f/8, 0x7F and 0xFF NaN, extremes 2^-9 and 448.
+    The reference decodes A[i][0]; with a second column of ones... a 1 x 1 product gives value^2,
+    and a 2-row problem gives value * 1."""
+    import math
+    for byte in range(256):
+        s_, e, f = byte >> 7, (byte >> 3) & 15, byte & 7
+        if e == 15 and f == 7:
+            want = math.nan
+        elif e == 0:
+            want = (-1.0) ** s_ * 2.0 ** -6 * (f / 8.0)
+        else:
+            want = (-1.0) ** s_ * 2.0 ** (e - 7) * (1.0 + f / 8.0)
+        A = np.array([[0x38], [byte]], dtype=np.uint8)               # 0x38 = 1.0
+        ref, bound = O.syrk_lower(A, None, 1.0, 0.0, O.DTYPE_E4M3_F32)
+        if math.isnan(want):
+            assert math.isnan(ref[1, 0]) and math.isnan(ref[1, 1]) and ref[0, 0] == 1.0
+        else:
+            assert ref[1, 0] == want and ref[1, 1] == want * want and bound[1, 0] == abs(want)
+    assert O.syrk_lower(np.array([[0x7E]], dtype=np.uint8), None, 1.0, 0.0, O.DTYPE_E4M3_F32)[0][0, 0] == 448.0 ** 2
+    assert O.syrk_lower(np.array([[0x01]], dtype=np.uint8), None, 1.0, 0.0, O.DTYPE_E4M3_F32)[0][0, 0] == 2.0 ** -18
+
+
+def test_e4m3_rounding_of_inputs_is_nearest_even_and_saturating():
+    # between 1.0 (0x38) and 1.125 (0x39): 1.0625 is a tie -> even code 0x38; 1.1875 ties 0x39/0x3A -> 0x3A
+    x = np.array([1.0625, 1.1875, 1.07, 1000.0, -1000.0, 2.0 ** -10, 0.0, -0.0], dtype=np.float32)
+    bits = I.f32_to_e4m3_bits(x)
+    assert list(bits) == [0x38, 0x3A, 0x39, 0x7E, 0xFE, 0x00, 0x00, 0x80]   # 2^-10 ties 0 / 2^-9 -> code 0
+    assert list(I.e4m3_bits_to_f32(bits)[:5]) == [1.0, 1.25, 1.125, 448.0, -448.0]
 
 
 def test_bf16_rounding_of_inputs_is_nearest_even():
