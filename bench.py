@@ -29,9 +29,10 @@ from paper_2202_10217_b200 import inputs as I
 
 METRIC = "syrk_tflops_N(N+1)M"
 UNIT = "TFLOP/s"
-DTYPE_NAME = {I.DTYPE_F64: "f64", I.DTYPE_BF16_F32: "bf16_in_f32_acc", I.DTYPE_TF32_F32: "tf32_in_f32_acc"}
-ELEM_A = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 2, I.DTYPE_TF32_F32: 4}
-ELEM_C = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 4, I.DTYPE_TF32_F32: 4}
+DTYPE_NAME = {I.DTYPE_F64: "f64", I.DTYPE_BF16_F32: "bf16_in_f32_acc", I.DTYPE_TF32_F32: "tf32_in_f32_acc",
+              I.DTYPE_E4M3_F32: "fp8_e4m3_in_f32_acc"}
+ELEM_A = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 2, I.DTYPE_TF32_F32: 4, I.DTYPE_E4M3_F32: 1}
+ELEM_C = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 4, I.DTYPE_TF32_F32: 4, I.DTYPE_E4M3_F32: 4}
 
 
 def measured_peaks():
@@ -191,7 +192,7 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
     N, M, dtype = wl.N, wl.M, wl.dtype
     A_host = wl.make_A()
     cdt = I.c_storage_dtype(dtype)
-    if dtype in (I.DTYPE_F64, I.DTYPE_TF32_F32):
+    if dtype in (I.DTYPE_F64, I.DTYPE_TF32_F32, I.DTYPE_E4M3_F32):
         A_pinned = torch.from_numpy(A_host).pin_memory()
         dA = A_pinned.cuda()
     else:
@@ -262,6 +263,10 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
         peak_note = ("FP64 tensor-core (DMMA) rate measured in this run by the library's register-only "
                      "mma.sync probe; MEASURED_PEAKS.json has no FP64 figure (bf16 %s %.1f x 40/2250 = %.1f)"
                      % (peak_kind, peaks["bf16_tflops"], peaks["bf16_tflops"] * 40.0 / 2250.0))
+    elif dtype == I.DTYPE_E4M3_F32:
+        # no measured FP8 figure: the measured bf16 burst peak times the nominal ratio 4.5 / 2.25 PFLOP/s
+        peak = float(peaks["bf16_tflops"]) * 2.0
+        peak_note = "cuBLAS bf16 burst, MEASURED_PEAKS.json (%s), x nominal fp8/bf16 ratio 2" % peak_kind
     elif dtype == I.DTYPE_TF32_F32:
         # no measured TF32 figure: the measured bf16 burst peak times the nominal ratio 1.1 / 2.25 PFLOP/s
         peak = float(peaks["bf16_tflops"]) * 1.1 / 2.25
@@ -449,7 +454,7 @@ def main():
     ap.add_argument("--lbc-n", type=int, default=32768, help="matrix size of --workload lbc")
     ap.add_argument("--block", type=int, default=0, help="panel width of --workload lbc (0 = library default)")
     ap.add_argument("--shape", default=None,
-                    help="N,M,dtype,alpha,beta (dtype f64|bf16|tf32): a custom seeded N(0,1) workload")
+                    help="N,M,dtype,alpha,beta (dtype f64|bf16|tf32|e4m3): a custom seeded N(0,1) workload")
     ap.add_argument("--kernel-only", action="store_true",
                     help="device-timed kernel steps only (no end-to-end leg, CPU baseline or peak probe); "
                          "for short profiler runs")
@@ -475,7 +480,7 @@ def main():
     wl = I.CONFIGS[args.workload]
     if args.shape:
         n, m, dt, al, be = args.shape.split(",")
-        dtype = {"f64": I.DTYPE_F64, "bf16": I.DTYPE_BF16_F32, "tf32": I.DTYPE_TF32_F32}[dt]
+        dtype = {"f64": I.DTYPE_F64, "bf16": I.DTYPE_BF16_F32, "tf32": I.DTYPE_TF32_F32, "e4m3": I.DTYPE_E4M3_F32}[dt]
         wl = I.Workload("custom_%s_%sx%s" % (dt, n, m), int(n), int(m), dtype, float(al), float(be), 99, "normal")
     if args.impl == "reference":
         run_reference(args, wl, rank)

@@ -37,6 +37,11 @@ extern "C" {
                                   kind::tf32).  The paper fixes no input precision; this is
                                   the same update on FP32 data.  syrk_lower_tn takes this
                                   type through the plain-load kernel only.                */
+#define SYRK_DTYPE_E4M3_F32 3  /* A bytes in the OCP FP8 format E4M3 (1 sign, 4 exponent bits
+                                  with bias 7, 3 fraction bits; no infinities; 0x7F and 0xFF
+                                  are NaN; largest value 448), C binary32; binary32
+                                  accumulation (tcgen05 kind::f8f6f4).  syrk_lower_tn takes
+                                  this type through the plain-load kernel only.           */
 
 /* return codes */
 #define SYRK_OK                 0

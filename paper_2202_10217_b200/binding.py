@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(HERE, "libtbsyrk.so")
 DTYPE_F64 = 0
 DTYPE_BF16_F32 = 1
 DTYPE_TF32_F32 = 2
+DTYPE_E4M3_F32 = 3
 SCHEDULE_TBS = 0
 SCHEDULE_SQUARE = 1
 ITEM_TRI, ITEM_RECT, ITEM_DIAG = 0, 1, 2

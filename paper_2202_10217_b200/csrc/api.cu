@@ -77,8 +77,9 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         if (beta == 1.0) return SYRK_OK;
         return launch_scale_lower(dtype, N, C, ldc, beta, stream) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
     }
-    // TF32 inputs stored M x N have no tensor-core path (MN-major TF32 operands are not used here).
-    if (!tma_ok(A, lda, dtype) || (a_is_m_by_n && dtype == SYRK_DTYPE_TF32_F32))
+    // TF32 and FP8 inputs stored M x N have no tensor-core path (MN-major operands are used for
+    // bfloat16 only).
+    if (!tma_ok(A, lda, dtype) || (a_is_m_by_n && dtype >= SYRK_DTYPE_TF32_F32))
         return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
     DevicePlan* dp = nullptr;
@@ -119,7 +120,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
                            encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
         e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
                              float(beta), split, ds->d_partial, dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, a_is_m_by_n,
-                             dtype == SYRK_DTYPE_TF32_F32, ds->d_status, ds->sm_count, stream);
+                             dtype - SYRK_DTYPE_BF16_F32, ds->d_status, ds->sm_count, stream);
     }
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }

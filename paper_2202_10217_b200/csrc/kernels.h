@@ -34,13 +34,14 @@ int f64_stages();
 // map over C for the asynchronous store path (32 x 32 FP32 boxes, 128-byte swizzle), or null
 // when C does not meet the TMA alignment rules.  With split_k == 1 and `d_cta_begin` given, block b
 // runs items [d_cta_begin[b], d_cta_begin[b+1]) of the list (n_ctas blocks).  `a_is_m_by_n`: A is
-// stored M x N row-major and `tmA` has boxes of 64 rows x 64 columns over that array.  `a_is_tf32`:
-// A holds binary32 values read as TF32 (N x M order only), `tmA` has boxes of 128 rows x 32 columns.
+// stored M x N row-major and `tmA` has boxes of 64 rows x 64 columns over that array.  `a_kind`:
+// 0 bfloat16; 1 binary32 read as TF32 (boxes of 128 rows x 32 columns); 2 FP8 E4M3 bytes (boxes of
+// 128 rows x 128 columns); kinds 1 and 2 in the N x M order only.
 cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                              int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
-                             int a_is_tf32, int* d_status, int sm_count, cudaStream_t stream);
+                             int a_kind, int* d_status, int sm_count, cudaStream_t stream);
 int bf16_tile();
 int bf16_bk();
 int bf16_stages();

@@ -26,9 +26,9 @@ KernelShape kernel_shape(int dtype) {
     } else {
         // 128-row segments, three per pipeline stage and three 128 x 128 FP32 accumulators in
         // TMEM: a triangle block with k = 3, or a 1 x 2 rectangle, or two diagonal tile rows.
-        // A stage row is 128 bytes: 64 bfloat16 or 32 binary32 (TF32) columns.
+        // A stage row is 128 bytes: 64 bfloat16, 32 binary32 (TF32) or 128 FP8 columns.
         s.tile = bf16_tile(); s.k = 3; s.rect_rows = 1; s.rect_cols = 2; s.diag_side = 2;
-        s.bk = (dtype == SYRK_DTYPE_TF32_F32) ? bf16_bk() / 2 : bf16_bk(); s.stages = bf16_stages();
+        s.bk = 128 / int(a_elem_size(dtype)); s.stages = bf16_stages();
         s.s_acc = int64_t(3) * s.tile * s.tile;
     }
     return s;
@@ -212,7 +212,8 @@ int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, i
     // TF32 operands travel as plain binary32 (bits untouched; the tensor core ignores the low 13).
     const CUtensorMapDataType dt =
         (dtype == SYRK_DTYPE_F64) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64
-        : (dtype == SYRK_DTYPE_TF32_F32) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+        : (dtype == SYRK_DTYPE_TF32_F32) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+        : (dtype == SYRK_DTYPE_E4M3_F32) ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUresult r = fn(tm, dt, 2, const_cast<void*>(A), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

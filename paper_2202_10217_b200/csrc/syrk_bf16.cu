@@ -1,6 +1,7 @@
-// BF16-in (or TF32-in) / FP32-accumulate triangle-block SYRK kernel for sm_100a (tcgen05 + TMEM).
-// With binary32 inputs read as TF32 a stage row of 128 bytes holds 32 columns instead of 64 and
-// the MMA is kind::tf32 with K = 8; everything else is shared.
+// BF16-in (or TF32-in, or FP8-E4M3-in) / FP32-accumulate triangle-block SYRK kernel for sm_100a
+// (tcgen05 + TMEM).  A stage row is 128 bytes for every input kind: 64 bfloat16 columns
+// (kind::f16, K = 16 per MMA), 32 binary32 columns read as TF32 (kind::tf32, K = 8) or 128 FP8
+// columns (kind::f8f6f4, K = 32); everything else is shared.
 //
 // Persistent kernel, one thread block per SM, work units dealt round-robin.  A work
 // unit is one item of the tiled TBS schedule (Algorithm 4 / Section 5.1.4 of the
@@ -62,15 +63,27 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]^T, FP32 accumulation, M = 128: BF16 inputs (K = 16 per
-// instruction) or, with kTF32, binary32 inputs read as TF32 (K = 8); 32 bytes of K either way.
-template <bool kTF32>
+// Input kinds of the kernel: what a 128-byte stage row holds and which MMA reads it.
+constexpr int kKindBF16 = 0;    // 64 bfloat16 columns, kind::f16, K = 16 per instruction
+constexpr int kKindTF32 = 1;    // 32 binary32 columns read as TF32, kind::tf32, K = 8
+constexpr int kKindE4M3 = 2;    // 128 FP8 E4M3 columns, kind::f8f6f4, K = 32
+template <int kKind> struct KindCols { static constexpr int value = kKind == kKindBF16 ? 64 : (kKind == kKindTF32 ? 32 : 128); };
+
+// D[tmem] (+)= A[smem] * B[smem]^T, FP32 accumulation, M = 128; 32 bytes of K per instruction for
+// every kind.
+template <int kKind>
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate) {
-    if (kTF32)
+    if (kKind == kKindTF32)
         asm volatile(
             "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
             "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else if (kKind == kKindE4M3)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
             ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
             : "memory");
     else
@@ -121,9 +134,10 @@ __device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
 }
 // Instruction descriptor, kind::f16: D = FP32, A = B = BF16, M = 128; both operands K-major, or
 // both MN-major (bits 15 and 16) when A is stored M x N.
-// kind::tf32 has the same fields with operand format 2 (TF32) in place of 1 (BF16).
-__device__ __forceinline__ uint32_t instr_desc(uint32_t n, bool mn_major, bool tf32) {
-    const uint32_t fmt = tf32 ? 2u : 1u;
+// The other kinds have the same fields; the operand format code is 1 (BF16) for kind::f16,
+// 2 (TF32) for kind::tf32 and 0 (E4M3) for kind::f8f6f4.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, bool mn_major, int kind) {
+    const uint32_t fmt = kind == kKindBF16 ? 1u : (kind == kKindTF32 ? 2u : 0u);
     return (1u << 4) | (fmt << 7) | (fmt << 10) | (mn_major ? (3u << 15) : 0u) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
@@ -176,7 +190,7 @@ __device__ __forceinline__ void layout_of(const WorkItem* it, int n_tile, uint32
     }
 }
 
-template <bool kTN, bool kTF32>
+template <bool kTN, int kKind>
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
                      const WorkItem* __restrict__ items, int64_t n_items, int64_t N, int32_t n_ksteps,
@@ -196,7 +210,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     __shared__ volatile int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    constexpr int kCols = kTF32 ? kBK / 2 : kBK;         // columns of A in a 128-byte stage row
+    constexpr int kCols = KindCols<kKind>::value;        // columns of A in a 128-byte stage row
     const int64_t n_units = n_items * split;
     // This block's units: its own contiguous range of a list ordered block by block on the host,
     // or (K-split calls) every gridDim.x-th unit of the slice-major list.
@@ -273,7 +287,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const int qq = q < L.n_grp ? q : 0;
                     a_lo[q] = (smem_base + uint32_t(L.gx[qq]) * kSegBytes) >> 4;
                     b_lo[q] = (smem_base + uint32_t(L.gy[qq]) * kSegBytes) >> 4;
-                    idesc[q] = instr_desc(uint32_t(L.gn[qq]), kTN, kTF32);
+                    idesc[q] = instr_desc(uint32_t(L.gn[qq]), kTN, kKind);
                     d_addr[q] = tmem_base + L.gcol[qq];
                 }
                 // accumulators of this item must have been drained by the epilogue
@@ -296,7 +310,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     for (int q = 0; q < L.n_grp; ++q) {
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk)
-                            tc_mma<kTF32>(d_addr[q], desc_hi | uint64_t(a_lo[q] + st_off + kk_step * kk),
+                            tc_mma<kKind>(d_addr[q], desc_hi | uint64_t(a_lo[q] + st_off + kk_step * kk),
                                         desc_hi | uint64_t(b_lo[q] + st_off + kk_step * kk), idesc[q],
                                         (kk > 0) ? 1u : first);
                     }
@@ -454,16 +468,17 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                              int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
-                             int a_is_tf32, int* d_status, int sm_count, cudaStream_t stream) {
+                             int a_kind, int* d_status, int sm_count, cudaStream_t stream) {
     // The shared-memory attribute belongs to a device's context: set it once per device.
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[3] = {reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, false>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, false>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, true>)};
+        const void* kernels[4] = {reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>),
+                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindBF16>),
+                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>),
+                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>)};
         for (const void* fn : kernels) {
             cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bf16::kSmemBytes);
             if (e != cudaSuccess) return e;
@@ -471,8 +486,8 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
         configured[dev] = true;
     }
     if (n_items == 0) return cudaSuccess;
-    if (a_is_tf32 && a_is_m_by_n) return cudaErrorInvalidValue;      // no such kernel
-    const int bk = a_is_tf32 ? bf16::kBK / 2 : bf16::kBK;
+    if (a_kind < 0 || a_kind > 2 || (a_kind != 0 && a_is_m_by_n)) return cudaErrorInvalidValue;   // no such kernel
+    const int bk = a_kind == bf16::kKindBF16 ? 64 : (a_kind == bf16::kKindTF32 ? 32 : 128);
     const int32_t n_ksteps = int32_t((M + bk - 1) / bk);
     const int split = split_k < 1 ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
     const int64_t n_units = n_items * split;
@@ -480,8 +495,10 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     const unsigned grid = ranges ? unsigned(n_ctas) : unsigned(n_units < sm_count ? n_units : sm_count);
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0) ? 1 : 0;
     CUtensorMap none{};
-    auto kernel = a_is_tf32 ? bf16::syrk_bf16_tbs_kernel<false, true>
-                  : a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, false> : bf16::syrk_bf16_tbs_kernel<false, false>;
+    auto kernel = a_kind == bf16::kKindTF32 ? bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>
+                  : a_kind == bf16::kKindE4M3 ? bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>
+                  : a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindBF16>
+                                : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>;
     kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
         tmA, tmC ? *tmC : none, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, split,
         d_partial, d_tile_base, total_tiles, ranges ? d_cta_begin : nullptr, d_status);

@@ -22,6 +22,16 @@ template <> struct Widen<float, float> {
     static __device__ float get(const float* p) { return __uint_as_float(__float_as_uint(*p) & 0xFFFFE000u); }
 };
 
+// FP8 E4M3 byte: (-1)^s * 2^(e-7) * (1 + f/8); e = 0: 2^-6 * f/8; e = 15, f = 7: NaN.
+template <> struct Widen<uint8_t, float> {
+    static __device__ float get(const uint8_t* p) {
+        const int b = *p, e = (b >> 3) & 15, f = b & 7;
+        float v = (e == 0) ? ldexpf(float(f), -9) : ldexpf(float(8 + f), e - 10);
+        if (e == 15 && f == 7) v = __int_as_float(0x7FC00000);
+        return (b & 0x80) ? -v : v;
+    }
+};
+
 template <typename TA, typename TC>
 __global__ void syrk_plain_kernel(int64_t N, int64_t M, const TA* __restrict__ A, int64_t row_stride,
                                   int64_t col_stride, TC* __restrict__ C, int64_t ldc, TC alpha, TC beta) {
@@ -60,6 +70,9 @@ cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, in
     if (dtype == 0)
         syrk_plain_kernel<double, double><<<grid2d(N, block), block, 0, stream>>>(
             N, M, static_cast<const double*>(A), rs, cs, static_cast<double*>(C), ldc, alpha, beta);
+    else if (dtype == 3)
+        syrk_plain_kernel<uint8_t, float><<<grid2d(N, block), block, 0, stream>>>(
+            N, M, static_cast<const uint8_t*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));
     else if (dtype == 2)
         syrk_plain_kernel<float, float><<<grid2d(N, block), block, 0, stream>>>(
             N, M, static_cast<const float*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));

@@ -14,11 +14,12 @@ SENTINEL = {np.dtype(np.float64): 0x7FF8DEADBEEF1234, np.dtype(np.float32): 0x7F
 
 
 def a_to_device(A: np.ndarray, dtype: int, lda: int | None = None, offset_elems: int = 0):
-    """Upload A (float64, uint16 bf16 bits, or float32 for TF32) with row pitch lda; returns
+    """Upload A (float64, uint16 bf16 bits, float32 for TF32, or uint8 FP8 bytes) with row pitch lda; returns
     (tensor_keepalive, ptr)."""
     N, M = A.shape
     lda = max(M, 1) if lda is None else lda
-    tdt = {B.DTYPE_F64: torch.float64, B.DTYPE_BF16_F32: torch.bfloat16, B.DTYPE_TF32_F32: torch.float32}[dtype]
+    tdt = {B.DTYPE_F64: torch.float64, B.DTYPE_BF16_F32: torch.bfloat16, B.DTYPE_TF32_F32: torch.float32,
+           B.DTYPE_E4M3_F32: torch.uint8}[dtype]
     buf = torch.zeros(offset_elems + max(N, 1) * lda, dtype=tdt, device="cuda")
     if N and M:
         host = torch.from_numpy(np.ascontiguousarray(A).view(np.int16) if dtype == B.DTYPE_BF16_F32

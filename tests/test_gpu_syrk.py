@@ -16,18 +16,20 @@ from paper_2202_10217_b200 import inputs as I
 from gpu_util import assert_within_tolerance, run_case
 
 pytestmark = pytest.mark.gpu
-BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32]     # every input type of the library
-DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "tf32"])
-A_NUMPY = {B.DTYPE_F64: np.float64, B.DTYPE_BF16_F32: np.uint16, B.DTYPE_TF32_F32: np.float32}
-ALIGN_ELEMS = {B.DTYPE_F64: 2, B.DTYPE_BF16_F32: 8, B.DTYPE_TF32_F32: 4}     # elements per 16 bytes
+BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32]     # every input type of the library
+DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "tf32", "e4m3"])
+A_NUMPY = {B.DTYPE_F64: np.float64, B.DTYPE_BF16_F32: np.uint16, B.DTYPE_TF32_F32: np.float32,
+           B.DTYPE_E4M3_F32: np.uint8}
+ALIGN_ELEMS = {B.DTYPE_F64: 2, B.DTYPE_BF16_F32: 8, B.DTYPE_TF32_F32: 4, B.DTYPE_E4M3_F32: 16}   # elements per 16 bytes
 
 
 def make_A(N, M, dtype, seed, kind="normal"):
     """Real-valued TF32 inputs keep their low-order bits: the library must ignore them."""
     if kind == "int":
         return {B.DTYPE_F64: I.small_int_f64, B.DTYPE_BF16_F32: I.small_int_bf16,
-                B.DTYPE_TF32_F32: I.small_int_f32}[dtype](N, M, seed)
-    return {B.DTYPE_F64: I.normal_f64, B.DTYPE_BF16_F32: I.normal_bf16, B.DTYPE_TF32_F32: I.normal_f32}[dtype](N, M, seed)
+                B.DTYPE_TF32_F32: I.small_int_f32, B.DTYPE_E4M3_F32: I.small_int_e4m3}[dtype](N, M, seed)
+    return {B.DTYPE_F64: I.normal_f64, B.DTYPE_BF16_F32: I.normal_bf16, B.DTYPE_TF32_F32: I.normal_f32,
+            B.DTYPE_E4M3_F32: I.normal_e4m3}[dtype](N, M, seed)
 
 
 # Sizes: below one tile, exact tiles, ragged tails in N and M, several tiles, and sizes
@@ -38,10 +40,13 @@ SIZES_BF16 = [(1, 8), (5, 24), (127, 64), (128, 64), (129, 72), (300, 200), (512
               (777, 136), (1100, 320), (2050, 72)]
 SIZES_TF32 = [(1, 4), (5, 12), (127, 32), (128, 64), (129, 36), (300, 100), (512, 256),
               (777, 68), (1100, 160), (2050, 44)]
+SIZES_E4M3 = [(1, 16), (5, 48), (127, 128), (128, 256), (129, 144), (300, 400), (512, 512),
+              (777, 272), (1100, 640), (2050, 144), (300, 77)]
 
 
 def sizes(dtype):
-    return {B.DTYPE_F64: SIZES_F64, B.DTYPE_BF16_F32: SIZES_BF16, B.DTYPE_TF32_F32: SIZES_TF32}[dtype]
+    return {B.DTYPE_F64: SIZES_F64, B.DTYPE_BF16_F32: SIZES_BF16, B.DTYPE_TF32_F32: SIZES_TF32,
+            B.DTYPE_E4M3_F32: SIZES_E4M3}[dtype]
 
 
 @DT
@@ -297,7 +302,8 @@ def test_tf32_low_order_bits_of_the_inputs_are_ignored():
 def test_host_buffer_entry_point_pipelined_blocks(dtype):
     """Inputs large enough for the host entry point to upload A in several column blocks and to
     bring C back in bands (A > 64 MB), with beta != 0, a ragged last block and host pitches."""
-    N, M = {B.DTYPE_F64: (1500, 9000), B.DTYPE_BF16_F32: (2304, 24000), B.DTYPE_TF32_F32: (1800, 12100)}[dtype]
+    N, M = {B.DTYPE_F64: (1500, 9000), B.DTYPE_BF16_F32: (2304, 24000), B.DTYPE_TF32_F32: (1800, 12100),
+            B.DTYPE_E4M3_F32: (2304, 48000)}[dtype]
     A = make_A(N, M, dtype, seed=51)
     lda, ldc = M + 16, N + 5
     Abig = np.zeros((N, lda), dtype=A.dtype)

@@ -107,9 +107,10 @@ def test_bf16_k_split_in_this_storage_order(split):
     assert_within_tolerance(got, ref, bound, M, 2.0, -1.0, Cin, B.DTYPE_BF16_F32)
 
 
-def test_tf32_inputs_in_this_storage_order_take_the_plain_kernel():
-    N, M = 264, 52
-    A = make_A(N, M, B.DTYPE_TF32_F32, seed=61)
-    Cin = I.random_c(N, 62, B.DTYPE_TF32_F32)
-    got, ref, bound = run_case(A, B.DTYPE_TF32_F32, -1.0, 1.0, Cin, tn=True)
-    assert_within_tolerance(got, ref, bound, M, -1.0, 1.0, Cin, B.DTYPE_TF32_F32)
+@pytest.mark.parametrize("dtype", [B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32], ids=["tf32", "e4m3"])
+def test_tf32_and_fp8_inputs_in_this_storage_order_take_the_plain_kernel(dtype):
+    N, M = 272, 52
+    A = make_A(N, M, dtype, seed=61)
+    Cin = I.random_c(N, 62, dtype)
+    got, ref, bound = run_case(A, dtype, -1.0, 1.0, Cin, tn=True)
+    assert_within_tolerance(got, ref, bound, M, -1.0, 1.0, Cin, dtype)
