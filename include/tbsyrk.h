@@ -123,9 +123,12 @@ int syrk_lower_tn(int64_t N, int64_t M,
  * Large inputs are pipelined: A is uploaded in blocks of columns (multiples of 256,
  * at least 32 MB each, at most 8) and each block's update
  * C <- alpha * A_c A_c^T + (beta for the first block, 1 after) * C runs while the next
- * block is in flight; the result comes back in four bands of rows that are moved into
- * the caller's C while the next band is copied.  The sum over k is thereby taken block
- * by block, which stays within the stated tolerance of the one-call result.
+ * block is in flight; the result comes back in up to 16 bands of rows: the rectangle left
+ * of a band's diagonal block is copied straight into the caller's C, the diagonal blocks'
+ * lower triangles come back packed and are put in place by the host meanwhile (with a
+ * pageable C the whole triangle comes back packed and host threads unpack it).  The sum
+ * over k is thereby taken block by block, which stays within the stated tolerance of the
+ * one-call result.
  */
 int syrk_lower_host(int64_t N, int64_t M,
                     const void* A, int64_t lda,

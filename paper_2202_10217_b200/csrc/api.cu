@@ -127,15 +127,19 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
 
 namespace {
 
-// Rows row0 .. row1 - 1 of the lower triangle of C (row pitch ldc) -> packed rows (row
-// i has i + 1 entries and starts at element i (i + 1) / 2), on device.
+// Rows [row0, row1) of the lower triangles of the diagonal blocks of side band_h of C (row pitch
+// ldc), packed: block b
+// starts at element b * band_h (band_h + 1) / 2 and its local row l has l + 1 entries starting at
+// l (l + 1) / 2.
 template <typename T>
-__global__ void pack_lower_kernel(int64_t row0, int64_t row1, const T* __restrict__ C, int64_t ldc,
-                                  T* __restrict__ packed) {
+__global__ void pack_diag_blocks_kernel(int64_t row0, int64_t row1, int64_t band_h, const T* __restrict__ C,
+                                        int64_t ldc, T* __restrict__ packed) {
+    const int64_t full = band_h * (band_h + 1) / 2;
     for (int64_t i = row0 + blockIdx.y; i < row1; i += gridDim.y) {
-        const T* src = C + i * ldc;
-        T* dst = packed + i * (i + 1) / 2;
-        for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j <= i; j += int64_t(gridDim.x) * blockDim.x)
+        const int64_t b = i / band_h, l = i - b * band_h;
+        const T* src = C + i * ldc + b * band_h;
+        T* dst = packed + b * full + l * (l + 1) / 2;
+        for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j <= l; j += int64_t(gridDim.x) * blockDim.x)
             dst[j] = src[j];
     }
 }
@@ -168,7 +172,7 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     DeviceState* ds = nullptr;
     rc = get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
-    constexpr int kMaxChunks = 8, kBands = 4;
+    constexpr int kMaxChunks = 8, kBands = 16;
     if (!ds->host_stream) {
         bool ok = cudaStreamCreateWithFlags(&ds->host_stream, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaStreamCreateWithFlags(&ds->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
@@ -181,7 +185,13 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     // device pitch of A rounded up so that the TMA path applies to any M
     const int64_t dlda = (std::max<int64_t>(M, 1) * int64_t(ea) + 15) / 16 * 16 / int64_t(ea);
     const int64_t dldc = (N + 1) / 2 * 2;
-    const size_t packed_bytes = size_t(N) * size_t(N + 1) / 2 * ec;
+    // packed lower triangles of the diagonal blocks of the download bands (see below)
+    cudaPointerAttributes c_attr{};
+    const bool c_pinned = cudaPointerGetAttributes(&c_attr, C) == cudaSuccess && c_attr.type == cudaMemoryTypeHost;
+    cudaGetLastError();
+    const int64_t pk_bands = c_pinned ? std::max<int64_t>(1, std::min<int64_t>(kBands, N / 256)) : 1;
+    const int64_t pk_h = (N + pk_bands - 1) / pk_bands;
+    const size_t packed_bytes = size_t(pk_bands) * size_t(pk_h) * size_t(pk_h + 1) / 2 * ec;
     if ((rc = ensure_device_bytes(&ds->d_a, &ds->d_a_bytes, size_t(N) * dlda * ea)) != SYRK_OK) return rc;
     if ((rc = ensure_device_bytes(&ds->d_c, &ds->d_c_bytes, size_t(N) * dldc * ec)) != SYRK_OK) return rc;
     if ((rc = ensure_device_bytes(&ds->d_packed, &ds->d_packed_bytes, packed_bytes)) != SYRK_OK) return rc;
@@ -217,46 +227,89 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
         if (rc != SYRK_OK) return rc;
     }
 
-    // Download and unpack overlap: the lower triangle comes back packed (row i has i + 1 entries) in
-    // bands of rows of about equal bytes; while band b + 1 is copied, host threads move band b into
-    // the caller's C.
-    int64_t band_row[kBands + 1];
-    for (int b = 0; b <= kBands; ++b) band_row[b] = (b == kBands) ? N : int64_t(double(N) * std::sqrt(double(b) / kBands));
-    for (int b = 0; b < kBands; ++b) {
-        const int64_t r0 = band_row[b], r1 = std::max(band_row[b + 1], band_row[b]);
-        band_row[b + 1] = r1;
-        if (r1 > r0) {
-            const dim3 grid(unsigned(std::min<int64_t>(64, (r1 + 255) / 256)), unsigned(std::min<int64_t>(r1 - r0, 32768)));
-            if (dtype == SYRK_DTYPE_F64)
-                pack_lower_kernel<double><<<grid, 256, 0, st>>>(r0, r1, static_cast<const double*>(ds->d_c), dldc,
-                                                                static_cast<double*>(ds->d_packed));
-            else
-                pack_lower_kernel<float><<<grid, 256, 0, st>>>(r0, r1, static_cast<const float*>(ds->d_c), dldc,
-                                                               static_cast<float*>(ds->d_packed));
-            const size_t off = size_t(r0) * size_t(r0 + 1) / 2 * ec, end = size_t(r1) * size_t(r1 + 1) / 2 * ec;
-            if (!chk(cudaGetLastError()) ||
-                !chk(cudaMemcpyAsync(static_cast<char*>(ds->h_packed) + off, static_cast<char*>(ds->d_packed) + off,
-                                     end - off, cudaMemcpyDeviceToHost, st)))
+    // Download: C is cut into bands of `band_h` rows.  The part of a band left of its diagonal block
+    // (rows [r0, r1) x columns [0, r0)) is a rectangle below the diagonal and is copied straight into
+    // the caller's C; the diagonal blocks' lower triangles (a few percent of the entries) come back
+    // packed and are put in place by the host while the rectangles are still being copied.
+    // (Copying straight into C pays only when C is page-locked; otherwise there is one band, i.e.
+    // the whole triangle comes back packed as one block.)
+    const int64_t n_bands = pk_bands;
+    const int64_t band_h = pk_h;
+    auto pack_rows = [&](int64_t r0, int64_t r1) {
+        const dim3 grid(unsigned(std::min<int64_t>(64, (band_h + 255) / 256)), unsigned(std::min<int64_t>(r1 - r0, 32768)));
+        if (dtype == SYRK_DTYPE_F64)
+            pack_diag_blocks_kernel<double><<<grid, 256, 0, st>>>(r0, r1, band_h, static_cast<const double*>(ds->d_c), dldc,
+                                                                  static_cast<double*>(ds->d_packed));
+        else
+            pack_diag_blocks_kernel<float><<<grid, 256, 0, st>>>(r0, r1, band_h, static_cast<const float*>(ds->d_c), dldc,
+                                                                 static_cast<float*>(ds->d_packed));
+        return cudaGetLastError() == cudaSuccess;
+    };
+    const char* psrc = static_cast<const char*>(ds->h_packed);
+    char* pdst = static_cast<char*>(C);
+    const size_t full = size_t(band_h) * size_t(band_h + 1) / 2;              // entries of a full diagonal block
+    auto unpack_rows = [=](int64_t i0, int64_t i1) {
+        for (int64_t i = i0; i < i1; ++i) {
+            const int64_t bnd = i / band_h, l = i - bnd * band_h;
+            std::memcpy(pdst + (size_t(i) * ldc + size_t(bnd) * band_h) * ec,
+                        psrc + (size_t(bnd) * full + size_t(l) * size_t(l + 1) / 2) * ec, size_t(l + 1) * ec);
+        }
+    };
+    const unsigned hw = std::thread::hardware_concurrency();
+    auto unpack_parallel = [&](int64_t i0, int64_t i1, size_t bytes, bool by_bytes) {
+        // a few host threads, about 4 MB each; `by_bytes`: shares of equal bytes of a triangle's rows
+        const int T = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(hw ? hw : 1), int64_t(8), int64_t(bytes >> 22)})));
+        std::vector<std::thread> pool;
+        int64_t lo = i0;
+        for (int t = 0; t < T; ++t) {
+            int64_t hi = i0 + (i1 - i0) * (t + 1) / T;
+            if (by_bytes) hi = int64_t(std::sqrt(double(i0) * i0 + (double(i1) * i1 - double(i0) * i0) * (t + 1) / T));
+            if (t == T - 1) hi = i1;
+            hi = std::min(std::max(hi, lo), i1);
+            if (t == T - 1) unpack_rows(lo, hi);
+            else pool.emplace_back(unpack_rows, lo, hi);
+            lo = hi;
+        }
+        for (std::thread& th : pool) th.join();
+    };
+    if (n_bands > 1) {
+        // page-locked C: diagonal blocks packed (one copy), rectangles copied in place
+        if (!pack_rows(0, N) ||
+            !chk(cudaMemcpyAsync(ds->h_packed, ds->d_packed, packed_bytes, cudaMemcpyDeviceToHost, st)) ||
+            !chk(cudaEventRecord(ds->host_events[0], st)))
+            return SYRK_ERR_CUDA;
+        for (int64_t r0 = band_h; r0 < N; r0 += band_h) {
+            const int64_t r1 = std::min(N, r0 + band_h);
+            if (!chk(cudaMemcpy2DAsync(static_cast<char*>(C) + size_t(r0) * ldc * ec, size_t(ldc) * ec,
+                                       static_cast<const char*>(ds->d_c) + size_t(r0) * dldc * ec, size_t(dldc) * ec,
+                                       size_t(r0) * ec, size_t(r1 - r0), cudaMemcpyDeviceToHost, st)))
                 return SYRK_ERR_CUDA;
         }
-        if (!chk(cudaEventRecord(ds->host_events[b], st))) return SYRK_ERR_CUDA;
-    }
-    const unsigned hw = std::thread::hardware_concurrency();
-    for (int b = 0; b < kBands; ++b) {
-        if (!chk(cudaEventSynchronize(ds->host_events[b]))) return SYRK_ERR_CUDA;
-        const int64_t r0 = band_row[b], r1 = band_row[b + 1];
-        if (r1 <= r0) continue;
-        const char* src = static_cast<const char*>(ds->h_packed);
-        char* dst = static_cast<char*>(C);
-        auto rows = [=](int64_t a0, int64_t a1) {
-            for (int64_t i = a0; i < a1; ++i)
-                std::memcpy(dst + size_t(i) * ldc * ec, src + size_t(i) * size_t(i + 1) / 2 * ec, size_t(i + 1) * ec);
-        };
-        const int T = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(hw ? hw : 1), int64_t(8), (r1 - r0) / 64})));
-        std::vector<std::thread> pool;
-        for (int t = 1; t < T; ++t) pool.emplace_back(rows, r0 + (r1 - r0) * t / T, r0 + (r1 - r0) * (t + 1) / T);
-        rows(r0, r0 + (r1 - r0) / T);
-        for (std::thread& th : pool) th.join();
+        if (!chk(cudaEventSynchronize(ds->host_events[0]))) return SYRK_ERR_CUDA;
+        unpack_parallel(0, N, packed_bytes, false);
+    } else {
+        // one block = the whole triangle, packed; it comes back in four groups of rows of about equal
+        // bytes, and host threads move group q into C while group q + 1 is copied
+        constexpr int kGroups = 4;
+        int64_t grp[kGroups + 1];
+        for (int q = 0; q <= kGroups; ++q) grp[q] = (q == kGroups) ? N : int64_t(double(N) * std::sqrt(double(q) / kGroups));
+        for (int q = 0; q < kGroups; ++q) {
+            grp[q + 1] = std::max(grp[q + 1], grp[q]);
+            const int64_t r0 = grp[q], r1 = grp[q + 1];
+            if (r1 > r0) {
+                const size_t off = size_t(r0) * size_t(r0 + 1) / 2 * ec, end = size_t(r1) * size_t(r1 + 1) / 2 * ec;
+                if (!pack_rows(r0, r1) ||
+                    !chk(cudaMemcpyAsync(static_cast<char*>(ds->h_packed) + off, static_cast<char*>(ds->d_packed) + off,
+                                         end - off, cudaMemcpyDeviceToHost, st)))
+                    return SYRK_ERR_CUDA;
+            }
+            if (!chk(cudaEventRecord(ds->host_events[q], st))) return SYRK_ERR_CUDA;
+        }
+        for (int q = 0; q < kGroups; ++q) {
+            if (!chk(cudaEventSynchronize(ds->host_events[q]))) return SYRK_ERR_CUDA;
+            if (grp[q + 1] > grp[q])
+                unpack_parallel(grp[q], grp[q + 1], size_t(grp[q + 1] - grp[q]) * size_t(grp[q + 1] + grp[q]) / 2 * ec, true);
+        }
     }
     if (!chk(cudaStreamSynchronize(st))) return SYRK_ERR_CUDA;
     int flag = 0;
