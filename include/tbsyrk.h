@@ -120,15 +120,19 @@ int syrk_lower_tn(int64_t N, int64_t M,
  * pinned; pinned memory copies faster).  The strict upper triangle of the host C is
  * left as it was.  The device and pinned staging buffers are kept by the library
  * (they only grow) and are released by syrk_shutdown().
- * Large inputs are pipelined: A is uploaded in blocks of columns (multiples of 256,
- * at least 32 MB each, at most 8) and each block's update
+ * Large inputs are pipelined.  With a page-locked C and N >= 4096 the call works band of
+ * rows by band of rows (up to 16): rows [r0, r1) of C need rows [0, r1) of A only, so A
+ * is uploaded band by band, a band's work items (square blocks in row order; this path
+ * does not use triangle blocks) run as soon as its rows have landed, and the band of C
+ * is downloaded while later bands are still uploaded and computed - the rectangle left
+ * of the band's diagonal block straight into the caller's C, the diagonal block's lower
+ * triangle packed and put in place by the host.  Otherwise A is uploaded in blocks of
+ * columns (multiples of 256, at least 32 MB each, at most 8) and each block's update
  * C <- alpha * A_c A_c^T + (beta for the first block, 1 after) * C runs while the next
- * block is in flight; the result comes back in up to 16 bands of rows: the rectangle left
- * of a band's diagonal block is copied straight into the caller's C, the diagonal blocks'
- * lower triangles come back packed and are put in place by the host meanwhile (with a
- * pageable C the whole triangle comes back packed and host threads unpack it).  The sum
- * over k is thereby taken block by block, which stays within the stated tolerance of the
- * one-call result.
+ * block is in flight (the sum over k is then taken block by block, within the stated
+ * tolerance of the one-call result), and C comes back after the last block: in bands as
+ * above when it is page-locked, else packed in four groups of rows that host threads
+ * unpack while the next group is copied.
  */
 int syrk_lower_host(int64_t N, int64_t M,
                     const void* A, int64_t lda,

@@ -66,6 +66,80 @@ int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk)
     return auto_split_k(dp->plan.items, M, bk, ds->sm_count, runtime().split_k);
 }
 
+// One launch of the item kernels over a list (the whole plan, or the items of one band of rows).
+int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkItem* d_items, int64_t n_items,
+                 int64_t N, int64_t M, void* C, int64_t ldc, double alpha, double beta, int split,
+                 const int64_t* d_tile_base, int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas,
+                 int f64_launch, int a_is_m_by_n, cudaStream_t stream) {
+    cudaError_t e;
+    if (dtype == SYRK_DTYPE_F64) {
+        CUtensorMap tmc;
+        const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
+                           encode_tensor_map_c_f64(&tmc, C, N, ldc, f64_tile()) == SYRK_OK;
+        // Persistent blocks hide each item's start-up (a few microseconds) behind the previous item.
+        // That pays when items are short (M <= 1024: at most 64 stages each) and the list fills the
+        // device several times over; for long items one block per item is the faster form.
+        const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
+        const bool persistent = mode == SYRK_F64_LAUNCH_PERSISTENT ||
+                                (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count));
+        int* tickets = persistent ? tickets_for_stream(ds, stream) : nullptr;
+        e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<double*>(C), ldc,
+                            alpha, beta, a_is_m_by_n, tickets, ds->sm_count, ds->d_status, stream);
+    } else {
+        CUtensorMap tmc;
+        const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
+                           encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
+        e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
+                             float(beta), split, ds->d_partial, d_tile_base, total_tiles, d_cta_begin, n_ctas, a_is_m_by_n,
+                             dtype - SYRK_DTYPE_BF16_F32, ds->d_status, ds->sm_count, stream);
+    }
+    return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
+// The row-ordered square-block list of (N, dtype), built and uploaded on first use.  Returns
+// SYRK_ERR_PLAN when the list cannot be cut into bands (the caller then takes another path).
+int get_banded_plan(DeviceState* ds, int64_t N, int dtype, int max_bands, BandedPlan** out) {
+    const KernelShape ks = kernel_shape(dtype);
+    const int64_t n_tiles = (N + ks.tile - 1) / ks.tile;
+    auto key = std::make_pair(n_tiles, dtype);
+    auto it = ds->banded.find(key);
+    if (it == ds->banded.end()) {
+        PlanParams p;
+        p.n_tiles = n_tiles; p.k = ks.k; p.rect_rows = ks.rect_rows; p.rect_cols = ks.rect_cols;
+        p.diag_side = ks.diag_side; p.schedule = SYRK_SCHEDULE_SQUARE;
+        Plan plan;
+        if (!build_plan(p, &plan) || plan.items.empty()) return SYRK_ERR_PLAN;
+        // Items come strip by strip (diag_side tile rows each, top to bottom); a band is a whole
+        // number of strips.
+        const int64_t n_strips = (n_tiles + ks.diag_side - 1) / ks.diag_side;
+        const int64_t n_bands = std::max<int64_t>(1, std::min<int64_t>(max_bands, n_strips));
+        const int64_t strips_per_band = (n_strips + n_bands - 1) / n_bands;
+        BandedPlan bp;
+        bp.band_rows = strips_per_band * ks.diag_side * ks.tile;
+        bp.items = plan.items;
+        int64_t band = 0;
+        for (size_t i = 0; i < bp.items.size(); ++i) {
+            const WorkItem& w = bp.items[i];
+            int64_t lo = INT64_MAX, hi = -1;
+            for (int t = 0; t < w.n_tile; ++t) {
+                lo = std::min<int64_t>(lo, w.seg[w.tile_x[t]]);
+                hi = std::max<int64_t>(hi, w.seg[w.tile_x[t]]);
+            }
+            const int64_t b_lo = lo * ks.tile / bp.band_rows, b_hi = hi * ks.tile / bp.band_rows;
+            if (b_lo != b_hi || b_hi < band) return SYRK_ERR_PLAN;      // straddles a boundary or out of order
+            while (band < b_hi) { bp.item_end.push_back(int64_t(i)); ++band; }
+        }
+        bp.item_end.push_back(int64_t(bp.items.size()));
+        if (cudaMalloc(&bp.d_items, bp.items.size() * sizeof(WorkItem)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
+        if (cudaMemcpy(bp.d_items, bp.items.data(), bp.items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError(); cudaFree(bp.d_items); return SYRK_ERR_CUDA;
+        }
+        it = ds->banded.emplace(key, std::move(bp)).first;
+    }
+    *out = &it->second;
+    return SYRK_OK;
+}
+
 }  // namespace
 
 int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
@@ -91,23 +165,9 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
     if (a_is_m_by_n) rc = encode_tensor_map_2d(&tm, dtype, A, M, N, lda, ks.bk, dtype == SYRK_DTYPE_F64 ? 16 : 64);
     else rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, ks.tile, ks.bk);
     if (rc != SYRK_OK) return rc;
-    const int64_t n_items = int64_t(dp->plan.items.size());
-    cudaError_t e;
-    if (dtype == SYRK_DTYPE_F64) {
-        CUtensorMap tmc;
-        const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
-                           encode_tensor_map_c_f64(&tmc, C, N, ldc, f64_tile()) == SYRK_OK;
-        // Persistent blocks hide each item's start-up (a few microseconds) behind the previous item.
-        // That pays when items are short (M <= 1024: at most 64 stages each) and the list fills the
-        // device several times over; for long items one block per item is the faster form.
-        const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
-        const bool persistent = mode == SYRK_F64_LAUNCH_PERSISTENT ||
-                                (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count));
-        int* tickets = persistent ? tickets_for_stream(ds, stream) : nullptr;
-        e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc,
-                            alpha, beta, a_is_m_by_n, tickets, ds->sm_count, ds->d_status, stream);
-    } else {
-        const int split = pick_split_k(ds, dp, M, ks.bk);
+    int split = 1;
+    if (is_tcgen05_dtype(dtype)) {
+        split = pick_split_k(ds, dp, M, ks.bk);
         if (split > 1) {
             const size_t want = size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float);
             void* p = ds->d_partial;
@@ -115,14 +175,9 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
             ds->d_partial = static_cast<float*>(p);
             if (rc != SYRK_OK) return rc;
         }
-        CUtensorMap tmc;
-        const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
-                           encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
-        e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
-                             float(beta), split, ds->d_partial, dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, a_is_m_by_n,
-                             dtype - SYRK_DTYPE_BF16_F32, ds->d_status, ds->sm_count, stream);
     }
-    return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+    return launch_items(ds, dtype, tm, dp->d_items, int64_t(dp->plan.items.size()), N, M, C, ldc, alpha, beta, split,
+                        dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, f64_launch, a_is_m_by_n, stream);
 }
 
 namespace {
@@ -175,9 +230,10 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     constexpr int kMaxChunks = 8, kBands = 16;
     if (!ds->host_stream) {
         bool ok = cudaStreamCreateWithFlags(&ds->host_stream, cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaStreamCreateWithFlags(&ds->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
-        for (int i = 0; ok && i < kMaxChunks; ++i)
-            ok = cudaEventCreateWithFlags(&ds->host_events[i], cudaEventDisableTiming) == cudaSuccess;
+                  cudaStreamCreateWithFlags(&ds->copy_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&ds->down_stream, cudaStreamNonBlocking) == cudaSuccess;
+        for (cudaStream_t& bs : ds->band_streams) ok = ok && cudaStreamCreateWithFlags(&bs, cudaStreamNonBlocking) == cudaSuccess;
+        for (cudaEvent_t& ev : ds->host_events) ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
         if (!ok) { cudaGetLastError(); return SYRK_ERR_CUDA; }
     }
     cudaStream_t st = ds->host_stream, cp = ds->copy_stream;
@@ -189,14 +245,95 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     cudaPointerAttributes c_attr{};
     const bool c_pinned = cudaPointerGetAttributes(&c_attr, C) == cudaSuccess && c_attr.type == cudaMemoryTypeHost;
     cudaGetLastError();
-    const int64_t pk_bands = c_pinned ? std::max<int64_t>(1, std::min<int64_t>(kBands, N / 256)) : 1;
-    const int64_t pk_h = (N + pk_bands - 1) / pk_bands;
+    // Large problems with a page-locked C are produced band by band (see below); the bands are then
+    // those of the row-ordered work list.
+    BandedPlan* bp = nullptr;
+    const bool banded = c_pinned && M > 0 && alpha != 0.0 && N >= 4096 &&
+                        get_banded_plan(ds, N, dtype, kBands, &bp) == SYRK_OK && bp->item_end.size() > 1;
+    const int64_t pk_h = banded ? bp->band_rows
+                                : (c_pinned ? (N + std::max<int64_t>(1, std::min<int64_t>(kBands, N / 256)) - 1) /
+                                                  std::max<int64_t>(1, std::min<int64_t>(kBands, N / 256))
+                                            : N);
+    const int64_t pk_bands = (N + pk_h - 1) / pk_h;
     const size_t packed_bytes = size_t(pk_bands) * size_t(pk_h) * size_t(pk_h + 1) / 2 * ec;
     if ((rc = ensure_device_bytes(&ds->d_a, &ds->d_a_bytes, size_t(N) * dlda * ea)) != SYRK_OK) return rc;
     if ((rc = ensure_device_bytes(&ds->d_c, &ds->d_c_bytes, size_t(N) * dldc * ec)) != SYRK_OK) return rc;
     if ((rc = ensure_device_bytes(&ds->d_packed, &ds->d_packed_bytes, packed_bytes)) != SYRK_OK) return rc;
     if ((rc = ensure_pinned_bytes(&ds->h_packed, &ds->h_packed_bytes, packed_bytes)) != SYRK_OK) return rc;
     auto chk = [](cudaError_t e) { if (e != cudaSuccess) { cudaGetLastError(); return false; } return true; };
+
+    if (banded) {
+        // Row-band pipeline.  Rows [r0, r1) of C need rows [0, r1) of A only, and in the row-ordered
+        // square-block list the items of band j write rows of band j only.  So A goes up band by band
+        // (copy stream), band j's items run as soon as its rows have landed (four compute streams in
+        // turn, so that short lists of long items overlap), and band j of C goes down (download
+        // stream) while later bands are still being uploaded and computed: the rectangle left of the
+        // diagonal block straight into C, the diagonal block packed.
+        const int64_t band_h = bp->band_rows, n_bands = int64_t(bp->item_end.size());
+        cudaStream_t dl = ds->down_stream;
+        const KernelShape ks = kernel_shape(dtype);
+        CUtensorMap tm;
+        if ((rc = encode_tensor_map_2d(&tm, dtype, ds->d_a, N, M, dlda, ks.tile, ks.bk)) != SYRK_OK) return rc;
+        cudaEvent_t* ev_up = ds->host_events;
+        cudaEvent_t* ev_done = ds->host_events + kBands;
+        cudaEvent_t* ev_packed = ds->host_events + 2 * kBands;
+        const size_t full = size_t(band_h) * size_t(band_h + 1) / 2;
+        for (int64_t j = 0; j < n_bands; ++j) {
+            const int64_t r0 = j * band_h, r1 = std::min(N, r0 + band_h);
+            cudaStream_t cs = ds->band_streams[j % 4];
+            bool ok = chk(cudaMemcpy2DAsync(static_cast<char*>(ds->d_a) + size_t(r0) * dlda * ea, dlda * ea,
+                                            static_cast<const char*>(A) + size_t(r0) * lda * ea, lda * ea, M * ea, r1 - r0,
+                                            cudaMemcpyHostToDevice, cp));
+            if (beta != 0.0)
+                ok = ok && chk(cudaMemcpy2DAsync(static_cast<char*>(ds->d_c) + size_t(r0) * dldc * ec, dldc * ec,
+                                                 static_cast<const char*>(C) + size_t(r0) * ldc * ec, ldc * ec, r1 * ec, r1 - r0,
+                                                 cudaMemcpyHostToDevice, cp));
+            ok = ok && chk(cudaEventRecord(ev_up[j], cp)) && chk(cudaStreamWaitEvent(cs, ev_up[j], 0));
+            if (!ok) return SYRK_ERR_CUDA;
+            const int64_t i0 = j == 0 ? 0 : bp->item_end[size_t(j - 1)], i1 = bp->item_end[size_t(j)];
+            if (i1 > i0) {
+                rc = launch_items(ds, dtype, tm, bp->d_items + i0, i1 - i0, N, M, ds->d_c, dldc, alpha, beta, 1, nullptr, 0,
+                                  nullptr, 0, -1, 0, cs);
+                if (rc != SYRK_OK) return rc;
+            }
+            ok = chk(cudaEventRecord(ev_done[j], cs)) && chk(cudaStreamWaitEvent(dl, ev_done[j], 0));
+            if (ok && r0 > 0)
+                ok = chk(cudaMemcpy2DAsync(static_cast<char*>(C) + size_t(r0) * ldc * ec, size_t(ldc) * ec,
+                                           static_cast<const char*>(ds->d_c) + size_t(r0) * dldc * ec, size_t(dldc) * ec,
+                                           size_t(r0) * ec, size_t(r1 - r0), cudaMemcpyDeviceToHost, dl));
+            if (!ok) return SYRK_ERR_CUDA;
+            const dim3 grid(unsigned(std::min<int64_t>(64, (band_h + 255) / 256)), unsigned(std::min<int64_t>(r1 - r0, 32768)));
+            if (dtype == SYRK_DTYPE_F64)
+                pack_diag_blocks_kernel<double><<<grid, 256, 0, dl>>>(r0, r1, band_h, static_cast<const double*>(ds->d_c), dldc,
+                                                                      static_cast<double*>(ds->d_packed));
+            else
+                pack_diag_blocks_kernel<float><<<grid, 256, 0, dl>>>(r0, r1, band_h, static_cast<const float*>(ds->d_c), dldc,
+                                                                     static_cast<float*>(ds->d_packed));
+            const size_t h = size_t(r1 - r0);
+            if (!chk(cudaGetLastError()) ||
+                !chk(cudaMemcpyAsync(static_cast<char*>(ds->h_packed) + size_t(j) * full * ec,
+                                     static_cast<const char*>(ds->d_packed) + size_t(j) * full * ec, h * (h + 1) / 2 * ec,
+                                     cudaMemcpyDeviceToHost, dl)) ||
+                !chk(cudaEventRecord(ev_packed[j], dl)))
+                return SYRK_ERR_CUDA;
+        }
+        const char* psrc = static_cast<const char*>(ds->h_packed);
+        char* pdst = static_cast<char*>(C);
+        for (int64_t j = 0; j < n_bands; ++j) {
+            if (!chk(cudaEventSynchronize(ev_packed[j]))) return SYRK_ERR_CUDA;
+            const int64_t r0 = j * band_h, r1 = std::min(N, r0 + band_h);
+            for (int64_t i = r0; i < r1; ++i) {
+                const int64_t l = i - r0;
+                std::memcpy(pdst + (size_t(i) * ldc + size_t(r0)) * ec,
+                            psrc + (size_t(j) * full + size_t(l) * size_t(l + 1) / 2) * ec, size_t(l + 1) * ec);
+            }
+        }
+        if (!chk(cudaStreamSynchronize(dl))) return SYRK_ERR_CUDA;
+        int flag = 0;
+        if (cudaMemcpy(&flag, ds->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+        if (flag != 0) { cudaMemset(ds->d_status, 0, sizeof(int)); return SYRK_ERR_DEVICE_WAIT; }
+        return SYRK_OK;
+    }
 
     // Upload and compute overlap: A goes up in column blocks on the copy stream and each block's
     // rank-update C <- alpha A_c A_c^T + (beta or 1) C runs on the compute stream as soon as its

@@ -298,6 +298,9 @@ void release_all() {
         if (ds.h_packed) cudaFreeHost(ds.h_packed);
         if (ds.host_stream) cudaStreamDestroy(ds.host_stream);
         if (ds.copy_stream) cudaStreamDestroy(ds.copy_stream);
+        if (ds.down_stream) cudaStreamDestroy(ds.down_stream);
+        for (cudaStream_t bs : ds.band_streams) if (bs) cudaStreamDestroy(bs);
+        for (auto& bk : ds.banded) if (bk.second.d_items) cudaFree(bk.second.d_items);
         for (cudaEvent_t ev : ds.host_events) if (ev) cudaEventDestroy(ev);
     }
     rt.devices.clear();

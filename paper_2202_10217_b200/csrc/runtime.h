@@ -5,6 +5,8 @@
 #include <map>
 #include <mutex>
 #include <tuple>
+#include <utility>
+#include <vector>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -37,6 +39,15 @@ struct DevicePlan {
     int n_ctas = 0;
 };
 
+// Square-block work list in row order for the host-buffer entry point: band j owns the rows
+// [j * band_rows, (j + 1) * band_rows) of C and the items [item_end[j-1], item_end[j]).
+struct BandedPlan {
+    std::vector<WorkItem> items;
+    WorkItem* d_items = nullptr;
+    int64_t band_rows = 0;
+    std::vector<int64_t> item_end;
+};
+
 struct DeviceState {
     int device = -1;
     int sm_count = 0;
@@ -55,7 +66,10 @@ struct DeviceState {
     void* h_packed = nullptr; size_t h_packed_bytes = 0;
     cudaStream_t host_stream = nullptr;      // compute stream of the host-buffer entry point
     cudaStream_t copy_stream = nullptr;      // its upload stream
-    cudaEvent_t host_events[8] = {};         // block-landed / band-ready events of that entry point
+    cudaStream_t down_stream = nullptr;      // its download stream
+    cudaStream_t band_streams[4] = {};       // its compute streams when C is produced band by band
+    cudaEvent_t host_events[48] = {};        // block-landed / band-computed / band-packed events of that entry point
+    std::map<std::pair<int64_t, int>, BandedPlan> banded;  // (n_tiles, dtype)
     std::map<std::tuple<int64_t, int, int>, DevicePlan> plans;  // (n_tiles, dtype, schedule)
 };
 

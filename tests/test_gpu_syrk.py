@@ -321,3 +321,38 @@ def test_host_buffer_entry_point_pipelined_blocks(dtype):
     iu = np.triu_indices(N, 1)
     assert np.array_equal(C[:, :N][iu], Cin[:, :N][iu])           # strict upper triangle untouched
     assert np.array_equal(C[:, N:], Cin[:, N:])                   # and the padding columns
+
+
+@DT
+def test_host_buffer_entry_point_row_band_pipeline(dtype):
+    """Page-locked host buffers and N >= 4096: the entry point uploads A, computes and downloads C
+    band of rows by band of rows.  Ragged N, pitches, beta != 0; sampled entries plus every entry
+    next to the band and tile boundaries of a few rows; upper triangle and padding untouched."""
+    import torch
+    N, M = {B.DTYPE_F64: (4100, 200), B.DTYPE_BF16_F32: (4500, 520), B.DTYPE_TF32_F32: (4230, 260),
+            B.DTYPE_E4M3_F32: (4400, 1040)}[dtype]
+    A = make_A(N, M, dtype, seed=71)
+    lda, ldc = M + 32, N + 6
+    Abig = np.zeros((N, lda), dtype=A.dtype)
+    Abig[:, :M] = A
+    Cin = I.random_c(N, 72, dtype, ldc)
+    hA = torch.from_numpy(Abig.view(np.int16) if dtype == B.DTYPE_BF16_F32 else Abig).pin_memory()
+    hC = torch.from_numpy(Cin.copy()).pin_memory()
+    for alpha, beta in ((0.5, -1.0), (1.0, 0.0)):
+        hC.copy_(torch.from_numpy(Cin))
+        B.syrk_lower_host(N, M, hA, lda, hC, ldc, alpha, beta, dtype)
+        C = hC.numpy()
+        rng = np.random.default_rng(73)
+        ii = rng.integers(0, N, size=30000)
+        jj = (rng.random(30000) * (ii + 1)).astype(np.int64)
+        rows = np.array([0, 127, 128, 255, 256, 257, 511, 512, 2047, 2048, 4095, 4096, N - 1])
+        rows = rows[rows < N]
+        ii = np.concatenate([ii] + [np.full(r + 1, r) for r in rows])
+        jj = np.concatenate([jj] + [np.arange(r + 1) for r in rows])
+        ref, bound = O.syrk_entries(ii, jj, A, None, alpha, 0.0, dtype)
+        ref = ref + beta * Cin[ii, jj].astype(np.float64)
+        tol = O.tolerance(M, bound, np.abs(Cin[ii, jj]), alpha, beta, dtype)
+        assert np.all(np.abs(C[ii, jj].astype(np.float64) - ref) <= tol)
+        iu = np.triu_indices(N, 1)
+        assert np.array_equal(C[:, :N][iu], Cin[:, :N][iu])
+        assert np.array_equal(C[:, N:], Cin[:, N:])
