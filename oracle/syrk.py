@@ -22,6 +22,7 @@ DTYPE_F64 = 0
 DTYPE_BF16_F32 = 1
 DTYPE_TF32_F32 = 2
 DTYPE_E4M3_F32 = 3
+DTYPE_F16_F32 = 4
 
 
 def build(force: bool = False) -> str:
@@ -58,7 +59,7 @@ def num_threads() -> int:
 
 def _check_inputs(A: np.ndarray, C_in, dtype: int):
     want_a = {DTYPE_F64: np.float64, DTYPE_BF16_F32: np.uint16, DTYPE_TF32_F32: np.float32,
-              DTYPE_E4M3_F32: np.uint8}[dtype]
+              DTYPE_E4M3_F32: np.uint8, DTYPE_F16_F32: np.uint16}[dtype]
     want_c = np.float64 if dtype == DTYPE_F64 else np.float32
     if A.dtype != want_a or A.ndim != 2 or (A.size > 0 and A.strides[1] != A.itemsize):
         raise ValueError("A must be a row-major 2-D array of %s" % want_a.__name__)
@@ -71,7 +72,8 @@ def syrk_lower(A: np.ndarray, C_in, alpha: float, beta: float, dtype: int):
     """Reference lower triangle and bound matrix.
 
     ``A`` is N x M (float64, uint16 holding bf16 bit patterns, or float32 read as TF32:
-    its 13 low-order bits are dropped, or uint8 holding FP8 E4M3 bytes); ``C_in`` is the
+    its 13 low-order bits are dropped, or uint8 holding FP8 E4M3 bytes, or uint16 holding
+    binary16 bit patterns for ``DTYPE_F16_F32``); ``C_in`` is the
     N x N prior value (float64 / float32) or None when beta == 0.  Returns
     ``(C_ref, B)``: N x N float64 arrays whose strict upper triangles are NaN
     (never written), with ``B[i, j] = sum_k |A[i,k]| |A[j,k]|``.
@@ -114,7 +116,7 @@ def syrk_entries(I, J, A: np.ndarray, C_in, alpha: float, beta: float, dtype: in
 
 # Parity tolerance: |C_gpu - C_ref| <= TOL[dtype] * M * (|alpha| B + |beta| |C_in|).
 TOL = {DTYPE_F64: 8.0 * 2.0 ** -53, DTYPE_BF16_F32: 4.0 * 2.0 ** -24, DTYPE_TF32_F32: 4.0 * 2.0 ** -24,
-       DTYPE_E4M3_F32: 4.0 * 2.0 ** -24}
+       DTYPE_E4M3_F32: 4.0 * 2.0 ** -24, DTYPE_F16_F32: 4.0 * 2.0 ** -24}
 
 
 def tolerance(M: int, bound, c_in_abs, alpha: float, beta: float, dtype: int):

@@ -28,6 +28,11 @@
  * subnormals f/8 * 2^-6; there are no infinities and the only NaN is exponent
  * and fraction all ones (0x7F, 0xFF); the largest finite value is 448.  Each
  * byte is decoded exactly; products have at most 8 significant bits.
+ * FP16 inputs are IEEE 754 binary16 bit patterns: 1 sign bit, 5 exponent bits
+ * (bias 15), 10 fraction bits; exponent field 0 holds zero and the subnormals
+ * f * 2^-24, exponent field 31 infinity (f = 0) and NaN.  Each pattern is
+ * decoded exactly; products have at most 22 significant bits and exponents of at
+ * least -48, so they are exact in binary64 (and in binary32).
  * The k-sum is sequential, with no reassociation and no fused multiply-add
  * (compile with -ffp-contract=off).
  *
@@ -50,7 +55,8 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_DTYPE_F64 = 0, ORACLE_DTYPE_BF16_F32 = 1, ORACLE_DTYPE_TF32_F32 = 2, ORACLE_DTYPE_E4M3_F32 = 3 };
+enum { ORACLE_DTYPE_F64 = 0, ORACLE_DTYPE_BF16_F32 = 1, ORACLE_DTYPE_TF32_F32 = 2, ORACLE_DTYPE_E4M3_F32 = 3,
+       ORACLE_DTYPE_F16_F32 = 4 };
 
 static inline double widen_bf16(uint16_t bits) {
     union { uint32_t u; float f; } x;
@@ -73,15 +79,25 @@ static inline double widen_e4m3(uint8_t bits) {
     return sign ? -v : v;
 }
 
+static inline double widen_f16(uint16_t bits) {
+    const int sign = bits >> 15, e = (bits >> 10) & 31, f = bits & 1023;
+    double v;
+    if (e == 31) v = f ? NAN : INFINITY;
+    else if (e == 0) v = ldexp((double)f, -24);           /* f/1024 * 2^-14 */
+    else v = ldexp((double)(1024 + f), e - 25);           /* (1 + f/1024) * 2^(e-15) */
+    return sign ? -v : v;
+}
+
 /* Element A[r][k] as a double, for any input type. */
 static inline double a_at(const void* A, int64_t lda, int dtype, int64_t r, int64_t k) {
     if (dtype == ORACLE_DTYPE_F64) return ((const double*)A)[r * lda + k];
     if (dtype == ORACLE_DTYPE_TF32_F32) return widen_tf32(((const uint32_t*)A)[r * lda + k]);
     if (dtype == ORACLE_DTYPE_E4M3_F32) return widen_e4m3(((const uint8_t*)A)[r * lda + k]);
+    if (dtype == ORACLE_DTYPE_F16_F32) return widen_f16(((const uint16_t*)A)[r * lda + k]);
     return widen_bf16(((const uint16_t*)A)[r * lda + k]);
 }
 
-/* Element C_in[i][j] as a double (binary64 C, or binary32 C for bf16, TF32 and FP8 inputs). */
+/* Element C_in[i][j] as a double (binary64 C, or binary32 C for bf16, TF32, FP8 and FP16 inputs). */
 static inline double c_at(const void* C, int64_t ldc, int dtype, int64_t i, int64_t j) {
     if (dtype == ORACLE_DTYPE_F64) return ((const double*)C)[i * ldc + j];
     return (double)((const float*)C)[i * ldc + j];
@@ -111,7 +127,7 @@ static void one_entry(int64_t M, const void* A, int64_t lda, int dtype,
 int oracle_syrk_lower(int64_t N, int64_t M, const void* A, int64_t lda,
                       const void* Cin, int64_t ldc, double alpha, double beta,
                       int dtype, double* Cref, double* Bound, int64_t ldr) {
-    if (N < 0 || M < 0 || dtype < ORACLE_DTYPE_F64 || dtype > ORACLE_DTYPE_E4M3_F32) return -1;
+    if (N < 0 || M < 0 || dtype < ORACLE_DTYPE_F64 || dtype > ORACLE_DTYPE_F16_F32) return -1;
     if (N > 0 && (!Cref || !Bound || ldr < N)) return -1;
     if (N > 0 && M > 0 && (!A || lda < M)) return -1;
     if (N > 0 && beta != 0.0 && (!Cin || ldc < N)) return -1;
@@ -135,7 +151,7 @@ int oracle_syrk_entries(int64_t P, const int64_t* I, const int64_t* J,
                         const void* Cin, int64_t ldc, double alpha, double beta,
                         int dtype, double* ref, double* bound) {
     if (P < 0 || N < 0 || M < 0) return -1;
-    if (dtype < ORACLE_DTYPE_F64 || dtype > ORACLE_DTYPE_E4M3_F32) return -1;
+    if (dtype < ORACLE_DTYPE_F64 || dtype > ORACLE_DTYPE_F16_F32) return -1;
     for (int64_t p = 0; p < P; ++p)
         if (I[p] < J[p] || J[p] < 0 || I[p] >= N) return -1;
 #pragma omp parallel for schedule(dynamic, 64)

@@ -7,7 +7,8 @@ and the CPU reference may take their inputs from it.  All generators are numpy
 on a GPU.
 
 bf16 values travel as ``uint16`` bit patterns and FP8 E4M3 values as ``uint8`` bytes (numpy has
-neither type).
+neither type); binary16 values travel as ``uint16`` bit patterns too, so that every 16-bit
+input reaches the library the same way.
 """
 from __future__ import annotations
 
@@ -20,6 +21,7 @@ DTYPE_F64 = 0        # A, C binary64
 DTYPE_BF16_F32 = 1   # A bfloat16, C binary32 (binary32 accumulation)
 DTYPE_TF32_F32 = 2   # A binary32 read as TF32 (19 high-order bits), C binary32
 DTYPE_E4M3_F32 = 3   # A FP8 E4M3 bytes (uint8), C binary32
+DTYPE_F16_F32 = 4    # A IEEE binary16 bit patterns (uint16), C binary32
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -33,6 +35,16 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
 def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     """Widen bfloat16 bit patterns to binary32 (exact)."""
     return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def f32_to_f16_bits(x: np.ndarray) -> np.ndarray:
+    """Round binary32 values to IEEE binary16 (nearest, ties to even; numpy's conversion); uint16 bits."""
+    return np.ascontiguousarray(x, dtype=np.float32).astype(np.float16).view(np.uint16)
+
+
+def f16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """Widen binary16 bit patterns to binary32 (exact)."""
+    return np.ascontiguousarray(bits, dtype=np.uint16).view(np.float16).astype(np.float32)
 
 
 def f32_keep_tf32_bits(x: np.ndarray) -> np.ndarray:
@@ -108,6 +120,16 @@ def small_int_e4m3(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.n
     return f32_to_e4m3_bits(np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float32))
 
 
+def normal_f16(N: int, M: int, seed: int, std: float = 1.0) -> np.ndarray:
+    """Entries i.i.d. N(0, std^2) rounded to binary16; uint16 bit patterns."""
+    return f32_to_f16_bits(_normal(np.random.default_rng(seed), (N, M), std))
+
+
+def small_int_f16(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
+    """Integer entries in [lo, hi] as binary16 bit patterns (exactly representable)."""
+    return f32_to_f16_bits(np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float32))
+
+
 def small_int_f64(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
     """Integer entries in [lo, hi] stored as binary64 (every partial sum is exact)."""
     return np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float64)
@@ -127,6 +149,8 @@ def ones(N: int, M: int, dtype: int) -> np.ndarray:
         return np.ones((N, M), dtype=np.float32)
     if dtype == DTYPE_E4M3_F32:
         return f32_to_e4m3_bits(np.ones((N, M), dtype=np.float32))
+    if dtype == DTYPE_F16_F32:
+        return f32_to_f16_bits(np.ones((N, M), dtype=np.float32))
     return f32_to_bf16_bits(np.ones((N, M), dtype=np.float32))
 
 
@@ -138,6 +162,8 @@ def to_storage(values: np.ndarray, dtype: int) -> np.ndarray:
         return np.ascontiguousarray(values, dtype=np.float32)
     if dtype == DTYPE_E4M3_F32:
         return f32_to_e4m3_bits(np.asarray(values, dtype=np.float32))
+    if dtype == DTYPE_F16_F32:
+        return f32_to_f16_bits(np.asarray(values, dtype=np.float32))
     return f32_to_bf16_bits(np.asarray(values, dtype=np.float32))
 
 
@@ -174,6 +200,8 @@ class Workload:
             return normal_f32(self.N, self.M, self.seed, self.std)
         if self.dtype == DTYPE_E4M3_F32:
             return normal_e4m3(self.N, self.M, self.seed, self.std)
+        if self.dtype == DTYPE_F16_F32:
+            return normal_f16(self.N, self.M, self.seed, self.std)
         return normal_bf16(self.N, self.M, self.seed, self.std)
 
     @property

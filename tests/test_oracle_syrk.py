@@ -14,7 +14,8 @@ from oracle import syrk as O
 from paper_2202_10217_b200 import inputs as I
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
-BOTH = [O.DTYPE_F64, O.DTYPE_BF16_F32, O.DTYPE_TF32_F32, O.DTYPE_E4M3_F32]      # every input type of the reference
+BOTH = [O.DTYPE_F64, O.DTYPE_BF16_F32, O.DTYPE_TF32_F32, O.DTYPE_E4M3_F32,
+        O.DTYPE_F16_F32]                                                      # every input type of the reference
 
 
 def lower(x):
@@ -28,6 +29,8 @@ def widen(A, dtype):
         return I.f32_keep_tf32_bits(A).astype(np.float64)
     if dtype == O.DTYPE_E4M3_F32:
         return I.e4m3_bits_to_f32(A).astype(np.float64)
+    if dtype == O.DTYPE_F16_F32:
+        return I.f16_bits_to_f32(A).astype(np.float64)
     return I.bf16_bits_to_f32(A).astype(np.float64)
 
 
@@ -38,6 +41,8 @@ def real_inputs(N, M, seed, dtype):
         return I.normal_f32(N, M, seed)          # low-order bits set: the reference must drop them
     if dtype == O.DTYPE_E4M3_F32:
         return I.normal_e4m3(N, M, seed)
+    if dtype == O.DTYPE_F16_F32:
+        return I.normal_f16(N, M, seed)
     return I.normal_bf16(N, M, seed)
 
 
@@ -128,8 +133,9 @@ def test_real_inputs_within_dot_product_bound_of_exact(dtype):
             err = abs(Fraction(ref[i, j]) - G[i][j])
             assert err <= Fraction(M * u * 1.01) * Fraction(bound[i, j])
     # the reference must not be exact-by-construction: some entry does round.  (FP8 products are
-    # multiples of 2^-18 below 2^18, so their binary64 sums are exact for any M used here.)
-    if dtype == O.DTYPE_E4M3_F32:
+    # multiples of 2^-18 below 2^18, so their binary64 sums are exact for any M used here; the
+    # binary16 products of this seeded input are multiples of 2^-48 below 2^5, exact as well.)
+    if dtype in (O.DTYPE_E4M3_F32, O.DTYPE_F16_F32):
         assert all(Fraction(ref[i, j]) == G[i][j] for i in range(N) for j in range(i + 1))
     else:
         assert any(Fraction(ref[i, j]) != G[i][j] for i in range(N) for j in range(i + 1))
@@ -180,7 +186,7 @@ def test_bf16_widening_bit_patterns():
 def test_leading_dimensions_and_entry_list(dtype):
     N, M, lda, ldc = 13, 21, 32, 20
     big = {O.DTYPE_F64: I.small_int_f64, O.DTYPE_BF16_F32: I.small_int_bf16, O.DTYPE_TF32_F32: I.small_int_f32,
-           O.DTYPE_E4M3_F32: I.small_int_e4m3}[dtype](N, lda, 4)
+           O.DTYPE_E4M3_F32: I.small_int_e4m3, O.DTYPE_F16_F32: I.small_int_f16}[dtype](N, lda, 4)
     A = big[:, :M]                                           # row pitch lda > M
     Cbig = I.random_c(N, 6, dtype, ldc)
     Cin = Cbig[:, :N]
@@ -231,6 +237,48 @@ def test_e4m3_decoding_of_every_byte():
             assert ref[1, 0] == want and ref[1, 1] == want * want and bound[1, 0] == abs(want)
     assert O.syrk_lower(np.array([[0x7E]], dtype=np.uint8), None, 1.0, 0.0, O.DTYPE_E4M3_F32)[0][0, 0] == 448.0 ** 2
     assert O.syrk_lower(np.array([[0x01]], dtype=np.uint8), None, 1.0, 0.0, O.DTYPE_E4M3_F32)[0][0, 0] == 2.0 ** -18
+
+
+def test_f16_decoding_of_every_bit_pattern():
+    """All 65536 binary16 patterns against the format's definition written out here:
+    value = (-1)^s * 2^(e-15) * (1 + f/1024); e = 0: (-1)^s * 2^-14 * f/1024; e = 31: infinity
+    (f = 0) or NaN.  Row 0 holds 1.0 (0x3C00), so entry (r, 0) of the result is the decoded
+    value of row r and entry (r, r) its square; hand values at the extremes follow."""
+    codes = np.arange(65536, dtype=np.uint32)
+    s_, e, f = codes >> 15, (codes >> 10) & 31, codes & 1023
+    want = np.where(e == 0, 2.0 ** -14 * (f / 1024.0), 2.0 ** (e.astype(np.float64) - 15) * (1.0 + f / 1024.0))
+    want = np.where(e == 31, np.where(f == 0, np.inf, np.nan), want)
+    want = np.where(s_ == 1, -want, want)
+    finite = np.isfinite(want)
+    for lo in range(0, 65536, 2048):                                 # 32 problems of 2049 rows, M = 1
+        block = codes[lo:lo + 2048].astype(np.uint16)
+        A = np.concatenate([np.array([0x3C00], dtype=np.uint16), block]).reshape(-1, 1)
+        I_ = np.arange(1, 2049)
+        v, b = O.syrk_entries(I_, np.zeros(2048, dtype=np.int64), A, None, 1.0, 0.0, O.DTYPE_F16_F32)
+        sq, _ = O.syrk_entries(I_, I_, A, None, 1.0, 0.0, O.DTYPE_F16_F32)
+        w, fin = want[lo:lo + 2048], finite[lo:lo + 2048]
+        assert np.array_equal(v[fin], w[fin]) and np.array_equal(b[fin], np.abs(w[fin]))
+        assert np.array_equal(sq[fin], w[fin] * w[fin])
+        assert np.array_equal(np.isnan(v), np.isnan(w)) and np.array_equal(np.isinf(v), np.isinf(w))
+    one = lambda bits: O.syrk_lower(np.array([[bits]], dtype=np.uint16), None, 1.0, 0.0, O.DTYPE_F16_F32)[0][0, 0]
+    assert one(0x7BFF) == 65504.0 ** 2            # largest finite value
+    assert one(0x0001) == 2.0 ** -48              # smallest subnormal, squared
+    assert one(0x0400) == 2.0 ** -28              # smallest normal 2^-14, squared
+    assert one(0x3555) == (1365.0 / 4096.0) ** 2  # 0.333251953125 = (1 + 341/1024) / 4
+    assert one(0xC000) == 4.0                     # -2
+    # the library that owns the type agrees (cross-check of the decoding, not the reference itself)
+    lib = np.arange(65536, dtype=np.uint32).astype(np.uint16).view(np.float16).astype(np.float64)
+    assert np.array_equal(lib[finite], want[finite])
+
+
+def test_f16_rounding_of_inputs_is_nearest_even():
+    # ulp of binary16 at 1 is 2^-10: 1 + 2^-11 ties to 1 (even), 1 + 3 * 2^-11 ties up to 1 + 2^-9;
+    # 65520 is the tie between 65504 and the overflow threshold -> infinity; 2^-25 ties to zero.
+    x = np.array([1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 1.0 + 2.0 ** -11 + 2.0 ** -20, 65519.0, 2.0 ** -25,
+                  -(2.0 ** -24)], dtype=np.float32)
+    bits = I.f32_to_f16_bits(x)
+    assert list(bits) == [0x3C00, 0x3C02, 0x3C01, 0x7BFF, 0x0000, 0x8001]
+    assert list(I.f16_bits_to_f32(bits)[:4]) == [1.0, 1.0 + 2.0 ** -9, 1.0 + 2.0 ** -10, 65504.0]
 
 
 def test_e4m3_rounding_of_inputs_is_nearest_even_and_saturating():
