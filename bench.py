@@ -30,9 +30,9 @@ from paper_2202_10217_b200 import inputs as I
 METRIC = "syrk_tflops_N(N+1)M"
 UNIT = "TFLOP/s"
 DTYPE_NAME = {I.DTYPE_F64: "f64", I.DTYPE_BF16_F32: "bf16_in_f32_acc", I.DTYPE_TF32_F32: "tf32_in_f32_acc",
-              I.DTYPE_E4M3_F32: "fp8_e4m3_in_f32_acc"}
-ELEM_A = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 2, I.DTYPE_TF32_F32: 4, I.DTYPE_E4M3_F32: 1}
-ELEM_C = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 4, I.DTYPE_TF32_F32: 4, I.DTYPE_E4M3_F32: 4}
+              I.DTYPE_E4M3_F32: "fp8_e4m3_in_f32_acc", I.DTYPE_F16_F32: "f16_in_f32_acc"}
+ELEM_A = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 2, I.DTYPE_TF32_F32: 4, I.DTYPE_E4M3_F32: 1, I.DTYPE_F16_F32: 2}
+ELEM_C = {I.DTYPE_F64: 8, I.DTYPE_BF16_F32: 4, I.DTYPE_TF32_F32: 4, I.DTYPE_E4M3_F32: 4, I.DTYPE_F16_F32: 4}
 
 
 def measured_peaks():
@@ -454,7 +454,7 @@ def main():
     ap.add_argument("--lbc-n", type=int, default=32768, help="matrix size of --workload lbc")
     ap.add_argument("--block", type=int, default=0, help="panel width of --workload lbc (0 = library default)")
     ap.add_argument("--shape", default=None,
-                    help="N,M,dtype,alpha,beta (dtype f64|bf16|tf32|e4m3): a custom seeded N(0,1) workload")
+                    help="N,M,dtype,alpha,beta (dtype f64|bf16|tf32|e4m3|f16): a custom seeded N(0,1) workload")
     ap.add_argument("--kernel-only", action="store_true",
                     help="device-timed kernel steps only (no end-to-end leg, CPU baseline or peak probe); "
                          "for short profiler runs")
@@ -480,7 +480,8 @@ def main():
     wl = I.CONFIGS[args.workload]
     if args.shape:
         n, m, dt, al, be = args.shape.split(",")
-        dtype = {"f64": I.DTYPE_F64, "bf16": I.DTYPE_BF16_F32, "tf32": I.DTYPE_TF32_F32, "e4m3": I.DTYPE_E4M3_F32}[dt]
+        dtype = {"f64": I.DTYPE_F64, "bf16": I.DTYPE_BF16_F32, "tf32": I.DTYPE_TF32_F32, "e4m3": I.DTYPE_E4M3_F32,
+                 "f16": I.DTYPE_F16_F32}[dt]
         wl = I.Workload("custom_%s_%sx%s" % (dt, n, m), int(n), int(m), dtype, float(al), float(be), 99, "normal")
     if args.impl == "reference":
         run_reference(args, wl, rank)

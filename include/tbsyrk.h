@@ -42,6 +42,10 @@ extern "C" {
                                   are NaN; largest value 448), C binary32; binary32
                                   accumulation (tcgen05 kind::f8f6f4).  syrk_lower_tn takes
                                   this type through the plain-load kernel only.           */
+#define SYRK_DTYPE_F16_F32  4  /* A IEEE 754 binary16 (1 sign, 5 exponent bits with bias 15,
+                                  10 fraction bits; subnormals, infinities and NaN as in
+                                  the standard), C binary32; binary32 accumulation (tcgen05
+                                  kind::f16).  Both storage orders run on the tensor cores. */
 
 /* return codes */
 #define SYRK_OK                 0
@@ -104,8 +108,8 @@ int syrk_lower(int64_t N, int64_t M,
  * Section 5.1.4), C, alpha, beta, dtype, stream, alignment rule (A 16-byte aligned and
  * lda * sizeof(element) a multiple of 16, else a slower plain-load kernel), ownership
  * and error codes are those of syrk_lower (SYRK_ERR_LD refers to lda < N here).
- * Both dtypes run on the tensor-core kernels (FP64: both launch forms; BF16: tcgen05
- * with MN-major operands, K-split included).
+ * FP64 and the 16-bit types run on the tensor-core kernels (FP64: both launch forms;
+ * bfloat16 and binary16: tcgen05 with MN-major operands, K-split included).
  */
 int syrk_lower_tn(int64_t N, int64_t M,
                   const void* A, int64_t lda,

@@ -16,6 +16,7 @@ DTYPE_F64 = 0
 DTYPE_BF16_F32 = 1
 DTYPE_TF32_F32 = 2
 DTYPE_E4M3_F32 = 3
+DTYPE_F16_F32 = 4
 SCHEDULE_TBS = 0
 SCHEDULE_SQUARE = 1
 ITEM_TRI, ITEM_RECT, ITEM_DIAG = 0, 1, 2

@@ -152,8 +152,8 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         return launch_scale_lower(dtype, N, C, ldc, beta, stream) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
     }
     // TF32 and FP8 inputs stored M x N have no tensor-core path (MN-major operands are used for
-    // bfloat16 only).
-    if (!tma_ok(A, lda, dtype) || (a_is_m_by_n && dtype >= SYRK_DTYPE_TF32_F32))
+    // the 16-bit types only).
+    if (!tma_ok(A, lda, dtype) || (a_is_m_by_n && (dtype == SYRK_DTYPE_TF32_F32 || dtype == SYRK_DTYPE_E4M3_F32)))
         return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
     DevicePlan* dp = nullptr;

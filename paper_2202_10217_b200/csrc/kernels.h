@@ -36,7 +36,7 @@ int f64_stages();
 // runs items [d_cta_begin[b], d_cta_begin[b+1]) of the list (n_ctas blocks).  `a_is_m_by_n`: A is
 // stored M x N row-major and `tmA` has boxes of 64 rows x 64 columns over that array.  `a_kind`:
 // 0 bfloat16; 1 binary32 read as TF32 (boxes of 128 rows x 32 columns); 2 FP8 E4M3 bytes (boxes of
-// 128 rows x 128 columns); kinds 1 and 2 in the N x M order only.
+// 128 rows x 128 columns); 3 IEEE binary16 (boxes as for bfloat16); kinds 1 and 2 in the N x M order only.
 cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                              int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,

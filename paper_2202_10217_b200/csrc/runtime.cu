@@ -213,7 +213,8 @@ int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, i
     const CUtensorMapDataType dt =
         (dtype == SYRK_DTYPE_F64) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64
         : (dtype == SYRK_DTYPE_TF32_F32) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
-        : (dtype == SYRK_DTYPE_E4M3_F32) ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+        : (dtype == SYRK_DTYPE_E4M3_F32) ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+        : (dtype == SYRK_DTYPE_F16_F32) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUresult r = fn(tm, dt, 2, const_cast<void*>(A), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

@@ -25,10 +25,10 @@ struct KernelShape {
 };
 KernelShape kernel_shape(int dtype);
 // Element sizes of A and C, and whether the dtype runs on the tcgen05 kernel (BF16, TF32 or FP8 inputs).
-inline size_t a_elem_size(int dtype) { return dtype == 0 ? 8 : (dtype == 1 ? 2 : (dtype == 2 ? 4 : 1)); }
+inline size_t a_elem_size(int dtype) { return dtype == 0 ? 8 : ((dtype == 1 || dtype == 4) ? 2 : (dtype == 2 ? 4 : 1)); }
 inline size_t c_elem_size(int dtype) { return dtype == 0 ? 8 : 4; }
-inline bool is_tcgen05_dtype(int dtype) { return dtype >= 1 && dtype <= 3; }
-inline bool known_dtype(int dtype) { return dtype >= 0 && dtype <= 3; }
+inline bool is_tcgen05_dtype(int dtype) { return dtype >= 1 && dtype <= 4; }
+inline bool known_dtype(int dtype) { return dtype >= 0 && dtype <= 4; }
 
 struct DevicePlan {
     Plan plan;

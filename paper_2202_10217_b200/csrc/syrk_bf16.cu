@@ -1,5 +1,5 @@
-// BF16-in (or TF32-in, or FP8-E4M3-in) / FP32-accumulate triangle-block SYRK kernel for sm_100a
-// (tcgen05 + TMEM).  A stage row is 128 bytes for every input kind: 64 bfloat16 columns
+// BF16-in (or FP16-in, TF32-in, FP8-E4M3-in) / FP32-accumulate triangle-block SYRK kernel for sm_100a
+// (tcgen05 + TMEM).  A stage row is 128 bytes for every input kind: 64 bfloat16 or binary16 columns
 // (kind::f16, K = 16 per MMA), 32 binary32 columns read as TF32 (kind::tf32, K = 8) or 128 FP8
 // columns (kind::f8f6f4, K = 32); everything else is shared.
 //
@@ -67,7 +67,10 @@ __device__ __forceinline__ void tc_commit(uint64_t* bar) {
 constexpr int kKindBF16 = 0;    // 64 bfloat16 columns, kind::f16, K = 16 per instruction
 constexpr int kKindTF32 = 1;    // 32 binary32 columns read as TF32, kind::tf32, K = 8
 constexpr int kKindE4M3 = 2;    // 128 FP8 E4M3 columns, kind::f8f6f4, K = 32
-template <int kKind> struct KindCols { static constexpr int value = kKind == kKindBF16 ? 64 : (kKind == kKindTF32 ? 32 : 128); };
+constexpr int kKindF16 = 3;     // 64 IEEE binary16 columns, kind::f16, K = 16
+template <int kKind> struct KindCols {
+    static constexpr int value = (kKind == kKindBF16 || kKind == kKindF16) ? 64 : (kKind == kKindTF32 ? 32 : 128);
+};
 
 // D[tmem] (+)= A[smem] * B[smem]^T, FP32 accumulation, M = 128; 32 bytes of K per instruction for
 // every kind.
@@ -134,8 +137,8 @@ __device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
 }
 // Instruction descriptor, kind::f16: D = FP32, A = B = BF16, M = 128; both operands K-major, or
 // both MN-major (bits 15 and 16) when A is stored M x N.
-// The other kinds have the same fields; the operand format code is 1 (BF16) for kind::f16,
-// 2 (TF32) for kind::tf32 and 0 (E4M3) for kind::f8f6f4.
+// The other kinds have the same fields; the operand format code is 1 (BF16) or 0 (binary16) for
+// kind::f16, 2 (TF32) for kind::tf32 and 0 (E4M3) for kind::f8f6f4.
 __device__ __forceinline__ uint32_t instr_desc(uint32_t n, bool mn_major, int kind) {
     const uint32_t fmt = kind == kKindBF16 ? 1u : (kind == kKindTF32 ? 2u : 0u);
     return (1u << 4) | (fmt << 7) | (fmt << 10) | (mn_major ? (3u << 15) : 0u) | ((n >> 3) << 17) | ((128u >> 4) << 24);
@@ -475,8 +478,10 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[4] = {reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>),
+        const void* kernels[6] = {reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>),
                                   reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindBF16>),
+                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindF16>),
+                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindF16>),
                                   reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>),
                                   reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>)};
         for (const void* fn : kernels) {
@@ -486,8 +491,9 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
         configured[dev] = true;
     }
     if (n_items == 0) return cudaSuccess;
-    if (a_kind < 0 || a_kind > 2 || (a_kind != 0 && a_is_m_by_n)) return cudaErrorInvalidValue;   // no such kernel
-    const int bk = a_kind == bf16::kKindBF16 ? 64 : (a_kind == bf16::kKindTF32 ? 32 : 128);
+    const bool two_byte = a_kind == bf16::kKindBF16 || a_kind == bf16::kKindF16;
+    if (a_kind < 0 || a_kind > 3 || (!two_byte && a_is_m_by_n)) return cudaErrorInvalidValue;   // no such kernel
+    const int bk = two_byte ? 64 : (a_kind == bf16::kKindTF32 ? 32 : 128);
     const int32_t n_ksteps = int32_t((M + bk - 1) / bk);
     const int split = split_k < 1 ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
     const int64_t n_units = n_items * split;
@@ -497,6 +503,8 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     CUtensorMap none{};
     auto kernel = a_kind == bf16::kKindTF32 ? bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>
                   : a_kind == bf16::kKindE4M3 ? bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>
+                  : a_kind == bf16::kKindF16 ? (a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindF16>
+                                                            : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindF16>)
                   : a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindBF16>
                                 : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>;
     kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(

@@ -5,6 +5,7 @@
 // inputs whose base address or row pitch is not a multiple of 16 bytes, for either storage
 // order of A (N x M, or M x N for the Gram form).
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "kernels.h"
 
@@ -15,6 +16,10 @@ template <typename TA, typename TC> struct Widen;
 template <> struct Widen<double, double> { static __device__ double get(const double* p) { return *p; } };
 template <> struct Widen<__nv_bfloat16, float> {
     static __device__ float get(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+};
+
+template <> struct Widen<__half, float> {
+    static __device__ float get(const __half* p) { return __half2float(*p); }
 };
 
 // binary32 read as TF32: the 13 low-order bits of the encoding are dropped.
@@ -73,6 +78,9 @@ cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, in
     else if (dtype == 3)
         syrk_plain_kernel<uint8_t, float><<<grid2d(N, block), block, 0, stream>>>(
             N, M, static_cast<const uint8_t*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));
+    else if (dtype == 4)
+        syrk_plain_kernel<__half, float><<<grid2d(N, block), block, 0, stream>>>(
+            N, M, static_cast<const __half*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));
     else if (dtype == 2)
         syrk_plain_kernel<float, float><<<grid2d(N, block), block, 0, stream>>>(
             N, M, static_cast<const float*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));

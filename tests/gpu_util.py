@@ -14,18 +14,18 @@ SENTINEL = {np.dtype(np.float64): 0x7FF8DEADBEEF1234, np.dtype(np.float32): 0x7F
 
 
 def a_to_device(A: np.ndarray, dtype: int, lda: int | None = None, offset_elems: int = 0):
-    """Upload A (float64, uint16 bf16 bits, float32 for TF32, or uint8 FP8 bytes) with row pitch lda; returns
+    """Upload A (float64, uint16 bf16 or binary16 bits, float32 for TF32, or uint8 FP8 bytes) with row pitch lda; returns
     (tensor_keepalive, ptr)."""
     N, M = A.shape
     lda = max(M, 1) if lda is None else lda
     tdt = {B.DTYPE_F64: torch.float64, B.DTYPE_BF16_F32: torch.bfloat16, B.DTYPE_TF32_F32: torch.float32,
-           B.DTYPE_E4M3_F32: torch.uint8}[dtype]
+           B.DTYPE_E4M3_F32: torch.uint8, B.DTYPE_F16_F32: torch.float16}[dtype]
     buf = torch.zeros(offset_elems + max(N, 1) * lda, dtype=tdt, device="cuda")
     if N and M:
-        host = torch.from_numpy(np.ascontiguousarray(A).view(np.int16) if dtype == B.DTYPE_BF16_F32
-                                else np.ascontiguousarray(A))
-        if dtype == B.DTYPE_BF16_F32:
-            host = host.view(torch.bfloat16)
+        two_byte = dtype in (B.DTYPE_BF16_F32, B.DTYPE_F16_F32)           # uint16 bit patterns
+        host = torch.from_numpy(np.ascontiguousarray(A).view(np.int16) if two_byte else np.ascontiguousarray(A))
+        if two_byte:
+            host = host.view(tdt)
         view = buf[offset_elems:offset_elems + N * lda].view(N, lda)
         view[:, :M].copy_(host)
     return buf, buf.data_ptr() + offset_elems * buf.element_size()

@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 def upload_A(A, dtype):
     if dtype in (B.DTYPE_F64, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32):
         return torch.from_numpy(A).cuda()
-    return torch.from_numpy(A.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(A.view(np.int16)).cuda().view(torch.float16 if dtype == B.DTYPE_F16_F32 else torch.bfloat16)
 
 
 def sample_pairs(N, count, tile, seed):
@@ -184,11 +184,12 @@ def test_forced_split_k_matches_reference(split):
 
 @pytest.mark.parametrize("dtype,N,M", [(B.DTYPE_BF16_F32, 20001, 104), (B.DTYPE_F64, 12003, 50),
                                        (B.DTYPE_TF32_F32, 16384, 4096), (B.DTYPE_TF32_F32, 20001, 52),
-                                       (B.DTYPE_E4M3_F32, 16384, 8192), (B.DTYPE_E4M3_F32, 20001, 208)])
+                                       (B.DTYPE_E4M3_F32, 16384, 8192), (B.DTYPE_E4M3_F32, 20001, 208),
+                                       (B.DTYPE_F16_F32, 16384, 4096), (B.DTYPE_F16_F32, 20001, 104)])
 def test_large_ragged_sizes_sampled(dtype, N, M):
     """Hundreds of tile rows with a ragged last tile and a ragged last K-step; alpha/beta general."""
     A = {B.DTYPE_F64: I.normal_f64, B.DTYPE_BF16_F32: I.normal_bf16, B.DTYPE_TF32_F32: I.normal_f32,
-         B.DTYPE_E4M3_F32: I.normal_e4m3}[dtype](N, M, 77)
+         B.DTYPE_E4M3_F32: I.normal_e4m3, B.DTYPE_F16_F32: I.normal_f16}[dtype](N, M, 77)
     dA = upload_A(A, dtype)
     tdt = torch.float64 if dtype == B.DTYPE_F64 else torch.float32
     gen = torch.Generator(device="cuda").manual_seed(5)

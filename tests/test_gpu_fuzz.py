@@ -13,7 +13,7 @@ from test_gpu_syrk import ALIGN_ELEMS, make_A
 
 pytestmark = pytest.mark.gpu
 
-DTYPES = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32]
+DTYPES = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32, B.DTYPE_F16_F32]
 SCALARS = [(1.0, 0.0), (-1.0, 1.0), (0.5, -2.0), (2.0, 0.0), (1.0, 1.0), (0.0, 0.5)]
 
 
@@ -21,7 +21,7 @@ SCALARS = [(1.0, 0.0), (-1.0, 1.0), (0.5, -2.0), (2.0, 0.0), (1.0, 1.0), (0.0, 0
 def test_random_cases(chunk):
     rng = np.random.default_rng(9000 + chunk)
     for case in range(12):
-        dtype = DTYPES[int(rng.integers(0, 4))]
+        dtype = DTYPES[int(rng.integers(0, len(DTYPES)))]
         tn = bool(rng.integers(0, 2))
         kind = "int" if rng.integers(0, 3) == 0 else "normal"
         N = int(rng.choice([int(rng.integers(1, 130)), int(rng.integers(130, 700)), int(rng.integers(700, 1700))]))

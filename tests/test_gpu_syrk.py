@@ -16,20 +16,23 @@ from paper_2202_10217_b200 import inputs as I
 from gpu_util import assert_within_tolerance, run_case
 
 pytestmark = pytest.mark.gpu
-BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32]     # every input type of the library
-DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "tf32", "e4m3"])
+BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32,
+        B.DTYPE_F16_F32]                                                     # every input type of the library
+DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "tf32", "e4m3", "f16"])
 A_NUMPY = {B.DTYPE_F64: np.float64, B.DTYPE_BF16_F32: np.uint16, B.DTYPE_TF32_F32: np.float32,
-           B.DTYPE_E4M3_F32: np.uint8}
-ALIGN_ELEMS = {B.DTYPE_F64: 2, B.DTYPE_BF16_F32: 8, B.DTYPE_TF32_F32: 4, B.DTYPE_E4M3_F32: 16}   # elements per 16 bytes
+           B.DTYPE_E4M3_F32: np.uint8, B.DTYPE_F16_F32: np.uint16}
+ALIGN_ELEMS = {B.DTYPE_F64: 2, B.DTYPE_BF16_F32: 8, B.DTYPE_TF32_F32: 4, B.DTYPE_E4M3_F32: 16,
+               B.DTYPE_F16_F32: 8}                                           # elements per 16 bytes
 
 
 def make_A(N, M, dtype, seed, kind="normal"):
     """Real-valued TF32 inputs keep their low-order bits: the library must ignore them."""
     if kind == "int":
         return {B.DTYPE_F64: I.small_int_f64, B.DTYPE_BF16_F32: I.small_int_bf16,
-                B.DTYPE_TF32_F32: I.small_int_f32, B.DTYPE_E4M3_F32: I.small_int_e4m3}[dtype](N, M, seed)
+                B.DTYPE_TF32_F32: I.small_int_f32, B.DTYPE_E4M3_F32: I.small_int_e4m3,
+                B.DTYPE_F16_F32: I.small_int_f16}[dtype](N, M, seed)
     return {B.DTYPE_F64: I.normal_f64, B.DTYPE_BF16_F32: I.normal_bf16, B.DTYPE_TF32_F32: I.normal_f32,
-            B.DTYPE_E4M3_F32: I.normal_e4m3}[dtype](N, M, seed)
+            B.DTYPE_E4M3_F32: I.normal_e4m3, B.DTYPE_F16_F32: I.normal_f16}[dtype](N, M, seed)
 
 
 # Sizes: below one tile, exact tiles, ragged tails in N and M, several tiles, and sizes
@@ -46,7 +49,7 @@ SIZES_E4M3 = [(1, 16), (5, 48), (127, 128), (128, 256), (129, 144), (300, 400), 
 
 def sizes(dtype):
     return {B.DTYPE_F64: SIZES_F64, B.DTYPE_BF16_F32: SIZES_BF16, B.DTYPE_TF32_F32: SIZES_TF32,
-            B.DTYPE_E4M3_F32: SIZES_E4M3}[dtype]
+            B.DTYPE_E4M3_F32: SIZES_E4M3, B.DTYPE_F16_F32: SIZES_BF16}[dtype]
 
 
 @DT
@@ -303,7 +306,7 @@ def test_host_buffer_entry_point_pipelined_blocks(dtype):
     """Inputs large enough for the host entry point to upload A in several column blocks and to
     bring C back in bands (A > 64 MB), with beta != 0, a ragged last block and host pitches."""
     N, M = {B.DTYPE_F64: (1500, 9000), B.DTYPE_BF16_F32: (2304, 24000), B.DTYPE_TF32_F32: (1800, 12100),
-            B.DTYPE_E4M3_F32: (2304, 48000)}[dtype]
+            B.DTYPE_E4M3_F32: (2304, 48000), B.DTYPE_F16_F32: (2304, 24000)}[dtype]
     A = make_A(N, M, dtype, seed=51)
     lda, ldc = M + 16, N + 5
     Abig = np.zeros((N, lda), dtype=A.dtype)
@@ -330,13 +333,13 @@ def test_host_buffer_entry_point_row_band_pipeline(dtype):
     next to the band and tile boundaries of a few rows; upper triangle and padding untouched."""
     import torch
     N, M = {B.DTYPE_F64: (4100, 200), B.DTYPE_BF16_F32: (4500, 520), B.DTYPE_TF32_F32: (4230, 260),
-            B.DTYPE_E4M3_F32: (4400, 1040)}[dtype]
+            B.DTYPE_E4M3_F32: (4400, 1040), B.DTYPE_F16_F32: (4500, 520)}[dtype]
     A = make_A(N, M, dtype, seed=71)
     lda, ldc = M + 32, N + 6
     Abig = np.zeros((N, lda), dtype=A.dtype)
     Abig[:, :M] = A
     Cin = I.random_c(N, 72, dtype, ldc)
-    hA = torch.from_numpy(Abig.view(np.int16) if dtype == B.DTYPE_BF16_F32 else Abig).pin_memory()
+    hA = torch.from_numpy(Abig.view(np.int16) if Abig.dtype == np.uint16 else Abig).pin_memory()
     hC = torch.from_numpy(Cin.copy()).pin_memory()
     for alpha, beta in ((0.5, -1.0), (1.0, 0.0)):
         hC.copy_(torch.from_numpy(Cin))

@@ -14,8 +14,8 @@ from gpu_util import assert_within_tolerance, run_case
 from test_gpu_syrk import make_A
 
 pytestmark = pytest.mark.gpu
-BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32]
-DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16"])
+BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_F16_F32]     # the types with a tensor-core path in this order
+DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "f16"])
 
 # N even keeps the pitch of the M x N array a multiple of 16 bytes (tensor-core path in FP64);
 # odd N takes the plain-load kernel.  Ragged tiles in N (not a multiple of 32) and ragged
@@ -24,6 +24,7 @@ SIZES = {B.DTYPE_F64: [(2, 1), (6, 3), (30, 17), (32, 16), (34, 50), (100, 64), 
                        (1000, 70), (1300, 40), (2500, 33), (33, 20), (257, 19)],
          B.DTYPE_BF16_F32: [(8, 8), (40, 24), (128, 64), (136, 72), (304, 200), (777, 136), (512, 256),
                             (1104, 320), (2056, 72), (1304, 1000)]}
+SIZES[B.DTYPE_F16_F32] = SIZES[B.DTYPE_BF16_F32]
 
 
 @DT
@@ -94,17 +95,18 @@ def test_leading_dimension_smaller_than_N_is_refused():
         B.syrk_lower_tn(64, 16, 8, 32, 8, 64, 1.0, 0.0, B.DTYPE_F64, stream=0)
 
 
+@pytest.mark.parametrize("dtype", [B.DTYPE_BF16_F32, B.DTYPE_F16_F32], ids=["bf16", "f16"])
 @pytest.mark.parametrize("split", [0, 2, 5])
-def test_bf16_k_split_in_this_storage_order(split):
+def test_bf16_k_split_in_this_storage_order(split, dtype):
     N, M = 704, 1280
-    A = I.small_int_bf16(N, M, seed=40 + split)
-    Cin = I.random_c(N, 41, B.DTYPE_BF16_F32)
+    A = make_A(N, M, dtype, seed=40 + split, kind="int")
+    Cin = I.random_c(N, 41, dtype)
     try:
         B.syrk_set_split_k(split)
-        got, ref, bound = run_case(A, B.DTYPE_BF16_F32, 2.0, -1.0, Cin, tn=True)
+        got, ref, bound = run_case(A, dtype, 2.0, -1.0, Cin, tn=True)
     finally:
         B.syrk_set_split_k(0)
-    assert_within_tolerance(got, ref, bound, M, 2.0, -1.0, Cin, B.DTYPE_BF16_F32)
+    assert_within_tolerance(got, ref, bound, M, 2.0, -1.0, Cin, dtype)
 
 
 @pytest.mark.parametrize("dtype", [B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32], ids=["tf32", "e4m3"])
