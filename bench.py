@@ -190,6 +190,9 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
         torch.cuda.synchronize()
 
     N, M, dtype = wl.N, wl.M, wl.dtype
+    if args.batch > 0:
+        run_batched(args, wl)
+        return
     A_host = wl.make_A()
     cdt = I.c_storage_dtype(dtype)
     if dtype in (I.DTYPE_F64, I.DTYPE_TF32_F32, I.DTYPE_E4M3_F32):
@@ -403,6 +406,51 @@ def run_sweep(args, rank: int, world: int, local_rank: int):
         dist.destroy_process_group()
 
 
+def run_batched(args, wl):
+    """--kernel-only --batch B: B seeded problems of the workload's shape through syrk_lower_batched,
+    beside the same B problems enqueued one by one with syrk_lower (device-timed, L2 flushed)."""
+    import torch
+    from paper_2202_10217_b200 import binding as B
+
+    N, M, dtype, nb = wl.N, wl.M, wl.dtype, args.batch
+    tall = I.Workload(wl.name, nb * N, M, dtype, wl.alpha, wl.beta, wl.seed, wl.dist, wl.std).make_A()
+    dA = torch.from_numpy(tall.view(np.int16) if tall.dtype == np.uint16 else tall).cuda()   # nb matrices, stride N * M
+    dC = torch.zeros((nb, N, N), dtype=torch.float64 if dtype == I.DTYPE_F64 else torch.float32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    ea, ec = dA.element_size(), dC.element_size()
+
+    def batched():
+        B.syrk_lower_batched(nb, N, M, dA, M, N * M, dC, N, N * N, wl.alpha, wl.beta, dtype)
+
+    def one_by_one():
+        for b in range(nb):
+            B.syrk_lower(N, M, dA.data_ptr() + b * N * M * ea, M, dC.data_ptr() + b * N * N * ec, N,
+                         wl.alpha, wl.beta, dtype)
+
+    out = {}
+    for name, call in (("batched", batched), ("one_by_one", one_by_one)):
+        for _ in range(max(args.warmup, 1)):
+            call()
+        torch.cuda.synchronize()
+        assert B.syrk_last_status() == 0
+        times = []
+        for _ in range(args.steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            call()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        out[name] = float(np.mean(times))
+    assert B.syrk_last_status() == 0
+    print(json.dumps({"metric": METRIC, "value": nb * wl.flops / (out["batched"] * 1e-3) * 1e-12, "unit": UNIT,
+                      "n_gpus": 1, "steps": args.steps, "ms_per_step": out["batched"], "kernel_only": True,
+                      "one_by_one_ms": out["one_by_one"],
+                      "one_by_one_value": nb * wl.flops / (out["one_by_one"] * 1e-3) * 1e-12,
+                      "config": {"workload": wl.name, "N": N, "M": M, "batch": nb}}))
+
+
 def run_cholesky(args, rank: int, world: int, local_rank: int):
     """Large Block Cholesky of a seeded 32768^2 FP64 matrix (n*I + G G^T / 512); a step is one
     factorisation (the matrix is restored from a device copy between steps, outside the timing)."""
@@ -460,8 +508,12 @@ def main():
                          "for short profiler runs")
     ap.add_argument("--gram", action="store_true",
                     help="with --kernel-only: hand the operand over stored M x N and time syrk_lower_tn (C = A^T A)")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="with --kernel-only: that many problems of the workload's shape through syrk_lower_batched")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
+    if args.batch > 0 and not args.kernel_only:
+        ap.error("--batch needs --kernel-only")
     if args.gram and not args.kernel_only:
         ap.error("--gram needs --kernel-only (the host-buffer entry point takes the N x M form)")
     rank = int(os.environ.get("RANK", "0"))

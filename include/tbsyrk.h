@@ -118,6 +118,31 @@ int syrk_lower_tn(int64_t N, int64_t M,
                   int dtype, void* stream);
 
 /*
+ * A strided batch of independent updates of the same shape:
+ *
+ *     C_b[i][j] = alpha * sum_k A_b[i][k] * A_b[j][k] + beta * C_b[i][j]    0 <= j <= i < N, 0 <= b < batch,
+ *
+ * i.e. Algorithm 1 of the paper applied to each of `batch` problems, with A_b = A + b * stride_a
+ * (N x M row-major, pitch lda) and C_b = C + b * stride_c (N x N row-major, pitch ldc), all DEVICE
+ * memory, strides in elements.  The paper states the update for one matrix; the batch exists because a
+ * small problem (tens of work items) cannot fill the GPU on its own: every matrix uses the work list
+ * of Algorithm 4 / Section 5.1.4 for its N, and one launch runs the (matrix, item) pairs of the whole
+ * batch (FP64: one thread block per pair; tcgen05 types: pairs dealt to the persistent blocks; the
+ * inner dimension is never split here).  Requirements for that single launch: A 16-byte aligned and
+ * lda * sizeof(element) and stride_a * sizeof(element) multiples of 16; otherwise, and for alpha == 0
+ * or M == 0, the matrices are enqueued one after the other exactly as `batch` syrk_lower calls.
+ * Matrices must not overlap: for batch > 1, stride_a >= (N-1) * lda + M and stride_c >= (N-1) * ldc + N
+ * (else SYRK_ERR_LD); batch < 0 or batch * items >= 2^31 gives SYRK_ERR_SIZE; batch == 0 returns at
+ * once.  Everything else (upper triangles untouched, beta == 0 not reading C, ownership, stream
+ * semantics, error codes) is as for syrk_lower.
+ */
+int syrk_lower_batched(int64_t batch, int64_t N, int64_t M,
+                       const void* A, int64_t lda, int64_t stride_a,
+                       void* C, int64_t ldc, int64_t stride_c,
+                       double alpha, double beta,
+                       int dtype, void* stream);
+
+/*
  * Same operation with HOST buffers: copies A (and C when beta != 0) to the
  * device, runs syrk_lower on a stream of the library, copies the lower triangle
  * back into C, and waits for completion.  A and C are host pointers (pageable or

@@ -219,6 +219,56 @@ int syrk_lower_tn(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int
     return syrk_run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream), -1, 1);
 }
 
+int syrk_lower_batched(int64_t batch, int64_t N, int64_t M, const void* A, int64_t lda, int64_t stride_a,
+                       void* C, int64_t ldc, int64_t stride_c, double alpha, double beta, int dtype, void* stream) {
+    if (batch < 0 || batch >= (int64_t(1) << 31)) return SYRK_ERR_SIZE;
+    int rc = validate(N, M, A, lda, C, ldc, dtype);
+    if (rc != SYRK_OK || N == 0 || batch == 0) return rc;
+    if (batch > 1 && ((M > 0 && stride_a < (N - 1) * lda + M) || stride_c < (N - 1) * ldc + N)) return SYRK_ERR_LD;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t ea = a_elem(dtype), ec = c_elem(dtype);
+    // One launch over all matrices needs 3-D tensor maps: base and both pitches of A multiples of 16
+    // bytes.  Otherwise (and for the quick returns) the matrices are enqueued one by one.
+    const bool one_launch = alpha != 0.0 && M > 0 && batch > 1 && tma_ok(A, lda, dtype) && (size_t(stride_a) * ea) % 16 == 0;
+    if (!one_launch) {
+        for (int64_t b = 0; b < batch; ++b) {
+            rc = syrk_run_device(N, M, static_cast<const char*>(A) + size_t(b) * size_t(stride_a) * ea, lda,
+                                 static_cast<char*>(C) + size_t(b) * size_t(stride_c) * ec, ldc, alpha, beta, dtype, st);
+            if (rc != SYRK_OK) return rc;
+        }
+        return SYRK_OK;
+    }
+    DeviceState* ds = nullptr;
+    rc = get_device_state(&ds);
+    if (rc != SYRK_OK) return rc;
+    DevicePlan* dp = nullptr;
+    rc = get_device_plan(ds, N, dtype, &dp);
+    if (rc != SYRK_OK) return rc;
+    const KernelShape ks = kernel_shape(dtype);
+    const int64_t n_items = int64_t(dp->plan.items.size());
+    if (n_items * batch >= (int64_t(1) << 31)) return SYRK_ERR_SIZE;
+    CUtensorMap tm, tmc;
+    rc = encode_tensor_map_batched(&tm, dtype, A, N, M, lda, stride_a, batch, ks.tile, ks.bk);
+    if (rc != SYRK_OK) return rc;
+    const bool c_aligned = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (size_t(ldc) * ec) % 16 == 0 &&
+                           (size_t(stride_c) * ec) % 16 == 0;
+    cudaError_t e;
+    if (dtype == SYRK_DTYPE_F64) {
+        const bool c_tma = beta != 0.0 && c_aligned &&
+                           encode_tensor_map_c_batched(&tmc, 1, C, N, ldc, stride_c, batch, f64_tile()) == SYRK_OK;
+        e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha,
+                            beta, 0, nullptr, 0, ds->d_status, st, batch, stride_c);
+    } else {
+        const bool c_tma = c_aligned &&
+                           encode_tensor_map_c_batched(&tmc, 0, C, N, ldc, stride_c, batch, bf16_store_box()) == SYRK_OK;
+        e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc,
+                             float(alpha), float(beta), 1, nullptr, dp->d_tile_base, dp->total_tiles, nullptr, 0, 0,
+                             dtype - SYRK_DTYPE_BF16_F32, ds->d_status, ds->sm_count, st, batch, stride_c);
+    }
+    return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
 int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
                     double beta, int dtype) {
     int rc = validate(N, M, A, lda, C, ldc, dtype);

@@ -87,6 +87,25 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
         : "memory");
 }
 
+// The same for a 3-D tensor map whose outermost coordinate z selects one matrix of a strided
+// batch (box depth 1): the box lands in shared memory exactly as a 2-D box would.
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* tmap, int32_t x,
+                                            int32_t y, int32_t z, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z),
+          "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Box load from a 2-D map (z < 0) or from matrix z of a batched 3-D map.
+__device__ __forceinline__ void tma_load_box(void* smem_dst, const CUtensorMap* tmap, int32_t x,
+                                             int32_t y, int32_t z, uint64_t* bar) {
+    if (z < 0) tma_load_2d(smem_dst, tmap, x, y, bar);
+    else tma_load_3d(smem_dst, tmap, x, y, z, bar);
+}
+
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }

@@ -14,10 +14,13 @@ namespace tbsyrk {
 // d_tickets[0] (d_tickets[0..1] must be zero and must not be shared with a launch that can run at
 // the same time; the kernel leaves them zero).  `a_is_m_by_n`: A is stored M x N row-major (the
 // Gram form C = A^T A); `tmA` then has boxes of 16 rows x 16 columns over that array.
+// `batch` > 0: strided batch of `batch` problems; `tmA` and `tmC` are then 3-D maps whose last
+// coordinate is the matrix number, matrix b of C starts at C + b * c_batch_stride, and the launch
+// has one block per (matrix, item).
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
-                            cudaStream_t stream);
+                            cudaStream_t stream, int64_t batch = 0, int64_t c_batch_stride = 0);
 // The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
 // P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
 // columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.
@@ -37,11 +40,14 @@ int f64_stages();
 // stored M x N row-major and `tmA` has boxes of 64 rows x 64 columns over that array.  `a_kind`:
 // 0 bfloat16; 1 binary32 read as TF32 (boxes of 128 rows x 32 columns); 2 FP8 E4M3 bytes (boxes of
 // 128 rows x 128 columns); 3 IEEE binary16 (boxes as for bfloat16); kinds 1 and 2 in the N x M order only.
+// `batch` > 0: strided batch (3-D maps as for the FP64 kernel); the units are then (matrix, item)
+// pairs dealt round-robin, split_k must be 1.
 cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                              int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
-                             int a_kind, int* d_status, int sm_count, cudaStream_t stream);
+                             int a_kind, int* d_status, int sm_count, cudaStream_t stream,
+                             int64_t batch = 0, int64_t c_batch_stride = 0);
 int bf16_tile();
 int bf16_bk();
 int bf16_stages();

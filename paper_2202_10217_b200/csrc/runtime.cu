@@ -234,6 +234,46 @@ int encode_tensor_map_c_f32(CUtensorMap* tm, const void* C, int64_t N, int64_t l
     return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
+// Strided batch: a third dimension of `batch` matrices `stride` elements apart (box depth 1).
+int encode_tensor_map_batched(CUtensorMap* tm, int dtype, const void* A, int64_t N, int64_t M, int64_t lda,
+                              int64_t stride, int64_t batch, int box_rows, int box_cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SYRK_ERR_CUDA;
+    const size_t es = a_elem_size(dtype);
+    const cuuint64_t dims[3] = {cuuint64_t(M), cuuint64_t(N), cuuint64_t(batch)};
+    const cuuint64_t strides[2] = {cuuint64_t(lda) * es, cuuint64_t(stride) * es};
+    const cuuint32_t box[3] = {cuuint32_t(box_cols), cuuint32_t(box_rows), 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUtensorMapDataType dt =
+        (dtype == SYRK_DTYPE_F64) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64
+        : (dtype == SYRK_DTYPE_TF32_F32) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+        : (dtype == SYRK_DTYPE_E4M3_F32) ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+        : (dtype == SYRK_DTYPE_F16_F32) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult r = fn(tm, dt, 3, const_cast<void*>(A), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
+// C of a strided batch: square boxes of `box` elements, 128-byte swizzle for binary32 (the store
+// path of the tcgen05 kernel), none for binary64 (old-C tiles of the FP64 kernel).
+int encode_tensor_map_c_batched(CUtensorMap* tm, int is_f64, const void* C, int64_t N, int64_t ldc,
+                                int64_t stride, int64_t batch, int box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SYRK_ERR_CUDA;
+    const size_t es = is_f64 ? 8 : 4;
+    const cuuint64_t dims[3] = {cuuint64_t(N), cuuint64_t(N), cuuint64_t(batch)};
+    const cuuint64_t strides[2] = {cuuint64_t(ldc) * es, cuuint64_t(stride) * es};
+    const cuuint32_t bx[3] = {cuuint32_t(box), cuuint32_t(box), 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = fn(tm, is_f64 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
+                          const_cast<void*>(C), dims, strides, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          is_f64 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                          is_f64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
 int encode_tensor_map_f64_plain(CUtensorMap* tm, const void* p, int64_t rows, int64_t cols, int64_t ld,
                                 int box_rows, int box_cols) {
     EncodeTiledFn fn = encode_fn();

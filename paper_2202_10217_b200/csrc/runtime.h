@@ -102,6 +102,10 @@ int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, i
                          int64_t lda, int box_rows, int box_cols);
 
 // 2-D row-major FP32 tensor map over C (N x N, pitch ldc) with box x box boxes, 128-byte swizzle.
+int encode_tensor_map_batched(CUtensorMap* tm, int dtype, const void* A, int64_t N, int64_t M, int64_t lda,
+                              int64_t stride, int64_t batch, int box_rows, int box_cols);
+int encode_tensor_map_c_batched(CUtensorMap* tm, int is_f64, const void* C, int64_t N, int64_t ldc,
+                                int64_t stride, int64_t batch, int box);
 int encode_tensor_map_c_f32(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box);
 // The same over an FP64 C, without swizzle (a box row of 32 doubles is 256 bytes).
 int encode_tensor_map_c_f64(CUtensorMap* tm, const void* C, int64_t N, int64_t ldc, int box);

@@ -150,19 +150,31 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, const void
                  ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(smem_src)) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
+// The same into matrix z of a strided batch (3-D map, box depth 1).
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tmap, const void* smem_src, int32_t x, int32_t y, int32_t z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(smem_u32(smem_src)) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
 __device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-struct Unit {       // one work unit: an item and a range of K-steps
+struct Unit {       // one work unit: an item and a range of K-steps (or a matrix of a strided batch)
     int64_t item;
     int32_t slice;
     int32_t k0, k1;
+    int32_t batch;      // matrix number, or -1 outside batched calls
 };
-__device__ __forceinline__ Unit unit_of(int64_t w, int64_t n_items, int32_t n_ksteps, int32_t split) {
+__device__ __forceinline__ Unit unit_of(int64_t w, int64_t n_items, int32_t n_ksteps, int32_t split, int32_t n_batch) {
     Unit u;
-    u.slice = int32_t(w / n_items);               // slice-major: a wave shares one K-slab of A
     u.item = w % n_items;
+    if (n_batch > 0) {                            // batched calls: matrix-major, whole inner dimension
+        u.batch = int32_t(w / n_items); u.slice = 0; u.k0 = 0; u.k1 = n_ksteps;
+        return u;
+    }
+    u.batch = -1;
+    u.slice = int32_t(w / n_items);               // slice-major: a wave shares one K-slab of A
     u.k0 = int32_t(int64_t(n_ksteps) * u.slice / split);
     u.k1 = int32_t(int64_t(n_ksteps) * (u.slice + 1) / split);
     return u;
@@ -199,7 +211,8 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                      const WorkItem* __restrict__ items, int64_t n_items, int64_t N, int32_t n_ksteps,
                      float* __restrict__ C, int64_t ldc, float alpha, float beta, int vec_ok, int tma_store_ok,
                      int32_t split, float* __restrict__ partial, const int64_t* __restrict__ tile_base,
-                     int64_t total_tiles, const int64_t* __restrict__ cta_begin, int* __restrict__ status) {
+                     int64_t total_tiles, const int64_t* __restrict__ cta_begin, int* __restrict__ status,
+                     int32_t n_batch, int64_t c_batch_stride) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* staging = smem + kStages * kStageBytes;
@@ -214,7 +227,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     constexpr int kCols = KindCols<kKind>::value;        // columns of A in a 128-byte stage row
-    const int64_t n_units = n_items * split;
+    const int64_t n_units = n_items * split * (n_batch > 0 ? n_batch : 1);
     // This block's units: its own contiguous range of a list ordered block by block on the host,
     // or (K-split calls) every gridDim.x-th unit of the slice-major list.
     const int64_t w_first = cta_begin ? cta_begin[blockIdx.x] : int64_t(blockIdx.x);
@@ -243,7 +256,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             prefetch_tensormap(&tmA);
             uint32_t g = 0;
             for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride) {
-                const Unit u = unit_of(w, n_items, n_ksteps, split);
+                const Unit u = unit_of(w, n_items, n_ksteps, split, n_batch);
                 const WorkItem* it = &items[u.item];
                 const int n_seg = it->n_seg;
                 int32_t rows[kSegSlots];
@@ -258,11 +271,11 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (kTN) {   // A stored M x N: two boxes of 64 k-rows x 64 columns per segment
                         for (int s = 0; s < n_seg; ++s)
                             for (int h = 0; h < 2; ++h)
-                                tma_load_2d(dst + s * kSegBytes + h * (kSegBytes / 2), &tmA, rows[s] + h * 64, ks * kCols,
-                                            &full_bar[st]);
+                                tma_load_box(dst + s * kSegBytes + h * (kSegBytes / 2), &tmA, rows[s] + h * 64, ks * kCols,
+                                             u.batch, &full_bar[st]);
                     } else {
                         for (int s = 0; s < n_seg; ++s)
-                            tma_load_2d(dst + s * kSegBytes, &tmA, ks * kCols, rows[s], &full_bar[st]);
+                            tma_load_box(dst + s * kSegBytes, &tmA, ks * kCols, rows[s], u.batch, &full_bar[st]);
                     }
                 }
             }
@@ -281,7 +294,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const uint64_t desc_hi = kTN ? smem_desc_mn_sw128(0) : smem_desc_sw128(0);
             constexpr uint32_t kk_step = kTN ? (2048u >> 4) : (32u >> 4);   // descriptor advance per K = 16
             for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride, ++n_done) {
-                const Unit u = unit_of(w, n_items, n_ksteps, split);
+                const Unit u = unit_of(w, n_items, n_ksteps, split, n_batch);
                 const WorkItem* it = &items[u.item];
                 Layout L;
                 layout_of(it, it->n_tile, (n_done & 1) ? 3u * kTile : 0u, L);
@@ -336,7 +349,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         uint8_t* my_staging = staging + (warp - 2) * 2 * kStageBufBytes;
         uint32_t n_done = 0, n_stores = 0;
         for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride, ++n_done) {
-            const Unit u = unit_of(w, n_items, n_ksteps, split);
+            const Unit u = unit_of(w, n_items, n_ksteps, split, n_batch);
             const WorkItem* it = &items[u.item];
             const int n_tile = it->n_tile;
             Layout L;
@@ -347,6 +360,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 tcol[t] = (t < n_tile) ? it->seg[it->tile_y[t]] : 0;
             }
             const int64_t slot0 = (split > 1) ? tile_base[u.item] : 0;
+            float* Cb = (u.batch > 0) ? C + int64_t(u.batch) * c_batch_stride : C;     // this unit's matrix
             if (!mbar_wait_bounded(tmem_full_bar, n_done & 1, &s_abort)) {
                 s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitMma); break;
             }
@@ -384,13 +398,15 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                                                 alpha * __uint_as_float(v[4 * j + 2]), alpha * __uint_as_float(v[4 * j + 3]));
                             fence_async_smem();
                             __syncwarp();
-                            if (lane == 0)
-                                tma_store_2d(&tmC, buf, int32_t(c0), int32_t(trow[t] * kTile + quarter * 32));
+                            if (lane == 0) {
+                                if (u.batch < 0) tma_store_2d(&tmC, buf, int32_t(c0), int32_t(trow[t] * kTile + quarter * 32));
+                                else tma_store_3d(&tmC, buf, int32_t(c0), int32_t(trow[t] * kTile + quarter * 32), u.batch);
+                            }
                             ++n_stores;
                             continue;
                         }
                         if (r >= N) continue;
-                        float* crow = C + r * ldc + c0;
+                        float* crow = Cb + r * ldc + c0;
                         if (c0 + 31 <= r && vec_ok) {
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
@@ -471,7 +487,8 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                              int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
-                             int a_kind, int* d_status, int sm_count, cudaStream_t stream) {
+                             int a_kind, int* d_status, int sm_count, cudaStream_t stream, int64_t batch,
+                             int64_t c_batch_stride) {
     // The shared-memory attribute belongs to a device's context: set it once per device.
     static bool configured[64] = {};
     int dev = 0;
@@ -496,10 +513,12 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     const int bk = two_byte ? 64 : (a_kind == bf16::kKindTF32 ? 32 : 128);
     const int32_t n_ksteps = int32_t((M + bk - 1) / bk);
     const int split = split_k < 1 ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
-    const int64_t n_units = n_items * split;
-    const bool ranges = (d_cta_begin != nullptr && split == 1 && n_ctas > 0);
+    if (batch > 0 && (split != 1 || batch >= (int64_t(1) << 31))) return cudaErrorInvalidValue;
+    const int64_t n_units = n_items * split * (batch > 0 ? batch : 1);
+    const bool ranges = (d_cta_begin != nullptr && split == 1 && n_ctas > 0 && batch <= 0);
     const unsigned grid = ranges ? unsigned(n_ctas) : unsigned(n_units < sm_count ? n_units : sm_count);
-    const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0) ? 1 : 0;
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
+                        (batch <= 0 || (c_batch_stride & 3) == 0)) ? 1 : 0;
     CUtensorMap none{};
     auto kernel = a_kind == bf16::kKindTF32 ? bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>
                   : a_kind == bf16::kKindE4M3 ? bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>
@@ -509,7 +528,8 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                                 : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>;
     kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
         tmA, tmC ? *tmC : none, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, split,
-        d_partial, d_tile_base, total_tiles, ranges ? d_cta_begin : nullptr, d_status);
+        d_partial, d_tile_base, total_tiles, ranges ? d_cta_begin : nullptr, d_status, int32_t(batch > 0 ? batch : 0),
+        c_batch_stride);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || split == 1) return e;
     bf16::splitk_reduce_kernel<<<dim3(unsigned(n_items), bf16::kMaxTiles), 256, 0, stream>>>(

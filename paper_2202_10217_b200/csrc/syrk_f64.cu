@@ -73,6 +73,7 @@ struct Call {
     int64_t ldc;
     double alpha, beta;
     int vec_ok, c_tma;
+    int32_t batch;                 // matrix of a strided batch the block works on (tensor maps are 3-D), or -1
     bool gemm;
 };
 
@@ -97,12 +98,12 @@ __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, 
             // (128-byte rows of 16 columns, one row per k), 2 KB each.
             for (int s = 0; s < n_seg; ++s)
                 for (int h = 0; h < 2; ++h)
-                    tma_load_2d(dst + s * kSegBytes + h * (kSegBytes / 2), k.tmA, it.seg[s] * kTile + h * 16, ks * kBK,
-                                &k.full_bar[st]);
+                    tma_load_box(dst + s * kSegBytes + h * (kSegBytes / 2), k.tmA, it.seg[s] * kTile + h * 16, ks * kBK,
+                                 k.batch, &k.full_bar[st]);
         } else {
             for (int s = 0; s < n_seg; ++s)
-                tma_load_2d(dst + s * kSegBytes, (k.gemm && s < it.pad) ? k.tmB : k.tmA, ks * kBK, it.seg[s] * kTile,
-                            &k.full_bar[st]);
+                tma_load_box(dst + s * kSegBytes, (k.gemm && s < it.pad) ? k.tmB : k.tmA, ks * kBK, it.seg[s] * kTile,
+                             k.batch, &k.full_bar[st]);
         }
     }
     // Old C: ring step j carries tiles 4j .. 4j+3 (8 KB each, row pitch 256 B), those below the diagonal.
@@ -120,7 +121,8 @@ __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, 
         uint8_t* dst = k.smem + st * kStageBytes;
         for (int tt = 4 * j; tt < n_tile && tt < 4 * j + 4; ++tt) {
             const int rx = it.seg[it.tile_x[tt]], cy = it.seg[it.tile_y[tt]];
-            if (k.gemm || rx != cy) tma_load_2d(dst + (tt & 3) * kCTileBytes, k.tmC, cy * kTile, rx * kTile, &k.full_bar[st]);
+            if (k.gemm || rx != cy)
+                tma_load_box(dst + (tt & 3) * kCTileBytes, k.tmC, cy * kTile, rx * kTile, k.batch, &k.full_bar[st]);
         }
     }
     return true;
@@ -405,7 +407,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
                     int64_t ncols, int32_t gemm_col_tiles, int32_t n_ksteps, double* __restrict__ C,
-                    int64_t ldc, double alpha, double beta, int vec_ok, int c_tma, int* __restrict__ status) {
+                    int64_t ldc, double alpha, double beta, int vec_ok, int c_tma, int* __restrict__ status,
+                    int64_t items_per_batch, int64_t c_batch_stride) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ WorkItem s_item;
@@ -421,6 +424,14 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     k.tmA = &tmA; k.tmB = &tmB; k.tmC = &tmC;
     k.N = N; k.ncols = ncols; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
     k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = gemm_col_tiles > 0;
+    // Strided batch: the grid holds the work list once per matrix; the tensor maps are 3-D.
+    k.batch = -1;
+    int64_t item_index = blockIdx.x;
+    if (items_per_batch > 0) {
+        k.batch = int32_t(int64_t(blockIdx.x) / items_per_batch);
+        item_index = int64_t(blockIdx.x) % items_per_batch;
+        k.C = C + int64_t(k.batch) * c_batch_stride;
+    }
 
     if (k.gemm) {
         if (tid == 0) {
@@ -437,7 +448,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             s_item.n_seg = nc + nr; s_item.n_tile = tt; s_item.kind = kRect; s_item.pad = nc;
         }
     } else if (tid < int(sizeof(WorkItem) / 4)) {
-        reinterpret_cast<int32_t*>(&s_item)[tid] = reinterpret_cast<const int32_t*>(&items[blockIdx.x])[tid];
+        reinterpret_cast<int32_t*>(&s_item)[tid] = reinterpret_cast<const int32_t*>(&items[item_index])[tid];
     }
     if (tid == 0) s_abort = 0;
     __syncthreads();
@@ -492,7 +503,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
     k.abort_flag = &s_abort; k.status = status;
     k.tmA = &tmA; k.tmB = &tmA; k.tmC = &tmC;
     k.N = N; k.ncols = N; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
-    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false;
+    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false; k.batch = -1;
 
     if (tid == 0) {
         s_abort = 0;
@@ -570,15 +581,25 @@ cudaError_t configure_f64_kernels() {
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, int64_t batch, int64_t c_batch_stride) {
     cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
-    const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0) ? 1 : 0;
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
+                        (batch <= 0 || (c_batch_stride & 1) == 0)) ? 1 : 0;
     const int32_t n_ksteps = int32_t((M + f64::kBK - 1) / f64::kBK);
     const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
     CUtensorMap none{};
     const dim3 threads(f64::kThreads);
+    if (batch > 0) {
+        // Strided batch (3-D tensor maps): one block per (matrix, item), matrix-major.
+        if (n_items * batch >= (int64_t(1) << 31)) return cudaErrorInvalidValue;
+        auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
+        kernel<<<dim3(unsigned(n_items * batch)), threads, f64::kSmemBytes, stream>>>(
+            tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
+            n_items, c_batch_stride);
+        return cudaGetLastError();
+    }
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true> : f64::syrk_f64_tbs_persistent_kernel<false>;
@@ -588,7 +609,8 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
     }
     auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
     kernel<<<dim3(unsigned(n_items)), threads, f64::kSmemBytes, stream>>>(
-        tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
+        tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
+        int64_t(0), int64_t(0));
     return cudaGetLastError();
 }
 
@@ -606,7 +628,7 @@ cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, c
     CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<false><<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmP, tmQ, c_tma ? *tmD : none, nullptr, nrows, ncols, int32_t(col_tiles), n_ksteps, D, ldd, alpha, beta,
-        vec_ok, c_tma, d_status);
+        vec_ok, c_tma, d_status, int64_t(0), int64_t(0));
     return cudaGetLastError();
 }
 
