@@ -35,13 +35,11 @@ extern "C" {
                                   fraction bits: the 13 low-order bits of every element are
                                   ignored), C binary32; binary32 accumulation (tcgen05
                                   kind::tf32).  The paper fixes no input precision; this is
-                                  the same update on FP32 data.  syrk_lower_tn takes this
-                                  type through the plain-load kernel only.                */
+                                  the same update on FP32 data.                           */
 #define SYRK_DTYPE_E4M3_F32 3  /* A bytes in the OCP FP8 format E4M3 (1 sign, 4 exponent bits
                                   with bias 7, 3 fraction bits; no infinities; 0x7F and 0xFF
                                   are NaN; largest value 448), C binary32; binary32
-                                  accumulation (tcgen05 kind::f8f6f4).  syrk_lower_tn takes
-                                  this type through the plain-load kernel only.           */
+                                  accumulation (tcgen05 kind::f8f6f4).                    */
 #define SYRK_DTYPE_F16_F32  4  /* A IEEE 754 binary16 (1 sign, 5 exponent bits with bias 15,
                                   10 fraction bits; subnormals, infinities and NaN as in
                                   the standard), C binary32; binary32 accumulation (tcgen05
@@ -108,8 +106,8 @@ int syrk_lower(int64_t N, int64_t M,
  * Section 5.1.4), C, alpha, beta, dtype, stream, alignment rule (A 16-byte aligned and
  * lda * sizeof(element) a multiple of 16, else a slower plain-load kernel), ownership
  * and error codes are those of syrk_lower (SYRK_ERR_LD refers to lda < N here).
- * FP64 and the 16-bit types run on the tensor-core kernels (FP64: both launch forms;
- * bfloat16 and binary16: tcgen05 with MN-major operands, K-split included).
+ * Every dtype runs on the tensor-core kernels (FP64: both launch forms; the others:
+ * tcgen05 with MN-major operands, K-split included).
  */
 int syrk_lower_tn(int64_t N, int64_t M,
                   const void* A, int64_t lda,

@@ -151,9 +151,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         if (beta == 1.0) return SYRK_OK;
         return launch_scale_lower(dtype, N, C, ldc, beta, stream) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
     }
-    // TF32 and FP8 inputs stored M x N have no tensor-core path (MN-major operands are used for
-    // the 16-bit types only).
-    if (!tma_ok(A, lda, dtype) || (a_is_m_by_n && (dtype == SYRK_DTYPE_TF32_F32 || dtype == SYRK_DTYPE_E4M3_F32)))
+    if (!tma_ok(A, lda, dtype))
         return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
     DevicePlan* dp = nullptr;
@@ -162,7 +160,8 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
     const KernelShape ks = kernel_shape(dtype);
     CUtensorMap tm;
     // A stored M x N: boxes of one stage's k-rows x 128 bytes of columns (16 doubles, 64 bf16)
-    if (a_is_m_by_n) rc = encode_tensor_map_2d(&tm, dtype, A, M, N, lda, ks.bk, dtype == SYRK_DTYPE_F64 ? 16 : 64);
+    if (a_is_m_by_n) rc = encode_tensor_map_2d(&tm, dtype, A, M, N, lda, ks.bk, 128 / int(a_elem(dtype)),
+                                               dtype == SYRK_DTYPE_TF32_F32);
     else rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, ks.tile, ks.bk);
     if (rc != SYRK_OK) return rc;
     int split = 1;

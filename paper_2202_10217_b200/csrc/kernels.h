@@ -37,9 +37,10 @@ int f64_stages();
 // map over C for the asynchronous store path (32 x 32 FP32 boxes, 128-byte swizzle), or null
 // when C does not meet the TMA alignment rules.  With split_k == 1 and `d_cta_begin` given, block b
 // runs items [d_cta_begin[b], d_cta_begin[b+1]) of the list (n_ctas blocks).  `a_is_m_by_n`: A is
-// stored M x N row-major and `tmA` has boxes of 64 rows x 64 columns over that array.  `a_kind`:
-// 0 bfloat16; 1 binary32 read as TF32 (boxes of 128 rows x 32 columns); 2 FP8 E4M3 bytes (boxes of
-// 128 rows x 128 columns); 3 IEEE binary16 (boxes as for bfloat16); kinds 1 and 2 in the N x M order only.
+// stored M x N row-major and `tmA` has square boxes of one stage's k-rows x 128 bytes of columns
+// over that array (64 x 64 for the 16-bit kinds, 32 x 32 for TF32, 128 x 128 for FP8).  `a_kind`:
+// 0 bfloat16; 1 binary32 read as TF32 (N x M order: boxes of 128 rows x 32 columns); 2 FP8 E4M3 bytes
+// (boxes of 128 rows x 128 columns); 3 IEEE binary16 (boxes as for bfloat16).
 // `batch` > 0: strided batch (3-D maps as for the FP64 kernel); the units are then (matrix, item)
 // pairs dealt round-robin, split_k must be 1.
 cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,

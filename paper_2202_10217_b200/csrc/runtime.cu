@@ -201,7 +201,7 @@ EncodeTiledFn encode_fn() {
 }  // namespace
 
 int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, int64_t M,
-                         int64_t lda, int box_rows, int box_cols) {
+                         int64_t lda, int box_rows, int box_cols, int swizzle_atom_32b) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return SYRK_ERR_CUDA;
     const size_t es = a_elem_size(dtype);
@@ -216,7 +216,8 @@ int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, i
         : (dtype == SYRK_DTYPE_E4M3_F32) ? CU_TENSOR_MAP_DATA_TYPE_UINT8
         : (dtype == SYRK_DTYPE_F16_F32) ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUresult r = fn(tm, dt, 2, const_cast<void*>(A), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          swizzle_atom_32b ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? SYRK_OK : SYRK_ERR_CUDA;
 }

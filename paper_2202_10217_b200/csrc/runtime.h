@@ -97,9 +97,10 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out);
 bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out);
 
 // 2-D row-major tensor map over A (N x M, pitch lda elements) with a box of
-// box_rows x box_cols elements and 128-byte swizzle.
+// box_rows x box_cols elements and 128-byte swizzle (16-byte atoms, or 32-byte atoms with
+// `swizzle_atom_32b`: the form MN-major binary32 operands of the tensor core need).
 int encode_tensor_map_2d(CUtensorMap* tm, int dtype, const void* A, int64_t N, int64_t M,
-                         int64_t lda, int box_rows, int box_cols);
+                         int64_t lda, int box_rows, int box_cols, int swizzle_atom_32b = 0);
 
 // 2-D row-major FP32 tensor map over C (N x N, pitch ldc) with box x box boxes, 128-byte swizzle.
 int encode_tensor_map_batched(CUtensorMap* tm, int dtype, const void* A, int64_t N, int64_t M, int64_t lda,

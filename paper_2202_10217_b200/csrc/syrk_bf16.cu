@@ -27,8 +27,9 @@
 //
 // Both MMA operands come from the same row-major A (K contiguous): segment x is the
 // M-operand, segment y (or the adjacent pair y, y+1) the N-operand, both K-major.  When A is
-// stored M x N (the Gram form) the stages hold 64 k-rows of 64 columns per box and both
-// operands are MN-major; everything after the MMA is the same.
+// stored M x N (the Gram form) the stages hold boxes of k-rows by columns and both
+// operands are MN-major (for every input kind; the boxes are then one stage's k-rows by 128 bytes
+// of columns); everything after the MMA is the same.
 #include "device_utils.cuh"
 #include "kernels.h"
 #include "tbs_plan.h"
@@ -123,16 +124,21 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return d;
 }
 // The same for an MN-major operand (A stored M x N: a segment's 128 columns are contiguous in
-// memory, one 128-byte row of 64 columns per k).  A segment slot holds two groups of 64 columns,
-// 8192 bytes apart (leading byte offset); within a group, 8-row k groups are 1024 bytes apart
-// (stride byte offset); `addr` advances by 2048 bytes per K = 16 step.
-__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
+// memory, one 128-byte row per k).  A 128-byte row holds 64 two-byte, 32 binary32 or 128 FP8
+// columns, so a segment slot holds 2, 4 or 1 column groups, each a box of one stage's k-rows,
+// `group_bytes` apart (leading byte offset; the N = 256 operand runs on into the next slot with
+// the same stride); within a group, 8-row k groups are 1024 bytes apart (stride byte offset);
+// `addr` advances by (k-rows per MMA) * 128 bytes per instruction.
+// binary32 (TF32) operands in this order use the 128-byte swizzle with 32-byte atoms instead (layout
+// code 1; the tensor map over A is encoded with the matching TMA mode): its pattern repeats every 4
+// k-rows, so the k groups are 512 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t group_bytes, bool atom32) {
     uint64_t d = 0;
     d |= uint64_t((addr & 0x3FFFF) >> 4);
-    d |= uint64_t(8192 >> 4) << 16;                // leading byte offset (between 64-column groups)
-    d |= uint64_t(1024 >> 4) << 32;                // stride byte offset (between 8-row k groups)
+    d |= uint64_t(group_bytes >> 4) << 16;         // leading byte offset (between column groups)
+    d |= uint64_t((atom32 ? 512 : 1024) >> 4) << 32;   // stride byte offset (between k groups of 4 or 8 rows)
     d |= uint64_t(1) << 46;
-    d |= uint64_t(2) << 61;
+    d |= uint64_t(atom32 ? 1 : 2) << 61;
     return d;
 }
 // Instruction descriptor, kind::f16: D = FP32, A = B = BF16, M = 128; both operands K-major, or
@@ -268,11 +274,13 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     }
                     mbar_arrive_expect_tx(&full_bar[st], uint32_t(n_seg) * kSegBytes);
                     uint8_t* dst = smem + st * kStageBytes;
-                    if (kTN) {   // A stored M x N: two boxes of 64 k-rows x 64 columns per segment
+                    if (kTN) {   // A stored M x N: per segment, boxes of one stage's k-rows x 128 bytes of columns
+                        constexpr int kGroupCols = kCols;                 // columns in a 128-byte row: 64, 32 or 128
+                        constexpr int kGroups = kTile / kGroupCols;
                         for (int s = 0; s < n_seg; ++s)
-                            for (int h = 0; h < 2; ++h)
-                                tma_load_box(dst + s * kSegBytes + h * (kSegBytes / 2), &tmA, rows[s] + h * 64, ks * kCols,
-                                             u.batch, &full_bar[st]);
+                            for (int h = 0; h < kGroups; ++h)
+                                tma_load_box(dst + s * kSegBytes + h * (kSegBytes / kGroups), &tmA, rows[s] + h * kGroupCols,
+                                             ks * kCols, u.batch, &full_bar[st]);
                     } else {
                         for (int s = 0; s < n_seg; ++s)
                             tma_load_box(dst + s * kSegBytes, &tmA, ks * kCols, rows[s], u.batch, &full_bar[st]);
@@ -291,8 +299,9 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if (lane == 0) {
             uint32_t g = 0, n_done = 0;
             const uint32_t smem_base = smem_u32(smem);
-            const uint64_t desc_hi = kTN ? smem_desc_mn_sw128(0) : smem_desc_sw128(0);
-            constexpr uint32_t kk_step = kTN ? (2048u >> 4) : (32u >> 4);   // descriptor advance per K = 16
+            // MN-major: a column group is one stage's k-rows (kCols) of 128 bytes; an MMA takes a quarter of them
+            const uint64_t desc_hi = kTN ? smem_desc_mn_sw128(0, uint32_t(kCols) * 128u, kKind == kKindTF32) : smem_desc_sw128(0);
+            constexpr uint32_t kk_step = kTN ? ((uint32_t(kCols) * 32u) >> 4) : (32u >> 4);   // descriptor advance per MMA
             for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride, ++n_done) {
                 const Unit u = unit_of(w, n_items, n_ksteps, split, n_batch);
                 const WorkItem* it = &items[u.item];
@@ -495,7 +504,9 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[6] = {reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>),
+        const void* kernels[8] = {reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>),
+                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindTF32>),
+                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindE4M3>),
                                   reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindBF16>),
                                   reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindF16>),
                                   reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindF16>),
@@ -509,7 +520,7 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     }
     if (n_items == 0) return cudaSuccess;
     const bool two_byte = a_kind == bf16::kKindBF16 || a_kind == bf16::kKindF16;
-    if (a_kind < 0 || a_kind > 3 || (!two_byte && a_is_m_by_n)) return cudaErrorInvalidValue;   // no such kernel
+    if (a_kind < 0 || a_kind > 3) return cudaErrorInvalidValue;   // no such kernel
     const int bk = two_byte ? 64 : (a_kind == bf16::kKindTF32 ? 32 : 128);
     const int32_t n_ksteps = int32_t((M + bk - 1) / bk);
     const int split = split_k < 1 ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
@@ -520,8 +531,10 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                         (batch <= 0 || (c_batch_stride & 3) == 0)) ? 1 : 0;
     CUtensorMap none{};
-    auto kernel = a_kind == bf16::kKindTF32 ? bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>
-                  : a_kind == bf16::kKindE4M3 ? bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>
+    auto kernel = a_kind == bf16::kKindTF32 ? (a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindTF32>
+                                                           : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>)
+                  : a_kind == bf16::kKindE4M3 ? (a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindE4M3>
+                                                             : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>)
                   : a_kind == bf16::kKindF16 ? (a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindF16>
                                                             : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindF16>)
                   : a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindBF16>

@@ -14,8 +14,8 @@ from gpu_util import assert_within_tolerance, run_case
 from test_gpu_syrk import make_A
 
 pytestmark = pytest.mark.gpu
-BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_F16_F32]     # the types with a tensor-core path in this order
-DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "f16"])
+BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_F16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32]
+DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "f16", "tf32", "e4m3"])
 
 # N even keeps the pitch of the M x N array a multiple of 16 bytes (tensor-core path in FP64);
 # odd N takes the plain-load kernel.  Ragged tiles in N (not a multiple of 32) and ragged
@@ -25,6 +25,10 @@ SIZES = {B.DTYPE_F64: [(2, 1), (6, 3), (30, 17), (32, 16), (34, 50), (100, 64), 
          B.DTYPE_BF16_F32: [(8, 8), (40, 24), (128, 64), (136, 72), (304, 200), (777, 136), (512, 256),
                             (1104, 320), (2056, 72), (1304, 1000)]}
 SIZES[B.DTYPE_F16_F32] = SIZES[B.DTYPE_BF16_F32]
+SIZES[B.DTYPE_TF32_F32] = [(4, 4), (40, 12), (128, 32), (132, 36), (304, 100), (777, 68), (512, 256), (1100, 160),
+                           (2052, 44), (1304, 500)]
+SIZES[B.DTYPE_E4M3_F32] = [(16, 16), (48, 48), (128, 128), (144, 272), (304, 400), (777, 144), (512, 512),
+                           (1104, 640), (2064, 144), (1312, 1008)]
 
 
 @DT
@@ -95,7 +99,8 @@ def test_leading_dimension_smaller_than_N_is_refused():
         B.syrk_lower_tn(64, 16, 8, 32, 8, 64, 1.0, 0.0, B.DTYPE_F64, stream=0)
 
 
-@pytest.mark.parametrize("dtype", [B.DTYPE_BF16_F32, B.DTYPE_F16_F32], ids=["bf16", "f16"])
+@pytest.mark.parametrize("dtype", [B.DTYPE_BF16_F32, B.DTYPE_F16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32],
+                         ids=["bf16", "f16", "tf32", "e4m3"])
 @pytest.mark.parametrize("split", [0, 2, 5])
 def test_bf16_k_split_in_this_storage_order(split, dtype):
     N, M = 704, 1280
@@ -109,10 +114,13 @@ def test_bf16_k_split_in_this_storage_order(split, dtype):
     assert_within_tolerance(got, ref, bound, M, 2.0, -1.0, Cin, dtype)
 
 
-@pytest.mark.parametrize("dtype", [B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32], ids=["tf32", "e4m3"])
-def test_tf32_and_fp8_inputs_in_this_storage_order_take_the_plain_kernel(dtype):
-    N, M = 272, 52
-    A = make_A(N, M, dtype, seed=61)
-    Cin = I.random_c(N, 62, dtype)
-    got, ref, bound = run_case(A, dtype, -1.0, 1.0, Cin, tn=True)
-    assert_within_tolerance(got, ref, bound, M, -1.0, 1.0, Cin, dtype)
+def test_tf32_low_order_bits_are_ignored_in_this_storage_order():
+    """The MN-major TF32 path reads the same 19 high-order bits as the N x M path."""
+    N, M = 264, 96
+    base = I.small_int_f32(N, M, seed=63, lo=-3, hi=3)
+    noise = np.random.default_rng(64).integers(0, 1 << 13, size=base.shape, dtype=np.uint32)
+    dirty = (base.view(np.uint32) | np.where(base != 0, noise, 0).astype(np.uint32)).view(np.float32)
+    got_dirty, ref, bound = run_case(dirty, B.DTYPE_TF32_F32, 1.0, 0.0, tn=True)
+    got_clean, _, _ = run_case(base, B.DTYPE_TF32_F32, 1.0, 0.0, tn=True)
+    il = np.tril_indices(N)
+    assert np.array_equal(got_dirty[il], got_clean[il]) and np.array_equal(got_dirty[il], ref[il])
