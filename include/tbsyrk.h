@@ -87,7 +87,12 @@ extern "C" {
  * K-split path, a device workspace; both are created on first use (that first
  * call allocates device memory) and released by syrk_shutdown().  Calls are
  * stream-ordered; concurrent calls on different streams that need the K-split
- * workspace are serialised by the caller.
+ * workspace are serialised by the caller.  The K-split path is taken when the
+ * work list is too short to fill the GPU and the inner dimension is long (FP64:
+ * fewer items than SMs and M >= 1024; the other types: a cost
+ * model over the work list, slices of at least 8 K-steps): the inner dimension is cut
+ * into slices, the slices' partial results go to the workspace and are summed in
+ * slice order (deterministic) before alpha and beta are applied.
  */
 int syrk_lower(int64_t N, int64_t M,
                const void* A, int64_t lda,
@@ -246,7 +251,7 @@ int syrk_set_schedule(int schedule);
  */
 int syrk_probe_f64_mma_peak(int iters, double* tflops);
 
-/* Force the number of K-slices (0 = automatic) used by later bf16 calls. */
+/* Force the number of K-slices (0 = automatic) used by later calls of every dtype. */
 int syrk_set_split_k(int slices);
 
 /*

@@ -62,6 +62,27 @@ int auto_split_k(const std::vector<WorkItem>& items, int64_t M, int bk, int sm_c
     return best;
 }
 
+// K-slices for an FP64 call (one block per item).  With fewer items than SMs the inner
+// dimension is cut so that more blocks run at once; the slices' partial matrices are
+// summed by a second kernel.  Model, in microseconds: a K-step of an item takes about 2, an item's
+// start-up and write-out about 6, the reduction streams slices * N^2 / 2 doubles at about 5 TB/s
+// after a launch gap of about 4.  A slice keeps at least 32 K-steps.
+int auto_split_k_f64(int64_t n_items, int64_t N, int64_t M, int bk, int sm_count, int forced) {
+    const int64_t ksteps = (M + bk - 1) / bk;
+    if (forced > 0) return int(std::max<int64_t>(1, std::min<int64_t>(forced, ksteps)));
+    if (n_items == 0 || n_items >= int64_t(sm_count) || ksteps < 64) return 1;
+    int best = 1;
+    double best_cost = 0.0;
+    for (int s = 1; s <= 16 && s <= ksteps / 32; ++s) {
+        if (s > 1 && double(s) * double(N) * double(N) * 8.0 > 512e6) break;        // workspace cap
+        const int64_t waves = (n_items * s + sm_count - 1) / sm_count;
+        double cost = double(waves) * (2.0 * double((ksteps + s - 1) / s) + 6.0);
+        if (s > 1) cost += 4.0 + double(s) * double(N) * double(N) * 4.0 / 5e6;
+        if (s == 1 || cost < best_cost) { best = s; best_cost = cost; }
+    }
+    return best;
+}
+
 int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk) {
     return auto_split_k(dp->plan.items, M, bk, ds->sm_count, runtime().split_k);
 }
@@ -82,9 +103,10 @@ int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkIt
         const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
         const bool persistent = mode == SYRK_F64_LAUNCH_PERSISTENT ||
                                 (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count));
-        int* tickets = persistent ? tickets_for_stream(ds, stream) : nullptr;
+        int* tickets = (persistent && split <= 1) ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<double*>(C), ldc,
-                            alpha, beta, a_is_m_by_n, tickets, ds->sm_count, ds->d_status, stream);
+                            alpha, beta, a_is_m_by_n, tickets, ds->sm_count, ds->d_status, stream, 0, 0, split,
+                            reinterpret_cast<double*>(ds->d_partial));
     } else {
         CUtensorMap tmc;
         const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
@@ -171,6 +193,16 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
             const size_t want = size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float);
             void* p = ds->d_partial;
             rc = ensure_device_bytes(&p, &ds->partial_bytes, want);
+            ds->d_partial = static_cast<float*>(p);
+            if (rc != SYRK_OK) return rc;
+        }
+    } else if (f64_launch < 0) {
+        // FP64 K-split (not for callers that fix the launch form: the Cholesky driver runs updates on
+        // two streams at once, and the workspace is one per device)
+        split = auto_split_k_f64(int64_t(dp->plan.items.size()), N, M, ks.bk, ds->sm_count, runtime().split_k);
+        if (split > 1) {
+            void* p = ds->d_partial;
+            rc = ensure_device_bytes(&p, &ds->partial_bytes, size_t(split) * size_t(N) * size_t(N) * sizeof(double));
             ds->d_partial = static_cast<float*>(p);
             if (rc != SYRK_OK) return rc;
         }

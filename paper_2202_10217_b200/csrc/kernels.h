@@ -16,11 +16,14 @@ namespace tbsyrk {
 // Gram form C = A^T A); `tmA` then has boxes of 16 rows x 16 columns over that array.
 // `batch` > 0: strided batch of `batch` problems; `tmA` and `tmC` are then 3-D maps whose last
 // coordinate is the matrix number, matrix b of C starts at C + b * c_batch_stride, and the launch
-// has one block per (matrix, item).
+// has one block per (matrix, item).  `split_k` > 1 with `d_partial` (split_k x N x N doubles): the
+// inner dimension is cut into that many slices, one block per (slice, item) writes partial
+// matrices and a second kernel sums them in slice order and applies alpha and beta.
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
-                            cudaStream_t stream, int64_t batch = 0, int64_t c_batch_stride = 0);
+                            cudaStream_t stream, int64_t batch = 0, int64_t c_batch_stride = 0, int split_k = 1,
+                            double* d_partial = nullptr);
 // The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
 // P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
 // columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.

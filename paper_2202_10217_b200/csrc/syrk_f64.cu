@@ -74,6 +74,7 @@ struct Call {
     double alpha, beta;
     int vec_ok, c_tma;
     int32_t batch;                 // matrix of a strided batch the block works on (tensor maps are 3-D), or -1
+    int32_t k0;                    // first K-step of the block's slice of the inner dimension (K-split calls)
     bool gemm;
 };
 
@@ -98,12 +99,12 @@ __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, 
             // (128-byte rows of 16 columns, one row per k), 2 KB each.
             for (int s = 0; s < n_seg; ++s)
                 for (int h = 0; h < 2; ++h)
-                    tma_load_box(dst + s * kSegBytes + h * (kSegBytes / 2), k.tmA, it.seg[s] * kTile + h * 16, ks * kBK,
-                                 k.batch, &k.full_bar[st]);
+                    tma_load_box(dst + s * kSegBytes + h * (kSegBytes / 2), k.tmA, it.seg[s] * kTile + h * 16,
+                                 (k.k0 + ks) * kBK, k.batch, &k.full_bar[st]);
         } else {
             for (int s = 0; s < n_seg; ++s)
-                tma_load_box(dst + s * kSegBytes, (k.gemm && s < it.pad) ? k.tmB : k.tmA, ks * kBK, it.seg[s] * kTile,
-                             k.batch, &k.full_bar[st]);
+                tma_load_box(dst + s * kSegBytes, (k.gemm && s < it.pad) ? k.tmB : k.tmA, (k.k0 + ks) * kBK,
+                             it.seg[s] * kTile, k.batch, &k.full_bar[st]);
         }
     }
     // Old C: ring step j carries tiles 4j .. 4j+3 (8 KB each, row pitch 256 B), those below the diagonal.
@@ -408,7 +409,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
                     int64_t ncols, int32_t gemm_col_tiles, int32_t n_ksteps, double* __restrict__ C,
                     int64_t ldc, double alpha, double beta, int vec_ok, int c_tma, int* __restrict__ status,
-                    int64_t items_per_batch, int64_t c_batch_stride) {
+                    int64_t items_per_batch, int64_t c_batch_stride, int32_t slice_ksteps) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ WorkItem s_item;
@@ -425,12 +426,20 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     k.N = N; k.ncols = ncols; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
     k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = gemm_col_tiles > 0;
     // Strided batch: the grid holds the work list once per matrix; the tensor maps are 3-D.
-    k.batch = -1;
+    // K-split (slice_ksteps > 0): the grid holds the list once per slice of the inner dimension;
+    // slice s takes K-steps [s * slice_ksteps, ...) of the 2-D maps and writes partial matrix s.
+    k.batch = -1; k.k0 = 0;
     int64_t item_index = blockIdx.x;
     if (items_per_batch > 0) {
-        k.batch = int32_t(int64_t(blockIdx.x) / items_per_batch);
+        const int32_t group = int32_t(int64_t(blockIdx.x) / items_per_batch);
         item_index = int64_t(blockIdx.x) % items_per_batch;
-        k.C = C + int64_t(k.batch) * c_batch_stride;
+        k.C = C + int64_t(group) * c_batch_stride;
+        if (slice_ksteps > 0) {
+            k.k0 = group * slice_ksteps;
+            k.n_ksteps = min(slice_ksteps, n_ksteps - k.k0);
+        } else {
+            k.batch = group;
+        }
     }
 
     if (k.gemm) {
@@ -503,7 +512,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
     k.abort_flag = &s_abort; k.status = status;
     k.tmA = &tmA; k.tmB = &tmA; k.tmC = &tmC;
     k.N = N; k.ncols = N; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
-    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false; k.batch = -1;
+    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false; k.batch = -1; k.k0 = 0;
 
     if (tid == 0) {
         s_abort = 0;
@@ -554,6 +563,20 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
     }
 }
 
+// K-split calls: lower triangle of C <- alpha * (sum of the slices' partial matrices, in slice
+// order) + beta * C.  Partial matrix s is N x N with row pitch N at partial + s * N * N.
+__global__ void __launch_bounds__(256)
+splitk_reduce_f64_kernel(int64_t N, int32_t slices, const double* __restrict__ partial, double* __restrict__ C,
+                         int64_t ldc, double alpha, double beta) {
+    const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
+    if (i >= N || j > i) return;
+    double s = 0.0;
+    for (int32_t sl = 0; sl < slices; ++sl) s += partial[(int64_t(sl) * N + i) * N + j];
+    double* c = C + i * ldc + j;
+    *c = (beta == 0.0) ? alpha * s : alpha * s + beta * *c;
+}
+
 }  // namespace f64
 
 namespace {
@@ -581,7 +604,8 @@ cudaError_t configure_f64_kernels() {
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
-                            cudaStream_t stream, int64_t batch, int64_t c_batch_stride) {
+                            cudaStream_t stream, int64_t batch, int64_t c_batch_stride, int split_k,
+                            double* d_partial) {
     cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
@@ -591,13 +615,30 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
     const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
     CUtensorMap none{};
     const dim3 threads(f64::kThreads);
+    if (split_k > 1 && batch <= 0 && d_partial != nullptr) {
+        // K-split: one block per (slice, item); slices write partial matrices (alpha = 1, beta = 0,
+        // old C not read), summed afterwards in slice order.
+        const int32_t slice_ksteps = (n_ksteps + split_k - 1) / split_k;
+        const int32_t slices = (n_ksteps + slice_ksteps - 1) / slice_ksteps;       // none of them empty
+        if (n_items * slices >= (int64_t(1) << 31)) return cudaErrorInvalidValue;
+        auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
+        kernel<<<dim3(unsigned(n_items * slices)), threads, f64::kSmemBytes, stream>>>(
+            tmA, tmA, none, d_items, N, N, 0, n_ksteps, d_partial, N, 1.0, 0.0, (N & 1) == 0 ? 1 : 0, 0, d_status,
+            n_items, N * N, slice_ksteps);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        const dim3 rb(32, 8);
+        f64::splitk_reduce_f64_kernel<<<dim3(unsigned((N + 31) / 32), unsigned((N + 7) / 8)), rb, 0, stream>>>(
+            N, slices, d_partial, C, ldc, alpha, beta);
+        return cudaGetLastError();
+    }
     if (batch > 0) {
         // Strided batch (3-D tensor maps): one block per (matrix, item), matrix-major.
         if (n_items * batch >= (int64_t(1) << 31)) return cudaErrorInvalidValue;
         auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
         kernel<<<dim3(unsigned(n_items * batch)), threads, f64::kSmemBytes, stream>>>(
             tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
-            n_items, c_batch_stride);
+            n_items, c_batch_stride, 0);
         return cudaGetLastError();
     }
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
@@ -610,7 +651,7 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
     auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
     kernel<<<dim3(unsigned(n_items)), threads, f64::kSmemBytes, stream>>>(
         tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
-        int64_t(0), int64_t(0));
+        int64_t(0), int64_t(0), 0);
     return cudaGetLastError();
 }
 
@@ -628,7 +669,7 @@ cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, c
     CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<false><<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmP, tmQ, c_tma ? *tmD : none, nullptr, nrows, ncols, int32_t(col_tiles), n_ksteps, D, ldd, alpha, beta,
-        vec_ok, c_tma, d_status, int64_t(0), int64_t(0));
+        vec_ok, c_tma, d_status, int64_t(0), int64_t(0), 0);
     return cudaGetLastError();
 }
 

@@ -39,7 +39,7 @@ def test_random_cases(chunk):
         Cin = I.random_c(N, int(rng.integers(0, 1 << 30)), dtype) if beta != 0.0 else None
         if Cin is not None and kind == "int":
             Cin = np.round(Cin * 4).astype(Cin.dtype)           # keeps every partial result exact
-        split = int(rng.choice([0, 0, 2, 3])) if dtype != B.DTYPE_F64 else 0
+        split = int(rng.choice([0, 0, 2, 3]))
         mode = int(rng.integers(0, 3)) if dtype == B.DTYPE_F64 else 0
         try:
             B.syrk_set_split_k(split)

@@ -281,6 +281,35 @@ def test_f64_call_inside_stream_capture_replays_correctly():
     assert np.array_equal(dC.cpu().numpy()[il], ref[il])
 
 
+@pytest.mark.parametrize("tn", [False, True], ids=["nxm", "mxn"])
+@pytest.mark.parametrize("split", [2, 3, 7])
+def test_f64_k_split_forced(split, tn):
+    """FP64 K-split: slices of the inner dimension into partial matrices, summed in slice order.
+    Ragged last slice and last K-step, ragged N, general alpha / beta, both storage orders; integer
+    inputs must still match bit for bit."""
+    for n, (N, M) in enumerate([(258, 1030), (1056, 2048), (64, 4099 if not tn else 4100), (700, 528)]):
+        A = make_A(N, M, B.DTYPE_F64, seed=900 + n)
+        Ai = make_A(N, M, B.DTYPE_F64, seed=950 + n, kind="int")
+        Cin = I.random_c(N, 960 + n, B.DTYPE_F64)
+        try:
+            B.syrk_set_split_k(split)
+            got, ref, bound = run_case(A, B.DTYPE_F64, -1.5, 0.5, Cin, tn=tn)
+            goti, refi, boundi = run_case(Ai, B.DTYPE_F64, 1.0, 0.0, poison=True, tn=tn)
+        finally:
+            B.syrk_set_split_k(0)
+        assert_within_tolerance(got, ref, bound, M, -1.5, 0.5, Cin, B.DTYPE_F64)
+        assert_within_tolerance(goti, refi, boundi, M, 1.0, 0.0, None, B.DTYPE_F64, exact=True)
+
+
+def test_f64_k_split_automatic_for_short_work_lists():
+    """N = 1024 has about 60 work items: with M = 8192 the library cuts the inner dimension by itself."""
+    N, M = 1024, 8192
+    A = make_A(N, M, B.DTYPE_F64, seed=980)
+    Cin = I.random_c(N, 981, B.DTYPE_F64)
+    got, ref, bound = run_case(A, B.DTYPE_F64, 1.0, -1.0, Cin, ldc=N + 3)
+    assert_within_tolerance(got, ref, bound, M, 1.0, -1.0, Cin, B.DTYPE_F64)
+
+
 def test_tf32_low_order_bits_of_the_inputs_are_ignored():
     """The tensor core reads the 19 high-order bits of every binary32 input.  With values whose
     low 13 bits are set the result must equal, bit for bit, the result for the same values with
