@@ -121,6 +121,38 @@ int syrk_lower_tn(int64_t N, int64_t M,
                   int dtype, void* stream);
 
 /*
+ * The general form: which triangle of C is stored and how the operand is stored.
+ *
+ *     uplo = SYRK_UPLO_LOWER: the entries C[i][j] with j <= i are updated (as syrk_lower);
+ *     uplo = SYRK_UPLO_UPPER: the entries C[i][j] with j >= i are updated, the strict lower
+ *                             triangle is never read or written;
+ *     trans = SYRK_OP_N: A is N x M row-major, C <- alpha * A A^T + beta * C  (as syrk_lower);
+ *     trans = SYRK_OP_T: A is M x N row-major, C <- alpha * A^T A + beta * C  (as syrk_lower_tn).
+ *
+ * The result is that of Algorithm 1 of the paper: C is symmetric, so the upper form holds the
+ * same numbers mirrored.  The paper works on the lower triangle only; the upper form runs the
+ * mirror image of the same work list (every tile (x, y) of Algorithm 4 / Section 5.1.4 becomes
+ * the tile (y, x), i.e. the roles of the two MMA operands are exchanged and the triangle mask
+ * is flipped), so the I/O count is unchanged.
+ * For callers holding COLUMN-major data (BLAS convention): a column-major N x K matrix with
+ * leading dimension lda is a row-major K x N array with pitch lda, and a column-major triangle
+ * 'L' is the row-major upper triangle.  Hence  xSYRK('L', 'N', n, k, alpha, A, lda, beta, C, ldc)
+ * == syrk_ex(SYRK_UPLO_UPPER, SYRK_OP_T, n, k, A, lda, C, ldc, alpha, beta, ...), 'U' maps to
+ * SYRK_UPLO_LOWER, and trans 'T' to SYRK_OP_N.
+ * Everything else (alignment rule and plain-load fallback, K-split, ownership, stream semantics,
+ * quick returns, error codes) is as for syrk_lower; an unknown uplo or trans gives SYRK_ERR_SIZE.
+ */
+#define SYRK_UPLO_LOWER 0
+#define SYRK_UPLO_UPPER 1
+#define SYRK_OP_N 0
+#define SYRK_OP_T 1
+int syrk_ex(int uplo, int trans, int64_t N, int64_t M,
+            const void* A, int64_t lda,
+            void* C, int64_t ldc,
+            double alpha, double beta,
+            int dtype, void* stream);
+
+/*
  * A strided batch of independent updates of the same shape:
  *
  *     C_b[i][j] = alpha * sum_k A_b[i][k] * A_b[j][k] + beta * C_b[i][j]    0 <= j <= i < N, 0 <= b < batch,

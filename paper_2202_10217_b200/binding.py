@@ -17,13 +17,15 @@ DTYPE_BF16_F32 = 1
 DTYPE_TF32_F32 = 2
 DTYPE_E4M3_F32 = 3
 DTYPE_F16_F32 = 4
+UPLO_LOWER, UPLO_UPPER = 0, 1
+OP_N, OP_T = 0, 1
 SCHEDULE_TBS = 0
 SCHEDULE_SQUARE = 1
 ITEM_TRI, ITEM_RECT, ITEM_DIAG = 0, 1, 2
 MAX_SEG, MAX_TILE = 8, 16
 
 EXPORTS = [
-    "syrk_lower", "syrk_lower_tn", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
+    "syrk_lower", "syrk_lower_tn", "syrk_ex", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_set_f64_launch", "syrk_get_schedule_stats",
     "syrk_probe_f64_mma_peak", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
     "tbs_plan_build", "tbs_plan_balance", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
@@ -64,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.syrk_lower.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
         L.syrk_lower_tn.restype = ci
         L.syrk_lower_tn.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
+        L.syrk_ex.restype = ci
+        L.syrk_ex.argtypes = [ci, ci, i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
         L.syrk_lower_batched.restype = ci
         L.syrk_lower_batched.argtypes = [i64, i64, i64, vp, i64, i64, vp, i64, i64, dbl, dbl, ci, vp]
         L.syrk_lower_host.restype = ci
@@ -153,6 +157,15 @@ def syrk_lower_tn(N: int, M: int, A, lda: int, C, ldc: int, alpha: float, beta: 
         import torch
         stream = torch.cuda.current_stream().cuda_stream
     _check(lib().syrk_lower_tn(N, M, _ptr(A), lda, _ptr(C), ldc, float(alpha), float(beta), dtype, stream))
+
+
+def syrk_ex(uplo: int, trans: int, N: int, M: int, A, lda: int, C, ldc: int, alpha: float, beta: float,
+            dtype: int, stream: Optional[int] = None) -> None:
+    """General form: stored triangle `uplo` of C <- alpha * op(A) op(A)^T + beta * C (device pointers)."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().syrk_ex(uplo, trans, N, M, _ptr(A), lda, _ptr(C), ldc, float(alpha), float(beta), dtype, stream))
 
 
 def syrk_lower_batched(batch: int, N: int, M: int, A, lda: int, stride_a: int, C, ldc: int, stride_c: int,

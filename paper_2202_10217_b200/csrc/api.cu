@@ -91,7 +91,7 @@ int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk)
 int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkItem* d_items, int64_t n_items,
                  int64_t N, int64_t M, void* C, int64_t ldc, double alpha, double beta, int split,
                  const int64_t* d_tile_base, int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas,
-                 int f64_launch, int a_is_m_by_n, cudaStream_t stream) {
+                 int f64_launch, int a_is_m_by_n, cudaStream_t stream, int upper = 0) {
     cudaError_t e;
     if (dtype == SYRK_DTYPE_F64) {
         CUtensorMap tmc;
@@ -101,19 +101,19 @@ int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkIt
         // That pays when items are short (M <= 1024: at most 64 stages each) and the list fills the
         // device several times over; for long items one block per item is the faster form.
         const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
-        const bool persistent = mode == SYRK_F64_LAUNCH_PERSISTENT ||
-                                (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count));
+        const bool persistent = !upper && (mode == SYRK_F64_LAUNCH_PERSISTENT ||
+                                (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count)));
         int* tickets = (persistent && split <= 1) ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<double*>(C), ldc,
                             alpha, beta, a_is_m_by_n, tickets, ds->sm_count, ds->d_status, stream, 0, 0, split,
-                            reinterpret_cast<double*>(ds->d_partial));
+                            reinterpret_cast<double*>(ds->d_partial), upper);
     } else {
         CUtensorMap tmc;
         const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                            encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
         e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
                              float(beta), split, ds->d_partial, d_tile_base, total_tiles, d_cta_begin, n_ctas, a_is_m_by_n,
-                             dtype - SYRK_DTYPE_BF16_F32, ds->d_status, ds->sm_count, stream);
+                             dtype - SYRK_DTYPE_BF16_F32, ds->d_status, ds->sm_count, stream, 0, 0, upper);
     }
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
@@ -165,19 +165,19 @@ int get_banded_plan(DeviceState* ds, int64_t N, int dtype, int max_bands, Banded
 }  // namespace
 
 int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
-                            double beta, int dtype, cudaStream_t stream, int f64_launch, int a_is_m_by_n) {
+                            double beta, int dtype, cudaStream_t stream, int f64_launch, int a_is_m_by_n, int upper) {
     DeviceState* ds = nullptr;
     int rc = get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
     if (alpha == 0.0 || M == 0) {
         if (beta == 1.0) return SYRK_OK;
-        return launch_scale_lower(dtype, N, C, ldc, beta, stream) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+        return launch_scale_lower(dtype, N, C, ldc, beta, stream, upper) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
     }
     if (!tma_ok(A, lda, dtype))
-        return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream) == cudaSuccess
+        return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream, upper) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
     DevicePlan* dp = nullptr;
-    rc = get_device_plan(ds, N, dtype, &dp);
+    rc = get_device_plan(ds, N, dtype, &dp, upper);
     if (rc != SYRK_OK) return rc;
     const KernelShape ks = kernel_shape(dtype);
     CUtensorMap tm;
@@ -208,7 +208,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         }
     }
     return launch_items(ds, dtype, tm, dp->d_items, int64_t(dp->plan.items.size()), N, M, C, ldc, alpha, beta, split,
-                        dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, f64_launch, a_is_m_by_n, stream);
+                        dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, f64_launch, a_is_m_by_n, stream, upper);
 }
 
 namespace {
@@ -248,6 +248,17 @@ int syrk_lower_tn(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int
     if (rc != SYRK_OK || N == 0) return rc;
     std::lock_guard<std::mutex> lock(runtime().mu);
     return syrk_run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream), -1, 1);
+}
+
+int syrk_ex(int uplo, int trans, int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc,
+            double alpha, double beta, int dtype, void* stream) {
+    if ((uplo != SYRK_UPLO_LOWER && uplo != SYRK_UPLO_UPPER) || (trans != SYRK_OP_N && trans != SYRK_OP_T))
+        return SYRK_ERR_SIZE;
+    int rc = validate(N, M, A, lda, C, ldc, dtype, trans == SYRK_OP_T);
+    if (rc != SYRK_OK || N == 0) return rc;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    return syrk_run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream), -1,
+                           trans == SYRK_OP_T ? 1 : 0, uplo == SYRK_UPLO_UPPER ? 1 : 0);
 }
 
 int syrk_lower_batched(int64_t batch, int64_t N, int64_t M, const void* A, int64_t lda, int64_t stride_a,

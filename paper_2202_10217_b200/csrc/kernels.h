@@ -18,12 +18,14 @@ namespace tbsyrk {
 // coordinate is the matrix number, matrix b of C starts at C + b * c_batch_stride, and the launch
 // has one block per (matrix, item).  `split_k` > 1 with `d_partial` (split_k x N x N doubles): the
 // inner dimension is cut into that many slices, one block per (slice, item) writes partial
-// matrices and a second kernel sums them in slice order and applies alpha and beta.
+// matrices and a second kernel sums them in slice order and applies alpha and beta.  `upper`: the
+// work list holds the tiles on and above the diagonal and entries with col >= row are written (one
+// block per item; not with `batch`).
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
                             cudaStream_t stream, int64_t batch = 0, int64_t c_batch_stride = 0, int split_k = 1,
-                            double* d_partial = nullptr);
+                            double* d_partial = nullptr, int upper = 0);
 // The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
 // P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
 // columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.
@@ -45,13 +47,14 @@ int f64_stages();
 // 0 bfloat16; 1 binary32 read as TF32 (N x M order: boxes of 128 rows x 32 columns); 2 FP8 E4M3 bytes
 // (boxes of 128 rows x 128 columns); 3 IEEE binary16 (boxes as for bfloat16).
 // `batch` > 0: strided batch (3-D maps as for the FP64 kernel); the units are then (matrix, item)
-// pairs dealt round-robin, split_k must be 1.
+// pairs dealt round-robin, split_k must be 1.  `upper`: the work list holds the tiles on and above
+// the diagonal and the entries with col >= row are written (not with `batch`).
 cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                              int64_t n_items, int64_t N, int64_t M, float* C, int64_t ldc, float alpha,
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
                              int a_kind, int* d_status, int sm_count, cudaStream_t stream,
-                             int64_t batch = 0, int64_t c_batch_stride = 0);
+                             int64_t batch = 0, int64_t c_batch_stride = 0, int upper = 0);
 int bf16_tile();
 int bf16_bk();
 int bf16_stages();
@@ -61,10 +64,11 @@ int bf16_store_box();
 // Plain-load kernels: one thread per lower-triangle entry.  Used when A does not meet
 // the TMA alignment rules; same result, much slower.
 cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, void* C,
-                              int64_t ldc, double alpha, double beta, int a_is_m_by_n, cudaStream_t stream);
+                              int64_t ldc, double alpha, double beta, int a_is_m_by_n, cudaStream_t stream,
+                              int upper = 0);
 
 // Lower triangle <- beta * lower triangle (zero when beta == 0, without reading C).
 cudaError_t launch_scale_lower(int dtype, int64_t N, void* C, int64_t ldc, double beta,
-                               cudaStream_t stream);
+                               cudaStream_t stream, int upper = 0);
 
 }  // namespace tbsyrk

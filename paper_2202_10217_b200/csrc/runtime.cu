@@ -34,13 +34,17 @@ KernelShape kernel_shape(int dtype) {
     return s;
 }
 
-bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out) {
+bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out, int upper) {
     const KernelShape ks = kernel_shape(dtype);
     PlanParams p;
     p.n_tiles = (N + ks.tile - 1) / ks.tile;
     p.k = ks.k;
-    p.rect_rows = ks.rect_rows;
-    p.rect_cols = ks.rect_cols;
+    // The upper-triangle form runs the mirror image of a lower-triangle list: a rectangle of r x c
+    // tiles below the diagonal becomes one of c x r above it, so the list is built with the
+    // rectangle's sides exchanged (the tcgen05 kernel wants one M-operand and two adjacent N-operands).
+    p.rect_rows = upper ? ks.rect_cols : ks.rect_rows;
+    p.rect_cols = upper ? ks.rect_rows : ks.rect_cols;
+    if (upper && ks.diag_side < p.rect_rows) return false;
     p.diag_side = ks.diag_side;
     p.schedule = schedule;
     if (!build_plan(p, out)) return false;
@@ -49,6 +53,20 @@ bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out) {
     if (dtype == SYRK_DTYPE_F64) balance_for_slots(out, 148);
     else std::stable_sort(out->items.begin(), out->items.end(),
                           [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
+    if (upper) {
+        for (WorkItem& it : out->items) {
+            for (int t = 0; t < it.n_tile; ++t) std::swap(it.tile_x[t], it.tile_y[t]);     // tile (x, y) -> (y, x)
+            if (dtype != SYRK_DTYPE_F64) {
+                // tcgen05 layout: tiles with the same M-operand and adjacent N-operands must follow each other
+                for (int a = 1; a < it.n_tile; ++a)
+                    for (int b = a; b > 0 && (it.tile_x[b] < it.tile_x[b - 1] ||
+                                              (it.tile_x[b] == it.tile_x[b - 1] && it.tile_y[b] < it.tile_y[b - 1])); --b) {
+                        std::swap(it.tile_x[b], it.tile_x[b - 1]);
+                        std::swap(it.tile_y[b], it.tile_y[b - 1]);
+                    }
+            }
+        }
+    }
     return true;
 }
 
@@ -87,14 +105,14 @@ int* tickets_for_stream(DeviceState* ds, cudaStream_t stream) {
     return ds->d_tickets + 2 * it->second;
 }
 
-int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out) {
+int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out, int upper) {
     const KernelShape ks = kernel_shape(dtype);
     const int64_t n_tiles = (N + ks.tile - 1) / ks.tile;
-    const auto key = std::make_tuple(n_tiles, dtype, runtime().schedule);
+    const auto key = std::make_tuple(n_tiles, dtype, runtime().schedule + (upper ? 16 : 0));
     auto it = ds->plans.find(key);
     if (it == ds->plans.end()) {
         DevicePlan dp;
-        if (!build_host_plan(N, dtype, runtime().schedule, &dp.plan)) return SYRK_ERR_PLAN;
+        if (!build_host_plan(N, dtype, runtime().schedule, &dp.plan, upper)) return SYRK_ERR_PLAN;
         const int max_seg = (dtype == SYRK_DTYPE_F64) ? kMaxSeg : bf16_seg_slots();
         const int max_tile = (dtype == SYRK_DTYPE_F64) ? kMaxTile : 3;
         for (const WorkItem& it : dp.plan.items) {

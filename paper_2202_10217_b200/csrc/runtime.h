@@ -91,10 +91,10 @@ Runtime& runtime();
 int get_device_state(DeviceState** out);
 
 // Plan for (N, dtype) under the current schedule, built and uploaded on first use.
-int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out);
+int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out, int upper = 0);
 
 // Host-only plan (no device).
-bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out);
+bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out, int upper = 0);
 
 // 2-D row-major tensor map over A (N x M, pitch lda elements) with a box of
 // box_rows x box_cols elements and 128-byte swizzle (16-byte atoms, or 32-byte atoms with
@@ -118,8 +118,10 @@ int encode_tensor_map_f64_plain(CUtensorMap* tm, const void* p, int64_t rows, in
 // The device path of syrk_lower (arguments already validated; the caller holds the runtime lock).
 // `f64_launch` >= 0 overrides the process-wide FP64 launch form for this call.  `a_is_m_by_n`: A is
 // stored M x N row-major (pitch lda >= N) and the call computes alpha * A^T A + beta * C.
+// `upper`: the entries with col >= row are updated instead of those with col <= row.
 int syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
-                    double beta, int dtype, cudaStream_t stream, int f64_launch = -1, int a_is_m_by_n = 0);
+                    double beta, int dtype, cudaStream_t stream, int f64_launch = -1, int a_is_m_by_n = 0,
+                    int upper = 0);
 
 void release_cholesky_workspaces();
 

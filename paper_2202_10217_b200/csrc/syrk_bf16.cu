@@ -211,7 +211,7 @@ __device__ __forceinline__ void layout_of(const WorkItem* it, int n_tile, uint32
     }
 }
 
-template <bool kTN, int kKind>
+template <bool kTN, int kKind, bool kUpper>
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
                      const WorkItem* __restrict__ items, int64_t n_items, int64_t N, int32_t n_ksteps,
@@ -416,7 +416,9 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         }
                         if (r >= N) continue;
                         float* crow = Cb + r * ldc + c0;
-                        if (c0 + 31 <= r && vec_ok) {
+                        // entries this row keeps: columns <= r (lower form) or r .. N-1 (upper form)
+                        const bool whole = kUpper ? (c0 >= r && c0 + 31 < N) : (c0 + 31 <= r);
+                        if (whole && vec_ok) {
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 float4 o = make_float4(alpha * __uint_as_float(v[4 * j]), alpha * __uint_as_float(v[4 * j + 1]),
@@ -431,7 +433,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                if (c0 + j <= r) {
+                                if (kUpper ? (c0 + j >= r && c0 + j < N) : (c0 + j <= r)) {
                                     float o = alpha * __uint_as_float(v[j]);
                                     if (beta != 0.f) o += beta * crow[j];
                                     crow[j] = o;
@@ -457,11 +459,12 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
 }
 
-// Sum of the K-slices' partial tiles in slice order, then alpha/beta and the triangle mask.
+// Sum of the K-slices' partial tiles in slice order, then alpha/beta and the triangle mask
+// (col <= row, or col >= row for the upper form).
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const WorkItem* __restrict__ items, const int64_t* __restrict__ tile_base,
                      int64_t total_tiles, int32_t split, const float* __restrict__ partial, int64_t N,
-                     float* __restrict__ C, int64_t ldc, float alpha, float beta) {
+                     float* __restrict__ C, int64_t ldc, float alpha, float beta, int upper) {
     const WorkItem* it = &items[blockIdx.x];
     const int t = blockIdx.y;
     if (t >= it->n_tile) return;
@@ -481,12 +484,31 @@ splitk_reduce_kernel(const WorkItem* __restrict__ items, const int64_t* __restri
         float* crow = C + r * ldc + col0 + cc;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (col0 + cc + j <= r) {
+            const int64_t c = col0 + cc + j;
+            if (upper ? (c >= r && c < N) : (c <= r)) {
                 float o = alpha * vals[j];
                 if (beta != 0.f) o += beta * crow[j];
                 crow[j] = o;
             }
         }
+    }
+}
+
+// The instantiation for an input kind, a storage order of A and a stored triangle of C.
+using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const WorkItem*, int64_t, int64_t, int32_t, float*, int64_t,
+                          float, float, int, int, int32_t, float*, const int64_t*, int64_t, const int64_t*, int*, int32_t,
+                          int64_t);
+template <int kKind>
+KernelFn kernel_of_kind(int tn, int upper) {
+    return tn ? (upper ? syrk_bf16_tbs_kernel<true, kKind, true> : syrk_bf16_tbs_kernel<true, kKind, false>)
+              : (upper ? syrk_bf16_tbs_kernel<false, kKind, true> : syrk_bf16_tbs_kernel<false, kKind, false>);
+}
+KernelFn kernel_for(int kind, int tn, int upper) {
+    switch (kind) {
+        case kKindTF32: return kernel_of_kind<kKindTF32>(tn, upper);
+        case kKindE4M3: return kernel_of_kind<kKindE4M3>(tn, upper);
+        case kKindF16: return kernel_of_kind<kKindF16>(tn, upper);
+        default: return kernel_of_kind<kKindBF16>(tn, upper);
     }
 }
 
@@ -497,21 +519,15 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
                              int a_kind, int* d_status, int sm_count, cudaStream_t stream, int64_t batch,
-                             int64_t c_batch_stride) {
+                             int64_t c_batch_stride, int upper) {
     // The shared-memory attribute belongs to a device's context: set it once per device.
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[8] = {reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindTF32>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindE4M3>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindBF16>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindF16>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<true, bf16::kKindF16>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>),
-                                  reinterpret_cast<const void*>(&bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>)};
+        const void* kernels[16];
+        for (int i = 0; i < 16; ++i) kernels[i] = reinterpret_cast<const void*>(bf16::kernel_for(i >> 2, (i >> 1) & 1, i & 1));
         for (const void* fn : kernels) {
             cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bf16::kSmemBytes);
             if (e != cudaSuccess) return e;
@@ -524,21 +540,14 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     const int bk = two_byte ? 64 : (a_kind == bf16::kKindTF32 ? 32 : 128);
     const int32_t n_ksteps = int32_t((M + bk - 1) / bk);
     const int split = split_k < 1 ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
-    if (batch > 0 && (split != 1 || batch >= (int64_t(1) << 31))) return cudaErrorInvalidValue;
+    if (batch > 0 && (split != 1 || upper || batch >= (int64_t(1) << 31))) return cudaErrorInvalidValue;
     const int64_t n_units = n_items * split * (batch > 0 ? batch : 1);
     const bool ranges = (d_cta_begin != nullptr && split == 1 && n_ctas > 0 && batch <= 0);
     const unsigned grid = ranges ? unsigned(n_ctas) : unsigned(n_units < sm_count ? n_units : sm_count);
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                         (batch <= 0 || (c_batch_stride & 3) == 0)) ? 1 : 0;
     CUtensorMap none{};
-    auto kernel = a_kind == bf16::kKindTF32 ? (a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindTF32>
-                                                           : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindTF32>)
-                  : a_kind == bf16::kKindE4M3 ? (a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindE4M3>
-                                                             : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindE4M3>)
-                  : a_kind == bf16::kKindF16 ? (a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindF16>
-                                                            : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindF16>)
-                  : a_is_m_by_n ? bf16::syrk_bf16_tbs_kernel<true, bf16::kKindBF16>
-                                : bf16::syrk_bf16_tbs_kernel<false, bf16::kKindBF16>;
+    auto kernel = bf16::kernel_for(a_kind, a_is_m_by_n, upper);
     kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
         tmA, tmC ? *tmC : none, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, split,
         d_partial, d_tile_base, total_tiles, ranges ? d_cta_begin : nullptr, d_status, int32_t(batch > 0 ? batch : 0),
@@ -546,7 +555,7 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || split == 1) return e;
     bf16::splitk_reduce_kernel<<<dim3(unsigned(n_items), bf16::kMaxTiles), 256, 0, stream>>>(
-        d_items, d_tile_base, total_tiles, split, d_partial, N, C, ldc, alpha, beta);
+        d_items, d_tile_base, total_tiles, split, d_partial, N, C, ldc, alpha, beta, upper);
     return cudaGetLastError();
 }
 

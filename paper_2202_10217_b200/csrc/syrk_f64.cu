@@ -141,7 +141,7 @@ __device__ void drain_producer(const Call& k, uint32_t g) {
 // whether it is a triangle block in the generator's tile order (x = 1..5, y < x): for those
 // the 16th MMA warp takes the last 8 x 8 block of every tile.  (One thread decides this once per
 // item; the MMA warps only read the flag.)
-__device__ bool prepare_item(const Call& k, WorkItem& it) {
+__device__ bool prepare_item(const Call& k, WorkItem& it, bool upper = false) {
     bool ok = it.n_seg >= 1 && it.n_seg <= kMaxSeg && it.n_tile >= 1 && it.n_tile <= kMmaWarps;
     for (int s = 0; ok && s < it.n_seg; ++s)
         ok = it.seg[s] >= 0 && int64_t(it.seg[s]) * kTile < ((k.gemm && s < it.pad) ? k.ncols : k.N);
@@ -149,7 +149,8 @@ __device__ bool prepare_item(const Call& k, WorkItem& it) {
     if (ok && !k.gemm) {
         bool tri = it.kind == kTri && it.n_seg == 6 && it.n_tile == 15;
         for (int x = 1, q = 0; tri && x < 6; ++x)
-            for (int y = 0; y < x; ++y, ++q) tri = tri && it.tile_x[q] == x && it.tile_y[q] == y;
+            for (int y = 0; y < x; ++y, ++q)      // the upper-triangle form holds the same tiles transposed
+                tri = tri && it.tile_x[q] == (upper ? y : x) && it.tile_y[q] == (upper ? x : y);
         it.pad = tri ? 1 : 0;
     }
     return ok;
@@ -265,7 +266,7 @@ __device__ __forceinline__ uint32_t fragment_offset_tn(int lane) {
 
 // 16th warp of a triangle block: the 15 left-out 8 x 8 blocks.  g0 = the item's first ring step,
 // n_c = its old-C steps.
-template <bool kTN>
+template <bool kTN, bool kUpper>
 __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, int lane) {
     const int gq = lane >> 2, t = lane & 3;
     const uint32_t gc = g0 + uint32_t(k.n_ksteps);
@@ -302,6 +303,27 @@ __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it
     for (int x = 1; x < 6; ++x)
 #pragma unroll
         for (int y = 0; y < x; ++y, ++q) {
+            if (kUpper) {
+                // The block belongs to the tile stored above the diagonal: rows of segment y, columns of
+                // segment x, i.e. the accumulator transposed: this lane's two values go to rows 2t, 2t+1,
+                // column gq of the 8 x 8 block.
+                const int64_t c = int64_t(seg[x]) * kTile + 24 + gq;
+                if (c >= k.N) continue;
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int64_t r = int64_t(seg[y]) * kTile + 24 + 2 * t + e;
+                    if (r >= k.N) continue;
+                    double* p = k.C + r * k.ldc + c;
+                    double v = k.alpha * sacc[q][e];
+                    if (n_c > 0)
+                        v += k.beta * *reinterpret_cast<const double*>(
+                                 k.smem + ((gc + (q >> 2)) % kStages) * kStageBytes + (q & 3) * kCTileBytes +
+                                 (24 + 2 * t + e) * (kTile * 8) + (24 + gq) * 8);
+                    else if (use_beta) v += k.beta * *p;
+                    *p = v;
+                }
+                continue;
+            }
             const int64_t r = int64_t(seg[x]) * kTile + 24 + gq;
             const int64_t c = int64_t(seg[y]) * kTile + 24 + 2 * t;
             if (r >= k.N) continue;                                 // tile below the diagonal: c + 1 < r
@@ -321,7 +343,7 @@ __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it
 }
 
 // A warp with a tile (tile number `warp` of the item).  `scavenge`: block (3, 3) is left to the 16th warp.
-template <bool kTN>
+template <bool kTN, bool kUpper>
 __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, bool scavenge,
                                           int warp, int lane) {
     const int gq = lane >> 2, t = lane & 3;
@@ -347,6 +369,33 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
     const uint8_t* old_tile = nullptr;                  // this warp's old C tile in shared memory
     if (n_c > 0 && (k.gemm || row0 != col0))
         old_tile = k.smem + ((gc + (warp >> 2)) % kStages) * kStageBytes + (warp & 3) * kCTileBytes;
+    if (kUpper) {
+        // Upper-triangle form: row r keeps columns r .. N-1; either value of a pair may be the one kept.
+#pragma unroll
+        for (int mi = 0; mi < 4; ++mi) {
+            const int64_t r = row0 + mi * 8 + gq;
+            if (r >= k.N) continue;
+            double* crow = k.C + r * k.ldc;
+#pragma unroll
+            for (int ni = 0; ni < 4; ++ni) {
+                if (scavenge && mi == 3 && ni == 3) continue;             // written by the 16th warp
+                const int64_t c = col0 + ni * 8 + 2 * t;
+                const bool ok0 = c >= r && c < k.N, ok1 = c + 1 >= r && c + 1 < k.N;
+                if (!ok0 && !ok1) continue;
+                double v0 = k.alpha * acc[mi][ni][0], v1 = k.alpha * acc[mi][ni][1];
+                if (use_beta) {
+                    double2 o = make_double2(0.0, 0.0);
+                    if (old_tile) o = *reinterpret_cast<const double2*>(old_tile + (mi * 8 + gq) * (kTile * 8) + (ni * 8 + 2 * t) * 8);
+                    else { if (ok0) o.x = crow[c]; if (ok1) o.y = crow[c + 1]; }
+                    v0 += k.beta * o.x; v1 += k.beta * o.y;
+                }
+                if (ok0 && ok1 && k.vec_ok) *reinterpret_cast<double2*>(crow + c) = make_double2(v0, v1);
+                else { if (ok0) crow[c] = v0; if (ok1) crow[c + 1] = v1; }
+            }
+        }
+        for (int j = 0; j < n_c; ++j) release(k, gc + j, lane);
+        return true;
+    }
 #pragma unroll
     for (int mi = 0; mi < 4; ++mi) {
         const int64_t r = row0 + mi * 8 + gq;
@@ -381,15 +430,15 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
 
 // One MMA warp's share of one item: its ring steps from global step g on, then its write-out.
 // Every warp waits for and releases every ring step of the item, with or without work in it.
-template <bool kTN>
+template <bool kTN, bool kUpper>
 __device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it, uint32_t& g, int warp, int lane) {
     const int n_tile = it.n_tile;
     const int n_c = c_steps_of(k, n_tile);
     const uint32_t g0 = g;
     g += uint32_t(k.n_ksteps + n_c);
     const bool scavenge = !k.gemm && it.pad != 0;      // set by prepare_item
-    if (scavenge && warp == kMmaWarps - 1) return scavenger_role<kTN>(k, it, g0, n_c, lane);
-    if (warp < n_tile) return tile_role<kTN>(k, it, g0, n_c, scavenge, warp, lane);
+    if (scavenge && warp == kMmaWarps - 1) return scavenger_role<kTN, kUpper>(k, it, g0, n_c, lane);
+    if (warp < n_tile) return tile_role<kTN, kUpper>(k, it, g0, n_c, scavenge, warp, lane);
     for (uint32_t s = g0; s < g; ++s) {                 // no tile in this item: keep the ring moving
         if (!wait_full(k, s, lane)) return false;
         release(k, s, lane);
@@ -403,7 +452,7 @@ __device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it,
 // groups), its column segments come from Q (tmB, the first `pad` segments), its row segments
 // from P (tmA).
 // ---------------------------------------------------------------------------------------------
-template <bool kTN>
+template <bool kTN, bool kUpper>
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
@@ -462,7 +511,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (tid == 0) s_abort = 0;
     __syncthreads();
     if (tid == 0) {
-        if (!prepare_item(k, s_item)) { s_abort = 1; atomicOr(status, kStatusBadItem); }
+        if (!prepare_item(k, s_item, kUpper)) { s_abort = 1; atomicOr(status, kStatusBadItem); }
         else {
             for (int s = 0; s < kStages; ++s) { mbar_init(&k.full_bar[s], 1); mbar_init(&k.empty_bar[s], kMmaWarps); }
             mbar_fence_init();
@@ -481,7 +530,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         return;
     }
-    mma_warp_item<kTN>(k, s_item, g, warp, lane);
+    mma_warp_item<kTN, kUpper>(k, s_item, g, warp, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -559,18 +608,18 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
         }
         const WorkItem& it = s_ring[slot % kItemRing];
         if (it.n_tile < 0) return;
-        if (!mma_warp_item<kTN>(k, it, g, warp, lane)) return;
+        if (!mma_warp_item<kTN, false>(k, it, g, warp, lane)) return;
     }
 }
 
-// K-split calls: lower triangle of C <- alpha * (sum of the slices' partial matrices, in slice
+// K-split calls: stored triangle of C <- alpha * (sum of the slices' partial matrices, in slice
 // order) + beta * C.  Partial matrix s is N x N with row pitch N at partial + s * N * N.
 __global__ void __launch_bounds__(256)
 splitk_reduce_f64_kernel(int64_t N, int32_t slices, const double* __restrict__ partial, double* __restrict__ C,
-                         int64_t ldc, double alpha, double beta) {
+                         int64_t ldc, double alpha, double beta, int upper) {
     const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
-    if (i >= N || j > i) return;
+    if (i >= N || j >= N || (upper ? j < i : j > i)) return;
     double s = 0.0;
     for (int32_t sl = 0; sl < slices; ++sl) s += partial[(int64_t(sl) * N + i) * N + j];
     double* c = C + i * ldc + j;
@@ -587,8 +636,10 @@ cudaError_t configure_f64_kernels() {
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[4] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false>),
-                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true>),
+        const void* kernels[6] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, false>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true>)};
         for (const void* fn : kernels) {
@@ -605,7 +656,7 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
                             cudaStream_t stream, int64_t batch, int64_t c_batch_stride, int split_k,
-                            double* d_partial) {
+                            double* d_partial, int upper) {
     cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
@@ -621,7 +672,8 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
         const int32_t slice_ksteps = (n_ksteps + split_k - 1) / split_k;
         const int32_t slices = (n_ksteps + slice_ksteps - 1) / slice_ksteps;       // none of them empty
         if (n_items * slices >= (int64_t(1) << 31)) return cudaErrorInvalidValue;
-        auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
+        auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, true> : f64::syrk_f64_tbs_kernel<false, true>)
+                            : (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, false> : f64::syrk_f64_tbs_kernel<false, false>);
         kernel<<<dim3(unsigned(n_items * slices)), threads, f64::kSmemBytes, stream>>>(
             tmA, tmA, none, d_items, N, N, 0, n_ksteps, d_partial, N, 1.0, 0.0, (N & 1) == 0 ? 1 : 0, 0, d_status,
             n_items, N * N, slice_ksteps);
@@ -629,26 +681,28 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
         if (e != cudaSuccess) return e;
         const dim3 rb(32, 8);
         f64::splitk_reduce_f64_kernel<<<dim3(unsigned((N + 31) / 32), unsigned((N + 7) / 8)), rb, 0, stream>>>(
-            N, slices, d_partial, C, ldc, alpha, beta);
+            N, slices, d_partial, C, ldc, alpha, beta, upper);
         return cudaGetLastError();
     }
     if (batch > 0) {
+        if (upper) return cudaErrorInvalidValue;
         // Strided batch (3-D tensor maps): one block per (matrix, item), matrix-major.
         if (n_items * batch >= (int64_t(1) << 31)) return cudaErrorInvalidValue;
-        auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
+        auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, false> : f64::syrk_f64_tbs_kernel<false, false>;
         kernel<<<dim3(unsigned(n_items * batch)), threads, f64::kSmemBytes, stream>>>(
             tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
             n_items, c_batch_stride, 0);
         return cudaGetLastError();
     }
-    if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
+    if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30) && !upper) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true> : f64::syrk_f64_tbs_persistent_kernel<false>;
         kernel<<<grid, threads, f64::kSmemBytes, stream>>>(tmA, c_tma ? *tmC : none, d_items, n_items, d_tickets, N,
                                                            n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
         return cudaGetLastError();
     }
-    auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true> : f64::syrk_f64_tbs_kernel<false>;
+    auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, true> : f64::syrk_f64_tbs_kernel<false, true>)
+                        : (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, false> : f64::syrk_f64_tbs_kernel<false, false>);
     kernel<<<dim3(unsigned(n_items)), threads, f64::kSmemBytes, stream>>>(
         tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
         int64_t(0), int64_t(0), 0);
@@ -667,7 +721,7 @@ cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, c
     const int64_t row_tiles = (nrows + f64::kTile - 1) / f64::kTile, col_tiles = (ncols + f64::kTile - 1) / f64::kTile;
     const int64_t blocks = ((row_tiles + 3) / 4) * ((col_tiles + 3) / 4);
     CUtensorMap none{};
-    f64::syrk_f64_tbs_kernel<false><<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
+    f64::syrk_f64_tbs_kernel<false, false><<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmP, tmQ, c_tma ? *tmD : none, nullptr, nrows, ncols, int32_t(col_tiles), n_ksteps, D, ldd, alpha, beta,
         vec_ok, c_tma, d_status, int64_t(0), int64_t(0), 0);
     return cudaGetLastError();

@@ -39,10 +39,10 @@ template <> struct Widen<uint8_t, float> {
 
 template <typename TA, typename TC>
 __global__ void syrk_plain_kernel(int64_t N, int64_t M, const TA* __restrict__ A, int64_t row_stride,
-                                  int64_t col_stride, TC* __restrict__ C, int64_t ldc, TC alpha, TC beta) {
+                                  int64_t col_stride, TC* __restrict__ C, int64_t ldc, TC alpha, TC beta, int upper) {
     const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
-    if (i >= N || j > i) return;
+    if (i >= N || j >= N || (upper ? j < i : j > i)) return;
     const TA* ai = A + i * row_stride;       // row i of the N x M operand, whichever way it is stored
     const TA* aj = A + j * row_stride;
     TC s = TC(0);
@@ -53,10 +53,10 @@ __global__ void syrk_plain_kernel(int64_t N, int64_t M, const TA* __restrict__ A
 }
 
 template <typename TC>
-__global__ void scale_lower_kernel(int64_t N, TC* __restrict__ C, int64_t ldc, TC beta) {
+__global__ void scale_lower_kernel(int64_t N, TC* __restrict__ C, int64_t ldc, TC beta, int upper) {
     const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
-    if (i >= N || j > i) return;
+    if (i >= N || j >= N || (upper ? j < i : j > i)) return;
     TC* c = C + i * ldc + j;
     *c = (beta == TC(0)) ? TC(0) : beta * *c;
 }
@@ -68,37 +68,37 @@ inline dim3 grid2d(int64_t N, dim3 block) {
 }  // namespace
 
 cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, void* C,
-                              int64_t ldc, double alpha, double beta, int a_is_m_by_n, cudaStream_t stream) {
+                              int64_t ldc, double alpha, double beta, int a_is_m_by_n, cudaStream_t stream, int upper) {
     if (N == 0) return cudaSuccess;
     const dim3 block(32, 8);
     const int64_t rs = a_is_m_by_n ? 1 : lda, cs = a_is_m_by_n ? lda : 1;
     if (dtype == 0)
         syrk_plain_kernel<double, double><<<grid2d(N, block), block, 0, stream>>>(
-            N, M, static_cast<const double*>(A), rs, cs, static_cast<double*>(C), ldc, alpha, beta);
+            N, M, static_cast<const double*>(A), rs, cs, static_cast<double*>(C), ldc, alpha, beta, upper);
     else if (dtype == 3)
         syrk_plain_kernel<uint8_t, float><<<grid2d(N, block), block, 0, stream>>>(
-            N, M, static_cast<const uint8_t*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));
+            N, M, static_cast<const uint8_t*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta), upper);
     else if (dtype == 4)
         syrk_plain_kernel<__half, float><<<grid2d(N, block), block, 0, stream>>>(
-            N, M, static_cast<const __half*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));
+            N, M, static_cast<const __half*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta), upper);
     else if (dtype == 2)
         syrk_plain_kernel<float, float><<<grid2d(N, block), block, 0, stream>>>(
-            N, M, static_cast<const float*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta));
+            N, M, static_cast<const float*>(A), rs, cs, static_cast<float*>(C), ldc, float(alpha), float(beta), upper);
     else
         syrk_plain_kernel<__nv_bfloat16, float><<<grid2d(N, block), block, 0, stream>>>(
             N, M, static_cast<const __nv_bfloat16*>(A), rs, cs, static_cast<float*>(C), ldc,
-            float(alpha), float(beta));
+            float(alpha), float(beta), upper);
     return cudaGetLastError();
 }
 
 cudaError_t launch_scale_lower(int dtype, int64_t N, void* C, int64_t ldc, double beta,
-                               cudaStream_t stream) {
+                               cudaStream_t stream, int upper) {
     if (N == 0) return cudaSuccess;
     const dim3 block(32, 8);
     if (dtype == 0)
-        scale_lower_kernel<double><<<grid2d(N, block), block, 0, stream>>>(N, static_cast<double*>(C), ldc, beta);
+        scale_lower_kernel<double><<<grid2d(N, block), block, 0, stream>>>(N, static_cast<double*>(C), ldc, beta, upper);
     else
-        scale_lower_kernel<float><<<grid2d(N, block), block, 0, stream>>>(N, static_cast<float*>(C), ldc, float(beta));
+        scale_lower_kernel<float><<<grid2d(N, block), block, 0, stream>>>(N, static_cast<float*>(C), ldc, float(beta), upper);
     return cudaGetLastError();
 }
 

@@ -39,31 +39,42 @@ def sentinel_array(shape, np_dtype):
 
 def run_case(A: np.ndarray, dtype: int, alpha: float, beta: float, Cin: np.ndarray | None = None,
              lda: int | None = None, ldc: int | None = None, a_offset: int = 0, c_offset: int = 0,
-             poison: bool = False, tn: bool = False):
+             poison: bool = False, tn: bool = False, upper: bool = False):
     """One call; returns (got, ref, bound).  Checks canaries and status itself.
 
     `A` is always the N x M operand of the reference.  With `tn` it is handed to the library
-    transposed (an M x N row-major array, pitch lda >= N) through syrk_lower_tn."""
+    transposed (an M x N row-major array, pitch lda >= N) through syrk_lower_tn.  With `upper`
+    the call goes through syrk_ex with the upper triangle stored: the prior values and the result
+    live at the mirrored positions (j, i), and `got` is returned transposed so that its lower
+    triangle compares with the reference as usual."""
     N, M = A.shape
     cdt = I.c_storage_dtype(dtype)
     ldc = max(N, 1) if ldc is None else ldc
     rows = N + 2 * GUARD
     host_c = sentinel_array((rows, ldc + c_offset), cdt)
     body = host_c[GUARD:GUARD + N, c_offset:c_offset + N] if N else host_c[0:0, 0:0]
+    stored = np.tril_indices(N)
+    if upper:
+        stored = (stored[1], stored[0])                      # entry (i, j), j <= i, lives at (j, i)
     if Cin is not None:
-        il = np.tril_indices(N)
-        body[il] = Cin[il]
+        body[stored] = Cin[np.tril_indices(N)]
     elif poison:
-        body[np.tril_indices(N)] = np.nan
+        body[stored] = np.nan
     before = host_c.copy()
     dev_c = torch.from_numpy(host_c).cuda()
     c_ptr = dev_c.data_ptr() + (GUARD * (ldc + c_offset) + c_offset) * dev_c.element_size()
     if tn:
         keep, a_ptr = a_to_device(np.ascontiguousarray(A.T), dtype, lda, a_offset)
-        B.syrk_lower_tn(N, M, a_ptr, max(N, 1) if lda is None else lda, c_ptr, ldc + c_offset, alpha, beta, dtype)
+        lda_eff = max(N, 1) if lda is None else lda
     else:
         keep, a_ptr = a_to_device(A, dtype, lda, a_offset)
-        B.syrk_lower(N, M, a_ptr, max(M, 1) if lda is None else lda, c_ptr, ldc + c_offset, alpha, beta, dtype)
+        lda_eff = max(M, 1) if lda is None else lda
+    if upper:
+        B.syrk_ex(B.UPLO_UPPER, B.OP_T if tn else B.OP_N, N, M, a_ptr, lda_eff, c_ptr, ldc + c_offset, alpha, beta, dtype)
+    elif tn:
+        B.syrk_lower_tn(N, M, a_ptr, lda_eff, c_ptr, ldc + c_offset, alpha, beta, dtype)
+    else:
+        B.syrk_lower(N, M, a_ptr, lda_eff, c_ptr, ldc + c_offset, alpha, beta, dtype)
     torch.cuda.synchronize()
     assert B.syrk_last_status() == 0
     after = dev_c.cpu().numpy()
@@ -72,9 +83,11 @@ def run_case(A: np.ndarray, dtype: int, alpha: float, beta: float, Cin: np.ndarr
     mask = np.ones(after.shape, dtype=bool)
     if N:
         m = mask[GUARD:GUARD + N, c_offset:c_offset + N]
-        m[np.tril_indices(N)] = False
-    assert np.array_equal(after.view(u)[mask], before.view(u)[mask]), "wrote outside the lower triangle"
+        m[stored] = False
+    assert np.array_equal(after.view(u)[mask], before.view(u)[mask]), "wrote outside the stored triangle"
     got = after[GUARD:GUARD + N, c_offset:c_offset + N].astype(np.float64)
+    if upper:
+        got = np.ascontiguousarray(got.T)
     ref, bound = O.syrk_lower(np.ascontiguousarray(A), None if Cin is None else np.ascontiguousarray(Cin),
                               alpha, beta if Cin is not None else 0.0, dtype)
     return got, ref, bound
