@@ -146,9 +146,9 @@ def run_reference(args, wl: I.Workload, rank: int):
 # captures summarised under profiles/.  Valid only for the kernel source it was taken on.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, sha256 of the kernel source at capture time)
-    "c2_f64_4096x4096": (777_209_088, "de13754c66e41a84278a15bcafeb6e1758756338eb3106d2a42b6f422c6761c4"),
-    "c3_bf16_16384x4096": (1_923_674_112, "e7088eee8b3a4de2d4426963ceffe7d3d18aac3a023a141dff24a45c2e2d4309"),
-    "c4_bf16_2048x262144": (2_854_155_264, "e7088eee8b3a4de2d4426963ceffe7d3d18aac3a023a141dff24a45c2e2d4309"),
+    "c2_f64_4096x4096": (779_726_336, "d1df95dc3b79669ebb072c7afbcfebc01663be171998e16610030920976908f8"),
+    "c3_bf16_16384x4096": (1_938_945_792, "4821ed7dd649bee40152f9f9c7cae9ba3a0f61e5860377e22447fa74776ae46e"),
+    "c4_bf16_2048x262144": (2_929_146_880, "4821ed7dd649bee40152f9f9c7cae9ba3a0f61e5860377e22447fa74776ae46e"),
 }
 
 
