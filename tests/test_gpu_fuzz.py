@@ -1,5 +1,5 @@
 """Seeded random sweep of the C-ABI surface on the GPU: every input type, both storage orders
-of the operand, aligned and unaligned bases and pitches, general alpha / beta, forced K-splits and
+of the operand, both stored triangles, aligned and unaligned bases and pitches, general alpha / beta, forced K-splits and
 both FP64 launch forms - each case compared entry by entry with the CPU reference under the
 tolerance of test_gpu_syrk.py (and bit for bit when the inputs are small integers)."""
 import numpy as np
@@ -17,12 +17,13 @@ DTYPES = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32, B.D
 SCALARS = [(1.0, 0.0), (-1.0, 1.0), (0.5, -2.0), (2.0, 0.0), (1.0, 1.0), (0.0, 0.5)]
 
 
-@pytest.mark.parametrize("chunk", range(6))
+@pytest.mark.parametrize("chunk", range(8))
 def test_random_cases(chunk):
     rng = np.random.default_rng(9000 + chunk)
     for case in range(12):
         dtype = DTYPES[int(rng.integers(0, len(DTYPES)))]
         tn = bool(rng.integers(0, 2))
+        upper = bool(rng.integers(0, 3) == 0)
         kind = "int" if rng.integers(0, 3) == 0 else "normal"
         N = int(rng.choice([int(rng.integers(1, 130)), int(rng.integers(130, 700)), int(rng.integers(700, 1700))]))
         M = int(rng.choice([int(rng.integers(1, 40)), int(rng.integers(40, 300)), int(rng.integers(300, 900))]))
@@ -45,12 +46,12 @@ def test_random_cases(chunk):
             B.syrk_set_split_k(split)
             B.syrk_set_f64_launch(mode)
             got, ref, bound = run_case(A, dtype, alpha, beta, Cin, lda=lda, ldc=ldc, a_offset=a_offset,
-                                       c_offset=c_offset, tn=tn)
+                                       c_offset=c_offset, tn=tn, upper=upper)
         finally:
             B.syrk_set_split_k(0)
             B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
-        where = "case %d.%d dtype=%d tn=%s N=%d M=%d lda=%d off=%d a=%g b=%g split=%d mode=%d" % (
-            chunk, case, dtype, tn, N, M, lda, a_offset, alpha, beta, split, mode)
+        where = "case %d.%d dtype=%d tn=%s upper=%s N=%d M=%d lda=%d off=%d a=%g b=%g split=%d mode=%d" % (
+            chunk, case, dtype, tn, upper, N, M, lda, a_offset, alpha, beta, split, mode)
         try:
             exact = kind == "int" and float(alpha).is_integer() and float(beta).is_integer()
             assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin, dtype, exact=exact)
