@@ -41,6 +41,15 @@ def test_strerror_and_argument_validation_need_no_device():
     assert L.syrk_lower(4, 4, p, 4, None, 4, 1.0, 0.0, 0, None) == -1        # null C
     assert L.syrk_lower(4, 4, p, 4, p, 4, 1.0, 0.0, 7, None) == -4           # dtype
     assert L.syrk_lower(0, 4, None, 4, None, 1, 1.0, 0.0, 0, None) == 0      # N == 0
+    assert L.syrk_ex(2, 0, 4, 4, p, 4, p, 4, 1.0, 0.0, 0, None) == -2           # unknown uplo
+    assert L.syrk_ex(1, 3, 4, 4, p, 4, p, 4, 1.0, 0.0, 0, None) == -2           # unknown trans
+    assert L.syrk_ex(1, 1, 4, 8, p, 3, p, 4, 1.0, 0.0, 0, None) == -3           # M x N operand: lda < N
+    assert L.syrk_ex(1, 0, 0, 8, None, 8, None, 1, 1.0, 0.0, 0, None) == 0      # N == 0
+    assert L.syrk_lower_batched(-1, 4, 4, p, 4, 16, p, 4, 16, 1.0, 0.0, 0, None) == -2      # negative batch
+    assert L.syrk_lower_batched(3, 4, 4, p, 4, 15, p, 4, 16, 1.0, 0.0, 0, None) == -3       # matrices of A overlap
+    assert L.syrk_lower_batched(3, 4, 4, p, 4, 16, p, 4, 15, 1.0, 0.0, 0, None) == -3       # matrices of C overlap
+    assert L.syrk_lower_batched(0, 4, 4, None, 4, 16, None, 4, 16, 1.0, 0.0, 0, None) == -1  # arguments are still checked
+    assert L.syrk_lower_batched(0, 4, 4, p, 4, 16, p, 4, 16, 1.0, 0.0, 0, None) == 0        # empty batch
     assert L.syrk_set_schedule(5) == -7
     assert B.Plan.__init__ is not None
     with pytest.raises(B.SyrkError):
