@@ -193,6 +193,9 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
     if args.batch > 0:
         run_batched(args, wl)
         return
+    if args.syr2k:
+        run_syr2k(args, wl)
+        return
     A_host = wl.make_A()
     cdt = I.c_storage_dtype(dtype)
     if dtype in (I.DTYPE_F64, I.DTYPE_TF32_F32, I.DTYPE_E4M3_F32):
@@ -451,6 +454,36 @@ def run_batched(args, wl):
                       "config": {"workload": wl.name, "N": N, "M": M, "batch": nb}}))
 
 
+def run_syr2k(args, wl):
+    """--kernel-only --syr2k: the rank-2k update alpha (A B^T + B A^T) + beta C of the workload's shape
+    (binary64; B drawn like A from the next seed); 2 N (N+1) M flops."""
+    import torch
+    from paper_2202_10217_b200 import binding as B
+
+    N, M = wl.N, wl.M
+    dA = torch.from_numpy(wl.make_A()).cuda()
+    dB = torch.from_numpy(I.Workload(wl.name, N, M, wl.dtype, wl.alpha, wl.beta, wl.seed + 1, wl.dist, wl.std).make_A()).cuda()
+    dC = torch.zeros((N, N), dtype=torch.float64, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for _ in range(max(args.warmup, 1)):
+        B.syr2k_lower(N, M, dA, M, dB, M, dC, N, wl.alpha, wl.beta)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(args.steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.syr2k_lower(N, M, dA, M, dB, M, dC, N, wl.alpha, wl.beta)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert B.syrk_last_status() == 0
+    ms = float(np.mean(times))
+    print(json.dumps({"metric": "syr2k_tflops_2N(N+1)M", "value": 2 * wl.flops / (ms * 1e-3) * 1e-12, "unit": UNIT,
+                      "n_gpus": 1, "steps": args.steps, "ms_per_step": ms, "kernel_only": True,
+                      "config": {"workload": wl.name, "N": N, "M": M, "op": "syr2k"}}))
+
+
 def run_cholesky(args, rank: int, world: int, local_rank: int):
     """Large Block Cholesky of a seeded 32768^2 FP64 matrix (n*I + G G^T / 512); a step is one
     factorisation (the matrix is restored from a device copy between steps, outside the timing)."""
@@ -510,8 +543,12 @@ def main():
                     help="with --kernel-only: hand the operand over stored M x N and time syrk_lower_tn (C = A^T A)")
     ap.add_argument("--batch", type=int, default=0,
                     help="with --kernel-only: that many problems of the workload's shape through syrk_lower_batched")
+    ap.add_argument("--syr2k", action="store_true",
+                    help="with --kernel-only and an f64 workload: time syr2k_lower (rank-2k update) instead")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
+    if args.syr2k and not args.kernel_only:
+        ap.error("--syr2k needs --kernel-only")
     if args.batch > 0 and not args.kernel_only:
         ap.error("--batch needs --kernel-only")
     if args.gram and not args.kernel_only:

@@ -153,6 +153,27 @@ int syrk_ex(int uplo, int trans, int64_t N, int64_t M,
             int dtype, void* stream);
 
 /*
+ * Symmetric rank-2k update on the lower triangle, binary64:
+ *
+ *     C[i][j] = alpha * sum_k (A[i][k] * B[j][k] + B[i][k] * A[j][k]) + beta * C[i][j]     0 <= j <= i < N,
+ *
+ * A and B DEVICE pointers to N x M row-major arrays (pitches lda, ldb >= max(1, M)), C as for
+ * syrk_lower.  The paper treats the rank-k update and names, in its conclusion, kernels that use
+ * the same input several times as the place its ideas extend to; this is that extension for the
+ * nearest such kernel.  The schedule is Algorithm 4 / Section 5.1.4 unchanged: a thread block owns
+ * the accumulators of every pair among k = 4 row segments and streams those rows of A and of B
+ * (8 segments per step, where a square block of the same 6 tiles would need more), every tile
+ * receiving both products.  FP64 tensor cores (DMMA); A and B 16-byte aligned with even pitches,
+ * else a plain-load kernel.  Quick returns, ownership, stream semantics and error codes as for
+ * syrk_lower (SYRK_ERR_LD also for ldb < max(1, M), SYRK_ERR_NULL for a null B with M > 0).
+ */
+int syr2k_lower(int64_t N, int64_t M,
+                const void* A, int64_t lda,
+                const void* B, int64_t ldb,
+                void* C, int64_t ldc,
+                double alpha, double beta, void* stream);
+
+/*
  * A strided batch of independent updates of the same shape:
  *
  *     C_b[i][j] = alpha * sum_k A_b[i][k] * A_b[j][k] + beta * C_b[i][j]    0 <= j <= i < N, 0 <= b < batch,

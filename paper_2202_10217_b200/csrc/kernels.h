@@ -26,6 +26,12 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
                             cudaStream_t stream, int64_t batch = 0, int64_t c_batch_stride = 0, int split_k = 1,
                             double* d_partial = nullptr, int upper = 0);
+// Rank-2k update C = alpha (A B^T + B A^T) + beta C on the lower triangle with the same kernel: the work
+// items name at most 4 segments and 8 tiles; every stage holds the segments' rows of A (tmA) and of
+// B (tmB); a tile is shared by two warps (16 rows each) that add both products.  One block per item.
+cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap* tmC,
+                             const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc,
+                             double alpha, double beta, int* d_status, cudaStream_t stream);
 // The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
 // P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
 // columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.
@@ -68,6 +74,10 @@ cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, in
                               int upper = 0);
 
 // Lower triangle <- beta * lower triangle (zero when beta == 0, without reading C).
+// Plain-load rank-2k update (binary64): one thread per lower-triangle entry; for unaligned operands.
+cudaError_t launch_syr2k_plain(int64_t N, int64_t M, const double* A, int64_t lda, const double* B, int64_t ldb,
+                               double* C, int64_t ldc, double alpha, double beta, cudaStream_t stream);
+
 cudaError_t launch_scale_lower(int dtype, int64_t N, void* C, int64_t ldc, double beta,
                                cudaStream_t stream, int upper = 0);
 

@@ -49,6 +49,7 @@ constexpr int kThreads = (kMmaWarps + 1) * 32;  // + producer warp
 constexpr int kCTileBytes = kTile * kTile * 8;  // one old C tile in a ring stage (4 per stage)
 constexpr int kSmemBytes = kStages * kStageBytes + 2 * kStages * 8 + 1024;
 constexpr int kItemRing = 16;                   // published items in flight (persistent form)
+constexpr int kSyr2kSlots = kMaxSeg / 2;        // rank-2k update: segments of A in slots 0..3, of B in slots 4..7
 
 __device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
@@ -75,6 +76,7 @@ struct Call {
     int vec_ok, c_tma;
     int32_t batch;                 // matrix of a strided batch the block works on (tensor maps are 3-D), or -1
     int32_t k0;                    // first K-step of the block's slice of the inner dimension (K-split calls)
+    bool syr2k;                    // rank-2k update: slots 0..3 hold segments of A, slots 4..7 the same rows of B (tmB)
     bool gemm;
 };
 
@@ -92,9 +94,14 @@ __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, 
         if (g >= kStages && !mbar_wait_bounded(&k.empty_bar[st], ((g / kStages) - 1) & 1, k.abort_flag)) {
             *k.abort_flag = 1; atomicOr(k.status, kStatusWaitEmpty); return false;
         }
-        mbar_arrive_expect_tx(&k.full_bar[st], uint32_t(n_seg) * kSegBytes);
+        mbar_arrive_expect_tx(&k.full_bar[st], uint32_t(k.syr2k ? 2 * n_seg : n_seg) * kSegBytes);
         uint8_t* dst = k.smem + st * kStageBytes;
-        if (kTN) {
+        if (k.syr2k) {
+            for (int s = 0; s < n_seg; ++s) {
+                tma_load_2d(dst + s * kSegBytes, k.tmA, (k.k0 + ks) * kBK, it.seg[s] * kTile, &k.full_bar[st]);
+                tma_load_2d(dst + (kSyr2kSlots + s) * kSegBytes, k.tmB, (k.k0 + ks) * kBK, it.seg[s] * kTile, &k.full_bar[st]);
+            }
+        } else if (kTN) {
             // A stored M x N: a segment's 32 columns x 16 rows of A arrive as two boxes of 16 x 16
             // (128-byte rows of 16 columns, one row per k), 2 KB each.
             for (int s = 0; s < n_seg; ++s)
@@ -143,11 +150,12 @@ __device__ void drain_producer(const Call& k, uint32_t g) {
 // item; the MMA warps only read the flag.)
 __device__ bool prepare_item(const Call& k, WorkItem& it, bool upper = false) {
     bool ok = it.n_seg >= 1 && it.n_seg <= kMaxSeg && it.n_tile >= 1 && it.n_tile <= kMmaWarps;
+    if (k.syr2k) ok = ok && it.n_seg <= kSyr2kSlots && it.n_tile <= kMmaWarps / 2;
     for (int s = 0; ok && s < it.n_seg; ++s)
         ok = it.seg[s] >= 0 && int64_t(it.seg[s]) * kTile < ((k.gemm && s < it.pad) ? k.ncols : k.N);
     for (int t = 0; ok && t < it.n_tile; ++t) ok = it.tile_x[t] < it.n_seg && it.tile_y[t] < it.n_seg;
     if (ok && !k.gemm) {
-        bool tri = it.kind == kTri && it.n_seg == 6 && it.n_tile == 15;
+        bool tri = !k.syr2k && it.kind == kTri && it.n_seg == 6 && it.n_tile == 15;
         for (int x = 1, q = 0; tri && x < 6; ++x)
             for (int y = 0; y < x; ++y, ++q)      // the upper-triangle form holds the same tiles transposed
                 tri = tri && it.tile_x[q] == (upper ? y : x) && it.tile_y[q] == (upper ? x : y);
@@ -428,14 +436,104 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
     return true;
 }
 
+// Rank-2k update: warp w owns rows 16 (w & 1) .. + 15 of tile w >> 1 and adds both products,
+// A_x B_y^T and B_x A_y^T, into the same 16 x 32 accumulator (2 x 4 blocks of m8n8k4): 16 DMMAs per
+// k-slice and warp, as for a whole tile of the rank-k update.  N x M operands, lower triangle.
+__device__ __forceinline__ bool syr2k_tile_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, int warp, int lane) {
+    const int gq = lane >> 2, t = lane & 3;
+    const int tile = warp >> 1, half = warp & 1;
+    const uint32_t gc = g0 + uint32_t(k.n_ksteps);
+    const bool use_beta = (k.beta != 0.0);
+    const uint32_t off0 = fragment_offset(lane);
+    const int sx = it.tile_x[tile], sy = it.tile_y[tile];
+    const int64_t row0 = int64_t(it.seg[sx]) * kTile, col0 = int64_t(it.seg[sy]) * kTile;
+    const uint32_t xa = uint32_t(sx) * kSegBytes, ya = uint32_t(sy) * kSegBytes;
+    const uint32_t xb = uint32_t(kSyr2kSlots + sx) * kSegBytes, yb = uint32_t(kSyr2kSlots + sy) * kSegBytes;
+
+    double acc[2][4][2];
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) acc[mi][ni][0] = acc[mi][ni][1] = 0.0;
+
+    uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;
+    for (int ks = 0; ks < k.n_ksteps; ++ks) {
+        if (!wait_full_at(k, st, parity, lane)) return false;
+        const uint32_t stage = k.smem32 + st * kStageBytes;
+        const uint32_t pxa = (stage + xa) | off0, pya = (stage + ya) | off0;
+        const uint32_t pxb = (stage + xb) | off0, pyb = (stage + yb) | off0;
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl) {
+            double a1[2], a2[2], b1[4], b2[4];
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi) {
+                a1[mi] = lds_f64(frag_addr<false>(pxa, 2 * half + mi, sl));
+                a2[mi] = lds_f64(frag_addr<false>(pxb, 2 * half + mi, sl));
+            }
+#pragma unroll
+            for (int ni = 0; ni < 4; ++ni) {
+                b1[ni] = lds_f64(frag_addr<false>(pyb, ni, sl));
+                b2[ni] = lds_f64(frag_addr<false>(pya, ni, sl));
+            }
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+                for (int ni = 0; ni < 4; ++ni) {
+                    dmma884(acc[mi][ni], a1[mi], b1[ni]);
+                    dmma884(acc[mi][ni], a2[mi], b2[ni]);
+                }
+        }
+        release_at(k, st, lane);
+        if (++st == kStages) { st = 0; parity ^= 1; }
+    }
+
+    for (int j = 0; j < n_c; ++j)
+        if (!wait_full(k, gc + j, lane)) return false;
+    const uint8_t* old_tile = nullptr;
+    if (n_c > 0 && row0 != col0)
+        old_tile = k.smem + ((gc + (tile >> 2)) % kStages) * kStageBytes + (tile & 3) * kCTileBytes;
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi) {
+        const int rr = (2 * half + mi) * 8 + gq;            // row inside the tile
+        const int64_t r = row0 + rr;
+        if (r >= k.N) continue;
+        double* crow = k.C + r * k.ldc;
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) {
+            const int64_t c = col0 + ni * 8 + 2 * t;
+            if (c > r) continue;
+            const bool both = (c + 1 <= r);
+            double v0 = k.alpha * acc[mi][ni][0], v1 = k.alpha * acc[mi][ni][1];
+            if (use_beta) {
+                double2 o = make_double2(0.0, 0.0);
+                if (old_tile) o = *reinterpret_cast<const double2*>(old_tile + rr * (kTile * 8) + (ni * 8 + 2 * t) * 8);
+                else { o.x = crow[c]; if (both) o.y = crow[c + 1]; }
+                v0 += k.beta * o.x; v1 += k.beta * o.y;
+            }
+            if (both && k.vec_ok) *reinterpret_cast<double2*>(crow + c) = make_double2(v0, v1);
+            else { crow[c] = v0; if (both) crow[c + 1] = v1; }
+        }
+    }
+    for (int j = 0; j < n_c; ++j) release(k, gc + j, lane);
+    return true;
+}
+
 // One MMA warp's share of one item: its ring steps from global step g on, then its write-out.
 // Every warp waits for and releases every ring step of the item, with or without work in it.
-template <bool kTN, bool kUpper>
+template <bool kTN, bool kUpper, bool kSyr2k = false>
 __device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it, uint32_t& g, int warp, int lane) {
     const int n_tile = it.n_tile;
     const int n_c = c_steps_of(k, n_tile);
     const uint32_t g0 = g;
     g += uint32_t(k.n_ksteps + n_c);
+    if (kSyr2k) {
+        if (warp < 2 * n_tile) return syr2k_tile_role(k, it, g0, n_c, warp, lane);
+        for (uint32_t s = g0; s < g; ++s) {             // no work in this item: keep the ring moving
+            if (!wait_full(k, s, lane)) return false;
+            release(k, s, lane);
+        }
+        return true;
+    }
     const bool scavenge = !k.gemm && it.pad != 0;      // set by prepare_item
     if (scavenge && warp == kMmaWarps - 1) return scavenger_role<kTN, kUpper>(k, it, g0, n_c, lane);
     if (warp < n_tile) return tile_role<kTN, kUpper>(k, it, g0, n_c, scavenge, warp, lane);
@@ -452,7 +550,7 @@ __device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it,
 // groups), its column segments come from Q (tmB, the first `pad` segments), its row segments
 // from P (tmA).
 // ---------------------------------------------------------------------------------------------
-template <bool kTN, bool kUpper>
+template <bool kTN, bool kUpper, bool kSyr2k = false>
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
@@ -473,7 +571,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     k.abort_flag = &s_abort; k.status = status;
     k.tmA = &tmA; k.tmB = &tmB; k.tmC = &tmC;
     k.N = N; k.ncols = ncols; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
-    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = gemm_col_tiles > 0;
+    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = gemm_col_tiles > 0; k.syr2k = kSyr2k;
     // Strided batch: the grid holds the work list once per matrix; the tensor maps are 3-D.
     // K-split (slice_ksteps > 0): the grid holds the list once per slice of the inner dimension;
     // slice s takes K-steps [s * slice_ksteps, ...) of the 2-D maps and writes partial matrix s.
@@ -524,13 +622,14 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == kMmaWarps) {
         if (lane == 0) {
             prefetch_tensormap(&tmA);
+            if (kSyr2k) prefetch_tensormap(&tmB);
             if (c_tma) prefetch_tensormap(&tmC);
             produce_item<kTN>(k, s_item, g);
             if (s_abort) drain_producer(k, g);
         }
         return;
     }
-    mma_warp_item<kTN, kUpper>(k, s_item, g, warp, lane);
+    mma_warp_item<kTN, kUpper, kSyr2k>(k, s_item, g, warp, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -561,7 +660,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
     k.abort_flag = &s_abort; k.status = status;
     k.tmA = &tmA; k.tmB = &tmA; k.tmC = &tmC;
     k.N = N; k.ncols = N; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
-    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false; k.batch = -1; k.k0 = 0;
+    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false; k.batch = -1; k.k0 = 0; k.syr2k = false;
 
     if (tid == 0) {
         s_abort = 0;
@@ -636,7 +735,8 @@ cudaError_t configure_f64_kernels() {
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[6] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false>),
+        const void* kernels[7] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, true>),
@@ -705,6 +805,22 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
                         : (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, false> : f64::syrk_f64_tbs_kernel<false, false>);
     kernel<<<dim3(unsigned(n_items)), threads, f64::kSmemBytes, stream>>>(
         tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
+        int64_t(0), int64_t(0), 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap* tmC,
+                             const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc,
+                             double alpha, double beta, int* d_status, cudaStream_t stream) {
+    cudaError_t e = configure_f64_kernels();
+    if (e != cudaSuccess) return e;
+    if (n_items == 0) return cudaSuccess;
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0) ? 1 : 0;
+    const int32_t n_ksteps = int32_t((M + f64::kBK - 1) / f64::kBK);
+    const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
+    CUtensorMap none{};
+    f64::syrk_f64_tbs_kernel<false, false, true><<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
+        tmA, tmB, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
         int64_t(0), int64_t(0), 0);
     return cudaGetLastError();
 }

@@ -52,6 +52,19 @@ __global__ void syrk_plain_kernel(int64_t N, int64_t M, const TA* __restrict__ A
     *c = (beta == TC(0)) ? alpha * s : alpha * s + beta * *c;
 }
 
+__global__ void syr2k_plain_kernel(int64_t N, int64_t M, const double* __restrict__ A, int64_t lda,
+                                   const double* __restrict__ B, int64_t ldb, double* __restrict__ C, int64_t ldc,
+                                   double alpha, double beta) {
+    const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
+    if (i >= N || j > i) return;
+    double s = 0.0;
+    for (int64_t k = 0; k < M; ++k)
+        s = fma(A[i * lda + k], B[j * ldb + k], fma(B[i * ldb + k], A[j * lda + k], s));
+    double* c = C + i * ldc + j;
+    *c = (beta == 0.0) ? alpha * s : alpha * s + beta * *c;
+}
+
 template <typename TC>
 __global__ void scale_lower_kernel(int64_t N, TC* __restrict__ C, int64_t ldc, TC beta, int upper) {
     const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -88,6 +101,14 @@ cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, in
         syrk_plain_kernel<__nv_bfloat16, float><<<grid2d(N, block), block, 0, stream>>>(
             N, M, static_cast<const __nv_bfloat16*>(A), rs, cs, static_cast<float*>(C), ldc,
             float(alpha), float(beta), upper);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_syr2k_plain(int64_t N, int64_t M, const double* A, int64_t lda, const double* B, int64_t ldb,
+                               double* C, int64_t ldc, double alpha, double beta, cudaStream_t stream) {
+    if (N == 0) return cudaSuccess;
+    const dim3 block(32, 8);
+    syr2k_plain_kernel<<<grid2d(N, block), block, 0, stream>>>(N, M, A, lda, B, ldb, C, ldc, alpha, beta);
     return cudaGetLastError();
 }
 
