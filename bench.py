@@ -208,6 +208,8 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
     dC = torch.zeros((N, N), dtype=C_pinned.dtype, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > L2 (126 MB)
 
+    if args.schedule != "tbs":                            # comparison schedules (kernel-only runs)
+        B.syrk_set_schedule({"square": B.SCHEDULE_SQUARE, "pair": B.SCHEDULE_PAIR_SQUARE}[args.schedule])
     B.syrk_plan_prepare(N, M, dtype)
     stats = B.syrk_get_schedule_stats(N, M, dtype)
     n_warm = args.warmup if args.kernel_only else max(args.warmup, 3)
@@ -242,7 +244,7 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
                               "steps": args.steps, "ms_per_step": ms_per_step, "kernel_only": True,
-                              "config": {"workload": wl.name, "N": N, "M": M,
+                              "config": {"workload": wl.name, "N": N, "M": M, "schedule": args.schedule,
                                          "operand": "M x N (Gram form)" if args.gram else "N x M"}}))
         return
 
@@ -543,10 +545,15 @@ def main():
                     help="with --kernel-only: hand the operand over stored M x N and time syrk_lower_tn (C = A^T A)")
     ap.add_argument("--batch", type=int, default=0,
                     help="with --kernel-only: that many problems of the workload's shape through syrk_lower_batched")
+    ap.add_argument("--schedule", default="tbs", choices=["tbs", "square", "pair"],
+                    help="with --kernel-only: the triangle-block schedule (default), the square-block comparison "
+                         "schedule, or square blocks on CTA pairs (16-bit types)")
     ap.add_argument("--syr2k", action="store_true",
                     help="with --kernel-only and an f64 workload: time syr2k_lower (rank-2k update) instead")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
+    if args.schedule != "tbs" and not args.kernel_only:
+        ap.error("--schedule needs --kernel-only")
     if args.syr2k and not args.kernel_only:
         ap.error("--syr2k needs --kernel-only")
     if args.batch > 0 and not args.kernel_only:

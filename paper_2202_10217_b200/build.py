@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtbsyrk.so")
-SOURCES = ["api.cu", "runtime.cu", "tbs_plan.cpp", "syrk_f64.cu", "syrk_bf16.cu", "syrk_plain.cu", "probe.cu", "syrk_static.cu", "cholesky_f64.cu"]
+SOURCES = ["api.cu", "runtime.cu", "tbs_plan.cpp", "syrk_f64.cu", "syrk_bf16.cu", "syrk_bf16_pair.cu", "syrk_plain.cu", "probe.cu", "syrk_static.cu", "cholesky_f64.cu"]
 HEADERS = ["kernels.h", "runtime.h", "tbs_plan.h", "device_utils.cuh",
            os.path.join("..", "..", "include", "tbsyrk.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",

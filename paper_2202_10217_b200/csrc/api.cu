@@ -164,6 +164,65 @@ int get_banded_plan(DeviceState* ds, int64_t N, int dtype, int max_bands, Banded
 
 }  // namespace
 
+namespace {
+// SYRK_SCHEDULE_PAIR_SQUARE for bfloat16 / binary16 operands stored N x M, lower triangle: the 256 x 256
+// blocks below the diagonal on the CTA-pair kernel, then the diagonal blocks (two tile rows each) on the
+// triangle-block kernel.  Returns SYRK_ERR_PLAN when the problem has fewer blocks than the GPU has pairs.
+int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc,
+                    double alpha, double beta, int dtype, cudaStream_t stream) {
+    const int tile = bf16_tile();
+    const int64_t n_tiles = (N + tile - 1) / tile, n_super = (n_tiles + 1) / 2;
+    if (n_super * (n_super - 1) / 2 < ds->sm_count / 2 || n_tiles >= (int64_t(1) << 20)) return SYRK_ERR_PLAN;
+    auto it = ds->pair_plans.find(n_tiles);
+    if (it == ds->pair_plans.end()) {
+        std::vector<int4> blocks;
+        std::vector<WorkItem> diag;
+        for (int64_t I = 0; I < n_super; ++I) {
+            for (int64_t J = 0; J < I; ++J)
+                blocks.push_back(make_int4(int(2 * I), int(2 * I + 1), int(2 * J), int(2 * J + 1)));
+            WorkItem w{};
+            w.kind = kDiag;
+            const int rows = int(std::min<int64_t>(2, n_tiles - 2 * I));
+            for (int x = 0; x < rows; ++x) w.seg[x] = int32_t(2 * I + x);
+            w.n_seg = rows;
+            int t = 0;
+            for (int x = 0; x < rows; ++x)
+                for (int y = 0; y <= x; ++y) { w.tile_x[t] = uint8_t(x); w.tile_y[t] = uint8_t(y); ++t; }
+            w.n_tile = t;
+            diag.push_back(w);
+        }
+        PairPlan pp;
+        pp.n_blocks = int32_t(blocks.size());
+        pp.n_diag = int64_t(diag.size());
+        bool ok = cudaMalloc(&pp.d_blocks, blocks.size() * sizeof(int4)) == cudaSuccess &&
+                  cudaMalloc(&pp.d_diag, diag.size() * sizeof(WorkItem)) == cudaSuccess;
+        ok = ok && cudaMemcpy(pp.d_blocks, blocks.data(), blocks.size() * sizeof(int4), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(pp.d_diag, diag.data(), diag.size() * sizeof(WorkItem), cudaMemcpyHostToDevice) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            if (pp.d_blocks) cudaFree(pp.d_blocks);
+            if (pp.d_diag) cudaFree(pp.d_diag);
+            return SYRK_ERR_ALLOC;
+        }
+        it = ds->pair_plans.emplace(n_tiles, pp).first;
+    }
+    const PairPlan& pp = it->second;
+    CUtensorMap tm, tmc;
+    int rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, tile, bf16_bk());
+    if (rc != SYRK_OK) return rc;
+    const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
+                       encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
+    cudaError_t e = launch_syrk_pair_square(tm, c_tma ? &tmc : nullptr, pp.d_blocks, pp.n_blocks, N, M, static_cast<float*>(C),
+                                            ldc, float(alpha), float(beta), dtype == SYRK_DTYPE_F16_F32, ds->d_status,
+                                            ds->sm_count, stream);
+    if (e != cudaSuccess) return SYRK_ERR_CUDA;
+    e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, pp.d_diag, pp.n_diag, N, M, static_cast<float*>(C), ldc, float(alpha),
+                         float(beta), 1, nullptr, nullptr, 0, nullptr, 0, 0, dtype - SYRK_DTYPE_BF16_F32, ds->d_status,
+                         ds->sm_count, stream);
+    return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+}
+}  // namespace
+
 int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
                             double beta, int dtype, cudaStream_t stream, int f64_launch, int a_is_m_by_n, int upper) {
     DeviceState* ds = nullptr;
@@ -176,6 +235,10 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
     if (!tma_ok(A, lda, dtype))
         return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream, upper) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
+    if (runtime().pair_square && (dtype == SYRK_DTYPE_BF16_F32 || dtype == SYRK_DTYPE_F16_F32) && !a_is_m_by_n && !upper) {
+        rc = run_pair_square(ds, N, M, A, lda, C, ldc, alpha, beta, dtype, stream);
+        if (rc != SYRK_ERR_PLAN) return rc;          // SYRK_ERR_PLAN: too few blocks for the pairs - the square list below
+    }
     DevicePlan* dp = nullptr;
     rc = get_device_plan(ds, N, dtype, &dp, upper);
     if (rc != SYRK_OK) return rc;
@@ -657,9 +720,11 @@ const char* syrk_strerror(int code) {
 }
 
 int syrk_set_schedule(int schedule) {
-    if (schedule != SYRK_SCHEDULE_TBS && schedule != SYRK_SCHEDULE_SQUARE) return SYRK_ERR_PLAN;
+    if (schedule != SYRK_SCHEDULE_TBS && schedule != SYRK_SCHEDULE_SQUARE && schedule != SYRK_SCHEDULE_PAIR_SQUARE)
+        return SYRK_ERR_PLAN;
     std::lock_guard<std::mutex> lock(runtime().mu);
-    runtime().schedule = schedule;
+    runtime().pair_square = schedule == SYRK_SCHEDULE_PAIR_SQUARE;
+    runtime().schedule = runtime().pair_square ? SYRK_SCHEDULE_SQUARE : schedule;
     return SYRK_OK;
 }
 

@@ -351,6 +351,10 @@ void release_all() {
             if (pk.second.d_tile_base) cudaFree(pk.second.d_tile_base);
             if (pk.second.d_cta_begin) cudaFree(pk.second.d_cta_begin);
         }
+        for (auto& pp : ds.pair_plans) {
+            if (pp.second.d_blocks) cudaFree(pp.second.d_blocks);
+            if (pp.second.d_diag) cudaFree(pp.second.d_diag);
+        }
         if (ds.d_status) cudaFree(ds.d_status);
         if (ds.d_tickets) cudaFree(ds.d_tickets);
         if (ds.d_partial) cudaFree(ds.d_partial);

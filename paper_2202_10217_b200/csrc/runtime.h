@@ -48,6 +48,15 @@ struct BandedPlan {
     std::vector<int64_t> item_end;
 };
 
+// Work lists of the CTA-pair square-block schedule: 256 x 256 blocks below the diagonal for the pair
+// kernel, and the diagonal blocks (two tile rows each) for the triangle-block kernel.
+struct PairPlan {
+    int4* d_blocks = nullptr;
+    int32_t n_blocks = 0;
+    WorkItem* d_diag = nullptr;
+    int64_t n_diag = 0;
+};
+
 struct DeviceState {
     int device = -1;
     int sm_count = 0;
@@ -57,6 +66,7 @@ struct DeviceState {
     // after another, so they can share a pair; launches on different streams cannot).
     int* d_tickets = nullptr;
     std::map<cudaStream_t, int> ticket_slot;
+    std::map<int64_t, PairPlan> pair_plans;   // by number of tile rows
     float* d_partial = nullptr;  // K-split workspace
     size_t partial_bytes = 0;
     // staging for the host-buffer entry point (grow-only)
@@ -77,6 +87,7 @@ struct Runtime {
     std::mutex mu;
     std::map<int, DeviceState> devices;
     int schedule = 0;
+    bool pair_square = false;   // SYRK_SCHEDULE_PAIR_SQUARE: square blocks, CTA-pair kernel where it applies
     int split_k = 0;
     int f64_launch = 0;
 };

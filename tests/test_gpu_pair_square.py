@@ -1,0 +1,65 @@
+"""GPU parity of the CTA-pair square-block schedule (SYRK_SCHEDULE_PAIR_SQUARE: 256 x 256 blocks on pairs
+of thread blocks, diagonal blocks on the triangle-block kernel) against the CPU reference, for the two
+16-bit input types: sizes with an even and an odd number of tile rows, ragged last tiles and K-steps,
+integer inputs bit for bit, general alpha / beta with pitches, NaN-poisoned C with beta = 0; the calls
+the schedule does not cover (small problems, the other storage order, the other types) must fall back
+and still match."""
+import numpy as np
+import pytest
+
+from paper_2202_10217_b200 import binding as B
+from paper_2202_10217_b200 import inputs as I
+
+from gpu_util import assert_within_tolerance, run_case
+from test_gpu_syrk import make_A
+
+pytestmark = pytest.mark.gpu
+DT = pytest.mark.parametrize("dtype", [B.DTYPE_BF16_F32, B.DTYPE_F16_F32], ids=["bf16", "f16"])
+
+
+@pytest.fixture(autouse=True)
+def pair_schedule():
+    B.syrk_set_schedule(B.SCHEDULE_PAIR_SQUARE)
+    yield
+    B.syrk_set_schedule(B.SCHEDULE_TBS)
+
+
+SIZES = [(3200, 136), (3328, 64), (4200, 320), (3500, 72), (6145, 200)]
+
+
+@DT
+def test_real_inputs_within_tolerance(dtype):
+    for n, (N, M) in enumerate(SIZES):
+        A = make_A(N, M, dtype, seed=7000 + n)
+        got, ref, bound = run_case(A, dtype, 1.0, 0.0)
+        assert_within_tolerance(got, ref, bound, M, 1.0, 0.0, None, dtype)
+
+
+@DT
+def test_integer_inputs_are_bit_exact(dtype):
+    for n, (N, M) in enumerate(SIZES[:4]):
+        A = make_A(N, M, dtype, seed=7100 + n, kind="int")
+        got, ref, bound = run_case(A, dtype, 1.0, 0.0)
+        assert_within_tolerance(got, ref, bound, M, 1.0, 0.0, None, dtype, exact=True)
+
+
+@DT
+@pytest.mark.parametrize("alpha,beta", [(-1.0, 1.0), (2.5, -0.5), (1.0, 0.0)])
+def test_alpha_beta_pitches_and_poison(dtype, alpha, beta):
+    N, M = 3300, 104
+    A = make_A(N, M, dtype, seed=7200, kind="int")
+    Cin = I.random_c(N, 7201, dtype)
+    got, ref, bound = run_case(A, dtype, alpha, beta, Cin if beta != 0.0 else None, lda=M + 16, ldc=N + 12,
+                               a_offset=8, c_offset=4, poison=(beta == 0.0))
+    assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin if beta != 0.0 else None, dtype)
+    got, ref, bound = run_case(A, dtype, alpha, beta, Cin if beta != 0.0 else None, ldc=N + 3)   # odd pitch: scalar stores
+    assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin if beta != 0.0 else None, dtype)
+
+
+def test_calls_outside_the_schedule_fall_back():
+    for dtype, N, M, tn, upper in [(B.DTYPE_BF16_F32, 700, 72, False, False), (B.DTYPE_BF16_F32, 3200, 72, True, False),
+                                   (B.DTYPE_F16_F32, 3200, 72, False, True), (B.DTYPE_F64, 1100, 48, False, False),
+                                   (B.DTYPE_E4M3_F32, 3200, 144, False, False)]:
+        A = make_A(N, M, dtype, seed=7300)
+        got, ref, bound = run_case(A, dtype, 1.0, 0.0, tn=tn, upper=upper)
+        assert_within_tolerance(got, ref, bound, M, 1.0, 0.0, None, dtype)
