@@ -166,8 +166,7 @@ int get_banded_plan(DeviceState* ds, int64_t N, int dtype, int max_bands, Banded
 
 namespace {
 // SYRK_SCHEDULE_PAIR_SQUARE for bfloat16 / binary16 operands stored N x M, lower triangle: the 256 x 256
-// blocks below the diagonal on the CTA-pair kernel, then the diagonal blocks (two tile rows each) on the
-// triangle-block kernel.  Returns SYRK_ERR_PLAN when the problem has fewer blocks than the GPU has pairs.
+// blocks below and on the diagonal on the CTA-pair kernel.  Returns SYRK_ERR_PLAN when the problem has fewer blocks than the GPU has pairs.
 int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc,
                     double alpha, double beta, int dtype, cudaStream_t stream) {
     const int tile = bf16_tile();
@@ -175,33 +174,20 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
     if (n_super * (n_super - 1) / 2 < ds->sm_count / 2 || n_tiles >= (int64_t(1) << 20)) return SYRK_ERR_PLAN;
     auto it = ds->pair_plans.find(n_tiles);
     if (it == ds->pair_plans.end()) {
+        // heaviest first is moot (all blocks cost the same); the diagonal blocks go last
         std::vector<int4> blocks;
-        std::vector<WorkItem> diag;
-        for (int64_t I = 0; I < n_super; ++I) {
+        for (int64_t I = 0; I < n_super; ++I)
             for (int64_t J = 0; J < I; ++J)
                 blocks.push_back(make_int4(int(2 * I), int(2 * I + 1), int(2 * J), int(2 * J + 1)));
-            WorkItem w{};
-            w.kind = kDiag;
-            const int rows = int(std::min<int64_t>(2, n_tiles - 2 * I));
-            for (int x = 0; x < rows; ++x) w.seg[x] = int32_t(2 * I + x);
-            w.n_seg = rows;
-            int t = 0;
-            for (int x = 0; x < rows; ++x)
-                for (int y = 0; y <= x; ++y) { w.tile_x[t] = uint8_t(x); w.tile_y[t] = uint8_t(y); ++t; }
-            w.n_tile = t;
-            diag.push_back(w);
-        }
+        for (int64_t I = 0; I < n_super; ++I)
+            blocks.push_back(make_int4(int(2 * I), int(2 * I + 1), int(2 * I), int(2 * I + 1)));
         PairPlan pp;
         pp.n_blocks = int32_t(blocks.size());
-        pp.n_diag = int64_t(diag.size());
-        bool ok = cudaMalloc(&pp.d_blocks, blocks.size() * sizeof(int4)) == cudaSuccess &&
-                  cudaMalloc(&pp.d_diag, diag.size() * sizeof(WorkItem)) == cudaSuccess;
-        ok = ok && cudaMemcpy(pp.d_blocks, blocks.data(), blocks.size() * sizeof(int4), cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMemcpy(pp.d_diag, diag.data(), diag.size() * sizeof(WorkItem), cudaMemcpyHostToDevice) == cudaSuccess;
+        bool ok = cudaMalloc(&pp.d_blocks, blocks.size() * sizeof(int4)) == cudaSuccess;
+        ok = ok && cudaMemcpy(pp.d_blocks, blocks.data(), blocks.size() * sizeof(int4), cudaMemcpyHostToDevice) == cudaSuccess;
         if (!ok) {
             cudaGetLastError();
             if (pp.d_blocks) cudaFree(pp.d_blocks);
-            if (pp.d_diag) cudaFree(pp.d_diag);
             return SYRK_ERR_ALLOC;
         }
         it = ds->pair_plans.emplace(n_tiles, pp).first;
@@ -215,10 +201,6 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
     cudaError_t e = launch_syrk_pair_square(tm, c_tma ? &tmc : nullptr, pp.d_blocks, pp.n_blocks, N, M, static_cast<float*>(C),
                                             ldc, float(alpha), float(beta), dtype == SYRK_DTYPE_F16_F32, ds->d_status,
                                             ds->sm_count, stream);
-    if (e != cudaSuccess) return SYRK_ERR_CUDA;
-    e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, pp.d_diag, pp.n_diag, N, M, static_cast<float*>(C), ldc, float(alpha),
-                         float(beta), 1, nullptr, nullptr, 0, nullptr, 0, 0, dtype - SYRK_DTYPE_BF16_F32, ds->d_status,
-                         ds->sm_count, stream);
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
 }  // namespace

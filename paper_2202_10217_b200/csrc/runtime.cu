@@ -353,7 +353,6 @@ void release_all() {
         }
         for (auto& pp : ds.pair_plans) {
             if (pp.second.d_blocks) cudaFree(pp.second.d_blocks);
-            if (pp.second.d_diag) cudaFree(pp.second.d_diag);
         }
         if (ds.d_status) cudaFree(ds.d_status);
         if (ds.d_tickets) cudaFree(ds.d_tickets);

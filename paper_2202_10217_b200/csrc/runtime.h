@@ -48,13 +48,10 @@ struct BandedPlan {
     std::vector<int64_t> item_end;
 };
 
-// Work lists of the CTA-pair square-block schedule: 256 x 256 blocks below the diagonal for the pair
-// kernel, and the diagonal blocks (two tile rows each) for the triangle-block kernel.
+// Work list of the CTA-pair square-block schedule: the 256 x 256 blocks below and on the diagonal.
 struct PairPlan {
     int4* d_blocks = nullptr;
     int32_t n_blocks = 0;
-    WorkItem* d_diag = nullptr;
-    int64_t n_diag = 0;
 };
 
 struct DeviceState {

@@ -8,8 +8,8 @@
 // the N-operand halves of both.  This shape does not fit triangle blocks (a pair shares its
 // N-operand; the left-over pairs of a triangle block have none in common), so the kernel runs the
 // square-block schedule of the paper's comparison algorithm (Section 5, the blocks of the generic
-// out-of-core scheme of Algorithm 3): off-diagonal 256 x 256 squares here, the diagonal blocks by
-// the triangle-block kernel's DIAG items.
+// out-of-core scheme of Algorithm 3): 256 x 256 squares, those on the diagonal included (a quarter of
+// such a block is computed in vain; they are one block in sixty-odd at the sizes this schedule is for).
 //
 // Per CTA: warp 0 = TMA producer (2 loads of 16 KB per stage, 6 stages, completion counted on the
 // LEADER CTA's full barrier), warp 1 = TMEM allocation (both CTAs) and, in the leader CTA (cluster
@@ -126,8 +126,9 @@ __device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// blocks[i] = {X0, X1, Y0, Y1}: tile rows of the 256 x 256 block i (X0 > Y1).  The pair with index p
-// runs blocks p, p + pairs, p + 2 pairs, ...
+// blocks[i] = {X0, X1, Y0, Y1}: tile rows of the 256 x 256 block i, below the diagonal (X0 > Y1) or on it
+// (X = Y: the two diagonal tiles are stored with the triangle mask, the tile above the diagonal is
+// computed but not stored).  The pair with index p runs blocks p, p + pairs, p + 2 pairs, ...
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
                         const int4* __restrict__ blocks, int32_t n_blocks, int64_t N, int32_t n_ksteps,
@@ -242,7 +243,9 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             for (int t = 0; t < 2; ++t) {
                 const int64_t tcol = t == 0 ? blk.z : blk.w;
                 const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccCols + uint32_t(t) * kTile;
-                const bool staged = tma_store_ok && beta == 0.f && trow * kTile + quarter * 32 < N;
+                if (tcol > trow) continue;                          // diagonal block: the tile above the diagonal is not stored
+                const bool on_diag = tcol == trow;
+                const bool staged = tma_store_ok && !on_diag && beta == 0.f && trow * kTile + quarter * 32 < N;
 #pragma unroll 1
                 for (int cb = 0; cb < kTile; cb += 32) {
                     uint32_t v[32];
@@ -264,8 +267,17 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         continue;
                     }
                     if (r >= N) continue;
-                    float* crow = C + r * ldc + c0;                  // strictly below the diagonal: every column kept
-                    if (vec_ok) {
+                    float* crow = C + r * ldc + c0;                  // below the diagonal every column is kept
+                    if (on_diag && c0 + 31 > r) {                    // diagonal tile: columns <= row only
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (c0 + j <= r) {
+                                float o = alpha * __uint_as_float(v[j]);
+                                if (beta != 0.f) o += beta * crow[j];
+                                crow[j] = o;
+                            }
+                        }
+                    } else if (vec_ok) {
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             float4 o = make_float4(alpha * __uint_as_float(v[4 * j]), alpha * __uint_as_float(v[4 * j + 1]),
