@@ -83,8 +83,11 @@ int auto_split_k_f64(int64_t n_items, int64_t N, int64_t M, int bk, int sm_count
     return best;
 }
 
-int pick_split_k(const DeviceState* ds, const DevicePlan* dp, int64_t M, int bk) {
-    return auto_split_k(dp->plan.items, M, bk, ds->sm_count, runtime().split_k);
+int pick_split_k(const DeviceState* ds, DevicePlan* dp, int64_t M, int bk) {
+    if (runtime().split_k > 0) return auto_split_k(dp->plan.items, M, bk, ds->sm_count, runtime().split_k);
+    auto it = dp->auto_split.find(M);
+    if (it == dp->auto_split.end()) it = dp->auto_split.emplace(M, auto_split_k(dp->plan.items, M, bk, ds->sm_count, 0)).first;
+    return it->second;
 }
 
 // One launch of the item kernels over a list (the whole plan, or the items of one band of rows).
@@ -171,7 +174,29 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
                     double alpha, double beta, int dtype, cudaStream_t stream) {
     const int tile = bf16_tile();
     const int64_t n_tiles = (N + tile - 1) / tile, n_super = (n_tiles + 1) / 2;
-    if (n_super * (n_super - 1) / 2 < ds->sm_count / 2 || n_tiles >= (int64_t(1) << 20)) return SYRK_ERR_PLAN;
+    const int64_t n_blk = n_super * (n_super + 1) / 2, pairs = ds->sm_count / 2;
+    const int64_t n_ksteps = (M + bf16_bk() - 1) / bf16_bk();
+    if (n_tiles >= (int64_t(1) << 15)) return SYRK_ERR_PLAN;
+    // K-slices: with fewer blocks than a few rounds of pairs the inner dimension is cut so that every pair
+    // has work; the number of slices minimises rounds x (K-steps per slice + 20) plus the partial traffic.
+    int split = 1;
+    if (runtime().split_k > 0) split = int(std::min<int64_t>(runtime().split_k, n_ksteps));
+    else if (n_blk < 4 * pairs) {
+        double best = 0.0;
+        for (int sp = 1; sp <= 32 && sp <= n_ksteps / 8; ++sp) {
+            const int64_t rounds = (n_blk * sp + pairs - 1) / pairs;
+            double cost = double(rounds) * (double((n_ksteps + sp - 1) / sp) + 20.0);
+            if (sp > 1) cost += 0.1 * double(sp) * double(n_blk) * 2.0 + 40.0;
+            if (sp == 1 || cost < best) { best = cost; split = sp; }
+        }
+    }
+    if (n_blk * split < pairs) return SYRK_ERR_PLAN;           // still too few units for the pairs
+    if (split > 1) {
+        void* p = ds->d_partial;
+        const int rc2 = ensure_device_bytes(&p, &ds->partial_bytes, size_t(split) * size_t(n_blk) * 4 * tile * tile * sizeof(float));
+        ds->d_partial = static_cast<float*>(p);
+        if (rc2 != SYRK_OK) return rc2;
+    }
     auto it = ds->pair_plans.find(n_tiles);
     if (it == ds->pair_plans.end()) {
         // heaviest first is moot (all blocks cost the same); the diagonal blocks go last
@@ -200,7 +225,7 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
                        encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
     cudaError_t e = launch_syrk_pair_square(tm, c_tma ? &tmc : nullptr, pp.d_blocks, pp.n_blocks, N, M, static_cast<float*>(C),
                                             ldc, float(alpha), float(beta), dtype == SYRK_DTYPE_F16_F32, ds->d_status,
-                                            ds->sm_count, stream);
+                                            ds->sm_count, stream, split, ds->d_partial);
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
 }  // namespace

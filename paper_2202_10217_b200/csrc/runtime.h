@@ -37,6 +37,8 @@ struct DevicePlan {
     int64_t total_tiles = 0;
     int64_t* d_cta_begin = nullptr;  // BF16: first item of each persistent thread block (n_ctas + 1)
     int n_ctas = 0;
+    std::map<int64_t, int> auto_split;   // tcgen05: modelled number of K-slices by inner dimension (the model
+                                         // walks every unit of every candidate: too slow to redo on every call)
 };
 
 // Square-block work list in row order for the host-buffer entry point: band j owns the rows

@@ -133,7 +133,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
                         const int4* __restrict__ blocks, int32_t n_blocks, int64_t N, int32_t n_ksteps,
                         float* __restrict__ C, int64_t ldc, float alpha, float beta, int vec_ok, int tma_store_ok,
-                        uint32_t fmt, int* __restrict__ status) {
+                        uint32_t fmt, int* __restrict__ status, int32_t split, float* __restrict__ partial) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* staging = smem + kStages * kStageBytes;
@@ -148,6 +148,9 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_rank();                  // 0 = leader of the pair
     const int32_t pair_id = int32_t(blockIdx.x >> 1), n_pairs = int32_t(gridDim.x >> 1);
+    // Units: (block, K-slice) pairs, slice-major (split == 1: the blocks themselves).  Unit w is block
+    // w % n_blocks restricted to K-steps [n_ksteps * s / split, n_ksteps * (s + 1) / split), s = w / n_blocks.
+    const int32_t n_units = n_blocks * split;
 
     if (tid == 0) {
         s_abort = 0;
@@ -169,11 +172,13 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         if (lane == 0) {
             prefetch_tensormap(&tmA);
             uint32_t g = 0;
-            for (int32_t b = pair_id; b < n_blocks && !s_abort; b += n_pairs) {
-                const int4 blk = blocks[b];
+            for (int32_t w = pair_id; w < n_units && !s_abort; w += n_pairs) {
+                const int4 blk = blocks[w % n_blocks];
+                const int32_t sl = w / n_blocks;
+                const int32_t k0 = int32_t(int64_t(n_ksteps) * sl / split), k1 = int32_t(int64_t(n_ksteps) * (sl + 1) / split);
                 const int32_t row_x = (rank == 0 ? blk.x : blk.y) * kTile;       // this CTA's M-operand rows
                 const int32_t row_y = (rank == 0 ? blk.z : blk.w) * kTile;       // this CTA's half of the N-operand
-                for (int ks = 0; ks < n_ksteps; ++ks, ++g) {
+                for (int ks = k0; ks < k1; ++ks, ++g) {
                     const uint32_t st = g % kStages;
                     if (g >= kStages && !mbar_wait_bounded(&empty_bar[st], ((g / kStages) - 1) & 1, &s_abort)) {
                         s_abort = 1; atomicOr(status, kStatusWaitEmpty); break;
@@ -194,7 +199,9 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             const uint32_t smem_base = smem_u32(smem);
             const uint64_t desc_hi = smem_desc_sw128(0);
             const uint32_t idesc = instr_desc_pair(fmt);
-            for (int32_t b = pair_id; b < n_blocks && !s_abort; b += n_pairs, ++n_done) {
+            for (int32_t w = pair_id; w < n_units && !s_abort; w += n_pairs, ++n_done) {
+                const int32_t sl = w / n_blocks;
+                const int32_t k0 = int32_t(int64_t(n_ksteps) * sl / split), k1 = int32_t(int64_t(n_ksteps) * (sl + 1) / split);
                 const uint32_t acc = n_done & 1;
                 if (n_done >= 2 && !mbar_wait_bounded(&tmem_empty_bar[acc], ((n_done >> 1) - 1) & 1, &s_abort)) {
                     s_abort = 1; atomicOr(status, kStatusWaitTmem); break;
@@ -202,7 +209,7 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 tc_fence_after();
                 const uint32_t d_addr = tmem_base + acc * kAccCols;
                 bool ok = true;
-                for (int ks = 0; ks < n_ksteps; ++ks, ++g) {
+                for (int ks = k0; ks < k1; ++ks, ++g) {
                     const uint32_t st = g % kStages;
                     if (!mbar_wait_bounded(&full_bar[st], (g / kStages) & 1, &s_abort)) {
                         s_abort = 1; atomicOr(status, kStatusWaitFull); ok = false; break;
@@ -212,7 +219,7 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
                     for (int kk = 0; kk < kBK / 16; ++kk)
                         tc_mma_pair(d_addr, desc_hi | uint64_t(a_lo + 2 * kk), desc_hi | uint64_t(b_lo + 2 * kk), idesc,
-                                    (kk > 0 || ks > 0) ? 1u : 0u);
+                                    (kk > 0 || ks > k0) ? 1u : 0u);
                     tc_commit_pair(&empty_bar[st]);          // both CTAs may refill the stage
                 }
                 if (!ok) break;
@@ -231,7 +238,8 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         const int row_in_tile = quarter * 32 + lane;
         uint8_t* my_staging = staging + (warp - 2) * 2 * kStageBufBytes;
         uint32_t n_done = 0, n_stores = 0;
-        for (int32_t b = pair_id; b < n_blocks && !s_abort; b += n_pairs, ++n_done) {
+        for (int32_t w = pair_id; w < n_units && !s_abort; w += n_pairs, ++n_done) {
+            const int32_t b = w % n_blocks, sl = w / n_blocks;
             const int4 blk = blocks[b];
             const uint32_t acc = n_done & 1;
             const int64_t trow = rank == 0 ? blk.x : blk.y;
@@ -245,11 +253,22 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccCols + uint32_t(t) * kTile;
                 if (tcol > trow) continue;                          // diagonal block: the tile above the diagonal is not stored
                 const bool on_diag = tcol == trow;
-                const bool staged = tma_store_ok && !on_diag && beta == 0.f && trow * kTile + quarter * 32 < N;
+                const bool staged = tma_store_ok && split == 1 && !on_diag && beta == 0.f && trow * kTile + quarter * 32 < N;
+                // K-split: raw partial tile (slice, block, rank, t), 128 x 128 binary32
+                float* part = split > 1 ? partial + (((int64_t(sl) * n_blocks + b) * 4 + int64_t(rank) * 2 + t) * kTile + row_in_tile) * kTile
+                                        : nullptr;
 #pragma unroll 1
                 for (int cb = 0; cb < kTile; cb += 32) {
                     uint32_t v[32];
                     tmem_ld_32x32(taddr + cb, v);
+                    if (split > 1) {
+                        float4* dst = reinterpret_cast<float4*>(part + cb);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                 __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        continue;
+                    }
                     const int64_t c0 = tcol * kTile + cb;
                     if (staged) {
                         uint8_t* buf = my_staging + (n_stores & 1) * kStageBufBytes;
@@ -317,11 +336,43 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     }
 }
 
+// K-split calls: stored entries of tile (rank, t) of block blockIdx.x <- alpha * (sum of the slices' partial
+// tiles, in slice order) + beta * C.
+__global__ void __launch_bounds__(256)
+pair_splitk_reduce_kernel(const int4* __restrict__ blocks, int32_t n_blocks, int32_t split, const float* __restrict__ partial,
+                          int64_t N, float* __restrict__ C, int64_t ldc, float alpha, float beta) {
+    const int4 blk = blocks[blockIdx.x];
+    const int rank = blockIdx.y >> 1, t = blockIdx.y & 1;
+    const int64_t trow = rank == 0 ? blk.x : blk.y, tcol = t == 0 ? blk.z : blk.w;
+    if (tcol > trow) return;
+    for (int e = threadIdx.x; e < kTile * kTile / 4; e += blockDim.x) {
+        const int rr = e / (kTile / 4), cc = (e % (kTile / 4)) * 4;
+        const int64_t r = trow * kTile + rr;
+        if (r >= N) continue;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sl = 0; sl < split; ++sl) {
+            const float4 p = *reinterpret_cast<const float4*>(
+                partial + (((int64_t(sl) * n_blocks + blockIdx.x) * 4 + blockIdx.y) * kTile + rr) * kTile + cc);
+            s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+        }
+        const float vals[4] = {s.x, s.y, s.z, s.w};
+        float* crow = C + r * ldc + tcol * kTile + cc;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (tcol * kTile + cc + j <= r) {
+                float o = alpha * vals[j];
+                if (beta != 0.f) o += beta * crow[j];
+                crow[j] = o;
+            }
+        }
+    }
+}
+
 }  // namespace pair
 
 cudaError_t launch_syrk_pair_square(const CUtensorMap& tmA, const CUtensorMap* tmC, const int4* d_blocks, int32_t n_blocks,
                                     int64_t N, int64_t M, float* C, int64_t ldc, float alpha, float beta, int is_f16,
-                                    int* d_status, int sm_count, cudaStream_t stream) {
+                                    int* d_status, int sm_count, cudaStream_t stream, int split_k, float* d_partial) {
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
@@ -333,13 +384,18 @@ cudaError_t launch_syrk_pair_square(const CUtensorMap& tmA, const CUtensorMap* t
     }
     if (n_blocks <= 0) return cudaSuccess;
     const int32_t n_ksteps = int32_t((M + pair::kBK - 1) / pair::kBK);
+    const int split = (split_k < 1 || d_partial == nullptr) ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
     int pairs = sm_count / 2;
-    if (pairs > n_blocks) pairs = n_blocks;
+    if (int64_t(pairs) > int64_t(n_blocks) * split) pairs = n_blocks * split;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0) ? 1 : 0;
     CUtensorMap none{};
     pair::syrk_pair_square_kernel<<<dim3(unsigned(2 * pairs)), pair::kThreads, pair::kSmemBytes, stream>>>(
         tmA, tmC ? *tmC : none, d_blocks, n_blocks, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0,
-        is_f16 ? 0u : 1u, d_status);
+        is_f16 ? 0u : 1u, d_status, split, d_partial);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || split == 1) return e;
+    pair::pair_splitk_reduce_kernel<<<dim3(unsigned(n_blocks), 4), 256, 0, stream>>>(d_blocks, n_blocks, split, d_partial, N, C,
+                                                                                     ldc, alpha, beta);
     return cudaGetLastError();
 }
 

@@ -56,6 +56,30 @@ def test_alpha_beta_pitches_and_poison(dtype, alpha, beta):
     assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin if beta != 0.0 else None, dtype)
 
 
+@DT
+def test_k_split_automatic_and_forced(dtype):
+    """Few blocks and a long inner dimension: (block, K-slice) units with partial tiles summed in slice order.
+    Automatic choice at 2048 x 16384 and 1100 x 8200 (odd number of tile rows, ragged last K-step); forced
+    2, 3 and 7 slices at a size that needs none; integer inputs bit for bit."""
+    for n, (N, M) in enumerate([(2048, 16384), (1100, 8200)]):
+        A = make_A(N, M, dtype, seed=7400 + n, kind="int")
+        Cin = np.round(I.random_c(N, 7401, dtype) * 4).astype(np.float32)
+        got, ref, bound = run_case(A, dtype, 1.0, -1.0, Cin)
+        assert_within_tolerance(got, ref, bound, M, 1.0, -1.0, Cin, dtype, exact=True)
+        A = make_A(N, M, dtype, seed=7410 + n)
+        got, ref, bound = run_case(A, dtype, 0.5, 0.0, poison=True)
+        assert_within_tolerance(got, ref, bound, M, 0.5, 0.0, None, dtype)
+    for split in (2, 3, 7):
+        A = make_A(3200, 1288, dtype, seed=7420 + split)
+        Cin = I.random_c(3200, 7421, dtype)
+        try:
+            B.syrk_set_split_k(split)
+            got, ref, bound = run_case(A, dtype, -1.0, 1.0, Cin, ldc=3203)
+        finally:
+            B.syrk_set_split_k(0)
+        assert_within_tolerance(got, ref, bound, 1288, -1.0, 1.0, Cin, dtype)
+
+
 def test_calls_outside_the_schedule_fall_back():
     for dtype, N, M, tn, upper in [(B.DTYPE_BF16_F32, 700, 72, False, False), (B.DTYPE_BF16_F32, 3200, 72, True, False),
                                    (B.DTYPE_F16_F32, 3200, 72, False, True), (B.DTYPE_F64, 1100, 48, False, False),
