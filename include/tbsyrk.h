@@ -64,9 +64,10 @@ extern "C" {
 #define SYRK_SCHEDULE_SQUARE  1    /* square and diagonal blocks only (comparison schedule) */
 #define SYRK_SCHEDULE_PAIR_SQUARE 2 /* square blocks of 256 x 256 on pairs of thread blocks (tcgen05
                                       cta_group::2: the pair shares the N-operand, which halves its
-                                      shared-memory traffic) for bfloat16 / binary16 operands stored
-                                      N x M, lower triangle, when the problem has at least as many
-                                      blocks as the GPU has pairs; every other call runs
+                                      shared-memory traffic) for the tcgen05 types (every dtype but
+                                      binary64), operands stored N x M, lower triangle, when the
+                                      problem (cut along the inner dimension if need be) gives every
+                                      pair a block; every other call runs
                                       SYRK_SCHEDULE_SQUARE.  A second comparison schedule: the pair
                                       form does not fit triangle blocks.                          */
 

@@ -168,14 +168,15 @@ int get_banded_plan(DeviceState* ds, int64_t N, int dtype, int max_bands, Banded
 }  // namespace
 
 namespace {
-// SYRK_SCHEDULE_PAIR_SQUARE for bfloat16 / binary16 operands stored N x M, lower triangle: the 256 x 256
+// SYRK_SCHEDULE_PAIR_SQUARE for tcgen05-type operands stored N x M, lower triangle: the 256 x 256
 // blocks below and on the diagonal on the CTA-pair kernel.  Returns SYRK_ERR_PLAN when the problem has fewer blocks than the GPU has pairs.
 int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc,
                     double alpha, double beta, int dtype, cudaStream_t stream) {
     const int tile = bf16_tile();
     const int64_t n_tiles = (N + tile - 1) / tile, n_super = (n_tiles + 1) / 2;
     const int64_t n_blk = n_super * (n_super + 1) / 2, pairs = ds->sm_count / 2;
-    const int64_t n_ksteps = (M + bf16_bk() - 1) / bf16_bk();
+    const int64_t bk = 128 / int64_t(a_elem(dtype));              // columns in a 128-byte stage row
+    const int64_t n_ksteps = (M + bk - 1) / bk;
     if (n_tiles >= (int64_t(1) << 15)) return SYRK_ERR_PLAN;
     // K-slices: with fewer blocks than a few rounds of pairs the inner dimension is cut so that every pair
     // has work; the number of slices minimises rounds x (K-steps per slice + 20) plus the partial traffic.
@@ -219,12 +220,12 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
     }
     const PairPlan& pp = it->second;
     CUtensorMap tm, tmc;
-    int rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, tile, bf16_bk());
+    int rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, tile, int(bk));
     if (rc != SYRK_OK) return rc;
     const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                        encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
     cudaError_t e = launch_syrk_pair_square(tm, c_tma ? &tmc : nullptr, pp.d_blocks, pp.n_blocks, N, M, static_cast<float*>(C),
-                                            ldc, float(alpha), float(beta), dtype == SYRK_DTYPE_F16_F32, ds->d_status,
+                                            ldc, float(alpha), float(beta), dtype - SYRK_DTYPE_BF16_F32, ds->d_status,
                                             ds->sm_count, stream, split, ds->d_partial);
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
@@ -242,7 +243,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
     if (!tma_ok(A, lda, dtype))
         return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream, upper) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
-    if (runtime().pair_square && (dtype == SYRK_DTYPE_BF16_F32 || dtype == SYRK_DTYPE_F16_F32) && !a_is_m_by_n && !upper) {
+    if (runtime().pair_square && is_tcgen05_dtype(dtype) && !a_is_m_by_n && !upper) {
         rc = run_pair_square(ds, N, M, A, lda, C, ldc, alpha, beta, dtype, stream);
         if (rc != SYRK_ERR_PLAN) return rc;          // SYRK_ERR_PLAN: too few blocks for the pairs - the square list below
     }

@@ -61,14 +61,14 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
                              int a_kind, int* d_status, int sm_count, cudaStream_t stream,
                              int64_t batch = 0, int64_t c_batch_stride = 0, int upper = 0);
-// Square-block comparison kernel on CTA pairs (tcgen05 cta_group::2) for bfloat16 / binary16 operands
-// stored N x M: block i of `d_blocks` = {X0, X1, Y0, Y1}, tile rows (128 rows each) of a 256 x 256 block
+// Square-block comparison kernel on CTA pairs (tcgen05 cta_group::2) for operands of input kind `a_kind`
+// (as launch_syrk_bf16) stored N x M: block i of `d_blocks` = {X0, X1, Y0, Y1}, tile rows (128 rows each) of a 256 x 256 block
 // strictly below the diagonal; pair p of the grid runs blocks p, p + pairs, ...  `tmA` and `tmC` as for
 // launch_syrk_bf16 (boxes of 128 rows x 64 columns; 32 x 32 binary32 boxes).  Lower triangle only.
 // Blocks with X = Y lie on the diagonal.  `split_k` > 1 with `d_partial` (split_k x n_blocks x 4 tiles of
 // 128 x 128 floats): units are (block, K-slice) pairs, partial tiles summed in slice order by a second kernel.
 cudaError_t launch_syrk_pair_square(const CUtensorMap& tmA, const CUtensorMap* tmC, const int4* d_blocks, int32_t n_blocks,
-                                    int64_t N, int64_t M, float* C, int64_t ldc, float alpha, float beta, int is_f16,
+                                    int64_t N, int64_t M, float* C, int64_t ldc, float alpha, float beta, int a_kind,
                                     int* d_status, int sm_count, cudaStream_t stream, int split_k = 1,
                                     float* d_partial = nullptr);
 int bf16_tile();

@@ -1,4 +1,5 @@
-// Square-block comparison kernel for the 16-bit types on CTA pairs (tcgen05 cta_group::2).
+// Square-block comparison kernel on CTA pairs (tcgen05 cta_group::2) for the tcgen05 input types
+// (bfloat16, binary16, binary32 read as TF32, FP8 E4M3; a stage row is 128 bytes for all of them).
 //
 // The triangle-block kernel (syrk_bf16.cu) is bound by shared-memory traffic: one SM feeds both
 // MMA operands from its own shared memory.  A CTA pair halves the N-operand traffic: the pair
@@ -24,9 +25,8 @@ namespace tbsyrk {
 namespace pair {
 
 constexpr int kTile = 128;
-constexpr int kBK = 64;                            // bf16 / f16 columns per stage (128 bytes)
 constexpr int kStages = 6;
-constexpr int kSegBytes = kTile * kBK * 2;         // 16384
+constexpr int kSegBytes = kTile * 128;             // 128 rows of 128 bytes: 64 two-byte, 32 binary32 or 128 FP8 columns
 constexpr int kStageBytes = 2 * kSegBytes;         // own X rows + own Y rows
 constexpr int kThreads = 192;
 constexpr int kStoreBox = 32;
@@ -84,12 +84,24 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(smem_u32(bar)), "h"(mask) : "memory");
 }
+// Input kinds as in the triangle-block kernel: 0 bfloat16, 1 TF32, 2 FP8 E4M3, 3 binary16.
+template <int kKind>
 __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (kKind == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    else if (kKind == 2)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -112,8 +124,8 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {   // K-majo
     d |= uint64_t(2) << 61;
     return d;
 }
-// kind::f16 instruction descriptor for the pair: D = FP32, A = B = format `fmt` (1 bfloat16, 0 binary16),
-// both K-major, N = 256, M = 256 (128 rows per CTA).
+// Instruction descriptor for the pair: D = FP32, A = B = format code `fmt` (kind::f16: 1 bfloat16, 0 binary16;
+// kind::tf32: 2; kind::f8f6f4: 0 = E4M3), both K-major, N = 256, M = 256 (128 rows per CTA).
 __device__ __forceinline__ uint32_t instr_desc_pair(uint32_t fmt) {
     return (1u << 4) | (fmt << 7) | (fmt << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
 }
@@ -129,6 +141,7 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 // blocks[i] = {X0, X1, Y0, Y1}: tile rows of the 256 x 256 block i, below the diagonal (X0 > Y1) or on it
 // (X = Y: the two diagonal tiles are stored with the triangle mask, the tile above the diagonal is
 // computed but not stored).  The pair with index p runs blocks p, p + pairs, p + 2 pairs, ...
+template <int kKind>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
                         const int4* __restrict__ blocks, int32_t n_blocks, int64_t N, int32_t n_ksteps,
@@ -146,6 +159,7 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     __shared__ volatile int s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr int kCols = kKind == 1 ? 32 : (kKind == 2 ? 128 : 64);   // columns of A in a 128-byte stage row
     const uint32_t rank = cluster_rank();                  // 0 = leader of the pair
     const int32_t pair_id = int32_t(blockIdx.x >> 1), n_pairs = int32_t(gridDim.x >> 1);
     // Units: (block, K-slice) pairs, slice-major (split == 1: the blocks themselves).  Unit w is block
@@ -186,8 +200,8 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     const uint32_t leader_full = map_to_cta(smem_u32(&full_bar[st]), 0);
                     remote_arrive_expect_tx(leader_full, uint32_t(kStageBytes));
                     uint8_t* dst = smem + st * kStageBytes;
-                    tma_load_2d_pair(dst, &tmA, ks * kBK, row_x, leader_full);
-                    tma_load_2d_pair(dst + kSegBytes, &tmA, ks * kBK, row_y, leader_full);
+                    tma_load_2d_pair(dst, &tmA, ks * kCols, row_x, leader_full);
+                    tma_load_2d_pair(dst + kSegBytes, &tmA, ks * kCols, row_y, leader_full);
                 }
             }
         }
@@ -217,8 +231,8 @@ syrk_pair_square_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     tc_fence_after();
                     const uint32_t a_lo = (smem_base + st * kStageBytes) >> 4, b_lo = a_lo + (kSegBytes >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < kBK / 16; ++kk)
-                        tc_mma_pair(d_addr, desc_hi | uint64_t(a_lo + 2 * kk), desc_hi | uint64_t(b_lo + 2 * kk), idesc,
+                    for (int kk = 0; kk < 4; ++kk)            // 32 bytes of K per instruction for every kind
+                        tc_mma_pair<kKind>(d_addr, desc_hi | uint64_t(a_lo + 2 * kk), desc_hi | uint64_t(b_lo + 2 * kk), idesc,
                                     (kk > 0 || ks > k0) ? 1u : 0u);
                     tc_commit_pair(&empty_bar[st]);          // both CTAs may refill the stage
                 }
@@ -370,29 +384,44 @@ pair_splitk_reduce_kernel(const int4* __restrict__ blocks, int32_t n_blocks, int
 
 }  // namespace pair
 
-cudaError_t launch_syrk_pair_square(const CUtensorMap& tmA, const CUtensorMap* tmC, const int4* d_blocks, int32_t n_blocks,
-                                    int64_t N, int64_t M, float* C, int64_t ldc, float alpha, float beta, int is_f16,
-                                    int* d_status, int sm_count, cudaStream_t stream, int split_k, float* d_partial) {
+namespace {
+template <int kKind>
+cudaError_t launch_pair_kind(const CUtensorMap& tmA, const CUtensorMap* tmC, const int4* d_blocks, int32_t n_blocks, int64_t N,
+                             int32_t n_ksteps, float* C, int64_t ldc, float alpha, float beta, int vec_ok, uint32_t fmt,
+                             int* d_status, int pairs, int split, float* d_partial, cudaStream_t stream) {
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(&pair::syrk_pair_square_kernel),
+        cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(&pair::syrk_pair_square_kernel<kKind>),
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, pair::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
+    CUtensorMap none{};
+    pair::syrk_pair_square_kernel<kKind><<<dim3(unsigned(2 * pairs)), pair::kThreads, pair::kSmemBytes, stream>>>(
+        tmA, tmC ? *tmC : none, d_blocks, n_blocks, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, fmt, d_status,
+        split, d_partial);
+    return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_syrk_pair_square(const CUtensorMap& tmA, const CUtensorMap* tmC, const int4* d_blocks, int32_t n_blocks,
+                                    int64_t N, int64_t M, float* C, int64_t ldc, float alpha, float beta, int a_kind,
+                                    int* d_status, int sm_count, cudaStream_t stream, int split_k, float* d_partial) {
     if (n_blocks <= 0) return cudaSuccess;
-    const int32_t n_ksteps = int32_t((M + pair::kBK - 1) / pair::kBK);
+    if (a_kind < 0 || a_kind > 3) return cudaErrorInvalidValue;
+    const int cols = a_kind == 1 ? 32 : (a_kind == 2 ? 128 : 64);
+    const int32_t n_ksteps = int32_t((M + cols - 1) / cols);
     const int split = (split_k < 1 || d_partial == nullptr) ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
     int pairs = sm_count / 2;
     if (int64_t(pairs) > int64_t(n_blocks) * split) pairs = n_blocks * split;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0) ? 1 : 0;
-    CUtensorMap none{};
-    pair::syrk_pair_square_kernel<<<dim3(unsigned(2 * pairs)), pair::kThreads, pair::kSmemBytes, stream>>>(
-        tmA, tmC ? *tmC : none, d_blocks, n_blocks, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0,
-        is_f16 ? 0u : 1u, d_status, split, d_partial);
-    cudaError_t e = cudaGetLastError();
+    const uint32_t fmt = a_kind == 0 ? 1u : (a_kind == 1 ? 2u : 0u);
+    cudaError_t e;
+    if (a_kind == 1) e = launch_pair_kind<1>(tmA, tmC, d_blocks, n_blocks, N, n_ksteps, C, ldc, alpha, beta, vec_ok, fmt, d_status, pairs, split, d_partial, stream);
+    else if (a_kind == 2) e = launch_pair_kind<2>(tmA, tmC, d_blocks, n_blocks, N, n_ksteps, C, ldc, alpha, beta, vec_ok, fmt, d_status, pairs, split, d_partial, stream);
+    else e = launch_pair_kind<0>(tmA, tmC, d_blocks, n_blocks, N, n_ksteps, C, ldc, alpha, beta, vec_ok, fmt, d_status, pairs, split, d_partial, stream);
     if (e != cudaSuccess || split == 1) return e;
     pair::pair_splitk_reduce_kernel<<<dim3(unsigned(n_blocks), 4), 256, 0, stream>>>(d_blocks, n_blocks, split, d_partial, N, C,
                                                                                      ldc, alpha, beta);
