@@ -76,9 +76,9 @@ extern "C" {
  *
  *   N, M     rows and columns of A; N == 0 returns at once.
  *   A        device pointer, row-major N x M, row pitch lda >= max(1, M) elements;
- *            read only.  binary64 for SYRK_DTYPE_F64, bfloat16 for SYRK_DTYPE_BF16_F32.
+ *            read only.  Element type as `dtype` says (binary64, bfloat16, binary32, FP8 bytes, binary16).
  *   C        device pointer, row-major N x N, row pitch ldc >= max(1, N) elements;
- *            binary64 / binary32 respectively.  Only j <= i is touched.  With
+ *            binary64 for SYRK_DTYPE_F64, binary32 for every other dtype.  Only j <= i is touched.  With
  *            beta == 0 the old C is not read (NaN or Inf there do not propagate).
  *   alpha, beta   scalars, passed through as given (non-finite values included).
  *            alpha == 0 or M == 0: the lower triangle becomes beta * C (zero when
