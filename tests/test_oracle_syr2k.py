@@ -15,6 +15,22 @@ def lower(x):
     return x[np.tril_indices(x.shape[0])]
 
 
+def test_hand_worked_example():
+    import os
+    rows = [l for l in open(os.path.join(os.path.dirname(__file__), "golden", "syr2k_3x2_by_hand.txt")) if not l.startswith("#")]
+    N, M = map(int, rows[0].split())
+    A = np.array([[float(v) for v in rows[1 + r].split()] for r in range(N)])
+    B = np.array([[float(v) for v in rows[1 + N + r].split()] for r in range(N)])
+    want = [[float(v) for v in rows[1 + 2 * N + r].split()] for r in range(N)]
+    ref, bound = R.syr2k_lower(A, B, None, 1.0, 0.0)
+    for i in range(N):
+        for j in range(i + 1):
+            assert ref[i, j] == want[i][j]
+    assert bound[2, 0] == 5 + 0 + 2 + 2 and bound[2, 2] == 2 * (10 + 6)      # the bound sums absolute products
+    ref, _ = R.syr2k_lower(A, B, np.ones((N, N)), 2.0, -3.0)                 # alpha = 2, beta = -3 on C = ones
+    assert ref[2, 1] == 2.0 * 8 - 3.0
+
+
 def test_b_equal_a_is_twice_the_syrk_reference():
     A = I.small_int_f64(23, 31, seed=1)                       # integers: every sum exact
     ref2, bd2 = R.syr2k_lower(A, A.copy(), None, 1.0, 0.0)
