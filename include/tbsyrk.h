@@ -312,6 +312,15 @@ int syrk_set_schedule(int schedule);
  */
 int syrk_probe_f64_mma_peak(int iters, double* tflops);
 
+/*
+ * Diagnostic, no counterpart in the paper: enqueues on `stream` a one-warp kernel that waits on a
+ * barrier nothing arrives on.  Every wait inside the library's kernels has a time limit (about two
+ * seconds); this call makes one run out on purpose, so that a caller (or a test) can see the whole
+ * path work: the kernel returns normally, and after the stream is synchronised syrk_last_status()
+ * reports SYRK_ERR_DEVICE_WAIT once, then SYRK_OK again; the context stays usable.
+ */
+int syrk_selftest_bounded_wait(void* stream);
+
 /* Force the number of K-slices (0 = automatic) used by later calls of every dtype. */
 int syrk_set_split_k(int slices);
 

@@ -28,7 +28,7 @@ MAX_SEG, MAX_TILE = 8, 16
 EXPORTS = [
     "syrk_lower", "syrk_lower_tn", "syrk_ex", "syr2k_lower", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_set_f64_launch", "syrk_get_schedule_stats",
-    "syrk_probe_f64_mma_peak", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
+    "syrk_probe_f64_mma_peak", "syrk_selftest_bounded_wait", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
     "tbs_plan_build", "tbs_plan_balance", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
 ]
 
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.syrk_get_schedule_stats.argtypes = [i64, i64, ci, ctypes.POINTER(ScheduleStats)]
         L.syrk_probe_f64_mma_peak.restype = ci
         L.syrk_probe_f64_mma_peak.argtypes = [ci, ctypes.POINTER(dbl)]
+        L.syrk_selftest_bounded_wait.restype = ci
+        L.syrk_selftest_bounded_wait.argtypes = [vp]
         L.syrk_lower_bf16_static.restype = ci
         L.syrk_lower_bf16_static.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
         L.cholesky_lower.restype = ci
@@ -234,6 +236,14 @@ def syrk_shutdown() -> None:
 
 def syrk_last_status(stream: Optional[int] = None) -> int:
     return int(lib().syrk_last_status(stream))
+
+
+def syrk_selftest_bounded_wait(stream: Optional[int] = None) -> None:
+    """Enqueue the kernel whose bounded wait runs out on purpose (about two seconds)."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().syrk_selftest_bounded_wait(stream))
 
 
 def syrk_set_schedule(schedule: int) -> None:

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 
 #include "../../include/tbsyrk.h"
+#include "device_utils.cuh"
+#include "runtime.h"
 
 namespace {
 
@@ -25,6 +27,22 @@ __global__ void __launch_bounds__(512) dmma_probe_kernel(double* out, int iters,
     for (int j = 0; j < 8; ++j)
         for (int i = 0; i < 4; ++i) s += c[j][i];
     out[blockIdx.x * blockDim.x + threadIdx.x] = s;
+}
+
+// Self-test of the bounded waits: one warp waits on an mbarrier that nothing ever arrives on.  The wait
+// gives up after its time limit (about two seconds), the kernel records the status bit and returns
+// normally, exactly as the SYRK kernels do when a pipeline stalls.
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(int* status) {
+    __shared__ uint64_t bar;
+    __shared__ volatile int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        tbsyrk::mbar_init(&bar, 1);
+        tbsyrk::mbar_fence_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0 && !tbsyrk::mbar_wait_bounded(&bar, 0, &abort_flag)) atomicOr(status, tbsyrk::kStatusWaitFull);
+    __syncwarp();
 }
 
 }  // namespace
@@ -62,4 +80,13 @@ extern "C" int syrk_probe_f64_mma_peak(int iters, double* tflops) {
     const double flops = double(blocks) * (threads / 32) * double(iters) * 8 * (2.0 * 16 * 8 * 8);
     *tflops = flops / (double(best) * 1e-3) * 1e-12;
     return SYRK_OK;
+}
+
+int syrk_selftest_bounded_wait(void* stream) {
+    std::lock_guard<std::mutex> lock(tbsyrk::runtime().mu);
+    tbsyrk::DeviceState* ds = nullptr;
+    int rc = tbsyrk::get_device_state(&ds);
+    if (rc != SYRK_OK) return rc;
+    bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ds->d_status);
+    return cudaGetLastError() == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
