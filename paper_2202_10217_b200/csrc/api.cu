@@ -34,7 +34,7 @@ bool tma_ok(const void* A, int64_t lda, int dtype) {
 // to min(units, SMs) thread blocks; with few items the inner dimension is cut so that every SM
 // has work.  The number of slices is the one with the smallest modelled makespan, in units of
 // one 128 x 128 x 64 tile step: a unit costs tiles x its K-steps plus about 20 per tile for the
-// write-out, and the reduction pass adds about 0.1 per partial tile.
+// write-out, and the reduction pass adds about 0.2 per partial tile.
 int auto_split_k(const std::vector<WorkItem>& items, int64_t M, int bk, int sm_count, int forced) {
     const int64_t ksteps = (M + bk - 1) / bk;
     if (forced > 0) return int(std::max<int64_t>(1, std::min<int64_t>(forced, ksteps)));
@@ -56,7 +56,7 @@ int auto_split_k(const std::vector<WorkItem>& items, int64_t M, int bk, int sm_c
             load[size_t(w % grid)] += double(it.n_tile) * double(kk + 20);
         }
         double cost = *std::max_element(load.begin(), load.end());
-        if (s > 1) cost += 0.1 * double(s) * double(total_tiles) + 40.0;
+        if (s > 1) cost += 0.2 * double(s) * double(total_tiles) + 40.0;
         if (s == 1 || cost < best_cost) { best = s; best_cost = cost; }
     }
     return best;
