@@ -209,7 +209,7 @@ def run_ours(args, wl: I.Workload, rank: int, world: int, local_rank: int):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > L2 (126 MB)
 
     if args.schedule != "tbs":                            # comparison schedules (kernel-only runs)
-        B.syrk_set_schedule({"square": B.SCHEDULE_SQUARE, "pair": B.SCHEDULE_PAIR_SQUARE}[args.schedule])
+        B.syrk_set_schedule({"square": B.SCHEDULE_SQUARE, "pair": B.SCHEDULE_PAIR_SQUARE, "auto": B.SCHEDULE_AUTO}[args.schedule])
     B.syrk_plan_prepare(N, M, dtype)
     stats = B.syrk_get_schedule_stats(N, M, dtype)
     n_warm = args.warmup if args.kernel_only else max(args.warmup, 3)
@@ -545,7 +545,7 @@ def main():
                     help="with --kernel-only: hand the operand over stored M x N and time syrk_lower_tn (C = A^T A)")
     ap.add_argument("--batch", type=int, default=0,
                     help="with --kernel-only: that many problems of the workload's shape through syrk_lower_batched")
-    ap.add_argument("--schedule", default="tbs", choices=["tbs", "square", "pair"],
+    ap.add_argument("--schedule", default="tbs", choices=["tbs", "square", "pair", "auto"],
                     help="with --kernel-only: the triangle-block schedule (default), the square-block comparison "
                          "schedule, or square blocks on CTA pairs (16-bit types)")
     ap.add_argument("--syr2k", action="store_true",

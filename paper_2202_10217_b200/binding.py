@@ -22,6 +22,7 @@ OP_N, OP_T = 0, 1
 SCHEDULE_TBS = 0
 SCHEDULE_SQUARE = 1
 SCHEDULE_PAIR_SQUARE = 2
+SCHEDULE_AUTO = 3
 ITEM_TRI, ITEM_RECT, ITEM_DIAG = 0, 1, 2
 MAX_SEG, MAX_TILE = 8, 16
 

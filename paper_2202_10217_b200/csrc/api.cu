@@ -191,7 +191,7 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
             if (sp == 1 || cost < best) { best = cost; split = sp; }
         }
     }
-    if (n_blk * split < pairs) return SYRK_ERR_PLAN;           // still too few units for the pairs
+    if (2 * n_blk * split < pairs) return SYRK_ERR_PLAN;       // still fewer units than half the pairs
     if (split > 1) {
         void* p = ds->d_partial;
         const int rc2 = ensure_device_bytes(&p, &ds->partial_bytes, size_t(split) * size_t(n_blk) * 4 * tile * tile * sizeof(float));
@@ -250,6 +250,13 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
     DevicePlan* dp = nullptr;
     rc = get_device_plan(ds, N, dtype, &dp, upper);
     if (rc != SYRK_OK) return rc;
+    // SYRK_SCHEDULE_AUTO: a triangle-block list shorter than the SM count fills the GPU only through a
+    // K-split of many short units; square blocks on CTA pairs (their own K-split) are the faster form there.
+    if (runtime().auto_pair && is_tcgen05_dtype(dtype) && !a_is_m_by_n && !upper &&
+        int64_t(dp->plan.items.size()) < int64_t(ds->sm_count)) {
+        rc = run_pair_square(ds, N, M, A, lda, C, ldc, alpha, beta, dtype, stream);
+        if (rc != SYRK_ERR_PLAN) return rc;
+    }
     const KernelShape ks = kernel_shape(dtype);
     CUtensorMap tm;
     // A stored M x N: boxes of one stage's k-rows x 128 bytes of columns (16 doubles, 64 bf16)
@@ -728,11 +735,13 @@ const char* syrk_strerror(int code) {
 }
 
 int syrk_set_schedule(int schedule) {
-    if (schedule != SYRK_SCHEDULE_TBS && schedule != SYRK_SCHEDULE_SQUARE && schedule != SYRK_SCHEDULE_PAIR_SQUARE)
+    if (schedule != SYRK_SCHEDULE_TBS && schedule != SYRK_SCHEDULE_SQUARE && schedule != SYRK_SCHEDULE_PAIR_SQUARE &&
+        schedule != SYRK_SCHEDULE_AUTO)
         return SYRK_ERR_PLAN;
     std::lock_guard<std::mutex> lock(runtime().mu);
     runtime().pair_square = schedule == SYRK_SCHEDULE_PAIR_SQUARE;
-    runtime().schedule = runtime().pair_square ? SYRK_SCHEDULE_SQUARE : schedule;
+    runtime().auto_pair = schedule == SYRK_SCHEDULE_AUTO;
+    runtime().schedule = runtime().pair_square ? SYRK_SCHEDULE_SQUARE : (runtime().auto_pair ? SYRK_SCHEDULE_TBS : schedule);
     return SYRK_OK;
 }
 

@@ -87,6 +87,7 @@ struct Runtime {
     std::map<int, DeviceState> devices;
     int schedule = 0;
     bool pair_square = false;   // SYRK_SCHEDULE_PAIR_SQUARE: square blocks, CTA-pair kernel where it applies
+    bool auto_pair = false;     // SYRK_SCHEDULE_AUTO: triangle blocks, but the pair kernel for short work lists
     int split_k = 0;
     int f64_launch = 0;
 };
