@@ -71,11 +71,11 @@ extern "C" {
                                       SYRK_SCHEDULE_SQUARE.  A second comparison schedule: the pair
                                       form does not fit triangle blocks.                          */
 #define SYRK_SCHEDULE_AUTO 3        /* triangle blocks, except that a tcgen05-type call (operand N x M,
-                                      lower triangle) whose triangle-block list is shorter than the
-                                      SM count - a small N with a long inner dimension - runs
-                                      SYRK_SCHEDULE_PAIR_SQUARE: there the list only fills the GPU as
-                                      many short K-slices, and the pair form is measured 1.3-1.4x
-                                      faster (2048 x 262144: 0.78 against 0.99 ms).               */
+                                      lower triangle) whose triangle-block list is shorter than four
+                                      times the SM count (N below about 7500) runs
+                                      SYRK_SCHEDULE_PAIR_SQUARE: such a list fills the GPU unevenly
+                                      or only as many short K-slices, and the pair form is measured
+                                      1.0-1.5x faster there (2048 x 262144: 0.78 against 0.99 ms).  */
 
 /*
  * The update itself (see the formula above).

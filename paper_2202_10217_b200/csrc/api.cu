@@ -250,10 +250,11 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
     DevicePlan* dp = nullptr;
     rc = get_device_plan(ds, N, dtype, &dp, upper);
     if (rc != SYRK_OK) return rc;
-    // SYRK_SCHEDULE_AUTO: a triangle-block list shorter than the SM count fills the GPU only through a
-    // K-split of many short units; square blocks on CTA pairs (their own K-split) are the faster form there.
+    // SYRK_SCHEDULE_AUTO: a triangle-block list shorter than a few rounds of SMs fills the GPU unevenly or
+    // only through a K-split of many short units; square blocks on CTA pairs (their own K-split, equal
+    // units) are the faster form there (measured 1.0-1.5x from 1024 to 7168 rows, never slower).
     if (runtime().auto_pair && is_tcgen05_dtype(dtype) && !a_is_m_by_n && !upper &&
-        int64_t(dp->plan.items.size()) < int64_t(ds->sm_count)) {
+        int64_t(dp->plan.items.size()) < 4 * int64_t(ds->sm_count)) {
         rc = run_pair_square(ds, N, M, A, lda, C, ldc, alpha, beta, dtype, stream);
         if (rc != SYRK_ERR_PLAN) return rc;
     }
