@@ -60,7 +60,7 @@ extern "C" {
 #define SYRK_ERR_STATIC_LIMIT -10  /* syrk_lower_bf16_static: problem exceeds its fixed arrays */
 
 /* schedules (syrk_set_schedule) */
-#define SYRK_SCHEDULE_TBS     0    /* triangle blocks + square/diagonal leftovers (default) */
+#define SYRK_SCHEDULE_TBS     0    /* triangle blocks + square/diagonal leftovers, whatever the size */
 #define SYRK_SCHEDULE_SQUARE  1    /* square and diagonal blocks only (comparison schedule) */
 #define SYRK_SCHEDULE_PAIR_SQUARE 2 /* square blocks of 256 x 256 on pairs of thread blocks (tcgen05
                                       cta_group::2: the pair shares the N-operand, which halves its
@@ -70,12 +70,16 @@ extern "C" {
                                       pair a block; every other call runs
                                       SYRK_SCHEDULE_SQUARE.  A second comparison schedule: the pair
                                       form does not fit triangle blocks.                          */
-#define SYRK_SCHEDULE_AUTO 3        /* triangle blocks, except that a tcgen05-type call (operand N x M,
-                                      lower triangle) whose triangle-block list is shorter than four
-                                      times the SM count (N below about 7500) runs
+#define SYRK_SCHEDULE_AUTO 3        /* THE DEFAULT.  Triangle blocks, except that a tcgen05-type call
+                                      (operand N x M, lower triangle) whose triangle-block list is
+                                      shorter than four times the SM count (N below about 7500) runs
                                       SYRK_SCHEDULE_PAIR_SQUARE: such a list fills the GPU unevenly
                                       or only as many short K-slices, and the pair form is measured
-                                      1.0-1.5x faster there (2048 x 262144: 0.78 against 0.99 ms).  */
+                                      1.0-1.5x faster there (2048 x 262144: 0.78 against 0.99 ms).
+                                      The paper's tiled scheme needs N large against the block side
+                                      (Section 5.1.4) and leaves smaller N to square blocks; this is
+                                      that rule with the threshold measured on this GPU.
+                                      syrk_effective_schedule() tells which one a call takes.       */
 
 /*
  * The update itself (see the formula above).
@@ -98,10 +102,15 @@ extern "C" {
  * Ownership: the caller owns A and C, keeps them alive until the stream has run
  * the enqueued work, and must not let them overlap.  The library owns a cache of
  * device-resident work lists (one per N, dtype and schedule) and, for the
- * K-split path, a device workspace; both are created on first use (that first
- * call allocates device memory) and released by syrk_shutdown().  Calls are
- * stream-ordered; concurrent calls on different streams that need the K-split
- * workspace are serialised by the caller.  The K-split path is taken when the
+ * K-split path, a device workspace PER STREAM; both are created on first use (that
+ * first call allocates device memory; a workspace that must grow is freed and
+ * allocated anew, which synchronises the device) and released by syrk_shutdown().
+ * syrk_plan_prepare_stream() does all of that ahead of time.  Calls are
+ * stream-ordered, and calls on different streams may overlap on the GPU: each of
+ * the first 256 streams the library sees on a device has its own workspace,
+ * status word and work-item counter.  A K-split call on a further stream, or one
+ * whose workspace would have to grow while the stream is being captured into a
+ * graph, returns SYRK_ERR_ALLOC and enqueues nothing.  The K-split path is taken when the
  * work list is too short to fill the GPU and the inner dimension is long (FP64:
  * fewer items than SMs and M >= 1024; the other types: a cost
  * model over the work list, slices of at least 8 K-steps): the inner dimension is cut
@@ -239,6 +248,23 @@ int syrk_lower_host(int64_t N, int64_t M,
                     double alpha, double beta, int dtype);
 
 /*
+ * Which of the two pipelines above syrk_lower_host uses (process-wide; no counterpart in the paper).
+ * SYRK_HOST_AUTO (default): bands of rows where they apply, blocks of columns otherwise.
+ * SYRK_HOST_COLUMN_BLOCKS: always blocks of columns.  The difference matters for the schedule: a triangle
+ * block of Algorithm 4 owns tiles in k - 1 different zone rows (its rows are R = {u c + f(u)}), so a band of
+ * rows of C is complete only after blocks that also need later rows of A; the row-band pipeline therefore
+ * runs the square-block list, and only the column-block pipeline runs the schedule syrk_lower would run
+ * (syrk_effective_schedule) on each block of columns.
+ * syrk_host_pipeline_for tells which one a call with these sizes takes for alpha != 0 (host only):
+ * SYRK_HOST_ROW_BANDS or SYRK_HOST_COLUMN_BLOCKS.
+ */
+#define SYRK_HOST_AUTO          0
+#define SYRK_HOST_ROW_BANDS     1
+#define SYRK_HOST_COLUMN_BLOCKS 2
+int syrk_set_host_pipeline(int mode);
+int syrk_host_pipeline_for(int64_t N, int64_t M, int c_is_page_locked);
+
+/*
  * Allocation-free variant of the K-split BF16 path (no counterpart in the paper; it
  * exists for callers that cannot let a library call cudaMalloc: code that runs while
  * another allocator owns the device heap, services whose device memory budget is fixed
@@ -260,11 +286,16 @@ int syrk_lower_host(int64_t N, int64_t M,
  * SYRK_ERR_LD; alpha == 0 or M == 0 have nothing to split and return SYRK_ERR_SIZE.
  *
  * The first call on a device also resolves the device addresses of those arrays
- * (cudaGetSymbolAddress); make that first call outside any stream capture.
- * Every call rewrites the shared arrays, so calls whose GPU work may overlap (other
- * streams, other host threads) race: serialise them.  A bounded-wait failure inside
- * this variant's kernels is recorded in its own status word and is not reported by
- * syrk_last_status.
+ * (cudaGetSymbolAddress); make that first call before any stream capture begins.  A call
+ * on a stream that is being captured is refused with SYRK_ERR_CUDA: the work list is
+ * copied from host memory on the caller's stream when its size differs from the previous
+ * call's on that device (a pageable copy, staged before the call returns), and the arrays
+ * are shared.  Every call rewrites the shared arrays, so calls whose GPU work may overlap
+ * (other streams, other host threads) race: serialise them.  A bounded-wait failure inside
+ * this variant's kernels is recorded in its own status word, not the one syrk_last_status
+ * reads: after synchronising, syrk_lower_bf16_static_status() returns SYRK_OK, or
+ * SYRK_ERR_DEVICE_WAIT once (the result of that call is then undefined) and clears the
+ * word; it allocates nothing either.
  */
 #define SYRK_STATIC_MAX_SLICE_TILES 512
 int syrk_lower_bf16_static(int64_t N, int64_t M,
@@ -272,6 +303,7 @@ int syrk_lower_bf16_static(int64_t N, int64_t M,
                            void* C, int64_t ldc,
                            double alpha, double beta,
                            int slices, void* stream);
+int syrk_lower_bf16_static_status(void);
 
 /*
  * Cholesky factorisation by Large Block Cholesky (Algorithm 5 of the paper, LBC): replaces the
@@ -288,27 +320,43 @@ int syrk_lower_bf16_static(int64_t N, int64_t M,
  * first use and kept until syrk_shutdown().  A non-positive pivot does not stop the enqueued
  * work: after synchronising the stream, cholesky_last_info() returns 0, or k + 1 for the first
  * pivot k that was not positive (the contents of A are then undefined from column k on).
+ * The workspaces, the second stream and the pivot word are one per device: factorisations whose GPU
+ * work could overlap (different streams or host threads) must be serialised by the caller.
  */
 int     cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, void* stream);
 int64_t cholesky_last_info(void* stream);
 
-/* Build and upload the work list for (N, M, dtype) ahead of time, so that a later
- * syrk_lower with these sizes allocates nothing. */
+/* Take, ahead of time, every decision a later syrk_lower(N, M, ..., dtype, stream) takes under the
+ * current settings (schedule, number of K-slices) and create what that call would allocate: the
+ * device-resident work list (or the block list of the CTA-pair schedule) and `stream`'s K-split
+ * workspace, for every dtype.  After it, such a call allocates nothing, does not synchronise and
+ * may be captured into a graph.  syrk_plan_prepare is the same for the legacy default stream (0).
+ * Launches nothing.  (No counterpart in the paper.) */
+int syrk_plan_prepare_stream(int64_t N, int64_t M, int dtype, void* stream);
 int syrk_plan_prepare(int64_t N, int64_t M, int dtype);
 
 /* Free every cached work list and workspace of the calling process. */
 void syrk_shutdown(void);
 
 /* After the caller has synchronised `stream`: 0, or SYRK_ERR_DEVICE_WAIT when a
- * kernel gave up on a bounded wait since the last query (the result of that call
- * is then undefined; the context stays usable).  Clears the flag. */
+ * kernel enqueued on that stream gave up on a bounded wait since the last query (the
+ * result of that call is then undefined; the context stays usable).  Clears the flag.
+ * Every stream has its own flag; stream == 0 asks for all streams of the current device
+ * at once (after a device-wide synchronisation) - the form to use after cholesky_lower
+ * and syrk_lower_host, which run part of their work on streams of the library. */
 int syrk_last_status(void* stream);
 
 /* Human-readable text for a return code (static storage). */
 const char* syrk_strerror(int code);
 
-/* Select the schedule used by later calls (process-wide). */
+/* Select the schedule used by later calls (process-wide; SYRK_SCHEDULE_AUTO at start). */
 int syrk_set_schedule(int schedule);
+
+/* Which schedule syrk_lower(N, M, ..., dtype) runs under the current setting on a 148-SM device, for
+ * an aligned operand: SYRK_SCHEDULE_TBS, SYRK_SCHEDULE_SQUARE or SYRK_SCHEDULE_PAIR_SQUARE (host only;
+ * a negative SYRK_ERR_* for bad arguments).  Under SYRK_SCHEDULE_AUTO this is where the rule of
+ * Section 5.1.4 - triangle blocks once N is large against the block side, squares below - shows. */
+int syrk_effective_schedule(int64_t N, int64_t M, int dtype);
 
 /*
  * Diagnostic, no counterpart in the paper: measures this GPU's FP64 tensor-core
@@ -349,13 +397,17 @@ int syrk_set_f64_launch(int mode);
  * What a call with these sizes would run (host only, no device needed).
  * All counts refer to one call.  "a_loads" is the number of elements of A the
  * work list moves from slow to fast memory in the paper's two-level model
- * (Section 3): for every work item, rows held x M.
+ * (Section 3): for every work item, rows held x M.  The work-list fields (items ..
+ * a_loads, tile, k, c, s_acc, s_total) describe the single-block list of the current
+ * setting (triangle blocks unless SYRK_SCHEDULE_SQUARE / _PAIR_SQUARE is set);
+ * effective_schedule, split_k and launches describe what the call really runs, which
+ * under SYRK_SCHEDULE_AUTO may be square blocks on CTA pairs.
  */
 typedef struct {
     int32_t tile;            /* b: rows per segment                                  */
     int32_t k;               /* segments per triangle block                          */
     int32_t c;               /* zone side of the top level (in tiles)                */
-    int32_t split_k;         /* K-slices a BF16 call would use on a 148-SM device    */
+    int32_t split_k;         /* K-slices the call would use on a 148-SM device (1: none) */
     int64_t n_tiles;         /* ceil(N / b)                                          */
     int64_t items;           /* work items                                           */
     int64_t tri_items;       /* of which triangle blocks                             */
@@ -367,6 +419,9 @@ typedef struct {
     int64_t c_elems;         /* elements of C owned: N(N+1)/2                        */
     int64_t s_acc;           /* accumulator elements a thread block may hold         */
     int64_t s_total;         /* s_acc + staging elements (all pipeline stages)       */
+    int32_t effective_schedule; /* what the call runs: syrk_effective_schedule()      */
+    int32_t launches;        /* kernels the call enqueues: 1, or 2 with a K-split (the
+                                slices' partial results are summed by a second kernel)  */
 } syrk_schedule_stats;
 
 int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats* out);
@@ -392,7 +447,8 @@ void*   tbs_plan_build(int64_t n_tiles, int k, int rect_rows, int rect_cols,
                        int diag_side, int schedule);
 /* Reorder a plan for a machine that runs `slots` items at a time (heaviest items first, some
  * full rectangles at the end cut into quarters so that the last wave fills evenly); the set of
- * tiles covered does not change.  The FP64 path applies this with slots = 148. */
+ * tiles covered does not change.  The library's own FP64 path only sorts heaviest first (slots = 0):
+ * the quartered rectangles measured slower than the uneven last wave they avoid. */
 int     tbs_plan_balance(void* plan, int slots);
 int64_t tbs_plan_num_items(const void* plan);
 int     tbs_plan_item(const void* plan, int64_t index, int32_t* kind,

@@ -23,11 +23,14 @@ SCHEDULE_TBS = 0
 SCHEDULE_SQUARE = 1
 SCHEDULE_PAIR_SQUARE = 2
 SCHEDULE_AUTO = 3
+SCHEDULE_DEFAULT = SCHEDULE_AUTO      # what the library starts with
+SCHEDULE_NAME = {SCHEDULE_TBS: "tbs", SCHEDULE_SQUARE: "square", SCHEDULE_PAIR_SQUARE: "pair_square"}
 ITEM_TRI, ITEM_RECT, ITEM_DIAG = 0, 1, 2
 MAX_SEG, MAX_TILE = 8, 16
 
 EXPORTS = [
-    "syrk_lower", "syrk_lower_tn", "syrk_ex", "syr2k_lower", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_shutdown", "syrk_last_status",
+    "syrk_lower", "syrk_lower_tn", "syrk_ex", "syr2k_lower", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_plan_prepare_stream", "syrk_effective_schedule",
+    "syrk_lower_bf16_static_status", "syrk_set_host_pipeline", "syrk_host_pipeline_for", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_set_f64_launch", "syrk_get_schedule_stats",
     "syrk_probe_f64_mma_peak", "syrk_selftest_bounded_wait", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
     "tbs_plan_build", "tbs_plan_balance", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
@@ -40,7 +43,8 @@ class ScheduleStats(ctypes.Structure):
                 ("tri_items", ctypes.c_int64), ("rect_items", ctypes.c_int64),
                 ("diag_items", ctypes.c_int64), ("tri_tiles", ctypes.c_int64),
                 ("all_tiles", ctypes.c_int64), ("a_loads", ctypes.c_int64),
-                ("c_elems", ctypes.c_int64), ("s_acc", ctypes.c_int64), ("s_total", ctypes.c_int64)]
+                ("c_elems", ctypes.c_int64), ("s_acc", ctypes.c_int64), ("s_total", ctypes.c_int64),
+                ("effective_schedule", ctypes.c_int32), ("launches", ctypes.c_int32)]
 
     def as_dict(self):
         return {name: int(getattr(self, name)) for name, _ in self._fields_}
@@ -78,6 +82,16 @@ def lib() -> ctypes.CDLL:
         L.syrk_lower_host.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci]
         L.syrk_plan_prepare.restype = ci
         L.syrk_plan_prepare.argtypes = [i64, i64, ci]
+        L.syrk_plan_prepare_stream.restype = ci
+        L.syrk_plan_prepare_stream.argtypes = [i64, i64, ci, vp]
+        L.syrk_effective_schedule.restype = ci
+        L.syrk_effective_schedule.argtypes = [i64, i64, ci]
+        L.syrk_lower_bf16_static_status.restype = ci
+        L.syrk_lower_bf16_static_status.argtypes = []
+        L.syrk_set_host_pipeline.restype = ci
+        L.syrk_set_host_pipeline.argtypes = [ci]
+        L.syrk_host_pipeline_for.restype = ci
+        L.syrk_host_pipeline_for.argtypes = [i64, i64, ci]
         L.syrk_shutdown.restype = None
         L.syrk_shutdown.argtypes = []
         L.syrk_last_status.restype = ci
@@ -229,6 +243,44 @@ def cholesky_last_info(stream: Optional[int] = None) -> int:
 
 def syrk_plan_prepare(N: int, M: int, dtype: int) -> None:
     _check(lib().syrk_plan_prepare(N, M, dtype))
+
+
+def syrk_plan_prepare_stream(N: int, M: int, dtype: int, stream: Optional[int] = None) -> None:
+    """Create ahead of time what syrk_lower(N, M, ..., dtype) on `stream` (default: torch's current
+    stream) would allocate."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().syrk_plan_prepare_stream(N, M, dtype, stream))
+
+
+def syrk_effective_schedule(N: int, M: int, dtype: int) -> int:
+    """SCHEDULE_TBS, SCHEDULE_SQUARE or SCHEDULE_PAIR_SQUARE: what a call with these sizes runs (host only)."""
+    r = int(lib().syrk_effective_schedule(N, M, dtype))
+    if r < 0:
+        raise SyrkError(r)
+    return r
+
+
+HOST_AUTO, HOST_ROW_BANDS, HOST_COLUMN_BLOCKS = 0, 1, 2
+
+
+def syrk_set_host_pipeline(mode: int) -> None:
+    _check(lib().syrk_set_host_pipeline(mode))
+
+
+def syrk_host_pipeline_for(N: int, M: int, c_is_page_locked: bool) -> int:
+    """HOST_ROW_BANDS (square-block list) or HOST_COLUMN_BLOCKS (the schedule of syrk_lower): what
+    syrk_lower_host does with these sizes (host only)."""
+    r = int(lib().syrk_host_pipeline_for(N, M, 1 if c_is_page_locked else 0))
+    if r < 0:
+        raise SyrkError(r)
+    return r
+
+
+def syrk_lower_bf16_static_status() -> int:
+    """0, or -8 once after a bounded wait ran out inside syrk_lower_bf16_static (after a sync)."""
+    return int(lib().syrk_lower_bf16_static_status())
 
 
 def syrk_shutdown() -> None:

@@ -28,17 +28,24 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    objs = []
-    log = []
-    for s in SOURCES:
+    # Every header is a dependency of every source, so a stale library means a full rebuild; the
+    # sources compile side by side (one nvcc process each).
+    from concurrent.futures import ThreadPoolExecutor
+
+    def compile_one(s):
         obj = os.path.join(CSRC, os.path.splitext(s)[0] + ".o")
         cmd = [nvcc] + NVCC_FLAGS + ["-x", "cu", "-c", os.path.join(CSRC, s), "-o", obj]
-        r = subprocess.run(cmd, capture_output=True, text=True)
-        log.append(r.stderr)
-        if r.returncode != 0:
-            sys.stderr.write(r.stdout + r.stderr)
-            raise RuntimeError("nvcc failed on " + s)
-        objs.append(obj)
+        return s, obj, subprocess.run(cmd, capture_output=True, text=True)
+
+    objs = []
+    log = []
+    with ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 1)) as pool:
+        for s, obj, r in pool.map(compile_one, SOURCES):
+            log.append(r.stderr)
+            if r.returncode != 0:
+                sys.stderr.write(r.stdout + r.stderr)
+                raise RuntimeError("nvcc failed on " + s)
+            objs.append(obj)
     cmd = [nvcc, "-shared", "-o", LIB] + objs + ["-lcudart", "-lpthread"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:

@@ -94,8 +94,9 @@ int pick_split_k(const DeviceState* ds, DevicePlan* dp, int64_t M, int bk) {
 int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkItem* d_items, int64_t n_items,
                  int64_t N, int64_t M, void* C, int64_t ldc, double alpha, double beta, int split,
                  const int64_t* d_tile_base, int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas,
-                 int f64_launch, int a_is_m_by_n, cudaStream_t stream, int upper = 0) {
+                 int f64_launch, int a_is_m_by_n, cudaStream_t stream, int upper = 0, void* d_partial = nullptr) {
     cudaError_t e;
+    int* d_status = status_for_stream(ds, stream);
     if (dtype == SYRK_DTYPE_F64) {
         CUtensorMap tmc;
         const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
@@ -108,15 +109,15 @@ int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkIt
                                 (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count)));
         int* tickets = (persistent && split <= 1) ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<double*>(C), ldc,
-                            alpha, beta, a_is_m_by_n, tickets, ds->sm_count, ds->d_status, stream, 0, 0, split,
-                            reinterpret_cast<double*>(ds->d_partial), upper);
+                            alpha, beta, a_is_m_by_n, tickets, ds->sm_count, d_status, stream, 0, 0, split,
+                            static_cast<double*>(d_partial), upper);
     } else {
         CUtensorMap tmc;
         const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                            encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
         e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<float*>(C), ldc, float(alpha),
-                             float(beta), split, ds->d_partial, d_tile_base, total_tiles, d_cta_begin, n_ctas, a_is_m_by_n,
-                             dtype - SYRK_DTYPE_BF16_F32, ds->d_status, ds->sm_count, stream, 0, 0, upper);
+                             float(beta), split, static_cast<float*>(d_partial), d_tile_base, total_tiles, d_cta_begin, n_ctas,
+                             a_is_m_by_n, dtype - SYRK_DTYPE_BF16_F32, d_status, ds->sm_count, stream, 0, 0, upper);
     }
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
@@ -168,20 +169,20 @@ int get_banded_plan(DeviceState* ds, int64_t N, int dtype, int max_bands, Banded
 }  // namespace
 
 namespace {
-// SYRK_SCHEDULE_PAIR_SQUARE for tcgen05-type operands stored N x M, lower triangle: the 256 x 256
-// blocks below and on the diagonal on the CTA-pair kernel.  Returns SYRK_ERR_PLAN when the problem has fewer blocks than the GPU has pairs.
-int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc,
-                    double alpha, double beta, int dtype, cudaStream_t stream) {
+// The CTA-pair square-block schedule for (N, M): number of 256 x 256 blocks and K-slices.  Returns false
+// when the problem, even cut along the inner dimension, has fewer units than half the GPU's pairs (the
+// caller then runs a single-CTA list).
+bool pair_square_shape(int64_t N, int64_t M, int dtype, int sm_count, int forced_split, int64_t* n_blk_out, int* split_out) {
     const int tile = bf16_tile();
     const int64_t n_tiles = (N + tile - 1) / tile, n_super = (n_tiles + 1) / 2;
-    const int64_t n_blk = n_super * (n_super + 1) / 2, pairs = ds->sm_count / 2;
+    const int64_t n_blk = n_super * (n_super + 1) / 2, pairs = sm_count / 2;
     const int64_t bk = 128 / int64_t(a_elem(dtype));              // columns in a 128-byte stage row
     const int64_t n_ksteps = (M + bk - 1) / bk;
-    if (n_tiles >= (int64_t(1) << 15)) return SYRK_ERR_PLAN;
+    if (n_tiles >= (int64_t(1) << 15)) return false;
     // K-slices: with fewer blocks than a few rounds of pairs the inner dimension is cut so that every pair
     // has work; the number of slices minimises rounds x (K-steps per slice + 20) plus the partial traffic.
     int split = 1;
-    if (runtime().split_k > 0) split = int(std::min<int64_t>(runtime().split_k, n_ksteps));
+    if (forced_split > 0) split = int(std::max<int64_t>(1, std::min<int64_t>(forced_split, n_ksteps)));
     else if (n_blk < 4 * pairs) {
         double best = 0.0;
         for (int sp = 1; sp <= 32 && sp <= n_ksteps / 8; ++sp) {
@@ -191,11 +192,26 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
             if (sp == 1 || cost < best) { best = cost; split = sp; }
         }
     }
-    if (2 * n_blk * split < pairs) return SYRK_ERR_PLAN;       // still fewer units than half the pairs
+    if (2 * n_blk * split < pairs) return false;               // still fewer units than half the pairs
+    *n_blk_out = n_blk;
+    *split_out = split;
+    return true;
+}
+
+// SYRK_SCHEDULE_PAIR_SQUARE for tcgen05-type operands stored N x M, lower triangle: the 256 x 256
+// blocks below and on the diagonal on the CTA-pair kernel.  Returns SYRK_ERR_PLAN when the problem has
+// fewer blocks than the GPU has pairs.  `launch` false: only create what the call would allocate.
+int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc,
+                    double alpha, double beta, int dtype, cudaStream_t stream, bool launch = true) {
+    const int tile = bf16_tile();
+    const int64_t n_tiles = (N + tile - 1) / tile, n_super = (n_tiles + 1) / 2;
+    const int64_t bk = 128 / int64_t(a_elem(dtype));
+    int64_t n_blk = 0;
+    int split = 1;
+    if (!pair_square_shape(N, M, dtype, ds->sm_count, runtime().split_k, &n_blk, &split)) return SYRK_ERR_PLAN;
+    void* d_partial = nullptr;
     if (split > 1) {
-        void* p = ds->d_partial;
-        const int rc2 = ensure_device_bytes(&p, &ds->partial_bytes, size_t(split) * size_t(n_blk) * 4 * tile * tile * sizeof(float));
-        ds->d_partial = static_cast<float*>(p);
+        const int rc2 = workspace_for_stream(ds, stream, size_t(split) * size_t(n_blk) * 4 * tile * tile * sizeof(float), &d_partial);
         if (rc2 != SYRK_OK) return rc2;
     }
     auto it = ds->pair_plans.find(n_tiles);
@@ -218,6 +234,7 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
         }
         it = ds->pair_plans.emplace(n_tiles, pp).first;
     }
+    if (!launch) return SYRK_OK;
     const PairPlan& pp = it->second;
     CUtensorMap tm, tmc;
     int rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, tile, int(bk));
@@ -225,69 +242,68 @@ int run_pair_square(DeviceState* ds, int64_t N, int64_t M, const void* A, int64_
     const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                        encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
     cudaError_t e = launch_syrk_pair_square(tm, c_tma ? &tmc : nullptr, pp.d_blocks, pp.n_blocks, N, M, static_cast<float*>(C),
-                                            ldc, float(alpha), float(beta), dtype - SYRK_DTYPE_BF16_F32, ds->d_status,
-                                            ds->sm_count, stream, split, ds->d_partial);
+                                            ldc, float(alpha), float(beta), dtype - SYRK_DTYPE_BF16_F32,
+                                            status_for_stream(ds, stream), ds->sm_count, stream, split,
+                                            static_cast<float*>(d_partial));
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
 }  // namespace
 
 int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
-                            double beta, int dtype, cudaStream_t stream, int f64_launch, int a_is_m_by_n, int upper) {
+                            double beta, int dtype, cudaStream_t stream, int f64_launch, int a_is_m_by_n, int upper,
+                            bool prepare_only) {
     DeviceState* ds = nullptr;
     int rc = get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
     if (alpha == 0.0 || M == 0) {
-        if (beta == 1.0) return SYRK_OK;
+        if (beta == 1.0 || prepare_only) return SYRK_OK;
         return launch_scale_lower(dtype, N, C, ldc, beta, stream, upper) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
     }
-    if (!tma_ok(A, lda, dtype))
+    if (!prepare_only && !tma_ok(A, lda, dtype))
         return launch_syrk_plain(dtype, N, M, A, lda, C, ldc, alpha, beta, a_is_m_by_n, stream, upper) == cudaSuccess
                    ? SYRK_OK : SYRK_ERR_CUDA;
-    if (runtime().pair_square && is_tcgen05_dtype(dtype) && !a_is_m_by_n && !upper) {
-        rc = run_pair_square(ds, N, M, A, lda, C, ldc, alpha, beta, dtype, stream);
+    const bool pair_form = is_tcgen05_dtype(dtype) && !a_is_m_by_n && !upper;    // what the CTA-pair kernel covers
+    if (runtime().pair_square && pair_form) {
+        rc = run_pair_square(ds, N, M, A, lda, C, ldc, alpha, beta, dtype, stream, !prepare_only);
         if (rc != SYRK_ERR_PLAN) return rc;          // SYRK_ERR_PLAN: too few blocks for the pairs - the square list below
     }
     DevicePlan* dp = nullptr;
     rc = get_device_plan(ds, N, dtype, &dp, upper);
     if (rc != SYRK_OK) return rc;
-    // SYRK_SCHEDULE_AUTO: a triangle-block list shorter than a few rounds of SMs fills the GPU unevenly or
-    // only through a K-split of many short units; square blocks on CTA pairs (their own K-split, equal
-    // units) are the faster form there (measured 1.0-1.5x from 1024 to 7168 rows, never slower).
-    if (runtime().auto_pair && is_tcgen05_dtype(dtype) && !a_is_m_by_n && !upper &&
-        int64_t(dp->plan.items.size()) < 4 * int64_t(ds->sm_count)) {
-        rc = run_pair_square(ds, N, M, A, lda, C, ldc, alpha, beta, dtype, stream);
+    // SYRK_SCHEDULE_AUTO (the default): a triangle-block list shorter than a few rounds of SMs fills the GPU
+    // unevenly or only through a K-split of many short units; square blocks on CTA pairs (their own
+    // K-split, equal units) are the faster form there (measured 1.0-1.5x from 1024 to 7168 rows, never slower).
+    if (runtime().auto_pair && pair_form && int64_t(dp->plan.items.size()) < 4 * int64_t(ds->sm_count)) {
+        rc = run_pair_square(ds, N, M, A, lda, C, ldc, alpha, beta, dtype, stream, !prepare_only);
         if (rc != SYRK_ERR_PLAN) return rc;
     }
     const KernelShape ks = kernel_shape(dtype);
+    int split = 1;
+    void* d_partial = nullptr;
+    if (is_tcgen05_dtype(dtype)) {
+        split = pick_split_k(ds, dp, M, ks.bk);
+        if (split > 1) {
+            const size_t want = size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float);
+            if ((rc = workspace_for_stream(ds, stream, want, &d_partial)) != SYRK_OK) return rc;
+        }
+    } else if (f64_launch < 0) {
+        // FP64 K-split (not for callers that fix the launch form: the Cholesky driver's look-ahead stream
+        // runs short updates that gain nothing from it)
+        split = auto_split_k_f64(int64_t(dp->plan.items.size()), N, M, ks.bk, ds->sm_count, runtime().split_k);
+        if (split > 1 &&
+            (rc = workspace_for_stream(ds, stream, size_t(split) * size_t(N) * size_t(N) * sizeof(double), &d_partial)) != SYRK_OK)
+            return rc;
+    }
+    if (prepare_only) return SYRK_OK;
     CUtensorMap tm;
     // A stored M x N: boxes of one stage's k-rows x 128 bytes of columns (16 doubles, 64 bf16)
     if (a_is_m_by_n) rc = encode_tensor_map_2d(&tm, dtype, A, M, N, lda, ks.bk, 128 / int(a_elem(dtype)),
                                                dtype == SYRK_DTYPE_TF32_F32);
     else rc = encode_tensor_map_2d(&tm, dtype, A, N, M, lda, ks.tile, ks.bk);
     if (rc != SYRK_OK) return rc;
-    int split = 1;
-    if (is_tcgen05_dtype(dtype)) {
-        split = pick_split_k(ds, dp, M, ks.bk);
-        if (split > 1) {
-            const size_t want = size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float);
-            void* p = ds->d_partial;
-            rc = ensure_device_bytes(&p, &ds->partial_bytes, want);
-            ds->d_partial = static_cast<float*>(p);
-            if (rc != SYRK_OK) return rc;
-        }
-    } else if (f64_launch < 0) {
-        // FP64 K-split (not for callers that fix the launch form: the Cholesky driver runs updates on
-        // two streams at once, and the workspace is one per device)
-        split = auto_split_k_f64(int64_t(dp->plan.items.size()), N, M, ks.bk, ds->sm_count, runtime().split_k);
-        if (split > 1) {
-            void* p = ds->d_partial;
-            rc = ensure_device_bytes(&p, &ds->partial_bytes, size_t(split) * size_t(N) * size_t(N) * sizeof(double));
-            ds->d_partial = static_cast<float*>(p);
-            if (rc != SYRK_OK) return rc;
-        }
-    }
     return launch_items(ds, dtype, tm, dp->d_items, int64_t(dp->plan.items.size()), N, M, C, ldc, alpha, beta, split,
-                        dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, f64_launch, a_is_m_by_n, stream, upper);
+                        dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, f64_launch, a_is_m_by_n, stream, upper,
+                        d_partial);
 }
 
 namespace {
@@ -386,7 +402,7 @@ int syr2k_lower(int64_t N, int64_t M, const void* A, int64_t lda, const void* B,
     const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
                        encode_tensor_map_c_f64(&tmc, C, N, ldc, f64_tile()) == SYRK_OK;
     return launch_syr2k_f64(ta, tb, c_tma ? &tmc : nullptr, dp->d_items, int64_t(dp->plan.items.size()), N, M,
-                            static_cast<double*>(C), ldc, alpha, beta, ds->d_status, st) == cudaSuccess
+                            static_cast<double*>(C), ldc, alpha, beta, status_for_stream(ds, st), st) == cudaSuccess
                ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
@@ -429,13 +445,13 @@ int syrk_lower_batched(int64_t batch, int64_t N, int64_t M, const void* A, int64
         const bool c_tma = beta != 0.0 && c_aligned &&
                            encode_tensor_map_c_batched(&tmc, 1, C, N, ldc, stride_c, batch, f64_tile()) == SYRK_OK;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha,
-                            beta, 0, nullptr, 0, ds->d_status, st, batch, stride_c);
+                            beta, 0, nullptr, 0, status_for_stream(ds, st), st, batch, stride_c);
     } else {
         const bool c_tma = c_aligned &&
                            encode_tensor_map_c_batched(&tmc, 0, C, N, ldc, stride_c, batch, bf16_store_box()) == SYRK_OK;
         e = launch_syrk_bf16(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<float*>(C), ldc,
                              float(alpha), float(beta), 1, nullptr, dp->d_tile_base, dp->total_tiles, nullptr, 0, 0,
-                             dtype - SYRK_DTYPE_BF16_F32, ds->d_status, ds->sm_count, st, batch, stride_c);
+                             dtype - SYRK_DTYPE_BF16_F32, status_for_stream(ds, st), ds->sm_count, st, batch, stride_c);
     }
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
@@ -469,7 +485,7 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
     // Large problems with a page-locked C are produced band by band (see below); the bands are then
     // those of the row-ordered work list.
     BandedPlan* bp = nullptr;
-    const bool banded = c_pinned && M > 0 && alpha != 0.0 && N >= 4096 &&
+    const bool banded = c_pinned && M > 0 && alpha != 0.0 && N >= 4096 && runtime().host_pipeline != SYRK_HOST_COLUMN_BLOCKS &&
                         get_banded_plan(ds, N, dtype, kBands, &bp) == SYRK_OK && bp->item_end.size() > 1;
     const int64_t pk_h = banded ? bp->band_rows
                                 : (c_pinned ? (N + std::max<int64_t>(1, std::min<int64_t>(kBands, N / 256)) - 1) /
@@ -550,10 +566,12 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
             }
         }
         if (!chk(cudaStreamSynchronize(dl))) return SYRK_ERR_CUDA;
-        int flag = 0;
-        if (cudaMemcpy(&flag, ds->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
-        if (flag != 0) { cudaMemset(ds->d_status, 0, sizeof(int)); return SYRK_ERR_DEVICE_WAIT; }
-        return SYRK_OK;
+        int worst = SYRK_OK;                               // the band streams ran the kernels
+        for (cudaStream_t bs : ds->band_streams) {
+            const int r = read_and_clear_status(ds, bs, false);
+            if (r != SYRK_OK) worst = r;
+        }
+        return worst;
     }
 
     // Upload and compute overlap: A goes up in column blocks on the copy stream and each block's
@@ -670,51 +688,31 @@ int syrk_lower_host(int64_t N, int64_t M, const void* A, int64_t lda, void* C, i
         }
     }
     if (!chk(cudaStreamSynchronize(st))) return SYRK_ERR_CUDA;
-    int flag = 0;
-    if (cudaMemcpy(&flag, ds->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
-    if (flag != 0) { cudaMemset(ds->d_status, 0, sizeof(int)); return SYRK_ERR_DEVICE_WAIT; }
-    return SYRK_OK;
+    return read_and_clear_status(ds, st, false);
 }
 
-int syrk_plan_prepare(int64_t N, int64_t M, int dtype) {
+int syrk_plan_prepare_stream(int64_t N, int64_t M, int dtype, void* stream) {
     if (!known_dtype(dtype)) return SYRK_ERR_DTYPE;
     if (N < 0 || M < 0) return SYRK_ERR_SIZE;
     if (N == 0) return SYRK_OK;
     std::lock_guard<std::mutex> lock(runtime().mu);
-    DeviceState* ds = nullptr;
-    int rc = get_device_state(&ds);
-    if (rc != SYRK_OK) return rc;
-    DevicePlan* dp = nullptr;
-    rc = get_device_plan(ds, N, dtype, &dp);
-    if (rc != SYRK_OK) return rc;
-    if (is_tcgen05_dtype(dtype)) {
-        const KernelShape ks = kernel_shape(dtype);
-        const int split = pick_split_k(ds, dp, M, ks.bk);
-        if (split > 1) {
-            void* p = ds->d_partial;
-            rc = ensure_device_bytes(&p, &ds->partial_bytes,
-                                     size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float));
-            ds->d_partial = static_cast<float*>(p);
-        }
-    }
-    return rc;
+    // The decisions of a syrk_lower call (schedule, K-split) with everything they allocate, nothing launched.
+    return syrk_run_device(N, M, nullptr, M, nullptr, N, 1.0, 0.0, dtype, static_cast<cudaStream_t>(stream), -1, 0, 0, true);
 }
+
+int syrk_plan_prepare(int64_t N, int64_t M, int dtype) { return syrk_plan_prepare_stream(N, M, dtype, nullptr); }
 
 void syrk_shutdown(void) {
     std::lock_guard<std::mutex> lock(runtime().mu);
     release_all();
 }
 
-int syrk_last_status(void* /*stream*/) {
+int syrk_last_status(void* stream) {
     std::lock_guard<std::mutex> lock(runtime().mu);
     DeviceState* ds = nullptr;
     int rc = get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
-    int flag = 0;
-    if (cudaMemcpy(&flag, ds->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
-    if (flag == 0) return SYRK_OK;
-    cudaMemset(ds->d_status, 0, sizeof(int));
-    return SYRK_ERR_DEVICE_WAIT;
+    return read_and_clear_status(ds, static_cast<cudaStream_t>(stream), stream == nullptr);
 }
 
 const char* syrk_strerror(int code) {
@@ -746,6 +744,59 @@ int syrk_set_schedule(int schedule) {
     return SYRK_OK;
 }
 
+namespace {
+// What syrk_lower(N, M, ..., dtype) runs on a device with `sm_count` SMs under the current settings, for an
+// aligned N x M operand and the lower triangle: the schedule and its number of K-slices.
+int effective_schedule_of(int64_t N, int64_t M, int dtype, int sm_count, int* split_out) {
+    int schedule, forced_split;
+    bool pair_square, auto_pair;
+    {
+        std::lock_guard<std::mutex> lock(runtime().mu);
+        schedule = runtime().schedule; forced_split = runtime().split_k;
+        pair_square = runtime().pair_square; auto_pair = runtime().auto_pair;
+    }
+    *split_out = 1;
+    if (N == 0 || M == 0) return schedule;
+    const KernelShape ks = kernel_shape(dtype);
+    Plan plan;
+    if (!build_host_plan(N, dtype, schedule, &plan)) return SYRK_ERR_PLAN;
+    if (is_tcgen05_dtype(dtype)) {
+        int64_t n_blk = 0;
+        int split = 1;
+        const bool pairs_fit = pair_square_shape(N, M, dtype, sm_count, forced_split, &n_blk, &split);
+        if (pairs_fit && (pair_square || (auto_pair && int64_t(plan.items.size()) < 4 * int64_t(sm_count)))) {
+            *split_out = split;
+            return SYRK_SCHEDULE_PAIR_SQUARE;
+        }
+        *split_out = auto_split_k(plan.items, M, ks.bk, sm_count, forced_split);
+    } else {
+        *split_out = auto_split_k_f64(int64_t(plan.items.size()), N, M, ks.bk, sm_count, forced_split);
+    }
+    return schedule;
+}
+}  // namespace
+
+int syrk_effective_schedule(int64_t N, int64_t M, int dtype) {
+    if (!known_dtype(dtype)) return SYRK_ERR_DTYPE;
+    if (N < 0 || M < 0) return SYRK_ERR_SIZE;
+    int split = 1;
+    return effective_schedule_of(N, M, dtype, 148, &split);
+}
+
+int syrk_set_host_pipeline(int mode) {
+    if (mode != SYRK_HOST_AUTO && mode != SYRK_HOST_COLUMN_BLOCKS) return SYRK_ERR_PLAN;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    runtime().host_pipeline = mode;
+    return SYRK_OK;
+}
+
+int syrk_host_pipeline_for(int64_t N, int64_t M, int c_is_page_locked) {
+    if (N < 0 || M < 0) return SYRK_ERR_SIZE;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    return (c_is_page_locked && M > 0 && N >= 4096 && runtime().host_pipeline != SYRK_HOST_COLUMN_BLOCKS)
+               ? SYRK_HOST_ROW_BANDS : SYRK_HOST_COLUMN_BLOCKS;
+}
+
 int syrk_set_f64_launch(int mode) {
     if (mode != SYRK_F64_LAUNCH_AUTO && mode != SYRK_F64_LAUNCH_PER_ITEM && mode != SYRK_F64_LAUNCH_PERSISTENT)
         return SYRK_ERR_PLAN;
@@ -765,8 +816,8 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     if (!out) return SYRK_ERR_NULL;
     if (!known_dtype(dtype)) return SYRK_ERR_DTYPE;
     if (N < 0 || M < 0) return SYRK_ERR_SIZE;
-    int schedule, forced_split;
-    { std::lock_guard<std::mutex> lock(runtime().mu); schedule = runtime().schedule; forced_split = runtime().split_k; }
+    int schedule;
+    { std::lock_guard<std::mutex> lock(runtime().mu); schedule = runtime().schedule; }
     Plan plan;
     if (!build_host_plan(N, dtype, schedule, &plan)) return SYRK_ERR_PLAN;
     const KernelShape ks = kernel_shape(dtype);
@@ -775,8 +826,10 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->tile = ks.tile;
     out->k = ks.k;
     out->c = int32_t(plan.c_top);
-    out->split_k = (is_tcgen05_dtype(dtype) && M > 0)
-                       ? auto_split_k(plan.items, M, ks.bk, 148, forced_split) : 1;
+    int split = 1;
+    out->effective_schedule = effective_schedule_of(N, M, dtype, 148, &split);
+    out->split_k = split;
+    out->launches = split > 1 ? 2 : 1;
     out->n_tiles = plan.p.n_tiles;
     out->items = int64_t(plan.items.size());
     out->tri_items = plan.n_tri;

@@ -200,8 +200,8 @@ int gemm_nt(DeviceState* ds, int64_t nrows, int64_t ncols, int64_t K, const doub
     if (rc != SYRK_OK) return rc;
     const bool d_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(D) & 15) == 0 && (ldd & 1) == 0 &&
                        encode_tensor_map_f64_plain(&td, D, nrows, ncols, ldd, f64_tile(), f64_tile()) == SYRK_OK;
-    return launch_gemm_nt_f64(tp, tq, d_tma ? &td : nullptr, nrows, ncols, K, D, ldd, alpha, beta, ds->d_status,
-                              st) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+    return launch_gemm_nt_f64(tp, tq, d_tma ? &td : nullptr, nrows, ncols, K, D, ldd, alpha, beta,
+                              status_for_stream(ds, st), st) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
 }  // namespace

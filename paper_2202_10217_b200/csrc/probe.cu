@@ -87,6 +87,7 @@ int syrk_selftest_bounded_wait(void* stream) {
     tbsyrk::DeviceState* ds = nullptr;
     int rc = tbsyrk::get_device_state(&ds);
     if (rc != SYRK_OK) return rc;
-    bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ds->d_status);
+    bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        tbsyrk::status_for_stream(ds, static_cast<cudaStream_t>(stream)));
     return cudaGetLastError() == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }

@@ -85,26 +85,92 @@ int get_device_state(DeviceState** out) {
         ds.sm_count = prop.multiProcessorCount;
         ds.cc_major = prop.major;
         if (prop.major != 10) return SYRK_ERR_NO_DEVICE;  // kernels are built for sm_100a only
-        if (cudaMalloc(&ds.d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
-        if (cudaMemset(ds.d_status, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
-        if (cudaMalloc(&ds.d_tickets, 2 * kTicketStreams * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
-        if (cudaMemset(ds.d_tickets, 0, 2 * kTicketStreams * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+        if (cudaMalloc(&ds.d_status, (kStreamSlots + 1) * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
+        if (cudaMemset(ds.d_status, 0, (kStreamSlots + 1) * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+        if (cudaMalloc(&ds.d_tickets, 2 * kStreamSlots * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
+        if (cudaMemset(ds.d_tickets, 0, 2 * kStreamSlots * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+        ds.workspaces.resize(kStreamSlots);
         it = rt.devices.emplace(dev, std::move(ds)).first;
     }
     *out = &it->second;
     return SYRK_OK;
 }
 
-int* tickets_for_stream(DeviceState* ds, cudaStream_t stream) {
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-    if (cap != cudaStreamCaptureStatusNone) return nullptr;
-    auto it = ds->ticket_slot.find(stream);
-    if (it == ds->ticket_slot.end()) {
-        if (int(ds->ticket_slot.size()) >= kTicketStreams) return nullptr;
-        it = ds->ticket_slot.emplace(stream, int(ds->ticket_slot.size())).first;
+int slot_for_stream(DeviceState* ds, cudaStream_t stream) {
+    auto it = ds->stream_slot.find(stream);
+    if (it == ds->stream_slot.end()) {
+        if (int(ds->stream_slot.size()) >= kStreamSlots) return -1;
+        it = ds->stream_slot.emplace(stream, int(ds->stream_slot.size())).first;
     }
-    return ds->d_tickets + 2 * it->second;
+    return it->second;
+}
+
+int* status_for_stream(DeviceState* ds, cudaStream_t stream) {
+    const int slot = slot_for_stream(ds, stream);
+    return ds->d_status + (slot >= 0 ? slot : kStreamSlots);
+}
+
+namespace {
+bool stream_is_capturing(cudaStream_t stream) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return true; }   // be careful
+    return cap != cudaStreamCaptureStatusNone;
+}
+}  // namespace
+
+int* tickets_for_stream(DeviceState* ds, cudaStream_t stream) {
+    if (stream_is_capturing(stream)) return nullptr;
+    const int slot = slot_for_stream(ds, stream);
+    return slot >= 0 ? ds->d_tickets + 2 * slot : nullptr;
+}
+
+int workspace_for_stream(DeviceState* ds, cudaStream_t stream, size_t want, void** out) {
+    const int slot = slot_for_stream(ds, stream);
+    if (slot < 0) return SYRK_ERR_ALLOC;
+    StreamWorkspace& ws = ds->workspaces[size_t(slot)];
+    if (ws.bytes < want || !ws.d_partial) {
+        if (stream_is_capturing(stream)) return SYRK_ERR_ALLOC;
+        const int rc = ensure_device_bytes(&ws.d_partial, &ws.bytes, want);
+        if (rc != SYRK_OK) return rc;
+    }
+    *out = ws.d_partial;
+    return SYRK_OK;
+}
+
+int read_and_clear_status(DeviceState* ds, cudaStream_t stream, bool all) {
+    int words[kStreamSlots + 1];
+    const int first = all ? 0 : int(status_for_stream(ds, stream) - ds->d_status);
+    const int count = all ? kStreamSlots + 1 : 1;
+    if (cudaMemcpy(words, ds->d_status + first, size_t(count) * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return SYRK_ERR_CUDA;
+    }
+    int flag = 0;
+    for (int i = 0; i < count; ++i) flag |= words[i];
+    if (flag == 0) return SYRK_OK;
+    cudaMemset(ds->d_status + first, 0, size_t(count) * sizeof(int));
+    return SYRK_ERR_DEVICE_WAIT;
+}
+
+bool items_fit_kernel(const std::vector<WorkItem>& items, int dtype) {
+    const int max_seg = (dtype == SYRK_DTYPE_F64) ? kMaxSeg : bf16_seg_slots();
+    const int max_tile = (dtype == SYRK_DTYPE_F64) ? kMaxTile : 3;
+    for (const WorkItem& it : items) {
+        if (it.n_seg < 1 || it.n_tile < 1 || it.n_seg > max_seg || it.n_tile > max_tile) return false;
+        for (int t = 0; t < it.n_tile; ++t)
+            if (it.tile_x[t] >= it.n_seg || it.tile_y[t] >= it.n_seg) return false;
+        if (is_tcgen05_dtype(dtype)) {   // TMEM layout: at most one lone tile and one adjacent pair
+            int lone = 0, pairs = 0;
+            for (int t = 0; t < it.n_tile;) {
+                const bool pair = t + 1 < it.n_tile && it.tile_x[t + 1] == it.tile_x[t] &&
+                                  it.tile_y[t + 1] == it.tile_y[t] + 1;
+                pair ? ++pairs : ++lone;
+                t += pair ? 2 : 1;
+            }
+            if (lone > 1 || pairs > 1) return false;
+        }
+    }
+    return true;
 }
 
 int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out, int upper) {
@@ -115,21 +181,7 @@ int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out, int
     if (it == ds->plans.end()) {
         DevicePlan dp;
         if (!build_host_plan(N, dtype, runtime().schedule, &dp.plan, upper)) return SYRK_ERR_PLAN;
-        const int max_seg = (dtype == SYRK_DTYPE_F64) ? kMaxSeg : bf16_seg_slots();
-        const int max_tile = (dtype == SYRK_DTYPE_F64) ? kMaxTile : 3;
-        for (const WorkItem& it : dp.plan.items) {
-            if (it.n_seg > max_seg || it.n_tile > max_tile) return SYRK_ERR_PLAN;
-            if (is_tcgen05_dtype(dtype)) {   // TMEM layout: at most one lone tile and one adjacent pair
-                int lone = 0, pairs = 0;
-                for (int t = 0; t < it.n_tile;) {
-                    const bool pair = t + 1 < it.n_tile && it.tile_x[t + 1] == it.tile_x[t] &&
-                                      it.tile_y[t + 1] == it.tile_y[t] + 1;
-                    pair ? ++pairs : ++lone;
-                    t += pair ? 2 : 1;
-                }
-                if (lone > 1 || pairs > 1) return SYRK_ERR_PLAN;
-            }
-        }
+        if (!items_fit_kernel(dp.plan.items, dtype)) return SYRK_ERR_PLAN;
         std::vector<int64_t> cta_begin;
         if (is_tcgen05_dtype(dtype) && !dp.plan.items.empty()) {
             // Persistent kernel: items go to thread blocks (one per SM) longest first, each to the
@@ -356,7 +408,7 @@ void release_all() {
         }
         if (ds.d_status) cudaFree(ds.d_status);
         if (ds.d_tickets) cudaFree(ds.d_tickets);
-        if (ds.d_partial) cudaFree(ds.d_partial);
+        for (StreamWorkspace& ws : ds.workspaces) if (ws.d_partial) cudaFree(ws.d_partial);
         if (ds.d_a) cudaFree(ds.d_a);
         if (ds.d_c) cudaFree(ds.d_c);
         if (ds.d_packed) cudaFree(ds.d_packed);

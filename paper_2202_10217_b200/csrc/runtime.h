@@ -56,18 +56,26 @@ struct PairPlan {
     int32_t n_blocks = 0;
 };
 
+// K-split workspace of one stream slot (grow-only).
+struct StreamWorkspace {
+    void* d_partial = nullptr;
+    size_t bytes = 0;
+};
+
 struct DeviceState {
     int device = -1;
     int sm_count = 0;
     int cc_major = 0;
+    // Per-stream state.  Work enqueued on one stream runs in order, so it can share a status word,
+    // a K-split workspace and a ticket pair; work on different streams may overlap on the GPU and
+    // must not.  Every stream the library sees gets a slot (first come, kStreamSlots per device).
+    // d_status holds one word per slot plus a last one shared by the streams that found no slot.
     int* d_status = nullptr;
-    // FP64 persistent launches: a pair of tickets per stream (launches on one stream run one
-    // after another, so they can share a pair; launches on different streams cannot).
+    // FP64 persistent launches: a pair of tickets per slot.
     int* d_tickets = nullptr;
-    std::map<cudaStream_t, int> ticket_slot;
+    std::map<cudaStream_t, int> stream_slot;
+    std::vector<StreamWorkspace> workspaces;   // K-split partial tiles, by slot
     std::map<int64_t, PairPlan> pair_plans;   // by number of tile rows
-    float* d_partial = nullptr;  // K-split workspace
-    size_t partial_bytes = 0;
     // staging for the host-buffer entry point (grow-only)
     void* d_a = nullptr; size_t d_a_bytes = 0;
     void* d_c = nullptr; size_t d_c_bytes = 0;
@@ -87,15 +95,27 @@ struct Runtime {
     std::map<int, DeviceState> devices;
     int schedule = 0;
     bool pair_square = false;   // SYRK_SCHEDULE_PAIR_SQUARE: square blocks, CTA-pair kernel where it applies
-    bool auto_pair = false;     // SYRK_SCHEDULE_AUTO: triangle blocks, but the pair kernel for short work lists
+    bool auto_pair = true;      // SYRK_SCHEDULE_AUTO (default): triangle blocks, but the pair kernel for short work lists
     int split_k = 0;
     int f64_launch = 0;
+    int host_pipeline = 0;      // syrk_set_host_pipeline
 };
-constexpr int kTicketStreams = 256;
+constexpr int kStreamSlots = 256;
 
+// Slot of `stream` on this device (assigned on first sight), or -1 when all slots are taken.
+int slot_for_stream(DeviceState* ds, cudaStream_t stream);
+// The status word kernels launched on `stream` report to (the shared last word without a slot).
+int* status_for_stream(DeviceState* ds, cudaStream_t stream);
 // The ticket pair of `stream` on this device, or null when the persistent form must not be used
-// (all pairs taken, or the stream is being captured into a graph, whose replays may overlap).
+// (no slot left, or the stream is being captured into a graph, whose replays may overlap).
 int* tickets_for_stream(DeviceState* ds, cudaStream_t stream);
+// K-split workspace of at least `want` bytes for work enqueued on `stream`.  SYRK_ERR_ALLOC when the
+// stream has no slot, when the allocation fails, or when the buffer would have to grow while the
+// stream is being captured (growing frees the old buffer, which synchronises the device).
+int workspace_for_stream(DeviceState* ds, cudaStream_t stream, size_t want, void** out);
+// Reads and clears the status word of `stream`, or of every stream when `all` is set; the caller
+// has synchronised.  Returns SYRK_OK, SYRK_ERR_DEVICE_WAIT or SYRK_ERR_CUDA.
+int read_and_clear_status(DeviceState* ds, cudaStream_t stream, bool all);
 Runtime& runtime();
 
 // Current device's state, created on first use.  Returns a SYRK_* code.
@@ -103,6 +123,11 @@ int get_device_state(DeviceState** out);
 
 // Plan for (N, dtype) under the current schedule, built and uploaded on first use.
 int get_device_plan(DeviceState* ds, int64_t N, int dtype, DevicePlan** out, int upper = 0);
+
+// Whether every item of a list can be run by the kernel of `dtype`: segment and tile counts, tile
+// indices, and for the tcgen05 kernel its accumulator layout (at most one lone tile and one pair of
+// tiles with the same M-operand and adjacent N-operands).  That kernel does not check items itself.
+bool items_fit_kernel(const std::vector<WorkItem>& items, int dtype);
 
 // Host-only plan (no device).
 bool build_host_plan(int64_t N, int dtype, int schedule, Plan* out, int upper = 0);
@@ -130,9 +155,11 @@ int encode_tensor_map_f64_plain(CUtensorMap* tm, const void* p, int64_t rows, in
 // `f64_launch` >= 0 overrides the process-wide FP64 launch form for this call.  `a_is_m_by_n`: A is
 // stored M x N row-major (pitch lda >= N) and the call computes alpha * A^T A + beta * C.
 // `upper`: the entries with col >= row are updated instead of those with col <= row.
+// `prepare_only`: take the call's decisions (schedule, K-split) and create what it would allocate (work
+// lists, the stream's workspace) for an aligned operand, launch nothing; A and C are not looked at.
 int syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
                     double beta, int dtype, cudaStream_t stream, int f64_launch = -1, int a_is_m_by_n = 0,
-                    int upper = 0);
+                    int upper = 0, bool prepare_only = false);
 
 void release_cholesky_workspaces();
 

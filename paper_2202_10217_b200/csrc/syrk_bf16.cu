@@ -30,6 +30,8 @@
 // stored M x N (the Gram form) the stages hold boxes of k-rows by columns and both
 // operands are MN-major (for every input kind; the boxes are then one stage's k-rows by 128 bytes
 // of columns); everything after the MMA is the same.
+#include <mutex>
+
 #include "device_utils.cuh"
 #include "kernels.h"
 #include "tbs_plan.h"
@@ -522,6 +524,8 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                              int64_t c_batch_stride, int upper) {
     // The shared-memory attribute belongs to a device's context: set it once per device.
     static bool configured[64] = {};
+    static std::mutex configured_mu;                 // launchers are reached under different locks
+    std::lock_guard<std::mutex> configured_lock(configured_mu);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;

@@ -32,6 +32,8 @@
 // Accumulators (the C block) stay on chip for the whole M loop and each entry of
 // C is read (beta != 0) and written exactly once, as in the paper's generic
 // out-of-core scheme (Algorithm 3).
+#include <mutex>
+
 #include "device_utils.cuh"
 #include "kernels.h"
 #include "tbs_plan.h"
@@ -731,6 +733,8 @@ namespace {
 cudaError_t configure_f64_kernels() {
     // The shared-memory attribute belongs to a device's context: set it once per device.
     static bool configured[64] = {};
+    static std::mutex configured_mu;                 // launchers are reached under different locks
+    std::lock_guard<std::mutex> configured_lock(configured_mu);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;

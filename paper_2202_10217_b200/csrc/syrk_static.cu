@@ -48,10 +48,15 @@ struct StaticAddrs {
     int64_t* tile_base = nullptr;
     int* status = nullptr;
     int sm_count = 0;
+    int64_t uploaded_tiles = -1;    // tile rows of the work list the device arrays hold (-1: none yet)
 };
 
 std::mutex g_mu;
 StaticAddrs g_addrs[64];   // per device ordinal
+// Host copies of the work list and of its tile offsets, the source of the upload: fixed storage that
+// outlives the call (the copy engine may read it after the call has returned).  Guarded by g_mu.
+WorkItem g_host_items[kStaticMaxItems];
+int64_t g_host_tile_base[kStaticMaxItems + 1];
 
 // Set-up, once per device, with that device current: resolve the device addresses of
 // the arrays above.  Happens inside the first call on a device.
@@ -95,16 +100,16 @@ extern "C" int syrk_lower_bf16_static(int64_t N, int64_t M, const void* A, int64
 
     const int64_t n_ksteps = (M + bf16_bk() - 1) / bf16_bk();
     if (slices > n_ksteps) return SYRK_ERR_SIZE;
+    const int64_t n_tiles = (N + bf16_tile() - 1) / bf16_tile();
+    // every output tile belongs to exactly one item, so the list has n_tiles (n_tiles + 1) / 2 tiles
+    if (n_tiles * (n_tiles + 1) / 2 * slices > kStaticMaxSliceTiles) return SYRK_ERR_STATIC_LIMIT;
 
-    // Host-side work list (the same generator and ordering as the regular path).
-    Plan plan;
-    if (!build_host_plan(N, SYRK_DTYPE_BF16_F32, SYRK_SCHEDULE_TBS, &plan)) return SYRK_ERR_PLAN;
-    const int64_t n_items = int64_t(plan.items.size());
-    if (n_items > kStaticMaxItems) return SYRK_ERR_STATIC_LIMIT;
-    std::vector<int64_t> base(size_t(n_items) + 1, 0);
-    for (int64_t i = 0; i < n_items; ++i) base[size_t(i) + 1] = base[size_t(i)] + plan.items[size_t(i)].n_tile;
-    const int64_t total_tiles = base[size_t(n_items)];
-    if (total_tiles * slices > kStaticMaxSliceTiles) return SYRK_ERR_STATIC_LIMIT;   // workspace beyond the fixed array
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The call copies its work list from host memory and shares device arrays with every other call:
+    // neither belongs in a captured graph, which would replay both at times of its own.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+    if (cap != cudaStreamCaptureStatusNone) return SYRK_ERR_CUDA;
 
     std::lock_guard<std::mutex> lock(g_mu);
     int dev = -1;
@@ -113,12 +118,37 @@ extern "C" int syrk_lower_bf16_static(int64_t N, int64_t M, const void* A, int64
     int rc = setup_device(dev, &a);
     if (rc != SYRK_OK) return rc;
 
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // The work list travels on the caller's stream, ahead of the kernels that read it.
-    if (cudaMemcpyAsync(a->items, plan.items.data(), size_t(n_items) * sizeof(WorkItem), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(a->tile_base, base.data(), (size_t(n_items) + 1) * sizeof(int64_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
-        cudaGetLastError();
-        return SYRK_ERR_CUDA;
+    // Host-side work list (the same generator and ordering as the regular path); it depends on the
+    // number of tile rows only, so a call that finds the device arrays holding that list already
+    // uploads nothing.
+    int64_t n_items = 0, total_tiles = 0;
+    {
+        Plan plan;
+        if (!build_host_plan(N, SYRK_DTYPE_BF16_F32, SYRK_SCHEDULE_TBS, &plan)) return SYRK_ERR_PLAN;
+        n_items = int64_t(plan.items.size());
+        if (n_items > kStaticMaxItems) return SYRK_ERR_STATIC_LIMIT;
+        if (!items_fit_kernel(plan.items, SYRK_DTYPE_BF16_F32)) return SYRK_ERR_PLAN;   // the kernel does not check items
+        for (int64_t i = 0; i < n_items; ++i) total_tiles += plan.items[size_t(i)].n_tile;
+        if (total_tiles * slices > kStaticMaxSliceTiles) return SYRK_ERR_STATIC_LIMIT;   // workspace beyond the fixed array
+        if (a->uploaded_tiles != n_tiles) {
+            g_host_tile_base[0] = 0;
+            for (int64_t i = 0; i < n_items; ++i) {
+                g_host_items[i] = plan.items[size_t(i)];
+                g_host_tile_base[i + 1] = g_host_tile_base[i] + plan.items[size_t(i)].n_tile;
+            }
+        }
+    }
+    if (a->uploaded_tiles != n_tiles) {
+        // The work list travels on the caller's stream, ahead of the kernels that read it.
+        a->uploaded_tiles = -1;
+        if (cudaMemcpyAsync(a->items, g_host_items, size_t(n_items) * sizeof(WorkItem), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(a->tile_base, g_host_tile_base, (size_t(n_items) + 1) * sizeof(int64_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return SYRK_ERR_CUDA;
+        }
+        // The copies above are from pageable memory: the runtime has staged them before returning,
+        // so the host arrays may be rewritten by the next call.
+        a->uploaded_tiles = n_tiles;
     }
     CUtensorMap tm;
     rc = encode_tensor_map_2d(&tm, SYRK_DTYPE_BF16_F32, A, N, M, lda, bf16_tile(), bf16_bk());
@@ -127,4 +157,18 @@ extern "C" int syrk_lower_bf16_static(int64_t N, int64_t M, const void* A, int64
                                            float(alpha), float(beta), slices, a->partial, a->tile_base,
                                            total_tiles, nullptr, 0, 0, 0, a->status, a->sm_count, st);
     return e == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
+extern "C" int syrk_lower_bf16_static_status(void) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_NO_DEVICE; }
+    if (dev < 0 || dev >= 64) return SYRK_ERR_NO_DEVICE;
+    const StaticAddrs& a = g_addrs[dev];
+    if (!a.ready) return SYRK_OK;                                    // no call on this device yet
+    int flag = 0;
+    if (cudaMemcpy(&flag, a.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+    if (flag == 0) return SYRK_OK;
+    if (cudaMemset(a.status, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_CUDA; }
+    return SYRK_ERR_DEVICE_WAIT;
 }

@@ -146,6 +146,35 @@ def test_schedule_stats_for_the_benchmark_shapes():
     # triangle blocks stream fewer rows of A than squares of the same accumulator budget
     B.syrk_set_schedule(B.SCHEDULE_SQUARE)
     sq = B.syrk_get_schedule_stats(4096, 4096, B.DTYPE_F64)
-    B.syrk_set_schedule(B.SCHEDULE_TBS)
+    B.syrk_set_schedule(B.SCHEDULE_DEFAULT)
     tb = B.syrk_get_schedule_stats(4096, 4096, B.DTYPE_F64)
     assert sq["tri_items"] == 0 and tb["a_loads"] < sq["a_loads"]
+
+
+def test_effective_schedule_follows_the_size_rule():
+    """Default setting: triangle blocks once the list is long (N large against the block side, as the
+    paper's tiled scheme asks), square blocks on CTA pairs below, binary64 always on triangle blocks; an
+    explicit setting is reported as set, with the single-CTA square list where the pair form has too
+    few blocks."""
+    assert B.syrk_effective_schedule(16384, 4096, B.DTYPE_BF16_F32) == B.SCHEDULE_TBS          # 2848 items
+    assert B.syrk_effective_schedule(2048, 262144, B.DTYPE_BF16_F32) == B.SCHEDULE_PAIR_SQUARE  # 55 items
+    assert B.syrk_effective_schedule(7168, 4096, B.DTYPE_E4M3_F32) == B.SCHEDULE_PAIR_SQUARE
+    assert B.syrk_effective_schedule(8192, 4096, B.DTYPE_F16_F32) == B.SCHEDULE_TBS
+    assert B.syrk_effective_schedule(300, 64, B.DTYPE_BF16_F32) == B.SCHEDULE_TBS               # too few blocks for the pairs
+    assert B.syrk_effective_schedule(4096, 4096, B.DTYPE_F64) == B.SCHEDULE_TBS
+    assert B.syrk_effective_schedule(512, 0, B.DTYPE_BF16_F32) == B.SCHEDULE_TBS
+    try:
+        B.syrk_set_schedule(B.SCHEDULE_TBS)
+        assert B.syrk_effective_schedule(2048, 262144, B.DTYPE_BF16_F32) == B.SCHEDULE_TBS
+        B.syrk_set_schedule(B.SCHEDULE_PAIR_SQUARE)
+        assert B.syrk_effective_schedule(16384, 4096, B.DTYPE_BF16_F32) == B.SCHEDULE_PAIR_SQUARE
+        assert B.syrk_effective_schedule(300, 64, B.DTYPE_BF16_F32) == B.SCHEDULE_SQUARE
+        assert B.syrk_effective_schedule(4096, 4096, B.DTYPE_F64) == B.SCHEDULE_SQUARE
+        B.syrk_set_schedule(B.SCHEDULE_SQUARE)
+        assert B.syrk_effective_schedule(16384, 4096, B.DTYPE_BF16_F32) == B.SCHEDULE_SQUARE
+    finally:
+        B.syrk_set_schedule(B.SCHEDULE_DEFAULT)
+    with pytest.raises(B.SyrkError):
+        B.syrk_effective_schedule(-1, 4, B.DTYPE_F64)
+    with pytest.raises(B.SyrkError):
+        B.syrk_effective_schedule(4, 4, 9)

@@ -22,7 +22,7 @@ DT = pytest.mark.parametrize("dtype", [B.DTYPE_BF16_F32, B.DTYPE_F16_F32, B.DTYP
 def pair_schedule():
     B.syrk_set_schedule(B.SCHEDULE_PAIR_SQUARE)
     yield
-    B.syrk_set_schedule(B.SCHEDULE_TBS)
+    B.syrk_set_schedule(B.SCHEDULE_DEFAULT)
 
 
 SIZES = [(3200, 144), (3328, 64), (4200, 320)]      # M: multiples of 16 bytes for every type

@@ -114,7 +114,7 @@ def test_square_schedule_and_argument_errors():
         B.syrk_set_schedule(B.SCHEDULE_SQUARE)
         got, ref, bound = run(A, Bm, -1.0, 1.0, Cin)
     finally:
-        B.syrk_set_schedule(B.SCHEDULE_TBS)
+        B.syrk_set_schedule(B.SCHEDULE_DEFAULT)
     check(got, ref, bound, M, -1.0, 1.0, Cin)
     d = torch.zeros(64 * 64, dtype=torch.float64, device="cuda")
     for kwargs, code in [(dict(ldb=15), -3), (dict(lda=15), -3), (dict(Bm=None), -1), (dict(N=-1), -2)]:

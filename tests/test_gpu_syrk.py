@@ -16,6 +16,19 @@ from paper_2202_10217_b200 import inputs as I
 from gpu_util import assert_within_tolerance, run_case
 
 pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def triangle_block_schedule():
+    """This file is the parity suite of the triangle-block kernels: the sizes an entry-by-entry reference
+    can check are all below the size at which the default schedule starts to use them for the tcgen05
+    types, so the schedule is pinned here (the default is covered by test_gpu_default_schedule.py,
+    test_gpu_configs.py and the random sweep)."""
+    B.syrk_set_schedule(B.SCHEDULE_TBS)
+    yield
+    B.syrk_set_schedule(B.SCHEDULE_DEFAULT)
+
+
 BOTH = [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_TF32_F32, B.DTYPE_E4M3_F32,
         B.DTYPE_F16_F32]                                                     # every input type of the library
 DT = pytest.mark.parametrize("dtype", BOTH, ids=["f64", "bf16", "tf32", "e4m3", "f16"])
@@ -149,7 +162,7 @@ def test_square_schedule_gives_the_same_result(dtype):
         B.syrk_set_schedule(B.SCHEDULE_SQUARE)
         got, ref, bound = run_case(A, dtype, 1.0, 0.0)
     finally:
-        B.syrk_set_schedule(B.SCHEDULE_TBS)
+        B.syrk_set_schedule(B.SCHEDULE_TBS)              # what the fixture of this file expects to undo
     assert_within_tolerance(got, ref, bound, M, 1.0, 0.0, None, dtype, exact=True)
 
 

@@ -93,7 +93,7 @@ def test_large_triangle_block_sizes_and_square_schedule():
             B.syrk_set_schedule(B.SCHEDULE_SQUARE)
             got2, _, _ = run_case(A, dtype, -1.0, 1.0, Cin, upper=True)
         finally:
-            B.syrk_set_schedule(B.SCHEDULE_TBS)
+            B.syrk_set_schedule(B.SCHEDULE_DEFAULT)
         assert_within_tolerance(got2, ref, bound, M, -1.0, 1.0, Cin, dtype)
 
 
