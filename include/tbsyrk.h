@@ -379,6 +379,21 @@ int syrk_selftest_bounded_wait(void* stream);
 int syrk_set_split_k(int slices);
 
 /*
+ * Tail K-split of binary64 calls (no counterpart in the paper; results within the stated tolerance, and
+ * the same bits from run to run).  In the one-block-per-item launch form the thread blocks of Algorithm 4's
+ * block loop reach the SMs in list order, and with a list of only a few rounds of long items the last round
+ * leaves SMs idle.  The library then runs the last items of the list as `slices` blocks each, one per slice
+ * of the inner dimension, and a second kernel adds the slices' partial tiles in slice order.
+ *   slices == 0 (default): automatic - a replay of the dispatch with a cost model decides whether, how many
+ *                          items and how many slices (used when modelled at least 1.5 % faster);
+ *   slices == 1: never;
+ *   slices >= 2: always, for the last `tail_items` items of the list (tests and measurements).
+ * Not used by the persistent launch form, the upper triangle, batches, or calls that cut every item
+ * (fewer items than SMs).  Process-wide.  SYRK_ERR_PLAN for slices outside 0..64 or tail_items < 0.
+ */
+int syrk_set_f64_tail_split(int slices, int64_t tail_items);
+
+/*
  * How later FP64 calls hand the work items of the schedule (Algorithm 4, tiled as in
  * Section 5.1.4) to thread blocks; the paper has no counterpart, results are the same
  * entry for entry.  PER_ITEM: one thread block per item.  PERSISTENT: one block per SM

@@ -31,7 +31,7 @@ MAX_SEG, MAX_TILE = 8, 16
 EXPORTS = [
     "syrk_lower", "syrk_lower_tn", "syrk_ex", "syr2k_lower", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_plan_prepare_stream", "syrk_effective_schedule",
     "syrk_lower_bf16_static_status", "syrk_set_host_pipeline", "syrk_host_pipeline_for", "syrk_shutdown", "syrk_last_status",
-    "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_set_f64_launch", "syrk_get_schedule_stats",
+    "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_set_f64_tail_split", "syrk_set_f64_launch", "syrk_get_schedule_stats",
     "syrk_probe_f64_mma_peak", "syrk_selftest_bounded_wait", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
     "tbs_plan_build", "tbs_plan_balance", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
 ]
@@ -102,6 +102,8 @@ def lib() -> ctypes.CDLL:
         L.syrk_set_schedule.argtypes = [ci]
         L.syrk_set_split_k.restype = ci
         L.syrk_set_split_k.argtypes = [ci]
+        L.syrk_set_f64_tail_split.restype = ci
+        L.syrk_set_f64_tail_split.argtypes = [ci, i64]
         L.syrk_set_f64_launch.restype = ci
         L.syrk_set_f64_launch.argtypes = [ci]
         L.syrk_get_schedule_stats.restype = ci
@@ -308,6 +310,11 @@ F64_LAUNCH_AUTO, F64_LAUNCH_PER_ITEM, F64_LAUNCH_PERSISTENT = 0, 1, 2
 
 def syrk_set_f64_launch(mode: int) -> None:
     _check(lib().syrk_set_f64_launch(mode))
+
+
+def syrk_set_f64_tail_split(slices: int, tail_items: int = 0) -> None:
+    """0: automatic; 1: never; >= 2: the last `tail_items` items of an FP64 list run in that many K-slices."""
+    _check(lib().syrk_set_f64_tail_split(slices, tail_items))
 
 
 def syrk_set_split_k(slices: int) -> None:

@@ -83,6 +83,55 @@ int auto_split_k_f64(int64_t n_items, int64_t N, int64_t M, int bk, int sm_count
     return best;
 }
 
+// Tail K-split of an FP64 call in the one-block-per-item form.  The hardware hands the blocks to SMs in
+// list order as SMs free up, so a call lasts as long as its most loaded SM; with long items (many K-steps)
+// and a list of only a few rounds, the last round leaves SMs idle for up to an item's duration.  Cutting
+// the last items along the inner dimension gives the last round smaller units.  This replays that
+// dispatch for the whole list and for a few (number of tail items, slices) candidates with a cost model -
+// an item takes 3 us plus, per K-step, 2.17 us times the share of the busiest of the SM's four DMMA pipes
+// (16 tiles = 1), a slice 1 us more for its partial tiles; fitted to forty measured (shape, tail, slices)
+// triples within 1 % - and returns the best candidate when it is modelled at least 1.5 % faster, else {n, 1}.
+struct TailSplit { int64_t first; int slices; };
+TailSplit plan_tail_split_f64(const std::vector<WorkItem>& items, int64_t ksteps, int sm_count) {
+    const int64_t n = int64_t(items.size());
+    TailSplit none{n, 1};
+    if (n < sm_count || n > 16 * int64_t(sm_count) || ksteps < 64) return none;
+    auto weight = [](const WorkItem& it) {
+        if (it.kind == kTri && it.n_tile == 15) return 15.0 / 16.0;        // the 16th warp evens the pipes out
+        return double((it.n_tile + 3) / 4) / 4.0;
+    };
+    constexpr double kFixedUs = 3.0, kStepUs = 2.17, kPartialUs = 1.0;
+    std::vector<double> free_at;
+    auto makespan = [&](int64_t first, int slices) {
+        free_at.assign(size_t(sm_count), 0.0);
+        std::make_heap(free_at.begin(), free_at.end(), std::greater<double>());
+        double end = 0.0;
+        auto run = [&](double cost) {
+            std::pop_heap(free_at.begin(), free_at.end(), std::greater<double>());
+            free_at.back() += cost;
+            end = std::max(end, free_at.back());
+            std::push_heap(free_at.begin(), free_at.end(), std::greater<double>());
+        };
+        for (int64_t i = 0; i < first; ++i) run(kFixedUs + kStepUs * double(ksteps) * weight(items[size_t(i)]));
+        for (int64_t i = first; i < n; ++i)
+            for (int sl = 0; sl < slices; ++sl) {
+                const int64_t kk = ksteps * (sl + 1) / slices - ksteps * sl / slices;
+                run(kFixedUs + kPartialUs + kStepUs * double(kk) * weight(items[size_t(i)]));
+            }
+        if (slices > 1) end += 5.0 + double(n - first) * double(slices) * 16.0 * 8192.0 / 4e6;   // the reduction pass
+        return end;
+    };
+    const double whole = makespan(n, 1);
+    TailSplit best = none;
+    double best_t = whole;
+    for (int slices = 2; slices <= 6 && ksteps / slices >= 16; ++slices)
+        for (int64_t tail = sm_count / 4; tail <= 3 * int64_t(sm_count) && tail <= n; tail += sm_count / 4) {
+            const double t = makespan(n - tail, slices);
+            if (t < best_t) { best_t = t; best = TailSplit{n - tail, slices}; }
+        }
+    return best_t < 0.985 * whole ? best : none;
+}
+
 int pick_split_k(const DeviceState* ds, DevicePlan* dp, int64_t M, int bk) {
     if (runtime().split_k > 0) return auto_split_k(dp->plan.items, M, bk, ds->sm_count, runtime().split_k);
     auto it = dp->auto_split.find(M);
@@ -94,7 +143,8 @@ int pick_split_k(const DeviceState* ds, DevicePlan* dp, int64_t M, int bk) {
 int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkItem* d_items, int64_t n_items,
                  int64_t N, int64_t M, void* C, int64_t ldc, double alpha, double beta, int split,
                  const int64_t* d_tile_base, int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas,
-                 int f64_launch, int a_is_m_by_n, cudaStream_t stream, int upper = 0, void* d_partial = nullptr) {
+                 int f64_launch, int a_is_m_by_n, cudaStream_t stream, int upper = 0, void* d_partial = nullptr,
+                 int64_t tail_first = 0, int tail_slices = 1) {
     cudaError_t e;
     int* d_status = status_for_stream(ds, stream);
     if (dtype == SYRK_DTYPE_F64) {
@@ -105,12 +155,12 @@ int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkIt
         // That pays when items are short (M <= 1024: at most 64 stages each) and the list fills the
         // device several times over; for long items one block per item is the faster form.
         const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
-        const bool persistent = !upper && (mode == SYRK_F64_LAUNCH_PERSISTENT ||
+        const bool persistent = !upper && tail_slices <= 1 && (mode == SYRK_F64_LAUNCH_PERSISTENT ||
                                 (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count)));
         int* tickets = (persistent && split <= 1) ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<double*>(C), ldc,
                             alpha, beta, a_is_m_by_n, tickets, ds->sm_count, d_status, stream, 0, 0, split,
-                            static_cast<double*>(d_partial), upper);
+                            static_cast<double*>(d_partial), upper, tail_first, tail_slices);
     } else {
         CUtensorMap tmc;
         const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
@@ -278,7 +328,8 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         if (rc != SYRK_ERR_PLAN) return rc;
     }
     const KernelShape ks = kernel_shape(dtype);
-    int split = 1;
+    int split = 1, tail_slices = 1;
+    int64_t tail_first = 0;
     void* d_partial = nullptr;
     if (is_tcgen05_dtype(dtype)) {
         split = pick_split_k(ds, dp, M, ks.bk);
@@ -293,6 +344,31 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         if (split > 1 &&
             (rc = workspace_for_stream(ds, stream, size_t(split) * size_t(N) * size_t(N) * sizeof(double), &d_partial)) != SYRK_OK)
             return rc;
+        // Otherwise, in the one-block-per-item form: the last round's items in slices (tail K-split).
+        const int64_t n_items = int64_t(dp->plan.items.size());
+        const int mode = runtime().f64_launch;
+        const bool per_item = upper || mode == SYRK_F64_LAUNCH_PER_ITEM ||
+                              (mode == SYRK_F64_LAUNCH_AUTO && !(M <= 1024 && n_items >= 4 * int64_t(ds->sm_count)));
+        if (split == 1 && per_item && !upper && runtime().f64_tail_slices != 1) {
+            TailSplit ts{n_items, 1};
+            const int64_t ksteps = (M + ks.bk - 1) / ks.bk;
+            if (runtime().f64_tail_slices >= 2) {                    // forced (tests, measurements)
+                const int64_t tail = std::min<int64_t>(n_items, std::max<int64_t>(1, runtime().f64_tail_items));
+                if (runtime().f64_tail_slices <= ksteps) ts = TailSplit{n_items - tail, runtime().f64_tail_slices};
+            } else {
+                auto it = dp->tail_split.find(ksteps);
+                if (it == dp->tail_split.end()) {
+                    const TailSplit t = plan_tail_split_f64(dp->plan.items, ksteps, ds->sm_count);
+                    it = dp->tail_split.emplace(ksteps, std::make_pair(t.first, t.slices)).first;
+                }
+                ts = TailSplit{it->second.first, it->second.second};
+            }
+            if (ts.slices > 1) {
+                const size_t want = size_t(f64_tail_partial_elems(n_items - ts.first, ts.slices)) * sizeof(double);
+                if ((rc = workspace_for_stream(ds, stream, want, &d_partial)) != SYRK_OK) return rc;
+                tail_first = ts.first; tail_slices = ts.slices;
+            }
+        }
     }
     if (prepare_only) return SYRK_OK;
     CUtensorMap tm;
@@ -303,7 +379,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
     if (rc != SYRK_OK) return rc;
     return launch_items(ds, dtype, tm, dp->d_items, int64_t(dp->plan.items.size()), N, M, C, ldc, alpha, beta, split,
                         dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, f64_launch, a_is_m_by_n, stream, upper,
-                        d_partial);
+                        d_partial, tail_first, tail_slices);
 }
 
 namespace {
@@ -802,6 +878,14 @@ int syrk_set_f64_launch(int mode) {
         return SYRK_ERR_PLAN;
     std::lock_guard<std::mutex> lock(runtime().mu);
     runtime().f64_launch = mode;
+    return SYRK_OK;
+}
+
+int syrk_set_f64_tail_split(int slices, int64_t tail_items) {
+    if (slices < 0 || slices > 64 || tail_items < 0) return SYRK_ERR_PLAN;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    runtime().f64_tail_slices = slices;
+    runtime().f64_tail_items = tail_items;
     return SYRK_OK;
 }
 

@@ -20,12 +20,17 @@ namespace tbsyrk {
 // inner dimension is cut into that many slices, one block per (slice, item) writes partial
 // matrices and a second kernel sums them in slice order and applies alpha and beta.  `upper`: the
 // work list holds the tiles on and above the diagonal and entries with col >= row are written (one
-// block per item; not with `batch`).
+// block per item; not with `batch`).  `tail_slices` > 1 (one block per item, lower triangle, split_k == 1):
+// the items from `tail_first` on run as tail_slices blocks each, one per slice of the inner dimension,
+// whose raw partial tiles (in `d_partial`) a second kernel sums in slice order: smaller units for the
+// last round of blocks, same bits whatever the order the blocks ran in.
 cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, const WorkItem* d_items,
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
                             cudaStream_t stream, int64_t batch = 0, int64_t c_batch_stride = 0, int split_k = 1,
-                            double* d_partial = nullptr, int upper = 0);
+                            double* d_partial = nullptr, int upper = 0, int64_t tail_first = 0, int tail_slices = 1);
+// Elements of `d_partial` a tail K-split needs: (n_items - tail_first) * tail_slices units of 16 tiles.
+int64_t f64_tail_partial_elems(int64_t n_tail_items, int tail_slices);
 // Rank-2k update C = alpha (A B^T + B A^T) + beta C on the lower triangle with the same kernel: the work
 // items name at most 4 segments and 8 tiles; every stage holds the segments' rows of A (tmA) and of
 // B (tmB); a tile is shared by two warps (16 rows each) that add both products.  One block per item.

@@ -39,6 +39,7 @@ struct DevicePlan {
     int n_ctas = 0;
     std::map<int64_t, int> auto_split;   // tcgen05: modelled number of K-slices by inner dimension (the model
                                          // walks every unit of every candidate: too slow to redo on every call)
+    std::map<int64_t, std::pair<int64_t, int>> tail_split;   // FP64: (first tail item, slices) by number of K-steps
 };
 
 // Square-block work list in row order for the host-buffer entry point: band j owns the rows
@@ -99,6 +100,8 @@ struct Runtime {
     int split_k = 0;
     int f64_launch = 0;
     int host_pipeline = 0;      // syrk_set_host_pipeline
+    int f64_tail_slices = 0;    // syrk_set_f64_tail_split: 0 automatic, 1 off, >= 2 forced
+    int64_t f64_tail_items = 0; //   forced number of tail items
 };
 constexpr int kStreamSlots = 256;
 

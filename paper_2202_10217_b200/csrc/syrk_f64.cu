@@ -81,6 +81,11 @@ struct Call {
     bool syr2k;                    // rank-2k update: slots 0..3 hold segments of A, slots 4..7 the same rows of B (tmB)
     bool gemm;
 };
+// Tail K-split units: bit 1 of Call::vec_ok is set and Call::C points at the unit's partial tiles (16 slots
+// of 32 x 32, slot q at q * 1024) instead of at the result matrix.
+constexpr int kVecOkPartial = 2;
+constexpr int kPartTileElems = kTile * kTile;            // 1024 doubles per partial tile
+constexpr int kPartUnitElems = kMmaWarps * kPartTileElems; // one unit: a slot per MMA warp
 
 // Ring steps of one item: its K-steps, then (c_tma) one step per group of four tiles of old C.
 __device__ __forceinline__ int c_steps_of(const Call& k, int n_tile) { return k.c_tma ? (n_tile + 3) / 4 : 0; }
@@ -334,6 +339,11 @@ __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it
                 }
                 continue;
             }
+            if (k.vec_ok & kVecOkPartial) {                         // partial tile q of a K-slice: raw sums, no mask
+                *reinterpret_cast<double2*>(k.C + q * kPartTileElems + (24 + gq) * kTile + 24 + 2 * t) =
+                    make_double2(sacc[q][0], sacc[q][1]);
+                continue;
+            }
             const int64_t r = int64_t(seg[x]) * kTile + 24 + gq;
             const int64_t c = int64_t(seg[y]) * kTile + 24 + 2 * t;
             if (r >= k.N) continue;                                 // tile below the diagonal: c + 1 < r
@@ -404,6 +414,20 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
             }
         }
         for (int j = 0; j < n_c; ++j) release(k, gc + j, lane);
+        return true;
+    }
+    if (!kUpper && (k.vec_ok & kVecOkPartial)) {
+        // A K-slice of a tail item: the raw sums of this warp's tile go to slot `warp` of the unit's partial
+        // tiles, all 32 x 32 entries (the reduction applies alpha, beta and the triangle mask).
+        double* out = k.C + warp * kPartTileElems;
+#pragma unroll
+        for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+            for (int ni = 0; ni < 4; ++ni) {
+                if (scavenge && mi == 3 && ni == 3) continue;             // written by the 16th warp
+                *reinterpret_cast<double2*>(out + (mi * 8 + gq) * kTile + ni * 8 + 2 * t) =
+                    make_double2(acc[mi][ni][0], acc[mi][ni][1]);
+            }
         return true;
     }
 #pragma unroll
@@ -558,7 +582,8 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
                     int64_t ncols, int32_t gemm_col_tiles, int32_t n_ksteps, double* __restrict__ C,
                     int64_t ldc, double alpha, double beta, int vec_ok, int c_tma, int* __restrict__ status,
-                    int64_t items_per_batch, int64_t c_batch_stride, int32_t slice_ksteps) {
+                    int64_t items_per_batch, int64_t c_batch_stride, int32_t slice_ksteps,
+                    int32_t tail_first, int32_t tail_slices, double* __restrict__ tail_partial) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ WorkItem s_item;
@@ -577,8 +602,21 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // Strided batch: the grid holds the work list once per matrix; the tensor maps are 3-D.
     // K-split (slice_ksteps > 0): the grid holds the list once per slice of the inner dimension;
     // slice s takes K-steps [s * slice_ksteps, ...) of the 2-D maps and writes partial matrix s.
+    // Tail K-split (tail_slices > 1): blocks [0, tail_first) run items 0 .. tail_first - 1 whole; the blocks
+    // after them run the remaining items in tail_slices slices of the inner dimension each (item-major),
+    // writing raw partial tiles that a second kernel sums in slice order.
     k.batch = -1; k.k0 = 0;
     int64_t item_index = blockIdx.x;
+    if (tail_slices > 1 && int64_t(blockIdx.x) >= int64_t(tail_first)) {
+        const int64_t u = int64_t(blockIdx.x) - tail_first;
+        const int32_t sl = int32_t(u % tail_slices);
+        item_index = tail_first + u / tail_slices;
+        k.k0 = int32_t(int64_t(n_ksteps) * sl / tail_slices);
+        k.n_ksteps = int32_t(int64_t(n_ksteps) * (sl + 1) / tail_slices) - k.k0;
+        k.C = tail_partial + u * kPartUnitElems;
+        k.vec_ok = 1 | kVecOkPartial;
+        k.c_tma = 0;
+    }
     if (items_per_batch > 0) {
         const int32_t group = int32_t(int64_t(blockIdx.x) / items_per_batch);
         item_index = int64_t(blockIdx.x) % items_per_batch;
@@ -727,6 +765,28 @@ splitk_reduce_f64_kernel(int64_t N, int32_t slices, const double* __restrict__ p
     *c = (beta == 0.0) ? alpha * s : alpha * s + beta * *c;
 }
 
+// Tail K-split: for tail item i (list entry tail_first + i) and each of its tiles, the stored triangle of C
+// <- alpha * (sum of the slices' partial tiles, in slice order) + beta * C.  Unit (i, slice) has its 16 tile
+// slots at partial + (i * slices + slice) * 16 * 1024.
+__global__ void __launch_bounds__(256)
+tail_reduce_f64_kernel(const WorkItem* __restrict__ items, int32_t tail_first, int32_t slices,
+                       const double* __restrict__ partial, int64_t N, double* __restrict__ C, int64_t ldc,
+                       double alpha, double beta) {
+    const WorkItem* it = &items[tail_first + blockIdx.x];
+    const int q = blockIdx.y;
+    if (q >= it->n_tile) return;
+    const int64_t row0 = int64_t(it->seg[it->tile_x[q]]) * kTile, col0 = int64_t(it->seg[it->tile_y[q]]) * kTile;
+    const double* src = partial + (int64_t(blockIdx.x) * slices * kMmaWarps + q) * kPartTileElems;
+    for (int e = threadIdx.x; e < kPartTileElems; e += blockDim.x) {
+        const int64_t r = row0 + e / kTile, c = col0 + e % kTile;
+        if (r >= N || c > r) continue;
+        double s = 0.0;
+        for (int32_t sl = 0; sl < slices; ++sl) s += src[int64_t(sl) * kPartUnitElems + e];
+        double* dst = C + r * ldc + c;
+        *dst = (beta == 0.0) ? alpha * s : alpha * s + beta * *dst;
+    }
+}
+
 }  // namespace f64
 
 namespace {
@@ -760,7 +820,7 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
                             int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc, double alpha,
                             double beta, int a_is_m_by_n, int* d_tickets, int n_blocks, int* d_status,
                             cudaStream_t stream, int64_t batch, int64_t c_batch_stride, int split_k,
-                            double* d_partial, int upper) {
+                            double* d_partial, int upper, int64_t tail_first, int tail_slices) {
     cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
@@ -780,7 +840,7 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
                             : (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, false> : f64::syrk_f64_tbs_kernel<false, false>);
         kernel<<<dim3(unsigned(n_items * slices)), threads, f64::kSmemBytes, stream>>>(
             tmA, tmA, none, d_items, N, N, 0, n_ksteps, d_partial, N, 1.0, 0.0, (N & 1) == 0 ? 1 : 0, 0, d_status,
-            n_items, N * N, slice_ksteps);
+            n_items, N * N, slice_ksteps, 0, 1, nullptr);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         const dim3 rb(32, 8);
@@ -795,7 +855,7 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
         auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, false> : f64::syrk_f64_tbs_kernel<false, false>;
         kernel<<<dim3(unsigned(n_items * batch)), threads, f64::kSmemBytes, stream>>>(
             tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
-            n_items, c_batch_stride, 0);
+            n_items, c_batch_stride, 0, 0, 1, nullptr);
         return cudaGetLastError();
     }
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30) && !upper) {
@@ -807,9 +867,23 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
     }
     auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, true> : f64::syrk_f64_tbs_kernel<false, true>)
                         : (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, false> : f64::syrk_f64_tbs_kernel<false, false>);
+    if (tail_slices > 1 && d_partial != nullptr && !upper && tail_first >= 0 && tail_first < n_items) {
+        // Tail K-split: the last n_items - tail_first items run as tail_slices blocks each (see the kernel).
+        const int64_t n_tail = n_items - tail_first;
+        const int64_t blocks = tail_first + n_tail * tail_slices;
+        if (blocks >= (int64_t(1) << 31) || n_tail >= 65536 || tail_slices > n_ksteps) return cudaErrorInvalidValue;
+        kernel<<<dim3(unsigned(blocks)), threads, f64::kSmemBytes, stream>>>(
+            tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
+            int64_t(0), int64_t(0), 0, int32_t(tail_first), int32_t(tail_slices), d_partial);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        f64::tail_reduce_f64_kernel<<<dim3(unsigned(n_tail), f64::kMmaWarps), 256, 0, stream>>>(
+            d_items, int32_t(tail_first), int32_t(tail_slices), d_partial, N, C, ldc, alpha, beta);
+        return cudaGetLastError();
+    }
     kernel<<<dim3(unsigned(n_items)), threads, f64::kSmemBytes, stream>>>(
         tmA, tmA, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
-        int64_t(0), int64_t(0), 0);
+        int64_t(0), int64_t(0), 0, 0, 1, nullptr);
     return cudaGetLastError();
 }
 
@@ -825,7 +899,7 @@ cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, con
     CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<false, false, true><<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmA, tmB, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
-        int64_t(0), int64_t(0), 0);
+        int64_t(0), int64_t(0), 0, 0, 1, nullptr);
     return cudaGetLastError();
 }
 
@@ -843,10 +917,13 @@ cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, c
     CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<false, false><<<dim3(unsigned(blocks)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmP, tmQ, c_tma ? *tmD : none, nullptr, nrows, ncols, int32_t(col_tiles), n_ksteps, D, ldd, alpha, beta,
-        vec_ok, c_tma, d_status, int64_t(0), int64_t(0), 0);
+        vec_ok, c_tma, d_status, int64_t(0), int64_t(0), 0, 0, 1, nullptr);
     return cudaGetLastError();
 }
 
+int64_t f64_tail_partial_elems(int64_t n_tail_items, int tail_slices) {
+    return n_tail_items * int64_t(tail_slices) * f64::kPartUnitElems;
+}
 int f64_tile() { return f64::kTile; }
 int f64_bk() { return f64::kBK; }
 int f64_stages() { return f64::kStages; }

@@ -323,6 +323,50 @@ def test_f64_k_split_automatic_for_short_work_lists():
     assert_within_tolerance(got, ref, bound, M, 1.0, -1.0, Cin, B.DTYPE_F64)
 
 
+@pytest.mark.parametrize("tn", [False, True], ids=["nxm", "mxn"])
+@pytest.mark.parametrize("slices,tail", [(2, 1), (3, 7), (5, 10 ** 6)])
+def test_f64_tail_k_split_forced(slices, tail, tn):
+    """FP64 tail K-split: the last `tail` items of the list run as `slices` blocks each and a second
+    kernel sums their partial tiles in slice order (one item, a few items spanning kinds, every item).
+    Triangle blocks with their 16th warp, rectangles and diagonal blocks, ragged N and last K-step,
+    general alpha / beta with a pitch, integer inputs bit for bit, and the same bits when repeated."""
+    for n, (N, M) in enumerate([(1056, 272), (2100, 130), (700, 1030)]):
+        A = make_A(N, M, B.DTYPE_F64, seed=1000 + n)
+        Ai = make_A(N, M, B.DTYPE_F64, seed=1050 + n, kind="int")
+        Cin = I.random_c(N, 1060 + n, B.DTYPE_F64)
+        try:
+            B.syrk_set_f64_launch(B.F64_LAUNCH_PER_ITEM)
+            B.syrk_set_f64_tail_split(slices, tail)
+            got, ref, bound = run_case(A, B.DTYPE_F64, -1.5, 0.5, Cin, ldc=N + 2, tn=tn)
+            again, _, _ = run_case(A, B.DTYPE_F64, -1.5, 0.5, Cin, ldc=N + 2, tn=tn)
+            goti, refi, boundi = run_case(Ai, B.DTYPE_F64, 1.0, 0.0, poison=True, tn=tn)
+        finally:
+            B.syrk_set_f64_tail_split(0)
+            B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+        assert_within_tolerance(got, ref, bound, M, -1.5, 0.5, Cin, B.DTYPE_F64)
+        assert np.array_equal(got[np.tril_indices(N)], again[np.tril_indices(N)])
+        assert_within_tolerance(goti, refi, boundi, M, 1.0, 0.0, None, B.DTYPE_F64, exact=True)
+
+
+def test_f64_tail_k_split_automatic():
+    """A list of a few rounds of long items (3000 x 2048: 319 items of 128 K-steps for 148 SMs): the library
+    cuts the tail by itself; switched off, the result agrees within tolerance (another summation order)."""
+    N, M = 3000, 2048
+    A = make_A(N, M, B.DTYPE_F64, seed=1100)
+    Cin = I.random_c(N, 1101, B.DTYPE_F64)
+    got, ref, bound = run_case(A, B.DTYPE_F64, 1.0, -1.0, Cin)
+    assert_within_tolerance(got, ref, bound, M, 1.0, -1.0, Cin, B.DTYPE_F64)
+    try:
+        B.syrk_set_f64_tail_split(1)
+        off, _, _ = run_case(A, B.DTYPE_F64, 1.0, -1.0, Cin)
+    finally:
+        B.syrk_set_f64_tail_split(0)
+    assert_within_tolerance(off, ref, bound, M, 1.0, -1.0, Cin, B.DTYPE_F64)
+    Ai = make_A(N, 1100, B.DTYPE_F64, seed=1102, kind="int")
+    goti, refi, boundi = run_case(Ai, B.DTYPE_F64, 1.0, 0.0)
+    assert_within_tolerance(goti, refi, boundi, 1100, 1.0, 0.0, None, B.DTYPE_F64, exact=True)
+
+
 def test_tf32_low_order_bits_of_the_inputs_are_ignored():
     """The tensor core reads the 19 high-order bits of every binary32 input.  With values whose
     low 13 bits are set the result must equal, bit for bit, the result for the same values with
