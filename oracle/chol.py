@@ -29,6 +29,8 @@ def _load():
         lib = ctypes.CDLL(build())
         lib.oracle_cholesky_lower.restype = ctypes.c_int64
         lib.oracle_cholesky_lower.argtypes = [ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64]
+        lib.oracle_cholesky_lower_leading.restype = ctypes.c_int64
+        lib.oracle_cholesky_lower_leading.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64]
         _lib = lib
     return _lib
 
@@ -45,6 +47,22 @@ def cholesky_lower(A: np.ndarray):
     info = int(_load().oracle_cholesky_lower(L.shape[0], L.ctypes.data, max(L.shape[0], 1)))
     if info < 0:
         raise ValueError("oracle_cholesky_lower rejected its arguments")
+    return L, info
+
+
+def cholesky_lower_leading(panel: np.ndarray):
+    """First ``c`` columns of the factor from the first ``c`` columns of the matrix.
+
+    ``panel`` is N x c (the leading columns of a symmetric positive definite N x N matrix; entries
+    above the diagonal are ignored).  Returns ``(Lc, info)`` with the N x c leading columns of L.
+    """
+    if panel.dtype != np.float64 or panel.ndim != 2 or panel.shape[1] > panel.shape[0]:
+        raise ValueError("panel must be a float64 N x c array with c <= N")
+    L = np.ascontiguousarray(panel).copy()
+    N, c = L.shape
+    info = int(_load().oracle_cholesky_lower_leading(N, c, L.ctypes.data, max(c, 1)))
+    if info < 0:
+        raise ValueError("oracle_cholesky_lower_leading rejected its arguments")
     return L, info
 
 

@@ -80,3 +80,39 @@ def test_indefinite_matrix_is_reported():
     assert info == 2
     _, info = K.cholesky_lower(np.array([[-1.0]]))
     assert info == 1
+
+
+def test_leading_columns_routine_equals_the_full_factorisation_bit_for_bit():
+    """The restricted loop performs, for the columns it keeps, the very operations of the full one."""
+    rng = np.random.default_rng(11)
+    for N in (1, 5, 64, 300):
+        G = rng.standard_normal((N, N + 3))
+        A = G @ G.T / N + np.eye(N)
+        full, info = K.cholesky_lower(A)
+        assert info == 0
+        for c in sorted({1, min(N, 17), N}):
+            panel = A[:, :c].copy()
+            panel[np.triu_indices(N, 1, c)] = np.nan               # entries above the diagonal are never read
+            Lc, info = K.cholesky_lower_leading(panel)
+            assert info == 0
+            il = np.tril_indices(N, 0, c)
+            assert np.array_equal(Lc[il], full[:, :c][il])
+            assert np.isnan(Lc[np.triu_indices(N, 1, c)]).all()  # ... nor written
+    # closed form: the first columns of the Pascal matrix's factor are binomial coefficients
+    N, c = 12, 5
+    P = np.array([[float(math.comb(i + j, i)) for j in range(N)] for i in range(N)])
+    Lc, info = K.cholesky_lower_leading(P[:, :c].copy())
+    want = np.array([[float(math.comb(i, j)) for j in range(c)] for i in range(N)])
+    assert info == 0 and np.array_equal(np.tril(Lc), want)
+    # the hand-worked 3 x 3 example, first two columns
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "cholesky_3x3_by_hand.txt")) if not l.startswith("#")]
+    A3 = np.zeros((3, 3)); W3 = np.zeros((3, 3))
+    for i in range(3):
+        A3[i, :i + 1] = [float(v) for v in rows[1 + i]]
+        W3[i, :i + 1] = [float(v) for v in rows[1 + 3 + i]]
+    L2, info = K.cholesky_lower_leading(A3[:, :2].copy())
+    assert info == 0 and np.array_equal(np.tril(L2), np.tril(W3[:, :2]))
+    # a non-positive pivot inside the kept columns is reported, one beyond them is not looked at
+    B3 = np.array([[4.0, 0.0, 0.0], [2.0, 1.0, 0.0], [0.0, 0.0, 1.0]])
+    assert K.cholesky_lower_leading(B3[:, :2].copy())[1] == 2
+    assert K.cholesky_lower_leading(B3[:, :1].copy())[1] == 0
