@@ -7,10 +7,11 @@
 //   3. A[I1, I1] <- A[I1, I1] - A[I1, I0] * A[I1, I0]^T      (TBS: syrk_lower with alpha = -1,
 //                                                             beta = 1, K = b, trailing view)
 // Steps 1 and 2 are only cited by the paper; here they run in 128-column sub-steps.  A leaf
-// kernel (one thread block) factors a 128 x 128 diagonal block in shared memory and inverts
-// the factor; the rows below are solved as a product with that inverse (FP64 tensor-core
-// kernel in two-operand mode) and the rest of the panel is updated by a small SYRK (inside the
-// panel) and a product (below it).  Step 3 is the library's triangle-block SYRK.
+// kernel (one thread block) factors a 128 x 128 diagonal block in shared memory; the rows below
+// are solved against it by blocked forward substitution (64 rows per thread block, in place) and
+// the rest of the panel is updated by a small SYRK (inside the panel) and a product (below it,
+// FP64 tensor-core kernel in two-operand mode).  No triangular factor is inverted anywhere.
+// Step 3 is the library's triangle-block SYRK.
 #include <algorithm>
 #include <mutex>
 
@@ -23,28 +24,57 @@ namespace {
 
 constexpr int kLeaf = 128;
 constexpr int kLeafThreads = 512;
-constexpr int kNb = 32;                                         // inner block of the leaf
-constexpr int kLs = kLeaf + 1;                                  // padded row pitch of the factor in shared memory
-constexpr int kWs = kNb + 1;                                    // padded row pitch of a 32 x 32 block
-constexpr int kLeafSmem = (kLeaf * kLs + 4 * kNb * kWs + kNb * kWs) * int(sizeof(double));
+constexpr int kNb = 32;                                         // inner block of the leaf and of the row solve
+constexpr int kLs = kLeaf + 1;                                  // padded row pitch of a 128-column block in shared memory
+constexpr int kLeafSmem = kLeaf * kLs * int(sizeof(double));
 
-// Factor the m x m block at A (lower triangle, row pitch lda) in place and write the inverse
-// of the factor, as a full 128 x 128 row-major matrix with zeros above the diagonal and
-// beyond m, to W.  On a non-positive pivot k, *info <- pivot_base + k + 1 if it is still 0.
+// Algorithm 2 of the paper on one 32 x 32 diagonal block D (row pitch kLs, shared memory) by one warp: lane r
+// holds row r in registers and values travel by shuffle.  A non-positive pivot k sets *info (if still 0) to
+// pivot_base + k + 1 and *bad_flag.  Kept out of line so that the row stays in registers (inlined into the
+// leaf kernel the compiler left it in local memory, which made the leaf three times slower).
+__device__ __noinline__ void factor_diag_block(double* D, int lane, long long* info, long long pivot_base, int* bad_flag) {
+    double row[kNb];
+#pragma unroll
+    for (int c = 0; c < kNb; ++c) row[c] = D[lane * kLs + c];
+    bool bad = false;
+#pragma unroll
+    for (int k = 0; k < kNb; ++k) {
+        const double p = __shfl_sync(0xffffffffu, row[k], k);
+        if (!(p > 0.0)) {                                  // same value in every lane
+            if (!bad && lane == 0) {
+                atomicCAS(reinterpret_cast<unsigned long long*>(info), 0ull,
+                          static_cast<unsigned long long>(pivot_base + k + 1));
+                *bad_flag = 1;
+            }
+            bad = true;
+        }
+        const double d = sqrt(bad ? 1.0 : p);
+        if (lane == k) row[k] = d;
+        if (lane > k) row[k] = row[k] / d;
+        const double l = row[k];                           // L[lane][k] for lane >= k
+#pragma unroll
+        for (int c = k + 1; c < kNb; ++c) {
+            const double lc = __shfl_sync(0xffffffffu, l, c);       // L[c][k]
+            if (lane >= c) row[c] -= l * lc;
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < kNb; ++c)
+        if (c <= lane) D[lane * kLs + c] = row[c];
+}
+
+// Factor the m x m block at A (lower triangle, row pitch lda) in place.  On a non-positive pivot k,
+// *info <- pivot_base + k + 1 if it is still 0, and A is left as it was.
 //
-// Blocked right-looking Cholesky on 32 x 32 blocks, all in shared memory (rows beyond m are
-// padded with the identity): one warp factors a diagonal block column by column (Algorithm 2)
-// and inverts it; all 16 warps then solve the block rows below with that inverse and update
-// the trailing blocks.  The inverse of the whole factor is assembled block by block,
-// W[I][J] = -W[I][I] * sum_{K=J}^{I-1} L[I][K] * W[K][J], over the storage of L's off-diagonal
-// blocks once L has been written back.
+// Blocked right-looking Cholesky on 32 x 32 blocks, all in shared memory (rows beyond m are padded with
+// the identity): one warp factors a diagonal block column by column (Algorithm 2 of the paper on the
+// block, a row per lane, values travelling by shuffle); all 16 warps then solve the block rows below by
+// forward substitution against that block (x L_JJ^T = p, one row per warp and pass: lane c divides, the
+// lanes after it subtract) and update the trailing blocks.  Nothing is inverted.
 __global__ void __launch_bounds__(kLeafThreads)
-chol_leaf_kernel(double* __restrict__ A, int64_t lda, int m, double* __restrict__ W,
-                 long long* __restrict__ info, long long pivot_base) {
+chol_leaf_kernel(double* __restrict__ A, int64_t lda, int m, long long* __restrict__ info, long long pivot_base) {
     extern __shared__ double leaf_smem[];
     double* Lf = leaf_smem;                                       // 128 x 129
-    double* Wd = leaf_smem + kLeaf * kLs;                         // 4 diagonal inverses, 32 x 33 each
-    double* Tb = Wd + 4 * kNb * kWs;                              // one 32 x 33 scratch block
     __shared__ int s_bad;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -56,62 +86,21 @@ chol_leaf_kernel(double* __restrict__ A, int64_t lda, int m, double* __restrict_
 
     for (int J = 0; J < kLeaf / kNb; ++J) {
         const int j0 = J * kNb;
-        double* Wj = Wd + J * kNb * kWs;
-        if (warp == 0) {
-            // ---- diagonal block in registers: lane r holds row r; values travel by shuffle ----
-            double* D = Lf + j0 * kLs + j0;
-            double row[kNb];
-#pragma unroll
-            for (int c = 0; c < kNb; ++c) row[c] = D[lane * kLs + c];
-            bool bad = false;
-#pragma unroll
-            for (int k = 0; k < kNb; ++k) {                        // Algorithm 2 on the block
-                const double p = __shfl_sync(0xffffffffu, row[k], k);
-                if (!(p > 0.0)) {                                  // same value in every lane
-                    if (!bad && lane == 0) {
-                        atomicCAS(reinterpret_cast<unsigned long long*>(info), 0ull,
-                                  static_cast<unsigned long long>(pivot_base + j0 + k + 1));
-                        s_bad = 1;
-                    }
-                    bad = true;
-                }
-                const double d = sqrt(bad ? 1.0 : p);
-                if (lane == k) row[k] = d;
-                if (lane > k) row[k] = row[k] / d;
-                const double l = row[k];                           // L[lane][k] for lane >= k
-#pragma unroll
-                for (int c = k + 1; c < kNb; ++c) {
-                    const double lc = __shfl_sync(0xffffffffu, l, c);       // L[c][k]
-                    if (lane >= c) row[c] -= l * lc;
-                }
-            }
-#pragma unroll
-            for (int c = 0; c < kNb; ++c)
-                if (c <= lane) D[lane * kLs + c] = row[c];
-            __syncwarp();
-            // ---- its inverse: lane j holds column j, W[i][j] = (delta_ij - sum_k L[i][k] W[k][j]) / L[i][i];
-            //      L[i][k] is read from shared memory (same address in every lane) ----
-            if (!bad) {
-                double w[kNb];
-#pragma unroll
-                for (int i = 0; i < kNb; ++i) {
-                    double sacc = (i == lane) ? 1.0 : 0.0;
-#pragma unroll
-                    for (int k = 0; k < i; ++k)
-                        if (k >= lane) sacc -= D[i * kLs + k] * w[k];
-                    w[i] = (i >= lane) ? sacc / D[i * kLs + i] : 0.0;
-                    Wj[i * kWs + lane] = w[i];
-                }
-            }
-        }
+        if (warp == 0) factor_diag_block(Lf + j0 * kLs + j0, lane, info, pivot_base + j0, &s_bad);
         __syncthreads();
         if (s_bad) break;
-        // ---- block rows below: X = P * W_JJ^T (each row belongs to one warp: read, then write) ----
+        // ---- block rows below: x L_JJ^T = p by forward substitution; lane c holds entry c of the row and
+        //      the reciprocal of L_JJ[c][c] (one division per pivot instead of one per row and pivot) ----
+        const double rdiag = 1.0 / Lf[(j0 + lane) * kLs + j0 + lane];
         for (int r = j0 + kNb + warp; r < kLeaf; r += kLeafThreads / 32) {
-            double acc = 0.0;
-            for (int k = 0; k <= lane; ++k) acc += Lf[r * kLs + j0 + k] * Wj[lane * kWs + k];
-            __syncwarp();
-            Lf[r * kLs + j0 + lane] = acc;
+            double p = Lf[r * kLs + j0 + lane];
+#pragma unroll 4
+            for (int c = 0; c < kNb; ++c) {
+                if (lane == c) p = p * rdiag;
+                const double x = __shfl_sync(0xffffffffu, p, c);
+                if (lane > c) p -= x * Lf[(j0 + lane) * kLs + j0 + c];          // L_JJ[lane][c]
+            }
+            Lf[r * kLs + j0 + lane] = p;
         }
         __syncthreads();
         // ---- trailing update: L[r][c] -= sum_k X[r][k] X[c][k], c <= r ----
@@ -125,64 +114,91 @@ chol_leaf_kernel(double* __restrict__ A, int64_t lda, int m, double* __restrict_
         }
         __syncthreads();
     }
-    const bool bad = s_bad != 0;
-
     // ---- the factor goes back to A ----
-    if (!bad)
+    if (!s_bad)
         for (int r = warp; r < m; r += kLeafThreads / 32)
             for (int c = lane; c <= r; c += 32) A[r * lda + c] = Lf[r * kLs + c];
+}
 
-    // ---- off-diagonal blocks of the inverse, in the place of L's ----
-    if (!bad) {
-        for (int I = 1; I < kLeaf / kNb; ++I) {
-            for (int J = 0; J < I; ++J) {
-                // T = sum_{K=J}^{I-1} L[I][K] * W[K][J]; two elements per thread (rows tid/32 and +16)
-                double t0 = 0.0, t1 = 0.0;
-                const int r0 = warp, r1 = warp + 16;
-                for (int K = J; K < I; ++K) {
-                    const double* Lik = Lf + (I * kNb) * kLs + K * kNb;
-                    const double* Wkj = (K == J) ? (Wd + J * kNb * kWs) : (Lf + (K * kNb) * kLs + J * kNb);
-                    const int wp = (K == J) ? kWs : kLs;
-#pragma unroll 8
-                    for (int k = 0; k < kNb; ++k) {
-                        const double w = Wkj[k * wp + lane];
-                        t0 += Lik[r0 * kLs + k] * w;
-                        t1 += Lik[r1 * kLs + k] * w;
-                    }
-                }
-                Tb[r0 * kWs + lane] = t0;
-                Tb[r1 * kWs + lane] = t1;
-                __syncthreads();
-                // W[I][J] = -W[I][I] * T
-                const double* Wi = Wd + I * kNb * kWs;
-                double o0 = 0.0, o1 = 0.0;
-                for (int k = 0; k <= r1; ++k) {
-                    const double tv = Tb[k * kWs + lane];
-                    if (k <= r0) o0 -= Wi[r0 * kWs + k] * tv;
-                    o1 -= Wi[r1 * kWs + k] * tv;
-                }
-                Lf[(I * kNb + r0) * kLs + J * kNb + lane] = o0;
-                Lf[(I * kNb + r1) * kLs + J * kNb + lane] = o1;
-                __syncthreads();
-            }
+// Rows below a factored leaf: P <- P L^-T for the n_rows x m block P (row pitch ldp), L the m x m lower
+// triangular factor at `L` (row pitch ldl), m <= 128 - the paper's OOC_TRSM step for one 128-column
+// sub-step, by blocked forward substitution (nothing is inverted, so the backward error does not depend on
+// the condition of L's diagonal blocks).  A thread block holds L and 64 rows of P in shared memory; per
+// 32-column block J: (a) x_J L_JJ^T = p_J row by row, a thread per row with the row in registers (L_JJ
+// is read by every lane at the same address; its diagonal enters as reciprocals), then (b) the blocks to its right lose x_J L_KJ^T, every warp
+// taking a share of the columns (two rows per lane, the L values again broadcast).
+constexpr int kTrsmRows = 64;
+constexpr int kTrsmThreads = 256;
+constexpr int kTrsmSmem = (kLeaf * kLs + kTrsmRows * kLs) * int(sizeof(double));
+
+template <int kCols>    // columns of the update a warp takes: 12, 8 or 4 (96, 64 or 32 columns over 8 warps)
+__device__ __forceinline__ void trsm_update(const double* __restrict__ Ls, double* __restrict__ Xs, int j0, int warp, int lane) {
+    const int c0 = j0 + kNb + warp * kCols;                       // this warp's first column
+    double acc[2][kCols];
+#pragma unroll
+    for (int e = 0; e < kCols; ++e) acc[0][e] = acc[1][e] = 0.0;
+#pragma unroll 4
+    for (int k = 0; k < kNb; ++k) {
+        const double x0 = Xs[lane * kLs + j0 + k], x1 = Xs[(lane + 32) * kLs + j0 + k];
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) {
+            const double l = Ls[(c0 + e) * kLs + j0 + k];          // same address in every lane
+            acc[0][e] += x0 * l;
+            acc[1][e] += x1 * l;
         }
     }
+#pragma unroll
+    for (int e = 0; e < kCols; ++e) {
+        Xs[lane * kLs + c0 + e] -= acc[0][e];
+        Xs[(lane + 32) * kLs + c0 + e] -= acc[1][e];
+    }
+}
 
-    // ---- the inverse goes to W (zeros above the diagonal and beyond m) ----
-    for (int r = warp; r < kLeaf; r += kLeafThreads / 32)
-        for (int c = lane; c < kLeaf; c += 32) {
-            double w = 0.0;
-            if (!bad && r < m && c <= r)
-                w = ((r / kNb) == (c / kNb)) ? Wd[(r / kNb) * kNb * kWs + (r % kNb) * kWs + (c % kNb)] : Lf[r * kLs + c];
-            W[r * kLeaf + c] = w;
+__global__ void __launch_bounds__(kTrsmThreads)
+trsm_rows_kernel(const double* __restrict__ L, int64_t ldl, int m, double* __restrict__ P, int64_t ldp, int64_t n_rows) {
+    extern __shared__ double trsm_smem[];
+    double* Ls = trsm_smem;                                        // 128 x 129: lower triangle of L, identity beyond m
+    double* Xs = trsm_smem + kLeaf * kLs;                          // 64 x 129: this block's rows of P
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t row0 = int64_t(blockIdx.x) * kTrsmRows;
+    for (int r = warp; r < kLeaf; r += kTrsmThreads / 32)
+        for (int c = lane; c < kLeaf; c += 32)
+            Ls[r * kLs + c] = (r < m && c <= r) ? L[r * ldl + c] : ((r == c) ? 1.0 : 0.0);
+    for (int r = warp; r < kTrsmRows; r += kTrsmThreads / 32)
+        for (int c = lane; c < kLeaf; c += 32)
+            Xs[r * kLs + c] = (row0 + r < n_rows && c < m) ? P[(row0 + r) * ldp + c] : 0.0;
+    __syncthreads();
+    // The diagonal of L is replaced by its reciprocals (one division per pivot for the whole block); the
+    // padding column of each row of Ls is free for that.
+    if (tid < kLeaf) Ls[tid * kLs + kLeaf] = 1.0 / Ls[tid * kLs + tid];
+    __syncthreads();
+    for (int J = 0; J < kLeaf / kNb; ++J) {
+        const int j0 = J * kNb;
+        if (tid < kTrsmRows) {                                     // (a) a row per thread
+            double p[kNb];
+#pragma unroll
+            for (int c = 0; c < kNb; ++c) p[c] = Xs[tid * kLs + j0 + c];
+#pragma unroll
+            for (int c = 0; c < kNb; ++c) {
+                p[c] = p[c] * Ls[(j0 + c) * kLs + kLeaf];
+#pragma unroll
+                for (int d = c + 1; d < kNb; ++d) p[d] -= p[c] * Ls[(j0 + d) * kLs + j0 + c];
+            }
+#pragma unroll
+            for (int c = 0; c < kNb; ++c) Xs[tid * kLs + j0 + c] = p[c];
         }
+        __syncthreads();
+        if (J == 0) trsm_update<12>(Ls, Xs, j0, warp, lane);       // (b)
+        else if (J == 1) trsm_update<8>(Ls, Xs, j0, warp, lane);
+        else if (J == 2) trsm_update<4>(Ls, Xs, j0, warp, lane);
+        __syncthreads();
+    }
+    for (int r = warp; r < kTrsmRows; r += kTrsmThreads / 32)
+        for (int c = lane; c < m; c += 32)
+            if (row0 + r < n_rows) P[(row0 + r) * ldp + c] = Xs[r * kLs + c];
 }
 
 struct CholWorkspace {
-    double* w = nullptr;          // (block / 128) inverses, 128 x 128 each
-    size_t w_bytes = 0;
-    double* t = nullptr;          // N x 128 staging of a solved column block
-    size_t t_bytes = 0;
     long long* info = nullptr;
     cudaStream_t panel_stream = nullptr;   // panel factorisations run here, ahead of the trailing update
     cudaEvent_t ev_panel = nullptr, ev_rest = nullptr;
@@ -227,12 +243,6 @@ extern "C" int cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, 
     CholWorkspace& ws = g_ws[ds->device];
     {
         std::lock_guard<std::mutex> l2(g_chol_mu);
-        void* p = ws.w;
-        if ((rc = ensure_device_bytes(&p, &ws.w_bytes, size_t(block / kLeaf) * kLeaf * kLeaf * sizeof(double))) != SYRK_OK) return rc;
-        ws.w = static_cast<double*>(p);
-        p = ws.t;
-        if ((rc = ensure_device_bytes(&p, &ws.t_bytes, size_t(N) * kLeaf * sizeof(double))) != SYRK_OK) return rc;
-        ws.t = static_cast<double*>(p);
         if (!ws.info && cudaMalloc(&ws.info, sizeof(long long)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
         if (!ws.panel_stream) {
             int lo = 0, hi = 0;
@@ -245,7 +255,8 @@ extern "C" int cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, 
         }
         static bool leaf_configured[64] = {};
         if (!leaf_configured[ds->device]) {
-            if (cudaFuncSetAttribute(chol_leaf_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLeafSmem) != cudaSuccess) {
+            if (cudaFuncSetAttribute(chol_leaf_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLeafSmem) != cudaSuccess ||
+                cudaFuncSetAttribute(trsm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTrsmSmem) != cudaSuccess) {
                 cudaGetLastError(); return SYRK_ERR_CUDA;
             }
             leaf_configured[ds->device] = true;
@@ -266,16 +277,15 @@ extern "C" int cholesky_lower(int64_t N, double* A, int64_t lda, int64_t block, 
         // ---- panel [o, o + bb) on the panel stream: factor, solve the rows below ----
         for (int64_t cj = o; cj < o + bb; cj += kLeaf) {
             const int m = int(std::min<int64_t>(kLeaf, o + bb - cj));
-            double* Wj = ws.w + size_t((cj - o) / kLeaf) * kLeaf * kLeaf;
-            chol_leaf_kernel<<<1, kLeafThreads, kLeafSmem, sp>>>(A + cj * lda + cj, lda, m, Wj, ws.info, cj);
+            chol_leaf_kernel<<<1, kLeafThreads, kLeafSmem, sp>>>(A + cj * lda + cj, lda, m, ws.info, cj);
             if (cudaGetLastError() != cudaSuccess) return SYRK_ERR_CUDA;
             const int64_t below = N - (cj + m);
             if (below <= 0) continue;
             double* panel = A + (cj + m) * lda + cj;              // rows below the leaf, its m columns
-            // solve: panel <- panel * L_jj^-T  (through the staging buffer: the product is not in place)
-            if ((rc = gemm_nt(ds, below, m, m, panel, lda, Wj, kLeaf, ws.t, kLeaf, 1.0, 0.0, sp)) != SYRK_OK) return rc;
-            if (!chk(cudaMemcpy2DAsync(panel, size_t(lda) * 8, ws.t, size_t(kLeaf) * 8, size_t(m) * 8, size_t(below),
-                                       cudaMemcpyDeviceToDevice, sp))) return SYRK_ERR_CUDA;
+            // solve in place: panel <- panel * L_jj^-T by forward substitution
+            trsm_rows_kernel<<<unsigned((below + kTrsmRows - 1) / kTrsmRows), kTrsmThreads, kTrsmSmem, sp>>>(
+                A + cj * lda + cj, lda, m, panel, lda, below);
+            if (cudaGetLastError() != cudaSuccess) return SYRK_ERR_CUDA;
             const int64_t rem = o + bb - (cj + m);                // panel columns still to be updated
             if (rem <= 0) continue;
             // inside the panel: square block [cj+m, o+bb)^2, lower triangle
@@ -330,8 +340,6 @@ namespace tbsyrk {
 void release_cholesky_workspaces() {
     std::lock_guard<std::mutex> l2(g_chol_mu);
     for (CholWorkspace& ws : g_ws) {
-        if (ws.w) cudaFree(ws.w);
-        if (ws.t) cudaFree(ws.t);
         if (ws.info) cudaFree(ws.info);
         if (ws.panel_stream) cudaStreamDestroy(ws.panel_stream);
         if (ws.ev_panel) cudaEventDestroy(ws.ev_panel);
