@@ -306,6 +306,23 @@ int syrk_lower_bf16_static(int64_t N, int64_t M,
 int syrk_lower_bf16_static_status(void);
 
 /*
+ * The lower triangle in packed form, for exchanging it between GPUs (no counterpart in the paper, which
+ * names parallel algorithms as future work).  Packed order: row i holds its i + 1 entries at
+ * [i (i + 1) / 2, (i + 1) (i + 2) / 2), N (N + 1) / 2 elements of C's type in all (binary64 for
+ * SYRK_DTYPE_F64, binary32 otherwise).  All pointers are DEVICE pointers; both calls only enqueue.
+ *   syrk_pack_lower:          packed[i (i + 1) / 2 + j] <- C[i][j] for every j <= i.
+ *   syrk_unpack_lower_axpby:  for the packed entries first .. first + count - 1, whose values are in
+ *                             packed[0 .. count): C[i][j] <- value + beta * C[i][j]  (beta == 0: C not read).
+ * Used by the K-sharded multi-GPU update: every GPU holds a block of columns of A, computes alpha times
+ * its own A_r A_r^T with syrk_lower (the sum over k of Algorithm 1 splits over the blocks), the packed
+ * triangles are summed across GPUs by one reduce-scatter, and each GPU adds beta times its share of C.
+ * SYRK_ERR_SIZE for a range outside the triangle, SYRK_ERR_LD for ldc < N.
+ */
+int syrk_pack_lower(int64_t N, const void* C, int64_t ldc, int dtype, void* packed, void* stream);
+int syrk_unpack_lower_axpby(int64_t N, int64_t first, int64_t count, const void* packed, double beta,
+                            void* C, int64_t ldc, int dtype, void* stream);
+
+/*
  * Cholesky factorisation by Large Block Cholesky (Algorithm 5 of the paper, LBC): replaces the
  * lower triangle of the symmetric positive definite FP64 matrix A (device pointer, row-major
  * N x N, row pitch lda >= N) by L with A = L * L^T.  Entries above the diagonal are never read

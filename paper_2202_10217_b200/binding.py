@@ -30,7 +30,7 @@ MAX_SEG, MAX_TILE = 8, 16
 
 EXPORTS = [
     "syrk_lower", "syrk_lower_tn", "syrk_ex", "syr2k_lower", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_plan_prepare_stream", "syrk_effective_schedule",
-    "syrk_lower_bf16_static_status", "syrk_set_host_pipeline", "syrk_host_pipeline_for", "syrk_shutdown", "syrk_last_status",
+    "syrk_lower_bf16_static_status", "syrk_set_host_pipeline", "syrk_host_pipeline_for", "syrk_pack_lower", "syrk_unpack_lower_axpby", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_set_f64_tail_split", "syrk_set_f64_launch", "syrk_get_schedule_stats",
     "syrk_probe_f64_mma_peak", "syrk_selftest_bounded_wait", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
     "tbs_plan_build", "tbs_plan_balance", "tbs_plan_num_items", "tbs_plan_item", "tbs_plan_free", "tbs_plan_simulate",
@@ -92,6 +92,10 @@ def lib() -> ctypes.CDLL:
         L.syrk_set_host_pipeline.argtypes = [ci]
         L.syrk_host_pipeline_for.restype = ci
         L.syrk_host_pipeline_for.argtypes = [i64, i64, ci]
+        L.syrk_pack_lower.restype = ci
+        L.syrk_pack_lower.argtypes = [i64, vp, i64, ci, vp, vp]
+        L.syrk_unpack_lower_axpby.restype = ci
+        L.syrk_unpack_lower_axpby.argtypes = [i64, i64, i64, vp, dbl, vp, i64, ci, vp]
         L.syrk_shutdown.restype = None
         L.syrk_shutdown.argtypes = []
         L.syrk_last_status.restype = ci
@@ -278,6 +282,23 @@ def syrk_host_pipeline_for(N: int, M: int, c_is_page_locked: bool) -> int:
     if r < 0:
         raise SyrkError(r)
     return r
+
+
+def syrk_pack_lower(N: int, C, ldc: int, dtype: int, packed, stream: Optional[int] = None) -> None:
+    """packed[i (i + 1) / 2 + j] <- C[i][j], j <= i (device pointers; enqueues)."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().syrk_pack_lower(N, _ptr(C), ldc, dtype, _ptr(packed), stream))
+
+
+def syrk_unpack_lower_axpby(N: int, first: int, count: int, packed, beta: float, C, ldc: int, dtype: int,
+                            stream: Optional[int] = None) -> None:
+    """C[i][j] <- packed value + beta * C[i][j] for the packed entries first .. first + count - 1."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().syrk_unpack_lower_axpby(N, first, count, _ptr(packed), float(beta), _ptr(C), ldc, dtype, stream))
 
 
 def syrk_lower_bf16_static_status() -> int:

@@ -401,9 +401,58 @@ __global__ void pack_diag_blocks_kernel(int64_t row0, int64_t row1, int64_t band
     }
 }
 
+// Entries [first, first + count) of the packed lower triangle (row i starts at i (i + 1) / 2):
+// C[i][j] <- packed[idx - first] + beta * C[i][j]  (C not read when beta == 0).
+template <typename T>
+__global__ void unpack_lower_axpby_kernel(int64_t first, int64_t count, const T* __restrict__ packed, double beta,
+                                          T* __restrict__ C, int64_t ldc) {
+    for (int64_t e = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; e < count; e += int64_t(gridDim.x) * blockDim.x) {
+        const int64_t idx = first + e;
+        int64_t i = int64_t((sqrt(8.0 * double(idx) + 1.0) - 1.0) * 0.5);
+        while (i * (i + 1) / 2 > idx) --i;                 // the square root may be off by one either way
+        while ((i + 1) * (i + 2) / 2 <= idx) ++i;
+        const int64_t j = idx - i * (i + 1) / 2;
+        T* c = C + i * ldc + j;
+        *c = (beta == 0.0) ? packed[e] : T(double(packed[e]) + beta * double(*c));
+    }
+}
+
 }  // namespace
 
 extern "C" {
+
+int syrk_pack_lower(int64_t N, const void* C, int64_t ldc, int dtype, void* packed, void* stream) {
+    if (!known_dtype(dtype)) return SYRK_ERR_DTYPE;
+    if (N < 0) return SYRK_ERR_SIZE;
+    if (N == 0) return SYRK_OK;
+    if (ldc < N) return SYRK_ERR_LD;
+    if (!C || !packed) return SYRK_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dim3 grid(unsigned(std::min<int64_t>(64, (N + 255) / 256)), unsigned(std::min<int64_t>(N, 32768)));
+    if (dtype == SYRK_DTYPE_F64)
+        pack_diag_blocks_kernel<double><<<grid, 256, 0, st>>>(0, N, N, static_cast<const double*>(C), ldc, static_cast<double*>(packed));
+    else
+        pack_diag_blocks_kernel<float><<<grid, 256, 0, st>>>(0, N, N, static_cast<const float*>(C), ldc, static_cast<float*>(packed));
+    return cudaGetLastError() == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
+int syrk_unpack_lower_axpby(int64_t N, int64_t first, int64_t count, const void* packed, double beta, void* C,
+                            int64_t ldc, int dtype, void* stream) {
+    if (!known_dtype(dtype)) return SYRK_ERR_DTYPE;
+    if (N < 0 || first < 0 || count < 0 || first + count > N * (N + 1) / 2) return SYRK_ERR_SIZE;
+    if (count == 0) return SYRK_OK;
+    if (ldc < N) return SYRK_ERR_LD;
+    if (!C || !packed) return SYRK_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const unsigned grid = unsigned(std::min<int64_t>((count + 255) / 256, 148 * 16));
+    if (dtype == SYRK_DTYPE_F64)
+        unpack_lower_axpby_kernel<double><<<grid, 256, 0, st>>>(first, count, static_cast<const double*>(packed), beta,
+                                                                static_cast<double*>(C), ldc);
+    else
+        unpack_lower_axpby_kernel<float><<<grid, 256, 0, st>>>(first, count, static_cast<const float*>(packed), beta,
+                                                               static_cast<float*>(C), ldc);
+    return cudaGetLastError() == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+}
 
 int syrk_lower(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha,
                double beta, int dtype, void* stream) {
