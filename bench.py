@@ -579,6 +579,46 @@ def run_ours(args, keys, headline, shape, rank: int, world: int, local_rank: int
         dist.destroy_process_group()
 
 
+# ---- K-sharded update over the ranks (strong scaling; the default N > 1 run is replicas) ----------------------------
+
+def run_kshard(args, key, shape, rank: int, world: int, local_rank: int):
+    """--kshard: one update of the workload with the inner dimension split over the ranks (every rank a
+    block of columns of A, one reduce-scatter of the packed lower triangles); a step is the whole
+    exchange-and-update, the value is the whole problem's flops over the slowest rank's time."""
+    import torch
+    import torch.distributed as dist
+    from paper_2202_10217_b200 import binding as B
+    from paper_2202_10217_b200 import distributed as D
+
+    torch.cuda.set_device(local_rank)
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29555")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", local_rank))
+    T = Timer(torch, local_rank, dist if world > 1 else None)
+    wl = shape or I.CONFIGS[key]
+    N, M, dtype = wl.N, wl.M, wl.dtype
+    k0, k1 = D.column_block(M, world, rank, dtype)
+    A_host = wl.make_A()                                      # every rank draws the same seeded matrix and keeps its block
+    _, dA = to_device(torch, np.ascontiguousarray(A_host[:, k0:k1]), dtype)
+    del A_host
+    cdt = torch.float64 if dtype == I.DTYPE_F64 else torch.float32
+    dC = torch.zeros((N, N), dtype=cdt, device="cuda")
+    chunk = D.packed_share(N, world, rank)[2]
+    ws = (torch.empty((N, N), dtype=cdt, device="cuda"), torch.zeros(world * chunk, dtype=cdt, device="cuda"))
+    call = lambda: D.syrk_lower_ksharded(N, k1 - k0, dA, max(k1 - k0, 1), dC, N, wl.alpha, wl.beta, dtype, workspace=ws)
+    ms_step, _, clocks = T.burst(call, args.steps, max(args.warmup, 3), flush=True)
+    assert B.syrk_last_status() == 0
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": wl.flops / (ms_step * 1e-3) * 1e-12, "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+                          "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": DTYPE_NAME[dtype],
+                          "data": "synthetic", "config": dict(config_of(key, shape), parallelism="k-sharded x%d" % world),
+                          "clocks": clocks, "exchange": {"collective": "reduce_scatter of the packed lower triangle",
+                                                         "bytes_per_rank": world * chunk * (8 if dtype == I.DTYPE_F64 else 4)}}))
+    dist.destroy_process_group()
+
+
 # ---- short device-timed runs for the profiler ------------------------------------------------------------------------
 
 def run_kernel_only(args, key, shape, rank: int, world: int, local_rank: int):
@@ -731,6 +771,9 @@ def main():
                          "square-block comparison schedule, or square blocks on CTA pairs")
     ap.add_argument("--syr2k", action="store_true",
                     help="with --kernel-only and an f64 workload: time syr2k_lower (rank-2k update) instead")
+    ap.add_argument("--kshard", action="store_true",
+                    help="split the inner dimension of the workload (default c4) over the ranks: K-sharded update with "
+                         "one reduce-scatter (strong scaling) instead of independent replicas")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     for flag, on in (("--schedule", args.schedule != "default"), ("--syr2k", args.syr2k), ("--batch", args.batch > 0),
@@ -752,6 +795,12 @@ def main():
             print(json.dumps({"impl": "reference", "unavailable": "the factorisation has no oracle timing leg; use --workload c5"}))
             return
         run_reference(args, headline, shape, rank)
+        return
+    if args.kshard:
+        key = "custom" if shape is not None else (args.workload or "c4")
+        if key in ("c5", "lbc"):
+            ap.error("--kshard takes a single-call workload")
+        run_kshard(args, key, shape, rank, world, local_rank)
         return
     if args.kernel_only:
         if rank == 0:
