@@ -65,15 +65,16 @@ def sweep_flops() -> int:
     return sum(n * (n + 1) * I.SWEEP_K for n in I.sweep_sizes(SWEEP_N, SWEEP_STEP))
 
 
-def config_of(key: str, shape: I.Workload | None = None) -> dict:
+def config_of(key: str, shape: I.Workload | None = None, world: int = 1) -> dict:
     """What a workload is, in words both arms print identically (no measured or device-side facts)."""
+    par = {"parallelism": "replicas only" if world > 1 else "1 gpu"}
     if key == "c5":
-        return {"workload": SWEEP_NAME, "calls_per_step": len(I.sweep_sizes(SWEEP_N, SWEEP_STEP)), "N": SWEEP_N,
-                "M": I.SWEEP_K, "alpha": -1.0, "beta": 1.0, "ldc": SWEEP_N, "l2": L2_LARGE}
+        return dict({"workload": SWEEP_NAME, "calls_per_step": len(I.sweep_sizes(SWEEP_N, SWEEP_STEP)), "N": SWEEP_N,
+                     "M": I.SWEEP_K, "alpha": -1.0, "beta": 1.0, "ldc": SWEEP_N, "l2": L2_LARGE}, **par)
     if key == "lbc":
-        return {"workload": "lbc_f64_%d" % SWEEP_N, "N": SWEEP_N, "l2": L2_LARGE}
+        return dict({"workload": "lbc_f64_%d" % SWEEP_N, "N": SWEEP_N, "l2": L2_LARGE}, **par)
     wl = shape or I.CONFIGS[key]
-    return {"workload": wl.name, "N": wl.N, "M": wl.M, "alpha": wl.alpha, "beta": wl.beta, "l2": L2_FLUSH}
+    return dict({"workload": wl.name, "N": wl.N, "M": wl.M, "alpha": wl.alpha, "beta": wl.beta, "l2": L2_FLUSH}, **par)
 
 
 class ClockSampler:
@@ -92,7 +93,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            time.sleep(0.15)                      # let the first samples arrive before the load starts
+            time.sleep(0.4)                       # let the first samples arrive before the load starts
         except Exception:
             self.proc = None
         return self
@@ -100,6 +101,7 @@ class ClockSampler:
     def __exit__(self, *exc):
         if self.proc is None:
             return
+        time.sleep(0.05)                          # one more sampling period, so that a short region is seen
         self.proc.terminate()                     # the exact process started above
         try:
             out, _ = self.proc.communicate(timeout=5)
@@ -122,9 +124,10 @@ class ClockSampler:
             for name, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        # "under load": samples drawing more than half of the largest power seen
-        top = max(power) if power else 0.0
-        load = [(c, w) for c, w in zip(sm, power) if w >= 0.5 * top]
+        # "under load": samples drawing more than half of the way from the lowest to the largest power seen
+        # (the sampler also sees the idle time before and after the region)
+        top, low = (max(power), min(power)) if power else (0.0, 0.0)
+        load = [(c, w) for c, w in zip(sm, power) if w >= low + 0.5 * (top - low)]
         return {"sm_mhz": float(np.median([c for c, _ in load])) if load else None, "sm_max_mhz": mx or None,
                 "reasons": sorted(reasons), "samples": len(sm), "samples_under_load": len(load),
                 "power_w_median": float(np.median([w for _, w in load])) if load else None,
@@ -188,7 +191,7 @@ def run_reference(args, key: str, shape, rank: int):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": DTYPE_NAME[dtype], "data": "synthetic",
-        "config": config_of(key, shape),
+        "config": config_of(key, shape, args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
                          "sample": "%s, once per step (%.3g flops)" % (words, flops)},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -202,6 +205,10 @@ def run_reference(args, key: str, shape, rank: int):
 # summarised under profiles/.  Valid only for the kernel source it was taken on: keyed by its SHA-256.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, kernel source file, sha256 of that file at capture time, square-schedule bytes or None)
+    "c2_f64_4096x4096": (832_195_584, "syrk_f64.cu", "dc0af5511d941afee99ca375ca5db108325e8474b096a5eaff9efcc6db1d6bef", 811_978_240),
+    "c3_bf16_16384x4096": (1_881_366_784, "syrk_bf16.cu", "b2b31371304f54522dd449d94e2448a596236a0881b9e215e356cf28aec88cd5", 3_712_474_624),
+    "c4_bf16_2048x262144": (1_159_163_136, "syrk_bf16_pair.cu", "1f007b0ed5552de540c0cf0f25685f828321404cc4f842d0dbfcbbdcc303fc01", 2_276_417_536),
+    "c5_call_n16384": (2_885_844_736, "syrk_f64.cu", "dc0af5511d941afee99ca375ca5db108325e8474b096a5eaff9efcc6db1d6bef", 2_724_991_232),
 }
 
 
@@ -561,7 +568,7 @@ def run_ours(args, keys, headline, shape, rank: int, world: int, local_rank: int
         "metric": head["metric"], "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": head["steps"],
         "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": head["dtype"], "data": "synthetic",
-        "config": dict(head["config"], parallelism="replicas only" if world > 1 else "1 gpu"),
+        "config": config_of(headline, shape, world),
         "schedule": head.get("schedule"),
         "clocks": head["clocks"],
         "value_sustained": head.get("value_sustained"), "sustained": head.get("sustained"),
