@@ -445,3 +445,45 @@ def test_host_buffer_entry_point_row_band_pipeline(dtype):
         iu = np.triu_indices(N, 1)
         assert np.array_equal(C[:, :N][iu], Cin[:, :N][iu])
         assert np.array_equal(C[:, N:], Cin[:, N:])
+
+
+@pytest.mark.parametrize("dtype", [B.DTYPE_F64, B.DTYPE_BF16_F32, B.DTYPE_E4M3_F32], ids=["f64", "bf16", "e4m3"])
+def test_host_buffer_entry_point_column_block_pipeline_with_page_locked_buffers(dtype):
+    """The same page-locked call as above with the column-block pipeline forced: A goes up in blocks of
+    columns, each block's update runs the device call's schedule (triangle blocks here: the file pins them)
+    while the next block travels, C comes down in bands afterwards.  A wide operand (several blocks, ragged
+    last one), ragged N, pitches, beta != 0; sampled entries plus whole rows at band and tile boundaries."""
+    import torch
+    N, M = {B.DTYPE_F64: (4100, 2300), B.DTYPE_BF16_F32: (4500, 9000), B.DTYPE_E4M3_F32: (4400, 17000)}[dtype]
+    assert B.syrk_host_pipeline_for(N, M, True) == B.HOST_ROW_BANDS and B.syrk_host_pipeline_for(N, M, False) == B.HOST_COLUMN_BLOCKS
+    A = make_A(N, M, dtype, seed=81)
+    lda, ldc = M + 32, N + 6
+    Abig = np.zeros((N, lda), dtype=A.dtype)
+    Abig[:, :M] = A
+    Cin = I.random_c(N, 82, dtype, ldc)
+    hA = torch.from_numpy(Abig.view(np.int16) if Abig.dtype == np.uint16 else Abig).pin_memory()
+    hC = torch.from_numpy(Cin.copy()).pin_memory()
+    alpha, beta = 0.5, -1.0
+    try:
+        B.syrk_set_host_pipeline(B.HOST_COLUMN_BLOCKS)
+        assert B.syrk_host_pipeline_for(N, M, True) == B.HOST_COLUMN_BLOCKS
+        B.syrk_lower_host(N, M, hA, lda, hC, ldc, alpha, beta, dtype)
+    finally:
+        B.syrk_set_host_pipeline(B.HOST_AUTO)
+    C = hC.numpy()
+    rng = np.random.default_rng(83)
+    ii = rng.integers(0, N, size=20000)
+    jj = (rng.random(20000) * (ii + 1)).astype(np.int64)
+    rows = np.array([0, 127, 128, 255, 256, 2047, 2048, 4095, 4096, N - 1])
+    rows = rows[rows < N]
+    ii = np.concatenate([ii] + [np.full(r + 1, r) for r in rows])
+    jj = np.concatenate([jj] + [np.arange(r + 1) for r in rows])
+    ref, bound = O.syrk_entries(ii, jj, A, None, alpha, 0.0, dtype)
+    ref = ref + beta * Cin[ii, jj].astype(np.float64)
+    tol = O.tolerance(M, bound, np.abs(Cin[ii, jj]), alpha, beta, dtype)
+    assert np.all(np.abs(C[ii, jj].astype(np.float64) - ref) <= tol)
+    iu = np.triu_indices(N, 1)
+    assert np.array_equal(C[:, :N][iu], Cin[:, :N][iu])
+    assert np.array_equal(C[:, N:], Cin[:, N:])
+    with pytest.raises(B.SyrkError):
+        B.syrk_set_host_pipeline(7)
