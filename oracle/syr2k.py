@@ -17,6 +17,9 @@ _LIB = os.path.join(_HERE, "libsyr2k_oracle.so")
 
 # Parity tolerance: |C_gpu - C_ref| <= TOL * 2M * (|alpha| Bd + |beta| |C_in|): 2M products per entry.
 TOL = 8.0 * 2.0 ** -53
+# ... and for the input types whose products are exact in binary32 and are accumulated in binary32 (bfloat16,
+# binary16, TF32, FP8 E4M3): the tolerance of the rank-k update on those types, again with 2M products.
+TOL_F32_ACC = 4.0 * 2.0 ** -24
 
 
 def build(force: bool = False) -> str:
@@ -65,8 +68,25 @@ def syr2k_lower(A: np.ndarray, B: np.ndarray, C_in, alpha: float, beta: float):
     return ref, bound
 
 
-def tolerance(M: int, bound, c_in_abs, alpha: float, beta: float):
+def syr2k_lower_typed(A: np.ndarray, B: np.ndarray, C_in, alpha: float, beta: float, dtype: int):
+    """The same reference for operands in one of the library's storage types (dtype codes of the rank-k
+    reference): both operands are decoded exactly to binary64 by that reference's decoder, a binary32 C_in
+    is widened exactly, and the binary64 definition above is applied (products of two decoded values have
+    at most 22 significant bits, so each product is exact; only the sums round, in binary64)."""
+    from . import syrk as _syrk
+    if dtype == _syrk.DTYPE_F64:
+        return syr2k_lower(A, B, C_in, alpha, beta)
+    A64, B64 = _syrk.widen(np.ascontiguousarray(A), dtype), _syrk.widen(np.ascontiguousarray(B), dtype)
+    C64 = None
+    if C_in is not None:
+        if C_in.dtype != np.float32:
+            raise ValueError("C must be float32 for this input type")
+        C64 = np.ascontiguousarray(C_in, dtype=np.float64)
+    return syr2k_lower(A64, B64, C64, alpha, beta)
+
+
+def tolerance(M: int, bound, c_in_abs, alpha: float, beta: float, f32_accumulate: bool = False):
     t = abs(alpha) * np.asarray(bound, dtype=np.float64)
     if beta != 0.0 and c_in_abs is not None:
         t = t + abs(beta) * np.asarray(c_in_abs, dtype=np.float64)
-    return TOL * 2 * max(int(M), 1) * t
+    return (TOL_F32_ACC if f32_accumulate else TOL) * 2 * max(int(M), 1) * t

@@ -49,6 +49,8 @@ def _load():
         lib.oracle_syrk_entries.argtypes = [i64, vp, vp, i64, i64, vp, i64, vp, i64,
                                             dbl, dbl, ctypes.c_int, vp, vp]
         lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_widen.restype = ctypes.c_int
+        lib.oracle_widen.argtypes = [i64, i64, vp, i64, ctypes.c_int, vp]
         _lib = lib
     return _lib
 
@@ -66,6 +68,18 @@ def _check_inputs(A: np.ndarray, C_in, dtype: int):
     if C_in is not None and (C_in.dtype != want_c or C_in.ndim != 2
                              or C_in.strides[1] != C_in.itemsize):
         raise ValueError("C must be a row-major 2-D array of %s" % want_c.__name__)
+
+
+def widen(A: np.ndarray, dtype: int) -> np.ndarray:
+    """The operand as binary64 values, every element decoded exactly from its storage format (bf16 or
+    binary16 bit patterns, binary32 read as TF32, FP8 E4M3 bytes) by the reference's own decoder."""
+    _check_inputs(A, None, dtype)
+    N, M = A.shape
+    out = np.empty((N, M), dtype=np.float64)
+    lda = max(A.strides[0] // A.itemsize, M, 1) if A.size > 0 else max(M, 1)
+    if _load().oracle_widen(N, M, A.ctypes.data, lda, dtype, out.ctypes.data) != 0:
+        raise ValueError("oracle_widen rejected its arguments")
+    return out
 
 
 def syrk_lower(A: np.ndarray, C_in, alpha: float, beta: float, dtype: int):

@@ -160,6 +160,17 @@ int oracle_syrk_entries(int64_t P, const int64_t* I, const int64_t* J,
     return 0;
 }
 
+/* The N x M operand (row pitch lda) widened element by element to binary64, exactly, by the functions above:
+ * dst is N x M, dense.  For references of other updates on the same input types (the rank-2k update), so
+ * that every reference reads a storage format through the one pinned decoder.  Returns 0, or -1 on a bad
+ * argument. */
+int oracle_widen(int64_t N, int64_t M, const void* A, int64_t lda, int dtype, double* dst) {
+    if (N < 0 || M < 0 || lda < (M > 1 ? M : 1) || dtype < 0 || dtype > 4 || ((N > 0 && M > 0) && (!A || !dst))) return -1;
+    for (int64_t r = 0; r < N; ++r)
+        for (int64_t k = 0; k < M; ++k) dst[r * M + k] = a_at(A, lda, dtype, r, k);
+    return 0;
+}
+
 /* Host threads the loops above run on. */
 int oracle_num_threads(void) {
 #ifdef _OPENMP

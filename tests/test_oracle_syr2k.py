@@ -109,3 +109,48 @@ def test_pitches():
     r1, _ = R.syr2k_lower(A, B, None, 1.0, 0.0)
     r2, _ = R.syr2k_lower(np.ascontiguousarray(A), np.ascontiguousarray(B), None, 1.0, 0.0)
     assert np.array_equal(lower(r1), lower(r2))
+
+
+def test_typed_reference_decodes_through_the_pinned_decoder_and_reduces_to_the_rank_k_reference():
+    """Operands in a storage type are decoded by the rank-k reference's decoder (pinned pattern by pattern in
+    test_oracle_syrk.py) and then go through the binary64 definition.  Pins: the decoder's output squared is
+    the rank-k reference of a one-column problem, bit for bit, for every 8-bit pattern and for sampled 16-bit
+    patterns; B = A gives twice the rank-k reference of the same type, bit for bit (all sums are of exactly
+    representable products, doubling is exact); the exchange of A and B changes no bit."""
+    from oracle import syrk as O
+    from paper_2202_10217_b200 import inputs as I
+    allbytes = np.arange(256, dtype=np.uint8).reshape(256, 1)
+    w = O.widen(allbytes, O.DTYPE_E4M3_F32)
+    ref, _ = O.syrk_lower(allbytes, None, 1.0, 0.0, O.DTYPE_E4M3_F32)
+    d = np.diag(ref)
+    ok = ~np.isnan(w[:, 0])
+    assert np.array_equal(d[ok], (w[:, 0] ** 2)[ok]) and np.isnan(d[~ok]).all() and (~ok).sum() == 2
+    for dtype in (O.DTYPE_BF16_F32, O.DTYPE_F16_F32):
+        pats = np.random.default_rng(5).integers(0, 1 << 16, size=(400, 1)).astype(np.uint16)
+        w = O.widen(pats, dtype)[:, 0]
+        d = np.diag(O.syrk_lower(pats, None, 1.0, 0.0, dtype)[0])
+        fin = np.isfinite(w)
+        assert np.array_equal(d[fin], (w ** 2)[fin])
+    x = np.array([[1.0 + 2.0 ** -10, 1.0 + 2.0 ** -11 + 2.0 ** -12]], dtype=np.float32)      # TF32 keeps 10 fraction bits
+    assert np.array_equal(O.widen(x, O.DTYPE_TF32_F32), np.array([[1.0 + 2.0 ** -10, 1.0]]))
+    N, M = 37, 29
+    for dtype, gen in ((O.DTYPE_BF16_F32, I.normal_bf16), (O.DTYPE_F16_F32, I.normal_f16), (O.DTYPE_TF32_F32, I.normal_f32),
+                       (O.DTYPE_E4M3_F32, I.normal_e4m3)):
+        A, Bm = gen(N, M, 3), gen(N, M, 4)
+        Cin = I.random_c(N, 5, dtype)
+        il = np.tril_indices(N)
+        twice, _ = R.syr2k_lower_typed(A, A, None, 1.0, 0.0, dtype)
+        once, _ = O.syrk_lower(A, None, 1.0, 0.0, dtype)
+        assert np.array_equal(twice[il], 2.0 * once[il])
+        ab, bd1 = R.syr2k_lower_typed(A, Bm, Cin, 0.5, -1.0, dtype)
+        ba, bd2 = R.syr2k_lower_typed(Bm, A, Cin, 0.5, -1.0, dtype)
+        assert np.array_equal(ab[il], ba[il]) and np.array_equal(bd1[il], bd2[il])
+        # against exact rational arithmetic on the decoded values (a k-outermost loop nest of its own)
+        from fractions import Fraction
+        A64, B64 = O.widen(A, dtype), O.widen(Bm, dtype)
+        for (i, j) in [(0, 0), (5, 2), (36, 35), (20, 20)]:
+            s = Fraction(0)
+            for k in range(M):
+                s += Fraction(float(A64[i, k])) * Fraction(float(B64[j, k])) + Fraction(float(B64[i, k])) * Fraction(float(A64[j, k]))
+            exact = Fraction(0.5) * s - Fraction(float(Cin[i, j]))
+            assert abs(Fraction(float(ab[i, j])) - exact) <= Fraction(2 * M * 2.0 ** -53) * Fraction(float(bd1[i, j]) + abs(float(Cin[i, j])))
