@@ -738,25 +738,26 @@ def run_batched(args, wl):
 
 
 def run_syr2k(args, wl):
-    """--kernel-only --syr2k: the rank-2k update alpha (A B^T + B A^T) + beta C of the workload's shape
-    (binary64; B drawn like A from the next seed); 2 N (N+1) M flops."""
+    """--kernel-only --syr2k: the rank-2k update alpha (A B^T + B A^T) + beta C of the workload's shape and type
+    (B drawn like A from the next seed); 2 N (N+1) M flops."""
     import torch
     from paper_2202_10217_b200 import binding as B
 
-    N, M = wl.N, wl.M
-    dA = torch.from_numpy(wl.make_A()).cuda()
-    dB = torch.from_numpy(I.Workload(wl.name, N, M, wl.dtype, wl.alpha, wl.beta, wl.seed + 1, wl.dist, wl.std).make_A()).cuda()
-    dC = torch.zeros((N, N), dtype=torch.float64, device="cuda")
+    N, M, dtype = wl.N, wl.M, wl.dtype
+    _, dA = to_device(torch, wl.make_A(), dtype)
+    _, dB = to_device(torch, I.Workload(wl.name, N, M, dtype, wl.alpha, wl.beta, wl.seed + 1, wl.dist, wl.std).make_A(), dtype)
+    dC = torch.zeros((N, N), dtype=torch.float64 if dtype == I.DTYPE_F64 else torch.float32, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    call = lambda: B.syr2k_lower_ex(N, M, dA, M, dB, M, dC, N, wl.alpha, wl.beta, dtype)
     for _ in range(max(args.warmup, 1)):
-        B.syr2k_lower(N, M, dA, M, dB, M, dC, N, wl.alpha, wl.beta)
+        call()
     torch.cuda.synchronize()
     times = []
     for _ in range(args.steps):
         flush.zero_()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        B.syr2k_lower(N, M, dA, M, dB, M, dC, N, wl.alpha, wl.beta)
+        call()
         e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
@@ -764,7 +765,7 @@ def run_syr2k(args, wl):
     ms = float(np.mean(times))
     print(json.dumps({"metric": "syr2k_tflops_2N(N+1)M", "value": 2 * wl.flops / (ms * 1e-3) * 1e-12, "unit": UNIT,
                       "n_gpus": 1, "steps": args.steps, "ms_per_step": ms, "kernel_only": True,
-                      "config": {"workload": wl.name, "N": N, "M": M, "op": "syr2k"}}))
+                      "config": {"workload": wl.name, "N": N, "M": M, "op": "syr2k", "dtype": DTYPE_NAME[dtype]}}))
 
 
 def main():
@@ -790,7 +791,7 @@ def main():
                     help="with --kernel-only: the library's default rule, triangle blocks at every size, the "
                          "square-block comparison schedule, or square blocks on CTA pairs")
     ap.add_argument("--syr2k", action="store_true",
-                    help="with --kernel-only and an f64 workload: time syr2k_lower (rank-2k update) instead")
+                    help="with --kernel-only: time syr2k_lower_ex (rank-2k update of the workload's type) instead")
     ap.add_argument("--kshard", action="store_true",
                     help="split the inner dimension of the workload (default c4) over the ranks: K-sharded update with "
                          "one reduce-scatter (strong scaling) instead of independent replicas")

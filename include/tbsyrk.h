@@ -197,6 +197,25 @@ int syr2k_lower(int64_t N, int64_t M,
                 double alpha, double beta, void* stream);
 
 /*
+ * The rank-2k update for every dtype of the library:
+ *
+ *     C[i][j] = alpha * sum_k (A[i][k] * B[j][k] + B[i][k] * A[j][k]) + beta * C[i][j]     0 <= j <= i < N,
+ *
+ * A and B of the element type `dtype` names, C binary64 (SYRK_DTYPE_F64, which is syr2k_lower) or binary32.
+ * For the tcgen05 types the work list is the rank-k update's (Algorithm 4 / Section 5.1.4: triangle blocks of
+ * k = 3 segments, or the square list when that schedule is set); a pipeline stage carries the block's rows of
+ * both operands and every accumulator takes both products, A_x B_y^T and B_x A_y^T, in binary32 (each
+ * product exact).  K-splits as for syrk_lower; operands that break the TMA rules (16-byte aligned, pitch a
+ * multiple of 16 bytes) take a plain-load kernel.  The CTA-pair schedule has no rank-2k form: the default rule
+ * runs triangle blocks here at every size.  Arguments, quick returns, ownership and errors as for syr2k_lower.
+ */
+int syr2k_lower_ex(int64_t N, int64_t M,
+                   const void* A, int64_t lda,
+                   const void* B, int64_t ldb,
+                   void* C, int64_t ldc,
+                   double alpha, double beta, int dtype, void* stream);
+
+/*
  * A strided batch of independent updates of the same shape:
  *
  *     C_b[i][j] = alpha * sum_k A_b[i][k] * A_b[j][k] + beta * C_b[i][j]    0 <= j <= i < N, 0 <= b < batch,

@@ -531,6 +531,49 @@ int syr2k_lower(int64_t N, int64_t M, const void* A, int64_t lda, const void* B,
                ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
+int syr2k_lower_ex(int64_t N, int64_t M, const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc,
+                   double alpha, double beta, int dtype, void* stream) {
+    if (dtype == SYRK_DTYPE_F64) return syr2k_lower(N, M, A, lda, B, ldb, C, ldc, alpha, beta, stream);
+    int rc = validate(N, M, A, lda, C, ldc, dtype);
+    if (rc != SYRK_OK || N == 0) return rc;
+    if (ldb < std::max<int64_t>(1, M)) return SYRK_ERR_LD;
+    if (M > 0 && !B) return SYRK_ERR_NULL;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceState* ds = nullptr;
+    rc = get_device_state(&ds);
+    if (rc != SYRK_OK) return rc;
+    if (alpha == 0.0 || M == 0) {
+        if (beta == 1.0) return SYRK_OK;
+        return launch_scale_lower(dtype, N, C, ldc, beta, st) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+    }
+    if (!tma_ok(A, lda, dtype) || !tma_ok(B, ldb, dtype))
+        return launch_syr2k_plain_f32(dtype, N, M, A, lda, B, ldb, static_cast<float*>(C), ldc, float(alpha), float(beta), st) ==
+                       cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+    // The work list of the rank-k update under the current setting (triangle blocks k = 3, or squares): same
+    // items, each stage carrying the items' rows of both operands.  The CTA-pair kernel has no rank-2k form.
+    DevicePlan* dp = nullptr;
+    rc = get_device_plan(ds, N, dtype, &dp);
+    if (rc != SYRK_OK) return rc;
+    const KernelShape ks = kernel_shape(dtype);
+    const int split = pick_split_k(ds, dp, M, ks.bk);
+    void* d_partial = nullptr;
+    if (split > 1) {
+        const size_t want = size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float);
+        if ((rc = workspace_for_stream(ds, st, want, &d_partial)) != SYRK_OK) return rc;
+    }
+    CUtensorMap ta, tb, tmc;
+    if ((rc = encode_tensor_map_2d(&ta, dtype, A, N, M, lda, ks.tile, ks.bk)) != SYRK_OK) return rc;
+    if ((rc = encode_tensor_map_2d(&tb, dtype, B, N, M, ldb, ks.tile, ks.bk)) != SYRK_OK) return rc;
+    const bool c_tma = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
+                       encode_tensor_map_c_f32(&tmc, C, N, ldc, bf16_store_box()) == SYRK_OK;
+    return launch_syrk_bf16(ta, c_tma ? &tmc : nullptr, dp->d_items, int64_t(dp->plan.items.size()), N, M,
+                            static_cast<float*>(C), ldc, float(alpha), float(beta), split, static_cast<float*>(d_partial),
+                            dp->d_tile_base, dp->total_tiles, dp->d_cta_begin, dp->n_ctas, 0, dtype - SYRK_DTYPE_BF16_F32,
+                            status_for_stream(ds, st), ds->sm_count, st, 0, 0, 0, &tb) == cudaSuccess
+               ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
 int syrk_lower_batched(int64_t batch, int64_t N, int64_t M, const void* A, int64_t lda, int64_t stride_a,
                        void* C, int64_t ldc, int64_t stride_c, double alpha, double beta, int dtype, void* stream) {
     if (batch < 0 || batch >= (int64_t(1) << 31)) return SYRK_ERR_SIZE;

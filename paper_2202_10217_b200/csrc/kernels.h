@@ -57,6 +57,8 @@ int f64_stages();
 // over that array (64 x 64 for the 16-bit kinds, 32 x 32 for TF32, 128 x 128 for FP8).  `a_kind`:
 // 0 bfloat16; 1 binary32 read as TF32 (N x M order: boxes of 128 rows x 32 columns); 2 FP8 E4M3 bytes
 // (boxes of 128 rows x 128 columns); 3 IEEE binary16 (boxes as for bfloat16).
+// `tmB` (N x M operands, lower triangle, no batch): the rank-2k update alpha (A B^T + B A^T) + beta C; `tmB`
+// is the map of B with the boxes of `tmA`; a stage then holds the segments of both operands (two stages).
 // `batch` > 0: strided batch (3-D maps as for the FP64 kernel); the units are then (matrix, item)
 // pairs dealt round-robin, split_k must be 1.  `upper`: the work list holds the tiles on and above
 // the diagonal and the entries with col >= row are written (not with `batch`).
@@ -65,7 +67,7 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
                              int a_kind, int* d_status, int sm_count, cudaStream_t stream,
-                             int64_t batch = 0, int64_t c_batch_stride = 0, int upper = 0);
+                             int64_t batch = 0, int64_t c_batch_stride = 0, int upper = 0, const CUtensorMap* tmB = nullptr);
 // Square-block comparison kernel on CTA pairs (tcgen05 cta_group::2) for operands of input kind `a_kind`
 // (as launch_syrk_bf16) stored N x M: block i of `d_blocks` = {X0, X1, Y0, Y1}, tile rows (128 rows each) of a 256 x 256 block
 // strictly below the diagonal; pair p of the grid runs blocks p, p + pairs, ...  `tmA` and `tmC` as for
@@ -92,6 +94,10 @@ cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, in
 // Plain-load rank-2k update (binary64): one thread per lower-triangle entry; for unaligned operands.
 cudaError_t launch_syr2k_plain(int64_t N, int64_t M, const double* A, int64_t lda, const double* B, int64_t ldb,
                                double* C, int64_t ldc, double alpha, double beta, cudaStream_t stream);
+
+// The same for the tcgen05 storage types (dtype 1..4; binary32 accumulation and C).
+cudaError_t launch_syr2k_plain_f32(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, const void* B, int64_t ldb,
+                                   float* C, int64_t ldc, float alpha, float beta, cudaStream_t stream);
 
 cudaError_t launch_scale_lower(int dtype, int64_t N, void* C, int64_t ldc, double beta,
                                cudaStream_t stream, int upper = 0);

@@ -213,9 +213,14 @@ __device__ __forceinline__ void layout_of(const WorkItem* it, int n_tile, uint32
     }
 }
 
-template <bool kTN, int kKind, bool kUpper>
+// kSyr2k: the rank-2k update alpha (A B^T + B A^T) + beta C on the same work list.  A stage then holds the
+// item's segments of A in slots 0-2 and the same rows of B (second tensor map) in slots 3-5 - 96 KB, so the
+// ring has two stages instead of four - and every accumulator group takes two MMAs per 32 bytes of K,
+// A_x B_y^T and B_x A_y^T.  Operands stored N x M, lower triangle.
+template <bool kTN, int kKind, bool kUpper, bool kSyr2k = false>
 __global__ void __launch_bounds__(kThreads, 1)
-syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
+syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const __grid_constant__ CUtensorMap tmC,
                      const WorkItem* __restrict__ items, int64_t n_items, int64_t N, int32_t n_ksteps,
                      float* __restrict__ C, int64_t ldc, float alpha, float beta, int vec_ok, int tma_store_ok,
                      int32_t split, float* __restrict__ partial, const int64_t* __restrict__ tile_base,
@@ -235,6 +240,9 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     constexpr int kCols = KindCols<kKind>::value;        // columns of A in a 128-byte stage row
+    constexpr int kSt = kSyr2k ? kStages / 2 : kStages;                 // ring depth
+    constexpr int kStB = kSyr2k ? 2 * kStageBytes : kStageBytes;        // bytes of a stage (same ring size either way)
+    static_assert(!kSyr2k || (!kTN && !kUpper), "the rank-2k form takes N x M operands and the lower triangle");
     const int64_t n_units = n_items * split * (n_batch > 0 ? n_batch : 1);
     // This block's units: its own contiguous range of a list ordered block by block on the host,
     // or (K-split calls) every gridDim.x-th unit of the slice-major list.
@@ -244,7 +252,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
     if (tid == 0) {
         s_abort = 0;
-        for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kSt; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         mbar_init(tmem_full_bar, 1);
         mbar_init(pair_free_bar, 4);
         mbar_init(&single_free_bar[0], 4);
@@ -262,6 +270,7 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             prefetch_tensormap(&tmA);
+            if (kSyr2k) prefetch_tensormap(&tmB);
             uint32_t g = 0;
             for (int64_t w = w_first; w < w_last && !s_abort; w += w_stride) {
                 const Unit u = unit_of(w, n_items, n_ksteps, split, n_batch);
@@ -270,13 +279,18 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 int32_t rows[kSegSlots];
                 for (int s = 0; s < kSegSlots; ++s) rows[s] = (s < n_seg) ? it->seg[s] * kTile : 0;
                 for (int ks = u.k0; ks < u.k1; ++ks, ++g) {
-                    const uint32_t st = g % kStages;
-                    if (g >= kStages && !mbar_wait_bounded(&empty_bar[st], ((g / kStages) - 1) & 1, &s_abort)) {
+                    const uint32_t st = g % kSt;
+                    if (g >= kSt && !mbar_wait_bounded(&empty_bar[st], ((g / kSt) - 1) & 1, &s_abort)) {
                         s_abort = 1; atomicOr(status, kStatusWaitEmpty); break;
                     }
-                    mbar_arrive_expect_tx(&full_bar[st], uint32_t(n_seg) * kSegBytes);
-                    uint8_t* dst = smem + st * kStageBytes;
-                    if (kTN) {   // A stored M x N: per segment, boxes of one stage's k-rows x 128 bytes of columns
+                    mbar_arrive_expect_tx(&full_bar[st], uint32_t(kSyr2k ? 2 * n_seg : n_seg) * kSegBytes);
+                    uint8_t* dst = smem + st * kStB;
+                    if (kSyr2k) {   // rows of A in slots 0-2, the same rows of B in slots 3-5
+                        for (int s = 0; s < n_seg; ++s) {
+                            tma_load_box(dst + s * kSegBytes, &tmA, ks * kCols, rows[s], u.batch, &full_bar[st]);
+                            tma_load_box(dst + (kSegSlots + s) * kSegBytes, &tmB, ks * kCols, rows[s], u.batch, &full_bar[st]);
+                        }
+                    } else if (kTN) {   // A stored M x N: per segment, boxes of one stage's k-rows x 128 bytes of columns
                         constexpr int kGroupCols = kCols;                 // columns in a 128-byte row: 64, 32 or 128
                         constexpr int kGroups = kTile / kGroupCols;
                         for (int s = 0; s < n_seg; ++s)
@@ -291,8 +305,8 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             }
             if (s_abort) {   // winding down: let the copies still in flight land first
                 volatile int dummy = 0;
-                for (uint32_t i = (g > kStages ? g - kStages : 0); i < g; ++i)
-                    mbar_wait_bounded(&full_bar[i % kStages], (i / kStages) & 1, &dummy);
+                for (uint32_t i = (g > kSt ? g - kSt : 0); i < g; ++i)
+                    mbar_wait_bounded(&full_bar[i % kSt], (i / kSt) & 1, &dummy);
             }
         }
         __syncwarp();
@@ -327,19 +341,29 @@ syrk_bf16_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 tc_fence_after();
                 bool ok = true;
                 for (int ks = u.k0; ks < u.k1; ++ks, ++g) {
-                    const uint32_t st = g % kStages;
-                    if (!mbar_wait_bounded(&full_bar[st], (g / kStages) & 1, &s_abort)) {
+                    const uint32_t st = g % kSt;
+                    if (!mbar_wait_bounded(&full_bar[st], (g / kSt) & 1, &s_abort)) {
                         s_abort = 1; atomicOr(status, kStatusWaitFull); ok = false; break;
                     }
                     tc_fence_after();
-                    const uint32_t st_off = (st * kStageBytes) >> 4;
+                    const uint32_t st_off = (st * kStB) >> 4;
                     const uint32_t first = (ks > u.k0) ? 1u : 0u;
+                    constexpr uint32_t kOther = (uint32_t(kSegSlots) * kSegBytes) >> 4;   // from a segment of A to the same rows of B
                     for (int q = 0; q < L.n_grp; ++q) {
 #pragma unroll
-                        for (int kk = 0; kk < kBK / 16; ++kk)
-                            tc_mma<kKind>(d_addr[q], desc_hi | uint64_t(a_lo[q] + st_off + kk_step * kk),
-                                        desc_hi | uint64_t(b_lo[q] + st_off + kk_step * kk), idesc[q],
-                                        (kk > 0) ? 1u : first);
+                        for (int kk = 0; kk < kBK / 16; ++kk) {
+                            if (kSyr2k) {   // A_x B_y^T, then B_x A_y^T into the same accumulator
+                                tc_mma<kKind>(d_addr[q], desc_hi | uint64_t(a_lo[q] + st_off + kk_step * kk),
+                                              desc_hi | uint64_t(b_lo[q] + kOther + st_off + kk_step * kk), idesc[q],
+                                              (kk > 0) ? 1u : first);
+                                tc_mma<kKind>(d_addr[q], desc_hi | uint64_t(a_lo[q] + kOther + st_off + kk_step * kk),
+                                              desc_hi | uint64_t(b_lo[q] + st_off + kk_step * kk), idesc[q], 1u);
+                            } else {
+                                tc_mma<kKind>(d_addr[q], desc_hi | uint64_t(a_lo[q] + st_off + kk_step * kk),
+                                              desc_hi | uint64_t(b_lo[q] + st_off + kk_step * kk), idesc[q],
+                                              (kk > 0) ? 1u : first);
+                            }
+                        }
                     }
                     tc_commit(&empty_bar[st]);    // stage reusable once these MMAs have read it
                 }
@@ -497,9 +521,9 @@ splitk_reduce_kernel(const WorkItem* __restrict__ items, const int64_t* __restri
 }
 
 // The instantiation for an input kind, a storage order of A and a stored triangle of C.
-using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const WorkItem*, int64_t, int64_t, int32_t, float*, int64_t,
-                          float, float, int, int, int32_t, float*, const int64_t*, int64_t, const int64_t*, int*, int32_t,
-                          int64_t);
+using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const WorkItem*, int64_t, int64_t, int32_t,
+                          float*, int64_t, float, float, int, int, int32_t, float*, const int64_t*, int64_t, const int64_t*, int*,
+                          int32_t, int64_t);
 template <int kKind>
 KernelFn kernel_of_kind(int tn, int upper) {
     return tn ? (upper ? syrk_bf16_tbs_kernel<true, kKind, true> : syrk_bf16_tbs_kernel<true, kKind, false>)
@@ -513,6 +537,14 @@ KernelFn kernel_for(int kind, int tn, int upper) {
         default: return kernel_of_kind<kKindBF16>(tn, upper);
     }
 }
+KernelFn syr2k_kernel_for(int kind) {
+    switch (kind) {
+        case kKindTF32: return syrk_bf16_tbs_kernel<false, kKindTF32, false, true>;
+        case kKindE4M3: return syrk_bf16_tbs_kernel<false, kKindE4M3, false, true>;
+        case kKindF16: return syrk_bf16_tbs_kernel<false, kKindF16, false, true>;
+        default: return syrk_bf16_tbs_kernel<false, kKindBF16, false, true>;
+    }
+}
 
 }  // namespace bf16
 
@@ -521,7 +553,7 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
                              float beta, int split_k, float* d_partial, const int64_t* d_tile_base,
                              int64_t total_tiles, const int64_t* d_cta_begin, int n_ctas, int a_is_m_by_n,
                              int a_kind, int* d_status, int sm_count, cudaStream_t stream, int64_t batch,
-                             int64_t c_batch_stride, int upper) {
+                             int64_t c_batch_stride, int upper, const CUtensorMap* tmB) {
     // The shared-memory attribute belongs to a device's context: set it once per device.
     static bool configured[64] = {};
     static std::mutex configured_mu;                 // launchers are reached under different locks
@@ -530,8 +562,9 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[16];
+        const void* kernels[20];
         for (int i = 0; i < 16; ++i) kernels[i] = reinterpret_cast<const void*>(bf16::kernel_for(i >> 2, (i >> 1) & 1, i & 1));
+        for (int i = 0; i < 4; ++i) kernels[16 + i] = reinterpret_cast<const void*>(bf16::syr2k_kernel_for(i));
         for (const void* fn : kernels) {
             cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bf16::kSmemBytes);
             if (e != cudaSuccess) return e;
@@ -545,15 +578,16 @@ cudaError_t launch_syrk_bf16(const CUtensorMap& tmA, const CUtensorMap* tmC, con
     const int32_t n_ksteps = int32_t((M + bk - 1) / bk);
     const int split = split_k < 1 ? 1 : (split_k > n_ksteps ? n_ksteps : split_k);
     if (batch > 0 && (split != 1 || upper || batch >= (int64_t(1) << 31))) return cudaErrorInvalidValue;
+    if (tmB != nullptr && (a_is_m_by_n || upper || batch > 0)) return cudaErrorInvalidValue;   // rank-2k: N x M operands, lower triangle
     const int64_t n_units = n_items * split * (batch > 0 ? batch : 1);
     const bool ranges = (d_cta_begin != nullptr && split == 1 && n_ctas > 0 && batch <= 0);
     const unsigned grid = ranges ? unsigned(n_ctas) : unsigned(n_units < sm_count ? n_units : sm_count);
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 3) == 0 &&
                         (batch <= 0 || (c_batch_stride & 3) == 0)) ? 1 : 0;
     CUtensorMap none{};
-    auto kernel = bf16::kernel_for(a_kind, a_is_m_by_n, upper);
+    auto kernel = tmB ? bf16::syr2k_kernel_for(a_kind) : bf16::kernel_for(a_kind, a_is_m_by_n, upper);
     kernel<<<grid, bf16::kThreads, bf16::kSmemBytes, stream>>>(
-        tmA, tmC ? *tmC : none, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, split,
+        tmA, tmB ? *tmB : none, tmC ? *tmC : none, d_items, n_items, N, n_ksteps, C, ldc, alpha, beta, vec_ok, tmC ? 1 : 0, split,
         d_partial, d_tile_base, total_tiles, ranges ? d_cta_begin : nullptr, d_status, int32_t(batch > 0 ? batch : 0),
         c_batch_stride);
     cudaError_t e = cudaGetLastError();

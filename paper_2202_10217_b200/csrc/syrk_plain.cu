@@ -65,6 +65,21 @@ __global__ void syr2k_plain_kernel(int64_t N, int64_t M, const double* __restric
     *c = (beta == 0.0) ? alpha * s : alpha * s + beta * *c;
 }
 
+// The same for the storage types that accumulate in binary32 (each product is exact in binary32).
+template <typename TA>
+__global__ void syr2k_plain_f32_kernel(int64_t N, int64_t M, const TA* __restrict__ A, int64_t lda, const TA* __restrict__ B,
+                                       int64_t ldb, float* __restrict__ C, int64_t ldc, float alpha, float beta) {
+    const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
+    if (i >= N || j > i) return;
+    float s = 0.f;
+    for (int64_t k = 0; k < M; ++k)
+        s = fmaf(Widen<TA, float>::get(A + i * lda + k), Widen<TA, float>::get(B + j * ldb + k),
+                 fmaf(Widen<TA, float>::get(B + i * ldb + k), Widen<TA, float>::get(A + j * lda + k), s));
+    float* c = C + i * ldc + j;
+    *c = (beta == 0.f) ? alpha * s : alpha * s + beta * *c;
+}
+
 template <typename TC>
 __global__ void scale_lower_kernel(int64_t N, TC* __restrict__ C, int64_t ldc, TC beta, int upper) {
     const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -109,6 +124,26 @@ cudaError_t launch_syr2k_plain(int64_t N, int64_t M, const double* A, int64_t ld
     if (N == 0) return cudaSuccess;
     const dim3 block(32, 8);
     syr2k_plain_kernel<<<grid2d(N, block), block, 0, stream>>>(N, M, A, lda, B, ldb, C, ldc, alpha, beta);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_syr2k_plain_f32(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, const void* B, int64_t ldb,
+                                   float* C, int64_t ldc, float alpha, float beta, cudaStream_t stream) {
+    if (N == 0) return cudaSuccess;
+    const dim3 block(32, 8);
+    const dim3 grid = grid2d(N, block);
+    if (dtype == 3)
+        syr2k_plain_f32_kernel<uint8_t><<<grid, block, 0, stream>>>(N, M, static_cast<const uint8_t*>(A), lda,
+                                                                    static_cast<const uint8_t*>(B), ldb, C, ldc, alpha, beta);
+    else if (dtype == 4)
+        syr2k_plain_f32_kernel<__half><<<grid, block, 0, stream>>>(N, M, static_cast<const __half*>(A), lda,
+                                                                   static_cast<const __half*>(B), ldb, C, ldc, alpha, beta);
+    else if (dtype == 2)
+        syr2k_plain_f32_kernel<float><<<grid, block, 0, stream>>>(N, M, static_cast<const float*>(A), lda,
+                                                                  static_cast<const float*>(B), ldb, C, ldc, alpha, beta);
+    else
+        syr2k_plain_f32_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(N, M, static_cast<const __nv_bfloat16*>(A), lda,
+                                                                          static_cast<const __nv_bfloat16*>(B), ldb, C, ldc, alpha, beta);
     return cudaGetLastError();
 }
 

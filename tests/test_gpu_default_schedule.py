@@ -149,3 +149,33 @@ def test_k_split_call_inside_stream_capture_needs_a_prepared_workspace():
     ref, _ = O.syrk_lower(A, None, 2.0, 0.0, B.DTYPE_BF16_F32)        # two accumulating replays
     il = np.tril_indices(N)
     assert np.array_equal(dC.cpu().numpy().astype(np.float64)[il], ref[il])
+
+
+@pytest.mark.parametrize("pinned", [False, True], ids=["pageable", "page-locked"])
+def test_host_buffer_entry_point_under_the_default_schedule(pinned):
+    """syrk_lower_host with a short-and-wide BF16 operand: below the band pipeline's size the call uploads A
+    in blocks of columns and runs each block through the device call, which under the default rule means
+    square blocks on CTA pairs with their own K-split; beta != 0, pitches, ragged last block."""
+    N, M = 2304, 24000
+    assert B.syrk_effective_schedule(N, M, B.DTYPE_BF16_F32) == B.SCHEDULE_PAIR_SQUARE
+    assert B.syrk_host_pipeline_for(N, M, pinned) == B.HOST_COLUMN_BLOCKS
+    A = make_A(N, M, B.DTYPE_BF16_F32, seed=8400)
+    lda, ldc = M + 16, N + 5
+    Abig = np.zeros((N, lda), dtype=A.dtype)
+    Abig[:, :M] = A
+    Cin = I.random_c(N, 8401, B.DTYPE_BF16_F32, ldc)
+    hA = torch.from_numpy(Abig.view(np.int16))
+    hC = torch.from_numpy(Cin.copy())
+    if pinned:
+        hA, hC = hA.pin_memory(), hC.pin_memory()
+    B.syrk_lower_host(N, M, hA, lda, hC, ldc, 0.5, -1.0, B.DTYPE_BF16_F32)
+    C = hC.numpy()
+    ii, jj = np.tril_indices(N)
+    pick = np.random.default_rng(8402).choice(ii.size, size=20000, replace=False)
+    ii, jj = ii[pick], jj[pick]
+    ref, bound = O.syrk_entries(ii, jj, A, None, 0.5, 0.0, B.DTYPE_BF16_F32)
+    ref = ref - Cin[ii, jj].astype(np.float64)
+    tol = O.tolerance(M, bound, np.abs(Cin[ii, jj]), 0.5, -1.0, B.DTYPE_BF16_F32)
+    assert np.all(np.abs(C[ii, jj].astype(np.float64) - ref) <= tol)
+    iu = np.triu_indices(N, 1)
+    assert np.array_equal(C[:, :N][iu], Cin[:, :N][iu]) and np.array_equal(C[:, N:], Cin[:, N:])
