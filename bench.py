@@ -205,10 +205,10 @@ def run_reference(args, key: str, shape, rank: int):
 # summarised under profiles/.  Valid only for the kernel source it was taken on: keyed by its SHA-256.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, kernel source file, sha256 of that file at capture time, square-schedule bytes or None)
-    "c2_f64_4096x4096": (832_195_584, "syrk_f64.cu", "dc0af5511d941afee99ca375ca5db108325e8474b096a5eaff9efcc6db1d6bef", 811_978_240),
-    "c3_bf16_16384x4096": (1_881_366_784, "syrk_bf16.cu", "b2b31371304f54522dd449d94e2448a596236a0881b9e215e356cf28aec88cd5", 3_712_474_624),
-    "c4_bf16_2048x262144": (1_159_163_136, "syrk_bf16_pair.cu", "1f007b0ed5552de540c0cf0f25685f828321404cc4f842d0dbfcbbdcc303fc01", 2_276_417_536),
-    "c5_call_n16384": (2_885_844_736, "syrk_f64.cu", "dc0af5511d941afee99ca375ca5db108325e8474b096a5eaff9efcc6db1d6bef", 2_724_991_232),
+    "c2_f64_4096x4096": (833_247_744, "syrk_f64.cu", "dc0af5511d941afee99ca375ca5db108325e8474b096a5eaff9efcc6db1d6bef", 815_276_288),
+    "c3_bf16_16384x4096": (1_898_579_968, "syrk_bf16.cu", "527f2140d892d840fb605c824d4e19c4706e87355a46c48bb934fb71b3a9a97b", 3_150_107_648),
+    "c4_bf16_2048x262144": (1_308_831_488, "syrk_bf16_pair.cu", "1f007b0ed5552de540c0cf0f25685f828321404cc4f842d0dbfcbbdcc303fc01", 2_332_056_832),
+    "c5_call_n16384": (2_882_612_224, "syrk_f64.cu", "dc0af5511d941afee99ca375ca5db108325e8474b096a5eaff9efcc6db1d6bef", 2_727_926_272),
 }
 
 

@@ -337,16 +337,16 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
             const size_t want = size_t(split) * size_t(dp->total_tiles) * ks.tile * ks.tile * sizeof(float);
             if ((rc = workspace_for_stream(ds, stream, want, &d_partial)) != SYRK_OK) return rc;
         }
-    } else if (f64_launch < 0) {
-        // FP64 K-split (not for callers that fix the launch form: the Cholesky driver's look-ahead stream
-        // runs short updates that gain nothing from it)
+    } else {
+        // FP64 K-split for lists shorter than the SM count (every stream has its own workspace, so the
+        // Cholesky driver's two streams may both use it)
         split = auto_split_k_f64(int64_t(dp->plan.items.size()), N, M, ks.bk, ds->sm_count, runtime().split_k);
         if (split > 1 &&
             (rc = workspace_for_stream(ds, stream, size_t(split) * size_t(N) * size_t(N) * sizeof(double), &d_partial)) != SYRK_OK)
             return rc;
         // Otherwise, in the one-block-per-item form: the last round's items in slices (tail K-split).
         const int64_t n_items = int64_t(dp->plan.items.size());
-        const int mode = runtime().f64_launch;
+        const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
         const bool per_item = upper || mode == SYRK_F64_LAUNCH_PER_ITEM ||
                               (mode == SYRK_F64_LAUNCH_AUTO && !(M <= 1024 && n_items >= 4 * int64_t(ds->sm_count)));
         if (split == 1 && per_item && !upper && runtime().f64_tail_slices != 1) {
