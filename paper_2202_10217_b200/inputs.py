@@ -135,6 +135,34 @@ def small_int_f64(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.nd
     return np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float64)
 
 
+def normal_c128(N: int, M: int, seed: int, std: float = 1.0) -> np.ndarray:
+    """Complex N x M with independent N(0, std^2) real and imaginary parts (complex128)."""
+    rng = np.random.default_rng(seed)
+    out = np.empty((N, M), dtype=np.complex128)
+    out.real = rng.standard_normal((N, M)) * std
+    out.imag = rng.standard_normal((N, M)) * std
+    return out
+
+
+def small_int_c128(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
+    """Gaussian integers with both parts in [lo, hi] (complex128): every sum of products is exact."""
+    rng = np.random.default_rng(seed)
+    out = np.empty((N, M), dtype=np.complex128)
+    out.real = rng.integers(lo, hi + 1, size=(N, M))
+    out.imag = rng.integers(lo, hi + 1, size=(N, M))
+    return out
+
+
+def random_c128(N: int, seed: int, ldc: Optional[int] = None) -> np.ndarray:
+    """A complex N x ldc array for C (uniform parts in [-1, 1)); the caller reads its lower triangle."""
+    rng = np.random.default_rng(seed)
+    ldc = N if ldc is None else ldc
+    out = np.empty((N, ldc), dtype=np.complex128)
+    out.real = rng.uniform(-1.0, 1.0, size=(N, ldc))
+    out.imag = rng.uniform(-1.0, 1.0, size=(N, ldc))
+    return out
+
+
 def small_int_bf16(N: int, M: int, seed: int, lo: int = -2, hi: int = 2) -> np.ndarray:
     """Integer entries in [lo, hi] as bfloat16 bit patterns (exactly representable)."""
     v = np.random.default_rng(seed).integers(lo, hi + 1, size=(N, M)).astype(np.float32)
