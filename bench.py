@@ -671,6 +671,8 @@ def run_kernel_only(args, key, shape, rank: int, world: int, local_rank: int):
             return run_batched(args, wl)
         if args.syr2k:
             return run_syr2k(args, wl)
+        if args.herk:
+            return run_herk(args, wl)
         _, dA = to_device(torch, wl.make_A(), dtype)
         dC = torch.zeros((N, N), dtype=torch.float64 if dtype == I.DTYPE_F64 else torch.float32, device="cuda")
         if args.gram:                                          # same operand stored M x N: C = A^T A
@@ -768,6 +770,39 @@ def run_syr2k(args, wl):
                       "config": {"workload": wl.name, "N": N, "M": M, "op": "syr2k", "dtype": DTYPE_NAME[dtype]}}))
 
 
+def run_herk(args, wl):
+    """--kernel-only --herk: the Hermitian rank-k update alpha A A^H + beta C of the workload's N x M with complex128
+    entries (both parts drawn N(0, 1)); 4 N (N+1) M real flops (a complex multiply-add counted as 8)."""
+    import torch
+    from paper_2202_10217_b200 import binding as B
+
+    N, M = wl.N, wl.M
+    if wl.dtype != I.DTYPE_F64:
+        raise SystemExit("--herk is a binary64 path: give an f64 workload or --shape N,M,f64,alpha,beta")
+    gen = torch.Generator(device="cuda").manual_seed(wl.seed)
+    dA = torch.view_as_complex(torch.randn((N, M, 2), dtype=torch.float64, device="cuda", generator=gen))
+    dC = torch.zeros((N, N), dtype=torch.complex128, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    call = lambda: B.herk_lower(N, M, dA, M, dC, N, wl.alpha, wl.beta)
+    for _ in range(max(args.warmup, 1)):
+        call()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(args.steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        call()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert B.syrk_last_status() == 0
+    ms = float(np.mean(times))
+    print(json.dumps({"metric": "herk_tflops_4N(N+1)M", "value": 4 * wl.flops / (ms * 1e-3) * 1e-12, "unit": UNIT,
+                      "n_gpus": 1, "steps": args.steps, "ms_per_step": ms, "kernel_only": True,
+                      "config": {"workload": wl.name, "N": N, "M": M, "op": "herk", "dtype": "c128"}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -792,13 +827,15 @@ def main():
                          "square-block comparison schedule, or square blocks on CTA pairs")
     ap.add_argument("--syr2k", action="store_true",
                     help="with --kernel-only: time syr2k_lower_ex (rank-2k update of the workload's type) instead")
+    ap.add_argument("--herk", action="store_true",
+                    help="with --kernel-only: time herk_lower (Hermitian rank-k update, complex128, of the workload's N x M)")
     ap.add_argument("--kshard", action="store_true",
                     help="split the inner dimension of the workload (default c4) over the ranks: K-sharded update with "
                          "one reduce-scatter (strong scaling) instead of independent replicas")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
-    for flag, on in (("--schedule", args.schedule != "default"), ("--syr2k", args.syr2k), ("--batch", args.batch > 0),
-                     ("--gram", args.gram), ("--sustained", args.sustained)):
+    for flag, on in (("--schedule", args.schedule != "default"), ("--syr2k", args.syr2k), ("--herk", args.herk),
+                     ("--batch", args.batch > 0), ("--gram", args.gram), ("--sustained", args.sustained)):
         if on and not args.kernel_only:
             ap.error(flag + " needs --kernel-only")
     rank = int(os.environ.get("RANK", "0"))

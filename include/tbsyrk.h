@@ -216,6 +216,33 @@ int syr2k_lower_ex(int64_t N, int64_t M,
                    double alpha, double beta, int dtype, void* stream);
 
 /*
+ * Hermitian rank-k update on the lower triangle, complex128:
+ *
+ *     C[i][j] = alpha * sum_k A[i][k] * conj(A[j][k]) + beta * C[i][j]     0 <= j <= i < N,
+ *
+ * alpha and beta real.  A is a DEVICE pointer to an N x M row-major array of complex numbers stored as
+ * (real, imaginary) pairs of binary64, pitch lda >= max(1, M) complex entries; C likewise N x N, pitch
+ * ldc >= max(1, N) complex entries.  Entries with j > i are never read or written.  The imaginary part
+ * of a diagonal entry is not read and is written as zero.  beta == 0: C is not read.
+ * This is Algorithm 1 of the paper over the complex numbers (second factor conjugated), one more of
+ * the kernels "which use the same input several times" of the paper's conclusion.  Schedule: Algorithm 4 /
+ * Section 5.1.4 unchanged - a thread block owns the accumulators of every pair among k = 4 row segments
+ * and streams those rows of A once; what changes is the arithmetic per pair: on the real view of A
+ * (2M reals per row) the real part is the symmetric update, and the imaginary part is the product of
+ * the same rows with those of i * A, which a warp forms from the neighbouring shared-memory word of
+ * the same stage (no second operand is loaded).  FP64 tensor cores (DMMA).
+ * A and C 16-byte aligned, else (and for the scale-only cases) a plain-load kernel (8-byte alignment,
+ * that of binary64, is the caller's to keep).  Quick returns: N == 0; (alpha == 0 or M == 0) and
+ * beta == 1: nothing is touched; alpha == 0 or M == 0: the lower triangle is scaled by beta (zeroed
+ * for beta == 0) and the diagonal's imaginary part is zeroed.  Ownership, stream semantics, status
+ * word and the other error codes as for syrk_lower.
+ */
+int herk_lower(int64_t N, int64_t M,
+               const void* A, int64_t lda,
+               void* C, int64_t ldc,
+               double alpha, double beta, void* stream);
+
+/*
  * A strided batch of independent updates of the same shape:
  *
  *     C_b[i][j] = alpha * sum_k A_b[i][k] * A_b[j][k] + beta * C_b[i][j]    0 <= j <= i < N, 0 <= b < batch,

@@ -29,7 +29,7 @@ ITEM_TRI, ITEM_RECT, ITEM_DIAG = 0, 1, 2
 MAX_SEG, MAX_TILE = 8, 16
 
 EXPORTS = [
-    "syrk_lower", "syrk_lower_tn", "syrk_ex", "syr2k_lower", "syr2k_lower_ex", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_plan_prepare_stream", "syrk_effective_schedule",
+    "syrk_lower", "syrk_lower_tn", "syrk_ex", "syr2k_lower", "syr2k_lower_ex", "herk_lower", "syrk_lower_batched", "syrk_lower_host", "syrk_plan_prepare", "syrk_plan_prepare_stream", "syrk_effective_schedule",
     "syrk_lower_bf16_static_status", "syrk_set_host_pipeline", "syrk_host_pipeline_for", "syrk_pack_lower", "syrk_unpack_lower_axpby", "syrk_shutdown", "syrk_last_status",
     "syrk_strerror", "syrk_set_schedule", "syrk_set_split_k", "syrk_set_f64_tail_split", "syrk_set_f64_launch", "syrk_get_schedule_stats",
     "syrk_probe_f64_mma_peak", "syrk_selftest_bounded_wait", "syrk_lower_bf16_static", "cholesky_lower", "cholesky_last_info",
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.syrk_lower_tn.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
         L.syrk_ex.restype = ci
         L.syrk_ex.argtypes = [ci, ci, i64, i64, vp, i64, vp, i64, dbl, dbl, ci, vp]
+        L.herk_lower.restype = ci
+        L.herk_lower.argtypes = [i64, i64, vp, i64, vp, i64, dbl, dbl, vp]
         L.syr2k_lower.restype = ci
         L.syr2k_lower.argtypes = [i64, i64, vp, i64, vp, i64, vp, i64, dbl, dbl, vp]
         L.syr2k_lower_ex.restype = ci
@@ -203,6 +205,16 @@ def syr2k_lower(N: int, M: int, A, lda: int, Bm, ldb: int, C, ldc: int, alpha: f
         import torch
         stream = torch.cuda.current_stream().cuda_stream
     _check(lib().syr2k_lower(N, M, _ptr(A), lda, _ptr(Bm), ldb, _ptr(C), ldc, float(alpha), float(beta), stream))
+
+
+def herk_lower(N: int, M: int, A, lda: int, C, ldc: int, alpha: float, beta: float,
+               stream: Optional[int] = None) -> None:
+    """Enqueue C_lower <- alpha * A A^H + beta * C_lower (complex128 as (re, im) pairs, device pointers,
+    pitches in complex entries)."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().herk_lower(N, M, _ptr(A), lda, _ptr(C), ldc, float(alpha), float(beta), stream))
 
 
 def syr2k_lower_ex(N: int, M: int, A, lda: int, Bm, ldb: int, C, ldc: int, alpha: float, beta: float, dtype: int,

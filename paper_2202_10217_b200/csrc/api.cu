@@ -481,6 +481,33 @@ int syrk_ex(int uplo, int trans, int64_t N, int64_t M, const void* A, int64_t ld
                            trans == SYRK_OP_T ? 1 : 0, uplo == SYRK_UPLO_UPPER ? 1 : 0);
 }
 
+// Work list of Algorithm 4 for the kernels' forms in which two warps share a tile (rank-2k and Hermitian
+// updates): triangle blocks with k = 4 (6 tiles; for the rank-2k update a stage holds the four segments of A
+// and the same rows of B), 2 x 2 rectangles, diagonal blocks of two rows.  Cached per device.
+static int get_two_warp_plan(DeviceState* ds, int64_t N, DevicePlan** out) {
+    const int64_t n_tiles = (N + f64_tile() - 1) / f64_tile();
+    const auto key = std::make_tuple(n_tiles, 64, runtime().schedule);       // 64: this list
+    auto it = ds->plans.find(key);
+    if (it == ds->plans.end()) {
+        DevicePlan dp;
+        PlanParams p;
+        p.n_tiles = n_tiles; p.k = 4; p.rect_rows = 2; p.rect_cols = 2; p.diag_side = 2; p.schedule = runtime().schedule;
+        if (!build_plan(p, &dp.plan)) return SYRK_ERR_PLAN;
+        std::stable_sort(dp.plan.items.begin(), dp.plan.items.end(),
+                         [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
+        const size_t n = dp.plan.items.size();
+        if (n > 0) {
+            if (cudaMalloc(&dp.d_items, n * sizeof(WorkItem)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
+            if (cudaMemcpy(dp.d_items, dp.plan.items.data(), n * sizeof(WorkItem), cudaMemcpyHostToDevice) != cudaSuccess) {
+                cudaGetLastError(); cudaFree(dp.d_items); return SYRK_ERR_CUDA;
+            }
+        }
+        it = ds->plans.emplace(key, std::move(dp)).first;
+    }
+    *out = &it->second;
+    return SYRK_OK;
+}
+
 int syr2k_lower(int64_t N, int64_t M, const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc,
                 double alpha, double beta, void* stream) {
     int rc = validate(N, M, A, lda, C, ldc, SYRK_DTYPE_F64);
@@ -499,28 +526,8 @@ int syr2k_lower(int64_t N, int64_t M, const void* A, int64_t lda, const void* B,
     if (!tma_ok(A, lda, SYRK_DTYPE_F64) || !tma_ok(B, ldb, SYRK_DTYPE_F64))
         return launch_syr2k_plain(N, M, static_cast<const double*>(A), lda, static_cast<const double*>(B), ldb,
                                   static_cast<double*>(C), ldc, alpha, beta, st) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
-    // Work list of Algorithm 4 for blocks of four segments (a stage holds the four segments of A and
-    // the same rows of B): triangle blocks with k = 4, 2 x 2 rectangles, diagonal blocks of two rows.
-    const int64_t n_tiles = (N + f64_tile() - 1) / f64_tile();
-    const auto key = std::make_tuple(n_tiles, 64, runtime().schedule);       // 64: the rank-2k list
-    auto it = ds->plans.find(key);
-    if (it == ds->plans.end()) {
-        DevicePlan dp;
-        PlanParams p;
-        p.n_tiles = n_tiles; p.k = 4; p.rect_rows = 2; p.rect_cols = 2; p.diag_side = 2; p.schedule = runtime().schedule;
-        if (!build_plan(p, &dp.plan)) return SYRK_ERR_PLAN;
-        std::stable_sort(dp.plan.items.begin(), dp.plan.items.end(),
-                         [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
-        const size_t n = dp.plan.items.size();
-        if (n > 0) {
-            if (cudaMalloc(&dp.d_items, n * sizeof(WorkItem)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
-            if (cudaMemcpy(dp.d_items, dp.plan.items.data(), n * sizeof(WorkItem), cudaMemcpyHostToDevice) != cudaSuccess) {
-                cudaGetLastError(); cudaFree(dp.d_items); return SYRK_ERR_CUDA;
-            }
-        }
-        it = ds->plans.emplace(key, std::move(dp)).first;
-    }
-    DevicePlan* dp = &it->second;
+    DevicePlan* dp = nullptr;
+    if ((rc = get_two_warp_plan(ds, N, &dp)) != SYRK_OK) return rc;
     CUtensorMap ta, tb, tmc;
     if ((rc = encode_tensor_map_2d(&ta, SYRK_DTYPE_F64, A, N, M, lda, f64_tile(), f64_bk())) != SYRK_OK) return rc;
     if ((rc = encode_tensor_map_2d(&tb, SYRK_DTYPE_F64, B, N, M, ldb, f64_tile(), f64_bk())) != SYRK_OK) return rc;
@@ -529,6 +536,30 @@ int syr2k_lower(int64_t N, int64_t M, const void* A, int64_t lda, const void* B,
     return launch_syr2k_f64(ta, tb, c_tma ? &tmc : nullptr, dp->d_items, int64_t(dp->plan.items.size()), N, M,
                             static_cast<double*>(C), ldc, alpha, beta, status_for_stream(ds, st), st) == cudaSuccess
                ? SYRK_OK : SYRK_ERR_CUDA;
+}
+
+int herk_lower(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_t ldc, double alpha, double beta,
+               void* stream) {
+    if (N < 0 || M < 0) return SYRK_ERR_SIZE;
+    if (lda < std::max<int64_t>(1, M) || ldc < std::max<int64_t>(1, N)) return SYRK_ERR_LD;
+    if (N == 0) return SYRK_OK;
+    if (!C || (M > 0 && !A)) return SYRK_ERR_NULL;
+    std::lock_guard<std::mutex> lock(runtime().mu);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceState* ds = nullptr;
+    int rc = get_device_state(&ds);
+    if (rc != SYRK_OK) return rc;
+    if ((alpha == 0.0 || M == 0) && beta == 1.0) return SYRK_OK;
+    // Scale-only calls and operands that are not 16-byte aligned take the plain-load kernel.
+    if (alpha == 0.0 || M == 0 || (reinterpret_cast<uintptr_t>(A) & 15) != 0 || (reinterpret_cast<uintptr_t>(C) & 15) != 0)
+        return launch_herk_plain(N, M, static_cast<const double*>(A), lda, static_cast<double*>(C), ldc, alpha, beta, st) ==
+                       cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+    DevicePlan* dp = nullptr;
+    if ((rc = get_two_warp_plan(ds, N, &dp)) != SYRK_OK) return rc;
+    CUtensorMap ta;          // the real view of A: N rows of 2M values, pitch 2 lda
+    if ((rc = encode_tensor_map_2d(&ta, SYRK_DTYPE_F64, A, N, 2 * M, 2 * lda, f64_tile(), f64_bk())) != SYRK_OK) return rc;
+    return launch_herk_f64(ta, dp->d_items, int64_t(dp->plan.items.size()), N, M, static_cast<double*>(C), ldc, alpha, beta,
+                           status_for_stream(ds, st), st) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
 int syr2k_lower_ex(int64_t N, int64_t M, const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc,

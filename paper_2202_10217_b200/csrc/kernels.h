@@ -37,6 +37,12 @@ int64_t f64_tail_partial_elems(int64_t n_tail_items, int tail_slices);
 cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap* tmC,
                              const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc,
                              double alpha, double beta, int* d_status, cudaStream_t stream);
+// Hermitian rank-k update C = alpha A A^H + beta C on the lower triangle with the same kernel: `tmA` covers
+// the real view of the complex operand (N rows of 2M binary64 values, re and im interleaved), C and ldc
+// address complex entries (C 16-byte aligned); work items as for the rank-2k update (at most 8 tiles, a
+// tile shared by two warps, each with a real and an imaginary accumulator).  One block per item.
+cudaError_t launch_herk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M,
+                            double* C, int64_t ldc, double alpha, double beta, int* d_status, cudaStream_t stream);
 // The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
 // P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
 // columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.
@@ -94,6 +100,12 @@ cudaError_t launch_syrk_plain(int dtype, int64_t N, int64_t M, const void* A, in
 // Plain-load rank-2k update (binary64): one thread per lower-triangle entry; for unaligned operands.
 cudaError_t launch_syr2k_plain(int64_t N, int64_t M, const double* A, int64_t lda, const double* B, int64_t ldb,
                                double* C, int64_t ldc, double alpha, double beta, cudaStream_t stream);
+
+// Plain-load Hermitian rank-k update (complex128 as pairs of binary64; pitches in complex entries): one thread
+// per lower-triangle entry; for unaligned operands, and (M == 0 or alpha == 0) for the scale-only case.  The
+// diagonal's imaginary part is written as zero and not read; beta == 0: C is not read.
+cudaError_t launch_herk_plain(int64_t N, int64_t M, const double* A, int64_t lda, double* C, int64_t ldc,
+                              double alpha, double beta, cudaStream_t stream);
 
 // The same for the tcgen05 storage types (dtype 1..4; binary32 accumulation and C).
 cudaError_t launch_syr2k_plain_f32(int dtype, int64_t N, int64_t M, const void* A, int64_t lda, const void* B, int64_t ldb,

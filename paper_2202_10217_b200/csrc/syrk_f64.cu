@@ -79,6 +79,7 @@ struct Call {
     int32_t batch;                 // matrix of a strided batch the block works on (tensor maps are 3-D), or -1
     int32_t k0;                    // first K-step of the block's slice of the inner dimension (K-split calls)
     bool syr2k;                    // rank-2k update: slots 0..3 hold segments of A, slots 4..7 the same rows of B (tmB)
+    bool herk;                     // Hermitian update: A is the real view (re, im interleaved) of a complex operand, C complex
     bool gemm;
 };
 // Tail K-split units: bit 1 of Call::vec_ok is set and Call::C points at the unit's partial tiles (16 slots
@@ -158,11 +159,12 @@ __device__ void drain_producer(const Call& k, uint32_t g) {
 __device__ bool prepare_item(const Call& k, WorkItem& it, bool upper = false) {
     bool ok = it.n_seg >= 1 && it.n_seg <= kMaxSeg && it.n_tile >= 1 && it.n_tile <= kMmaWarps;
     if (k.syr2k) ok = ok && it.n_seg <= kSyr2kSlots && it.n_tile <= kMmaWarps / 2;
+    if (k.herk) ok = ok && it.n_tile <= kMmaWarps / 2;
     for (int s = 0; ok && s < it.n_seg; ++s)
         ok = it.seg[s] >= 0 && int64_t(it.seg[s]) * kTile < ((k.gemm && s < it.pad) ? k.ncols : k.N);
     for (int t = 0; ok && t < it.n_tile; ++t) ok = it.tile_x[t] < it.n_seg && it.tile_y[t] < it.n_seg;
     if (ok && !k.gemm) {
-        bool tri = !k.syr2k && it.kind == kTri && it.n_seg == 6 && it.n_tile == 15;
+        bool tri = !k.syr2k && !k.herk && it.kind == kTri && it.n_seg == 6 && it.n_tile == 15;
         for (int x = 1, q = 0; tri && x < 6; ++x)
             for (int y = 0; y < x; ++y, ++q)      // the upper-triangle form holds the same tiles transposed
                 tri = tri && it.tile_x[q] == (upper ? y : x) && it.tile_y[q] == (upper ? x : y);
@@ -544,16 +546,101 @@ __device__ __forceinline__ bool syr2k_tile_role(const Call& k, const WorkItem& i
     return true;
 }
 
+// Hermitian rank-k update, C <- alpha * A * A^H + beta * C with A complex N x M (pairs re, im) and C complex:
+// the stages hold the real view of A (row i = 2M reals).  With A[i][k] = a + b i and A[j][k] = c + d i,
+//     Re C[i][j] = sum a c + b d = (row i of the view) . (row j of the view),
+//     Im C[i][j] = sum b c - a d = (row i of the view) . (row j of the view of i * A),   i * (c + d i) = -d + c i.
+// Lanes t and t ^ 1 of a fragment hold the two parts of one complex number (k = ... + (t & 1)), so the
+// fragment of i * A is the partner's shared-memory word (address ^ 8) with the sign changed in the even lanes.
+// Warp w owns rows 16 (w & 1) .. + 15 of tile w >> 1 with one 16 x 32 accumulator per part: 16 DMMAs per
+// k-slice and warp, as for a whole tile of the rank-k update.  Lower triangle; the diagonal's imaginary part is
+// written as zero and not read.  k.C and k.ldc address complex elements (two doubles each).
+__device__ __forceinline__ double flip_sign(double v, uint32_t mask) {
+    return __hiloint2double(__double2hiint(v) ^ int(mask), __double2loint(v));
+}
+__device__ __forceinline__ bool herk_tile_role(const Call& k, const WorkItem& it, uint32_t g0, int warp, int lane) {
+    const int gq = lane >> 2, t = lane & 3;
+    const int tile = warp >> 1, half = warp & 1;
+    const bool use_beta = (k.beta != 0.0);
+    const uint32_t off0 = fragment_offset(lane);
+    const uint32_t flip = (t & 1) ? 0u : 0x80000000u;
+    const int sx = it.tile_x[tile], sy = it.tile_y[tile];
+    const int64_t row0 = int64_t(it.seg[sx]) * kTile, col0 = int64_t(it.seg[sy]) * kTile;
+    const uint32_t xa = uint32_t(sx) * kSegBytes, ya = uint32_t(sy) * kSegBytes;
+
+    double re[2][4][2], im[2][4][2];
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) re[mi][ni][0] = re[mi][ni][1] = im[mi][ni][0] = im[mi][ni][1] = 0.0;
+
+    uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;
+    for (int ks = 0; ks < k.n_ksteps; ++ks) {
+        if (!wait_full_at(k, st, parity, lane)) return false;
+        const uint32_t stage = k.smem32 + st * kStageBytes;
+        const uint32_t px = (stage + xa) | off0, py = (stage + ya) | off0;
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl) {
+            double a[2], b[4], r[4];
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi) a[mi] = lds_f64(frag_addr<false>(px, 2 * half + mi, sl));
+#pragma unroll
+            for (int ni = 0; ni < 4; ++ni) {
+                const uint32_t addr = frag_addr<false>(py, ni, sl);
+                b[ni] = lds_f64(addr);
+                r[ni] = flip_sign(lds_f64(addr ^ 8u), flip);
+            }
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+                for (int ni = 0; ni < 4; ++ni) {
+                    dmma884(re[mi][ni], a[mi], b[ni]);
+                    dmma884(im[mi][ni], a[mi], r[ni]);
+                }
+        }
+        release_at(k, st, lane);
+        if (++st == kStages) { st = 0; parity ^= 1; }
+    }
+
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi) {
+        const int64_t r = row0 + (2 * half + mi) * 8 + gq;
+        if (r >= k.N) continue;
+        double* crow = k.C + 2 * r * k.ldc;
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) {
+            const int64_t c = col0 + ni * 8 + 2 * t;
+            if (c > r) continue;
+            const bool both = (c + 1 <= r);
+            double2 v0 = make_double2(k.alpha * re[mi][ni][0], k.alpha * im[mi][ni][0]);
+            double2 v1 = make_double2(k.alpha * re[mi][ni][1], k.alpha * im[mi][ni][1]);
+            if (use_beta) {
+                const double2 o0 = *reinterpret_cast<const double2*>(crow + 2 * c);
+                v0.x += k.beta * o0.x; v0.y += k.beta * o0.y;
+                if (both) {
+                    const double2 o1 = *reinterpret_cast<const double2*>(crow + 2 * c + 2);
+                    v1.x += k.beta * o1.x; v1.y += k.beta * o1.y;
+                }
+            }
+            if (c == r) v0.y = 0.0;
+            if (c + 1 == r) v1.y = 0.0;
+            *reinterpret_cast<double2*>(crow + 2 * c) = v0;
+            if (both) *reinterpret_cast<double2*>(crow + 2 * c + 2) = v1;
+        }
+    }
+    return true;
+}
+
 // One MMA warp's share of one item: its ring steps from global step g on, then its write-out.
 // Every warp waits for and releases every ring step of the item, with or without work in it.
-template <bool kTN, bool kUpper, bool kSyr2k = false>
+template <bool kTN, bool kUpper, bool kSyr2k = false, bool kHerk = false>
 __device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it, uint32_t& g, int warp, int lane) {
     const int n_tile = it.n_tile;
     const int n_c = c_steps_of(k, n_tile);
     const uint32_t g0 = g;
     g += uint32_t(k.n_ksteps + n_c);
-    if (kSyr2k) {
-        if (warp < 2 * n_tile) return syr2k_tile_role(k, it, g0, n_c, warp, lane);
+    if (kSyr2k || kHerk) {
+        if (warp < 2 * n_tile) return kHerk ? herk_tile_role(k, it, g0, warp, lane) : syr2k_tile_role(k, it, g0, n_c, warp, lane);
         for (uint32_t s = g0; s < g; ++s) {             // no work in this item: keep the ring moving
             if (!wait_full(k, s, lane)) return false;
             release(k, s, lane);
@@ -576,7 +663,7 @@ __device__ __forceinline__ bool mma_warp_item(const Call& k, const WorkItem& it,
 // groups), its column segments come from Q (tmB, the first `pad` segments), its row segments
 // from P (tmA).
 // ---------------------------------------------------------------------------------------------
-template <bool kTN, bool kUpper, bool kSyr2k = false>
+template <bool kTN, bool kUpper, bool kSyr2k = false, bool kHerk = false>
 __global__ void __launch_bounds__(kThreads, 1)
 syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const WorkItem* __restrict__ items, int64_t N,
@@ -598,7 +685,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     k.abort_flag = &s_abort; k.status = status;
     k.tmA = &tmA; k.tmB = &tmB; k.tmC = &tmC;
     k.N = N; k.ncols = ncols; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
-    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = gemm_col_tiles > 0; k.syr2k = kSyr2k;
+    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = gemm_col_tiles > 0; k.syr2k = kSyr2k; k.herk = kHerk;
     // Strided batch: the grid holds the work list once per matrix; the tensor maps are 3-D.
     // K-split (slice_ksteps > 0): the grid holds the list once per slice of the inner dimension;
     // slice s takes K-steps [s * slice_ksteps, ...) of the 2-D maps and writes partial matrix s.
@@ -669,7 +756,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         return;
     }
-    mma_warp_item<kTN, kUpper, kSyr2k>(k, s_item, g, warp, lane);
+    mma_warp_item<kTN, kUpper, kSyr2k, kHerk>(k, s_item, g, warp, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -700,7 +787,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
     k.abort_flag = &s_abort; k.status = status;
     k.tmA = &tmA; k.tmB = &tmA; k.tmC = &tmC;
     k.N = N; k.ncols = N; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
-    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false; k.batch = -1; k.k0 = 0; k.syr2k = false;
+    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false; k.batch = -1; k.k0 = 0; k.syr2k = false; k.herk = false;
 
     if (tid == 0) {
         s_abort = 0;
@@ -799,7 +886,8 @@ cudaError_t configure_f64_kernels() {
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[7] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, true>),
+        const void* kernels[8] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, true>),
@@ -899,6 +987,20 @@ cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, con
     CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<false, false, true><<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmA, tmB, c_tma ? *tmC : none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status,
+        int64_t(0), int64_t(0), 0, 0, 1, nullptr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_herk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M,
+                            double* C, int64_t ldc, double alpha, double beta, int* d_status, cudaStream_t stream) {
+    cudaError_t e = configure_f64_kernels();
+    if (e != cudaSuccess) return e;
+    if (n_items == 0) return cudaSuccess;
+    if ((reinterpret_cast<uintptr_t>(C) & 15) != 0) return cudaErrorInvalidValue;     // complex entries move as 16-byte words
+    const int32_t n_ksteps = int32_t((2 * M + f64::kBK - 1) / f64::kBK);             // the real view has 2M columns
+    CUtensorMap none{};
+    f64::syrk_f64_tbs_kernel<false, false, false, true><<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
+        tmA, tmA, none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, 1, 0, d_status,
         int64_t(0), int64_t(0), 0, 0, 1, nullptr);
     return cudaGetLastError();
 }

@@ -65,6 +65,27 @@ __global__ void syr2k_plain_kernel(int64_t N, int64_t M, const double* __restric
     *c = (beta == 0.0) ? alpha * s : alpha * s + beta * *c;
 }
 
+// Hermitian rank-k update, one thread per entry (i, j), j <= i; complex numbers as (re, im) pairs.
+__global__ void herk_plain_kernel(int64_t N, int64_t M, const double* __restrict__ A, int64_t lda,
+                                  double* __restrict__ C, int64_t ldc, double alpha, double beta) {
+    const int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t i = int64_t(blockIdx.y) * blockDim.y + threadIdx.y;
+    if (i >= N || j > i) return;
+    const double* ai = A + 2 * i * lda;
+    const double* aj = A + 2 * j * lda;
+    double sr = 0.0, si = 0.0;
+    for (int64_t k = 0; k < M; ++k) {
+        const double a = ai[2 * k], b = ai[2 * k + 1], c = aj[2 * k], d = aj[2 * k + 1];
+        sr = fma(a, c, fma(b, d, sr));
+        si = fma(b, c, fma(-a, d, si));
+    }
+    double* c = C + 2 * (i * ldc + j);
+    double vr = alpha * sr, vi = alpha * si;
+    if (beta != 0.0) { vr += beta * c[0]; if (i != j) vi += beta * c[1]; }
+    c[0] = vr;
+    c[1] = (i == j) ? 0.0 : vi;
+}
+
 // The same for the storage types that accumulate in binary32 (each product is exact in binary32).
 template <typename TA>
 __global__ void syr2k_plain_f32_kernel(int64_t N, int64_t M, const TA* __restrict__ A, int64_t lda, const TA* __restrict__ B,
@@ -124,6 +145,14 @@ cudaError_t launch_syr2k_plain(int64_t N, int64_t M, const double* A, int64_t ld
     if (N == 0) return cudaSuccess;
     const dim3 block(32, 8);
     syr2k_plain_kernel<<<grid2d(N, block), block, 0, stream>>>(N, M, A, lda, B, ldb, C, ldc, alpha, beta);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_herk_plain(int64_t N, int64_t M, const double* A, int64_t lda, double* C, int64_t ldc,
+                              double alpha, double beta, cudaStream_t stream) {
+    if (N == 0) return cudaSuccess;
+    const dim3 block(32, 8);
+    herk_plain_kernel<<<grid2d(N, block), block, 0, stream>>>(N, alpha == 0.0 ? 0 : M, A, lda, C, ldc, alpha, beta);
     return cudaGetLastError();
 }
 

@@ -22,7 +22,7 @@ def built():
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "tbsyrk.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b((?:syrk|syr2k|tbs|cholesky)_[a-z_0-9]+)\s*\(", header))
+    declared = set(re.findall(r"\b((?:syrk|syr2k|herk|tbs|cholesky)_[a-z_0-9]+)\s*\(", header))
     assert declared == set(B.EXPORTS)
     L = ctypes.CDLL(B.LIB_PATH)
     for name in declared:
