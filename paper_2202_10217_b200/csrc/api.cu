@@ -64,20 +64,20 @@ int auto_split_k(const std::vector<WorkItem>& items, int64_t M, int bk, int sm_c
 
 // K-slices for an FP64 call (one block per item).  With fewer items than SMs the inner
 // dimension is cut so that more blocks run at once; the slices' partial matrices are
-// summed by a second kernel.  Model, in microseconds: a K-step of an item takes about 2, an item's
-// start-up and write-out about 6, the reduction streams slices * N^2 / 2 doubles at about 5 TB/s
-// after a launch gap of about 4.  A slice keeps at least 32 K-steps.
+// summed by a second kernel.  Model, in microseconds, fitted to measured calls of 512 to 1024 rows and 256 to
+// 1024 columns under 1 to 16 slices: 4 for the launch; per round of blocks 4.3 plus 2.14 per K-step of a
+// slice; for the reduction 3 plus 0.25 per slice and 512 x 512 entries.  A slice keeps at least 2 K-steps.
 int auto_split_k_f64(int64_t n_items, int64_t N, int64_t M, int bk, int sm_count, int forced) {
     const int64_t ksteps = (M + bk - 1) / bk;
     if (forced > 0) return int(std::max<int64_t>(1, std::min<int64_t>(forced, ksteps)));
-    if (n_items == 0 || n_items >= int64_t(sm_count) || ksteps < 64) return 1;
+    if (n_items == 0 || n_items >= int64_t(sm_count) || ksteps < 4) return 1;
     int best = 1;
     double best_cost = 0.0;
-    for (int s = 1; s <= 16 && s <= ksteps / 32; ++s) {
+    for (int s = 1; s <= 16 && s <= ksteps / 2; ++s) {
         if (s > 1 && double(s) * double(N) * double(N) * 8.0 > 512e6) break;        // workspace cap
-        const int64_t waves = (n_items * s + sm_count - 1) / sm_count;
-        double cost = double(waves) * (2.0 * double((ksteps + s - 1) / s) + 6.0);
-        if (s > 1) cost += 4.0 + double(s) * double(N) * double(N) * 4.0 / 5e6;
+        const int64_t rounds = (n_items * s + sm_count - 1) / sm_count;
+        double cost = 4.0 + double(rounds) * (2.14 * double((ksteps + s - 1) / s) + 4.3);
+        if (s > 1) cost += 3.0 + 0.25 * double(s) * double(N) * double(N) / (512.0 * 512.0);
         if (s == 1 || cost < best_cost) { best = s; best_cost = cost; }
     }
     return best;
