@@ -460,10 +460,14 @@ int syrk_set_f64_tail_split(int slices, int64_t tail_items);
  * How later FP64 calls hand the work items of the schedule (Algorithm 4, tiled as in
  * Section 5.1.4) to thread blocks; the paper has no counterpart, results are the same
  * entry for entry.  PER_ITEM: one thread block per item.  PERSISTENT: one block per SM
- * that draws items from a device-side counter, so an item's first loads overlap the
- * previous item's write-out; used only outside stream capture and for at most 256
- * distinct streams per device, else the call falls back to PER_ITEM.  AUTO (default):
- * PERSISTENT when M <= 1024 and the list has at least four items per SM.
+ * that draws items from a device-side counter; its MMA warps leave each item's
+ * accumulators in shared memory and separate warps write them out during the next item's
+ * M loop (beta == 0: stores; beta == 1: one floating-point add per entry done by the memory
+ * system, the correctly rounded sum; another beta: a multiply-add in those warps, which is slow
+ * because the tensor-core work holds the FP64 pipes).  Used only outside stream capture and for
+ * at most 256 distinct streams per device, else the call falls back to PER_ITEM.  AUTO (default):
+ * PERSISTENT for beta == 0 or 1 when the list has at least eight items per SM, or at least
+ * one per SM with M at most 300 columns per round of items; PER_ITEM otherwise.
  * Returns SYRK_ERR_PLAN for another value.  Process-wide.
  */
 #define SYRK_F64_LAUNCH_AUTO 0

@@ -62,6 +62,16 @@ int auto_split_k(const std::vector<WorkItem>& items, int64_t M, int bk, int sm_c
     return best;
 }
 
+// The automatic choice of the FP64 launch form.  Persistent blocks hide every item's write-out behind the next
+// item's M loop (for beta == 0 and beta == 1, see the kernel); one block per item has the tail K-split to even out
+// the last round of a list of a few rounds of long items.  Measured on 2048 to 16384 rows and 256 to 4096 columns:
+// persistent blocks win from about nine rounds of items on whatever the inner dimension, and on shorter lists
+// while an item is short against the list (M up to about 300 columns per round).
+bool f64_persistent_pays(int64_t M, int64_t n_items, double beta, int sm_count) {
+    if (!(beta == 0.0 || beta == 1.0) || n_items < int64_t(sm_count)) return false;
+    return n_items >= 8 * int64_t(sm_count) || M * int64_t(sm_count) <= 300 * n_items;
+}
+
 // K-slices for an FP64 call (one block per item).  With fewer items than SMs the inner
 // dimension is cut so that more blocks run at once; the slices' partial matrices are
 // summed by a second kernel.  Model, in microseconds, fitted to measured calls of 512 to 1024 rows and 256 to
@@ -151,12 +161,11 @@ int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkIt
         CUtensorMap tmc;
         const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
                            encode_tensor_map_c_f64(&tmc, C, N, ldc, f64_tile()) == SYRK_OK;
-        // Persistent blocks hide each item's start-up (a few microseconds) behind the previous item.
-        // That pays when items are short (M <= 1024: at most 64 stages each) and the list fills the
-        // device several times over; for long items one block per item is the faster form.
+        // Persistent blocks hide each item's start-up and write-out behind the next item's M loop
+        // (see f64_persistent_pays for when that is the faster form).
         const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
         const bool persistent = !upper && tail_slices <= 1 && (mode == SYRK_F64_LAUNCH_PERSISTENT ||
-                                (mode == SYRK_F64_LAUNCH_AUTO && M <= 1024 && n_items >= 4 * int64_t(ds->sm_count)));
+                                (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(M, n_items, beta, ds->sm_count)));
         int* tickets = (persistent && split <= 1) ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<double*>(C), ldc,
                             alpha, beta, a_is_m_by_n, tickets, ds->sm_count, d_status, stream, 0, 0, split,
@@ -348,7 +357,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         const int64_t n_items = int64_t(dp->plan.items.size());
         const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
         const bool per_item = upper || mode == SYRK_F64_LAUNCH_PER_ITEM ||
-                              (mode == SYRK_F64_LAUNCH_AUTO && !(M <= 1024 && n_items >= 4 * int64_t(ds->sm_count)));
+                              (mode == SYRK_F64_LAUNCH_AUTO && !f64_persistent_pays(M, n_items, beta, ds->sm_count));
         if (split == 1 && per_item && !upper && runtime().f64_tail_slices != 1) {
             TailSplit ts{n_items, 1};
             const int64_t ksteps = (M + ks.bk - 1) / ks.bk;

@@ -9,10 +9,11 @@
 namespace tbsyrk {
 
 // FP64 triangle-block kernel.  `tmC` (may be null): tensor map over C with 32 x 32 FP64 boxes, no
-// swizzle, through which the old C tiles are fetched when beta != 0.  With `d_tickets` null there
-// is one thread block per work item; otherwise `n_blocks` persistent blocks draw the items from
-// d_tickets[0] (d_tickets[0..1] must be zero and must not be shared with a launch that can run at
-// the same time; the kernel leaves them zero).  `a_is_m_by_n`: A is stored M x N row-major (the
+// swizzle, through which the old C tiles are fetched when beta != 0 (one block per item).  With
+// `d_tickets` null there is one thread block per work item; otherwise `n_blocks` persistent blocks
+// draw the items from d_tickets[0] (d_tickets[0..1] must be zero and must not be shared with a launch
+// that can run at the same time; the kernel leaves them zero); that form writes C from three extra
+// warps per block and reads old C from memory.  `a_is_m_by_n`: A is stored M x N row-major (the
 // Gram form C = A^T A); `tmA` then has boxes of 16 rows x 16 columns over that array.
 // `batch` > 0: strided batch of `batch` problems; `tmA` and `tmC` are then 3-D maps whose last
 // coordinate is the matrix number, matrix b of C starts at C + b * c_batch_stride, and the launch

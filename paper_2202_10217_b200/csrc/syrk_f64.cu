@@ -26,8 +26,9 @@
 // out the items; used for short lists and for the two-operand mode), and a persistent form,
 // one block per SM, whose producer draws the next item from a global counter and publishes
 // it to the MMA warps through a small ring in shared memory: the ring of stages then runs on
-// across items and the next item's first stages are in flight while the current one is
-// finished and written out.
+// across items.  In the persistent form the MMA warps do not write C themselves: they leave their
+// accumulators in a shared-memory image and three more warps write it out (reading old C from memory
+// when beta != 0) while the next item's M loop runs; its ring has three stages.
 //
 // Accumulators (the C block) stay on chip for the whole M loop and each entry of
 // C is read (beta != 0) and written exactly once, as in the paper's generic
@@ -63,6 +64,7 @@ __device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
 struct Call {
     uint8_t* smem;                 // the ring of stages
     uint32_t smem32, bars32;       // shared-space addresses of the ring and of full_bar[0] (MMA warps use these)
+    uint32_t empties32;            // ... and of empty_bar[0]
     uint64_t* full_bar;
     uint64_t* empty_bar;           // 16 arrivals (one per MMA warp) free a stage
     volatile int* abort_flag;
@@ -94,12 +96,12 @@ __device__ __forceinline__ int c_steps_of(const Call& k, int n_tile) { return k.
 // ---------------------------------------------------------------------------------------------
 // Producer (one thread): fetch one item's ring steps, starting at global step g.
 // ---------------------------------------------------------------------------------------------
-template <bool kTN>
+template <bool kTN, int kSt = kStages>
 __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, uint32_t& g) {
     const int n_seg = it.n_seg, n_tile = it.n_tile;
     for (int ks = 0; ks < k.n_ksteps; ++ks, ++g) {
-        const uint32_t st = g % kStages;
-        if (g >= kStages && !mbar_wait_bounded(&k.empty_bar[st], ((g / kStages) - 1) & 1, k.abort_flag)) {
+        const uint32_t st = g % kSt;
+        if (g >= kSt && !mbar_wait_bounded(&k.empty_bar[st], ((g / kSt) - 1) & 1, k.abort_flag)) {
             *k.abort_flag = 1; atomicOr(k.status, kStatusWaitEmpty); return false;
         }
         mbar_arrive_expect_tx(&k.full_bar[st], uint32_t(k.syr2k ? 2 * n_seg : n_seg) * kSegBytes);
@@ -125,8 +127,8 @@ __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, 
     // Old C: ring step j carries tiles 4j .. 4j+3 (8 KB each, row pitch 256 B), those below the diagonal.
     const int n_c = c_steps_of(k, n_tile);
     for (int j = 0; j < n_c; ++j, ++g) {
-        const uint32_t st = g % kStages;
-        if (g >= kStages && !mbar_wait_bounded(&k.empty_bar[st], ((g / kStages) - 1) & 1, k.abort_flag)) {
+        const uint32_t st = g % kSt;
+        if (g >= kSt && !mbar_wait_bounded(&k.empty_bar[st], ((g / kSt) - 1) & 1, k.abort_flag)) {
             *k.abort_flag = 1; atomicOr(k.status, kStatusWaitEmpty); return false;
         }
         int below = 0;
@@ -145,10 +147,11 @@ __device__ __forceinline__ bool produce_item(const Call& k, const WorkItem& it, 
 }
 
 // After a give-up: let the copies still in flight land before the block exits.
+template <int kSt = kStages>
 __device__ void drain_producer(const Call& k, uint32_t g) {
-    for (uint32_t i = (g > kStages ? g - kStages : 0); i < g; ++i) {
+    for (uint32_t i = (g > kSt ? g - kSt : 0); i < g; ++i) {
         volatile int dummy = 0;
-        mbar_wait_bounded(&k.full_bar[i % kStages], (i / kStages) & 1, &dummy);
+        mbar_wait_bounded(&k.full_bar[i % kSt], (i / kSt) & 1, &dummy);
     }
 }
 
@@ -211,7 +214,7 @@ __device__ __forceinline__ bool wait_full_at(const Call& k, uint32_t st, uint32_
 }
 __device__ __forceinline__ void release_at(const Call& k, uint32_t st, int lane) {
     __syncwarp();
-    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(k.bars32 + (kStages + st) * 8) : "memory");
+    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(k.empties32 + st * 8) : "memory");
 }
 __device__ __forceinline__ bool wait_full(const Call& k, uint32_t g, int lane) {
     return wait_full_at(k, g % kStages, (g / kStages) & 1, lane);
@@ -229,10 +232,10 @@ __device__ __forceinline__ uint32_t frag_addr(uint32_t p, int j, int sl) {
     return (p ^ uint32_t(sl << 4)) + uint32_t(j * 1024);
 }
 
-template <bool kSkipLast, bool kTN>
+template <bool kSkipLast, bool kTN, int kSt = kStages>
 __device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const Call& k, uint32_t xbase, uint32_t ybase,
                                               uint32_t off0, uint32_t g0, int lane) {
-    uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;      // stage and phase, advanced step by step
+    uint32_t st = g0 % kSt, parity = (g0 / kSt) & 1;              // stage and phase, advanced step by step
     for (int ks = 0; ks < k.n_ksteps; ++ks) {
         if (!wait_full_at(k, st, parity, lane)) return false;
         const uint32_t stage = k.smem32 + st * kStageBytes;
@@ -252,7 +255,7 @@ __device__ __forceinline__ bool tile_mainloop(double (&acc)[4][4][2], const Call
                     if (!(kSkipLast && mi == 3 && ni == 3)) dmma884(acc[mi][ni], a[mi], b[ni]);
         }
         release_at(k, st, lane);
-        if (++st == kStages) { st = 0; parity ^= 1; }
+        if (++st == kSt) { st = 0; parity ^= 1; }
     }
     return true;
 }
@@ -281,21 +284,13 @@ __device__ __forceinline__ uint32_t fragment_offset_tn(int lane) {
     return uint32_t(k_lane * 128 + ((((g >> 1) ^ k_lane)) << 4) + ((g & 1) << 3));
 }
 
-// 16th warp of a triangle block: the 15 left-out 8 x 8 blocks.  g0 = the item's first ring step,
-// n_c = its old-C steps.
-template <bool kTN, bool kUpper>
-__device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, int lane) {
-    const int gq = lane >> 2, t = lane & 3;
-    const uint32_t gc = g0 + uint32_t(k.n_ksteps);
-    const bool use_beta = (k.beta != 0.0);
-    const uint32_t off0 = kTN ? fragment_offset_tn(lane) : fragment_offset(lane);
-    int32_t seg[6];
-#pragma unroll
-    for (int s = 0; s < 6; ++s) seg[s] = it.seg[s];
-    double sacc[15][2];
+// The M loop of the 16th warp of a triangle block: block q = (x, y), y < x, of the 15 left-out 8 x 8 blocks
+// is the product of rows 24..31 of segments x and y.
+template <bool kTN, int kSt = kStages>
+__device__ __forceinline__ bool scavenger_mainloop(double (&sacc)[15][2], const Call& k, uint32_t off0, uint32_t g0, int lane) {
 #pragma unroll
     for (int q = 0; q < 15; ++q) sacc[q][0] = sacc[q][1] = 0.0;
-    uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;
+    uint32_t st = g0 % kSt, parity = (g0 / kSt) & 1;
     for (int ks = 0; ks < k.n_ksteps; ++ks) {
         if (!wait_full_at(k, st, parity, lane)) return false;
         const uint32_t base = (k.smem32 + st * kStageBytes) | off0;
@@ -311,8 +306,24 @@ __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it
                 for (int y = 0; y < x; ++y, ++q) dmma884(sacc[q], f[x], f[y]);
         }
         release_at(k, st, lane);
-        if (++st == kStages) { st = 0; parity ^= 1; }
+        if (++st == kSt) { st = 0; parity ^= 1; }
     }
+    return true;
+}
+
+// 16th warp of a triangle block: the 15 left-out 8 x 8 blocks.  g0 = the item's first ring step,
+// n_c = its old-C steps.
+template <bool kTN, bool kUpper>
+__device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, int lane) {
+    const int gq = lane >> 2, t = lane & 3;
+    const uint32_t gc = g0 + uint32_t(k.n_ksteps);
+    const bool use_beta = (k.beta != 0.0);
+    const uint32_t off0 = kTN ? fragment_offset_tn(lane) : fragment_offset(lane);
+    int32_t seg[6];
+#pragma unroll
+    for (int s = 0; s < 6; ++s) seg[s] = it.seg[s];
+    double sacc[15][2];
+    if (!scavenger_mainloop<kTN>(sacc, k, off0, g0, lane)) return false;
     for (int j = 0; j < n_c; ++j)
         if (!wait_full(k, gc + j, lane)) return false;
     int q = 0;
@@ -681,7 +692,7 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     k.smem = smem;
     k.full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
     k.empty_bar = k.full_bar + kStages;
-    k.smem32 = smem_u32(smem); k.bars32 = smem_u32(k.full_bar);
+    k.smem32 = smem_u32(smem); k.bars32 = smem_u32(k.full_bar); k.empties32 = k.bars32 + kStages * 8;
     k.abort_flag = &s_abort; k.status = status;
     k.tmA = &tmA; k.tmB = &tmB; k.tmC = &tmC;
     k.N = N; k.ncols = ncols; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
@@ -762,16 +773,147 @@ syrk_f64_tbs_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 // ---------------------------------------------------------------------------------------------
 // Persistent form: one block per SM; the producer draws items from counter[0] (zero at launch;
 // counter[1] counts the producers that are done) and publishes them through a ring of kItemRing
-// slots.  The producer is never more than
-// kStages ring steps - hence fewer than kItemRing items - ahead of the slowest MMA warp, so a
-// slot is rewritten only after every warp has read it.
+// slots.  The producer is never more than kPStages ring steps - hence fewer than kItemRing items -
+// ahead of the slowest MMA warp, so a slot is rewritten only after every warp has read it.
+//
+// Write-out off the MMA warps: at the end of an item an MMA warp only copies its accumulators into a
+// 128 KB image in shared memory (one 32 x 32 slot per tile) and goes on with the next item's stages, which
+// are already in the ring; three write-out warps then form alpha * acc + beta * C from the image and store
+// it while the DMMA pipes work on the next item.  (With the write-out in the MMA warps all sixteen do it at
+// once and the pipes idle for the 128 KB that one SM has to move per item.)  The image takes the room of
+// three of the six stages: this form runs a 3-stage ring, and old C is read from memory by the write-out
+// warps, which have an item's duration to hide that latency.
 // ---------------------------------------------------------------------------------------------
+constexpr int kPStages = 3;
+constexpr int kOutWarps = 3;
+constexpr int kOutBatch = 4;                     // row pairs of a tile a write-out warp has in flight
+constexpr int kPThreads = (kMmaWarps + 1 + kOutWarps) * 32;
+constexpr int kImageBytes = kMmaWarps * kCTileBytes;
+constexpr int kPSmemBytes = kPStages * kStageBytes + kImageBytes + (2 * kPStages + 2) * 8 + 1024;
+
+// Entry (row r, 16-byte chunk c) of a tile's image: chunk index flipped in bit 2 on odd rows, so that both the
+// fragment-shaped stores of the MMA warps (rows g, g + 1 x chunks 4 ni + t per quarter warp) and the row-shaped
+// loads of the write-out warps are free of bank conflicts.
+__device__ __forceinline__ uint32_t image_offset(int r, int c) { return uint32_t(r * 256 + ((c ^ ((r & 1) << 2)) << 4)); }
+__device__ __forceinline__ void sts_f64x2(uint32_t addr, double v0, double v1) {
+    asm volatile("st.shared.v2.f64 [%0], {%1, %2};" ::"r"(addr), "d"(v0), "d"(v1) : "memory");
+}
+__device__ __forceinline__ double2 lds_f64x2(uint32_t addr) {
+    double2 v;
+    asm volatile("ld.shared.v2.f64 {%0, %1}, [%2];" : "=d"(v.x), "=d"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+
+// What the persistent form adds to Call: the image and its two barriers (full: 16 arrivals, one per MMA warp
+// and item; empty: one arrival per write-out warp and item).
+struct Image {
+    uint32_t base32, full32, empty32;
+};
+
+__device__ __forceinline__ bool wait_image_empty(const Call& k, const Image& im, uint32_t item_no, int lane) {
+    if (item_no == 0) return true;
+    const uint32_t parity = (item_no - 1) & 1;
+    if (try_wait32(im.empty32, parity)) return true;
+    return wait_full_slow(im.empty32, parity, k.abort_flag, k.status, lane);
+}
+
+// One MMA warp's share of item number item_no of its block: the M loop, then its accumulators into the image.
 template <bool kTN>
-__global__ void __launch_bounds__(kThreads, 1)
-syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmC,
-                               const WorkItem* __restrict__ items, int64_t n_items, int* __restrict__ counter,
-                               int64_t N, int32_t n_ksteps, double* __restrict__ C, int64_t ldc, double alpha,
-                               double beta, int vec_ok, int c_tma, int* __restrict__ status) {
+__device__ __forceinline__ bool mma_warp_item_p(const Call& k, const Image& im, const WorkItem& it, uint32_t& g,
+                                                uint32_t item_no, int warp, int lane) {
+    const int gq = lane >> 2, t = lane & 3;
+    const int n_tile = it.n_tile;
+    const uint32_t g0 = g;
+    g += uint32_t(k.n_ksteps);
+    const bool scavenge = it.pad != 0;                  // set by prepare_item
+    const uint32_t off0 = kTN ? fragment_offset_tn(lane) : fragment_offset(lane);
+    if (scavenge && warp == kMmaWarps - 1) {
+        double sacc[15][2];
+        if (!scavenger_mainloop<kTN, kPStages>(sacc, k, off0, g0, lane)) return false;
+        if (!wait_image_empty(k, im, item_no, lane)) return false;
+#pragma unroll
+        for (int q = 0; q < 15; ++q)                    // block (3, 3) of tile q
+            sts_f64x2(im.base32 + q * kCTileBytes + image_offset(24 + gq, 12 + t), k.alpha * sacc[q][0], k.alpha * sacc[q][1]);
+    } else if (warp < n_tile) {
+        const uint32_t xbase = uint32_t(it.tile_x[warp]) * kSegBytes, ybase = uint32_t(it.tile_y[warp]) * kSegBytes;
+        double acc[4][4][2];
+#pragma unroll
+        for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+            for (int ni = 0; ni < 4; ++ni) acc[mi][ni][0] = acc[mi][ni][1] = 0.0;
+        const bool alive = scavenge ? tile_mainloop<true, kTN, kPStages>(acc, k, xbase, ybase, off0, g0, lane)
+                                    : tile_mainloop<false, kTN, kPStages>(acc, k, xbase, ybase, off0, g0, lane);
+        if (!alive) return false;
+        if (!wait_image_empty(k, im, item_no, lane)) return false;
+        const uint32_t tile32 = im.base32 + warp * kCTileBytes;
+#pragma unroll
+        for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+            for (int ni = 0; ni < 4; ++ni) {
+                if (scavenge && mi == 3 && ni == 3) continue;         // written by the 16th warp
+                sts_f64x2(tile32 + image_offset(mi * 8 + gq, ni * 4 + t), k.alpha * acc[mi][ni][0], k.alpha * acc[mi][ni][1]);
+            }
+    } else {
+        uint32_t st = g0 % kPStages, parity = (g0 / kPStages) & 1;    // no tile in this item: keep the ring moving
+        for (int ks = 0; ks < k.n_ksteps; ++ks) {
+            if (!wait_full_at(k, st, parity, lane)) return false;
+            release_at(k, st, lane);
+            if (++st == kPStages) { st = 0; parity ^= 1; }
+        }
+    }
+    __syncwarp();
+    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(im.full32) : "memory");
+    return true;
+}
+
+// A write-out warp's share of one item: tiles out_warp, out_warp + 3, ... of the image, which holds alpha * acc.
+// A warp instruction covers two rows of a tile (16 lanes x 16 bytes each): 256 contiguous bytes of C per row.
+// The DMMA pipes are the FP64 pipes, and the MMA warps keep them full: an FP64 instruction issued from here
+// waits behind them for most of an item.  So beta == 0 is a copy, and beta == 1 an addition done by the
+// memory system (red.global.add.f64, one per entry and call: the result does not depend on any order, and it is
+// the correctly rounded sum that the multiply-add of the other launch form gives for beta == 1); any other
+// beta does its multiply-add here and is slow - the automatic choice of the launch form avoids it.
+__device__ __forceinline__ void red_add_f64(double* p, double v) {
+    asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p), "d"(v) : "memory");
+}
+__device__ __forceinline__ void write_out_item(const Call& k, const Image& im, const WorkItem& it, int out_warp, int lane) {
+    const int mode = (k.beta == 0.0) ? 0 : (k.beta == 1.0 ? 1 : 2);
+    const int half = lane >> 4, c16 = lane & 15;
+    for (int q = out_warp; q < it.n_tile; q += kOutWarps) {
+        const int64_t row0 = int64_t(it.seg[it.tile_x[q]]) * kTile, col0 = int64_t(it.seg[it.tile_y[q]]) * kTile;
+        const uint32_t tile32 = im.base32 + q * kCTileBytes;
+        for (int i0 = 0; i0 < 16; i0 += kOutBatch) {
+            double2 v[kOutBatch];
+#pragma unroll
+            for (int i = 0; i < kOutBatch; ++i) v[i] = lds_f64x2(tile32 + uint32_t((2 * (i0 + i) + half) * 256 + (c16 << 4)));
+#pragma unroll
+            for (int i = 0; i < kOutBatch; ++i) {
+                const int r = 2 * (i0 + i) + half;
+                const int64_t R = row0 + r, c = col0 + 2 * (c16 ^ ((r & 1) << 2));
+                if (R >= k.N || c > R) continue;                       // beyond the last row, or above the diagonal
+                double* p = k.C + R * k.ldc + c;
+                const bool both = (c + 1 <= R);
+                if (mode == 0) {
+                    if (both && (k.vec_ok & 1)) *reinterpret_cast<double2*>(p) = v[i];
+                    else { p[0] = v[i].x; if (both) p[1] = v[i].y; }
+                } else if (mode == 1) {
+                    red_add_f64(p, v[i].x);
+                    if (both) red_add_f64(p + 1, v[i].y);
+                } else {
+                    p[0] = v[i].x + k.beta * p[0];
+                    if (both) p[1] = v[i].y + k.beta * p[1];
+                }
+            }
+        }
+    }
+}
+
+template <bool kTN>
+__global__ void __launch_bounds__(kPThreads, 1)
+syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __restrict__ items,
+                               int64_t n_items, int* __restrict__ counter, int64_t N, int32_t n_ksteps,
+                               double* __restrict__ C, int64_t ldc, double alpha, double beta, int vec_ok,
+                               int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ WorkItem s_ring[kItemRing];
@@ -781,27 +923,34 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
 
     Call k;
     k.smem = smem;
-    k.full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
-    k.empty_bar = k.full_bar + kStages;
-    k.smem32 = smem_u32(smem); k.bars32 = smem_u32(k.full_bar);
+    k.full_bar = reinterpret_cast<uint64_t*>(smem + kPStages * kStageBytes + kImageBytes);
+    k.empty_bar = k.full_bar + kPStages;
+    uint64_t* image_bar = k.empty_bar + kPStages;            // [0] full, [1] empty
+    k.smem32 = smem_u32(smem); k.bars32 = smem_u32(k.full_bar); k.empties32 = k.bars32 + kPStages * 8;
     k.abort_flag = &s_abort; k.status = status;
-    k.tmA = &tmA; k.tmB = &tmA; k.tmC = &tmC;
+    k.tmA = &tmA; k.tmB = &tmA; k.tmC = &tmA;
     k.N = N; k.ncols = N; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
-    k.vec_ok = vec_ok; k.c_tma = c_tma; k.gemm = false; k.batch = -1; k.k0 = 0; k.syr2k = false; k.herk = false;
+    k.vec_ok = vec_ok; k.c_tma = 0; k.gemm = false; k.batch = -1; k.k0 = 0; k.syr2k = false; k.herk = false;
+    Image im;
+    im.base32 = k.smem32 + kPStages * kStageBytes;
+    im.full32 = smem_u32(&image_bar[0]);
+    im.empty32 = smem_u32(&image_bar[1]);
 
     if (tid == 0) {
         s_abort = 0;
-        for (int s = 0; s < kStages; ++s) { mbar_init(&k.full_bar[s], 1); mbar_init(&k.empty_bar[s], kMmaWarps); }
+        for (int s = 0; s < kPStages; ++s) { mbar_init(&k.full_bar[s], 1); mbar_init(&k.empty_bar[s], kMmaWarps); }
+        mbar_init(&image_bar[0], kMmaWarps);
+        mbar_init(&image_bar[1], kOutWarps);
         for (int s = 0; s < kItemRing; ++s) mbar_init(&s_item_bar[s], 1);
         mbar_fence_init();
     }
     __syncthreads();
 
+    // Warps 0..2 write out, warp 3 produces, warps 4..19 are MMA warps 0..15 (four per scheduler).
     uint32_t g = 0;
-    if (warp == kMmaWarps) {
+    if (warp == kOutWarps) {
         if (lane == 0) {
             prefetch_tensormap(&tmA);
-            if (c_tma) prefetch_tensormap(&tmC);
             for (uint32_t slot = 0;; ++slot) {
                 WorkItem& dst = s_ring[slot % kItemRing];
                 const int64_t idx = s_abort ? n_items : int64_t(atomicAdd(counter, 1));
@@ -814,19 +963,38 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                 if (last) dst.n_tile = -1;                        // end marker
                 mbar_arrive(&s_item_bar[slot % kItemRing]);       // publishes the slot (release)
                 if (last) break;
-                if (!produce_item<kTN>(k, dst, g)) {                   // gave up: tell the MMA warps to stop as well
+                if (!produce_item<kTN, kPStages>(k, dst, g)) {     // gave up: tell the other warps to stop as well
                     WorkItem& end = s_ring[(slot + 1) % kItemRing];
                     end.n_tile = -1;
                     mbar_arrive(&s_item_bar[(slot + 1) % kItemRing]);
                     break;
                 }
             }
-            if (s_abort) drain_producer(k, g);
+            if (s_abort) drain_producer<kPStages>(k, g);
             // The last producer to get here puts both tickets back to zero for the next launch
             // on this stream: by then no block draws any more.
             if (atomicAdd(counter + 1, 1) == int(gridDim.x) - 1) { atomicExch(counter, 0); atomicExch(counter + 1, 0); }
         }
         return;
+    }
+    if (warp < kOutWarps) {
+        // Write-out warps: item after item, one item behind the MMA warps at most (they wait for the image to be
+        // empty before they fill it again), so the slot of the item ring is still the item's.
+        const int out_warp = warp;
+        for (uint32_t slot = 0;; ++slot) {
+            if (!mbar_wait_bounded(&s_item_bar[slot % kItemRing], (slot / kItemRing) & 1, &s_abort)) {
+                s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); return;
+            }
+            const WorkItem& it = s_ring[slot % kItemRing];
+            if (it.n_tile < 0) return;
+            if (!mbar_wait_bounded(&image_bar[0], slot & 1, &s_abort)) {
+                if (s_abort == 0) { s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); }
+                return;
+            }
+            write_out_item(k, im, it, out_warp, lane);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&image_bar[1]);
+        }
     }
     for (uint32_t slot = 0;; ++slot) {
         if (!mbar_wait_bounded(&s_item_bar[slot % kItemRing], (slot / kItemRing) & 1, &s_abort)) {
@@ -834,7 +1002,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
         }
         const WorkItem& it = s_ring[slot % kItemRing];
         if (it.n_tile < 0) return;
-        if (!mma_warp_item<kTN, false>(k, it, g, warp, lane)) return;
+        if (!mma_warp_item_p<kTN>(k, im, it, g, slot, warp - kOutWarps - 1, lane)) return;
     }
 }
 
@@ -895,7 +1063,9 @@ cudaError_t configure_f64_kernels() {
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true>)};
         for (const void* fn : kernels) {
-            cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, f64::kSmemBytes);
+            const bool persistent = fn == kernels[6] || fn == kernels[7];
+            cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 persistent ? f64::kPSmemBytes : f64::kSmemBytes);
             if (e != cudaSuccess) return e;
         }
         configured[dev] = true;
@@ -949,8 +1119,8 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30) && !upper) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true> : f64::syrk_f64_tbs_persistent_kernel<false>;
-        kernel<<<grid, threads, f64::kSmemBytes, stream>>>(tmA, c_tma ? *tmC : none, d_items, n_items, d_tickets, N,
-                                                           n_ksteps, C, ldc, alpha, beta, vec_ok, c_tma, d_status);
+        kernel<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, d_items, n_items, d_tickets, N, n_ksteps, C, ldc,
+                                                                         alpha, beta, vec_ok, d_status);
         return cudaGetLastError();
     }
     auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, true> : f64::syrk_f64_tbs_kernel<false, true>)
