@@ -205,10 +205,10 @@ def run_reference(args, key: str, shape, rank: int):
 # summarised under profiles/.  Valid only for the kernel source it was taken on: keyed by its SHA-256.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, kernel source file, sha256 of that file at capture time, square-schedule bytes or None)
-    "c2_f64_4096x4096": (833_247_744, "syrk_f64.cu", "dc0af5511d941afee99ca375ca5db108325e8474b096a5eaff9efcc6db1d6bef", 815_276_288),
+    "c2_f64_4096x4096": (829_197_312, "syrk_f64.cu", "6cfcb5d4ea6d5daaa57917c2f53b5ff04c792125d6983bf1e21a58e50e141e4d", 814_020_096),
     "c3_bf16_16384x4096": (1_898_579_968, "syrk_bf16.cu", "527f2140d892d840fb605c824d4e19c4706e87355a46c48bb934fb71b3a9a97b", 3_150_107_648),
     "c4_bf16_2048x262144": (1_308_831_488, "syrk_bf16_pair.cu", "1f007b0ed5552de540c0cf0f25685f828321404cc4f842d0dbfcbbdcc303fc01", 2_332_056_832),
-    "c5_call_n16384": (2_882_612_224, "syrk_f64.cu", "dc0af5511d941afee99ca375ca5db108325e8474b096a5eaff9efcc6db1d6bef", 2_727_926_272),
+    "c5_call_n16384": (2_698_881_536, "syrk_f64.cu", "6cfcb5d4ea6d5daaa57917c2f53b5ff04c792125d6983bf1e21a58e50e141e4d", 2_519_901_440),
 }
 
 
@@ -460,7 +460,8 @@ def record_sweep(args, T: Timer, B, torch, world, want_e2e: bool, peak_cache: di
         "value_sustained": whole_job_tflops(flops, world, sus_ms * 1e-3),
         "sustained": {"ms_per_step": sus_ms, "calls": sus_calls * len(sizes), "l2": "no flush, sweeps back to back",
                       "clocks": sus_clocks},
-        "gpu_launches": args.steps * len(sizes),
+        # one kernel per call, plus the reduction kernel of the few smallest calls that run in K-slices
+        "gpu_launches": args.steps * sum(B.syrk_get_schedule_stats(n, M, I.DTYPE_F64)["launches"] for n in sizes),
         "roofline": roofline_record(flops / len(sizes), kernel_ms / len(sizes), sus_ms / len(sizes), peak, peak_sus, note,
                                     traffic, None, {"launches_per_step": len(sizes)}),
     }

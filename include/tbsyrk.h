@@ -502,8 +502,9 @@ typedef struct {
     int64_t s_acc;           /* accumulator elements a thread block may hold         */
     int64_t s_total;         /* s_acc + staging elements (all pipeline stages)       */
     int32_t effective_schedule; /* what the call runs: syrk_effective_schedule()      */
-    int32_t launches;        /* kernels the call enqueues: 1, or 2 with a K-split (the
-                                slices' partial results are summed by a second kernel)  */
+    int32_t launches;        /* kernels the call enqueues: 1, or 2 with a K-split of the whole
+                                list or of its tail (the slices' partial results are summed
+                                by a second kernel); under the automatic FP64 settings     */
 } syrk_schedule_stats;
 
 int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats* out);

@@ -1046,6 +1046,17 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->effective_schedule = effective_schedule_of(N, M, dtype, 148, &split);
     out->split_k = split;
     out->launches = split > 1 ? 2 : 1;
+    if (dtype == SYRK_DTYPE_F64 && split == 1 && out->effective_schedule != SYRK_SCHEDULE_PAIR_SQUARE) {
+        // the tail K-split of the one-block-per-item form adds its reduction kernel (the launch form is taken as
+        // for beta == 0 or 1; the automatic settings are assumed)
+        int mode, tail_setting;
+        { std::lock_guard<std::mutex> lock(runtime().mu); mode = runtime().f64_launch; tail_setting = runtime().f64_tail_slices; }
+        const int64_t n_items = int64_t(plan.items.size());
+        const bool per_item = mode == SYRK_F64_LAUNCH_PER_ITEM ||
+                              (mode == SYRK_F64_LAUNCH_AUTO && !f64_persistent_pays(M, n_items, 0.0, 148));
+        if (per_item && tail_setting == 0 && plan_tail_split_f64(plan.items, (M + ks.bk - 1) / ks.bk, 148).slices > 1)
+            out->launches = 2;
+    }
     out->n_tiles = plan.p.n_tiles;
     out->items = int64_t(plan.items.size());
     out->tri_items = plan.n_tri;
