@@ -60,6 +60,12 @@ __device__ __forceinline__ void dmma884(double (&c)[2], double a, double b) {
                  : "d"(a), "d"(b));
 }
 
+// The write-out arithmetic, alpha * acc + beta * old, in one fixed rounding sequence - the product alpha * acc
+// rounded, then one fused multiply-add - so that every role and both launch forms give the same bits whatever
+// the compiler would contract.  (With beta == 1 the second step is the correctly rounded sum.)
+__device__ __forceinline__ double scaled(double alpha, double acc) { return __dmul_rn(alpha, acc); }
+__device__ __forceinline__ double plus_old(double v, double beta, double old) { return __fma_rn(beta, old, v); }
+
 // What every role of a block needs to know about the call.
 struct Call {
     uint8_t* smem;                 // the ring of stages
@@ -342,12 +348,12 @@ __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it
                     const int64_t r = int64_t(seg[y]) * kTile + 24 + 2 * t + e;
                     if (r >= k.N) continue;
                     double* p = k.C + r * k.ldc + c;
-                    double v = k.alpha * sacc[q][e];
+                    double v = scaled(k.alpha, sacc[q][e]);
                     if (n_c > 0)
-                        v += k.beta * *reinterpret_cast<const double*>(
+                        v = plus_old(v, k.beta, *reinterpret_cast<const double*>(
                                  k.smem + ((gc + (q >> 2)) % kStages) * kStageBytes + (q & 3) * kCTileBytes +
-                                 (24 + 2 * t + e) * (kTile * 8) + (24 + gq) * 8);
-                    else if (use_beta) v += k.beta * *p;
+                                 (24 + 2 * t + e) * (kTile * 8) + (24 + gq) * 8));
+                    else if (use_beta) v = plus_old(v, k.beta, *p);
                     *p = v;
                 }
                 continue;
@@ -361,13 +367,13 @@ __device__ __forceinline__ bool scavenger_role(const Call& k, const WorkItem& it
             const int64_t c = int64_t(seg[y]) * kTile + 24 + 2 * t;
             if (r >= k.N) continue;                                 // tile below the diagonal: c + 1 < r
             double* p = k.C + r * k.ldc + c;
-            double v0 = k.alpha * sacc[q][0], v1 = k.alpha * sacc[q][1];
+            double v0 = scaled(k.alpha, sacc[q][0]), v1 = scaled(k.alpha, sacc[q][1]);
             if (n_c > 0) {
                 const double2 o = *reinterpret_cast<const double2*>(
                     k.smem + ((gc + (q >> 2)) % kStages) * kStageBytes + (q & 3) * kCTileBytes +
                     (24 + gq) * (kTile * 8) + (24 + 2 * t) * 8);
-                v0 += k.beta * o.x; v1 += k.beta * o.y;
-            } else if (use_beta) { v0 += k.beta * p[0]; v1 += k.beta * p[1]; }
+                v0 = plus_old(v0, k.beta, o.x); v1 = plus_old(v1, k.beta, o.y);
+            } else if (use_beta) { v0 = plus_old(v0, k.beta, p[0]); v1 = plus_old(v1, k.beta, p[1]); }
             if (k.vec_ok) *reinterpret_cast<double2*>(p) = make_double2(v0, v1);
             else { p[0] = v0; p[1] = v1; }
         }
@@ -415,12 +421,12 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
                 const int64_t c = col0 + ni * 8 + 2 * t;
                 const bool ok0 = c >= r && c < k.N, ok1 = c + 1 >= r && c + 1 < k.N;
                 if (!ok0 && !ok1) continue;
-                double v0 = k.alpha * acc[mi][ni][0], v1 = k.alpha * acc[mi][ni][1];
+                double v0 = scaled(k.alpha, acc[mi][ni][0]), v1 = scaled(k.alpha, acc[mi][ni][1]);
                 if (use_beta) {
                     double2 o = make_double2(0.0, 0.0);
                     if (old_tile) o = *reinterpret_cast<const double2*>(old_tile + (mi * 8 + gq) * (kTile * 8) + (ni * 8 + 2 * t) * 8);
                     else { if (ok0) o.x = crow[c]; if (ok1) o.y = crow[c + 1]; }
-                    v0 += k.beta * o.x; v1 += k.beta * o.y;
+                    v0 = plus_old(v0, k.beta, o.x); v1 = plus_old(v1, k.beta, o.y);
                 }
                 if (ok0 && ok1 && k.vec_ok) *reinterpret_cast<double2*>(crow + c) = make_double2(v0, v1);
                 else { if (ok0) crow[c] = v0; if (ok1) crow[c + 1] = v1; }
@@ -455,13 +461,13 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
             const int64_t c = col0 + ni * 8 + 2 * t;
             if (c > cmax) continue;
             const bool both = (c + 1 <= cmax);
-            double v0 = k.alpha * acc[mi][ni][0], v1 = k.alpha * acc[mi][ni][1];
+            double v0 = scaled(k.alpha, acc[mi][ni][0]), v1 = scaled(k.alpha, acc[mi][ni][1]);
             if (use_beta) {
                 double2 o = make_double2(0.0, 0.0);
                 if (old_tile) o = *reinterpret_cast<const double2*>(old_tile + (mi * 8 + gq) * (kTile * 8) + (ni * 8 + 2 * t) * 8);
                 else if (both && k.vec_ok) o = *reinterpret_cast<const double2*>(crow + c);
                 else { o.x = crow[c]; if (both) o.y = crow[c + 1]; }
-                v0 += k.beta * o.x; v1 += k.beta * o.y;
+                v0 = plus_old(v0, k.beta, o.x); v1 = plus_old(v1, k.beta, o.y);
             }
             if (both) {
                 if (k.vec_ok) *reinterpret_cast<double2*>(crow + c) = make_double2(v0, v1);
@@ -542,12 +548,12 @@ __device__ __forceinline__ bool syr2k_tile_role(const Call& k, const WorkItem& i
             const int64_t c = col0 + ni * 8 + 2 * t;
             if (c > r) continue;
             const bool both = (c + 1 <= r);
-            double v0 = k.alpha * acc[mi][ni][0], v1 = k.alpha * acc[mi][ni][1];
+            double v0 = scaled(k.alpha, acc[mi][ni][0]), v1 = scaled(k.alpha, acc[mi][ni][1]);
             if (use_beta) {
                 double2 o = make_double2(0.0, 0.0);
                 if (old_tile) o = *reinterpret_cast<const double2*>(old_tile + rr * (kTile * 8) + (ni * 8 + 2 * t) * 8);
                 else { o.x = crow[c]; if (both) o.y = crow[c + 1]; }
-                v0 += k.beta * o.x; v1 += k.beta * o.y;
+                v0 = plus_old(v0, k.beta, o.x); v1 = plus_old(v1, k.beta, o.y);
             }
             if (both && k.vec_ok) *reinterpret_cast<double2*>(crow + c) = make_double2(v0, v1);
             else { crow[c] = v0; if (both) crow[c + 1] = v1; }
@@ -623,14 +629,14 @@ __device__ __forceinline__ bool herk_tile_role(const Call& k, const WorkItem& it
             const int64_t c = col0 + ni * 8 + 2 * t;
             if (c > r) continue;
             const bool both = (c + 1 <= r);
-            double2 v0 = make_double2(k.alpha * re[mi][ni][0], k.alpha * im[mi][ni][0]);
-            double2 v1 = make_double2(k.alpha * re[mi][ni][1], k.alpha * im[mi][ni][1]);
+            double2 v0 = make_double2(scaled(k.alpha, re[mi][ni][0]), scaled(k.alpha, im[mi][ni][0]));
+            double2 v1 = make_double2(scaled(k.alpha, re[mi][ni][1]), scaled(k.alpha, im[mi][ni][1]));
             if (use_beta) {
                 const double2 o0 = *reinterpret_cast<const double2*>(crow + 2 * c);
-                v0.x += k.beta * o0.x; v0.y += k.beta * o0.y;
+                v0.x = plus_old(v0.x, k.beta, o0.x); v0.y = plus_old(v0.y, k.beta, o0.y);
                 if (both) {
                     const double2 o1 = *reinterpret_cast<const double2*>(crow + 2 * c + 2);
-                    v1.x += k.beta * o1.x; v1.y += k.beta * o1.y;
+                    v1.x = plus_old(v1.x, k.beta, o1.x); v1.y = plus_old(v1.y, k.beta, o1.y);
                 }
             }
             if (c == r) v0.y = 0.0;
@@ -833,7 +839,7 @@ __device__ __forceinline__ bool mma_warp_item_p(const Call& k, const Image& im, 
         if (!wait_image_empty(k, im, item_no, lane)) return false;
 #pragma unroll
         for (int q = 0; q < 15; ++q)                    // block (3, 3) of tile q
-            sts_f64x2(im.base32 + q * kCTileBytes + image_offset(24 + gq, 12 + t), k.alpha * sacc[q][0], k.alpha * sacc[q][1]);
+            sts_f64x2(im.base32 + q * kCTileBytes + image_offset(24 + gq, 12 + t), scaled(k.alpha, sacc[q][0]), scaled(k.alpha, sacc[q][1]));
     } else if (warp < n_tile) {
         const uint32_t xbase = uint32_t(it.tile_x[warp]) * kSegBytes, ybase = uint32_t(it.tile_y[warp]) * kSegBytes;
         double acc[4][4][2];
@@ -851,7 +857,7 @@ __device__ __forceinline__ bool mma_warp_item_p(const Call& k, const Image& im, 
 #pragma unroll
             for (int ni = 0; ni < 4; ++ni) {
                 if (scavenge && mi == 3 && ni == 3) continue;         // written by the 16th warp
-                sts_f64x2(tile32 + image_offset(mi * 8 + gq, ni * 4 + t), k.alpha * acc[mi][ni][0], k.alpha * acc[mi][ni][1]);
+                sts_f64x2(tile32 + image_offset(mi * 8 + gq, ni * 4 + t), scaled(k.alpha, acc[mi][ni][0]), scaled(k.alpha, acc[mi][ni][1]));
             }
     } else {
         uint32_t st = g0 % kPStages, parity = (g0 / kPStages) & 1;    // no tile in this item: keep the ring moving
@@ -900,8 +906,8 @@ __device__ __forceinline__ void write_out_item(const Call& k, const Image& im, c
                     red_add_f64(p, v[i].x);
                     if (both) red_add_f64(p + 1, v[i].y);
                 } else {
-                    p[0] = v[i].x + k.beta * p[0];
-                    if (both) p[1] = v[i].y + k.beta * p[1];
+                    p[0] = plus_old(v[i].x, k.beta, p[0]);
+                    if (both) p[1] = plus_old(v[i].y, k.beta, p[1]);
                 }
             }
         }
@@ -1017,7 +1023,7 @@ splitk_reduce_f64_kernel(int64_t N, int32_t slices, const double* __restrict__ p
     double s = 0.0;
     for (int32_t sl = 0; sl < slices; ++sl) s += partial[(int64_t(sl) * N + i) * N + j];
     double* c = C + i * ldc + j;
-    *c = (beta == 0.0) ? alpha * s : alpha * s + beta * *c;
+    *c = (beta == 0.0) ? scaled(alpha, s) : plus_old(scaled(alpha, s), beta, *c);
 }
 
 // Tail K-split: for tail item i (list entry tail_first + i) and each of its tiles, the stored triangle of C
@@ -1038,7 +1044,7 @@ tail_reduce_f64_kernel(const WorkItem* __restrict__ items, int32_t tail_first, i
         double s = 0.0;
         for (int32_t sl = 0; sl < slices; ++sl) s += src[int64_t(sl) * kPartUnitElems + e];
         double* dst = C + r * ldc + c;
-        *dst = (beta == 0.0) ? alpha * s : alpha * s + beta * *dst;
+        *dst = (beta == 0.0) ? scaled(alpha, s) : plus_old(scaled(alpha, s), beta, *dst);
     }
 }
 

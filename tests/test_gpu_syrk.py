@@ -217,11 +217,13 @@ def test_two_streams_back_to_back():
 
 # ---- FP64 launch forms: one block per item / persistent blocks drawing items from a counter ----
 
-@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-1.0, 1.0)])
+@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-1.0, 1.0), (2.5, -0.5)])
 def test_f64_launch_forms_agree_bit_for_bit(alpha, beta):
     """Both forms run every tile with the same arithmetic in the same order: identical bits,
     and both within tolerance of the reference.  Sizes span one item, a ragged edge, and a list
-    several times longer than the SM count."""
+    several times longer than the SM count.  The persistent form writes C from separate warps: stores for
+    beta = 0, one memory-side addition per entry for beta = 1 (the correctly rounded sum, as the other form's
+    multiply-add gives), a multiply-add for any other beta."""
     for n, (N, M) in enumerate([(33, 50), (1000, 70), (1300, 40), (2500, 33), (5000, 48)]):
         A = make_A(N, M, B.DTYPE_F64, seed=300 + n)
         Cin = I.random_c(N, 7, B.DTYPE_F64) if beta != 0.0 else None
@@ -236,6 +238,28 @@ def test_f64_launch_forms_agree_bit_for_bit(alpha, beta):
             outs.append(got)
         il = np.tril_indices(N)
         assert np.array_equal(outs[0][il], outs[1][il]) and np.array_equal(outs[0][il], outs[2][il])
+
+
+@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-1.0, 1.0), (0.5, 3.0)])
+@pytest.mark.parametrize("ldc_pad,c_offset", [(3, 0), (0, 1), (5, 1)])
+def test_f64_persistent_write_out_with_odd_pitch_or_offset_of_c(alpha, beta, ldc_pad, c_offset):
+    """C off the 16-byte boundary or with an odd pitch: the write-out warps fall back to 8-byte accesses; same
+    bits as the one-block-per-item form, canaries around C untouched (run_case checks them)."""
+    N, M = 1400, 72
+    A = make_A(N, M, B.DTYPE_F64, seed=340)
+    Cin = I.random_c(N, 341, B.DTYPE_F64) if beta != 0.0 else None
+    outs = []
+    for mode in (B.F64_LAUNCH_PER_ITEM, B.F64_LAUNCH_PERSISTENT):
+        try:
+            B.syrk_set_f64_launch(mode)
+            got, ref, bound = run_case(A, B.DTYPE_F64, alpha, beta, Cin, ldc=N + ldc_pad, c_offset=c_offset,
+                                       poison=(beta == 0.0))
+        finally:
+            B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+        assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin, B.DTYPE_F64)
+        outs.append(got)
+    il = np.tril_indices(N)
+    assert np.array_equal(outs[0][il], outs[1][il])
 
 
 def test_f64_persistent_form_repeated_and_on_two_streams():
