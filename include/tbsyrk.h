@@ -500,7 +500,8 @@ typedef struct {
     int64_t a_loads;         /* elements of A loaded (two-level model)               */
     int64_t c_elems;         /* elements of C owned: N(N+1)/2                        */
     int64_t s_acc;           /* accumulator elements a thread block may hold         */
-    int64_t s_total;         /* s_acc + staging elements (all pipeline stages)       */
+    int64_t s_total;         /* s_acc + staging elements (all pipeline stages; for the
+                                persistent FP64 form also the accumulators' image)   */
     int32_t effective_schedule; /* what the call runs: syrk_effective_schedule()      */
     int32_t launches;        /* kernels the call enqueues: 1, or 2 with a K-split of the whole
                                 list or of its tail (the slices' partial results are summed

@@ -1046,6 +1046,7 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->effective_schedule = effective_schedule_of(N, M, dtype, 148, &split);
     out->split_k = split;
     out->launches = split > 1 ? 2 : 1;
+    bool f64_persistent = false;
     if (dtype == SYRK_DTYPE_F64 && split == 1 && out->effective_schedule != SYRK_SCHEDULE_PAIR_SQUARE) {
         // the tail K-split of the one-block-per-item form adds its reduction kernel (the launch form is taken as
         // for beta == 0 or 1; the automatic settings are assumed)
@@ -1056,6 +1057,7 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
                               (mode == SYRK_F64_LAUNCH_AUTO && !f64_persistent_pays(M, n_items, 0.0, 148));
         if (per_item && tail_setting == 0 && plan_tail_split_f64(plan.items, (M + ks.bk - 1) / ks.bk, 148).slices > 1)
             out->launches = 2;
+        f64_persistent = !per_item;
     }
     out->n_tiles = plan.p.n_tiles;
     out->items = int64_t(plan.items.size());
@@ -1069,6 +1071,8 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->s_acc = ks.s_acc;
     out->s_total = ks.s_acc + int64_t(kMaxSeg) * ks.tile * ks.bk * ks.stages;
     if (is_tcgen05_dtype(dtype)) out->s_total = ks.s_acc + int64_t(bf16_seg_slots()) * ks.tile * ks.bk * ks.stages;
+    // the persistent FP64 form: the accumulators, their shared-memory image, and its shorter ring of stages
+    if (f64_persistent) out->s_total = 2 * ks.s_acc + int64_t(kMaxSeg) * ks.tile * ks.bk * f64_persistent_stages();
     return SYRK_OK;
 }
 

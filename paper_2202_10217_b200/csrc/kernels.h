@@ -53,6 +53,7 @@ cudaError_t launch_gemm_nt_f64(const CUtensorMap& tmP, const CUtensorMap& tmQ, c
 int f64_tile();
 int f64_bk();
 int f64_stages();
+int f64_persistent_stages();    // ring depth of the persistent launch form
 
 // BF16 -> FP32 triangle-block kernel (tcgen05 / TMEM): persistent, one thread block per SM.
 // `split_k` > 1 makes every item run once per K-slice, partial tiles going to `d_partial`

@@ -1205,5 +1205,6 @@ int64_t f64_tail_partial_elems(int64_t n_tail_items, int tail_slices) {
 int f64_tile() { return f64::kTile; }
 int f64_bk() { return f64::kBK; }
 int f64_stages() { return f64::kStages; }
+int f64_persistent_stages() { return f64::kPStages; }
 
 }  // namespace tbsyrk
