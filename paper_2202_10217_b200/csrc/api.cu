@@ -164,7 +164,7 @@ int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkIt
         // Persistent blocks hide each item's start-up and write-out behind the next item's M loop
         // (see f64_persistent_pays for when that is the faster form).
         const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
-        const bool persistent = !upper && tail_slices <= 1 && (mode == SYRK_F64_LAUNCH_PERSISTENT ||
+        const bool persistent = tail_slices <= 1 && (mode == SYRK_F64_LAUNCH_PERSISTENT ||
                                 (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(M, n_items, beta, ds->sm_count)));
         int* tickets = (persistent && split <= 1) ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<double*>(C), ldc,
@@ -356,7 +356,7 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         // Otherwise, in the one-block-per-item form: the last round's items in slices (tail K-split).
         const int64_t n_items = int64_t(dp->plan.items.size());
         const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
-        const bool per_item = upper || mode == SYRK_F64_LAUNCH_PER_ITEM ||
+        const bool per_item = mode == SYRK_F64_LAUNCH_PER_ITEM ||
                               (mode == SYRK_F64_LAUNCH_AUTO && !f64_persistent_pays(M, n_items, beta, ds->sm_count));
         if (split == 1 && per_item && !upper && runtime().f64_tail_slices != 1) {
             TailSplit ts{n_items, 1};
@@ -426,6 +426,33 @@ __global__ void unpack_lower_axpby_kernel(int64_t first, int64_t count, const T*
     }
 }
 
+// Work list of Algorithm 4 for the kernels' forms in which two warps share a tile (rank-2k and Hermitian
+// updates): triangle blocks with k = 4 (6 tiles; for the rank-2k update a stage holds the four segments of A
+// and the same rows of B), 2 x 2 rectangles, diagonal blocks of two rows.  Cached per device.
+int get_two_warp_plan(DeviceState* ds, int64_t N, DevicePlan** out) {
+    const int64_t n_tiles = (N + f64_tile() - 1) / f64_tile();
+    const auto key = std::make_tuple(n_tiles, 64, runtime().schedule);       // 64: this list
+    auto it = ds->plans.find(key);
+    if (it == ds->plans.end()) {
+        DevicePlan dp;
+        PlanParams p;
+        p.n_tiles = n_tiles; p.k = 4; p.rect_rows = 2; p.rect_cols = 2; p.diag_side = 2; p.schedule = runtime().schedule;
+        if (!build_plan(p, &dp.plan)) return SYRK_ERR_PLAN;
+        std::stable_sort(dp.plan.items.begin(), dp.plan.items.end(),
+                         [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
+        const size_t n = dp.plan.items.size();
+        if (n > 0) {
+            if (cudaMalloc(&dp.d_items, n * sizeof(WorkItem)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
+            if (cudaMemcpy(dp.d_items, dp.plan.items.data(), n * sizeof(WorkItem), cudaMemcpyHostToDevice) != cudaSuccess) {
+                cudaGetLastError(); cudaFree(dp.d_items); return SYRK_ERR_CUDA;
+            }
+        }
+        it = ds->plans.emplace(key, std::move(dp)).first;
+    }
+    *out = &it->second;
+    return SYRK_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -488,33 +515,6 @@ int syrk_ex(int uplo, int trans, int64_t N, int64_t M, const void* A, int64_t ld
     std::lock_guard<std::mutex> lock(runtime().mu);
     return syrk_run_device(N, M, A, lda, C, ldc, alpha, beta, dtype, static_cast<cudaStream_t>(stream), -1,
                            trans == SYRK_OP_T ? 1 : 0, uplo == SYRK_UPLO_UPPER ? 1 : 0);
-}
-
-// Work list of Algorithm 4 for the kernels' forms in which two warps share a tile (rank-2k and Hermitian
-// updates): triangle blocks with k = 4 (6 tiles; for the rank-2k update a stage holds the four segments of A
-// and the same rows of B), 2 x 2 rectangles, diagonal blocks of two rows.  Cached per device.
-static int get_two_warp_plan(DeviceState* ds, int64_t N, DevicePlan** out) {
-    const int64_t n_tiles = (N + f64_tile() - 1) / f64_tile();
-    const auto key = std::make_tuple(n_tiles, 64, runtime().schedule);       // 64: this list
-    auto it = ds->plans.find(key);
-    if (it == ds->plans.end()) {
-        DevicePlan dp;
-        PlanParams p;
-        p.n_tiles = n_tiles; p.k = 4; p.rect_rows = 2; p.rect_cols = 2; p.diag_side = 2; p.schedule = runtime().schedule;
-        if (!build_plan(p, &dp.plan)) return SYRK_ERR_PLAN;
-        std::stable_sort(dp.plan.items.begin(), dp.plan.items.end(),
-                         [](const WorkItem& a, const WorkItem& b) { return a.n_tile > b.n_tile; });
-        const size_t n = dp.plan.items.size();
-        if (n > 0) {
-            if (cudaMalloc(&dp.d_items, n * sizeof(WorkItem)) != cudaSuccess) { cudaGetLastError(); return SYRK_ERR_ALLOC; }
-            if (cudaMemcpy(dp.d_items, dp.plan.items.data(), n * sizeof(WorkItem), cudaMemcpyHostToDevice) != cudaSuccess) {
-                cudaGetLastError(); cudaFree(dp.d_items); return SYRK_ERR_CUDA;
-            }
-        }
-        it = ds->plans.emplace(key, std::move(dp)).first;
-    }
-    *out = &it->second;
-    return SYRK_OK;
 }
 
 int syr2k_lower(int64_t N, int64_t M, const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc,

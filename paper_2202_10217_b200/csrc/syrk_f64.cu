@@ -291,8 +291,9 @@ __device__ __forceinline__ uint32_t fragment_offset_tn(int lane) {
 }
 
 // The M loop of the 16th warp of a triangle block: block q = (x, y), y < x, of the 15 left-out 8 x 8 blocks
-// is the product of rows 24..31 of segments x and y.
-template <bool kTN, int kSt = kStages>
+// is the product of rows 24..31 of segments x and y (kSwap: of y and x, the block as the tile stored above
+// the diagonal holds it).
+template <bool kTN, int kSt = kStages, bool kSwap = false>
 __device__ __forceinline__ bool scavenger_mainloop(double (&sacc)[15][2], const Call& k, uint32_t off0, uint32_t g0, int lane) {
 #pragma unroll
     for (int q = 0; q < 15; ++q) sacc[q][0] = sacc[q][1] = 0.0;
@@ -309,7 +310,7 @@ __device__ __forceinline__ bool scavenger_mainloop(double (&sacc)[15][2], const 
 #pragma unroll
             for (int x = 1; x < 6; ++x)
 #pragma unroll
-                for (int y = 0; y < x; ++y, ++q) dmma884(sacc[q], f[x], f[y]);
+                for (int y = 0; y < x; ++y, ++q) dmma884(sacc[q], kSwap ? f[y] : f[x], kSwap ? f[x] : f[y]);
         }
         release_at(k, st, lane);
         if (++st == kSt) { st = 0; parity ^= 1; }
@@ -824,7 +825,7 @@ __device__ __forceinline__ bool wait_image_empty(const Call& k, const Image& im,
 }
 
 // One MMA warp's share of item number item_no of its block: the M loop, then its accumulators into the image.
-template <bool kTN>
+template <bool kTN, bool kUpper>
 __device__ __forceinline__ bool mma_warp_item_p(const Call& k, const Image& im, const WorkItem& it, uint32_t& g,
                                                 uint32_t item_no, int warp, int lane) {
     const int gq = lane >> 2, t = lane & 3;
@@ -835,7 +836,7 @@ __device__ __forceinline__ bool mma_warp_item_p(const Call& k, const Image& im, 
     const uint32_t off0 = kTN ? fragment_offset_tn(lane) : fragment_offset(lane);
     if (scavenge && warp == kMmaWarps - 1) {
         double sacc[15][2];
-        if (!scavenger_mainloop<kTN, kPStages>(sacc, k, off0, g0, lane)) return false;
+        if (!scavenger_mainloop<kTN, kPStages, kUpper>(sacc, k, off0, g0, lane)) return false;
         if (!wait_image_empty(k, im, item_no, lane)) return false;
 #pragma unroll
         for (int q = 0; q < 15; ++q)                    // block (3, 3) of tile q
@@ -882,6 +883,7 @@ __device__ __forceinline__ bool mma_warp_item_p(const Call& k, const Image& im, 
 __device__ __forceinline__ void red_add_f64(double* p, double v) {
     asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p), "d"(v) : "memory");
 }
+template <bool kUpper>
 __device__ __forceinline__ void write_out_item(const Call& k, const Image& im, const WorkItem& it, int out_warp, int lane) {
     const int mode = (k.beta == 0.0) ? 0 : (k.beta == 1.0 ? 1 : 2);
     const int half = lane >> 4, c16 = lane & 15;
@@ -896,25 +898,28 @@ __device__ __forceinline__ void write_out_item(const Call& k, const Image& im, c
             for (int i = 0; i < kOutBatch; ++i) {
                 const int r = 2 * (i0 + i) + half;
                 const int64_t R = row0 + r, c = col0 + 2 * (c16 ^ ((r & 1) << 2));
-                if (R >= k.N || c > R) continue;                       // beyond the last row, or above the diagonal
+                if (R >= k.N) continue;                                // beyond the last row
+                // the entries of the pair (c, c + 1) that lie in the stored triangle
+                const bool ok0 = kUpper ? (c >= R && c < k.N) : (c <= R);
+                const bool ok1 = kUpper ? (c + 1 >= R && c + 1 < k.N) : (c + 1 <= R);
+                if (!ok0 && !ok1) continue;
                 double* p = k.C + R * k.ldc + c;
-                const bool both = (c + 1 <= R);
                 if (mode == 0) {
-                    if (both && (k.vec_ok & 1)) *reinterpret_cast<double2*>(p) = v[i];
-                    else { p[0] = v[i].x; if (both) p[1] = v[i].y; }
+                    if (ok0 && ok1 && (k.vec_ok & 1)) *reinterpret_cast<double2*>(p) = v[i];
+                    else { if (ok0) p[0] = v[i].x; if (ok1) p[1] = v[i].y; }
                 } else if (mode == 1) {
-                    red_add_f64(p, v[i].x);
-                    if (both) red_add_f64(p + 1, v[i].y);
+                    if (ok0) red_add_f64(p, v[i].x);
+                    if (ok1) red_add_f64(p + 1, v[i].y);
                 } else {
-                    p[0] = plus_old(v[i].x, k.beta, p[0]);
-                    if (both) p[1] = plus_old(v[i].y, k.beta, p[1]);
+                    if (ok0) p[0] = plus_old(v[i].x, k.beta, p[0]);
+                    if (ok1) p[1] = plus_old(v[i].y, k.beta, p[1]);
                 }
             }
         }
     }
 }
 
-template <bool kTN>
+template <bool kTN, bool kUpper>
 __global__ void __launch_bounds__(kPThreads, 1)
 syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __restrict__ items,
                                int64_t n_items, int* __restrict__ counter, int64_t N, int32_t n_ksteps,
@@ -964,7 +969,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const Wo
                 if (!last) {
                     for (int w = 0; w < int(sizeof(WorkItem) / 4); ++w)
                         reinterpret_cast<int32_t*>(&dst)[w] = reinterpret_cast<const int32_t*>(&items[idx])[w];
-                    if (!prepare_item(k, dst)) { s_abort = 1; atomicOr(status, kStatusBadItem); last = true; }
+                    if (!prepare_item(k, dst, kUpper)) { s_abort = 1; atomicOr(status, kStatusBadItem); last = true; }
                 }
                 if (last) dst.n_tile = -1;                        // end marker
                 mbar_arrive(&s_item_bar[slot % kItemRing]);       // publishes the slot (release)
@@ -997,7 +1002,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const Wo
                 if (s_abort == 0) { s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); }
                 return;
             }
-            write_out_item(k, im, it, out_warp, lane);
+            write_out_item<kUpper>(k, im, it, out_warp, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(&image_bar[1]);
         }
@@ -1008,7 +1013,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const Wo
         }
         const WorkItem& it = s_ring[slot % kItemRing];
         if (it.n_tile < 0) return;
-        if (!mma_warp_item_p<kTN>(k, im, it, g, slot, warp - kOutWarps - 1, lane)) return;
+        if (!mma_warp_item_p<kTN, kUpper>(k, im, it, g, slot, warp - kOutWarps - 1, lane)) return;
     }
 }
 
@@ -1060,16 +1065,18 @@ cudaError_t configure_f64_kernels() {
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[8] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
+        const void* kernels[10] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, true>),
-                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false>),
-                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true>)};
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, false>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, true>)};
         for (const void* fn : kernels) {
-            const bool persistent = fn == kernels[6] || fn == kernels[7];
+            const bool persistent = fn == kernels[6] || fn == kernels[7] || fn == kernels[8] || fn == kernels[9];
             cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  persistent ? f64::kPSmemBytes : f64::kSmemBytes);
             if (e != cudaSuccess) return e;
@@ -1122,9 +1129,10 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
             n_items, c_batch_stride, 0, 0, 1, nullptr);
         return cudaGetLastError();
     }
-    if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30) && !upper) {
+    if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
-        auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true> : f64::syrk_f64_tbs_persistent_kernel<false>;
+        auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, true> : f64::syrk_f64_tbs_persistent_kernel<false, true>)
+                            : (a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false> : f64::syrk_f64_tbs_persistent_kernel<false, false>);
         kernel<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, d_items, n_items, d_tickets, N, n_ksteps, C, ldc,
                                                                          alpha, beta, vec_ok, d_status);
         return cudaGetLastError();

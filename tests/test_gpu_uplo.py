@@ -110,3 +110,27 @@ def test_lower_form_of_syrk_ex_is_syrk_lower_and_bad_flags_are_refused():
         with pytest.raises(B.SyrkError) as e:
             B.syrk_ex(uplo, trans, N, M, A, M, C2, N, 1.0, 0.0, B.DTYPE_F64)
         assert e.value.code == -2
+
+
+@TN
+@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-1.0, 1.0), (2.5, -0.5)])
+def test_f64_launch_forms_agree_bit_for_bit_on_the_upper_triangle(tn, alpha, beta):
+    """The persistent FP64 form (write-out by separate warps) with the upper triangle stored: same bits as the
+    one-block-per-item form, within tolerance of the reference, ragged last tile row and column, odd pitch of C."""
+    for n, (N, M, pad) in enumerate([(1304, 40, 0), (2500, 33, 3), (5008, 48, 0)]):
+        if tn and N % 2:
+            continue
+        A = make_A(N, M, B.DTYPE_F64, seed=4500 + n)
+        Cin = I.random_c(N, 4501, B.DTYPE_F64) if beta != 0.0 else None
+        outs = []
+        for mode in (B.F64_LAUNCH_PER_ITEM, B.F64_LAUNCH_PERSISTENT):
+            try:
+                B.syrk_set_f64_launch(mode)
+                got, ref, bound = run_case(A, B.DTYPE_F64, alpha, beta, Cin, ldc=N + pad, tn=tn, upper=True,
+                                           poison=(beta == 0.0))
+            finally:
+                B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+            assert_within_tolerance(got, ref, bound, M, alpha, beta, Cin, B.DTYPE_F64)
+            outs.append(got)
+        il = np.tril_indices(N)
+        assert np.array_equal(outs[0][il], outs[1][il])
