@@ -426,6 +426,14 @@ __global__ void unpack_lower_axpby_kernel(int64_t first, int64_t count, const T*
     }
 }
 
+// The launch form of the rank-2k and Hermitian updates (inner dimension in binary64 columns of a stage row):
+// as set by syrk_set_f64_launch, the automatic rule being that of the rank-k update.
+bool two_warp_form_is_persistent(int64_t columns, int64_t n_items, double beta, int sm_count) {
+    const int mode = runtime().f64_launch;
+    return mode == SYRK_F64_LAUNCH_PERSISTENT ||
+           (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(columns, n_items, beta, sm_count));
+}
+
 // Work list of Algorithm 4 for the kernels' forms in which two warps share a tile (rank-2k and Hermitian
 // updates): triangle blocks with k = 4 (6 tiles; for the rank-2k update a stage holds the four segments of A
 // and the same rows of B), 2 x 2 rectangles, diagonal blocks of two rows.  Cached per device.
@@ -542,8 +550,10 @@ int syr2k_lower(int64_t N, int64_t M, const void* A, int64_t lda, const void* B,
     if ((rc = encode_tensor_map_2d(&tb, SYRK_DTYPE_F64, B, N, M, ldb, f64_tile(), f64_bk())) != SYRK_OK) return rc;
     const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
                        encode_tensor_map_c_f64(&tmc, C, N, ldc, f64_tile()) == SYRK_OK;
-    return launch_syr2k_f64(ta, tb, c_tma ? &tmc : nullptr, dp->d_items, int64_t(dp->plan.items.size()), N, M,
-                            static_cast<double*>(C), ldc, alpha, beta, status_for_stream(ds, st), st) == cudaSuccess
+    const int64_t n_items = int64_t(dp->plan.items.size());
+    int* tickets = two_warp_form_is_persistent(M, n_items, beta, ds->sm_count) ? tickets_for_stream(ds, st) : nullptr;
+    return launch_syr2k_f64(ta, tb, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha,
+                            beta, status_for_stream(ds, st), st, tickets, ds->sm_count) == cudaSuccess
                ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
@@ -567,8 +577,10 @@ int herk_lower(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_
     if ((rc = get_two_warp_plan(ds, N, &dp)) != SYRK_OK) return rc;
     CUtensorMap ta;          // the real view of A: N rows of 2M values, pitch 2 lda
     if ((rc = encode_tensor_map_2d(&ta, SYRK_DTYPE_F64, A, N, 2 * M, 2 * lda, f64_tile(), f64_bk())) != SYRK_OK) return rc;
-    return launch_herk_f64(ta, dp->d_items, int64_t(dp->plan.items.size()), N, M, static_cast<double*>(C), ldc, alpha, beta,
-                           status_for_stream(ds, st), st) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
+    const int64_t n_items = int64_t(dp->plan.items.size());
+    int* tickets = two_warp_form_is_persistent(2 * M, n_items, beta, ds->sm_count) ? tickets_for_stream(ds, st) : nullptr;
+    return launch_herk_f64(ta, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha, beta, status_for_stream(ds, st),
+                           st, tickets, ds->sm_count) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
 
 int syr2k_lower_ex(int64_t N, int64_t M, const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc,

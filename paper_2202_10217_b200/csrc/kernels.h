@@ -34,16 +34,20 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
 int64_t f64_tail_partial_elems(int64_t n_tail_items, int tail_slices);
 // Rank-2k update C = alpha (A B^T + B A^T) + beta C on the lower triangle with the same kernel: the work
 // items name at most 4 segments and 8 tiles; every stage holds the segments' rows of A (tmA) and of
-// B (tmB); a tile is shared by two warps (16 rows each) that add both products.  One block per item.
+// B (tmB); a tile is shared by two warps (16 rows each) that add both products.  One block per item, or, with
+// `d_tickets` (as for launch_syrk_f64), `n_blocks` persistent blocks whose write-out warps store C.
 cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap* tmC,
                              const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc,
-                             double alpha, double beta, int* d_status, cudaStream_t stream);
+                             double alpha, double beta, int* d_status, cudaStream_t stream, int* d_tickets = nullptr,
+                             int n_blocks = 0);
 // Hermitian rank-k update C = alpha A A^H + beta C on the lower triangle with the same kernel: `tmA` covers
 // the real view of the complex operand (N rows of 2M binary64 values, re and im interleaved), C and ldc
 // address complex entries (C 16-byte aligned); work items as for the rank-2k update (at most 8 tiles, a
-// tile shared by two warps, each with a real and an imaginary accumulator).  One block per item.
+// tile shared by two warps, each with a real and an imaginary accumulator).  One block per item, or persistent
+// blocks when `d_tickets` is given.
 cudaError_t launch_herk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M,
-                            double* C, int64_t ldc, double alpha, double beta, int* d_status, cudaStream_t stream);
+                            double* C, int64_t ldc, double alpha, double beta, int* d_status, cudaStream_t stream,
+                            int* d_tickets = nullptr, int n_blocks = 0);
 // The same kernel in two-operand mode: D (nrows x ncols, pitch ldd) = alpha * P * Q^T + beta * D with
 // P nrows x K and Q ncols x K, both row-major through their tensor maps (boxes of 32 rows x 16
 // columns, 128-byte swizzle); `tmD` (may be null) as `tmC` above.  Requires K > 0.

@@ -485,24 +485,16 @@ __device__ __forceinline__ bool tile_role(const Call& k, const WorkItem& it, uin
 // Rank-2k update: warp w owns rows 16 (w & 1) .. + 15 of tile w >> 1 and adds both products,
 // A_x B_y^T and B_x A_y^T, into the same 16 x 32 accumulator (2 x 4 blocks of m8n8k4): 16 DMMAs per
 // k-slice and warp, as for a whole tile of the rank-k update.  N x M operands, lower triangle.
-__device__ __forceinline__ bool syr2k_tile_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, int warp, int lane) {
-    const int gq = lane >> 2, t = lane & 3;
-    const int tile = warp >> 1, half = warp & 1;
-    const uint32_t gc = g0 + uint32_t(k.n_ksteps);
-    const bool use_beta = (k.beta != 0.0);
-    const uint32_t off0 = fragment_offset(lane);
-    const int sx = it.tile_x[tile], sy = it.tile_y[tile];
-    const int64_t row0 = int64_t(it.seg[sx]) * kTile, col0 = int64_t(it.seg[sy]) * kTile;
+template <int kSt = kStages>
+__device__ __forceinline__ bool syr2k_mainloop(double (&acc)[2][4][2], const Call& k, int sx, int sy, int half,
+                                               uint32_t off0, uint32_t g0, int lane) {
     const uint32_t xa = uint32_t(sx) * kSegBytes, ya = uint32_t(sy) * kSegBytes;
     const uint32_t xb = uint32_t(kSyr2kSlots + sx) * kSegBytes, yb = uint32_t(kSyr2kSlots + sy) * kSegBytes;
-
-    double acc[2][4][2];
 #pragma unroll
     for (int mi = 0; mi < 2; ++mi)
 #pragma unroll
         for (int ni = 0; ni < 4; ++ni) acc[mi][ni][0] = acc[mi][ni][1] = 0.0;
-
-    uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;
+    uint32_t st = g0 % kSt, parity = (g0 / kSt) & 1;
     for (int ks = 0; ks < k.n_ksteps; ++ks) {
         if (!wait_full_at(k, st, parity, lane)) return false;
         const uint32_t stage = k.smem32 + st * kStageBytes;
@@ -530,8 +522,21 @@ __device__ __forceinline__ bool syr2k_tile_role(const Call& k, const WorkItem& i
                 }
         }
         release_at(k, st, lane);
-        if (++st == kStages) { st = 0; parity ^= 1; }
+        if (++st == kSt) { st = 0; parity ^= 1; }
     }
+    return true;
+}
+
+__device__ __forceinline__ bool syr2k_tile_role(const Call& k, const WorkItem& it, uint32_t g0, int n_c, int warp, int lane) {
+    const int gq = lane >> 2, t = lane & 3;
+    const int tile = warp >> 1, half = warp & 1;
+    const uint32_t gc = g0 + uint32_t(k.n_ksteps);
+    const bool use_beta = (k.beta != 0.0);
+    const int sx = it.tile_x[tile], sy = it.tile_y[tile];
+    const int64_t row0 = int64_t(it.seg[sx]) * kTile, col0 = int64_t(it.seg[sy]) * kTile;
+
+    double acc[2][4][2];
+    if (!syr2k_mainloop(acc, k, sx, sy, half, fragment_offset(lane), g0, lane)) return false;
 
     for (int j = 0; j < n_c; ++j)
         if (!wait_full(k, gc + j, lane)) return false;
@@ -576,23 +581,17 @@ __device__ __forceinline__ bool syr2k_tile_role(const Call& k, const WorkItem& i
 __device__ __forceinline__ double flip_sign(double v, uint32_t mask) {
     return __hiloint2double(__double2hiint(v) ^ int(mask), __double2loint(v));
 }
-__device__ __forceinline__ bool herk_tile_role(const Call& k, const WorkItem& it, uint32_t g0, int warp, int lane) {
-    const int gq = lane >> 2, t = lane & 3;
-    const int tile = warp >> 1, half = warp & 1;
-    const bool use_beta = (k.beta != 0.0);
+template <int kSt = kStages>
+__device__ __forceinline__ bool herk_mainloop(double (&re)[2][4][2], double (&im)[2][4][2], const Call& k, int sx, int sy,
+                                              int half, uint32_t g0, int lane) {
     const uint32_t off0 = fragment_offset(lane);
-    const uint32_t flip = (t & 1) ? 0u : 0x80000000u;
-    const int sx = it.tile_x[tile], sy = it.tile_y[tile];
-    const int64_t row0 = int64_t(it.seg[sx]) * kTile, col0 = int64_t(it.seg[sy]) * kTile;
+    const uint32_t flip = (lane & 1) ? 0u : 0x80000000u;
     const uint32_t xa = uint32_t(sx) * kSegBytes, ya = uint32_t(sy) * kSegBytes;
-
-    double re[2][4][2], im[2][4][2];
 #pragma unroll
     for (int mi = 0; mi < 2; ++mi)
 #pragma unroll
         for (int ni = 0; ni < 4; ++ni) re[mi][ni][0] = re[mi][ni][1] = im[mi][ni][0] = im[mi][ni][1] = 0.0;
-
-    uint32_t st = g0 % kStages, parity = (g0 / kStages) & 1;
+    uint32_t st = g0 % kSt, parity = (g0 / kSt) & 1;
     for (int ks = 0; ks < k.n_ksteps; ++ks) {
         if (!wait_full_at(k, st, parity, lane)) return false;
         const uint32_t stage = k.smem32 + st * kStageBytes;
@@ -617,8 +616,20 @@ __device__ __forceinline__ bool herk_tile_role(const Call& k, const WorkItem& it
                 }
         }
         release_at(k, st, lane);
-        if (++st == kStages) { st = 0; parity ^= 1; }
+        if (++st == kSt) { st = 0; parity ^= 1; }
     }
+    return true;
+}
+
+__device__ __forceinline__ bool herk_tile_role(const Call& k, const WorkItem& it, uint32_t g0, int warp, int lane) {
+    const int gq = lane >> 2, t = lane & 3;
+    const int tile = warp >> 1, half = warp & 1;
+    const bool use_beta = (k.beta != 0.0);
+    const int sx = it.tile_x[tile], sy = it.tile_y[tile];
+    const int64_t row0 = int64_t(it.seg[sx]) * kTile, col0 = int64_t(it.seg[sy]) * kTile;
+
+    double re[2][4][2], im[2][4][2];
+    if (!herk_mainloop(re, im, k, sx, sy, half, g0, lane)) return false;
 
 #pragma unroll
     for (int mi = 0; mi < 2; ++mi) {
@@ -817,6 +828,10 @@ struct Image {
     uint32_t base32, full32, empty32;
 };
 
+// Every MMA warp, with or without a tile in the item, passes this wait before its arrival on the image's full
+// barrier: a warp's arrival for item i + 1 then cannot fall into the barrier phase of item i (the image of item
+// i is only released after that phase has completed and the write-out warps have read it).  The ring of stages
+// alone does not guarantee that for items of three K-steps or fewer.
 __device__ __forceinline__ bool wait_image_empty(const Call& k, const Image& im, uint32_t item_no, int lane) {
     if (item_no == 0) return true;
     const uint32_t parity = (item_no - 1) & 1;
@@ -824,14 +839,69 @@ __device__ __forceinline__ bool wait_image_empty(const Call& k, const Image& im,
     return wait_full_slow(im.empty32, parity, k.abort_flag, k.status, lane);
 }
 
+// The update a persistent launch runs: rank-k, rank-2k (two warps per tile, the rows of B in the stages' upper
+// slots) or Hermitian (two warps per tile, a real and an imaginary accumulator; the image holds complex entries,
+// 16 KB per tile, 16-byte entries with the index flipped in bit 0 on odd rows).
+constexpr int kModeSyrk = 0, kModeSyr2k = 1, kModeHerk = 2;
+
+// Keeps the ring moving for a warp without work in an item.
+__device__ __forceinline__ bool idle_mainloop_p(const Call& k, uint32_t g0, int lane) {
+    uint32_t st = g0 % kPStages, parity = (g0 / kPStages) & 1;
+    for (int ks = 0; ks < k.n_ksteps; ++ks) {
+        if (!wait_full_at(k, st, parity, lane)) return false;
+        release_at(k, st, lane);
+        if (++st == kPStages) { st = 0; parity ^= 1; }
+    }
+    return true;
+}
+
 // One MMA warp's share of item number item_no of its block: the M loop, then its accumulators into the image.
-template <bool kTN, bool kUpper>
+template <bool kTN, bool kUpper, int kMode>
 __device__ __forceinline__ bool mma_warp_item_p(const Call& k, const Image& im, const WorkItem& it, uint32_t& g,
                                                 uint32_t item_no, int warp, int lane) {
     const int gq = lane >> 2, t = lane & 3;
     const int n_tile = it.n_tile;
     const uint32_t g0 = g;
     g += uint32_t(k.n_ksteps);
+    if (kMode != kModeSyrk) {
+        if (warp < 2 * n_tile) {
+            const int tile = warp >> 1, half = warp & 1;
+            const int sx = it.tile_x[tile], sy = it.tile_y[tile];
+            if (kMode == kModeSyr2k) {
+                double acc[2][4][2];
+                if (!syr2k_mainloop<kPStages>(acc, k, sx, sy, half, fragment_offset(lane), g0, lane)) return false;
+                if (!wait_image_empty(k, im, item_no, lane)) return false;
+                const uint32_t tile32 = im.base32 + tile * kCTileBytes;
+#pragma unroll
+                for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+                    for (int ni = 0; ni < 4; ++ni)
+                        sts_f64x2(tile32 + image_offset((2 * half + mi) * 8 + gq, ni * 4 + t), scaled(k.alpha, acc[mi][ni][0]),
+                                  scaled(k.alpha, acc[mi][ni][1]));
+            } else {
+                double re[2][4][2], imag[2][4][2];
+                if (!herk_mainloop<kPStages>(re, imag, k, sx, sy, half, g0, lane)) return false;
+                if (!wait_image_empty(k, im, item_no, lane)) return false;
+                const uint32_t tile32 = im.base32 + tile * 2 * kCTileBytes;
+                const int diag = int(it.seg[sx] == it.seg[sy]);          // a tile on the diagonal: Im C[i][i] = 0
+#pragma unroll
+                for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+                    for (int ni = 0; ni < 4; ++ni)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int r = (2 * half + mi) * 8 + gq, c = ni * 8 + 2 * t + e;
+                            sts_f64x2(tile32 + uint32_t(r * 512 + ((c ^ (r & 1)) << 4)), scaled(k.alpha, re[mi][ni][e]),
+                                      (diag && r == c) ? 0.0 : scaled(k.alpha, imag[mi][ni][e]));
+                        }
+            }
+        } else if (!idle_mainloop_p(k, g0, lane) || !wait_image_empty(k, im, item_no, lane)) {
+            return false;
+        }
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(im.full32) : "memory");
+        return true;
+    }
     const bool scavenge = it.pad != 0;                  // set by prepare_item
     const uint32_t off0 = kTN ? fragment_offset_tn(lane) : fragment_offset(lane);
     if (scavenge && warp == kMmaWarps - 1) {
@@ -860,13 +930,8 @@ __device__ __forceinline__ bool mma_warp_item_p(const Call& k, const Image& im, 
                 if (scavenge && mi == 3 && ni == 3) continue;         // written by the 16th warp
                 sts_f64x2(tile32 + image_offset(mi * 8 + gq, ni * 4 + t), scaled(k.alpha, acc[mi][ni][0]), scaled(k.alpha, acc[mi][ni][1]));
             }
-    } else {
-        uint32_t st = g0 % kPStages, parity = (g0 / kPStages) & 1;    // no tile in this item: keep the ring moving
-        for (int ks = 0; ks < k.n_ksteps; ++ks) {
-            if (!wait_full_at(k, st, parity, lane)) return false;
-            release_at(k, st, lane);
-            if (++st == kPStages) { st = 0; parity ^= 1; }
-        }
+    } else if (!idle_mainloop_p(k, g0, lane) || !wait_image_empty(k, im, item_no, lane)) {   // no tile in this item
+        return false;
     }
     __syncwarp();
     if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(im.full32) : "memory");
@@ -919,9 +984,41 @@ __device__ __forceinline__ void write_out_item(const Call& k, const Image& im, c
     }
 }
 
-template <bool kTN, bool kUpper>
+// The same for the Hermitian update: complex entries (re, im) of 16 bytes, a warp instruction covers one row of a
+// tile (512 contiguous bytes of C); lower triangle; the diagonal's imaginary part is stored as zero, never read.
+__device__ __forceinline__ void write_out_item_herk(const Call& k, const Image& im, const WorkItem& it, int out_warp, int lane) {
+    const int mode = (k.beta == 0.0) ? 0 : (k.beta == 1.0 ? 1 : 2);
+    for (int q = out_warp; q < it.n_tile; q += kOutWarps) {
+        const int64_t row0 = int64_t(it.seg[it.tile_x[q]]) * kTile, col0 = int64_t(it.seg[it.tile_y[q]]) * kTile;
+        const uint32_t tile32 = im.base32 + q * 2 * kCTileBytes;
+        for (int r0 = 0; r0 < kTile; r0 += kOutBatch) {
+            double2 v[kOutBatch];
+#pragma unroll
+            for (int i = 0; i < kOutBatch; ++i) v[i] = lds_f64x2(tile32 + uint32_t((r0 + i) * 512 + (lane << 4)));
+#pragma unroll
+            for (int i = 0; i < kOutBatch; ++i) {
+                const int r = r0 + i;
+                const int64_t R = row0 + r, c = col0 + (lane ^ (r & 1));
+                if (R >= k.N || c > R) continue;
+                double* p = k.C + 2 * (R * k.ldc + c);
+                if (mode == 0) {
+                    *reinterpret_cast<double2*>(p) = v[i];
+                } else if (mode == 1) {
+                    red_add_f64(p, v[i].x);
+                    if (c == R) p[1] = 0.0; else red_add_f64(p + 1, v[i].y);
+                } else {
+                    p[0] = plus_old(v[i].x, k.beta, p[0]);
+                    p[1] = (c == R) ? 0.0 : plus_old(v[i].y, k.beta, p[1]);
+                }
+            }
+        }
+    }
+}
+
+template <bool kTN, bool kUpper, int kMode = kModeSyrk>
 __global__ void __launch_bounds__(kPThreads, 1)
-syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const WorkItem* __restrict__ items,
+syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                               const WorkItem* __restrict__ items,
                                int64_t n_items, int* __restrict__ counter, int64_t N, int32_t n_ksteps,
                                double* __restrict__ C, int64_t ldc, double alpha, double beta, int vec_ok,
                                int* __restrict__ status) {
@@ -939,9 +1036,10 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const Wo
     uint64_t* image_bar = k.empty_bar + kPStages;            // [0] full, [1] empty
     k.smem32 = smem_u32(smem); k.bars32 = smem_u32(k.full_bar); k.empties32 = k.bars32 + kPStages * 8;
     k.abort_flag = &s_abort; k.status = status;
-    k.tmA = &tmA; k.tmB = &tmA; k.tmC = &tmA;
+    k.tmA = &tmA; k.tmB = &tmB; k.tmC = &tmA;
     k.N = N; k.ncols = N; k.n_ksteps = n_ksteps; k.C = C; k.ldc = ldc; k.alpha = alpha; k.beta = beta;
-    k.vec_ok = vec_ok; k.c_tma = 0; k.gemm = false; k.batch = -1; k.k0 = 0; k.syr2k = false; k.herk = false;
+    k.vec_ok = vec_ok; k.c_tma = 0; k.gemm = false; k.batch = -1; k.k0 = 0;
+    k.syr2k = kMode == kModeSyr2k; k.herk = kMode == kModeHerk;
     Image im;
     im.base32 = k.smem32 + kPStages * kStageBytes;
     im.full32 = smem_u32(&image_bar[0]);
@@ -962,6 +1060,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const Wo
     if (warp == kOutWarps) {
         if (lane == 0) {
             prefetch_tensormap(&tmA);
+            if (kMode == kModeSyr2k) prefetch_tensormap(&tmB);
             for (uint32_t slot = 0;; ++slot) {
                 WorkItem& dst = s_ring[slot % kItemRing];
                 const int64_t idx = s_abort ? n_items : int64_t(atomicAdd(counter, 1));
@@ -1002,7 +1101,8 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const Wo
                 if (s_abort == 0) { s_abort = 1; if (lane == 0) atomicOr(status, kStatusWaitFull); }
                 return;
             }
-            write_out_item<kUpper>(k, im, it, out_warp, lane);
+            if (kMode == kModeHerk) write_out_item_herk(k, im, it, out_warp, lane);
+            else write_out_item<kUpper>(k, im, it, out_warp, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(&image_bar[1]);
         }
@@ -1013,7 +1113,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const Wo
         }
         const WorkItem& it = s_ring[slot % kItemRing];
         if (it.n_tile < 0) return;
-        if (!mma_warp_item_p<kTN, kUpper>(k, im, it, g, slot, warp - kOutWarps - 1, lane)) return;
+        if (!mma_warp_item_p<kTN, kUpper, kMode>(k, im, it, g, slot, warp - kOutWarps - 1, lane)) return;
     }
 }
 
@@ -1065,7 +1165,7 @@ cudaError_t configure_f64_kernels() {
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[10] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
+        const void* kernels[12] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, false>),
@@ -1074,9 +1174,12 @@ cudaError_t configure_f64_kernels() {
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, true>),
-                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, true>)};
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyr2k>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeHerk>)};
         for (const void* fn : kernels) {
-            const bool persistent = fn == kernels[6] || fn == kernels[7] || fn == kernels[8] || fn == kernels[9];
+            bool persistent = false;
+            for (int i = 6; i < 12; ++i) persistent = persistent || fn == kernels[i];
             cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  persistent ? f64::kPSmemBytes : f64::kSmemBytes);
             if (e != cudaSuccess) return e;
@@ -1133,8 +1236,8 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, true> : f64::syrk_f64_tbs_persistent_kernel<false, true>)
                             : (a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false> : f64::syrk_f64_tbs_persistent_kernel<false, false>);
-        kernel<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, d_items, n_items, d_tickets, N, n_ksteps, C, ldc,
-                                                                         alpha, beta, vec_ok, d_status);
+        kernel<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, tmA, d_items, n_items, d_tickets, N, n_ksteps, C,
+                                                                         ldc, alpha, beta, vec_ok, d_status);
         return cudaGetLastError();
     }
     auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, true> : f64::syrk_f64_tbs_kernel<false, true>)
@@ -1161,12 +1264,18 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
 
 cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap* tmC,
                              const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M, double* C, int64_t ldc,
-                             double alpha, double beta, int* d_status, cudaStream_t stream) {
+                             double alpha, double beta, int* d_status, cudaStream_t stream, int* d_tickets, int n_blocks) {
     cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0) ? 1 : 0;
     const int32_t n_ksteps = int32_t((M + f64::kBK - 1) / f64::kBK);
+    if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
+        const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
+        f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyr2k><<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(
+            tmA, tmB, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, vec_ok, d_status);
+        return cudaGetLastError();
+    }
     const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
     CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<false, false, true><<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
@@ -1176,12 +1285,19 @@ cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, con
 }
 
 cudaError_t launch_herk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int64_t n_items, int64_t N, int64_t M,
-                            double* C, int64_t ldc, double alpha, double beta, int* d_status, cudaStream_t stream) {
+                            double* C, int64_t ldc, double alpha, double beta, int* d_status, cudaStream_t stream,
+                            int* d_tickets, int n_blocks) {
     cudaError_t e = configure_f64_kernels();
     if (e != cudaSuccess) return e;
     if (n_items == 0) return cudaSuccess;
     if ((reinterpret_cast<uintptr_t>(C) & 15) != 0) return cudaErrorInvalidValue;     // complex entries move as 16-byte words
     const int32_t n_ksteps = int32_t((2 * M + f64::kBK - 1) / f64::kBK);             // the real view has 2M columns
+    if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
+        const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
+        f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeHerk><<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(
+            tmA, tmA, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, 1, d_status);
+        return cudaGetLastError();
+    }
     CUtensorMap none{};
     f64::syrk_f64_tbs_kernel<false, false, false, true><<<dim3(unsigned(n_items)), dim3(f64::kThreads), f64::kSmemBytes, stream>>>(
         tmA, tmA, none, d_items, N, N, 0, n_ksteps, C, ldc, alpha, beta, 1, 0, d_status,

@@ -185,3 +185,25 @@ def test_larger_problem_on_sampled_entries():
             assert C[i, j].imag == 0.0
     d = np.einsum("ik,ik->i", A, A.conj()).real
     assert np.all(np.diag(C).imag == 0.0) and np.allclose(np.diag(C).real, d, rtol=1e-12)
+
+
+@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-1.0, 1.0), (2.5, -0.5)])
+def test_launch_forms_agree_bit_for_bit(alpha, beta):
+    """One block per item and persistent blocks (whose write-out warps store C: a copy for beta = 0, memory-side
+    additions for beta = 1 with the diagonal's imaginary part stored as zero) run the same arithmetic: identical
+    bits, both within the bound; a NaN imaginary diagonal in C is never read."""
+    for n, (N, M, ldc_pad) in enumerate([(40, 25, 0), (1000, 35, 0), (1300, 20, 3), (2500, 17, 0), (4100, 24, 1)]):
+        A = I.normal_c128(N, M, seed=600 + n)
+        Cin = I.random_c128(N, 700 + n) if beta != 0.0 else None
+        outs = []
+        for mode in (B.F64_LAUNCH_PER_ITEM, B.F64_LAUNCH_PERSISTENT):
+            try:
+                B.syrk_set_f64_launch(mode)
+                got, ref, bound = run_herk(A, alpha, beta, Cin=Cin, ldc=N + ldc_pad, poison=(beta == 0.0),
+                                           nan_diag=(beta != 0.0))
+            finally:
+                B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+            check(got, ref, bound, M, Cin, alpha, beta)
+            outs.append(got)
+        il = np.tril_indices(N)
+        assert np.array_equal(outs[0][il].view(np.uint64), outs[1][il].view(np.uint64))

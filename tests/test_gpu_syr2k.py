@@ -123,3 +123,23 @@ def test_square_schedule_and_argument_errors():
         with pytest.raises(B.SyrkError) as e:
             B.syr2k_lower(**args)
         assert e.value.code == code
+
+
+@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-1.0, 1.0), (2.5, -0.5)])
+def test_launch_forms_agree_bit_for_bit(alpha, beta):
+    """One block per item and persistent blocks (whose write-out warps store C: a copy for beta = 0, a
+    memory-side addition for beta = 1) run the same arithmetic: identical bits, both within tolerance."""
+    for n, (N, M, ldc_pad) in enumerate([(40, 50, 0), (1000, 70, 0), (1300, 40, 3), (2500, 33, 0), (4100, 48, 2)]):
+        A, Bm = I.normal_f64(N, M, seed=7000 + n), I.normal_f64(N, M, seed=7100 + n)
+        Cin = I.random_c(N, 7200 + n, B.DTYPE_F64) if beta != 0.0 else None
+        outs = []
+        for mode in (B.F64_LAUNCH_PER_ITEM, B.F64_LAUNCH_PERSISTENT):
+            try:
+                B.syrk_set_f64_launch(mode)
+                got, ref, bound = run(A, Bm, alpha, beta, Cin, ldc=N + ldc_pad, poison=(beta == 0.0))
+            finally:
+                B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+            check(got, ref, bound, M, alpha, beta, Cin)
+            outs.append(got)
+        il = np.tril_indices(N)
+        assert np.array_equal(outs[0][il], outs[1][il])

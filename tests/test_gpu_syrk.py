@@ -8,6 +8,7 @@ Integer-valued inputs must match bit for bit whatever the summation order.
 """
 import numpy as np
 import pytest
+import torch
 
 from oracle import syrk as O
 from paper_2202_10217_b200 import binding as B
@@ -260,6 +261,28 @@ def test_f64_persistent_write_out_with_odd_pitch_or_offset_of_c(alpha, beta, ldc
         outs.append(got)
     il = np.tril_indices(N)
     assert np.array_equal(outs[0][il], outs[1][il])
+
+
+@pytest.mark.parametrize("M", [5, 16, 33, 48])
+def test_f64_persistent_form_with_items_of_one_to_three_k_steps(M):
+    """Items shorter than the ring of stages (one to three K-steps of 16 columns): the hand-over of the
+    accumulators' image between the MMA warps and the write-out warps must not depend on the ring to keep the
+    warps of one item together - warps without a tile in an item run ahead.  Long list, ragged edge, repeated."""
+    N = 4100
+    A = make_A(N, M, B.DTYPE_F64, seed=350 + M, kind="int")
+    dA = torch.from_numpy(A).cuda()
+    ref, _ = O.syrk_lower(A, None, 1.0, 0.0, B.DTYPE_F64)
+    il = np.tril_indices(N)
+    try:
+        B.syrk_set_f64_launch(B.F64_LAUNCH_PERSISTENT)
+        for rep in range(3):
+            dC = torch.full((N, N), float("nan"), dtype=torch.float64, device="cuda")
+            B.syrk_lower(N, M, dA, M, dC, N, 1.0, 0.0, B.DTYPE_F64)
+            torch.cuda.synchronize()
+            assert B.syrk_last_status() == 0
+            assert np.array_equal(dC.cpu().numpy()[il], ref[il]), rep
+    finally:
+        B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
 
 
 def test_f64_persistent_form_repeated_and_on_two_streams():
