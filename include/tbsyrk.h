@@ -457,8 +457,8 @@ int syrk_set_split_k(int slices);
 int syrk_set_f64_tail_split(int slices, int64_t tail_items);
 
 /*
- * How later FP64 calls hand the work items of the schedule (Algorithm 4, tiled as in
- * Section 5.1.4) to thread blocks; the paper has no counterpart, results are the same
+ * How later FP64 calls (syrk_lower and its variants, syr2k_lower, herk_lower) hand the work items
+ * of the schedule (Algorithm 4, tiled as in Section 5.1.4) to thread blocks; the paper has no counterpart, results are the same
  * entry for entry.  PER_ITEM: one thread block per item.  PERSISTENT: one block per SM
  * that draws items from a device-side counter; its MMA warps leave each item's
  * accumulators in shared memory and separate warps write them out during the next item's
