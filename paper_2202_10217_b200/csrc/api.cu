@@ -664,8 +664,13 @@ int syrk_lower_batched(int64_t batch, int64_t N, int64_t M, const void* A, int64
     if (dtype == SYRK_DTYPE_F64) {
         const bool c_tma = beta != 0.0 && c_aligned &&
                            encode_tensor_map_c_batched(&tmc, 1, C, N, ldc, stride_c, batch, f64_tile()) == SYRK_OK;
+        // persistent blocks over the (matrix, item) pairs when the launch-form rule says so for that many units
+        const int mode = runtime().f64_launch;
+        const bool persistent = mode == SYRK_F64_LAUNCH_PERSISTENT ||
+                                (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(M, n_items * batch, beta, ds->sm_count));
+        int* tickets = persistent ? tickets_for_stream(ds, st) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha,
-                            beta, 0, nullptr, 0, status_for_stream(ds, st), st, batch, stride_c);
+                            beta, 0, tickets, ds->sm_count, status_for_stream(ds, st), st, batch, stride_c);
     } else {
         const bool c_tma = c_aligned &&
                            encode_tensor_map_c_batched(&tmc, 0, C, N, ldc, stride_c, batch, bf16_store_box()) == SYRK_OK;

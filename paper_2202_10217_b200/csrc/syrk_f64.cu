@@ -949,7 +949,7 @@ __device__ __forceinline__ void red_add_f64(double* p, double v) {
     asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p), "d"(v) : "memory");
 }
 template <bool kUpper>
-__device__ __forceinline__ void write_out_item(const Call& k, const Image& im, const WorkItem& it, int out_warp, int lane) {
+__device__ __forceinline__ void write_out_item(const Call& k, const Image& im, const WorkItem& it, double* C, int out_warp, int lane) {
     const int mode = (k.beta == 0.0) ? 0 : (k.beta == 1.0 ? 1 : 2);
     const int half = lane >> 4, c16 = lane & 15;
     for (int q = out_warp; q < it.n_tile; q += kOutWarps) {
@@ -968,7 +968,7 @@ __device__ __forceinline__ void write_out_item(const Call& k, const Image& im, c
                 const bool ok0 = kUpper ? (c >= R && c < k.N) : (c <= R);
                 const bool ok1 = kUpper ? (c + 1 >= R && c + 1 < k.N) : (c + 1 <= R);
                 if (!ok0 && !ok1) continue;
-                double* p = k.C + R * k.ldc + c;
+                double* p = C + R * k.ldc + c;
                 if (mode == 0) {
                     if (ok0 && ok1 && (k.vec_ok & 1)) *reinterpret_cast<double2*>(p) = v[i];
                     else { if (ok0) p[0] = v[i].x; if (ok1) p[1] = v[i].y; }
@@ -1021,10 +1021,11 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                                const WorkItem* __restrict__ items,
                                int64_t n_items, int* __restrict__ counter, int64_t N, int32_t n_ksteps,
                                double* __restrict__ C, int64_t ldc, double alpha, double beta, int vec_ok,
-                               int* __restrict__ status) {
+                               int* __restrict__ status, int64_t items_per_batch, int64_t c_batch_stride) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ WorkItem s_ring[kItemRing];
+    __shared__ int32_t s_batch[kItemRing];        // strided batch (items_per_batch > 0): the matrix an item belongs to, else 0
     __shared__ uint64_t s_item_bar[kItemRing];
     __shared__ volatile int s_abort;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1066,8 +1067,14 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                 const int64_t idx = s_abort ? n_items : int64_t(atomicAdd(counter, 1));
                 bool last = idx >= n_items;
                 if (!last) {
+                    // strided batch: tickets run over (matrix, item) pairs, matrix-major; the 3-D tensor map takes the
+                    // matrix as its last coordinate
+                    const int64_t item_idx = items_per_batch > 0 ? idx % items_per_batch : idx;
+                    const int32_t matrix = items_per_batch > 0 ? int32_t(idx / items_per_batch) : 0;
+                    k.batch = items_per_batch > 0 ? matrix : -1;
+                    s_batch[slot % kItemRing] = matrix;
                     for (int w = 0; w < int(sizeof(WorkItem) / 4); ++w)
-                        reinterpret_cast<int32_t*>(&dst)[w] = reinterpret_cast<const int32_t*>(&items[idx])[w];
+                        reinterpret_cast<int32_t*>(&dst)[w] = reinterpret_cast<const int32_t*>(&items[item_idx])[w];
                     if (!prepare_item(k, dst, kUpper)) { s_abort = 1; atomicOr(status, kStatusBadItem); last = true; }
                 }
                 if (last) dst.n_tile = -1;                        // end marker
@@ -1102,7 +1109,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                 return;
             }
             if (kMode == kModeHerk) write_out_item_herk(k, im, it, out_warp, lane);
-            else write_out_item<kUpper>(k, im, it, out_warp, lane);
+            else write_out_item<kUpper>(k, im, it, k.C + int64_t(s_batch[slot % kItemRing]) * c_batch_stride, out_warp, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(&image_bar[1]);
         }
@@ -1224,6 +1231,15 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
     }
     if (batch > 0) {
         if (upper) return cudaErrorInvalidValue;
+        if (d_tickets != nullptr && n_blocks > 0 && n_items * batch < (int64_t(1) << 30)) {
+            // Strided batch on persistent blocks: tickets over the (matrix, item) pairs.
+            const int64_t units = n_items * batch;
+            const dim3 grid(unsigned(units < n_blocks ? units : int64_t(n_blocks)));
+            auto pk = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false> : f64::syrk_f64_tbs_persistent_kernel<false, false>;
+            pk<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, tmA, d_items, units, d_tickets, N, n_ksteps, C, ldc, alpha,
+                                                                     beta, vec_ok, d_status, n_items, c_batch_stride);
+            return cudaGetLastError();
+        }
         // Strided batch (3-D tensor maps): one block per (matrix, item), matrix-major.
         if (n_items * batch >= (int64_t(1) << 31)) return cudaErrorInvalidValue;
         auto kernel = a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, false> : f64::syrk_f64_tbs_kernel<false, false>;
@@ -1237,7 +1253,7 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
         auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, true> : f64::syrk_f64_tbs_persistent_kernel<false, true>)
                             : (a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false> : f64::syrk_f64_tbs_persistent_kernel<false, false>);
         kernel<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, tmA, d_items, n_items, d_tickets, N, n_ksteps, C,
-                                                                         ldc, alpha, beta, vec_ok, d_status);
+                                                                         ldc, alpha, beta, vec_ok, d_status, int64_t(0), int64_t(0));
         return cudaGetLastError();
     }
     auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, true> : f64::syrk_f64_tbs_kernel<false, true>)
@@ -1273,7 +1289,7 @@ cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, con
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyr2k><<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(
-            tmA, tmB, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, vec_ok, d_status);
+            tmA, tmB, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, vec_ok, d_status, int64_t(0), int64_t(0));
         return cudaGetLastError();
     }
     const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
@@ -1295,7 +1311,7 @@ cudaError_t launch_herk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeHerk><<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(
-            tmA, tmA, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, 1, d_status);
+            tmA, tmA, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, 1, d_status, int64_t(0), int64_t(0));
         return cudaGetLastError();
     }
     CUtensorMap none{};

@@ -157,3 +157,25 @@ def test_batch_of_one_and_of_zero_and_argument_errors():
         assert e.value.code == code
     torch.cuda.synchronize()
     assert bool((dC == 3.0).all())
+
+
+@pytest.mark.parametrize("alpha,beta", [(1.0, 0.0), (-1.0, 1.0), (2.5, -0.5)])
+def test_f64_launch_forms_agree_bit_for_bit(alpha, beta):
+    """FP64 batches on persistent blocks (tickets over the (matrix, item) pairs, C written by the write-out warps)
+    against one block per (matrix, item): identical bits, both within tolerance; gaps between the matrices, an odd
+    stride of C (8-byte accesses), and short inner dimensions (items of one to three K-steps)."""
+    for n, (batch, N, M, c_gap) in enumerate([(40, 96, 32, 0), (300, 70, 20, 0), (9, 520, 100, 8), (6, 1056, 48, 3)]):
+        As = [make_A(N, M, B.DTYPE_F64, seed=2900 + 10 * n + b) for b in range(batch)]
+        Cins = [I.random_c(N, 2950 + 10 * n + b, B.DTYPE_F64) for b in range(batch)] if beta != 0.0 else None
+        outs = []
+        for mode in (B.F64_LAUNCH_PER_ITEM, B.F64_LAUNCH_PERSISTENT):
+            try:
+                B.syrk_set_f64_launch(mode)
+                got = run_batched(As, B.DTYPE_F64, alpha, beta, Cins, stride_c=N * N + c_gap, poison=(beta == 0.0))
+            finally:
+                B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+            check(As, got, B.DTYPE_F64, alpha, beta, Cins)
+            outs.append(got)
+        il = np.tril_indices(N)
+        for b in range(batch):
+            assert np.array_equal(outs[0][b][il], outs[1][b][il]), (n, b)
