@@ -7,8 +7,8 @@
 // K-step where a square block of the same accumulator count streams 8.
 //
 //   producer warp : plain TMA tile loads (no multicast) of the item's segments,
-//                   16 columns of A per stage, into a 6-stage shared-memory ring
-//                   (128-byte swizzle), signalled through mbarriers;
+//                   16 columns of A per stage, into a shared-memory ring of stages
+//                   (128-byte swizzle; six stages, three in the persistent form), signalled through mbarriers;
 //   16 MMA warps  : warp w owns tile w: a 32 x 32 accumulator held in registers as
 //                   4 x 4 blocks of mma.sync m8n8k4 (FP64 tensor core, DMMA).  Each of the
 //                   SM's four schedulers has its own DMMA pipe, so an item lasts as long as
@@ -16,7 +16,7 @@
 //                   leave out their last 8 x 8 block and the 16th warp owns those 15 blocks -
 //                   itself a triangle block over the last 8 rows of the six segments - so
 //                   that every warp issues 15 DMMAs per k-slice instead of 16, 16, 16, 12;
-//   epilogue      : alpha * acc (+ beta * C) written for entries with col <= row
+//   epilogue      : (one block per item) alpha * acc (+ beta * C) written for entries with col <= row
 //                   only, two doubles per store where alignment allows.  With beta != 0
 //                   the producer also TMA-loads the item's old C tiles (those below the
 //                   diagonal) into the ring's stages as the last K-steps release them, so
@@ -27,8 +27,8 @@
 // one block per SM, whose producer draws the next item from a global counter and publishes
 // it to the MMA warps through a small ring in shared memory: the ring of stages then runs on
 // across items.  In the persistent form the MMA warps do not write C themselves: they leave their
-// accumulators in a shared-memory image and three more warps write it out (reading old C from memory
-// when beta != 0) while the next item's M loop runs; its ring has three stages.
+// accumulators in a shared-memory image and three more warps write it out while the next item's M loop
+// runs.  The same two forms serve the rank-2k and the Hermitian updates (two warps per tile) and strided batches.
 //
 // Accumulators (the C block) stay on chip for the whole M loop and each entry of
 // C is read (beta != 0) and written exactly once, as in the paper's generic
