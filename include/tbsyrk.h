@@ -252,7 +252,8 @@ int herk_lower(int64_t N, int64_t M,
  * memory, strides in elements.  The paper states the update for one matrix; the batch exists because a
  * small problem (tens of work items) cannot fill the GPU on its own: every matrix uses the work list
  * of Algorithm 4 / Section 5.1.4 for its N, and one launch runs the (matrix, item) pairs of the whole
- * batch (FP64: one thread block per pair; tcgen05 types: pairs dealt to the persistent blocks; the
+ * batch (FP64: one thread block per pair, or persistent blocks drawing the pairs from a counter,
+ * by the rule of syrk_set_f64_launch; tcgen05 types: pairs dealt to the persistent blocks; the
  * inner dimension is never split here).  Requirements for that single launch: A 16-byte aligned and
  * lda * sizeof(element) and stride_a * sizeof(element) multiples of 16; otherwise, and for alpha == 0
  * or M == 0, the matrices are enqueued one after the other exactly as `batch` syrk_lower calls.
