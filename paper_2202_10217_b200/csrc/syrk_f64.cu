@@ -1015,7 +1015,7 @@ __device__ __forceinline__ void write_out_item_herk(const Call& k, const Image& 
     }
 }
 
-template <bool kTN, bool kUpper, int kMode = kModeSyrk>
+template <bool kTN, bool kUpper, int kMode = kModeSyrk, bool kBatched = false>
 __global__ void __launch_bounds__(kPThreads, 1)
 syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                                const WorkItem* __restrict__ items,
@@ -1025,7 +1025,7 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ WorkItem s_ring[kItemRing];
-    __shared__ int32_t s_batch[kItemRing];        // strided batch (items_per_batch > 0): the matrix an item belongs to, else 0
+    __shared__ int32_t s_batch[kItemRing];        // strided batch (kBatched): the matrix an item belongs to
     __shared__ uint64_t s_item_bar[kItemRing];
     __shared__ volatile int s_abort;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1068,11 +1068,17 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                 bool last = idx >= n_items;
                 if (!last) {
                     // strided batch: tickets run over (matrix, item) pairs, matrix-major; the 3-D tensor map takes the
-                    // matrix as its last coordinate
-                    const int64_t item_idx = items_per_batch > 0 ? idx % items_per_batch : idx;
-                    const int32_t matrix = items_per_batch > 0 ? int32_t(idx / items_per_batch) : 0;
-                    k.batch = items_per_batch > 0 ? matrix : -1;
-                    s_batch[slot % kItemRing] = matrix;
+                    // matrix as its last coordinate.  (A template parameter: with k.batch a constant the producer's loads
+                    // are the 2-D ones without a branch: a few instructions more per load in this thread cost 0.5 % of a
+                    // call.  Issuing the loads from several lanes, fetching the next item ahead of time, or moving this
+                    // warp to another scheduler gained nothing - all measured.)
+                    int64_t item_idx = idx;
+                    if (kBatched) {
+                        const int32_t matrix = int32_t(uint32_t(idx) / uint32_t(items_per_batch));
+                        item_idx = idx - int64_t(matrix) * items_per_batch;
+                        k.batch = matrix;
+                        s_batch[slot % kItemRing] = matrix;
+                    }
                     for (int w = 0; w < int(sizeof(WorkItem) / 4); ++w)
                         reinterpret_cast<int32_t*>(&dst)[w] = reinterpret_cast<const int32_t*>(&items[item_idx])[w];
                     if (!prepare_item(k, dst, kUpper)) { s_abort = 1; atomicOr(status, kStatusBadItem); last = true; }
@@ -1109,7 +1115,8 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                 return;
             }
             if (kMode == kModeHerk) write_out_item_herk(k, im, it, out_warp, lane);
-            else write_out_item<kUpper>(k, im, it, k.C + int64_t(s_batch[slot % kItemRing]) * c_batch_stride, out_warp, lane);
+            else write_out_item<kUpper>(k, im, it, kBatched ? k.C + int64_t(s_batch[slot % kItemRing]) * c_batch_stride : k.C,
+                                        out_warp, lane);
             __syncwarp();
             if (lane == 0) mbar_arrive(&image_bar[1]);
         }
@@ -1172,7 +1179,7 @@ cudaError_t configure_f64_kernels() {
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[12] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
+        const void* kernels[14] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, false>),
@@ -1183,10 +1190,12 @@ cudaError_t configure_f64_kernels() {
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyr2k>),
-                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeHerk>)};
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeHerk>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyrk, true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, false, f64::kModeSyrk, true>)};
         for (const void* fn : kernels) {
             bool persistent = false;
-            for (int i = 6; i < 12; ++i) persistent = persistent || fn == kernels[i];
+            for (int i = 6; i < 14; ++i) persistent = persistent || fn == kernels[i];
             cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  persistent ? f64::kPSmemBytes : f64::kSmemBytes);
             if (e != cudaSuccess) return e;
@@ -1235,7 +1244,8 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
             // Strided batch on persistent blocks: tickets over the (matrix, item) pairs.
             const int64_t units = n_items * batch;
             const dim3 grid(unsigned(units < n_blocks ? units : int64_t(n_blocks)));
-            auto pk = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false> : f64::syrk_f64_tbs_persistent_kernel<false, false>;
+            auto pk = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false, f64::kModeSyrk, true>
+                                  : f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyrk, true>;
             pk<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, tmA, d_items, units, d_tickets, N, n_ksteps, C, ldc, alpha,
                                                                      beta, vec_ok, d_status, n_items, c_batch_stride);
             return cudaGetLastError();
