@@ -452,8 +452,8 @@ int syrk_set_split_k(int slices);
  *                          items and how many slices (used when modelled at least 1.5 % faster);
  *   slices == 1: never;
  *   slices >= 2: always, for the last `tail_items` items of the list (tests and measurements).
- * Not used by the persistent launch form, the upper triangle, batches, or calls that cut every item
- * (fewer items than SMs).  Process-wide.  SYRK_ERR_PLAN for slices outside 0..64 or tail_items < 0.
+ * Both launch forms take it (in the persistent form the slices are further tickets).  Not used by the
+ * upper triangle, batches, or calls that cut every item (fewer items than SMs).  Process-wide.  SYRK_ERR_PLAN for slices outside 0..64 or tail_items < 0.
  */
 int syrk_set_f64_tail_split(int slices, int64_t tail_items);
 
@@ -467,8 +467,9 @@ int syrk_set_f64_tail_split(int slices, int64_t tail_items);
  * system, the correctly rounded sum; another beta: a multiply-add in those warps, which is slow
  * because the tensor-core work holds the FP64 pipes).  Used only outside stream capture and for
  * at most 256 distinct streams per device, else the call falls back to PER_ITEM.  AUTO (default):
- * PERSISTENT for beta == 0 or 1 when the list has at least eight items per SM, or at least
- * one per SM with M at most 300 columns per round of items; PER_ITEM otherwise.
+ * PERSISTENT for beta == 0 or 1 when the list has at least one item per SM; PER_ITEM otherwise.
+ * Both forms cut the last items of a list of a few rounds of long items into K-slices
+ * (syrk_set_f64_tail_split).
  * Returns SYRK_ERR_PLAN for another value.  Process-wide.
  */
 #define SYRK_F64_LAUNCH_AUTO 0

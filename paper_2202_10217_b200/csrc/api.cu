@@ -62,14 +62,12 @@ int auto_split_k(const std::vector<WorkItem>& items, int64_t M, int bk, int sm_c
     return best;
 }
 
-// The automatic choice of the FP64 launch form.  Persistent blocks hide every item's write-out behind the next
-// item's M loop (for beta == 0 and beta == 1, see the kernel); one block per item has the tail K-split to even out
-// the last round of a list of a few rounds of long items.  Measured on 2048 to 16384 rows and 256 to 4096 columns:
-// persistent blocks win from about nine rounds of items on whatever the inner dimension, and on shorter lists
-// while an item is short against the list (M up to about 300 columns per round).
-bool f64_persistent_pays(int64_t M, int64_t n_items, double beta, int sm_count) {
-    if (!(beta == 0.0 || beta == 1.0) || n_items < int64_t(sm_count)) return false;
-    return n_items >= 8 * int64_t(sm_count) || M * int64_t(sm_count) <= 300 * n_items;
+// The automatic choice of the FP64 launch form.  Persistent blocks hide every item's start-up and write-out behind
+// the next item's M loop (for beta == 0 and beta == 1, see the kernel) and take the tail K-split as the other form does.
+// Measured on 2048 to 16384 rows and 256 to 8192 columns, they win or tie wherever the list has an item per SM; shorter
+// lists run one block per (item, K-slice).
+bool f64_persistent_pays(int64_t n_items, double beta, int sm_count) {
+    return (beta == 0.0 || beta == 1.0) && n_items >= int64_t(sm_count);
 }
 
 // K-slices for an FP64 call (one block per item).  With fewer items than SMs the inner
@@ -164,8 +162,8 @@ int launch_items(DeviceState* ds, int dtype, const CUtensorMap& tm, const WorkIt
         // Persistent blocks hide each item's start-up and write-out behind the next item's M loop
         // (see f64_persistent_pays for when that is the faster form).
         const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
-        const bool persistent = tail_slices <= 1 && (mode == SYRK_F64_LAUNCH_PERSISTENT ||
-                                (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(M, n_items, beta, ds->sm_count)));
+        const bool persistent = mode == SYRK_F64_LAUNCH_PERSISTENT ||
+                                (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(n_items, beta, ds->sm_count));
         int* tickets = (persistent && split <= 1) ? tickets_for_stream(ds, stream) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, d_items, n_items, N, M, static_cast<double*>(C), ldc,
                             alpha, beta, a_is_m_by_n, tickets, ds->sm_count, d_status, stream, 0, 0, split,
@@ -353,12 +351,9 @@ int tbsyrk::syrk_run_device(int64_t N, int64_t M, const void* A, int64_t lda, vo
         if (split > 1 &&
             (rc = workspace_for_stream(ds, stream, size_t(split) * size_t(N) * size_t(N) * sizeof(double), &d_partial)) != SYRK_OK)
             return rc;
-        // Otherwise, in the one-block-per-item form: the last round's items in slices (tail K-split).
+        // Otherwise: the last round's items in slices (tail K-split), in either launch form.
         const int64_t n_items = int64_t(dp->plan.items.size());
-        const int mode = f64_launch >= 0 ? f64_launch : runtime().f64_launch;
-        const bool per_item = mode == SYRK_F64_LAUNCH_PER_ITEM ||
-                              (mode == SYRK_F64_LAUNCH_AUTO && !f64_persistent_pays(M, n_items, beta, ds->sm_count));
-        if (split == 1 && per_item && !upper && runtime().f64_tail_slices != 1) {
+        if (split == 1 && !upper && runtime().f64_tail_slices != 1) {
             TailSplit ts{n_items, 1};
             const int64_t ksteps = (M + ks.bk - 1) / ks.bk;
             if (runtime().f64_tail_slices >= 2) {                    // forced (tests, measurements)
@@ -426,12 +421,12 @@ __global__ void unpack_lower_axpby_kernel(int64_t first, int64_t count, const T*
     }
 }
 
-// The launch form of the rank-2k and Hermitian updates (inner dimension in binary64 columns of a stage row):
-// as set by syrk_set_f64_launch, the automatic rule being that of the rank-k update.
-bool two_warp_form_is_persistent(int64_t columns, int64_t n_items, double beta, int sm_count) {
+// The launch form of the rank-2k and Hermitian updates: as set by syrk_set_f64_launch, the automatic rule being
+// that of the rank-k update.
+bool two_warp_form_is_persistent(int64_t n_items, double beta, int sm_count) {
     const int mode = runtime().f64_launch;
     return mode == SYRK_F64_LAUNCH_PERSISTENT ||
-           (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(columns, n_items, beta, sm_count));
+           (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(n_items, beta, sm_count));
 }
 
 // Work list of Algorithm 4 for the kernels' forms in which two warps share a tile (rank-2k and Hermitian
@@ -551,7 +546,7 @@ int syr2k_lower(int64_t N, int64_t M, const void* A, int64_t lda, const void* B,
     const bool c_tma = beta != 0.0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc & 1) == 0 &&
                        encode_tensor_map_c_f64(&tmc, C, N, ldc, f64_tile()) == SYRK_OK;
     const int64_t n_items = int64_t(dp->plan.items.size());
-    int* tickets = two_warp_form_is_persistent(M, n_items, beta, ds->sm_count) ? tickets_for_stream(ds, st) : nullptr;
+    int* tickets = two_warp_form_is_persistent(n_items, beta, ds->sm_count) ? tickets_for_stream(ds, st) : nullptr;
     return launch_syr2k_f64(ta, tb, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha,
                             beta, status_for_stream(ds, st), st, tickets, ds->sm_count) == cudaSuccess
                ? SYRK_OK : SYRK_ERR_CUDA;
@@ -578,7 +573,7 @@ int herk_lower(int64_t N, int64_t M, const void* A, int64_t lda, void* C, int64_
     CUtensorMap ta;          // the real view of A: N rows of 2M values, pitch 2 lda
     if ((rc = encode_tensor_map_2d(&ta, SYRK_DTYPE_F64, A, N, 2 * M, 2 * lda, f64_tile(), f64_bk())) != SYRK_OK) return rc;
     const int64_t n_items = int64_t(dp->plan.items.size());
-    int* tickets = two_warp_form_is_persistent(2 * M, n_items, beta, ds->sm_count) ? tickets_for_stream(ds, st) : nullptr;
+    int* tickets = two_warp_form_is_persistent(n_items, beta, ds->sm_count) ? tickets_for_stream(ds, st) : nullptr;
     return launch_herk_f64(ta, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha, beta, status_for_stream(ds, st),
                            st, tickets, ds->sm_count) == cudaSuccess ? SYRK_OK : SYRK_ERR_CUDA;
 }
@@ -667,7 +662,7 @@ int syrk_lower_batched(int64_t batch, int64_t N, int64_t M, const void* A, int64
         // persistent blocks over the (matrix, item) pairs when the launch-form rule says so for that many units
         const int mode = runtime().f64_launch;
         const bool persistent = mode == SYRK_F64_LAUNCH_PERSISTENT ||
-                                (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(M, n_items * batch, beta, ds->sm_count));
+                                (mode == SYRK_F64_LAUNCH_AUTO && f64_persistent_pays(n_items * batch, beta, ds->sm_count));
         int* tickets = persistent ? tickets_for_stream(ds, st) : nullptr;
         e = launch_syrk_f64(tm, c_tma ? &tmc : nullptr, dp->d_items, n_items, N, M, static_cast<double*>(C), ldc, alpha,
                             beta, 0, tickets, ds->sm_count, status_for_stream(ds, st), st, batch, stride_c);
@@ -1065,14 +1060,14 @@ int syrk_get_schedule_stats(int64_t N, int64_t M, int dtype, syrk_schedule_stats
     out->launches = split > 1 ? 2 : 1;
     bool f64_persistent = false;
     if (dtype == SYRK_DTYPE_F64 && split == 1 && out->effective_schedule != SYRK_SCHEDULE_PAIR_SQUARE) {
-        // the tail K-split of the one-block-per-item form adds its reduction kernel (the launch form is taken as
-        // for beta == 0 or 1; the automatic settings are assumed)
+        // the tail K-split (either launch form) adds its reduction kernel; the launch form is taken as for
+        // beta == 0 or 1
         int mode, tail_setting;
         { std::lock_guard<std::mutex> lock(runtime().mu); mode = runtime().f64_launch; tail_setting = runtime().f64_tail_slices; }
         const int64_t n_items = int64_t(plan.items.size());
         const bool per_item = mode == SYRK_F64_LAUNCH_PER_ITEM ||
-                              (mode == SYRK_F64_LAUNCH_AUTO && !f64_persistent_pays(M, n_items, 0.0, 148));
-        if (per_item && tail_setting == 0 && plan_tail_split_f64(plan.items, (M + ks.bk - 1) / ks.bk, 148).slices > 1)
+                              (mode == SYRK_F64_LAUNCH_AUTO && !f64_persistent_pays(n_items, 0.0, 148));
+        if (tail_setting == 0 && plan_tail_split_f64(plan.items, (M + ks.bk - 1) / ks.bk, 148).slices > 1)
             out->launches = 2;
         f64_persistent = !per_item;
     }

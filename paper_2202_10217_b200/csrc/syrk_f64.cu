@@ -984,6 +984,23 @@ __device__ __forceinline__ void write_out_item(const Call& k, const Image& im, c
     }
 }
 
+// A K-slice of a tail item (tail K-split, persistent form): the raw sums of every tile go to the unit's partial
+// tiles (slot q at q * 1024 doubles, row-major 32 x 32), all entries; the reduction kernel applies alpha, beta and
+// the triangle mask.
+__device__ __forceinline__ void write_out_partial(const Image& im, const WorkItem& it, double* unit, int out_warp, int lane) {
+    const int half = lane >> 4, c16 = lane & 15;
+    for (int q = out_warp; q < it.n_tile; q += kOutWarps) {
+        const uint32_t tile32 = im.base32 + q * kCTileBytes;
+        double* dst = unit + q * kPartTileElems;
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {
+            const int r = 2 * i + half;
+            const double2 v = lds_f64x2(tile32 + uint32_t(r * 256 + (c16 << 4)));
+            *reinterpret_cast<double2*>(dst + r * kTile + 2 * (c16 ^ ((r & 1) << 2))) = v;
+        }
+    }
+}
+
 // The same for the Hermitian update: complex entries (re, im) of 16 bytes, a warp instruction covers one row of a
 // tile (512 contiguous bytes of C); lower triangle; the diagonal's imaginary part is stored as zero, never read.
 __device__ __forceinline__ void write_out_item_herk(const Call& k, const Image& im, const WorkItem& it, int out_warp, int lane) {
@@ -1015,17 +1032,23 @@ __device__ __forceinline__ void write_out_item_herk(const Call& k, const Image& 
     }
 }
 
-template <bool kTN, bool kUpper, int kMode = kModeSyrk, bool kBatched = false>
+// kTail (rank-k update, lower triangle): tickets [0, tail_first) are the list's first items, whole; the tickets after
+// them are the remaining items in tail_slices slices of the inner dimension each (item-major), whose raw sums go to
+// `tail_partial` for tail_reduce_f64_kernel - smaller units for the last round, as in the one-block-per-item form.
+template <bool kTN, bool kUpper, int kMode = kModeSyrk, bool kBatched = false, bool kTail = false>
 __global__ void __launch_bounds__(kPThreads, 1)
 syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                                const WorkItem* __restrict__ items,
                                int64_t n_items, int* __restrict__ counter, int64_t N, int32_t n_ksteps,
                                double* __restrict__ C, int64_t ldc, double alpha, double beta, int vec_ok,
-                               int* __restrict__ status, int64_t items_per_batch, int64_t c_batch_stride) {
+                               int* __restrict__ status, int64_t items_per_batch, int64_t c_batch_stride,
+                               int32_t tail_first, int32_t tail_slices, double* __restrict__ tail_partial) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ WorkItem s_ring[kItemRing];
     __shared__ int32_t s_batch[kItemRing];        // strided batch (kBatched): the matrix an item belongs to
+    __shared__ int32_t s_unit[kItemRing];         // kTail: the slice unit an entry of the ring is (-1: a whole item) ...
+    __shared__ int32_t s_nk[kItemRing];           // ... and its number of K-steps
     __shared__ uint64_t s_item_bar[kItemRing];
     __shared__ volatile int s_abort;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1079,6 +1102,19 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                         k.batch = matrix;
                         s_batch[slot % kItemRing] = matrix;
                     }
+                    if (kTail) {
+                        int32_t unit = -1, k0 = 0, nk = n_ksteps;
+                        if (idx >= tail_first) {
+                            unit = int32_t(idx) - tail_first;
+                            const int32_t sl = unit % tail_slices;
+                            item_idx = tail_first + unit / tail_slices;
+                            k0 = int32_t(int64_t(n_ksteps) * sl / tail_slices);
+                            nk = int32_t(int64_t(n_ksteps) * (sl + 1) / tail_slices) - k0;
+                        }
+                        k.k0 = k0; k.n_ksteps = nk;
+                        s_unit[slot % kItemRing] = unit;
+                        s_nk[slot % kItemRing] = nk;
+                    }
                     for (int w = 0; w < int(sizeof(WorkItem) / 4); ++w)
                         reinterpret_cast<int32_t*>(&dst)[w] = reinterpret_cast<const int32_t*>(&items[item_idx])[w];
                     if (!prepare_item(k, dst, kUpper)) { s_abort = 1; atomicOr(status, kStatusBadItem); last = true; }
@@ -1115,6 +1151,8 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
                 return;
             }
             if (kMode == kModeHerk) write_out_item_herk(k, im, it, out_warp, lane);
+            else if (kTail && s_unit[slot % kItemRing] >= 0)
+                write_out_partial(im, it, tail_partial + int64_t(s_unit[slot % kItemRing]) * kPartUnitElems, out_warp, lane);
             else write_out_item<kUpper>(k, im, it, kBatched ? k.C + int64_t(s_batch[slot % kItemRing]) * c_batch_stride : k.C,
                                         out_warp, lane);
             __syncwarp();
@@ -1127,6 +1165,10 @@ syrk_f64_tbs_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __
         }
         const WorkItem& it = s_ring[slot % kItemRing];
         if (it.n_tile < 0) return;
+        if (kTail) {                                       // a slice's raw sums are left unscaled
+            k.n_ksteps = s_nk[slot % kItemRing];
+            k.alpha = s_unit[slot % kItemRing] >= 0 ? 1.0 : alpha;
+        }
         if (!mma_warp_item_p<kTN, kUpper, kMode>(k, im, it, g, slot, warp - kOutWarps - 1, lane)) return;
     }
 }
@@ -1179,7 +1221,7 @@ cudaError_t configure_f64_kernels() {
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        const void* kernels[14] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
+        const void* kernels[16] = {reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false, true>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<false, false>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_kernel<true, false>),
@@ -1192,10 +1234,12 @@ cudaError_t configure_f64_kernels() {
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyr2k>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeHerk>),
                                   reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyrk, true>),
-                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, false, f64::kModeSyrk, true>)};
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, false, f64::kModeSyrk, true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyrk, false, true>),
+                                  reinterpret_cast<const void*>(&f64::syrk_f64_tbs_persistent_kernel<true, false, f64::kModeSyrk, false, true>)};
         for (const void* fn : kernels) {
             bool persistent = false;
-            for (int i = 6; i < 14; ++i) persistent = persistent || fn == kernels[i];
+            for (int i = 6; i < 16; ++i) persistent = persistent || fn == kernels[i];
             cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  persistent ? f64::kPSmemBytes : f64::kSmemBytes);
             if (e != cudaSuccess) return e;
@@ -1247,7 +1291,7 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
             auto pk = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false, f64::kModeSyrk, true>
                                   : f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyrk, true>;
             pk<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, tmA, d_items, units, d_tickets, N, n_ksteps, C, ldc, alpha,
-                                                                     beta, vec_ok, d_status, n_items, c_batch_stride);
+                                                                     beta, vec_ok, d_status, n_items, c_batch_stride, 0, 1, nullptr);
             return cudaGetLastError();
         }
         // Strided batch (3-D tensor maps): one block per (matrix, item), matrix-major.
@@ -1258,12 +1302,30 @@ cudaError_t launch_syrk_f64(const CUtensorMap& tmA, const CUtensorMap* tmC, cons
             n_items, c_batch_stride, 0, 0, 1, nullptr);
         return cudaGetLastError();
     }
+    if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30) && tail_slices > 1 && d_partial != nullptr && !upper &&
+        tail_first >= 0 && tail_first < n_items) {
+        // Persistent blocks with a tail K-split: the last n_items - tail_first items as tail_slices tickets each.
+        const int64_t n_tail = n_items - tail_first;
+        const int64_t units = tail_first + n_tail * tail_slices;
+        if (units >= (int64_t(1) << 30) || n_tail >= 65536 || tail_slices > n_ksteps) return cudaErrorInvalidValue;
+        const dim3 grid(unsigned(units < n_blocks ? units : int64_t(n_blocks)));
+        auto pk = a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false, f64::kModeSyrk, false, true>
+                              : f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyrk, false, true>;
+        pk<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, tmA, d_items, units, d_tickets, N, n_ksteps, C, ldc, alpha,
+                                                                 beta, vec_ok, d_status, int64_t(0), int64_t(0), int32_t(tail_first),
+                                                                 int32_t(tail_slices), d_partial);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        f64::tail_reduce_f64_kernel<<<dim3(unsigned(n_tail), f64::kMmaWarps), 256, 0, stream>>>(
+            d_items, int32_t(tail_first), int32_t(tail_slices), d_partial, N, C, ldc, alpha, beta);
+        return cudaGetLastError();
+    }
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, true> : f64::syrk_f64_tbs_persistent_kernel<false, true>)
                             : (a_is_m_by_n ? f64::syrk_f64_tbs_persistent_kernel<true, false> : f64::syrk_f64_tbs_persistent_kernel<false, false>);
         kernel<<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(tmA, tmA, d_items, n_items, d_tickets, N, n_ksteps, C,
-                                                                         ldc, alpha, beta, vec_ok, d_status, int64_t(0), int64_t(0));
+                                                                         ldc, alpha, beta, vec_ok, d_status, int64_t(0), int64_t(0), 0, 1, nullptr);
         return cudaGetLastError();
     }
     auto kernel = upper ? (a_is_m_by_n ? f64::syrk_f64_tbs_kernel<true, true> : f64::syrk_f64_tbs_kernel<false, true>)
@@ -1299,7 +1361,7 @@ cudaError_t launch_syr2k_f64(const CUtensorMap& tmA, const CUtensorMap& tmB, con
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeSyr2k><<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(
-            tmA, tmB, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, vec_ok, d_status, int64_t(0), int64_t(0));
+            tmA, tmB, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, vec_ok, d_status, int64_t(0), int64_t(0), 0, 1, nullptr);
         return cudaGetLastError();
     }
     const int c_tma = (tmC != nullptr && beta != 0.0 && vec_ok) ? 1 : 0;
@@ -1321,7 +1383,7 @@ cudaError_t launch_herk_f64(const CUtensorMap& tmA, const WorkItem* d_items, int
     if (d_tickets != nullptr && n_blocks > 0 && n_items < (int64_t(1) << 30)) {
         const dim3 grid(unsigned(n_items < n_blocks ? n_items : int64_t(n_blocks)));
         f64::syrk_f64_tbs_persistent_kernel<false, false, f64::kModeHerk><<<grid, dim3(f64::kPThreads), f64::kPSmemBytes, stream>>>(
-            tmA, tmA, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, 1, d_status, int64_t(0), int64_t(0));
+            tmA, tmA, d_items, n_items, d_tickets, N, n_ksteps, C, ldc, alpha, beta, 1, d_status, int64_t(0), int64_t(0), 0, 1, nullptr);
         return cudaGetLastError();
     }
     CUtensorMap none{};

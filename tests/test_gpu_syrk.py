@@ -381,18 +381,25 @@ def test_f64_tail_k_split_forced(slices, tail, tn):
         A = make_A(N, M, B.DTYPE_F64, seed=1000 + n)
         Ai = make_A(N, M, B.DTYPE_F64, seed=1050 + n, kind="int")
         Cin = I.random_c(N, 1060 + n, B.DTYPE_F64)
-        try:
-            B.syrk_set_f64_launch(B.F64_LAUNCH_PER_ITEM)
-            B.syrk_set_f64_tail_split(slices, tail)
-            got, ref, bound = run_case(A, B.DTYPE_F64, -1.5, 0.5, Cin, ldc=N + 2, tn=tn)
-            again, _, _ = run_case(A, B.DTYPE_F64, -1.5, 0.5, Cin, ldc=N + 2, tn=tn)
-            goti, refi, boundi = run_case(Ai, B.DTYPE_F64, 1.0, 0.0, poison=True, tn=tn)
-        finally:
-            B.syrk_set_f64_tail_split(0)
-            B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
-        assert_within_tolerance(got, ref, bound, M, -1.5, 0.5, Cin, B.DTYPE_F64)
-        assert np.array_equal(got[np.tril_indices(N)], again[np.tril_indices(N)])
-        assert_within_tolerance(goti, refi, boundi, M, 1.0, 0.0, None, B.DTYPE_F64, exact=True)
+        il = np.tril_indices(N)
+        by_form = []
+        for form in (B.F64_LAUNCH_PER_ITEM, B.F64_LAUNCH_PERSISTENT):      # blocks per slice / slices as further tickets
+            try:
+                B.syrk_set_f64_launch(form)
+                B.syrk_set_f64_tail_split(slices, tail)
+                got, ref, bound = run_case(A, B.DTYPE_F64, -1.5, 0.5, Cin, ldc=N + 2, tn=tn)
+                again, _, _ = run_case(A, B.DTYPE_F64, -1.5, 0.5, Cin, ldc=N + 2, tn=tn)
+                got1, ref1, bound1 = run_case(A, B.DTYPE_F64, -1.0, 1.0, Cin, tn=tn)
+                goti, refi, boundi = run_case(Ai, B.DTYPE_F64, 1.0, 0.0, poison=True, tn=tn)
+            finally:
+                B.syrk_set_f64_tail_split(0)
+                B.syrk_set_f64_launch(B.F64_LAUNCH_AUTO)
+            assert_within_tolerance(got, ref, bound, M, -1.5, 0.5, Cin, B.DTYPE_F64)
+            assert_within_tolerance(got1, ref1, bound1, M, -1.0, 1.0, Cin, B.DTYPE_F64)
+            assert np.array_equal(got[il], again[il])
+            assert_within_tolerance(goti, refi, boundi, M, 1.0, 0.0, None, B.DTYPE_F64, exact=True)
+            by_form.append((got[il], got1[il]))
+        assert np.array_equal(by_form[0][0], by_form[1][0]) and np.array_equal(by_form[0][1], by_form[1][1])
 
 
 def test_f64_tail_k_split_automatic():
