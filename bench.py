@@ -205,10 +205,10 @@ def run_reference(args, key: str, shape, rank: int):
 # summarised under profiles/.  Valid only for the kernel source it was taken on: keyed by its SHA-256.
 NCU_TRAFFIC = {
     # workload: (bytes per launch, kernel source file, sha256 of that file at capture time, square-schedule bytes or None)
-    "c2_f64_4096x4096": (828_744_448, "syrk_f64.cu", "aaff98b8281e9f400fdc495d28f82b12729f8aae146acccbc8ca953d5bc93ce7", 815_202_816),
+    "c2_f64_4096x4096": (822_442_496, "syrk_f64.cu", "b7220ccfcf5f6537b1b742a9ff9c2f3bd738d45ad98f75423b3ab2b781f45979", 809_468_160),
     "c3_bf16_16384x4096": (1_898_579_968, "syrk_bf16.cu", "527f2140d892d840fb605c824d4e19c4706e87355a46c48bb934fb71b3a9a97b", 3_150_107_648),
     "c4_bf16_2048x262144": (1_308_831_488, "syrk_bf16_pair.cu", "1f007b0ed5552de540c0cf0f25685f828321404cc4f842d0dbfcbbdcc303fc01", 2_332_056_832),
-    "c5_call_n16384": (2_695_872_768, "syrk_f64.cu", "aaff98b8281e9f400fdc495d28f82b12729f8aae146acccbc8ca953d5bc93ce7", 2_493_814_272),
+    "c5_call_n16384": (2_697_048_064, "syrk_f64.cu", "b7220ccfcf5f6537b1b742a9ff9c2f3bd738d45ad98f75423b3ab2b781f45979", 2_507_285_760),
 }
 
 
